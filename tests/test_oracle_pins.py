@@ -1,0 +1,273 @@
+"""Pins for the CPU oracle: closed forms, brute force through a second formulation,
+library routines on special cases, and the paper's worked examples.  No GPU."""
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.signal
+import scipy.special
+
+from oracle import oracle as orc
+from paper_2201_05587_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def im2col_conv(x, w, bias, stride, pad):
+    """Second, independent formulation: explicit padding, patch matrix, fp64 matmul."""
+    x = x.astype(np.float64)
+    w = w.astype(np.float64)
+    n, c, h, wd = x.shape
+    k, _, r, s = w.shape
+    xp = np.zeros((n, c, h + 2 * pad[0], wd + 2 * pad[1]))
+    xp[:, :, pad[0]:pad[0] + h, pad[1]:pad[1] + wd] = x
+    p = (h + 2 * pad[0] - r) // stride[0] + 1
+    q = (wd + 2 * pad[1] - s) // stride[1] + 1
+    cols = np.zeros((n, c * r * s, p * q))
+    for ci in range(c):
+        for ri in range(r):
+            for si in range(s):
+                patch = xp[:, ci, ri:ri + stride[0] * p:stride[0], si:si + stride[1] * q:stride[1]]
+                cols[:, (ci * r + ri) * s + si, :] = patch.reshape(n, -1)
+    y = np.einsum("kj,njp->nkp", w.reshape(k, -1), cols).reshape(n, k, p, q)
+    if bias is not None:
+        y = y + bias.astype(np.float64)[None, :, None, None]
+    return y
+
+
+@pytest.mark.parametrize("stride", [(1, 1), (2, 2), (1, 2)])
+@pytest.mark.parametrize("pad", [(0, 0), (1, 1), (2, 1)])
+@pytest.mark.parametrize("rs", [(3, 3), (1, 1), (2, 3)])
+def test_conv_brute_force_second_formulation(stride, pad, rs):
+    x = inputs.uniform((2, 2, 5, 4), 11, 0)
+    w = inputs.uniform((3, 2) + rs, 11, 1)
+    b = inputs.uniform((3,), 11, 2)
+    if 5 + 2 * pad[0] < rs[0] or 4 + 2 * pad[1] < rs[1]:
+        pytest.skip("filter larger than padded input")
+    y = orc.conv2d(x, w, b, stride=stride, pad=pad)
+    ref = im2col_conv(x, w, b, stride, pad)
+    assert y.shape == ref.shape
+    np.testing.assert_allclose(y, ref.astype(np.float32), rtol=0, atol=1e-6)
+
+
+def test_conv_is_cross_correlation_scipy():
+    """One channel, one filter, no padding: the library's 'valid' correlation (no flip)."""
+    x = inputs.uniform((1, 1, 9, 8), 12, 0)
+    w = inputs.uniform((1, 1, 3, 3), 12, 1)
+    y = orc.conv2d(x, w)
+    ref = scipy.signal.correlate2d(x[0, 0].astype(np.float64), w[0, 0].astype(np.float64), mode="valid")
+    np.testing.assert_allclose(y[0, 0], ref.astype(np.float32), atol=1e-6)
+    flipped = scipy.signal.convolve2d(x[0, 0].astype(np.float64), w[0, 0].astype(np.float64), mode="valid")
+    assert np.abs(y[0, 0] - flipped).max() > 1e-3
+
+
+@pytest.mark.parametrize("c0,r0,s0", [(0, 0, 0), (1, 1, 1), (2, 2, 0), (1, 0, 2)])
+def test_conv_delta_filter_is_shift(c0, r0, s0):
+    """A filter with a single 1 at (c0,r0,s0) copies input channel c0 shifted by (r0-1, s0-1), zeros outside."""
+    x = inputs.uniform((1, 3, 6, 7), 13, 0)
+    w = np.zeros((2, 3, 3, 3), np.float32)
+    w[1, c0, r0, s0] = 1.0
+    y = orc.conv2d(x, w, pad=(1, 1))
+    assert np.all(y[0, 0] == 0)
+    exp = np.zeros((6, 7), np.float32)
+    for p in range(6):
+        for q in range(7):
+            ih, iw = p + r0 - 1, q + s0 - 1
+            if 0 <= ih < 6 and 0 <= iw < 7:
+                exp[p, q] = x[0, c0, ih, iw]
+    np.testing.assert_array_equal(y[0, 1], exp)
+
+
+def test_conv_all_ones_filter_is_window_sum():
+    x = inputs.uniform((1, 2, 8, 9), 14, 0)
+    w = np.ones((1, 2, 3, 3), np.float32)
+    y = orc.conv2d(x, w, pad=(1, 1))
+    # summed-area table over the zero-padded channel sum
+    cs = x.astype(np.float64).sum(axis=1)[0]
+    padded = np.zeros((8 + 2, 9 + 2))
+    padded[1:-1, 1:-1] = cs
+    sat = np.zeros((11, 12))
+    sat[1:, 1:] = padded.cumsum(0).cumsum(1)
+    exp = sat[3:, 3:] - sat[:-3, 3:] - sat[3:, :-3] + sat[:-3, :-3]
+    np.testing.assert_allclose(y[0, 0], exp.astype(np.float32), atol=1e-5)
+
+
+def test_conv_1x1_equals_dense_on_reshaped_tensor():
+    x = inputs.uniform((1, 5, 4, 3), 15, 0)
+    w = inputs.uniform((6, 5, 1, 1), 15, 1)
+    b = inputs.uniform((6,), 15, 2)
+    y = orc.conv2d(x, w, b)
+    pix = x[0].reshape(5, 12).T.copy()                 # [pixels, C]
+    d = orc.dense(pix, w.reshape(6, 5), b)             # [pixels, K]
+    np.testing.assert_array_equal(y[0].reshape(6, 12), d.T)
+
+
+def test_conv_stride2_is_subsampled_stride1():
+    x = inputs.uniform((1, 3, 9, 9), 16, 0)
+    w = inputs.uniform((4, 3, 3, 3), 16, 1)
+    y1 = orc.conv2d(x, w, pad=(1, 1))
+    y2 = orc.conv2d(x, w, stride=(2, 2), pad=(1, 1))
+    np.testing.assert_array_equal(y2, y1[:, :, ::2, ::2])
+
+
+def test_conv_bias_only_and_activations():
+    x = inputs.uniform((1, 2, 4, 4), 17, 0)
+    w = np.zeros((3, 2, 3, 3), np.float32)
+    b = np.array([-1.5, 2.0, 7.25], np.float32)
+    y = orc.conv2d(x, w, b, pad=(1, 1), act=orc.ACT_RELU)
+    assert np.all(y[0, 0] == 0) and np.all(y[0, 1] == 2.0) and np.all(y[0, 2] == 7.25)
+    y6 = orc.conv2d(x, w, b, pad=(1, 1), act=orc.ACT_RELU6)
+    assert np.all(y6[0, 0] == 0) and np.all(y6[0, 1] == 2.0) and np.all(y6[0, 2] == 6.0)
+    yn = orc.conv2d(x, w, b, pad=(1, 1))
+    assert np.all(yn[0, 0] == -1.5)
+
+
+def test_conv_linearity_and_residual():
+    x1 = inputs.uniform((1, 2, 5, 5), 18, 0)
+    x2 = inputs.uniform((1, 2, 5, 5), 18, 1)
+    w = inputs.uniform((3, 2, 3, 3), 18, 2)
+    ya = orc.conv2d(x1, w, pad=(1, 1)).astype(np.float64)
+    yb = orc.conv2d(x2, w, pad=(1, 1)).astype(np.float64)
+    ys = orc.conv2d((x1 + 2 * x2), w, pad=(1, 1)).astype(np.float64)
+    np.testing.assert_allclose(ys, ya + 2 * yb, atol=2e-5)
+    res = inputs.uniform((1, 3, 5, 5), 18, 3)
+    yr = orc.conv2d(x1, w, pad=(1, 1), residual=res, act=orc.ACT_RELU)
+    np.testing.assert_allclose(yr, np.maximum(ya + res, 0).astype(np.float32), atol=1e-6)
+
+
+@pytest.mark.parametrize("stride", [1, 2])
+def test_depthwise_equals_block_diagonal_full_conv(stride):
+    c = 4
+    x = inputs.uniform((2, c, 7, 6), 19, 0)
+    w = inputs.uniform((c, 1, 3, 3), 19, 1)
+    b = inputs.uniform((c,), 19, 2)
+    y = orc.dwconv2d(x, w, b, stride=(stride, stride), pad=(1, 1), act=orc.ACT_RELU6)
+    full = np.zeros((c, c, 3, 3), np.float32)
+    for i in range(c):
+        full[i, i] = w[i, 0]
+    ref = orc.conv2d(x, full, b, stride=(stride, stride), pad=(1, 1), act=orc.ACT_RELU6)
+    np.testing.assert_array_equal(y, ref)
+
+
+def test_depthwise_delta_and_ones():
+    x = inputs.uniform((1, 3, 5, 5), 20, 0)
+    w = np.zeros((3, 1, 3, 3), np.float32)
+    w[:, 0, 1, 1] = 1.0
+    np.testing.assert_array_equal(orc.dwconv2d(x, w, pad=(1, 1)), x)
+    w[:] = 1.0
+    y = orc.dwconv2d(x, w, pad=(0, 0))
+    exp = sum(x[:, :, r:r + 3, s:s + 3].astype(np.float64) for r in range(3) for s in range(3))
+    np.testing.assert_allclose(y, exp.astype(np.float32), atol=1e-6)
+
+
+def test_matmul_algorithm1_against_numpy_and_closed_forms():
+    a = inputs.uniform((1, 7, 5), 21, 0)
+    b = inputs.uniform((1, 5, 6), 21, 1)
+    c = orc.batch_matmul(a, b)
+    ref = a[0].astype(np.float64) @ b[0].astype(np.float64)
+    np.testing.assert_allclose(c[0], ref.astype(np.float32), atol=1e-6)
+    # identity weight copies, ones give row sums
+    x = inputs.uniform((4, 6), 21, 2)
+    np.testing.assert_array_equal(orc.dense(x, np.eye(6, dtype=np.float32)), x)
+    rs = orc.dense(x, np.ones((3, 6), np.float32))
+    np.testing.assert_allclose(rs, np.repeat(x.astype(np.float64).sum(1, keepdims=True), 3, 1).astype(np.float32),
+                               atol=1e-6)
+    # a non-symmetric case separates a transposed operand from the right one
+    w = inputs.uniform((3, 6), 21, 3)
+    bias = inputs.uniform((3,), 21, 4)
+    d = orc.dense(x, w, bias)
+    np.testing.assert_allclose(d, (x.astype(np.float64) @ w.astype(np.float64).T + bias).astype(np.float32),
+                               atol=1e-6)
+
+
+def test_batch_matmul_nt_nn_consistency_and_batch1_dense():
+    a = inputs.uniform((3, 4, 5), 22, 0)
+    b = inputs.uniform((3, 6, 5), 22, 1)            # [B, M, K]
+    nt = orc.batch_matmul(a, b, trans_b=True)
+    nn = orc.batch_matmul(a, np.ascontiguousarray(b.transpose(0, 2, 1)), trans_b=False)
+    np.testing.assert_array_equal(nt, nn)
+    for i in range(3):
+        np.testing.assert_array_equal(nt[i], orc.dense(a[i], b[i]))
+    ident = np.broadcast_to(np.eye(5, dtype=np.float32), (3, 5, 5)).copy()
+    np.testing.assert_array_equal(orc.batch_matmul(a, ident), a)
+
+
+def test_softmax_pins():
+    s = inputs.normal((3, 4, 17), 23, 0, std=3.0)
+    p = orc.softmax(s, scale=0.125)
+    np.testing.assert_allclose(p.astype(np.float64).sum(-1), 1.0, atol=1e-6)
+    np.testing.assert_allclose(p, scipy.special.softmax(0.125 * s.astype(np.float64), axis=-1).astype(np.float32),
+                               atol=1e-7)
+    shifted = orc.softmax(s + np.float32(8.0), scale=0.125)
+    np.testing.assert_allclose(shifted, p, atol=1e-6)
+    u = orc.softmax(np.full((2, 8), 3.5, np.float32))
+    np.testing.assert_array_equal(u, np.full((2, 8), 0.125, np.float32))
+    # large magnitudes must not overflow
+    big = orc.softmax(np.array([[1000.0, 1000.0, -1000.0]], np.float32))
+    np.testing.assert_allclose(big, [[0.5, 0.5, 0.0]], atol=1e-7)
+
+
+def test_activation_pins():
+    x = np.array([[-3.0, -1.0, 0.0, 0.5, 1.0, 6.0, 7.5]], np.float32)
+    eye = np.eye(7, dtype=np.float32)
+    r6 = orc.dense(x, eye, act=orc.ACT_RELU6)
+    np.testing.assert_array_equal(r6, [[0, 0, 0, 0.5, 1.0, 6.0, 6.0]])
+    r = orc.dense(x, eye, act=orc.ACT_RELU)
+    np.testing.assert_array_equal(r, [[0, 0, 0, 0.5, 1.0, 6.0, 7.5]])
+    g = orc.dense(x, eye, act=orc.ACT_GELU_ERF).astype(np.float64)
+    gm = orc.dense(-x, eye, act=orc.ACT_GELU_ERF).astype(np.float64)
+    assert g[0, 2] == 0.0
+    np.testing.assert_allclose(g - gm, x, atol=1e-6)             # GELU(x) - GELU(-x) = x
+    assert abs(g[0, 4] - 0.8413447460685429) < 1e-7              # GELU(1) = Phi(1)
+    assert abs(g[0, 4] - 0.5 * (1 + math.tanh(math.sqrt(2 / math.pi) * (1 + 0.044715)))) > 1e-5  # not the tanh form
+
+
+def test_tf32_modes_are_diagnostics_close_to_exact():
+    x = inputs.uniform((8, 64), 24, 0)
+    w = inputs.uniform((16, 64), 24, 1)
+    exact = orc.dense(x, w)
+    for mode in (orc.MODE_TF32_TRUNC, orc.MODE_TF32_ROUND):
+        e = orc.rel_l2(orc.dense(x, w, mode=mode), exact)
+        assert 1e-6 < e < 2e-3
+    # values already representable with 10 mantissa bits are unchanged by either mode
+    xi = np.round(x * 64) / 64
+    wi = np.round(w * 64) / 64
+    np.testing.assert_array_equal(orc.dense(xi, wi, mode=orc.MODE_TF32_TRUNC), orc.dense(xi, wi))
+    np.testing.assert_array_equal(orc.dense(xi, wi, mode=orc.MODE_TF32_ROUND), orc.dense(xi, wi))
+
+
+def test_thread_count_does_not_change_results():
+    x = inputs.uniform((1, 8, 12, 12), 25, 0)
+    w = inputs.uniform((8, 8, 3, 3), 25, 1)
+    y1 = orc.conv2d(x, w, pad=(1, 1), threads=1)
+    yn, used = orc.conv2d(x, w, pad=(1, 1), threads=0, return_threads=True)
+    assert used >= 1
+    np.testing.assert_array_equal(y1, yn)
+
+
+def test_split_rules_match_paper_examples():
+    with open(os.path.join(GOLDEN, "split_validity.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            extent, form, factors, valid = line.split()
+            extent, valid = int(extent), bool(int(valid))
+            fs = [int(v) for v in factors.split(",")]
+            if form == "fixed":
+                assert orc.split_covers(extent, fs) == valid, line
+            elif form == "reform":
+                assert orc.split_reformulated_valid(extent, fs[0]) == valid, line
+            else:
+                assert orc.factor_fits(extent, fs[0]) == valid, line
+    assert not orc.same_class(("conv2d", "bias", "relu"), ("dense", "add"))
+    assert orc.same_class(("conv2d", "bias", "relu"), ("conv2d", "bias", "relu"))
+
+
+def test_select_hand_tables():
+    t = [5.0, 3.0, -1.0, 3.0,     # tie between 1 and 3 -> lowest index
+         -1.0, -1.0, -1.0, -1.0,  # nothing valid
+         2.0, -1.0, 1.5, 9.0]
+    assert orc.select(t, 3, 4) == [1, -1, 2]
+    assert orc.model_latency([2, 1, 3], t, [1, -1, 2], 4) == pytest.approx(2 * 3.0 + 3 * 1.5)
