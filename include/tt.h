@@ -1,0 +1,252 @@
+/*
+ * tt.h — C ABI of the transfer-tuning hot path on B200 (sm_100a).
+ *
+ * Transfer-tuning (Gibson & Cano, PACT '22) reuses schedules tuned for the kernels
+ * of one model on the kernels of another: every kernel of the target model is run
+ * standalone under every compatible schedule of a pool, timed, and the fastest
+ * schedule that produced valid code is kept (Section 4.3).  A kernel is a fused
+ * group of operators identified by its class (operator sequence) and its data
+ * sizes (Section 4.2); a schedule is the list of transformations applied to the
+ * kernel's loop nest (Section 2, Algorithm 1).
+ *
+ * Here a schedule is a fixed-size record of the choices those transformations make
+ * on a GPU (tile sizes, pipeline depth, split-K, tile order, vector width ...), and
+ * applying it to a kernel of another shape legalises it or declares it invalid.
+ *
+ * General conventions
+ *   - Every function returns a tt_status; nothing throws or aborts across the ABI.
+ *   - Handles (tt_workload*) are owned by the library and released by *_destroy.
+ *   - Tensor pointers in tt_tensors are DEVICE pointers owned by the caller, fp32,
+ *     dense row-major in the layouts stated at tt_op; they are borrowed for the
+ *     call and never retained.  tt_run_host takes HOST pointers instead.
+ *   - The only device memory the library owns is a per-workload workspace (split-K
+ *     partial sums and a status word), allocated by tt_schedule_apply and released
+ *     by tt_workload_destroy or the next apply.
+ *   - Launches are asynchronous on the given CUDA stream (a cudaStream_t passed as
+ *     void*; NULL is the default stream).  tt_time, tt_transfer_tune, tt_grid_tune
+ *     and tt_run_host synchronise that stream before returning.
+ *   - One handle must not be used from two threads at once.
+ *   - A CUDA device must be present for everything except the pure host calls
+ *     (tt_workload_create/key/class/gemm_view, tt_default_schedule, tt_schedule_check,
+ *     tt_select, tt_model_latency, tt_split_check, tt_status_string); there is no
+ *     CPU fallback: without a device the others return TT_ERR_CUDA.
+ */
+#ifndef TT_H_
+#define TT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TT_OK = 0,
+    TT_ERR_INVALID_ARG = 1,       /* null pointer, non-positive extent, unknown enum */
+    TT_ERR_INVALID_SCHEDULE = 2,  /* the record cannot be applied to this shape ("invalid code", Section 4.2) */
+    TT_ERR_CLASS_MISMATCH = 3,    /* record of another kernel family/class (always invalid, Section 4.2) */
+    TT_ERR_RESOURCE = 4,          /* legal record, but exceeds shared memory / tensor memory / thread limits */
+    TT_ERR_NOT_APPLIED = 5,       /* tt_run / tt_time before a successful tt_schedule_apply */
+    TT_ERR_CUDA = 6,              /* a CUDA runtime or driver call failed (or no device) */
+    TT_ERR_TIMEOUT = 7,           /* a bounded wait inside a kernel expired; the context stays usable */
+    TT_ERR_OOM = 8,               /* workspace allocation failed */
+    TT_ERR_NOT_IMPLEMENTED = 9
+} tt_status;
+
+/* Operators (each is one fused kernel; bias and activation are applied as soon as an
+ * output's partial sums are complete, Section 4.2).
+ *   TT_OP_CONV2D        Algorithm 2: y = act(conv2d(pad(x), w) + bias [+ residual]).
+ *                       x [n,c,h,w]  w [k,c,r,s]  bias [k]  residual,y [n,k,p,q]; cross-correlation,
+ *                       zero padding pad_h/pad_w per side, p = (h + 2 pad_h - r)/stride_h + 1.
+ *   TT_OP_DWCONV2D      the same with one r x s filter per channel: w [c,1,r,s], bias [c], y [n,c,p,q].
+ *   TT_OP_DENSE         y[m,nn] = act(bias[nn] + sum_kk x[m,kk] w[nn,kk]); x [m,kk], w [nn,kk] (Algorithm 1 with
+ *                       the second operand stored transposed), bias [nn].
+ *   TT_OP_BATCH_MATMUL  y[b,m,nn] = sum_kk x[b,m,kk] * w[b,nn,kk] (trans_b = 1) or * w[b,kk,nn] (trans_b = 0);
+ *                       Algorithm 1 per batch entry.
+ *   TT_OP_SOFTMAX       y[row,:] = softmax(scale * x[row,:]) over nn columns, rows = batch*m.
+ */
+typedef enum { TT_OP_CONV2D = 0, TT_OP_DWCONV2D = 1, TT_OP_DENSE = 2, TT_OP_BATCH_MATMUL = 3, TT_OP_SOFTMAX = 4 } tt_op;
+typedef enum { TT_ACT_NONE = 0, TT_ACT_RELU = 1, TT_ACT_RELU6 = 2, TT_ACT_GELU_ERF = 3 } tt_act;
+
+/* Kernel families: the loop structure a record was written for.  A record only applies inside its family. */
+typedef enum { TT_FAMILY_GEMM_TC = 0,   /* tcgen05 TF32 contraction: conv2d (implicit GEMM), dense, batch_matmul */
+               TT_FAMILY_DW_SIMT = 1,   /* fp32 SIMT depthwise convolution */
+               TT_FAMILY_ROW_SIMT = 2   /* fp32 SIMT row-wise kernels (softmax) */
+} tt_family;
+
+typedef struct tt_shapes {
+    int32_t n, c, h, w, k, r, s, stride_h, stride_w, pad_h, pad_w; /* conv2d, dwconv2d (k ignored for depthwise) */
+    int32_t batch, m, nn, kk, trans_b;                             /* dense (batch=1), batch_matmul, softmax */
+    int32_t has_bias, has_residual;
+    int32_t act;                                                   /* tt_act */
+    float scale;                                                   /* softmax only */
+} tt_shapes;
+
+#define TT_RECORD_VERSION 1u
+
+/* A schedule record.  Correspondence with the primitives listed under Algorithm 1:
+ *   Split     -> tile_m, tile_n, tile_k (CTA tile of the output and of the reduction), split_k
+ *   Reorder   -> raster (order in which output tiles are handed to CTAs), mma_m_axis (which output loop is the
+ *                accumulator's row loop)
+ *   Fuse+Parallel -> the (tile_m x tile_n x split_k x batch) grid
+ *   cache buffer / ComputeAt -> the accumulator lives in tensor memory and the bias/activation run on read-out;
+ *                               `stages` shared-memory buffers decouple loading from the multiply
+ *   Vectorize -> vec_width;   Unroll -> unroll / items_per_thread
+ * GEMM_TC uses tile_m, tile_n, tile_k, stages, split_k, raster, mma_m_axis.
+ * DW_SIMT uses tile_m (channels per CTA), block_y x block_x (output rows x columns per CTA tile),
+ *         items_per_thread (consecutive outputs along the width per thread), vec_width, threads.
+ * ROW_SIMT uses block_x (threads cooperating on one row: 1..32, power of two), block_y (rows per CTA), vec_width.
+ * origin_* say which kernel the record was tuned on (its "native" kernel, Section 3). */
+typedef struct tt_schedule_record {
+    uint32_t version;      /* TT_RECORD_VERSION */
+    uint32_t family;       /* tt_family */
+    int32_t origin_op;     /* tt_op */
+    tt_shapes origin;
+    int32_t tile_m, tile_n, tile_k;
+    int32_t stages, split_k, raster;
+    int32_t block_x, block_y, items_per_thread, vec_width, unroll, threads;
+    int32_t mma_m_axis;    /* GEMM_TC: which output axis rides the 128 accumulator rows: 0 library's choice by shape,
+                              1 output rows (conv filters, dense/bmm rows m), 2 output columns (conv pixels, nn) */
+    int32_t reserved[3];
+} tt_schedule_record;
+
+typedef struct tt_tensors {
+    const void* x;
+    const void* w;
+    const void* bias;      /* NULL when has_bias == 0 */
+    const void* residual;  /* NULL when has_residual == 0 */
+    void* y;
+} tt_tensors;
+
+/* The contraction a GEMM_TC workload is lowered to, and its algorithmic work:
+ * flops = 2*batch*gm*gn*gk (depthwise: 2*outputs*r*s; softmax: 5 per element), bytes = 4 * (every tensor once). */
+typedef struct tt_gemm_view {
+    int32_t batch, gm, gn, gk;
+    double flops, bytes;
+} tt_gemm_view;
+
+/* What tt_schedule_apply / tt_schedule_check decided. */
+typedef struct tt_apply_info {
+    tt_schedule_record legal;   /* the record after legalisation: what will actually run */
+    int32_t changed;            /* bit mask of fields legalisation had to change (TT_CHG_*) */
+    int32_t grid_x, grid_y, grid_z, threads;
+    int32_t smem_bytes, tmem_cols;
+    int64_t workspace_bytes;
+    int32_t launches;           /* kernels per tt_run (2 with split-K) */
+} tt_apply_info;
+
+enum { TT_CHG_TILE_M = 1, TT_CHG_TILE_N = 2, TT_CHG_TILE_K = 4, TT_CHG_STAGES = 8, TT_CHG_SPLIT_K = 16,
+       TT_CHG_VEC = 32, TT_CHG_BLOCK = 64, TT_CHG_ITEMS = 128 };
+
+/* Validity modes for mapping a record onto another shape (Section 4.1).
+ *   TT_MODE_LEGALISE  reformulate: clamp/round tile sizes to the new extents and the hardware's legal set,
+ *                     lower the vector width to what divides the row, clamp split_k to the reduction tiles;
+ *                     invalid only when resources are exceeded or a field is nonsensical.
+ *   TT_MODE_STRICT    no reformulation: a record whose tile factor exceeds the loop extent, whose split_k
+ *                     exceeds the number of reduction tiles, or that needs any rounding is invalid. */
+typedef enum { TT_MODE_LEGALISE = 0, TT_MODE_STRICT = 1 } tt_mode;
+
+typedef struct tt_timing_opts {
+    int32_t warmup_batches;   /* default 3 */
+    int32_t batches;          /* default 10; the median over batches is reported (evaluation protocol, Section 5.1) */
+    int32_t min_batch_us;     /* each batch repeats the launch until it lasts at least this long; default 200 */
+    int32_t max_repeats;      /* cap on launches per batch; default 4096 */
+    int32_t use_graph;        /* 1: replay each batch as a CUDA graph (no CPU launch gaps) */
+    int32_t reserved[3];
+} tt_timing_opts;
+
+typedef struct tt_timing {
+    float median_us, min_us, max_us, q1_us, q3_us;  /* per launch of the whole workload (all its kernels) */
+    int32_t repeats, batches;
+} tt_timing;
+
+typedef struct tt_tune_opts {
+    tt_timing_opts timing;
+    int32_t mode;            /* tt_mode */
+    int32_t strict_class;    /* 1: the record's origin kernel class (op, bias, activation, residual) must equal the
+                                workload's (the paper's rule); 0: same family suffices */
+    int32_t include_default; /* 1 (default): column 0 of the table is the workload's default ("untuned") record */
+    int32_t reserved[5];
+} tt_tune_opts;
+
+/* Result arrays are allocated by the caller.  n_cols = n_pool + 1; column 0 is the default record, column j+1 is
+ * pool[j].  times_us < 0 marks an invalid pair (plotted as -1 in the paper's Figure 4). */
+typedef struct tt_tune_result {
+    int32_t* chosen;        /* [n_wl]        column index of the fastest valid record, -1 if none */
+    float* best_us;         /* [n_wl]        */
+    float* times_us;        /* [n_wl*n_cols] */
+    int32_t* status;        /* [n_wl*n_cols] tt_status of apply/timing for the pair */
+    double search_seconds;  /* wall time of the call: apply + warm-up + timing + selection */
+    int32_t pairs_timed, pairs_invalid;
+} tt_tune_result;
+
+typedef struct tt_workload tt_workload;
+
+const char* tt_status_string(tt_status s);
+
+/* Create a kernel from its operator and data sizes (Section 4.2: a kernel is its class plus its sizes).
+ * Validates the shape (positive extents, filter fits the padded input). */
+tt_status tt_workload_create(tt_op op, const tt_shapes* shapes, tt_workload** out);
+tt_status tt_workload_destroy(tt_workload* w);
+/* Workload ID: hash of operator type and sizes; identical kernels share schedules and are tuned once (Section 2). */
+tt_status tt_workload_key(const tt_workload* w, uint64_t* key);
+/* Kernel class: hash of (operator, bias, activation, residual) only, regardless of sizes (Section 4.2). */
+tt_status tt_workload_class(const tt_workload* w, uint64_t* cls);
+tt_status tt_workload_family(const tt_workload* w, int32_t* family);
+tt_status tt_workload_gemm_view(const tt_workload* w, tt_gemm_view* out);
+/* The built-in "untuned" record of the workload's family: baseline of every speedup and fallback when no
+ * pool record is valid (Section 4.3). */
+tt_status tt_default_schedule(const tt_workload* w, tt_schedule_record* out);
+
+/* Host-only: legalise and validate `rec` against `w` without touching the device. */
+tt_status tt_schedule_check(const tt_workload* w, const tt_schedule_record* rec, int32_t mode, int32_t strict_class,
+                            tt_apply_info* info_out);
+/* Legalise, validate and bind `rec` to `w` (tensor maps, descriptors, grid, workspace).  info_out may be NULL.
+ * Uses TT_MODE_LEGALISE and family matching; tt_schedule_apply_ex takes both options. */
+tt_status tt_schedule_apply(tt_workload* w, const tt_schedule_record* rec, tt_apply_info* info_out);
+tt_status tt_schedule_apply_ex(tt_workload* w, const tt_schedule_record* rec, int32_t mode, int32_t strict_class,
+                               tt_apply_info* info_out);
+/* Literal form of the split example of Section 4.1: does splitting a loop of `extent` iterations by the given
+ * factors traverse it exactly?  reformulate != 0 tests Split(N, N/f, f) for the single factor f instead. */
+tt_status tt_split_check(int64_t extent, const int64_t* factors, size_t n_factors, int32_t reformulate, int32_t* valid);
+
+/* Run the workload once under the applied record (device pointers). */
+tt_status tt_run(tt_workload* w, const tt_tensors* t, void* cuda_stream);
+/* The same with HOST pointers: copies x, w, bias, residual to library-owned device buffers, runs, copies y back,
+ * synchronises.  bytes_h2d/bytes_d2h (may be NULL) receive the bytes copied. */
+tt_status tt_run_host(tt_workload* w, const tt_tensors* host, void* cuda_stream, int64_t* bytes_h2d, int64_t* bytes_d2h);
+/* Read and clear the device status word of the last runs (TT_OK or TT_ERR_TIMEOUT); synchronises the stream. */
+tt_status tt_workload_status(tt_workload* w, void* cuda_stream);
+
+/* Time the applied record: warm-up batches, then `batches` batches of back-to-back launches between two CUDA
+ * events.  `sets` holds n_sets tensor sets used round-robin (n_sets > 1 with a footprint beyond L2 gives cold-cache
+ * times). */
+tt_status tt_time(tt_workload* w, const tt_tensors* sets, size_t n_sets, void* cuda_stream, const tt_timing_opts* o,
+                  tt_timing* out);
+
+/* Pure host: per row of times_us[n_wl x n_cols] the column of the smallest non-negative time, ties to the lowest
+ * column, -1 when the row has none. */
+tt_status tt_select(const float* times_us, size_t n_wl, size_t n_cols, int32_t* chosen);
+/* Pure host: sum_w use_count[w] * times_us[w, chosen[w]] (kernels assumed independent, Section 2). */
+tt_status tt_model_latency(const float* times_us, size_t n_wl, size_t n_cols, const int32_t* chosen,
+                           const int32_t* use_count, double* latency_us);
+
+/* The evaluator of Section 4.3: every workload x every compatible pool record (plus the default), standalone, on
+ * the workload's own tensors; invalid pairs are recorded, not fatal.  On return each workload is left with its
+ * chosen record applied.  tensors[i] belongs to model_workloads[i]. */
+tt_status tt_transfer_tune(tt_workload* const* model_workloads, const tt_tensors* tensors, size_t n_wl,
+                           const tt_schedule_record* pool, size_t n_pool, const tt_tune_opts* o, void* cuda_stream,
+                           tt_tune_result* out);
+
+/* Native tuning of one workload (stands in for the auto-scheduler that fills a pool, Section 2): exhaustive walk
+ * over a grid of records of the workload's family, each timed with `o`; writes the best `top_k` records (fastest
+ * first) to out_records/out_us and their number to n_out.  level 0 = coarse grid, 1 = full grid. */
+tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, const tt_timing_opts* o, int32_t level,
+                       size_t top_k, tt_schedule_record* out_records, float* out_us, size_t* n_out,
+                       int32_t* n_tried);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TT_H_ */

@@ -1,0 +1,351 @@
+"""ctypes binding of libtt.so: argument marshalling only.
+
+Names mirror ``include/tt.h``.  Torch tensors supply device memory and the current
+stream; every step of the hot path runs inside the library's CUDA kernels.  There
+is no fallback: if the library is missing or no GPU is present the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+from . import build as _build
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+# enums
+TT_OK, TT_ERR_INVALID_ARG, TT_ERR_INVALID_SCHEDULE, TT_ERR_CLASS_MISMATCH, TT_ERR_RESOURCE, \
+    TT_ERR_NOT_APPLIED, TT_ERR_CUDA, TT_ERR_TIMEOUT, TT_ERR_OOM, TT_ERR_NOT_IMPLEMENTED = range(10)
+TT_OP_CONV2D, TT_OP_DWCONV2D, TT_OP_DENSE, TT_OP_BATCH_MATMUL, TT_OP_SOFTMAX = range(5)
+TT_ACT_NONE, TT_ACT_RELU, TT_ACT_RELU6, TT_ACT_GELU_ERF = range(4)
+TT_FAMILY_GEMM_TC, TT_FAMILY_DW_SIMT, TT_FAMILY_ROW_SIMT = range(3)
+TT_MODE_LEGALISE, TT_MODE_STRICT = 0, 1
+TT_RECORD_VERSION = 1
+TT_CHG_TILE_M, TT_CHG_TILE_N, TT_CHG_TILE_K, TT_CHG_STAGES, TT_CHG_SPLIT_K, TT_CHG_VEC, TT_CHG_BLOCK, TT_CHG_ITEMS = \
+    1, 2, 4, 8, 16, 32, 64, 128
+
+i32, u32, f32 = C.c_int32, C.c_uint32, C.c_float
+
+
+class tt_shapes(C.Structure):
+    _fields_ = [(n, i32) for n in ("n", "c", "h", "w", "k", "r", "s", "stride_h", "stride_w", "pad_h", "pad_w",
+                                   "batch", "m", "nn", "kk", "trans_b", "has_bias", "has_residual", "act")] + \
+               [("scale", f32)]
+
+
+class tt_schedule_record(C.Structure):
+    _fields_ = [("version", u32), ("family", u32), ("origin_op", i32), ("origin", tt_shapes)] + \
+               [(n, i32) for n in ("tile_m", "tile_n", "tile_k", "stages", "split_k", "raster", "block_x", "block_y",
+                                   "items_per_thread", "vec_width", "unroll", "threads", "mma_m_axis")] + \
+               [("reserved", i32 * 3)]
+
+    FIELDS = ("tile_m", "tile_n", "tile_k", "stages", "split_k", "raster", "block_x", "block_y",
+              "items_per_thread", "vec_width", "unroll", "threads", "mma_m_axis")
+
+    def as_dict(self):
+        d = {"family": int(self.family), "origin_op": int(self.origin_op)}
+        d.update({k: int(getattr(self, k)) for k in self.FIELDS})
+        return d
+
+    def short(self):
+        if self.family == TT_FAMILY_GEMM_TC:
+            return (f"tc[{self.tile_m}x{self.tile_n}x{self.tile_k} st{self.stages} sk{self.split_k} "
+                    f"r{self.raster} ax{self.mma_m_axis}]")
+        if self.family == TT_FAMILY_DW_SIMT:
+            return (f"dw[c{self.tile_m} {self.block_y}x{self.block_x} it{self.items_per_thread} "
+                    f"v{self.vec_width} t{self.threads}]")
+        return f"row[{self.block_x}x{self.block_y} v{self.vec_width}]"
+
+
+class tt_tensors(C.Structure):
+    _fields_ = [("x", C.c_void_p), ("w", C.c_void_p), ("bias", C.c_void_p), ("residual", C.c_void_p), ("y", C.c_void_p)]
+
+
+class tt_gemm_view(C.Structure):
+    _fields_ = [("batch", i32), ("gm", i32), ("gn", i32), ("gk", i32), ("flops", C.c_double), ("bytes", C.c_double)]
+
+
+class tt_apply_info(C.Structure):
+    _fields_ = [("legal", tt_schedule_record), ("changed", i32), ("grid_x", i32), ("grid_y", i32), ("grid_z", i32),
+                ("threads", i32), ("smem_bytes", i32), ("tmem_cols", i32), ("workspace_bytes", C.c_int64),
+                ("launches", i32)]
+
+
+class tt_timing_opts(C.Structure):
+    _fields_ = [("warmup_batches", i32), ("batches", i32), ("min_batch_us", i32), ("max_repeats", i32),
+                ("use_graph", i32), ("reserved", i32 * 3)]
+
+
+class tt_timing(C.Structure):
+    _fields_ = [("median_us", f32), ("min_us", f32), ("max_us", f32), ("q1_us", f32), ("q3_us", f32),
+                ("repeats", i32), ("batches", i32)]
+
+
+class tt_tune_opts(C.Structure):
+    _fields_ = [("timing", tt_timing_opts), ("mode", i32), ("strict_class", i32), ("include_default", i32),
+                ("reserved", i32 * 5)]
+
+
+class tt_tune_result(C.Structure):
+    _fields_ = [("chosen", C.POINTER(i32)), ("best_us", C.POINTER(f32)), ("times_us", C.POINTER(f32)),
+                ("status", C.POINTER(i32)), ("search_seconds", C.c_double), ("pairs_timed", i32),
+                ("pairs_invalid", i32)]
+
+
+EXPORTS = {
+    "tt_status_string": (C.c_char_p, [i32]),
+    "tt_workload_create": (i32, [i32, C.POINTER(tt_shapes), C.POINTER(C.c_void_p)]),
+    "tt_workload_destroy": (i32, [C.c_void_p]),
+    "tt_workload_key": (i32, [C.c_void_p, C.POINTER(C.c_uint64)]),
+    "tt_workload_class": (i32, [C.c_void_p, C.POINTER(C.c_uint64)]),
+    "tt_workload_family": (i32, [C.c_void_p, C.POINTER(i32)]),
+    "tt_workload_gemm_view": (i32, [C.c_void_p, C.POINTER(tt_gemm_view)]),
+    "tt_default_schedule": (i32, [C.c_void_p, C.POINTER(tt_schedule_record)]),
+    "tt_schedule_check": (i32, [C.c_void_p, C.POINTER(tt_schedule_record), i32, i32, C.POINTER(tt_apply_info)]),
+    "tt_schedule_apply": (i32, [C.c_void_p, C.POINTER(tt_schedule_record), C.POINTER(tt_apply_info)]),
+    "tt_schedule_apply_ex": (i32, [C.c_void_p, C.POINTER(tt_schedule_record), i32, i32, C.POINTER(tt_apply_info)]),
+    "tt_split_check": (i32, [C.c_int64, C.POINTER(C.c_int64), C.c_size_t, i32, C.POINTER(i32)]),
+    "tt_run": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p]),
+    "tt_run_host": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
+    "tt_workload_status": (i32, [C.c_void_p, C.c_void_p]),
+    "tt_time": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_size_t, C.c_void_p, C.POINTER(tt_timing_opts),
+                      C.POINTER(tt_timing)]),
+    "tt_select": (i32, [C.POINTER(f32), C.c_size_t, C.c_size_t, C.POINTER(i32)]),
+    "tt_model_latency": (i32, [C.POINTER(f32), C.c_size_t, C.c_size_t, C.POINTER(i32), C.POINTER(i32),
+                               C.POINTER(C.c_double)]),
+    "tt_transfer_tune": (i32, [C.POINTER(C.c_void_p), C.POINTER(tt_tensors), C.c_size_t, C.POINTER(tt_schedule_record),
+                               C.c_size_t, C.POINTER(tt_tune_opts), C.c_void_p, C.POINTER(tt_tune_result)]),
+    "tt_grid_tune": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(tt_timing_opts), i32, C.c_size_t,
+                           C.POINTER(tt_schedule_record), C.POINTER(f32), C.POINTER(C.c_size_t), C.POINTER(i32)]),
+}
+
+_lib = None
+
+
+def lib():
+    """Load libtt.so (building it with nvcc first if the sources are newer).  Raises if that fails."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if _build.needs_build():
+            path = _build.build()
+        handle = C.CDLL(path)
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(handle, name)          # AttributeError if a declared symbol is missing
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+class TTError(RuntimeError):
+    def __init__(self, status, what=""):
+        self.status = int(status)
+        msg = lib().tt_status_string(self.status).decode()
+        super().__init__(f"{what}: {msg} (tt_status {self.status})" if what else f"{msg} (tt_status {self.status})")
+
+
+def _check(status, what=""):
+    if status != TT_OK:
+        raise TTError(status, what)
+
+
+def status_string(s: int) -> str:
+    return lib().tt_status_string(int(s)).decode()
+
+
+def make_shapes(**kw) -> tt_shapes:
+    s = tt_shapes()
+    for k, v in kw.items():
+        if not hasattr(s, k):
+            raise KeyError(k)
+        setattr(s, k, v)
+    return s
+
+
+def conv2d_shapes(n, c, h, w, k, r, s, stride=1, pad=0, has_bias=True, act=TT_ACT_RELU, has_residual=False):
+    return make_shapes(n=n, c=c, h=h, w=w, k=k, r=r, s=s, stride_h=stride, stride_w=stride, pad_h=pad, pad_w=pad,
+                       has_bias=int(has_bias), act=act, has_residual=int(has_residual))
+
+
+def dense_shapes(m, nn, kk, has_bias=True, act=TT_ACT_NONE):
+    return make_shapes(batch=1, m=m, nn=nn, kk=kk, trans_b=1, has_bias=int(has_bias), act=act)
+
+
+def bmm_shapes(batch, m, nn, kk, trans_b=True):
+    return make_shapes(batch=batch, m=m, nn=nn, kk=kk, trans_b=int(trans_b))
+
+
+def softmax_shapes(batch, m, nn, scale=1.0):
+    return make_shapes(batch=batch, m=m, nn=nn, scale=scale)
+
+
+def make_record(family, **kw) -> tt_schedule_record:
+    r = tt_schedule_record()
+    r.version = TT_RECORD_VERSION
+    r.family = family
+    defaults = dict(tile_m=128, tile_n=128, tile_k=32, stages=4, split_k=1, raster=0, block_x=32, block_y=4,
+                    items_per_thread=1, vec_width=1, unroll=1, threads=128, mma_m_axis=0)
+    defaults.update(kw)
+    for k, v in defaults.items():
+        setattr(r, k, v)
+    return r
+
+
+def split_check(extent, factors, reformulate=False) -> bool:
+    arr = (C.c_int64 * len(factors))(*factors)
+    v = i32(0)
+    _check(lib().tt_split_check(extent, arr, len(factors), int(reformulate), C.byref(v)), "tt_split_check")
+    return bool(v.value)
+
+
+def select(times, n_wl, n_cols):
+    arr = (f32 * (n_wl * n_cols))(*[float(t) for t in times])
+    out = (i32 * n_wl)()
+    _check(lib().tt_select(arr, n_wl, n_cols, out), "tt_select")
+    return list(out)
+
+
+def model_latency(times, n_wl, n_cols, chosen, use_count) -> float:
+    arr = (f32 * (n_wl * n_cols))(*[float(t) for t in times])
+    ch = (i32 * n_wl)(*chosen)
+    uc = (i32 * n_wl)(*use_count)
+    out = C.c_double(0)
+    _check(lib().tt_model_latency(arr, n_wl, n_cols, ch, uc, C.byref(out)), "tt_model_latency")
+    return out.value
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def tensors(x, w=None, bias=None, residual=None, y=None) -> tt_tensors:
+    """Device pointers of torch CUDA tensors (or host pointers of CPU tensors for tt_run_host)."""
+    t = tt_tensors()
+    t.x, t.w, t.bias, t.residual, t.y = _ptr(x), _ptr(w), _ptr(bias), _ptr(residual), _ptr(y)
+    return t
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+class Workload:
+    """Owns one tt_workload handle."""
+
+    def __init__(self, op, shapes: tt_shapes, name: str = "", use_count: int = 1):
+        self.op, self.shapes, self.name, self.use_count = op, shapes, name, use_count
+        h = C.c_void_p()
+        _check(lib().tt_workload_create(op, C.byref(shapes), C.byref(h)), f"tt_workload_create({name})")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().tt_workload_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+    def key(self) -> int:
+        v = C.c_uint64()
+        _check(lib().tt_workload_key(self.handle, C.byref(v)))
+        return v.value
+
+    def kernel_class(self) -> int:
+        v = C.c_uint64()
+        _check(lib().tt_workload_class(self.handle, C.byref(v)))
+        return v.value
+
+    def family(self) -> int:
+        v = i32()
+        _check(lib().tt_workload_family(self.handle, C.byref(v)))
+        return v.value
+
+    def gemm_view(self) -> tt_gemm_view:
+        v = tt_gemm_view()
+        _check(lib().tt_workload_gemm_view(self.handle, C.byref(v)))
+        return v
+
+    def default_schedule(self) -> tt_schedule_record:
+        r = tt_schedule_record()
+        _check(lib().tt_default_schedule(self.handle, C.byref(r)))
+        return r
+
+    def check(self, rec, mode=TT_MODE_LEGALISE, strict_class=False):
+        """Returns (status, tt_apply_info); never raises for an invalid record."""
+        info = tt_apply_info()
+        st = lib().tt_schedule_check(self.handle, C.byref(rec), mode, int(strict_class), C.byref(info))
+        return st, info
+
+    def apply(self, rec, mode=TT_MODE_LEGALISE, strict_class=False) -> tt_apply_info:
+        info = tt_apply_info()
+        _check(lib().tt_schedule_apply_ex(self.handle, C.byref(rec), mode, int(strict_class), C.byref(info)),
+               f"tt_schedule_apply({self.name})")
+        return info
+
+    def try_apply(self, rec, mode=TT_MODE_LEGALISE, strict_class=False):
+        info = tt_apply_info()
+        st = lib().tt_schedule_apply_ex(self.handle, C.byref(rec), mode, int(strict_class), C.byref(info))
+        return st, info
+
+    def run(self, t: tt_tensors):
+        _check(lib().tt_run(self.handle, C.byref(t), _stream()), f"tt_run({self.name})")
+
+    def run_host(self, t: tt_tensors):
+        up, down = C.c_int64(), C.c_int64()
+        _check(lib().tt_run_host(self.handle, C.byref(t), _stream(), C.byref(up), C.byref(down)),
+               f"tt_run_host({self.name})")
+        return up.value, down.value
+
+    def status(self) -> int:
+        return lib().tt_workload_status(self.handle, _stream())
+
+    def time(self, sets, opts: tt_timing_opts | None = None) -> tt_timing:
+        if isinstance(sets, tt_tensors):
+            sets = [sets]
+        arr = (tt_tensors * len(sets))(*sets)
+        out = tt_timing()
+        _check(lib().tt_time(self.handle, arr, len(sets), _stream(), C.byref(opts) if opts else None, C.byref(out)),
+               f"tt_time({self.name})")
+        return out
+
+    def grid_tune(self, t: tt_tensors, opts: tt_timing_opts | None = None, level=0, top_k=1):
+        recs = (tt_schedule_record * top_k)()
+        us = (f32 * top_k)()
+        n = C.c_size_t()
+        tried = i32()
+        _check(lib().tt_grid_tune(self.handle, C.byref(t), _stream(), C.byref(opts) if opts else None, level, top_k,
+                                  recs, us, C.byref(n), C.byref(tried)), f"tt_grid_tune({self.name})")
+        out = []
+        for i in range(n.value):
+            r = tt_schedule_record()
+            C.memmove(C.byref(r), C.byref(recs[i]), C.sizeof(r))
+            out.append((r, float(us[i])))
+        return out, tried.value
+
+
+def transfer_tune(workloads, tensor_sets, pool, opts: tt_tune_opts | None = None):
+    """Evaluate every workload under the default record and every pool record; returns a dict with
+    chosen (column index per workload), best_us, times_us [n_wl][n_pool+1], status, search_seconds, counts."""
+    n_wl, n_pool = len(workloads), len(pool)
+    n_cols = n_pool + 1
+    handles = (C.c_void_p * n_wl)(*[w.handle for w in workloads])
+    tens = (tt_tensors * n_wl)(*tensor_sets)
+    parr = (tt_schedule_record * max(n_pool, 1))(*pool)
+    chosen = (i32 * n_wl)()
+    best = (f32 * n_wl)()
+    times = (f32 * (n_wl * n_cols))()
+    status = (i32 * (n_wl * n_cols))()
+    res = tt_tune_result()
+    res.chosen, res.best_us, res.times_us, res.status = chosen, best, times, status
+    if opts is None:
+        opts = tt_tune_opts()
+        opts.include_default = 1
+    _check(lib().tt_transfer_tune(handles, tens, n_wl, parr, n_pool, C.byref(opts), _stream(), C.byref(res)),
+           "tt_transfer_tune")
+    return {
+        "chosen": list(chosen), "best_us": list(best),
+        "times_us": [[times[i * n_cols + j] for j in range(n_cols)] for i in range(n_wl)],
+        "status": [[status[i * n_cols + j] for j in range(n_cols)] for i in range(n_wl)],
+        "search_seconds": res.search_seconds, "pairs_timed": res.pairs_timed, "pairs_invalid": res.pairs_invalid,
+    }

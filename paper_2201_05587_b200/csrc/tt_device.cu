@@ -1,0 +1,479 @@
+// Device-facing half of the C ABI: binding a legalised record to a workload (workspace, tensor maps), running,
+// the device-timed evaluator (Section 4.3 of the paper), the native grid tuner that fills pools.
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <algorithm>
+#include <chrono>
+#include <cstring>
+#include <vector>
+#include "tt_internal.h"
+
+namespace tt {
+
+cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const ReduceArgs& red, const void* tmap_a,
+                        const void* tmap_b, cudaStream_t st);
+cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st);
+cudaError_t launch_row(const tt_apply_info& I, const RowArgs& row, cudaStream_t st);
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver entry point is looked up through the runtime, so the library links against cudart only and loads
+// on machines without a driver.
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+bool device_present() {
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess) { cudaGetLastError(); return false; }
+    return n > 0;
+}
+
+// K-major operand [batch][rows][K] -> 3-D tensor map, box = [atom_k, box_rows, 1], swizzle span = one box row.
+tt_status encode_operand(void* out, const float* base, int K, int rows, int batch, long long rs, long long bs,
+                         bool batched, int atom_k, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return TT_ERR_CUDA;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0) return TT_ERR_INVALID_ARG;
+    const cuuint64_t nb = batched ? (cuuint64_t)batch : 1;
+    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, nb};
+    cuuint64_t strides[2] = {(cuuint64_t)rs * 4, (cuuint64_t)(batched ? bs : (long long)rows * rs) * 4};
+    cuuint32_t box[3] = {(cuuint32_t)atom_k, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    const int row_bytes = atom_k * 4;
+    const CUtensorMapSwizzle swz = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                 : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+    CUresult r = fn(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base),
+                    dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? TT_OK : TT_ERR_CUDA;
+}
+
+const void* pick(const tt_tensors* t, int which) { return which == 0 ? t->x : t->w; }
+
+}  // namespace
+
+void release_device(tt_workload* w) {
+    if (w->workspace) cudaFree(w->workspace);
+    if (w->status_word) cudaFree(w->status_word);
+    for (int i = 0; i < 5; ++i) if (w->hbuf[i]) cudaFree(w->hbuf[i]);
+    w->workspace = nullptr; w->workspace_bytes = 0; w->status_word = nullptr;
+    for (int i = 0; i < 5; ++i) { w->hbuf[i] = nullptr; w->hbytes[i] = 0; }
+    cudaGetLastError();
+}
+
+tt_status bind_device(tt_workload* w) {
+    if (!device_present()) return TT_ERR_CUDA;
+    const size_t need = (size_t)w->plan.info.workspace_bytes;
+    if (need > w->workspace_bytes) {
+        if (w->workspace) cudaFree(w->workspace);
+        w->workspace = nullptr; w->workspace_bytes = 0;
+        if (cudaMalloc(&w->workspace, need) != cudaSuccess) { cudaGetLastError(); return TT_ERR_OOM; }
+        w->workspace_bytes = need;
+    }
+    if (!w->status_word) {
+        if (cudaMalloc(reinterpret_cast<void**>(&w->status_word), 16) != cudaSuccess) { cudaGetLastError(); return TT_ERR_OOM; }
+        if (cudaMemset(w->status_word, 0, 16) != cudaSuccess) return TT_ERR_CUDA;
+    }
+    w->tmaps.clear();
+    return TT_OK;
+}
+
+static tt_status tensor_maps_for(tt_workload* w, const void* a_ptr, const void* b_ptr, const TmapPair** out) {
+    for (const TmapPair& e : w->tmaps)
+        if (e.a_ptr == a_ptr && e.b_ptr == b_ptr) { *out = &e; return TT_OK; }
+    const GemmArgs& g = w->plan.g;
+    TmapPair e;
+    std::memset(&e, 0, sizeof e);
+    e.a_ptr = a_ptr; e.b_ptr = b_ptr;
+    // An operand that is gathered still needs a well-formed map in the kernel's parameter slot: encode the
+    // other operand's (or a self-describing dummy over the A tensor) so no parameter is uninitialised.
+    tt_status st = TT_OK;
+    if (g.a_mode == OPM_TMA)
+        st = encode_operand(e.a, static_cast<const float*>(a_ptr), g.K, g.M, g.batch, g.a_rs, g.a_bs, g.a_tma_batched != 0,
+                            g.atom_k, kHwTileM);
+    if (st != TT_OK) return st;
+    if (g.b_mode == OPM_TMA)
+        st = encode_operand(e.b, static_cast<const float*>(b_ptr), g.K, g.N, g.batch, g.b_rs, g.b_bs, g.b_tma_batched != 0,
+                            g.atom_k, g.tile_n);
+    if (st != TT_OK) return st;
+    if (w->tmaps.size() >= 256) w->tmaps.clear();
+    w->tmaps.push_back(e);
+    *out = &w->tmaps.back();
+    return TT_OK;
+}
+
+tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
+    if (!w || !t) return TT_ERR_INVALID_ARG;
+    if (!w->plan.applied) return TT_ERR_NOT_APPLIED;
+    if (!t->x || !t->y) return TT_ERR_INVALID_ARG;
+    if (w->op != TT_OP_SOFTMAX && !t->w) return TT_ERR_INVALID_ARG;
+    if (w->sh.has_bias && !t->bias) return TT_ERR_INVALID_ARG;
+    if (w->sh.has_residual && !t->residual) return TT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaSuccess;
+    const Plan& p = w->plan;
+    if (w->family == TT_FAMILY_GEMM_TC) {
+        GemmArgs g = p.g;
+        ReduceArgs red = p.red;
+        const void* a_ptr = pick(t, p.a_tensor);
+        const void* b_ptr = pick(t, p.b_tensor);
+        const TmapPair* maps = nullptr;
+        tt_status s = tensor_maps_for(w, a_ptr, b_ptr, &maps);
+        if (s != TT_OK) return s;
+        g.a = static_cast<const float*>(a_ptr);
+        g.b = static_cast<const float*>(b_ptr);
+        g.y = static_cast<float*>(t->y);
+        g.bias = w->sh.has_bias ? static_cast<const float*>(t->bias) : nullptr;
+        g.residual = w->sh.has_residual ? static_cast<const float*>(t->residual) : nullptr;
+        g.partial = static_cast<float*>(w->workspace);
+        g.status = w->status_word;
+        if ((reinterpret_cast<uintptr_t>(t->y) & 15u) != 0) { g.vec_store = 0; red.vec = 0; }
+        red.partial = g.partial; red.y = g.y; red.bias = g.bias; red.residual = g.residual;
+        e = launch_gemm(p.info, g, red, maps->a, maps->b, st);
+    } else if (w->family == TT_FAMILY_DW_SIMT) {
+        DwArgs d = p.dw;
+        d.x = static_cast<const float*>(t->x); d.w = static_cast<const float*>(t->w);
+        d.bias = w->sh.has_bias ? static_cast<const float*>(t->bias) : nullptr;
+        d.y = static_cast<float*>(t->y);
+        if ((reinterpret_cast<uintptr_t>(t->y) & 15u) != 0) d.vec = 1;
+        e = launch_dw(p.info, d, st);
+    } else {
+        RowArgs r = p.row;
+        r.x = static_cast<const float*>(t->x); r.y = static_cast<float*>(t->y);
+        if (((reinterpret_cast<uintptr_t>(t->y) | reinterpret_cast<uintptr_t>(t->x)) & 15u) != 0) r.vec = 1;
+        e = launch_row(p.info, r, st);
+    }
+    if (e != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    return TT_OK;
+}
+
+static tt_status read_status(tt_workload* w, cudaStream_t st) {
+    if (!w->status_word) return TT_ERR_NOT_APPLIED;
+    if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    unsigned v = 0;
+    if (cudaMemcpy(&v, w->status_word, 4, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    if (v != 0) {
+        cudaMemset(w->status_word, 0, 4);
+        return (tt_status)(v & 0xffu);
+    }
+    return TT_OK;
+}
+
+static void default_timing(tt_timing_opts* o) {
+    if (o->warmup_batches <= 0) o->warmup_batches = 3;
+    if (o->batches <= 0) o->batches = 10;
+    if (o->min_batch_us <= 0) o->min_batch_us = 200;
+    if (o->max_repeats <= 0) o->max_repeats = 4096;
+}
+
+static float median_of(std::vector<float>& v, float* q1, float* q3) {
+    std::sort(v.begin(), v.end());
+    const size_t n = v.size();
+    auto at = [&](double pos) {
+        const size_t lo = (size_t)pos;
+        const size_t hi = std::min(lo + 1, n - 1);
+        const double f = pos - (double)lo;
+        return (float)(v[lo] * (1.0 - f) + v[hi] * f);
+    };
+    if (q1) *q1 = at(0.25 * (n - 1));
+    if (q3) *q3 = at(0.75 * (n - 1));
+    // even count: mean of the two middle order statistics
+    return (n & 1) ? v[n / 2] : 0.5f * (v[n / 2 - 1] + v[n / 2]);
+}
+
+static tt_status time_applied(tt_workload* w, const tt_tensors* sets, size_t n_sets, cudaStream_t st,
+                              const tt_timing_opts* oin, tt_timing* out) {
+    tt_timing_opts o{};
+    if (oin) o = *oin;
+    default_timing(&o);
+    if (n_sets == 0) return TT_ERR_INVALID_ARG;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    cudaStream_t cap = nullptr;
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t gexec = nullptr;
+    tt_status rc = TT_OK;
+    size_t next = 0;
+    auto fail = [&](tt_status s) { rc = s; };
+    auto run_n = [&](int n, cudaStream_t s) -> tt_status {
+        for (int i = 0; i < n; ++i) {
+            tt_status r = launch(w, &sets[next], s);
+            next = (next + 1) % n_sets;
+            if (r != TT_OK) return r;
+        }
+        return TT_OK;
+    };
+    do {
+        if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) { fail(TT_ERR_CUDA); break; }
+        // first launch alone: surfaces launch errors and a tripped wait before anything is timed
+        if ((rc = run_n(1, st)) != TT_OK) break;
+        if ((rc = read_status(w, st)) != TT_OK) break;
+        // calibrate the number of launches per batch
+        float ms = 0.f;
+        const int probe = 4;
+        cudaEventRecord(e0, st);
+        if ((rc = run_n(probe, st)) != TT_OK) break;
+        cudaEventRecord(e1, st);
+        if (cudaEventSynchronize(e1) != cudaSuccess) { fail(TT_ERR_CUDA); break; }
+        cudaEventElapsedTime(&ms, e0, e1);
+        const double est_us = std::max(0.2, (double)ms * 1000.0 / probe);
+        int reps = (int)std::min<double>((double)o.max_repeats, std::max(1.0, std::ceil(o.min_batch_us / est_us)));
+        if (o.use_graph) {
+            // one batch = one graph of `reps` launches: no CPU launch gaps between them
+            reps = (int)((reps + n_sets - 1) / n_sets * n_sets);      // every replay walks the sets identically
+            if (cudaStreamCreateWithFlags(&cap, cudaStreamNonBlocking) != cudaSuccess) { fail(TT_ERR_CUDA); break; }
+            // tensor maps must exist before capture (encoding is host work, but keep the capture pure launches)
+            if (cudaStreamBeginCapture(cap, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { fail(TT_ERR_CUDA); break; }
+            tt_status r = run_n(reps, cap);
+            cudaError_t ce = cudaStreamEndCapture(cap, &graph);
+            if (r != TT_OK) { fail(r); break; }
+            if (ce != cudaSuccess || !graph) { fail(TT_ERR_CUDA); break; }
+            if (cudaGraphInstantiate(&gexec, graph, 0) != cudaSuccess) { fail(TT_ERR_CUDA); break; }
+        }
+        std::vector<float> per;
+        per.reserve(o.batches);
+        for (int b = 0; b < o.warmup_batches + o.batches; ++b) {
+            cudaEventRecord(e0, st);
+            if (gexec) {
+                if (cudaGraphLaunch(gexec, st) != cudaSuccess) { fail(TT_ERR_CUDA); break; }
+            } else if ((rc = run_n(reps, st)) != TT_OK) break;
+            cudaEventRecord(e1, st);
+            if (cudaEventSynchronize(e1) != cudaSuccess) { fail(TT_ERR_CUDA); break; }
+            cudaEventElapsedTime(&ms, e0, e1);
+            if (b >= o.warmup_batches) per.push_back(ms * 1000.f / (float)reps);
+        }
+        if (rc != TT_OK) break;
+        if ((rc = read_status(w, st)) != TT_OK) break;
+        tt_timing t{};
+        t.repeats = reps; t.batches = (int)per.size();
+        t.median_us = median_of(per, &t.q1_us, &t.q3_us);
+        t.min_us = per.front(); t.max_us = per.back();
+        *out = t;
+    } while (false);
+    if (gexec) cudaGraphExecDestroy(gexec);
+    if (graph) cudaGraphDestroy(graph);
+    if (cap) cudaStreamDestroy(cap);
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    if (rc == TT_ERR_CUDA) cudaGetLastError();
+    return rc;
+}
+
+static tt_status apply_impl(tt_workload* w, const tt_schedule_record* rec, int mode, int strict_class, tt_apply_info* info) {
+    if (!w || !rec) return TT_ERR_INVALID_ARG;
+    Plan np;
+    tt_status s = legalise(w, rec, mode, strict_class, &np);
+    if (info && (s == TT_OK || s == TT_ERR_RESOURCE)) *info = np.info;
+    if (s != TT_OK) return s;                     // the previously applied record, if any, stays in force
+    Plan old = w->plan;
+    w->plan = np;
+    s = bind_device(w);
+    if (s != TT_OK) { w->plan = old; w->plan.applied = false; return s; }
+    w->plan.applied = true;
+    return TT_OK;
+}
+
+}  // namespace tt
+
+using namespace tt;
+
+extern "C" {
+
+tt_status tt_schedule_apply(tt_workload* w, const tt_schedule_record* rec, tt_apply_info* info_out) {
+    return apply_impl(w, rec, TT_MODE_LEGALISE, 0, info_out);
+}
+
+tt_status tt_schedule_apply_ex(tt_workload* w, const tt_schedule_record* rec, int32_t mode, int32_t strict_class,
+                               tt_apply_info* info_out) {
+    if (mode != TT_MODE_LEGALISE && mode != TT_MODE_STRICT) return TT_ERR_INVALID_ARG;
+    return apply_impl(w, rec, mode, strict_class, info_out);
+}
+
+tt_status tt_run(tt_workload* w, const tt_tensors* t, void* cuda_stream) { return launch(w, t, cuda_stream); }
+
+tt_status tt_workload_status(tt_workload* w, void* cuda_stream) {
+    if (!w) return TT_ERR_INVALID_ARG;
+    return read_status(w, static_cast<cudaStream_t>(cuda_stream));
+}
+
+tt_status tt_run_host(tt_workload* w, const tt_tensors* host, void* cuda_stream, int64_t* bytes_h2d, int64_t* bytes_d2h) {
+    if (!w || !host) return TT_ERR_INVALID_ARG;
+    if (!w->plan.applied) return TT_ERR_NOT_APPLIED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const void* src[4] = {host->x, host->w, host->bias, host->residual};
+    int64_t up = 0;
+    for (int i = 0; i < 5; ++i) {
+        const size_t bytes = tensor_elems(w, i) * 4;
+        if (bytes == 0) continue;
+        if (i < 4 && !src[i]) return TT_ERR_INVALID_ARG;
+        if (bytes > w->hbytes[i]) {
+            if (w->hbuf[i]) cudaFree(w->hbuf[i]);
+            w->hbuf[i] = nullptr; w->hbytes[i] = 0;
+            if (cudaMalloc(&w->hbuf[i], bytes) != cudaSuccess) { cudaGetLastError(); return TT_ERR_OOM; }
+            w->hbytes[i] = bytes;
+        }
+        if (i < 4) {
+            if (cudaMemcpyAsync(w->hbuf[i], src[i], bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+            up += (int64_t)bytes;
+        }
+    }
+    if (!host->y) return TT_ERR_INVALID_ARG;
+    tt_tensors dev{w->hbuf[0], w->hbuf[1], w->hbuf[2], w->hbuf[3], w->hbuf[4]};
+    tt_status s = launch(w, &dev, st);
+    if (s != TT_OK) return s;
+    const size_t ybytes = tensor_elems(w, 4) * 4;
+    if (cudaMemcpyAsync(host->y, w->hbuf[4], ybytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    s = read_status(w, st);
+    if (bytes_h2d) *bytes_h2d = up;
+    if (bytes_d2h) *bytes_d2h = (int64_t)ybytes;
+    return s;
+}
+
+tt_status tt_time(tt_workload* w, const tt_tensors* sets, size_t n_sets, void* cuda_stream, const tt_timing_opts* o,
+                  tt_timing* out) {
+    if (!w || !sets || !out) return TT_ERR_INVALID_ARG;
+    if (!w->plan.applied) return TT_ERR_NOT_APPLIED;
+    return time_applied(w, sets, n_sets, static_cast<cudaStream_t>(cuda_stream), o, out);
+}
+
+tt_status tt_transfer_tune(tt_workload* const* wls, const tt_tensors* tensors, size_t n_wl, const tt_schedule_record* pool,
+                           size_t n_pool, const tt_tune_opts* oin, void* cuda_stream, tt_tune_result* out) {
+    if (!wls || !tensors || !out || (n_pool && !pool) || !out->chosen || !out->best_us || !out->times_us || !out->status)
+        return TT_ERR_INVALID_ARG;
+    tt_tune_opts o{};
+    o.include_default = 1;
+    if (oin) o = *oin;
+    if (!device_present()) return TT_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const auto t_begin = std::chrono::steady_clock::now();
+    const size_t n_cols = n_pool + 1;
+    int timed = 0, invalid = 0;
+    std::vector<tt_schedule_record> cols(n_cols);
+    for (size_t i = 0; i < n_wl; ++i) {
+        tt_workload* w = wls[i];
+        if (!w) return TT_ERR_INVALID_ARG;
+        tt_default_schedule(w, &cols[0]);
+        for (size_t j = 0; j < n_pool; ++j) cols[j + 1] = pool[j];
+        for (size_t j = 0; j < n_cols; ++j) {
+            float& cell = out->times_us[i * n_cols + j];
+            int32_t& cst = out->status[i * n_cols + j];
+            cell = -1.f;
+            if (j == 0 && !o.include_default) { cst = TT_ERR_INVALID_SCHEDULE; continue; }
+            // the default record is the workload's own: never subject to the class rule
+            tt_status s = apply_impl(w, &cols[j], j == 0 ? TT_MODE_LEGALISE : o.mode, j == 0 ? 0 : o.strict_class, nullptr);
+            if (s == TT_OK) {
+                tt_timing tm{};
+                s = time_applied(w, &tensors[i], 1, st, &o.timing, &tm);
+                if (s == TT_OK) { cell = tm.median_us; ++timed; }
+            }
+            cst = s;
+            if (s != TT_OK) {
+                if (s == TT_ERR_CUDA || s == TT_ERR_OOM) return s;   // the device is unwell: stop, do not mislabel
+                ++invalid;                                          // an invalid pair is a result, not a failure
+            }
+        }
+        tt_select(&out->times_us[i * n_cols], 1, n_cols, &out->chosen[i]);
+        const int c = out->chosen[i];
+        out->best_us[i] = c >= 0 ? out->times_us[i * n_cols + c] : -1.f;
+        if (c >= 0) {
+            tt_status s = apply_impl(w, &cols[c], c == 0 ? TT_MODE_LEGALISE : o.mode, c == 0 ? 0 : o.strict_class, nullptr);
+            if (s != TT_OK) return s;
+        }
+    }
+    out->pairs_timed = timed; out->pairs_invalid = invalid;
+    out->search_seconds = std::chrono::duration<double>(std::chrono::steady_clock::now() - t_begin).count();
+    return TT_OK;
+}
+
+tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, const tt_timing_opts* o, int32_t level,
+                       size_t top_k, tt_schedule_record* out_records, float* out_us, size_t* n_out, int32_t* n_tried) {
+    if (!w || !t || !out_records || !out_us || !n_out || top_k == 0) return TT_ERR_INVALID_ARG;
+    if (!device_present()) return TT_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    tt_schedule_record base;
+    tt_default_schedule(w, &base);
+    std::vector<tt_schedule_record> cand;
+    auto push = [&](const tt_schedule_record& r) {
+        // keep only records that are legal as written: a record that needs rounding duplicates another candidate
+        tt_apply_info info;
+        if (tt_schedule_check(w, &r, TT_MODE_LEGALISE, 0, &info) != TT_OK) return;
+        if (info.changed & ~TT_CHG_TILE_M) return;
+        cand.push_back(info.legal);
+    };
+    const bool full = level > 0;
+    if (w->family == TT_FAMILY_GEMM_TC) {
+        const std::vector<int> tns = full ? std::vector<int>{16, 32, 48, 64, 96, 128, 192, 256} : std::vector<int>{32, 64, 128, 256};
+        const std::vector<int> tks = full ? std::vector<int>{8, 16, 32, 64, 128} : std::vector<int>{16, 32, 64};
+        const std::vector<int> sts = full ? std::vector<int>{2, 3, 4, 6} : std::vector<int>{2, 4};
+        const std::vector<int> sks = full ? std::vector<int>{1, 2, 3, 4, 6, 8, 12, 16, 24, 32} : std::vector<int>{1, 2, 4, 8, 16};
+        const std::vector<int> ras = full ? std::vector<int>{0, 1} : std::vector<int>{0};
+        for (int ax : {1, 2}) for (int tn : tns) for (int tk : tks) for (int sg : sts) for (int sk : sks) for (int ra : ras) {
+            tt_schedule_record r = base;
+            r.mma_m_axis = ax; r.tile_m = kHwTileM; r.tile_n = tn; r.tile_k = tk; r.stages = sg; r.split_k = sk; r.raster = ra;
+            push(r);
+        }
+    } else if (w->family == TT_FAMILY_DW_SIMT) {
+        const std::vector<int> tcs = full ? std::vector<int>{1, 2, 4, 8, 16, 32} : std::vector<int>{1, 4, 16};
+        const std::vector<int> bys = full ? std::vector<int>{1, 2, 4, 7, 8, 14, 16, 28} : std::vector<int>{4, 8, 16};
+        const std::vector<int> bxs = full ? std::vector<int>{8, 16, 28, 32, 56, 64, 112} : std::vector<int>{16, 32, 64};
+        const std::vector<int> its = full ? std::vector<int>{1, 2, 4, 8} : std::vector<int>{1, 4};
+        for (int tc : tcs) for (int by : bys) for (int bx : bxs) for (int it : its) for (int vw : {1, 4}) for (int th : {128, 256}) {
+            tt_schedule_record r = base;
+            r.tile_m = tc; r.block_y = by; r.block_x = bx; r.items_per_thread = it; r.vec_width = vw; r.threads = th;
+            push(r);
+        }
+    } else {
+        for (int bx : {4, 8, 16, 32}) for (int by : {1, 2, 4, 8, 16}) for (int vw : {1, 2, 4}) {
+            tt_schedule_record r = base;
+            r.block_x = bx; r.block_y = by; r.vec_width = vw;
+            push(r);
+        }
+    }
+    // drop exact duplicates (legalisation can map different inputs to one record)
+    std::vector<tt_schedule_record> uniq;
+    for (const auto& r : cand) {
+        bool dup = false;
+        for (const auto& u : uniq) if (std::memcmp(&u, &r, sizeof r) == 0) { dup = true; break; }
+        if (!dup) uniq.push_back(r);
+    }
+    std::vector<std::pair<float, size_t>> timed;
+    for (size_t i = 0; i < uniq.size(); ++i) {
+        tt_status s = apply_impl(w, &uniq[i], TT_MODE_LEGALISE, 0, nullptr);
+        if (s == TT_ERR_OOM || s == TT_ERR_CUDA) return s;
+        if (s != TT_OK) continue;
+        tt_timing tm{};
+        s = time_applied(w, t, 1, st, o, &tm);
+        if (s == TT_ERR_CUDA || s == TT_ERR_OOM) return s;
+        if (s == TT_OK) timed.emplace_back(tm.median_us, i);
+    }
+    if (n_tried) *n_tried = (int32_t)uniq.size();
+    std::stable_sort(timed.begin(), timed.end(), [](const auto& a, const auto& b) { return a.first < b.first; });
+    const size_t n = std::min(top_k, timed.size());
+    for (size_t i = 0; i < n; ++i) {
+        out_records[i] = uniq[timed[i].second];
+        out_records[i].origin_op = w->op;
+        out_records[i].origin = w->sh;
+        out_us[i] = timed[i].first;
+    }
+    *n_out = n;
+    if (n > 0) return apply_impl(w, &out_records[0], TT_MODE_LEGALISE, 0, nullptr);
+    return TT_ERR_INVALID_SCHEDULE;
+}
+
+}  // extern "C"

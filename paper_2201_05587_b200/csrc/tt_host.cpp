@@ -1,0 +1,491 @@
+// Host logic of libtt: workloads, kernel classes, schedule records, the transfer /
+// legalisation / validity layer, the selector.  Nothing here touches the device.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include "tt_internal.h"
+
+using namespace tt;
+
+namespace {
+
+uint64_t fnv1a(const void* data, size_t n, uint64_t h = 1469598103934665603ull) {
+    const unsigned char* p = static_cast<const unsigned char*>(data);
+    for (size_t i = 0; i < n; ++i) { h ^= p[i]; h *= 1099511628211ull; }
+    return h;
+}
+
+int round_up(int v, int m) { return (v + m - 1) / m * m; }
+int pow2_ceil(int v) { int p = 1; while (p < v) p <<= 1; return p; }
+int pow2_floor(int v) { int p = 1; while (p * 2 <= v) p <<= 1; return p; }
+
+int family_of(tt_op op) {
+    switch (op) {
+        case TT_OP_CONV2D: case TT_OP_DENSE: case TT_OP_BATCH_MATMUL: return TT_FAMILY_GEMM_TC;
+        case TT_OP_DWCONV2D: return TT_FAMILY_DW_SIMT;
+        case TT_OP_SOFTMAX: return TT_FAMILY_ROW_SIMT;
+    }
+    return -1;
+}
+
+bool conv_like(tt_op op) { return op == TT_OP_CONV2D || op == TT_OP_DWCONV2D; }
+
+}  // namespace
+
+namespace tt {
+
+uint64_t class_hash(int op, const tt_shapes& s) {
+    // A kernel class is the sequence of operators, regardless of data sizes (Section 4.2).
+    int32_t v[5] = {op, s.has_bias != 0, s.act, s.has_residual != 0, op == TT_OP_BATCH_MATMUL ? (s.trans_b != 0) : 0};
+    return fnv1a(v, sizeof v);
+}
+
+size_t tensor_elems(const tt_workload* w, int which) {
+    const tt_shapes& s = w->sh;
+    switch (w->op) {
+        case TT_OP_CONV2D:
+            switch (which) {
+                case 0: return (size_t)s.n * s.c * s.h * s.w;
+                case 1: return (size_t)s.k * s.c * s.r * s.s;
+                case 2: return s.has_bias ? (size_t)s.k : 0;
+                case 3: return s.has_residual ? (size_t)s.n * s.k * w->P * w->Q : 0;
+                default: return (size_t)s.n * s.k * w->P * w->Q;
+            }
+        case TT_OP_DWCONV2D:
+            switch (which) {
+                case 0: return (size_t)s.n * s.c * s.h * s.w;
+                case 1: return (size_t)s.c * s.r * s.s;
+                case 2: return s.has_bias ? (size_t)s.c : 0;
+                case 3: return 0;
+                default: return (size_t)s.n * s.c * w->P * w->Q;
+            }
+        case TT_OP_DENSE:
+        case TT_OP_BATCH_MATMUL:
+            switch (which) {
+                case 0: return (size_t)s.batch * s.m * s.kk;
+                case 1: return (size_t)s.batch * s.nn * s.kk;
+                case 2: return s.has_bias ? (size_t)s.nn : 0;
+                case 3: return s.has_residual ? (size_t)s.batch * s.m * s.nn : 0;
+                default: return (size_t)s.batch * s.m * s.nn;
+            }
+        case TT_OP_SOFTMAX:
+            return (which == 0 || which == 4) ? (size_t)s.batch * s.m * s.nn : 0;
+    }
+    return 0;
+}
+
+// ---- legalisation -------------------------------------------------------------------------------------------
+
+static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* rec, int mode, Plan* plan) {
+    tt_schedule_record L = *rec;
+    int changed = 0;
+    const bool strict = mode == TT_MODE_STRICT;
+    if (rec->tile_m <= 0 || rec->tile_n <= 0 || rec->tile_k <= 0 || rec->stages <= 0 || rec->split_k <= 0 ||
+        rec->raster < 0 || rec->raster > 1 || rec->mma_m_axis < 0 || rec->mma_m_axis > 2)
+        return TT_ERR_INVALID_SCHEDULE;
+    // Which output axis becomes the accumulator's 128 rows.  Left to the library (0), the shorter-than-a-tile
+    // axis goes to the MMA's N side, where 16..256 columns are legal.
+    const tt_shapes& s = w->sh;
+    bool swap = rec->mma_m_axis == 2;
+    if (rec->mma_m_axis == 0) swap = w->view.gm <= 64 && w->view.gn > w->view.gm;
+    L.mma_m_axis = swap ? 2 : 1;
+    plan->swap_ab = swap;
+    plan->gm = swap ? w->view.gn : w->view.gm;
+    plan->gn = swap ? w->view.gm : w->view.gn;
+    const int M = plan->gm, N = plan->gn, K = plan->gk, B = plan->gbatch;
+    // A split factor larger than the loop itself is invalid code when nothing may be reformulated (Section 4.2).
+    if (strict && (rec->tile_m > round_up(M, 32) || rec->tile_n > round_up(N, 16) || rec->tile_k > round_up(K, 8)))
+        return TT_ERR_INVALID_SCHEDULE;
+    // tile_m: the accumulator always spans 128 tensor-memory lanes; smaller logical tiles leave rows idle.
+    L.tile_m = kHwTileM;
+    if (L.tile_m != rec->tile_m) changed |= TT_CHG_TILE_M;
+    // tile_n: legal MMA N for M = 128 is a multiple of 16 in [16, 256]; no wider than the padded extent.
+    int tn = std::min(256, std::max(16, round_up(rec->tile_n, 16)));
+    tn = std::min(tn, round_up(N, 16));
+    if (tn != rec->tile_n) changed |= TT_CHG_TILE_N;
+    L.tile_n = tn;
+    // tile_k: power of two in [8, 128] (one to four 128-byte swizzle atoms, or one 32/64-byte atom).
+    int tk = std::min(128, std::max(8, pow2_floor(rec->tile_k)));
+    tk = std::min(tk, std::max(8, pow2_ceil(K)));
+    if (tk != rec->tile_k) changed |= TT_CHG_TILE_K;
+    L.tile_k = tk;
+    int st = std::min(kMaxStages, rec->stages);
+    if (st != rec->stages) changed |= TT_CHG_STAGES;
+    L.stages = st;
+    const int k_tiles = (K + tk - 1) / tk;
+    int sk = rec->split_k;
+    if (sk > k_tiles) {
+        if (strict) return TT_ERR_INVALID_SCHEDULE;
+        sk = k_tiles;
+    }
+    const int per_split = (k_tiles + sk - 1) / sk;
+    sk = (k_tiles + per_split - 1) / per_split;          // every split owns at least one reduction tile
+    if (sk != rec->split_k) changed |= TT_CHG_SPLIT_K;
+    L.split_k = sk;
+    if (strict && (changed & ~TT_CHG_TILE_M)) return TT_ERR_INVALID_SCHEDULE;
+
+    const int atom_k = std::min(tk, 32), n_atoms = tk / atom_k, row_bytes = atom_k * 4;
+    const unsigned a_stage = (unsigned)n_atoms * kHwTileM * row_bytes;
+    const unsigned b_stage = (unsigned)n_atoms * tn * row_bytes;
+    const long long smem = (long long)st * (a_stage + b_stage) + 1024;
+    int tmem_cols = std::max(32, pow2_ceil(tn));
+    const int tiles_m = (M + kHwTileM - 1) / kHwTileM, tiles_n = (N + tn - 1) / tn;
+    if ((long long)tiles_m * tiles_n > 0x7fffffffLL || sk > 65535 || B > 65535) return TT_ERR_RESOURCE;
+
+    tt_apply_info& I = plan->info;
+    I = tt_apply_info{};
+    I.legal = L;
+    I.changed = changed;
+    I.grid_x = tiles_m * tiles_n; I.grid_y = sk; I.grid_z = B;
+    I.threads = kGemmThreads;
+    I.smem_bytes = (int)std::min<long long>(smem, 0x7fffffff);
+    I.tmem_cols = tmem_cols;
+    I.workspace_bytes = sk > 1 ? (int64_t)sk * B * M * N * 4 : 0;
+    I.launches = sk > 1 ? 2 : 1;
+    if (smem > kDynSmemLimit) return TT_ERR_RESOURCE;
+
+    GemmArgs& g = plan->g;
+    g = GemmArgs{};
+    g.M = M; g.N = N; g.K = K; g.batch = B;
+    g.tile_n = tn; g.tile_k = tk; g.stages = st;
+    g.k_tiles = k_tiles; g.k_tiles_per_split = per_split; g.split_k = sk;
+    g.tiles_m = tiles_m; g.tiles_n = tiles_n; g.raster = L.raster;
+    g.atom_k = atom_k; g.n_atoms = n_atoms; g.row_bytes = row_bytes;
+    g.swz_mask = row_bytes == 128 ? 7 : (row_bytes == 64 ? 3 : 1);
+    g.a_stage_bytes = a_stage; g.b_stage_bytes = b_stage;
+    g.tmem_cols = (unsigned)tmem_cols;
+    // Instruction descriptor, kind::tf32: D = F32 (bits 4-5 = 1), A and B = TF32 (bits 7-9, 10-12 = 2), both
+    // K-major (bits 15, 16 = 0), N >> 3 at bits 17-22, M >> 4 at bits 24-28.
+    g.idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(tn >> 3) << 17) | ((unsigned)(kHwTileM >> 4) << 24);
+    // Operands of the logical contraction Y[b][i][j] = sum_k U[b][i][k] V[b][j][k], then the optional swap.
+    struct Opnd { int mode; long long rs, ks, bs; int batched; } U{}, V{};
+    long long y_is, y_js, y_bs;
+    int bias_on;   // 1: bias indexed by i, 2: by j
+    const bool k4 = (K % 4) == 0;
+    if (w->op == TT_OP_CONV2D) {
+        U = {k4 ? OPM_TMA : OPM_GATHER_K, K, 1, 0, 0};                         // filters [k][c*r*s], shared by images
+        V = {OPM_IM2COL, 0, 0, (long long)s.c * s.h * s.w, 1};                 // pixels x (c,r,s) gathered from NCHW
+        y_is = (long long)w->P * w->Q; y_js = 1; y_bs = (long long)s.k * w->P * w->Q; bias_on = 1;
+    } else if (w->op == TT_OP_DENSE) {
+        U = {k4 ? OPM_TMA : OPM_GATHER_K, K, 1, 0, 0};
+        V = {k4 ? OPM_TMA : OPM_GATHER_K, K, 1, 0, 0};
+        y_is = s.nn; y_js = 1; y_bs = 0; bias_on = 2;
+    } else {
+        U = {k4 ? OPM_TMA : OPM_GATHER_K, K, 1, (long long)s.m * K, 1};
+        if (s.trans_b) V = {k4 ? OPM_TMA : OPM_GATHER_K, K, 1, (long long)s.nn * K, 1};
+        else V = {OPM_GATHER_ROWS, 1, s.nn, (long long)s.nn * K, 1};           // w[b][k][j]: rows j are contiguous
+        y_is = s.nn; y_js = 1; y_bs = (long long)s.m * s.nn; bias_on = 2;
+    }
+    const int u_tensor = w->op == TT_OP_CONV2D ? 1 : 0;       // conv: U is the filter tensor; dense/bmm: U is x
+    plan->a_tensor = swap ? 1 - u_tensor : u_tensor;
+    plan->b_tensor = 1 - plan->a_tensor;
+    const Opnd& A = swap ? V : U;
+    const Opnd& Bo = swap ? U : V;
+    g.a_mode = A.mode; g.a_rs = A.rs; g.a_ks = A.ks; g.a_bs = A.bs; g.a_tma_batched = A.batched;
+    g.b_mode = Bo.mode; g.b_rs = Bo.rs; g.b_ks = Bo.ks; g.b_bs = Bo.bs; g.b_tma_batched = Bo.batched;
+    g.y_ms = swap ? y_js : y_is; g.y_ns = swap ? y_is : y_js; g.y_bs = y_bs;
+    g.bias_mode = s.has_bias ? (swap ? 3 - bias_on : bias_on) : 0;
+    g.act = s.act;
+    g.C = s.c; g.H = s.h; g.W = s.w; g.R = s.r; g.S = s.s; g.Q = w->Q;
+    g.sh = s.stride_h; g.sw = s.stride_w; g.ph = s.pad_h; g.pw = s.pad_w;
+    g.tx_bytes = (A.mode == OPM_TMA ? a_stage : 0) + (Bo.mode == OPM_TMA ? b_stage : 0);
+    g.vec_store = (g.y_ns == 1 && g.y_ms % 4 == 0 && g.y_bs % 4 == 0) ? 1 : 0;
+    // the split-K reduction kernel reads [split][batch][M][N] and writes y through the same strides
+    ReduceArgs& r = plan->red;
+    r = ReduceArgs{};
+    r.split_k = sk; r.batch = B; r.M = M; r.N = N; r.y_ms = g.y_ms; r.y_ns = g.y_ns; r.y_bs = g.y_bs;
+    r.bias_mode = g.bias_mode; r.act = g.act; r.vec = (g.vec_store && N % 4 == 0) ? 1 : 0;
+    return TT_OK;
+}
+
+static tt_status legalise_dw(const tt_workload* w, const tt_schedule_record* rec, int mode, Plan* plan) {
+    const tt_shapes& s = w->sh;
+    const bool strict = mode == TT_MODE_STRICT;
+    tt_schedule_record L = *rec;
+    int changed = 0;
+    if (rec->tile_m <= 0 || rec->block_x <= 0 || rec->block_y <= 0 || rec->items_per_thread <= 0 ||
+        rec->vec_width <= 0 || rec->threads <= 0)
+        return TT_ERR_INVALID_SCHEDULE;
+    if (strict && (rec->tile_m > s.c || rec->block_y > w->P || rec->block_x > round_up(w->Q, 4)))
+        return TT_ERR_INVALID_SCHEDULE;
+    L.tile_m = std::min(rec->tile_m, s.c);
+    if (L.tile_m != rec->tile_m) changed |= TT_CHG_TILE_M;
+    L.block_y = std::min(rec->block_y, w->P);
+    int vec = rec->vec_width >= 4 ? 4 : (rec->vec_width >= 2 ? 2 : 1);
+    while (vec > 1 && (w->Q % vec) != 0) vec >>= 1;        // rows of y must stay vector-aligned
+    int items = std::min(8, pow2_floor(rec->items_per_thread));
+    items = std::max(items, vec);
+    int bx = std::min(rec->block_x, round_up(w->Q, items));
+    bx = round_up(bx, items);
+    if (bx != rec->block_x || L.block_y != rec->block_y) changed |= TT_CHG_BLOCK;
+    L.block_x = bx;
+    if (items != rec->items_per_thread) changed |= TT_CHG_ITEMS;
+    L.items_per_thread = items;
+    if (vec != rec->vec_width) changed |= TT_CHG_VEC;
+    L.vec_width = vec;
+    int th = std::min(1024, std::max(32, round_up(rec->threads, 32)));
+    if (th != rec->threads) changed |= TT_CHG_BLOCK;
+    L.threads = th;
+    if (strict && changed) return TT_ERR_INVALID_SCHEDULE;
+
+    DwArgs& d = plan->dw;
+    d = DwArgs{};
+    d.N = s.n; d.C = s.c; d.H = s.h; d.W = s.w; d.R = s.r; d.S = s.s; d.P = w->P; d.Q = w->Q;
+    d.sh = s.stride_h; d.sw = s.stride_w; d.ph = s.pad_h; d.pw = s.pad_w; d.act = s.act;
+    d.tile_c = L.tile_m; d.tile_h = L.block_y; d.tile_w = L.block_x;
+    d.in_h = (d.tile_h - 1) * d.sh + d.R;
+    d.in_w = (d.tile_w - 1) * d.sw + d.S;
+    d.items = items; d.vec = vec;
+    d.tiles_c = (s.c + d.tile_c - 1) / d.tile_c;
+    d.tiles_h = (w->P + d.tile_h - 1) / d.tile_h;
+    d.tiles_w = (w->Q + d.tile_w - 1) / d.tile_w;
+    const long long smem = (long long)d.tile_c * ((long long)d.in_h * d.in_w + d.R * d.S + 1) * 4;
+    tt_apply_info& I = plan->info;
+    I = tt_apply_info{};
+    I.legal = L; I.changed = changed;
+    const long long gx = (long long)d.tiles_w * d.tiles_h * d.tiles_c;
+    I.grid_x = (int)std::min<long long>(gx, 0x7fffffff); I.grid_y = s.n; I.grid_z = 1;
+    I.threads = th; I.smem_bytes = (int)std::min<long long>(smem, 0x7fffffff);
+    I.launches = 1;
+    if (smem > kDynSmemLimit || gx > 0x7fffffffLL || s.n > 65535) return TT_ERR_RESOURCE;
+    return TT_OK;
+}
+
+static tt_status legalise_row(const tt_workload* w, const tt_schedule_record* rec, int mode, Plan* plan) {
+    const tt_shapes& s = w->sh;
+    const bool strict = mode == TT_MODE_STRICT;
+    tt_schedule_record L = *rec;
+    int changed = 0;
+    if (rec->block_x <= 0 || rec->block_y <= 0 || rec->vec_width <= 0) return TT_ERR_INVALID_SCHEDULE;
+    const long long rows = (long long)s.batch * s.m;
+    int lanes = std::min(32, pow2_floor(rec->block_x));
+    int vec = rec->vec_width >= 4 ? 4 : (rec->vec_width >= 2 ? 2 : 1);
+    while (vec > 1 && (s.nn % vec) != 0) vec >>= 1;
+    if (strict && (long long)rec->block_x * rec->vec_width > round_up(s.nn, 4)) return TT_ERR_INVALID_SCHEDULE;
+    int rpc = rec->block_y;
+    while ((rpc * lanes) % 32 != 0) ++rpc;                 // whole warps
+    if ((long long)rpc * lanes > 1024) rpc = 1024 / lanes;
+    if (lanes != rec->block_x || rpc != rec->block_y) changed |= TT_CHG_BLOCK;
+    if (vec != rec->vec_width) changed |= TT_CHG_VEC;
+    L.block_x = lanes; L.block_y = rpc; L.vec_width = vec;
+    if (strict && changed) return TT_ERR_INVALID_SCHEDULE;
+    RowArgs& r = plan->row;
+    r = RowArgs{};
+    r.rows = rows; r.cols = s.nn; r.scale = s.scale; r.lanes_per_row = lanes; r.rows_per_cta = rpc; r.vec = vec;
+    tt_apply_info& I = plan->info;
+    I = tt_apply_info{};
+    I.legal = L; I.changed = changed;
+    const long long gx = (rows + rpc - 1) / rpc;
+    I.grid_x = (int)std::min<long long>(gx, 0x7fffffff); I.grid_y = 1; I.grid_z = 1;
+    I.threads = rpc * lanes; I.launches = 1;
+    if (gx > 0x7fffffffLL) return TT_ERR_RESOURCE;
+    return TT_OK;
+}
+
+tt_status legalise(const tt_workload* w, const tt_schedule_record* rec, int mode, int strict_class, Plan* plan) {
+    if (!w || !rec || !plan) return TT_ERR_INVALID_ARG;
+    if (rec->version != TT_RECORD_VERSION) return TT_ERR_INVALID_SCHEDULE;
+    // A schedule written for another loop structure tries to transform loops that do not exist (Section 4.2).
+    if ((int)rec->family != w->family) return TT_ERR_CLASS_MISMATCH;
+    if (strict_class && class_hash(rec->origin_op, rec->origin) != class_hash(w->op, w->sh)) return TT_ERR_CLASS_MISMATCH;
+    plan->gm = w->view.gm; plan->gn = w->view.gn; plan->gk = w->view.gk; plan->gbatch = w->view.batch;
+    switch (w->family) {
+        case TT_FAMILY_GEMM_TC: return legalise_gemm(w, rec, mode, plan);
+        case TT_FAMILY_DW_SIMT: return legalise_dw(w, rec, mode, plan);
+        case TT_FAMILY_ROW_SIMT: return legalise_row(w, rec, mode, plan);
+    }
+    return TT_ERR_INVALID_ARG;
+}
+
+}  // namespace tt
+
+// ---- C ABI (host-only entry points) -------------------------------------------------------------------------
+
+extern "C" {
+
+const char* tt_status_string(tt_status s) {
+    switch (s) {
+        case TT_OK: return "ok";
+        case TT_ERR_INVALID_ARG: return "invalid argument";
+        case TT_ERR_INVALID_SCHEDULE: return "schedule invalid for this workload";
+        case TT_ERR_CLASS_MISMATCH: return "schedule belongs to another kernel class";
+        case TT_ERR_RESOURCE: return "schedule exceeds hardware resources";
+        case TT_ERR_NOT_APPLIED: return "no schedule applied";
+        case TT_ERR_CUDA: return "CUDA error";
+        case TT_ERR_TIMEOUT: return "device wait timed out";
+        case TT_ERR_OOM: return "out of device memory";
+        case TT_ERR_NOT_IMPLEMENTED: return "not implemented";
+    }
+    return "unknown status";
+}
+
+tt_status tt_workload_create(tt_op op, const tt_shapes* sp, tt_workload** out) {
+    if (!sp || !out) return TT_ERR_INVALID_ARG;
+    *out = nullptr;
+    const int fam = family_of(op);
+    if (fam < 0) return TT_ERR_INVALID_ARG;
+    tt_shapes s = *sp;
+    if (s.act < TT_ACT_NONE || s.act > TT_ACT_GELU_ERF) return TT_ERR_INVALID_ARG;
+    int P = 0, Q = 0;
+    tt_gemm_view v{};
+    if (conv_like(op)) {
+        if (s.n <= 0 || s.c <= 0 || s.h <= 0 || s.w <= 0 || s.r <= 0 || s.s <= 0 || s.stride_h <= 0 || s.stride_w <= 0 ||
+            s.pad_h < 0 || s.pad_w < 0)
+            return TT_ERR_INVALID_ARG;
+        if (op == TT_OP_CONV2D && s.k <= 0) return TT_ERR_INVALID_ARG;
+        if (s.h + 2 * s.pad_h < s.r || s.w + 2 * s.pad_w < s.s) return TT_ERR_INVALID_ARG;
+        if (op == TT_OP_DWCONV2D) { s.k = s.c; if (s.has_residual) return TT_ERR_INVALID_ARG; }
+        P = (s.h + 2 * s.pad_h - s.r) / s.stride_h + 1;
+        Q = (s.w + 2 * s.pad_w - s.s) / s.stride_w + 1;
+        s.batch = s.m = s.nn = s.kk = s.trans_b = 0;
+        if (op == TT_OP_CONV2D) {
+            // implicit GEMM: rows = filters, columns = output pixels, reduction = (c, r, s), one GEMM per image
+            v.batch = s.n; v.gm = s.k; v.gn = P * Q; v.gk = s.c * s.r * s.s;
+            v.flops = 2.0 * v.batch * v.gm * (double)v.gn * v.gk;
+            v.bytes = 4.0 * ((double)s.n * s.c * s.h * s.w + (double)s.k * v.gk + (s.has_bias ? s.k : 0) +
+                             (double)s.n * s.k * P * Q * (s.has_residual ? 2 : 1));
+        } else {
+            v.batch = s.n; v.gm = s.c; v.gn = P * Q; v.gk = s.r * s.s;
+            v.flops = 2.0 * s.n * s.c * (double)P * Q * s.r * s.s;
+            v.bytes = 4.0 * ((double)s.n * s.c * s.h * s.w + (double)s.c * s.r * s.s + (s.has_bias ? s.c : 0) +
+                             (double)s.n * s.c * P * Q);
+        }
+    } else {
+        if (op == TT_OP_DENSE) { s.batch = 1; s.trans_b = 1; }
+        if (s.batch <= 0 || s.m <= 0 || s.nn <= 0) return TT_ERR_INVALID_ARG;
+        if (op != TT_OP_SOFTMAX && s.kk <= 0) return TT_ERR_INVALID_ARG;
+        if (op == TT_OP_SOFTMAX) { s.kk = 0; s.has_bias = 0; s.has_residual = 0; s.act = TT_ACT_NONE; s.trans_b = 0; }
+        s.n = s.c = s.h = s.w = s.k = s.r = s.s = s.stride_h = s.stride_w = s.pad_h = s.pad_w = 0;
+        v.batch = s.batch; v.gm = s.m; v.gn = s.nn; v.gk = s.kk;
+        if (op == TT_OP_SOFTMAX) {
+            v.flops = 5.0 * s.batch * (double)s.m * s.nn;
+            v.bytes = 8.0 * s.batch * (double)s.m * s.nn;
+        } else {
+            v.flops = 2.0 * s.batch * (double)s.m * s.nn * s.kk;
+            v.bytes = 4.0 * ((double)s.batch * s.m * s.kk + (double)s.batch * s.nn * s.kk + (s.has_bias ? s.nn : 0) +
+                             (double)s.batch * s.m * s.nn * (s.has_residual ? 2 : 1));
+        }
+    }
+    if (op != TT_OP_SOFTMAX) s.scale = 0.f;
+    s.has_bias = s.has_bias != 0; s.has_residual = s.has_residual != 0;
+    tt_workload* w = new (std::nothrow) tt_workload();
+    if (!w) return TT_ERR_OOM;
+    w->op = op; w->sh = s; w->family = fam; w->P = P; w->Q = Q; w->view = v;
+    *out = w;
+    return TT_OK;
+}
+
+tt_status tt_workload_destroy(tt_workload* w) {
+    if (!w) return TT_ERR_INVALID_ARG;
+    tt::release_device(w);
+    delete w;
+    return TT_OK;
+}
+
+tt_status tt_workload_key(const tt_workload* w, uint64_t* key) {
+    if (!w || !key) return TT_ERR_INVALID_ARG;
+    int32_t op = w->op;
+    uint64_t h = fnv1a(&op, sizeof op);
+    // field by field: padding bytes of the struct never enter the hash
+    const tt_shapes& s = w->sh;
+    const int32_t f[] = {s.n, s.c, s.h, s.w, s.k, s.r, s.s, s.stride_h, s.stride_w, s.pad_h, s.pad_w,
+                         s.batch, s.m, s.nn, s.kk, s.trans_b, s.has_bias, s.has_residual, s.act};
+    h = fnv1a(f, sizeof f, h);
+    h = fnv1a(&s.scale, sizeof s.scale, h);
+    *key = h;
+    return TT_OK;
+}
+
+tt_status tt_workload_class(const tt_workload* w, uint64_t* cls) {
+    if (!w || !cls) return TT_ERR_INVALID_ARG;
+    *cls = tt::class_hash(w->op, w->sh);
+    return TT_OK;
+}
+
+tt_status tt_workload_family(const tt_workload* w, int32_t* family) {
+    if (!w || !family) return TT_ERR_INVALID_ARG;
+    *family = w->family;
+    return TT_OK;
+}
+
+tt_status tt_workload_gemm_view(const tt_workload* w, tt_gemm_view* out) {
+    if (!w || !out) return TT_ERR_INVALID_ARG;
+    *out = w->view;
+    return TT_OK;
+}
+
+tt_status tt_default_schedule(const tt_workload* w, tt_schedule_record* out) {
+    if (!w || !out) return TT_ERR_INVALID_ARG;
+    tt_schedule_record r;
+    std::memset(&r, 0, sizeof r);
+    r.version = TT_RECORD_VERSION;
+    r.family = (uint32_t)w->family;
+    r.origin_op = w->op;
+    r.origin = w->sh;
+    // One generic, shape-blind record per family: the counterpart of a compiler's default schedule.
+    r.tile_m = 128; r.tile_n = 128; r.tile_k = 32; r.stages = 4; r.split_k = 1; r.raster = 0;
+    r.block_x = 32; r.block_y = 4; r.items_per_thread = 1; r.vec_width = 1; r.unroll = 1; r.threads = 128;
+    if (w->family == TT_FAMILY_DW_SIMT) { r.tile_m = 1; r.block_x = 32; r.block_y = 8; }
+    if (w->family == TT_FAMILY_ROW_SIMT) { r.block_x = 32; r.block_y = 4; }
+    *out = r;
+    return TT_OK;
+}
+
+tt_status tt_schedule_check(const tt_workload* w, const tt_schedule_record* rec, int32_t mode, int32_t strict_class,
+                            tt_apply_info* info_out) {
+    if (!w || !rec) return TT_ERR_INVALID_ARG;
+    tt::Plan* p = new (std::nothrow) tt::Plan();
+    if (!p) return TT_ERR_OOM;
+    tt_status st = tt::legalise(w, rec, mode, strict_class, p);
+    if (info_out && (st == TT_OK || st == TT_ERR_RESOURCE)) *info_out = p->info;
+    delete p;
+    return st;
+}
+
+tt_status tt_split_check(int64_t extent, const int64_t* factors, size_t n, int32_t reformulate, int32_t* valid) {
+    if (!factors || !valid || n == 0 || extent <= 0) return TT_ERR_INVALID_ARG;
+    if (reformulate) {
+        // Split(N, N/f, f): the outer range adapts to the extent, so only divisibility remains.
+        *valid = factors[0] > 0 && extent % factors[0] == 0;
+        return TT_OK;
+    }
+    // Split(N, f0, f1, ...): fixed ranges must traverse the loop exactly.
+    __int128 prod = 1;
+    for (size_t i = 0; i < n; ++i) {
+        if (factors[i] <= 0) { *valid = 0; return TT_OK; }
+        prod *= factors[i];
+        if (prod > (__int128)extent) { *valid = 0; return TT_OK; }
+    }
+    *valid = prod == (__int128)extent;
+    return TT_OK;
+}
+
+tt_status tt_select(const float* times_us, size_t n_wl, size_t n_cols, int32_t* chosen) {
+    if (!times_us || !chosen || n_cols == 0) return TT_ERR_INVALID_ARG;
+    for (size_t i = 0; i < n_wl; ++i) {
+        int best = -1;
+        float bt = 0.f;
+        for (size_t j = 0; j < n_cols; ++j) {
+            const float t = times_us[i * n_cols + j];
+            if (!(t >= 0.f) || !std::isfinite(t)) continue;     // negative = invalid pair, NaN never wins
+            if (best < 0 || t < bt) { best = (int)j; bt = t; }
+        }
+        chosen[i] = best;
+    }
+    return TT_OK;
+}
+
+tt_status tt_model_latency(const float* times_us, size_t n_wl, size_t n_cols, const int32_t* chosen,
+                           const int32_t* use_count, double* latency_us) {
+    if (!times_us || !chosen || !use_count || !latency_us) return TT_ERR_INVALID_ARG;
+    double sum = 0.0;
+    for (size_t i = 0; i < n_wl; ++i) {
+        if (chosen[i] < 0 || (size_t)chosen[i] >= n_cols) continue;
+        sum += (double)use_count[i] * (double)times_us[i * n_cols + chosen[i]];
+    }
+    *latency_us = sum;
+    return TT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,110 @@
+// Internal declarations shared by the host logic and the CUDA launchers of libtt.
+#pragma once
+#include <cstdint>
+#include <cstddef>
+#include <vector>
+#include "tt.h"
+
+namespace tt {
+
+constexpr int kHwTileM = 128;           // tcgen05 accumulator rows per CTA (cta_group::1, M = 128)
+constexpr int kMaxStages = 8;
+constexpr int kSmemLimit = 232448;      // 227 KB opt-in shared memory per CTA on sm_100
+constexpr int kDynSmemLimit = kSmemLimit - 1024;  // what is left for dynamic shared memory beside barriers
+constexpr int kGemmThreads = 192;       // warp 0 TMA, warp 1 MMA + TMEM, warps 2-5 gather + epilogue
+
+// How one operand of the contraction reaches shared memory.
+enum OperandMode : int {
+    OPM_TMA = 0,          // K-major 2-D/3-D tensor map, hardware swizzle
+    OPM_GATHER_ROWS = 1,  // strided view, lanes walk rows (row stride 1): 16-byte swizzled stores
+    OPM_GATHER_K = 2,     // strided view, lanes walk k (k stride 1): 4-byte swizzled stores
+    OPM_IM2COL = 3        // rows are output pixels, k = (c, r, s): gathered from NCHW
+};
+
+// Device-side arguments of the GEMM_TC kernel (plain data, passed by value).
+struct GemmArgs {
+    int M, N, K, batch;
+    int tile_n, tile_k, stages;
+    int k_tiles, k_tiles_per_split, split_k;
+    int tiles_m, tiles_n, raster;
+    int atom_k, n_atoms, swz_mask, row_bytes;
+    int a_mode, b_mode;
+    const float* a; long long a_rs, a_ks, a_bs; int a_tma_batched;
+    const float* b; long long b_rs, b_ks, b_bs; int b_tma_batched;
+    int C, H, W, R, S, Q, sh, sw, ph, pw;       // im2col geometry of operand B
+    float* y; long long y_ms, y_ns, y_bs;
+    const float* bias; int bias_mode;           // 0 none, 1 per row (m), 2 per column (n)
+    int act;
+    const float* residual;
+    float* partial;                             // split-K partial sums [split][batch][M][N]
+    unsigned* status;
+    unsigned idesc, tmem_cols;
+    unsigned a_stage_bytes, b_stage_bytes, tx_bytes;
+    int vec_store;                              // 1: y rows allow aligned float4 stores
+};
+
+struct ReduceArgs {
+    const float* partial; float* y; const float* bias; const float* residual;
+    int split_k, batch, M, N; long long y_ms, y_ns, y_bs; int bias_mode, act, vec;
+};
+
+struct DwArgs {
+    const float* x; const float* w; const float* bias; float* y;
+    int N, C, H, W, R, S, P, Q, sh, sw, ph, pw, act;
+    int tile_c, tile_h, tile_w, in_h, in_w, items, vec;
+    int tiles_c, tiles_h, tiles_w;
+};
+
+struct RowArgs {
+    const float* x; float* y; long long rows; int cols; float scale;
+    int lanes_per_row, rows_per_cta, vec;
+};
+
+// Host-side plan of an applied record.
+struct Plan {
+    bool applied = false;
+    tt_apply_info info{};
+    // GEMM lowering
+    int gm = 0, gn = 0, gk = 0, gbatch = 1;
+    bool swap_ab = false;
+    int a_tensor = 0, b_tensor = 1;   // which caller tensor feeds operand A / B: 0 = x, 1 = w
+    GemmArgs g{};
+    ReduceArgs red{};
+    DwArgs dw{};
+    RowArgs row{};
+};
+
+struct TmapPair {
+    const void* a_ptr; const void* b_ptr;
+    alignas(64) unsigned char a[128];
+    alignas(64) unsigned char b[128];
+};
+
+}  // namespace tt
+
+struct tt_workload {
+    tt_op op;
+    tt_shapes sh;
+    int family;
+    int P, Q;                    // conv output size
+    tt_gemm_view view;
+    tt::Plan plan;
+    void* workspace = nullptr;   // device: split-K partials
+    size_t workspace_bytes = 0;
+    unsigned* status_word = nullptr;  // device
+    // device staging buffers of tt_run_host
+    void* hbuf[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    size_t hbytes[5] = {0, 0, 0, 0, 0};
+    std::vector<tt::TmapPair> tmaps;  // tensor maps encoded so far for the applied record, by operand pointers
+};
+
+namespace tt {
+// host logic (tt_host.cpp)
+tt_status legalise(const tt_workload* w, const tt_schedule_record* rec, int mode, int strict_class, Plan* plan);
+uint64_t class_hash(int op, const tt_shapes& s);
+size_t tensor_elems(const tt_workload* w, int which);   // 0 x, 1 w, 2 bias, 3 residual, 4 y
+// device side (launch.cu)
+tt_status bind_device(tt_workload* w);                          // workspace + status word
+tt_status launch(tt_workload* w, const tt_tensors* t, void* stream);
+void release_device(tt_workload* w);
+}  // namespace tt

@@ -1,0 +1,254 @@
+"""Workload inventories shaped like the paper's models, and seeded inputs for them.
+
+The paper evaluates ImageNet CNNs and BERT (Section 5.1); a schedule depends only on
+the operator and the data sizes of a kernel (Section 2), never on weight values, so
+each model is represented by the list of its unique kernels (operator, sizes, use
+count) with synthetic tensors.  No dataset item or trained weight is involved.
+
+Kernel classes follow Table 1: conv2d_add (class A: 1x1 stride-2 downsample, no
+activation), conv2d_bias_relu (class E), dense_add (class D).  Residual-add variants
+(class F/G/K) share the shape of their class-E sibling and are counted with it.
+"""
+from __future__ import annotations
+
+import math
+from collections import OrderedDict
+
+import numpy as np
+
+from . import binding as B
+from . import inputs
+
+
+class Spec:
+    """One unique kernel of a model: operator, sizes, how often the model uses it, and a label."""
+
+    def __init__(self, op, shapes, use_count=1, name="", init="he"):
+        self.op, self.shapes, self.use_count, self.name, self.init = op, shapes, use_count, name, init
+
+    def workload(self) -> "B.Workload":
+        return B.Workload(self.op, self.shapes, self.name, self.use_count)
+
+
+def _conv(c, hw, k, r, stride, pad, act=B.TT_ACT_RELU, use=1, name=None, bias=True):
+    nm = name or f"conv{r}x{r}s{stride}_{c}x{hw}->{k}"
+    return Spec(B.TT_OP_CONV2D, B.conv2d_shapes(1, c, hw, hw, k, r, r, stride, pad, bias, act), use, nm)
+
+
+def _dw(c, hw, stride, r=3, act=B.TT_ACT_RELU6, use=1):
+    s = B.make_shapes(n=1, c=c, h=hw, w=hw, k=c, r=r, s=r, stride_h=stride, stride_w=stride, pad_h=r // 2, pad_w=r // 2,
+                      has_bias=1, act=act)
+    return Spec(B.TT_OP_DWCONV2D, s, use, f"dw{r}x{r}s{stride}_{c}x{hw}")
+
+
+def _dense(m, kk, nn, act=B.TT_ACT_NONE, use=1, init="he", name=None):
+    return Spec(B.TT_OP_DENSE, B.dense_shapes(m, nn, kk, True, act), use, name or f"dense_{m}x{kk}->{nn}", init)
+
+
+def _dedup(specs):
+    """Identical kernels (same workload ID: operator + sizes) are one kernel with a summed use count."""
+    seen = OrderedDict()
+    for sp in specs:
+        key = (sp.op, bytes(sp.shapes))
+        if key in seen:
+            seen[key].use_count += sp.use_count
+        else:
+            seen[key] = sp
+    return list(seen.values())
+
+
+def single_conv():
+    """One conv2d+bias+ReLU: C=16, 14x14, 32 filters 3x3, stride 1, pad 1."""
+    return [Spec(B.TT_OP_CONV2D, B.conv2d_shapes(1, 16, 14, 14, 32, 3, 3, 1, 1, True, B.TT_ACT_RELU), 1,
+                 "conv3x3s1_16x14->32", init="uniform")]
+
+
+def single_conv_pool():
+    """Four records sized for a C=32, 28x28, K=64 conv: tile M/N/K in {32,64}x{32,64}x{8,16}, 2-3 stages."""
+    origin = B.conv2d_shapes(1, 32, 28, 28, 64, 3, 3, 1, 1, True, B.TT_ACT_RELU)
+    recs = []
+    for tm, tn, tk, st in ((32, 32, 8, 2), (64, 32, 16, 2), (32, 64, 8, 3), (64, 64, 16, 3)):
+        r = B.make_record(B.TT_FAMILY_GEMM_TC, tile_m=tm, tile_n=tn, tile_k=tk, stages=st)
+        r.origin_op = B.TT_OP_CONV2D
+        r.origin = origin
+        recs.append(r)
+    return recs
+
+
+def resnet18():
+    """Table 1 (classes A, E+F merged per shape, D): 12 unique kernels."""
+    specs = [_conv(3, 224, 64, 7, 2, 3, name="stem7x7s2_3x224->64")]
+    ch, hw = 64, 56
+    for stage, k in enumerate((64, 128, 256, 512)):
+        if stage > 0:
+            specs.append(_conv(ch, hw, k, 3, 2, 1))                                     # first 3x3, strided
+            specs.append(_conv(ch, hw, k, 1, 2, 0, act=B.TT_ACT_NONE))                  # downsample (class A)
+            hw //= 2
+            specs.append(_conv(k, hw, k, 3, 1, 1, use=3))
+        else:
+            specs.append(_conv(ch, hw, k, 3, 1, 1, use=4))
+        ch = k
+    specs.append(_dense(1, 512, 1000))
+    return _dedup(specs)
+
+
+def resnet50():
+    """Bottleneck 1x1 / 3x3 / 1x1 kernels (stride on the 3x3), 1x1 downsamples, the 2048->1000 dense layer."""
+    specs = [_conv(3, 224, 64, 7, 2, 3, name="stem7x7s2_3x224->64")]
+    in_ch, hw = 64, 56
+    for stage, (mid, blocks) in enumerate(((64, 3), (128, 4), (256, 6), (512, 3))):
+        out_ch = mid * 4
+        stride = 1 if stage == 0 else 2
+        for b in range(blocks):
+            s = stride if b == 0 else 1
+            specs.append(_conv(in_ch, hw, mid, 1, 1, 0))                                # reduce
+            specs.append(_conv(mid, hw, mid, 3, s, 1))                                  # 3x3
+            if b == 0:
+                specs.append(_conv(in_ch, hw, out_ch, 1, s, 0, act=B.TT_ACT_NONE))      # downsample
+            hw2 = hw // s
+            specs.append(_conv(mid, hw2, out_ch, 1, 1, 0))                              # expand (+residual in-model)
+            in_ch, hw = out_ch, hw2
+    specs.append(_dense(1, 2048, 1000))
+    return _dedup(specs)
+
+
+def vgg16():
+    specs = []
+    ch, hw = 3, 224
+    for k, n in ((64, 2), (128, 2), (256, 3), (512, 3), (512, 3)):
+        for _ in range(n):
+            specs.append(_conv(ch, hw, k, 3, 1, 1))
+            ch = k
+        hw //= 2
+    specs += [_dense(1, 25088, 4096, B.TT_ACT_RELU), _dense(1, 4096, 4096, B.TT_ACT_RELU), _dense(1, 4096, 1000)]
+    return _dedup(specs)
+
+
+_MBV2 = ((1, 16, 1, 1), (6, 24, 2, 2), (6, 32, 3, 2), (6, 64, 4, 2), (6, 96, 3, 1), (6, 160, 3, 2), (6, 320, 1, 1))
+
+
+def mobilenet_v2():
+    specs = [_conv(3, 224, 32, 3, 2, 1, act=B.TT_ACT_RELU6, name="stem3x3s2_3x224->32")]
+    ch, hw = 32, 112
+    for t, c, n, s in _MBV2:
+        for i in range(n):
+            stride = s if i == 0 else 1
+            hid = ch * t
+            if t != 1:
+                specs.append(_conv(ch, hw, hid, 1, 1, 0, act=B.TT_ACT_RELU6))           # expand
+            specs.append(_dw(hid, hw, stride))
+            hw //= stride
+            specs.append(_conv(hid, hw, c, 1, 1, 0, act=B.TT_ACT_NONE))                 # project
+            ch = c
+    specs.append(_conv(320, 7, 1280, 1, 1, 0, act=B.TT_ACT_RELU6))
+    specs.append(_dense(1, 1280, 1000))
+    return _dedup(specs)
+
+
+def efficientnet_b0_like():
+    """1x1 expand/project, depthwise 3x3/5x5 and dense shapes of an EfficientNet-B0-shaped network (pool source)."""
+    cfg = ((1, 16, 1, 1, 3), (6, 24, 2, 2, 3), (6, 40, 2, 2, 5), (6, 80, 3, 2, 3), (6, 112, 3, 1, 5), (6, 192, 4, 2, 5),
+           (6, 320, 1, 1, 3))
+    specs = []
+    ch, hw = 32, 112
+    for t, c, n, s, r in cfg:
+        for i in range(n):
+            stride = s if i == 0 else 1
+            hid = ch * t
+            if t != 1:
+                specs.append(_conv(ch, hw, hid, 1, 1, 0, act=B.TT_ACT_RELU6))
+            specs.append(_dw(hid, hw, stride, r=r))
+            hw //= stride
+            specs.append(_conv(hid, hw, c, 1, 1, 0, act=B.TT_ACT_NONE))
+            ch = c
+    specs.append(_conv(320, 7, 1280, 1, 1, 0, act=B.TT_ACT_RELU6))
+    specs.append(_dense(1, 1280, 1000))
+    return _dedup(specs)
+
+
+def bert_base(seq=128, hidden=768, heads=12, ffn=3072, layers=12):
+    d = hidden // heads
+    return [
+        _dense(seq, hidden, hidden, use=4 * layers, init="bert", name=f"dense_{seq}x{hidden}->{hidden}"),
+        _dense(seq, hidden, ffn, act=B.TT_ACT_GELU_ERF, use=layers, init="bert", name=f"dense_gelu_{seq}x{hidden}->{ffn}"),
+        _dense(seq, ffn, hidden, use=layers, init="bert", name=f"dense_{seq}x{ffn}->{hidden}"),
+        Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(heads, seq, seq, d, True), layers, "bmm_qk_nt", "bert"),
+        Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(heads, seq, d, seq, False), layers, "bmm_pv_nn", "bert"),
+        Spec(B.TT_OP_SOFTMAX, B.softmax_shapes(heads, seq, seq, 1.0 / math.sqrt(d)), layers, "softmax", "bert"),
+    ]
+
+
+MODELS = {
+    "single_conv": single_conv, "resnet18": resnet18, "resnet50": resnet50, "vgg16": vgg16,
+    "mobilenet_v2": mobilenet_v2, "efficientnet_b0_like": efficientnet_b0_like, "bert_base": bert_base,
+}
+
+# target model -> models whose natively tuned records form its schedule pool
+POOL_SOURCES = {
+    "resnet18": ("resnet50",),
+    "resnet50": ("resnet18", "vgg16"),
+    "mobilenet_v2": ("resnet50", "efficientnet_b0_like"),
+    "bert_base": ("resnet50", "mobilenet_v2"),
+}
+
+
+def tensor_shapes(spec: Spec):
+    """Shapes of (x, w, bias, residual, y) for a spec; None where the tensor does not exist."""
+    s = spec.shapes
+    if spec.op in (B.TT_OP_CONV2D, B.TT_OP_DWCONV2D):
+        p = (s.h + 2 * s.pad_h - s.r) // s.stride_h + 1
+        q = (s.w + 2 * s.pad_w - s.s) // s.stride_w + 1
+        if spec.op == B.TT_OP_CONV2D:
+            wshape, k = (s.k, s.c, s.r, s.s), s.k
+        else:
+            wshape, k = (s.c, 1, s.r, s.s), s.c
+        y = (s.n, k, p, q)
+        return (s.n, s.c, s.h, s.w), wshape, (k,) if s.has_bias else None, y if s.has_residual else None, y
+    if spec.op == B.TT_OP_DENSE:
+        return (s.m, s.kk), (s.nn, s.kk), (s.nn,) if s.has_bias else None, None, (s.m, s.nn)
+    if spec.op == B.TT_OP_BATCH_MATMUL:
+        wshape = (s.batch, s.nn, s.kk) if s.trans_b else (s.batch, s.kk, s.nn)
+        return (s.batch, s.m, s.kk), wshape, None, None, (s.batch, s.m, s.nn)
+    return (s.batch, s.m, s.nn), None, None, None, (s.batch, s.m, s.nn)
+
+
+def make_inputs(spec: Spec, seed: int, index: int = 0):
+    """Seeded numpy tensors {x, w, bias, residual} for a spec.
+
+    init "uniform": everything U[-1,1].  "he": activations U[-1,1], weights N(0, 2/fan_in), bias U[-0.1,0.1].
+    "bert": activations N(0,1), weights N(0,0.02), bias U[-0.1,0.1]; the batch_matmul operands are N(0,1).
+    """
+    xs, ws, bs, rs, _ = tensor_shapes(spec)
+    tid = index * 8
+    out = {"x": None, "w": None, "bias": None, "residual": None}
+    if spec.init == "uniform":
+        out["x"] = inputs.uniform(xs, seed, tid)
+        if ws:
+            out["w"] = inputs.uniform(ws, seed, tid + 1)
+        if bs:
+            out["bias"] = inputs.uniform(bs, seed, tid + 2)
+    elif spec.init == "bert":
+        out["x"] = inputs.normal(xs, seed, tid)
+        if ws:
+            std = 1.0 if spec.op == B.TT_OP_BATCH_MATMUL else 0.02
+            out["w"] = inputs.normal(ws, seed, tid + 1, std=std)
+        if bs:
+            out["bias"] = inputs.uniform(bs, seed, tid + 2, -0.1, 0.1)
+    else:
+        out["x"] = inputs.uniform(xs, seed, tid)
+        if ws:
+            fan_in = int(np.prod(ws[1:]))
+            out["w"] = inputs.normal(ws, seed, tid + 1, std=math.sqrt(2.0 / fan_in))
+        if bs:
+            out["bias"] = inputs.uniform(bs, seed, tid + 2, -0.1, 0.1)
+    if rs:
+        out["residual"] = inputs.uniform(rs, seed, tid + 3)
+    return out
+
+
+def device_tensors(spec: Spec, arrays, device="cuda"):
+    """Copy the numpy inputs to torch tensors on `device`, allocate y; returns (dict of tensors, tt_tensors)."""
+    import torch
+    t = {k: (None if v is None else torch.from_numpy(v).to(device)) for k, v in arrays.items()}
+    t["y"] = torch.empty(tensor_shapes(spec)[4], dtype=torch.float32, device=device)
+    return t, B.tensors(t["x"], t["w"], t["bias"], t["residual"], t["y"])
