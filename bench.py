@@ -1,0 +1,364 @@
+#!/usr/bin/env python
+"""Benchmark of the transfer-tuning hot path on B200.
+
+One step = one pass over every kernel of the target model (use counts included), each run under the record the
+evaluator selected from a pool tuned on *other* models.  Before the timed region the pool is built (native grid
+tuning of the source models' kernels) and the evaluator runs every (kernel, record) pair; both are reported but
+not part of a step.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--model resnet18] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "TFLOP/s (model pass under transferred schedules)"
+UNIT = "TFLOP/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d.get("hbm_gbs", 6650.0), "bf16_tflops": d.get("bf16_tflops", 1590.0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz, self.stop_flag = index, [], set(), None, False
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                     nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                     nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                     nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
+            while not self.stop_flag:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                time.sleep(0.05)
+        except Exception as e:  # NVML missing: report that, do not fail the bench
+            self.reasons.add(f"nvml_unavailable:{type(e).__name__}")
+
+    def summary(self):
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def cpu_baseline_oracle(specs, arrays, budget_s, threads=0):
+    """Time the oracle as it stands on the host cores over a bounded sample of the model's unique kernels."""
+    from oracle import oracle as orc
+    orc.build()
+    flops, secs, used, names = 0.0, 0.0, 1, []
+    order = sorted(range(len(specs)), key=lambda i: -specs[i].workload().gemm_view().flops)
+    for i in order:
+        v = specs[i].workload().gemm_view()
+        est = v.flops / 2.0e9
+        if secs > 0 and secs + est > budget_s:
+            continue
+        t0 = time.perf_counter()
+        orc.reference(specs[i].op, specs[i].shapes, arrays[i], threads=threads)
+        secs += time.perf_counter() - t0
+        flops += v.flops
+        names.append(specs[i].name)
+        if secs > budget_s:
+            break
+    used = orc.max_threads() if threads == 0 else threads
+    return flops, secs, used, names
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, rank 0 only, on bounded samples of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_2201_05587_b200 import workloads as W
+    specs = W.MODELS[args.model]()
+    arrays = [W.make_inputs(sp, args.seed, i) for i, sp in enumerate(specs)]
+    total = args.steps + args.warmup
+    per_step = max(1.0, 150.0 / max(total, 1))
+    flops = secs = 0.0
+    used, names = 1, []
+    for step in range(total):
+        f, s, used, names = cpu_baseline_oracle(specs, arrays, per_step)
+        if step >= args.warmup:
+            flops += f
+            secs += s
+    value = flops / secs / 1e12
+    sample = f"{len(names)} of {len(specs)} unique kernels per step, once each: " + ",".join(names[:4]) + ("..." if len(names) > 4 else "")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": secs / max(args.steps, 1) * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"{args.model}-shaped inference, batch 1, fp32, pool from {','.join(W.POOL_SOURCES[args.model])}"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def tf32_peak(torch):
+    """cuBLAS TF32 matmul 8192^3, best of 10: the tensor-pipe denominator for this path (library call, not the product)."""
+    old = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = True
+    n = 8192
+    a = torch.randn(n, n, device="cuda")
+    b = torch.randn(n, n, device="cuda")
+    for _ in range(3):
+        a @ b
+    best = 1e9
+    for _ in range(10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        a @ b
+        e1.record()
+        e1.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    torch.backends.cuda.matmul.allow_tf32 = old
+    del a, b
+    return 2.0 * n ** 3 / (best * 1e-3) / 1e12
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--model", default="resnet18", choices=["resnet18", "resnet50", "mobilenet_v2", "bert_base"])
+    ap.add_argument("--seed", type=int, default=2)
+    ap.add_argument("--tune-level", type=int, default=0)
+    ap.add_argument("--top-k", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--report", default="", help="write the per-kernel table (JSON) to this file")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2201_05587_b200 import binding as B
+    from paper_2201_05587_b200 import replicas
+    from paper_2201_05587_b200 import workloads as W
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    rank, local_rank, world = replicas.init("nccl")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    B.lib()
+    peaks = measured_peaks()
+
+    # ---- target model, pool sources, tensors -------------------------------------------------------------
+    specs = W.MODELS[args.model]()
+    arrays = [W.make_inputs(sp, args.seed, i) for i, sp in enumerate(specs)]
+    wls = [sp.workload() for sp in specs]
+    dev_t, tts = zip(*[W.device_tensors(sp, a, dev) for sp, a in zip(specs, arrays)])
+
+    topts = B.tt_timing_opts()
+    topts.warmup_batches, topts.batches, topts.min_batch_us, topts.use_graph = 2, 5, 100, 1
+    t0 = time.perf_counter()
+    pool, n_tried = [], 0
+    for src in W.POOL_SOURCES[args.model]:
+        for j, sp in enumerate(W.MODELS[src]()):
+            a = W.make_inputs(sp, args.seed + 100, j)
+            swl = sp.workload()
+            _, stt = W.device_tensors(sp, a, dev)
+            best, tried = swl.grid_tune(stt, topts, level=args.tune_level, top_k=args.top_k)
+            n_tried += tried
+            pool += [r for r, _ in best]
+            swl.close()
+    pool_seconds = time.perf_counter() - t0
+
+    # ---- the evaluator: every kernel x every pool record (+ default) -------------------------------------
+    o = B.tt_tune_opts()
+    o.include_default = 1
+    o.timing.warmup_batches, o.timing.batches, o.timing.min_batch_us, o.timing.use_graph = 3, 10, 200, 1
+    res = B.transfer_tune(list(wls), list(tts), pool, o)
+    n_cols = len(pool) + 1
+    chosen = res["chosen"]
+    use = [sp.use_count for sp in specs]
+    flat = [v for row in res["times_us"] for v in row]
+    lat_best = B.model_latency(flat, len(wls), n_cols, chosen, use)
+    lat_default = B.model_latency(flat, len(wls), n_cols, [0] * len(wls), use)
+
+    views = [w.gemm_view() for w in wls]
+    flops_pass = sum(v.flops * u for v, u in zip(views, use))
+    bytes_pass = sum(v.bytes * u for v, u in zip(views, use))
+    launches_pass = 0
+    for w, u, c in zip(wls, use, chosen):
+        rec = w.default_schedule() if c == 0 else pool[c - 1]
+        launches_pass += w.check(rec)[1].launches * u
+
+    # ---- one model pass as a CUDA graph --------------------------------------------------------------------
+    def model_pass():
+        for w, t, u in zip(wls, tts, use):
+            for _ in range(u):
+                w.run(t)
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        model_pass()
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        model_pass()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)          # larger than the 126 MB L2
+
+    def timed_steps(n, body):
+        ms = 0.0
+        for _ in range(n):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            body()
+            e1.record()
+            e1.synchronize()
+            ms += e0.elapsed_time(e1)
+        return ms
+
+    timed_steps(args.warmup, graph.replay)
+    replicas.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ms_total = timed_steps(args.steps, graph.replay)
+    torch.cuda.synchronize()
+    replicas.barrier()
+    sampler.stop_flag = True
+    sampler.join(timeout=2)
+    for w in wls:
+        st = w.status()
+        if st != B.TT_OK:
+            raise SystemExit(f"device status {st} after the timed region")
+    value, slowest_s = replicas.aggregate(flops_pass * args.steps / 1e12, ms_total * 1e-3, dev)
+    ms_per_step = slowest_s * 1e3 / args.steps
+
+    # ---- end to end through the C ABI with host buffers -----------------------------------------------------
+    host_sets = []
+    for sp, a in zip(specs, arrays):
+        h = {k: (None if v is None else torch.from_numpy(v).pin_memory()) for k, v in a.items()}
+        h["y"] = torch.empty(W.tensor_shapes(sp)[4], dtype=torch.float32).pin_memory()
+        host_sets.append((h, B.tensors(h["x"], h["w"], h["bias"], h["residual"], h["y"])))
+    bytes_up = bytes_down = 0
+
+    def e2e_pass():
+        nonlocal bytes_up, bytes_down
+        bytes_up = bytes_down = 0
+        for w, (h, ht), u in zip(wls, host_sets, use):
+            for _ in range(u):
+                up, down = w.run_host(ht)
+                bytes_up += up
+                bytes_down += down
+
+    timed_steps(3, e2e_pass)
+    e2e_steps = max(3, min(args.steps, 10))
+    replicas.barrier()
+    e2e_ms = timed_steps(e2e_steps, e2e_pass)
+    replicas.barrier()
+    e2e_value, _ = replicas.aggregate(flops_pass * e2e_steps / 1e12, e2e_ms * 1e-3, dev)
+
+    # ---- roofline of the dominant kernel family (live, standalone, cold L2) ------------------------------
+    # Rotating tensor sets whose footprint exceeds twice the L2 make every launch miss; times are CUDA events
+    # around batches of launches on the launching stream.
+    rows = []
+    cold = B.tt_timing_opts()
+    cold.warmup_batches, cold.batches, cold.min_batch_us, cold.use_graph = 2, 5, 200, 1
+    gemm_flops = gemm_bytes = gemm_cold_us = gemm_launches = 0.0
+    tf32 = tf32_peak(torch) if rank == 0 else 0.0
+    for i, (sp, w, v, a) in enumerate(zip(specs, wls, views, arrays)):
+        n_sets = int(min(1024, max(2, (2 * 126e6) // max(v.bytes, 1) + 1)))
+        sets, keep = [], []
+        for _ in range(n_sets):
+            t, tt = W.device_tensors(sp, a, dev)
+            keep.append(t)
+            sets.append(tt)
+        tm = w.time(sets, cold)
+        warm = res["best_us"][i]
+        rec = w.default_schedule() if chosen[i] == 0 else pool[chosen[i] - 1]
+        info = w.check(rec)[1]
+        rows.append({"kernel": sp.name, "use": sp.use_count, "mflop": v.flops / 1e6, "mbytes": v.bytes / 1e6,
+                     "record": info.legal.short(), "grid": [info.grid_x, info.grid_y, info.grid_z],
+                     "warm_us": warm, "default_us": res["times_us"][i][0], "cold_us": tm.median_us,
+                     "tflops_warm": v.flops / warm / 1e6, "gbs_cold": v.bytes / tm.median_us / 1e3,
+                     "valid_records": sum(1 for s in res["status"][i] if s == 0), "origin": chosen[i]})
+        if w.family() == B.TT_FAMILY_GEMM_TC:
+            gemm_flops += v.flops * sp.use_count
+            gemm_bytes += v.bytes * sp.use_count
+            gemm_cold_us += tm.median_us * sp.use_count
+            gemm_launches += info.launches * sp.use_count
+        del keep, sets
+    ai = gemm_flops / max(gemm_bytes, 1)
+    ridge = tf32 * 1e12 / (peaks["hbm_gbs"] * 1e9) if tf32 else 107.0
+    if ai < ridge:
+        roof = {"bound": "hbm", "achieved": gemm_bytes / gemm_cold_us / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"bound": "tensor", "achieved": gemm_flops / gemm_cold_us / 1e6, "peak": tf32, "unit": "TFLOP/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = None
+    roof.update({"kernel": "tt_gemm_tc_kernel", "peak_source": peaks["source"] + (" hbm copy" if roof["bound"] == "hbm" else " cuBLAS TF32 8192^3, this run"),
+                 "launches_per_pass": gemm_launches, "avg_launch_us": gemm_cold_us / max(gemm_launches, 1),
+                 "algorithmic_mbytes_per_pass": gemm_bytes / 1e6, "algorithmic_gflop_per_pass": gemm_flops / 1e9,
+                 "tf32_peak_tflops_this_run": tf32, "tensor_frac": (gemm_flops / gemm_cold_us / 1e6) / tf32 if tf32 else None,
+                 "l2": "cold (rotating tensor sets > 2x L2)"})
+
+    line = None
+    if rank == 0:
+        cpu = None
+        if not args.no_cpu_baseline:
+            f, s, used, names = cpu_baseline_oracle(specs, arrays, 20.0)
+            cpu = {"value": f / s / 1e12, "unit": UNIT, "cores": used, "kind": "oracle",
+                   "sample": f"{len(names)} of {len(specs)} unique kernels once each ({f / 1e9:.2f} GFLOP in {s:.1f} s)"}
+        clocks = sampler.summary()
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "tf32",
+            "data": "synthetic",
+            "config": {"workload": f"{args.model}-shaped inference, batch 1, fp32 NCHW, {len(specs)} unique kernels / "
+                                   f"{sum(use)} per pass, pool from {','.join(W.POOL_SOURCES[args.model])}-shaped kernels",
+                       "l2": "flushed between steps (256 MB write)", "replay": "one CUDA graph per model pass",
+                       "multi_gpu": "independent replicas"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bytes_up, "d2h_bytes_per_step": bytes_down,
+                    "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+            "gpu_launches": int(launches_pass * args.steps),
+            "clocks": clocks,
+            "roofline": roof,
+            "cpu_baseline": cpu,
+            "model_latency_us": {"transferred_sum_standalone": lat_best, "default_sum_standalone": lat_default,
+                                 "speedup_over_default": lat_default / lat_best if lat_best else None,
+                                 "measured_pass_cold_l2": ms_per_step * 1e3},
+            "search": {"pairs_timed": res["pairs_timed"], "pairs_invalid": res["pairs_invalid"],
+                       "seconds": res["search_seconds"], "pool_records": len(pool), "pool_build_seconds": pool_seconds,
+                       "pool_candidates_tried": n_tried},
+        }
+        if args.report:
+            with open(args.report, "w") as fh:
+                json.dump({"line": line, "kernels": rows}, fh, indent=1)
+        print(json.dumps(line))
+    replicas.finalize()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -151,6 +151,28 @@ def softmax(s, scale=1.0, threads=0):
     return p
 
 
+# operator numbering of the C ABI under test (tt_op in include/tt.h), restated here: the oracle imports nothing
+OP_CONV2D, OP_DWCONV2D, OP_DENSE, OP_BATCH_MATMUL, OP_SOFTMAX = range(5)
+
+
+def reference(op: int, s, a, mode=MODE_EXACT, threads=0):
+    """Reference output of one kernel: `s` carries the size fields of the ABI's shape struct (any object with
+    those attributes), `a` maps 'x', 'w', 'bias', 'residual' to numpy arrays or None."""
+    if op == OP_CONV2D:
+        return conv2d(a["x"], a["w"], a.get("bias"), (s.stride_h, s.stride_w), (s.pad_h, s.pad_w), s.act,
+                      a.get("residual"), mode=mode, threads=threads)
+    if op == OP_DWCONV2D:
+        return dwconv2d(a["x"], a["w"], a.get("bias"), (s.stride_h, s.stride_w), (s.pad_h, s.pad_w), s.act,
+                        threads=threads)
+    if op == OP_DENSE:
+        return dense(a["x"], a["w"], a.get("bias"), s.act, mode=mode, threads=threads)
+    if op == OP_BATCH_MATMUL:
+        return batch_matmul(a["x"], a["w"], None, bool(s.trans_b), s.act, mode=mode, threads=threads)
+    if op == OP_SOFTMAX:
+        return softmax(a["x"], s.scale, threads=threads)
+    raise ValueError(f"unknown operator {op}")
+
+
 def rel_l2(y, ref) -> float:
     """||y - ref||_2 / ||ref||_2 in double; absolute norm of y when ref is all zero."""
     y = np.asarray(y, dtype=np.float64).ravel()

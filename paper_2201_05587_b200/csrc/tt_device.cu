@@ -102,8 +102,7 @@ static tt_status tensor_maps_for(tt_workload* w, const void* a_ptr, const void* 
     TmapPair e;
     std::memset(&e, 0, sizeof e);
     e.a_ptr = a_ptr; e.b_ptr = b_ptr;
-    // An operand that is gathered still needs a well-formed map in the kernel's parameter slot: encode the
-    // other operand's (or a self-describing dummy over the A tensor) so no parameter is uninitialised.
+    // A gathered operand keeps an all-zero map in its parameter slot; the kernel never issues a TMA load on it.
     tt_status st = TT_OK;
     if (g.a_mode == OPM_TMA)
         st = encode_operand(e.a, static_cast<const float*>(a_ptr), g.K, g.M, g.batch, g.a_rs, g.a_bs, g.a_tma_batched != 0,
@@ -113,7 +112,7 @@ static tt_status tensor_maps_for(tt_workload* w, const void* a_ptr, const void* 
         st = encode_operand(e.b, static_cast<const float*>(b_ptr), g.K, g.N, g.batch, g.b_rs, g.b_bs, g.b_tma_batched != 0,
                             g.atom_k, g.tile_n);
     if (st != TT_OK) return st;
-    if (w->tmaps.size() >= 256) w->tmaps.clear();
+    if (w->tmaps.size() >= 4096) w->tmaps.clear();
     w->tmaps.push_back(e);
     *out = &w->tmaps.back();
     return TT_OK;

@@ -1,0 +1,280 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded inputs."""
+import ctypes
+import itertools
+
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_2201_05587_b200 import binding as B
+from paper_2201_05587_b200 import workloads as W
+import util
+
+pytestmark = pytest.mark.gpu
+
+
+def tc(**kw):
+    return B.make_record(B.TT_FAMILY_GEMM_TC, **kw)
+
+
+def run_spec(spec, rec, arrays, ref=None, tol=None, mode=B.TT_MODE_LEGALISE):
+    import torch
+    wl = spec.workload()
+    wl.apply(rec, mode=mode)
+    t, tt = W.device_tensors(spec, arrays)
+    t["y"].fill_(float("nan"))
+    wl.run(tt)
+    assert wl.status() == B.TT_OK
+    y = t["y"].cpu().numpy()
+    wl.close()
+    assert not np.isnan(y).any(), "kernel left outputs unwritten"
+    if ref is not None:
+        err = util.rel_l2(y, ref)
+        assert err <= (tol or util.tolerance(spec.op)), f"{spec.name} {rec.short()} rel-L2 {err:.3e}"
+    return y
+
+
+GEMM_RECORDS = [
+    tc(tile_n=128, tile_k=32, stages=4, mma_m_axis=1),
+    tc(tile_n=64, tile_k=16, stages=3, mma_m_axis=1),
+    tc(tile_n=16, tile_k=8, stages=2, mma_m_axis=1),
+    tc(tile_n=256, tile_k=64, stages=2, mma_m_axis=1),
+    tc(tile_n=48, tile_k=32, stages=1, raster=1, mma_m_axis=1),
+    tc(tile_n=96, tile_k=32, stages=6, split_k=3, mma_m_axis=1),
+    tc(tile_n=128, tile_k=64, stages=3, split_k=2, mma_m_axis=2),
+    tc(tile_n=32, tile_k=128, stages=2, split_k=1, raster=1, mma_m_axis=2),
+    tc(tile_n=192, tile_k=16, stages=4, split_k=5, mma_m_axis=2),
+]
+
+
+def check_all_records(spec, seed, records=GEMM_RECORDS):
+    a = W.make_inputs(spec, seed)
+    ref = util.oracle_ref(spec, a)
+    outs = [run_spec(spec, r, a, ref) for r in records]
+    # a schedule changes speed, never semantics: every valid record gives the same output (up to summation order)
+    for y in outs[1:]:
+        assert util.rel_l2(y, outs[0]) <= 1e-6
+    return outs
+
+
+@pytest.mark.parametrize("spec", [
+    W._dense(128, 768, 768, name="bert_dense"),
+    W._dense(200, 300, 100, act=B.TT_ACT_RELU, name="ragged_dense"),        # ragged M, N, K tails; K % 8 != 0
+    W._dense(129, 147, 257, act=B.TT_ACT_GELU_ERF, name="odd_dense_gatherK"),   # K % 4 != 0: gathered operands
+    W._dense(1, 512, 1000, name="head_m1"),
+    W._dense(1, 1, 1, name="one_by_one"),
+    W._dense(3, 5, 7, name="tiny"),
+], ids=lambda s: s.name)
+def test_dense_parity_all_records(spec):
+    check_all_records(spec, seed=31)
+
+
+@pytest.mark.parametrize("spec", [
+    W.single_conv()[0],
+    W._conv(3, 32, 64, 7, 2, 3, name="stem_like_7x7s2"),                    # reduction 147: gathered filters
+    W._conv(24, 15, 40, 3, 2, 1, name="conv3x3s2_odd"),
+    W._conv(32, 14, 64, 1, 1, 0, act=B.TT_ACT_RELU6, name="conv1x1_relu6"),
+    W._conv(64, 14, 128, 1, 2, 0, act=B.TT_ACT_NONE, name="downsample_1x1s2"),
+    W._conv(20, 7, 24, 3, 1, 1, name="conv3x3_7x7"),
+    W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(2, 8, 9, 11, 12, 3, 3, 1, 1, True, B.TT_ACT_RELU, True), 1, "batch2_residual", "uniform"),
+    W.Spec(B.TT_OP_CONV2D, B.make_shapes(n=1, c=6, h=10, w=12, k=9, r=3, s=2, stride_h=2, stride_w=1, pad_h=0, pad_w=1,
+                                         has_bias=0, act=B.TT_ACT_NONE), 1, "asym_nobias", "uniform"),
+], ids=lambda s: s.name)
+def test_conv_parity_all_records(spec):
+    check_all_records(spec, seed=32)
+
+
+@pytest.mark.parametrize("spec", [
+    W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(12, 128, 128, 64, True), 1, "qk_nt", "bert"),
+    W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(12, 128, 64, 128, False), 1, "pv_nn", "bert"),
+    W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(3, 50, 70, 36, False), 1, "ragged_nn", "bert"),
+    W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(2, 33, 17, 10, True), 1, "ragged_nt_k10", "bert"),
+], ids=lambda s: s.name)
+def test_batch_matmul_parity_all_records(spec):
+    check_all_records(spec, seed=33)
+
+
+def test_config1_every_pool_record_and_selection():
+    spec = W.single_conv()[0]
+    a = W.make_inputs(spec, 1)
+    ref = util.oracle_ref(spec, a)
+    pool = W.single_conv_pool()
+    outs = [run_spec(spec, r, a, ref) for r in pool]
+    for y in outs[1:]:
+        assert util.rel_l2(y, outs[0]) <= 1e-6
+    wl = spec.workload()
+    t, tt = W.device_tensors(spec, a)
+    res = B.transfer_tune([wl], [tt], pool)
+    assert res["pairs_timed"] == 5 and res["pairs_invalid"] == 0
+    times = res["times_us"][0]
+    assert all(v > 0 for v in times)
+    # selection is the oracle's argmin on the measured table
+    assert res["chosen"] == orc.select(times, 1, 5) == B.select(times, 1, 5)
+    assert res["best_us"][0] == pytest.approx(min(times))
+    # the chosen record is left applied: running now reproduces the oracle
+    t["y"].zero_()
+    wl.run(tt)
+    assert wl.status() == B.TT_OK
+    assert util.rel_l2(t["y"].cpu().numpy(), ref) <= util.TOL_TF32
+
+
+def test_evaluator_records_invalid_pairs_and_falls_back_to_default():
+    conv = W._conv(16, 12, 24, 3, 1, 1)
+    dw = W._dw(16, 12, 1)
+    a1, a2 = W.make_inputs(conv, 7), W.make_inputs(dw, 7, 1)
+    w1, w2 = conv.workload(), dw.workload()
+    t1, tt1 = W.device_tensors(conv, a1)
+    t2, tt2 = W.device_tensors(dw, a2)
+    fat = tc(tile_n=256, tile_k=128, stages=8, mma_m_axis=1)           # legal fields, too much shared memory... on big shapes
+    nonsense = tc(tile_n=64, tile_k=32, stages=0)
+    pool = [tc(tile_n=32, tile_k=16, stages=2), nonsense, B.make_record(B.TT_FAMILY_ROW_SIMT)]
+    res = B.transfer_tune([w1, w2], [tt1, tt2], pool)
+    st = res["status"]
+    assert st[0][0] == B.TT_OK and st[0][1] == B.TT_OK
+    assert st[0][2] == B.TT_ERR_INVALID_SCHEDULE and st[0][3] == B.TT_ERR_CLASS_MISMATCH
+    assert res["times_us"][0][2] == -1.0 and res["times_us"][0][3] == -1.0
+    # the depthwise kernel has no compatible record in this pool: it keeps its default schedule
+    assert st[1][1] == st[1][2] == st[1][3] == B.TT_ERR_CLASS_MISMATCH
+    assert res["chosen"][1] == 0 and res["best_us"][1] > 0
+    assert res["pairs_invalid"] == 5 and res["pairs_timed"] == 3
+    w2.run(tt2)
+    assert util.rel_l2(t2["y"].cpu().numpy(), util.oracle_ref(dw, a2)) <= util.TOL_FP32
+    del fat
+
+
+@pytest.mark.parametrize("spec", [s for s in W.mobilenet_v2() if s.op == B.TT_OP_DWCONV2D][::3] + [
+    W._dw(5, 9, 2), W._dw(40, 28, 1, r=5), W._dw(1, 1, 1),
+    W.Spec(B.TT_OP_DWCONV2D, B.make_shapes(n=3, c=7, h=13, w=10, r=3, s=3, stride_h=1, stride_w=2, pad_h=1, pad_w=0,
+                                           has_bias=0, act=B.TT_ACT_RELU), 1, "dw_batch3_asym", "uniform"),
+], ids=lambda s: s.name)
+def test_depthwise_parity_records(spec):
+    a = W.make_inputs(spec, 34)
+    ref = util.oracle_ref(spec, a)
+    recs = [spec.workload().default_schedule()]
+    for tcn, by, bx, it, vw, th in ((4, 8, 32, 4, 4, 256), (16, 4, 16, 2, 2, 128), (1, 16, 64, 8, 4, 64), (32, 7, 7, 1, 1, 512),
+                                    (3, 5, 24, 8, 1, 96)):
+        recs.append(B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=tcn, block_y=by, block_x=bx, items_per_thread=it,
+                                  vec_width=vw, threads=th))
+    outs = [run_spec(spec, r, a, ref) for r in recs]
+    for y in outs[1:]:
+        np.testing.assert_array_equal(y, outs[0])       # same fp32 operations in the same order: bit-identical
+
+
+@pytest.mark.parametrize("shape", [(12, 128, 128), (1, 1, 1), (3, 5, 37), (2, 9, 1000), (1, 300, 6)])
+def test_softmax_parity_records(shape):
+    spec = W.Spec(B.TT_OP_SOFTMAX, B.softmax_shapes(*shape, scale=0.125), 1, "softmax", "bert")
+    a = W.make_inputs(spec, 35)
+    a["x"] = a["x"] * 6.0
+    ref = util.oracle_ref(spec, a)
+    for bx, by, vw in ((32, 4, 1), (8, 16, 4), (1, 32, 1), (16, 3, 2), (4, 64, 4)):
+        run_spec(spec, B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=bx, block_y=by, vec_width=vw), a, ref)
+
+
+def test_split_k_is_bit_reproducible():
+    spec = W._dense(128, 3072, 768)
+    a = W.make_inputs(spec, 36)
+    r = tc(tile_n=128, tile_k=32, stages=4, split_k=8, mma_m_axis=1)
+    y1 = run_spec(spec, r, a)
+    y2 = run_spec(spec, r, a)
+    np.testing.assert_array_equal(y1, y2)
+
+
+def test_run_requires_apply_and_pointers():
+    spec = W._dense(8, 16, 8)
+    wl = spec.workload()
+    a = W.make_inputs(spec, 37)
+    t, tt = W.device_tensors(spec, a)
+    assert B.lib().tt_run(wl.handle, ctypes.byref(tt), None) == B.TT_ERR_NOT_APPLIED
+    wl.apply(wl.default_schedule())
+    bad = B.tensors(t["x"], t["w"], None, None, t["y"])
+    assert B.lib().tt_run(wl.handle, ctypes.byref(bad), None) == B.TT_ERR_INVALID_ARG
+    # an invalid record leaves the applied one in force
+    st, _ = wl.try_apply(tc(stages=0))
+    assert st == B.TT_ERR_INVALID_SCHEDULE
+    wl.run(tt)
+    assert util.rel_l2(t["y"].cpu().numpy(), util.oracle_ref(spec, a)) <= util.TOL_TF32
+
+
+def test_run_host_matches_oracle():
+    import torch
+    spec = W._conv(16, 14, 32, 3, 1, 1)
+    a = W.make_inputs(spec, 38)
+    wl = spec.workload()
+    wl.apply(tc(tile_n=64, tile_k=32, stages=3))
+    host = {k: (None if v is None else torch.from_numpy(v).pin_memory()) for k, v in a.items()}
+    y = torch.empty(W.tensor_shapes(spec)[4], dtype=torch.float32).pin_memory()
+    up, down = wl.run_host(B.tensors(host["x"], host["w"], host["bias"], None, y))
+    assert up == 4 * (a["x"].size + a["w"].size + a["bias"].size) and down == 4 * y.numel()
+    assert util.rel_l2(y.numpy(), util.oracle_ref(spec, a)) <= util.TOL_TF32
+
+
+def test_timing_and_grid_tuner_smoke():
+    spec = W._conv(32, 14, 64, 3, 1, 1)
+    a = W.make_inputs(spec, 39)
+    wl = spec.workload()
+    t, tt = W.device_tensors(spec, a)
+    wl.apply(wl.default_schedule())
+    o = B.tt_timing_opts()
+    o.batches, o.warmup_batches, o.min_batch_us = 4, 1, 50
+    tm = wl.time(tt, o)
+    assert 0 < tm.min_us <= tm.median_us <= tm.max_us and tm.batches == 4
+    o.use_graph = 1
+    tg = wl.time([tt, tt], o)
+    assert tg.median_us > 0
+    best, tried = wl.grid_tune(tt, o, level=0, top_k=3)
+    assert tried > 10 and 1 <= len(best) <= 3
+    assert best[0][1] <= best[-1][1]
+    assert best[0][0].origin_op == B.TT_OP_CONV2D and best[0][0].origin.c == 32
+    wl.run(tt)                                     # the best record is left applied
+    assert util.rel_l2(t["y"].cpu().numpy(), util.oracle_ref(spec, a)) <= util.TOL_TF32
+
+
+def _model_parity(model, seed, recs):
+    specs = W.MODELS[model]()
+    for i, spec in enumerate(specs):
+        a = W.make_inputs(spec, seed, i)
+        ref = util.oracle_ref(spec, a)
+        rr = [spec.workload().default_schedule()] + (recs if spec.op in (B.TT_OP_CONV2D, B.TT_OP_DENSE, B.TT_OP_BATCH_MATMUL) else [])
+        for r in rr:
+            run_spec(spec, r, a, ref)
+
+
+def test_resnet18_full_size_every_kernel():
+    _model_parity("resnet18", 2, [tc(tile_n=64, tile_k=64, stages=3, split_k=4, mma_m_axis=2),
+                                  tc(tile_n=256, tile_k=32, stages=3, split_k=1, raster=1, mma_m_axis=1)])
+
+
+def test_mobilenet_v2_full_size_every_kernel():
+    _model_parity("mobilenet_v2", 4, [tc(tile_n=32, tile_k=16, stages=4, split_k=2, mma_m_axis=2)])
+
+
+def test_bert_base_full_size_every_kernel():
+    _model_parity("bert_base", 5, [tc(tile_n=64, tile_k=32, stages=4, split_k=3, mma_m_axis=1)])
+
+
+def test_resnet50_full_size_sampled_filters():
+    """Full-size kernels, outputs sampled by filter: a convolution restricted to some filters is exactly those
+    output channels, so the oracle computes only them."""
+    import torch
+    specs = W.resnet50()
+    rec = tc(tile_n=128, tile_k=32, stages=4, split_k=2, mma_m_axis=1)
+    for i, spec in enumerate(specs):
+        a = W.make_inputs(spec, 3, i)
+        y = run_spec(spec, rec, a)
+        if spec.op == B.TT_OP_CONV2D:
+            ks = sorted({0, spec.shapes.k // 3, spec.shapes.k - 1})
+            sub = orc.conv2d(a["x"], a["w"][ks], a["bias"][ks], (spec.shapes.stride_h,) * 2, (spec.shapes.pad_h,) * 2,
+                             spec.shapes.act)
+            assert util.rel_l2(y[:, ks], sub) <= util.TOL_TF32, spec.name
+        else:
+            assert util.rel_l2(y, util.oracle_ref(spec, a)) <= util.TOL_TF32
+
+
+def test_largest_dense_sampled_outputs():
+    """The largest kernel of the pool sources (25088 -> 4096, 411 MB of weights), checked on sampled out-features."""
+    spec = W._dense(1, 25088, 4096, B.TT_ACT_RELU)
+    a = W.make_inputs(spec, 40)
+    y = run_spec(spec, tc(tile_n=16, tile_k=64, stages=4, split_k=16), a)
+    rows = [0, 1, 127, 128, 2047, 4000, 4095]
+    sub = orc.dense(a["x"], a["w"][rows], a["bias"][rows], B.TT_ACT_RELU)
+    assert util.rel_l2(y[:, rows], sub) <= util.TOL_TF32

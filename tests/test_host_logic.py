@@ -1,0 +1,212 @@
+"""Host logic of the library (no GPU): ABI exports, workloads, classes, legaliser/validator, selector."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from oracle import oracle as orc
+from paper_2201_05587_b200 import binding as B
+from paper_2201_05587_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+GOLDEN = os.path.join(ROOT, "tests", "golden")
+
+
+def test_library_exports_every_declared_symbol():
+    text = open(os.path.join(ROOT, "include", "tt.h")).read()
+    declared = set(re.findall(r"\b(tt_[a-z_]+)\s*\(", text))
+    declared -= {"tt_op", "tt_act"}
+    assert declared, "no declarations found"
+    lib = B.lib()
+    for name in sorted(declared):
+        assert hasattr(lib, name), f"{name} declared in tt.h but not exported"
+        assert name in B.EXPORTS, f"{name} has no binding"
+    assert set(B.EXPORTS) <= declared
+
+
+def test_struct_sizes_match_header_layout():
+    assert ctypes.sizeof(B.tt_shapes) == 20 * 4
+    assert ctypes.sizeof(B.tt_schedule_record) == 3 * 4 + 80 + 16 * 4
+    assert B.status_string(B.TT_ERR_INVALID_SCHEDULE) != B.status_string(B.TT_OK)
+
+
+def test_split_check_matches_paper_examples_and_oracle():
+    with open(os.path.join(GOLDEN, "split_validity.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            extent, form, factors, valid = line.split()
+            extent, valid = int(extent), bool(int(valid))
+            fs = [int(v) for v in factors.split(",")]
+            if form == "fixed":
+                assert B.split_check(extent, fs) == valid == orc.split_covers(extent, fs), line
+            elif form == "reform":
+                assert B.split_check(extent, fs, reformulate=True) == valid, line
+    for n in (1, 7, 8, 24, 49, 196, 1000, 4096):
+        for f in (1, 2, 3, 8, 16):
+            assert B.split_check(n, [f], True) == orc.split_reformulated_valid(n, f)
+            assert B.split_check(n, [n // f if n % f == 0 else 1, f]) == orc.split_covers(n, [n // f if n % f == 0 else 1, f])
+
+
+def test_select_matches_oracle_on_hand_tables():
+    t = [5.0, 3.0, -1.0, 3.0, -1.0, -1.0, -1.0, -1.0, 2.0, -1.0, 1.5, 9.0, float("nan"), 4.0, 4.0, -1.0]
+    assert B.select(t, 4, 4) == orc.select(t, 4, 4) == [1, -1, 2, 1]
+    lat = B.model_latency(t, 4, 4, [1, -1, 2, 1], [2, 5, 3, 1])
+    assert lat == pytest.approx(orc.model_latency([2, 5, 3, 1], [0 if v != v else v for v in t], [1, -1, 2, 1], 4))
+    # deterministic: same table, same answer
+    assert all(B.select(t, 4, 4) == [1, -1, 2, 1] for _ in range(5))
+
+
+def test_resnet18_inventory_matches_table1():
+    rows = []
+    with open(os.path.join(GOLDEN, "resnet18_table1.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                i, cls, ic, ihw, oc, ohw, use = line.split()
+                rows.append((cls, int(ic), int(ihw), int(oc), int(ohw), int(use)))
+    specs = W.resnet18()
+    assert len(specs) == 12
+    # merge the table's E and F rows per shape (residual variants share the shape), keep A and D
+    want = {}
+    for cls, ic, ihw, oc, ohw, use in rows:
+        kind = "A" if cls == "A" else ("D" if cls == "D" else "E")
+        want[(kind, ic, ihw, oc, ohw)] = want.get((kind, ic, ihw, oc, ohw), 0) + use
+    got = {}
+    for sp in specs:
+        s = sp.shapes
+        if sp.op == B.TT_OP_DENSE:
+            got[("D", s.kk, 1, s.nn, 1)] = sp.use_count
+        else:
+            p = (s.h + 2 * s.pad_h - s.r) // s.stride_h + 1
+            kind = "A" if (s.r == 1 and s.act == B.TT_ACT_NONE) else "E"
+            got[(kind, s.c, s.h, s.k, p)] = sp.use_count
+    assert got == want
+    assert sum(sp.use_count for sp in specs) == 21          # 20 convolutions + 1 dense
+
+
+def test_unique_kernel_counts_of_table2():
+    """Table 2: ResNet50 A4 E16 G4 D1; VGG-16 E9 (+ 3 dense shapes); MobileNetV2 A7+K5 J8 L10 D1; BERT Q3 R2."""
+    r50 = W.resnet50()
+    convs = [s for s in r50 if s.op == B.TT_OP_CONV2D]
+    down = [s for s in convs if s.shapes.act == B.TT_ACT_NONE]
+    assert len(down) == 4 and len(convs) - len(down) == 20 and len(r50) == 25    # 16 (E) + 4 (G) share code here
+    vgg = W.vgg16()
+    assert len([s for s in vgg if s.op == B.TT_OP_CONV2D]) == 9 and len(vgg) == 12
+    mb = W.mobilenet_v2()
+    dw = [s for s in mb if s.op == B.TT_OP_DWCONV2D]
+    proj = [s for s in mb if s.op == B.TT_OP_CONV2D and s.shapes.act == B.TT_ACT_NONE]
+    relu6 = [s for s in mb if s.op == B.TT_OP_CONV2D and s.shapes.act == B.TT_ACT_RELU6]
+    assert (len(dw), len(proj), len(relu6)) == (10, 12, 8)
+    bert = W.bert_base()
+    assert len([s for s in bert if s.op == B.TT_OP_DENSE]) == 3
+    assert len([s for s in bert if s.op == B.TT_OP_BATCH_MATMUL]) == 2
+
+
+def test_workload_key_and_class():
+    a = W._conv(64, 56, 64, 3, 1, 1).workload()
+    b = W._conv(64, 56, 64, 3, 1, 1).workload()
+    c = W._conv(128, 28, 128, 3, 1, 1).workload()
+    d = W._conv(64, 56, 128, 1, 2, 0, act=B.TT_ACT_NONE).workload()
+    e = W._dense(1, 512, 1000).workload()
+    assert a.key() == b.key() != c.key()
+    assert a.kernel_class() == c.kernel_class()          # same operators, other sizes: same class
+    assert a.kernel_class() != d.kernel_class()          # conv2d_add is another class than conv2d_bias_relu
+    assert a.kernel_class() != e.kernel_class()
+    assert a.family() == e.family() == B.TT_FAMILY_GEMM_TC
+    v = a.gemm_view()
+    assert (v.batch, v.gm, v.gn, v.gk) == (1, 64, 3136, 576)
+    assert v.flops == pytest.approx(2 * 64 * 3136 * 576)
+
+
+def test_workload_create_rejects_bad_shapes():
+    for bad in (B.conv2d_shapes(1, 0, 8, 8, 4, 3, 3), B.conv2d_shapes(1, 4, 2, 2, 4, 5, 5), B.conv2d_shapes(1, 4, 8, 8, 4, 3, 3, 0)):
+        h = ctypes.c_void_p()
+        assert B.lib().tt_workload_create(B.TT_OP_CONV2D, ctypes.byref(bad), ctypes.byref(h)) == B.TT_ERR_INVALID_ARG
+    h = ctypes.c_void_p()
+    assert B.lib().tt_workload_create(99, ctypes.byref(B.dense_shapes(1, 2, 3)), ctypes.byref(h)) == B.TT_ERR_INVALID_ARG
+
+
+def test_cross_family_and_cross_class_records_are_invalid():
+    conv = W._conv(64, 56, 64, 3, 1, 1).workload()
+    dw = W._dw(32, 112, 1).workload()
+    dense = W._dense(1, 512, 1000).workload()
+    st, _ = dw.check(conv.default_schedule())
+    assert st == B.TT_ERR_CLASS_MISMATCH
+    st, _ = conv.check(dw.default_schedule())
+    assert st == B.TT_ERR_CLASS_MISMATCH
+    # the paper's rule: a conv schedule on a dense kernel is always invalid
+    rec = conv.default_schedule()
+    st, _ = dense.check(rec, strict_class=True)
+    assert st == B.TT_ERR_CLASS_MISMATCH
+    # with family matching (the stated extension) the same record applies
+    st, _ = dense.check(rec, strict_class=False)
+    assert st == B.TT_OK
+    # same class, other sizes: valid in both
+    other = W._conv(256, 14, 256, 3, 1, 1).workload()
+    assert other.check(rec, strict_class=True)[0] == B.TT_OK
+
+
+def test_legaliser_clamps_and_strict_mode_rejects():
+    wl = W.single_conv()[0].workload()         # GEMM view 32 x 196 x 144
+    for rec in W.single_conv_pool():
+        st, info = wl.check(rec)
+        assert st == B.TT_OK
+        L = info.legal
+        assert L.tile_m == 128 and L.tile_n % 16 == 0 and L.tile_k in (8, 16)
+        assert info.changed & B.TT_CHG_TILE_M
+    big = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=256, tile_k=64, stages=2, split_k=64, mma_m_axis=1)
+    st, info = wl.check(big)
+    assert st == B.TT_OK
+    assert info.legal.tile_n == 208 and info.legal.split_k == 3 and info.changed & B.TT_CHG_SPLIT_K
+    # strict: a factor larger than the loop, or more splits than reduction tiles, is invalid code
+    assert wl.check(big, mode=B.TT_MODE_STRICT)[0] == B.TT_ERR_INVALID_SCHEDULE
+    ok = B.make_record(B.TT_FAMILY_GEMM_TC, tile_m=32, tile_n=64, tile_k=16, stages=2, split_k=3, mma_m_axis=1)
+    assert wl.check(ok, mode=B.TT_MODE_STRICT)[0] == B.TT_OK
+    # resources: 8 stages of 128x256x128 do not fit shared memory
+    fat = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=256, tile_k=128, stages=8, mma_m_axis=1)
+    huge = W._dense(512, 4096, 4096).workload()
+    st, info = huge.check(fat)
+    assert st == B.TT_ERR_RESOURCE and info.smem_bytes > 227 * 1024
+    # nonsense fields
+    for kw in (dict(tile_n=0), dict(stages=0), dict(split_k=-1), dict(raster=5), dict(mma_m_axis=7)):
+        assert wl.check(B.make_record(B.TT_FAMILY_GEMM_TC, **kw))[0] == B.TT_ERR_INVALID_SCHEDULE
+    bad = B.make_record(B.TT_FAMILY_GEMM_TC)
+    bad.version = 77
+    assert wl.check(bad)[0] == B.TT_ERR_INVALID_SCHEDULE
+
+
+def test_gemm_records_transfer_between_512_and_1024():
+    """The GEMM example of Section 4.1: records of the 512^3 and 1024^3 kernels apply to each other unchanged."""
+    a, b = W._dense(512, 512, 512).workload(), W._dense(1024, 1024, 1024).workload()
+    ra = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=128, tile_k=32, stages=4, split_k=2, mma_m_axis=1)
+    rb = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=256, tile_k=64, stages=2, split_k=1, raster=1, mma_m_axis=1)
+    for wl in (a, b):
+        for r in (ra, rb):
+            st, info = wl.check(r, mode=B.TT_MODE_STRICT)
+            assert st == B.TT_OK and info.changed == 0
+
+
+def test_simt_legalisers():
+    dw = W._dw(96, 7, 1).workload()
+    r = B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=2048, block_y=16, block_x=64, items_per_thread=4, vec_width=4, threads=256)
+    st, info = dw.check(r)
+    assert st == B.TT_OK
+    L = info.legal
+    assert L.tile_m == 96 and L.block_y == 7 and L.vec_width == 1 and L.block_x % L.items_per_thread == 0
+    assert dw.check(r, mode=B.TT_MODE_STRICT)[0] == B.TT_ERR_INVALID_SCHEDULE
+    sm = W.bert_base()[5].workload()
+    st, info = sm.check(B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=24, block_y=3, vec_width=4))
+    assert st == B.TT_OK and info.legal.block_x == 16 and info.threads % 32 == 0 and info.legal.vec_width == 4
+
+
+def test_device_calls_fail_loudly_without_gpu():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("GPU present")
+    wl = W._dense(8, 16, 8).workload()
+    st, _ = wl.try_apply(wl.default_schedule())
+    assert st == B.TT_ERR_CUDA                      # no CPU fallback
+    t = B.tt_tensors()
+    assert B.lib().tt_run(wl.handle, ctypes.byref(t), None) == B.TT_ERR_NOT_APPLIED

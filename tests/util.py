@@ -13,18 +13,7 @@ def tolerance(op):
 
 
 def oracle_ref(spec, a, mode=orc.MODE_EXACT, threads=0):
-    s = spec.shapes
-    if spec.op == B.TT_OP_CONV2D:
-        return orc.conv2d(a["x"], a["w"], a["bias"], (s.stride_h, s.stride_w), (s.pad_h, s.pad_w), s.act,
-                          a.get("residual"), mode=mode, threads=threads)
-    if spec.op == B.TT_OP_DWCONV2D:
-        return orc.dwconv2d(a["x"], a["w"], a["bias"], (s.stride_h, s.stride_w), (s.pad_h, s.pad_w), s.act,
-                            threads=threads)
-    if spec.op == B.TT_OP_DENSE:
-        return orc.dense(a["x"], a["w"], a["bias"], s.act, mode=mode, threads=threads)
-    if spec.op == B.TT_OP_BATCH_MATMUL:
-        return orc.batch_matmul(a["x"], a["w"], None, bool(s.trans_b), s.act, mode=mode, threads=threads)
-    return orc.softmax(a["x"], s.scale, threads=threads)
+    return orc.reference(spec.op, spec.shapes, a, mode=mode, threads=threads)
 
 
 def rel_l2(y, ref):
