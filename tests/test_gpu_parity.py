@@ -12,6 +12,8 @@ import util
 
 pytestmark = pytest.mark.gpu
 
+INVARIANCE_TOL = 1e-5   # between two valid records on the same precision path
+
 
 def tc(**kw):
     return B.make_record(B.TT_FAMILY_GEMM_TC, **kw)
@@ -51,9 +53,10 @@ def check_all_records(spec, seed, records=GEMM_RECORDS):
     a = W.make_inputs(spec, seed)
     ref = util.oracle_ref(spec, a)
     outs = [run_spec(spec, r, a, ref) for r in records]
-    # a schedule changes speed, never semantics: every valid record gives the same output (up to summation order)
+    # a schedule changes speed, never semantics: every valid record gives the same output up to the order of the
+    # fp32 additions (tile_k and split_k regroup them): sqrt(K) * 2^-24 is about 4e-6 at the largest K here
     for y in outs[1:]:
-        assert util.rel_l2(y, outs[0]) <= 1e-6
+        assert util.rel_l2(y, outs[0]) <= INVARIANCE_TOL
     return outs
 
 
@@ -101,7 +104,7 @@ def test_config1_every_pool_record_and_selection():
     pool = W.single_conv_pool()
     outs = [run_spec(spec, r, a, ref) for r in pool]
     for y in outs[1:]:
-        assert util.rel_l2(y, outs[0]) <= 1e-6
+        assert util.rel_l2(y, outs[0]) <= INVARIANCE_TOL
     wl = spec.workload()
     t, tt = W.device_tensors(spec, a)
     res = B.transfer_tune([wl], [tt], pool)
