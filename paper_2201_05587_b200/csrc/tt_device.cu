@@ -10,8 +10,7 @@
 
 namespace tt {
 
-cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const ReduceArgs& red, const void* tmap_a,
-                        const void* tmap_b, cudaStream_t st);
+cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, cudaStream_t st);
 cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st);
 cudaError_t launch_row(const tt_apply_info& I, const RowArgs& row, cudaStream_t st);
 
@@ -87,9 +86,14 @@ tt_status bind_device(tt_workload* w) {
         if (cudaMalloc(&w->workspace, need) != cudaSuccess) { cudaGetLastError(); return TT_ERR_OOM; }
         w->workspace_bytes = need;
     }
+    if (need > 0) {
+        // arrival counters start at zero; each launch leaves them at zero again
+        const size_t off = (size_t)w->plan.partial_bytes;
+        if (cudaMemset(static_cast<char*>(w->workspace) + off, 0, need - off) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    }
     if (!w->status_word) {
-        if (cudaMalloc(reinterpret_cast<void**>(&w->status_word), 16) != cudaSuccess) { cudaGetLastError(); return TT_ERR_OOM; }
-        if (cudaMemset(w->status_word, 0, 16) != cudaSuccess) return TT_ERR_CUDA;
+        if (cudaMalloc(reinterpret_cast<void**>(&w->status_word), 512) != cudaSuccess) { cudaGetLastError(); return TT_ERR_OOM; }
+        if (cudaMemset(w->status_word, 0, 512) != cudaSuccess) return TT_ERR_CUDA;
     }
     w->tmaps.clear();
     return TT_OK;
@@ -130,7 +134,6 @@ tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
     const Plan& p = w->plan;
     if (w->family == TT_FAMILY_GEMM_TC) {
         GemmArgs g = p.g;
-        ReduceArgs red = p.red;
         const void* a_ptr = pick(t, p.a_tensor);
         const void* b_ptr = pick(t, p.b_tensor);
         const TmapPair* maps = nullptr;
@@ -142,10 +145,12 @@ tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
         g.bias = w->sh.has_bias ? static_cast<const float*>(t->bias) : nullptr;
         g.residual = w->sh.has_residual ? static_cast<const float*>(t->residual) : nullptr;
         g.partial = static_cast<float*>(w->workspace);
+        g.counters = reinterpret_cast<unsigned*>(static_cast<char*>(w->workspace) + p.partial_bytes);
         g.status = w->status_word;
-        if ((reinterpret_cast<uintptr_t>(t->y) & 15u) != 0) { g.vec_store = 0; red.vec = 0; }
-        red.partial = g.partial; red.y = g.y; red.bias = g.bias; red.residual = g.residual;
-        e = launch_gemm(p.info, g, red, maps->a, maps->b, st);
+        if ((reinterpret_cast<uintptr_t>(t->y) & 15u) != 0 ||
+            (g.residual && (reinterpret_cast<uintptr_t>(g.residual) & 15u) != 0)) g.vec_store = 0;
+        if (g.bias && (reinterpret_cast<uintptr_t>(g.bias) & 15u) == 0) g.vec_store |= 2;
+        e = launch_gemm(p.info, g, maps->a, maps->b, st);
     } else if (w->family == TT_FAMILY_DW_SIMT) {
         DwArgs d = p.dw;
         d.x = static_cast<const float*>(t->x); d.w = static_cast<const float*>(t->w);
@@ -305,6 +310,16 @@ tt_status tt_schedule_apply_ex(tt_workload* w, const tt_schedule_record* rec, in
 }
 
 tt_status tt_run(tt_workload* w, const tt_tensors* t, void* cuda_stream) { return launch(w, t, cuda_stream); }
+
+#ifdef TT_PHASE_TIMERS
+// Diagnostic build only: copy the 10 phase stamps (global timer ns, SM clock) of the last GEMM launch.
+tt_status tt_debug_read_timers(tt_workload* w, unsigned long long* out50) {
+    if (!w || !w->status_word || !out50) return TT_ERR_INVALID_ARG;
+    cudaDeviceSynchronize();
+    return cudaMemcpy(out50, reinterpret_cast<char*>(w->status_word) + 16, 50 * 8, cudaMemcpyDeviceToHost) == cudaSuccess
+               ? TT_OK : TT_ERR_CUDA;
+}
+#endif
 
 tt_status tt_workload_status(tt_workload* w, void* cuda_stream) {
     if (!w) return TT_ERR_INVALID_ARG;

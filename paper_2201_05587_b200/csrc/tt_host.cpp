@@ -128,7 +128,15 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     const int atom_k = std::min(tk, 32), n_atoms = tk / atom_k, row_bytes = atom_k * 4;
     const unsigned a_stage = (unsigned)n_atoms * kHwTileM * row_bytes;
     const unsigned b_stage = (unsigned)n_atoms * tn * row_bytes;
-    const long long smem = (long long)st * (a_stage + b_stage) + 1024;
+    // pipeline buffers, reused by the epilogue as a 32 x 36-float staging area per warp; then the im2col k-table
+    // (one word per reduction index of a CTA's K range); 1 KB of alignment slack
+    const long long pipe = std::max<long long>((long long)st * (a_stage + b_stage), (long long)kGatherWarps * 32 * 36 * 4);
+    const long long ktab = w->op == TT_OP_CONV2D ? (long long)per_split * tk * 4 : 0;
+    const long long smem = pipe + ktab + 1024;
+    if (w->op == TT_OP_CONV2D) {
+        // table packing: element offsets below 2^26, tap indices below 63
+        if ((long long)s.c * s.h * s.w >= (1ll << 26) || s.r * s.s > 63) return TT_ERR_RESOURCE;
+    }
     int tmem_cols = std::max(32, pow2_ceil(tn));
     const int tiles_m = (M + kHwTileM - 1) / kHwTileM, tiles_n = (N + tn - 1) / tn;
     if ((long long)tiles_m * tiles_n > 0x7fffffffLL || sk > 65535 || B > 65535) return TT_ERR_RESOURCE;
@@ -141,8 +149,10 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     I.threads = kGemmThreads;
     I.smem_bytes = (int)std::min<long long>(smem, 0x7fffffff);
     I.tmem_cols = tmem_cols;
-    I.workspace_bytes = sk > 1 ? (int64_t)sk * B * M * N * 4 : 0;
-    I.launches = sk > 1 ? 2 : 1;
+    // split-K workspace: partial tiles, then one arrival counter per (batch, tile)
+    plan->partial_bytes = sk > 1 ? (((long long)sk * B * M * N * 4 + 255) / 256) * 256 : 0;
+    I.workspace_bytes = sk > 1 ? plan->partial_bytes + (int64_t)B * tiles_m * tiles_n * 4 : 0;
+    I.launches = 1;
     if (smem > kDynSmemLimit) return TT_ERR_RESOURCE;
 
     GemmArgs& g = plan->g;
@@ -154,6 +164,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     g.atom_k = atom_k; g.n_atoms = n_atoms; g.row_bytes = row_bytes;
     g.swz_mask = row_bytes == 128 ? 7 : (row_bytes == 64 ? 3 : 1);
     g.a_stage_bytes = a_stage; g.b_stage_bytes = b_stage;
+    g.ktab_off = (unsigned)pipe;
     g.tmem_cols = (unsigned)tmem_cols;
     // Instruction descriptor, kind::tf32: D = F32 (bits 4-5 = 1), A and B = TF32 (bits 7-9, 10-12 = 2), both
     // K-major (bits 15, 16 = 0), N >> 3 at bits 17-22, M >> 4 at bits 24-28.
@@ -191,11 +202,6 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     g.sh = s.stride_h; g.sw = s.stride_w; g.ph = s.pad_h; g.pw = s.pad_w;
     g.tx_bytes = (A.mode == OPM_TMA ? a_stage : 0) + (Bo.mode == OPM_TMA ? b_stage : 0);
     g.vec_store = (g.y_ns == 1 && g.y_ms % 4 == 0 && g.y_bs % 4 == 0) ? 1 : 0;
-    // the split-K reduction kernel reads [split][batch][M][N] and writes y through the same strides
-    ReduceArgs& r = plan->red;
-    r = ReduceArgs{};
-    r.split_k = sk; r.batch = B; r.M = M; r.N = N; r.y_ms = g.y_ms; r.y_ns = g.y_ns; r.y_bs = g.y_bs;
-    r.bias_mode = g.bias_mode; r.act = g.act; r.vec = (g.vec_store && N % 4 == 0) ? 1 : 0;
     return TT_OK;
 }
 

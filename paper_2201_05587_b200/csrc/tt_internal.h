@@ -10,8 +10,10 @@ namespace tt {
 constexpr int kHwTileM = 128;           // tcgen05 accumulator rows per CTA (cta_group::1, M = 128)
 constexpr int kMaxStages = 8;
 constexpr int kSmemLimit = 232448;      // 227 KB opt-in shared memory per CTA on sm_100
-constexpr int kDynSmemLimit = kSmemLimit - 1024;  // what is left for dynamic shared memory beside barriers
-constexpr int kGemmThreads = 192;       // warp 0 TMA, warp 1 MMA + TMEM, warps 2-5 gather + epilogue
+constexpr int kDynSmemLimit = kSmemLimit - 6144;  // what is left for dynamic shared memory beside barriers
+constexpr int kGatherWarps = 8;
+constexpr int kGatherThreads = kGatherWarps * 32;
+constexpr int kGemmThreads = 64 + kGatherThreads;   // warp 0 TMA, warp 1 MMA + TMEM, warps 2-9 gather + epilogue
 
 // How one operand of the contraction reaches shared memory.
 enum OperandMode : int {
@@ -37,15 +39,12 @@ struct GemmArgs {
     int act;
     const float* residual;
     float* partial;                             // split-K partial sums [split][batch][M][N]
+    unsigned* counters;                         // split-K arrival counters [batch][tiles], zero between launches
     unsigned* status;
     unsigned idesc, tmem_cols;
     unsigned a_stage_bytes, b_stage_bytes, tx_bytes;
-    int vec_store;                              // 1: y rows allow aligned float4 stores
-};
-
-struct ReduceArgs {
-    const float* partial; float* y; const float* bias; const float* residual;
-    int split_k, batch, M, N; long long y_ms, y_ns, y_bs; int bias_mode, act, vec;
+    unsigned ktab_off;                          // im2col k-table: byte offset from the aligned tile base
+    int vec_store;                              // bit 0: y rows allow aligned float4 stores; bit 1: so does bias
 };
 
 struct DwArgs {
@@ -69,7 +68,7 @@ struct Plan {
     bool swap_ab = false;
     int a_tensor = 0, b_tensor = 1;   // which caller tensor feeds operand A / B: 0 = x, 1 = w
     GemmArgs g{};
-    ReduceArgs red{};
+    long long partial_bytes = 0;      // counters start here inside the workspace
     DwArgs dw{};
     RowArgs row{};
 };

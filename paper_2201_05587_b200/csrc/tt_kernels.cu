@@ -1,8 +1,9 @@
 // Device code of libtt for sm_100a: the schedule-parameterised kernel families.
 //
 //   GEMM_TC  tcgen05.mma kind::tf32, accumulator in tensor memory, operands staged in shared memory by TMA
-//            (K-major tensors) or by gather warps (im2col of NCHW activations, strided views), `stages`-deep
-//            mbarrier pipeline, bias/activation fused into the accumulator read-out, deterministic split-K.
+//            (K-major tensors) or by gather warps issuing cp.async (im2col of NCHW activations, strided views),
+//            `stages`-deep mbarrier pipeline, bias/activation fused into the accumulator read-out, split-K with
+//            an in-kernel reduction in fixed split order by the last-arriving CTA of each tile.
 //   DW_SIMT  depthwise convolution, shared-memory halo tile, fp32 FMA.
 //   ROW_SIMT row softmax with sub-warp shuffles.
 //
@@ -50,10 +51,24 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second per wait, then give up
 
+// Diagnostic build only (-DTT_PHASE_TIMERS): CTA (0,0,0) stamps the global timer and the SM clock at the phase
+// boundaries of the GEMM kernel into the 64-bit slots that follow the status word.
+#ifdef TT_PHASE_TIMERS
+__device__ unsigned long long* g_tt_dbg = nullptr;       // set by CTA (0,0,0) before its first barrier
+__device__ __forceinline__ void tt_stamp(int slot) {
+    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && g_tt_dbg) {
+        g_tt_dbg[2 * slot] = global_timer_ns();
+        g_tt_dbg[2 * slot + 1] = (unsigned long long)clock64();
+    }
+}
+#define TT_STAMP(slot) tt_stamp(slot)
+#else
+#define TT_STAMP(slot) do { } while (0)
+#endif
+
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
-                                       unsigned where) {
-    if (mbar_try_wait(bar, parity)) return true;
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
+                                            unsigned where) {
     const unsigned long long t0 = global_timer_ns();
     unsigned spins = 0;
     for (;;) {
@@ -67,6 +82,12 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
             }
         }
     }
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
+                                          unsigned where) {
+    if (mbar_try_wait(bar, parity)) return true;         // the common case costs one instruction
+    return mbar_wait_slow(bar, parity, abort_flag, status, where);
 }
 
 __device__ __forceinline__ void fence_proxy_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -142,76 +163,211 @@ __device__ __forceinline__ uint32_t swz_off(uint32_t row, uint32_t kbyte, uint32
 }
 
 // ------------------------------------------------------------------------------------------------------------
-// Gather producers: fill one operand tile of one pipeline stage with generic-proxy stores.
-// `rows` tile rows starting at global row row0 (valid below row_extent), reduction indices k0 .. k0 + tile_k.
+// Gather producers.  The 8 gather warps form 1, 2 or 4 groups; group g fills pipeline stages g, g + groups, ...
+// so that the global-memory latency of one stage overlaps the other groups' stages.  Within a stage a warp
+// takes (32-row block, 4-wide k chunk) tasks: lanes walk rows (coalesced loads), each lane assembles four
+// consecutive reduction indices of its row in registers and writes one 16-byte chunk into the swizzled K-major
+// tile.  Loads of four tasks are issued before the first store, so 16 loads per lane are in flight.
 // ------------------------------------------------------------------------------------------------------------
 struct Im2col { int C, H, W, R, S, Q, sh, sw, ph, pw; };
 
-__device__ __forceinline__ void gather_tile(int mode, uint32_t tile_smem, int rows, int row0, int row_extent,
-                                            const float* __restrict__ src, long long rs, long long ks,
-                                            const Im2col& ic, int k0, int K, int tile_k, int atom_k, int row_bytes,
-                                            int swz_mask, int gw, int n_gw, int lane) {
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, float a, float b, float c, float d) {
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ void st_shared_f32(uint32_t addr, float a) {
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(a) : "memory");
+}
+
+// One stage of an operand whose rows are contiguous across lanes: IM2COL (rows = output pixels of an NCHW
+// image, k = (c, r, s)) or GATHER_ROWS (strided view with unit row stride).
+// IM2COL reads two shared-memory tables built once per CTA: ktab[k] = (element offset c*H*W + r*W + s) << 6 |
+// tap index r*S + s (63 for k beyond K), and rowinfo[row] = {ih0*W + iw0, in-bounds tap mask low, high, -} of the
+// row's output pixel (mask 0 for rows past the extent), so the inner loop holds neither a division nor a
+// bounds comparison: one table word per k (warp-uniform), one mask bit test and one add per element.
+template <int MODE>
+__device__ __forceinline__ void gather_rows_stage(uint32_t tile_smem, int rows, const float* __restrict__ src,
+                                                  long long rs, long long ks, const int4* rowinfo, const uint32_t* ktab,
+                                                  int row0, int row_extent, int k0, int K, int tile_k, int atom_k,
+                                                  int row_bytes, int swz_mask, int wig, int wpg, int lane) {
+    const int atom_shift = atom_k == 32 ? 5 : (atom_k == 16 ? 4 : 3);
+    const int shift = row_bytes == 128 ? 0 : (row_bytes == 64 ? 1 : 2);
     const uint32_t atom_bytes = (uint32_t)rows * (uint32_t)row_bytes;
-    if (mode == OPM_GATHER_K) {
-        // lanes walk k (contiguous in memory): 4-byte stores, conflict-free inside a row
-        for (int r = gw; r < rows; r += n_gw) {
-            const int grow = row0 + r;
-            const bool rv = grow < row_extent;
-            for (int kk = lane; kk < tile_k; kk += 32) {
-                const int k = k0 + kk;
-                float v = 0.f;
-                if (rv && k < K) v = __ldg(src + (long long)grow * rs + (long long)k * ks);
-                const int atom = kk / atom_k, ka = kk - atom * atom_k;
-                const uint32_t addr = tile_smem + atom * atom_bytes + swz_off(r, ka * 4, row_bytes, swz_mask);
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
-            }
-        }
-        return;
-    }
-    // lanes walk rows; each thread assembles 4 consecutive k of its row and writes one 16-byte chunk
-    const int row_groups = (rows + 31) >> 5;
-    const int k_chunks = tile_k >> 2;
-    const int units = row_groups * k_chunks;
-    const int RS = ic.R * ic.S;
-    for (int u = gw; u < units; u += n_gw) {
-        const int rg = u % row_groups, kc = u / row_groups;
-        const int r = rg * 32 + lane;
-        if (r >= rows) continue;
-        const int grow = row0 + r;
-        const int kb = k0 + kc * 4;
-        float v[4] = {0.f, 0.f, 0.f, 0.f};
-        if (grow < row_extent) {
-            if (mode == OPM_IM2COL) {
-                const int p = grow / ic.Q, q = grow - p * ic.Q;
-                const int ih0 = p * ic.sh - ic.ph, iw0 = q * ic.sw - ic.pw;
+    const int n_rb = (rows + 31) >> 5;
+    const int n_ch = tile_k >> 2;
+    const int my_ch = (n_ch - wig + wpg - 1) / wpg;      // chunks wig, wig + wpg, ... belong to this warp
+    const int n_tasks = my_ch > 0 ? my_ch * n_rb : 0;    // task = (chunk, 32-row block)
+    const uint32_t inv_rb = (65536u + (uint32_t)n_rb - 1u) / (uint32_t)n_rb;     // t / n_rb == (t * inv_rb) >> 16 for small t
+    constexpr int kBatch = 8;                            // tasks whose loads are issued before the first store
+    for (int t0 = 0; t0 < n_tasks; t0 += kBatch) {
+        float val[kBatch][4];
+        uint32_t dst[kBatch];
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+            const int t = t0 + b;
+            const bool live = t < n_tasks;               // warp-uniform
+            const int tt = live ? t : 0;
+            const int ci = (int)(((uint32_t)tt * inv_rb) >> 16);
+            const int rb = tt - ci * n_rb;
+            const int kk = (wig + ci * wpg) * 4;
+            const int row = rb * 32 + lane;
+            const bool in_tile = live && row < rows;
+            dst[b] = in_tile ? tile_smem + (uint32_t)(kk >> atom_shift) * atom_bytes + (uint32_t)row * (uint32_t)row_bytes +
+                                   ((uint32_t)((kk & (atom_k - 1)) << 2) ^ ((uint32_t)((row >> shift) & swz_mask) << 4))
+                             : 0xffffffffu;
+            if (MODE == OPM_IM2COL) {
+                const uint4 e = *reinterpret_cast<const uint4*>(ktab + kk);      // same address in every lane
+                const int4 info = rowinfo[row < rows ? row : 0];
+                const uint32_t ev[4] = {e.x, e.y, e.z, e.w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const int k = kb + j;
-                    if (k < K) {
-                        const int c = k / RS, rs_ = k - c * RS;
-                        const int fr = rs_ / ic.S, fs = rs_ - fr * ic.S;
-                        const int ih = ih0 + fr, iw = iw0 + fs;
-                        if (ih >= 0 && ih < ic.H && iw >= 0 && iw < ic.W)
-                            v[j] = __ldg(src + ((long long)c * ic.H + ih) * ic.W + iw);
-                    }
+                    const uint32_t tap = ev[j] & 63u;
+                    const uint32_t word = tap < 32u ? (uint32_t)info.y : (uint32_t)info.z;
+                    const bool ok = in_tile && ((word >> (tap & 31u)) & 1u) != 0u;
+                    val[b][j] = ok ? __ldg(src + ((int)(ev[j] >> 6) + info.x)) : 0.f;
                 }
             } else {
+                const int grow = row0 + row;
+                const bool rv = in_tile && grow < row_extent;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const int k = kb + j;
-                    if (k < K) v[j] = __ldg(src + (long long)grow * rs + (long long)k * ks);
+                    const int k = k0 + kk + j;
+                    val[b][j] = (rv && k < K) ? __ldg(src + (long long)grow * rs + (long long)k * ks) : 0.f;
                 }
             }
         }
-        const int kk = kc * 4;
-        const int atom = kk / atom_k, ka = kk - atom * atom_k;
-        const uint32_t addr = tile_smem + atom * atom_bytes + swz_off(r, ka * 4, row_bytes, swz_mask);
-        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b)
+            if (dst[b] != 0xffffffffu) st_shared_v4(dst[b], val[b][0], val[b][1], val[b][2], val[b][3]);
+    }
+}
+
+// One stage of an operand whose reduction index is contiguous in memory but cannot go through TMA (K % 4 != 0):
+// a warp takes rows, its lanes walk k; 4-byte stores stay inside one swizzled row (conflict-free).
+__device__ __forceinline__ void gather_k_stage(uint32_t tile_smem, int rows, const float* __restrict__ src, long long rs,
+                                               long long ks, int row0, int row_extent, int k0, int K, int tile_k,
+                                               int atom_k, int row_bytes, int swz_mask, int wig, int wpg, int lane) {
+    const int atom_shift = atom_k == 32 ? 5 : (atom_k == 16 ? 4 : 3);
+    const int shift = row_bytes == 128 ? 0 : (row_bytes == 64 ? 1 : 2);
+    const uint32_t atom_bytes = (uint32_t)rows * (uint32_t)row_bytes;
+    for (int kk = lane; kk < tile_k; kk += 32) {
+        const int k = k0 + kk;
+        const uint32_t kterm = (uint32_t)(kk >> atom_shift) * atom_bytes;
+        const uint32_t kb = (uint32_t)((kk & (atom_k - 1)) << 2);
+        for (int r0 = wig; r0 < rows; r0 += wpg * 4) {
+            float val[4];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int r = r0 + b * wpg;
+                const int grow = row0 + r;
+                val[b] = (r < rows && grow < row_extent && k < K) ? __ldg(src + (long long)grow * rs + (long long)k * ks) : 0.f;
+            }
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int r = r0 + b * wpg;
+                if (r < rows)
+                    st_shared_f32(tile_smem + kterm + (uint32_t)r * (uint32_t)row_bytes + (kb ^ ((uint32_t)((r >> shift) & swz_mask) << 4)), val[b]);
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void gather_stage(int mode, uint32_t tile_smem, int rows, const float* __restrict__ src,
+                                             long long rs, long long ks, const int4* rowinfo, const uint32_t* ktab,
+                                             int row0, int row_extent, int k0, int K, int tile_k, int atom_k, int row_bytes,
+                                             int swz_mask, int wig, int wpg, int lane) {
+    if (mode == OPM_IM2COL)
+        gather_rows_stage<OPM_IM2COL>(tile_smem, rows, src, rs, ks, rowinfo, ktab, row0, row_extent, k0, K, tile_k, atom_k, row_bytes, swz_mask, wig, wpg, lane);
+    else if (mode == OPM_GATHER_ROWS)
+        gather_rows_stage<OPM_GATHER_ROWS>(tile_smem, rows, src, rs, ks, rowinfo, ktab, row0, row_extent, k0, K, tile_k, atom_k, row_bytes, swz_mask, wig, wpg, lane);
+    else
+        gather_k_stage(tile_smem, rows, src, rs, ks, row0, row_extent, k0, K, tile_k, atom_k, row_bytes, swz_mask, wig, wpg, lane);
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// Epilogue helpers
+// ------------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+
+constexpr int kStagePitch = 36;                          // floats per staged row: 16-byte accesses stay conflict-free
+constexpr int kStageBytesPerWarp = 32 * kStagePitch * 4;
+
+// ReLU, ReLU6 and "none" are one clamp with per-kernel bounds (no branch per element); GELU is a separate path.
+struct EpiArgs {
+    float* ybase; const float* rbase; long long y_ms, y_ns; int M; float lo, hi; bool gelu, vec;
+};
+
+__device__ __forceinline__ float finish_one(float v, const EpiArgs& e) {
+    if (e.gelu) return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f));     // uniform per kernel
+    return fminf(fmaxf(v, e.lo), e.hi);
+}
+
+// Store one 32-row x 32-column block of pre-activation values (bias already added) whose rows are this warp's
+// lanes.  Row-major outputs (y_ns == 1) are transposed through the warp's shared-memory staging area so that
+// eight lanes write one 128-byte row segment; otherwise lanes are contiguous in memory and each column is one
+// coalesced store.  FULL: all 32 rows and 32 columns exist and 16-byte accesses are aligned.
+// POST: a residual is added, so the activation runs here, after it; otherwise the values arrive activated.
+template <bool FULL, bool POST>
+__device__ __forceinline__ void epilogue_block(float (&v)[32], const EpiArgs& e, int m_first, int nb, int cnt,
+                                               uint32_t stg, int lane, bool transposed) {
+    if (transposed) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) st_shared_v4(stg + (uint32_t)(lane * kStagePitch + j) * 4u, v[j], v[j + 1], v[j + 2], v[j + 3]);
+        __syncwarp();
+        const int cc = (lane & 7) * 4;
+#pragma unroll
+        for (int itr = 0; itr < 8; ++itr) {
+            const int rr = itr * 4 + (lane >> 3);
+            const int m = m_first + rr;
+            float4 t;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w)
+                         : "r"(stg + (uint32_t)(rr * kStagePitch + cc) * 4u));
+            const long long o = (long long)m * e.y_ms + nb + cc;
+            if (FULL) {
+                if (POST) {
+                    const float4 r4 = __ldg(reinterpret_cast<const float4*>(e.rbase + o));
+                    t.x = finish_one(t.x + r4.x, e); t.y = finish_one(t.y + r4.y, e);
+                    t.z = finish_one(t.z + r4.z, e); t.w = finish_one(t.w + r4.w, e);
+                }
+                *reinterpret_cast<float4*>(e.ybase + o) = t;
+            } else {
+                const float tv[4] = {t.x, t.y, t.z, t.w};
+                const bool row_ok = m < e.M;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const bool ok = row_ok && cc + j < cnt;
+                    float out = tv[j];
+                    if (POST) out = finish_one(out + (ok ? __ldg(e.rbase + o + j) : 0.f), e);
+                    if (ok) e.ybase[o + j] = out;
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        const int m = m_first + lane;
+        const bool row_ok = FULL || m < e.M;
+        long long o = (long long)m * e.y_ms + (long long)nb * e.y_ns;
+#pragma unroll
+        for (int j = 0; j < 32; ++j, o += e.y_ns) {
+            const bool ok = row_ok && (FULL || j < cnt);
+            float out = v[j];
+            if (POST) out = finish_one(out + (ok ? __ldg(e.rbase + o) : 0.f), e);
+            if (ok) e.ybase[o] = out;
+        }
     }
 }
 
 // ------------------------------------------------------------------------------------------------------------
-// GEMM_TC kernel.  grid = (tiles_m * tiles_n, split_k, batch), block = 192 threads.
+// GEMM_TC kernel.  grid = (tiles_m * tiles_n, split_k, batch), block = 320 threads:
+// warp 0 TMA producer, warp 1 MMA issuer + tensor-memory owner, warps 2-9 gather producers, then epilogue.
 // ------------------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kGemmThreads, 1)
 tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const GemmArgs g) {
@@ -221,9 +377,17 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __shared__ uint64_t accum_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ int last_split_flag;
+    __shared__ __align__(16) float s_bias[256];
+    __shared__ int4 s_rowinfo[256];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int* abortp = &abort_flag;
+#ifdef TT_PHASE_TIMERS
+    if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+        g_tt_dbg = reinterpret_cast<unsigned long long*>(g.status) + 2;
+#endif
+    if (threadIdx.x == 0) TT_STAMP(0);
 
     // tile coordinates
     int tm, tn;
@@ -239,16 +403,19 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const uint32_t stage_bytes = g.a_stage_bytes + g.b_stage_bytes;
     const bool a_tma = g.a_mode == OPM_TMA, b_tma = g.b_mode == OPM_TMA;
     const bool any_tma = a_tma || b_tma, any_gather = !a_tma || !b_tma;
-    constexpr int kGatherWarps = 4;
+    // gather groups: 4 groups of 2 warps from 4 stages up, 2 groups of 4 warps for 2-3 stages, else one group
+    const int n_groups = g.stages >= 4 ? 4 : (g.stages >= 2 ? 2 : 1);
+    const int wpg = kGatherWarps / n_groups;
 
     if (threadIdx.x == 0) {
-        const uint32_t full_count = (any_tma ? 1u : 0u) + (any_gather ? (uint32_t)kGatherWarps : 0u);
+        const uint32_t full_count = (any_tma ? 1u : 0u) + (any_gather ? (uint32_t)wpg : 0u);
         for (int s = 0; s < g.stages; ++s) {
             mbar_init(smem_u32(&full_bar[s]), full_count);
             mbar_init(smem_u32(&empty_bar[s]), 1u);
         }
         mbar_init(smem_u32(&accum_bar), 1u);
         abort_flag = 0;
+        last_split_flag = 0;
         fence_mbar_init();
         fence_proxy_async_shared();
     }
@@ -260,24 +427,34 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *(volatile uint32_t*)&tmem_slot;
+    if (threadIdx.x == 0) TT_STAMP(1);
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0 && any_tma) {
             int armed = 0;   // stages whose loads were issued
-            for (int it = 0; it < iters; ++it) {
-                const int s = it % g.stages;
-                const uint32_t ph = (uint32_t)(it / g.stages) & 1u;
-                if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abortp, g.status, 1u)) break;
-                const uint32_t fb = smem_u32(&full_bar[s]);
+            uint32_t st = 0, ph = 0;
+            const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+            const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes), b_atom = (uint32_t)(g.tile_n * g.row_bytes);
+            const int a_bz = g.a_tma_batched ? bz : 0, b_bz = g.b_tma_batched ? bz : 0;
+            int k0 = kt_begin * g.tile_k;
+            for (int it = 0; it < iters; ++it, k0 += g.tile_k) {
+                if (!mbar_wait(empty0 + st * 8u, ph ^ 1u, abortp, g.status, 1u)) break;
+                const uint32_t fb = full0 + st * 8u;
                 mbar_expect_tx(fb, g.tx_bytes);
-                const uint32_t a_s = tiles_base + s * stage_bytes, b_s = a_s + g.a_stage_bytes;
-                const int k0 = (kt_begin + it) * g.tile_k;
-                for (int at = 0; at < g.n_atoms; ++at) {
-                    if (a_tma) tma_load_3d(a_s + at * (kHwTileM * g.row_bytes), &tmap_a, fb, k0 + at * g.atom_k, m0, g.a_tma_batched ? bz : 0);
-                    if (b_tma) tma_load_3d(b_s + at * (g.tile_n * g.row_bytes), &tmap_b, fb, k0 + at * g.atom_k, n0, g.b_tma_batched ? bz : 0);
+                const uint32_t a_s = tiles_base + st * stage_bytes, b_s = a_s + g.a_stage_bytes;
+                if (a_tma) {
+#pragma unroll 1
+                    for (int at = 0; at < g.n_atoms; ++at) tma_load_3d(a_s + at * a_atom, &tmap_a, fb, k0 + at * g.atom_k, m0, a_bz);
+                }
+                if (b_tma) {
+#pragma unroll 1
+                    for (int at = 0; at < g.n_atoms; ++at) tma_load_3d(b_s + at * b_atom, &tmap_b, fb, k0 + at * g.atom_k, n0, b_bz);
                 }
                 armed = it + 1;
+                if (it == 5) TT_STAMP(10);
+                if (it == 6) TT_STAMP(11);
+                if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
             }
             if (*abortp) {
                 // let copies in flight land before shared memory is given back (bounded)
@@ -294,104 +471,241 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             bool ok = true;
-            for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % g.stages;
-                const uint32_t ph = (uint32_t)(it / g.stages) & 1u;
-                if (!mbar_wait(smem_u32(&full_bar[s]), ph, abortp, g.status, 2u)) { ok = false; break; }
+            uint32_t st = 0, ph = 0;
+            const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+            // descriptors differ only in their 14-bit start-address field: keep the constant upper word, step the
+            // lower word by (bytes >> 4) per stage, per atom and per 8-wide K slice
+            const uint64_t d0 = make_desc(0u, g.row_bytes);
+            const uint32_t d_hi = (uint32_t)(d0 >> 32), d_lo = (uint32_t)d0;
+            const uint32_t a_lo0 = d_lo + ((tiles_base & 0x3FFFFu) >> 4);
+            const uint32_t b_lo0 = a_lo0 + (g.a_stage_bytes >> 4);
+            const uint32_t stage_step = stage_bytes >> 4;
+            const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes) >> 4, b_atom = (uint32_t)(g.tile_n * g.row_bytes) >> 4;
+            const int k8_per_atom = g.atom_k >> 3;
+            const int k8_shift = k8_per_atom == 4 ? 2 : (k8_per_atom == 2 ? 1 : 0);
+            const int n_mma = g.tile_k >> 3;
+            uint32_t accumulate = 0u;
+            for (int it = 0; it < iters; ++it) {
+                if (!mbar_wait(full0 + st * 8u, ph, abortp, g.status, 2u)) { ok = false; break; }
+                if (it == 0) TT_STAMP(2);
+                if (it == 5) TT_STAMP(12);
+                if (it == 6) TT_STAMP(13);
                 tc_fence_after();
-                const uint32_t a_s = tiles_base + s * stage_bytes, b_s = a_s + g.a_stage_bytes;
-                const int k8_per_atom = g.atom_k >> 3;
-                for (int at = 0; at < g.n_atoms; ++at) {
-                    const uint64_t ad = make_desc(a_s + at * (kHwTileM * g.row_bytes), g.row_bytes);
-                    const uint64_t bd = make_desc(b_s + at * (g.tile_n * g.row_bytes), g.row_bytes);
-                    for (int k8 = 0; k8 < k8_per_atom; ++k8) {
-                        // 8 TF32 = 32 bytes further along K inside the swizzle atom: start address + 2 (16-byte units)
-                        mma_tf32(tmem_base, ad + (uint64_t)(k8 * 2), bd + (uint64_t)(k8 * 2), g.idesc,
-                                 (it > 0 || at > 0 || k8 > 0) ? 1u : 0u);
-                    }
+                const uint32_t a_lo = a_lo0 + st * stage_step, b_lo = b_lo0 + st * stage_step;
+#pragma unroll 4
+                for (int i8 = 0; i8 < n_mma; ++i8) {
+                    const uint32_t at = (uint32_t)i8 >> k8_shift, k8 = (uint32_t)i8 & (uint32_t)(k8_per_atom - 1);
+                    // 8 TF32 = 32 bytes further along K inside the swizzle atom: start address + 2 (16-byte units)
+                    const uint64_t ad = ((uint64_t)d_hi << 32) | (uint64_t)(a_lo + at * a_atom + k8 * 2u);
+                    const uint64_t bd = ((uint64_t)d_hi << 32) | (uint64_t)(b_lo + at * b_atom + k8 * 2u);
+                    mma_tf32(tmem_base, ad, bd, g.idesc, accumulate);
+                    accumulate = 1u;
                 }
-                mma_commit(smem_u32(&empty_bar[s]));     // stage reusable once these MMAs have read it
+                mma_commit(empty0 + st * 8u);            // stage reusable once these MMAs have read it
+                if (it == 5) TT_STAMP(14);
+                if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
             }
             if (ok) mma_commit(smem_u32(&accum_bar));    // accumulator complete
+            TT_STAMP(3);
         }
     } else {
         // ---------------- gather producers, then epilogue ----------------
         const int gw = warp - 2;
+        const int gt = (int)threadIdx.x - 64;
+        const int quad = warp & 3;                       // tensor-memory lane quadrant this warp may read
+        const int m = m0 + quad * 32 + lane;
+        // bias is fetched now so that its latency hides behind the main loop
+        if (g.bias_mode == 2 && gt < g.tile_n) s_bias[gt] = (n0 + gt < g.N) ? __ldg(g.bias + n0 + gt) : 0.f;
+        const float bias_row = (g.bias_mode == 1 && m < g.M) ? __ldg(g.bias + m) : 0.f;
         if (any_gather) {
-            Im2col ic{g.C, g.H, g.W, g.R, g.S, g.Q, g.sh, g.sw, g.ph, g.pw};
+            const Im2col ic{g.C, g.H, g.W, g.R, g.S, g.Q, g.sh, g.sw, g.ph, g.pw};
             const float* a_src = g.a + (long long)bz * g.a_bs;
             const float* b_src = g.b + (long long)bz * g.b_bs;
-            for (int it = 0; it < iters; ++it) {
-                const int s = it % g.stages;
-                const uint32_t ph = (uint32_t)(it / g.stages) & 1u;
-                if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abortp, g.status, 3u)) break;
-                const uint32_t a_s = tiles_base + s * stage_bytes, b_s = a_s + g.a_stage_bytes;
+            uint32_t* ktab = reinterpret_cast<uint32_t*>(smem_raw + (tiles_base - smem_u32(smem_raw)) + g.ktab_off);
+            if (g.a_mode == OPM_IM2COL || g.b_mode == OPM_IM2COL) {
+                // Tables of the im2col operand, built once per CTA.
+                // rowinfo: per tile row, where its pixel's receptive field starts and which filter taps fall
+                // inside the image (bit r*S + s); ktab: per reduction index of this CTA's K range, the element
+                // offset of (c, r, s) and its tap index.
+                const bool on_a = g.a_mode == OPM_IM2COL;
+                const int rows = on_a ? kHwTileM : g.tile_n, row0 = on_a ? m0 : n0, ext = on_a ? g.M : g.N;
+                if (gt < rows) {
+                    const int grow = row0 + gt;
+                    int4 info = make_int4(0, 0, 0, 0);
+                    if (grow < ext) {
+                        const int p = grow / ic.Q, q = grow - p * ic.Q;
+                        const int ih0 = p * ic.sh - ic.ph, iw0 = q * ic.sw - ic.pw;
+                        const int s_lo = max(0, -iw0), s_hi = min(ic.S, ic.W - iw0);      // taps s_lo .. s_hi-1 are in range
+                        const unsigned long long colmask = s_hi > s_lo ? (((1ull << s_hi) - 1ull) & ~((1ull << s_lo) - 1ull)) : 0ull;
+                        unsigned long long mask = 0ull;
+                        for (int fr = 0; fr < ic.R; ++fr)
+                            if ((unsigned)(ih0 + fr) < (unsigned)ic.H) mask |= colmask << (fr * ic.S);
+                        info.x = ih0 * ic.W + iw0; info.y = (int)(uint32_t)mask; info.z = (int)(uint32_t)(mask >> 32);
+                    }
+                    s_rowinfo[gt] = info;
+                }
+                const int RS = ic.R * ic.S, HW = ic.H * ic.W;
+                const int kbeg = kt_begin * g.tile_k;
+                for (int i = gt; i < iters * g.tile_k; i += kGatherThreads) {
+                    const int k = kbeg + i;
+                    uint32_t ent = 63u;                  // beyond K: a tap no mask ever enables
+                    if (k < g.K) {
+                        const int c = k / RS, rem = k - c * RS, fr = rem / ic.S, fs = rem - fr * ic.S;
+                        ent = ((uint32_t)(c * HW + fr * ic.W + fs) << 6) | (uint32_t)rem;
+                    }
+                    ktab[i] = ent;
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kGatherThreads) : "memory");
+            }
+            const int grp = gw / wpg, wig = gw - grp * wpg;
+            const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+            int st = grp % g.stages;
+            uint32_t ph = (uint32_t)(grp / g.stages) & 1u;
+            for (int it = grp; it < iters; it += n_groups) {
+                if (!mbar_wait(empty0 + (uint32_t)st * 8u, ph ^ 1u, abortp, g.status, 3u)) break;
+                const uint32_t a_s = tiles_base + (uint32_t)st * stage_bytes, b_s = a_s + g.a_stage_bytes;
                 const int k0 = (kt_begin + it) * g.tile_k;
-                if (!a_tma) gather_tile(g.a_mode, a_s, kHwTileM, m0, g.M, a_src, g.a_rs, g.a_ks, ic, k0, g.K, g.tile_k,
-                                        g.atom_k, g.row_bytes, g.swz_mask, gw, kGatherWarps, lane);
-                if (!b_tma) gather_tile(g.b_mode, b_s, g.tile_n, n0, g.N, b_src, g.b_rs, g.b_ks, ic, k0, g.K, g.tile_k,
-                                        g.atom_k, g.row_bytes, g.swz_mask, gw, kGatherWarps, lane);
+                if (threadIdx.x == 64 && it == 4) TT_STAMP(15);
+                const uint32_t* kt = ktab + (it * g.tile_k);
+                if (!a_tma) gather_stage(g.a_mode, a_s, kHwTileM, a_src, g.a_rs, g.a_ks, s_rowinfo, kt, m0, g.M, k0, g.K, g.tile_k,
+                                         g.atom_k, g.row_bytes, g.swz_mask, wig, wpg, lane);
+                if (!b_tma) gather_stage(g.b_mode, b_s, g.tile_n, b_src, g.b_rs, g.b_ks, s_rowinfo, kt, n0, g.N, k0, g.K, g.tile_k,
+                                         g.atom_k, g.row_bytes, g.swz_mask, wig, wpg, lane);
+                if (threadIdx.x == 64 && it == 4) TT_STAMP(16);
                 fence_proxy_async_shared();              // generic-proxy stores -> visible to the tensor core's reads
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&full_bar[s]));
+                if (lane == 0) mbar_arrive(full0 + (uint32_t)st * 8u);
+                if (threadIdx.x == 64 && it == 4) TT_STAMP(17);
+                st += n_groups;
+                while (st >= g.stages) { st -= g.stages; ph ^= 1u; }
             }
         }
-        // epilogue: warp (warp % 4) owns tensor-memory lanes 32*(warp % 4) .. +31
+        // epilogue: warp w owns tensor-memory lanes 32*(w % 4) .. +31; the two warps of a lane quadrant take
+        // alternate 32-column blocks
         const bool have_acc = mbar_wait(smem_u32(&accum_bar), 0u, abortp, g.status, 4u);
-        if (have_acc) {
+        // every epilogue thread takes the same decision (named barrier 1 over the epilogue threads); the barrier
+        // also orders the bias staging above against its readers below
+        uint32_t all_acc;
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "setp.ne.u32 q, %1, 0;\n\t"
+            "bar.red.and.pred p, 1, %2, q;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(all_acc) : "r"((uint32_t)have_acc), "n"(kGatherThreads) : "memory");
+        if (threadIdx.x == 64) TT_STAMP(4);
+        if (all_acc) {
             tc_fence_after();
-            const int quad = warp & 3;
-            const int m = m0 + quad * 32 + lane;
+            const int half = gw >> 2;
             const bool m_ok = m < g.M;
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
-            const bool to_partial = g.split_k > 1;
-            float bias_m = 0.f;
-            if (!to_partial && g.bias_mode == 1 && m_ok) bias_m = __ldg(g.bias + m);
-            float* yrow;
-            long long ns;
-            if (to_partial) {
-                yrow = g.partial + (((long long)split * g.batch + bz) * g.M + m) * (long long)g.N;
-                ns = 1;
-            } else {
-                yrow = g.y + (long long)bz * g.y_bs + (long long)m * g.y_ms;
-                ns = g.y_ns;
+            const bool split_mode = g.split_k > 1;
+            // split-K workspace [split][batch][N][M]: a column of the tile is contiguous across lanes
+            const long long per_split = (long long)g.batch * g.M * (long long)g.N;
+            float* pcol = g.partial + (long long)bz * g.M * (long long)g.N + m;
+            if (split_mode) {
+                // 1. park this split's partial tile in the workspace
+                float* pmine = pcol + (long long)split * per_split;
+#pragma unroll 1
+                for (int c0 = half * 32; c0 < g.tile_n; c0 += 64) {
+                    uint32_t r[32];
+                    tmem_ld32(t_row + (uint32_t)c0, r);
+                    tmem_wait_ld();
+                    const int nb = n0 + c0;
+                    const int cnt = min(g.N - nb, g.tile_n - c0);
+                    if (!m_ok || cnt <= 0) continue;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < cnt) __stcg(pmine + (long long)(nb + j) * g.M, __uint_as_float(r[j]));
+                }
+                // 2. the split that arrives last at this tile's counter reduces all of them, in split order
+                __threadfence();
+                asm volatile("bar.sync 1, %0;" ::"n"(kGatherThreads) : "memory");
+                if (threadIdx.x == 64) {
+                    unsigned* ctr = g.counters + (size_t)bz * gridDim.x + blockIdx.x;
+                    const unsigned old = atomicAdd(ctr, 1u);
+                    const int last = old == (unsigned)(g.split_k - 1);
+                    if (last) *ctr = 0u;                 // all splits have arrived: ready for the next launch
+                    last_split_flag = last;
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(kGatherThreads) : "memory");
             }
-            const float* rrow = (!to_partial && g.residual) ? g.residual + (long long)bz * g.y_bs + (long long)m * g.y_ms : nullptr;
-            const bool vec = to_partial ? ((g.N & 3) == 0) : (g.vec_store != 0);
-            for (int c0 = 0; c0 < g.tile_n; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld16(t_row + (uint32_t)c0, r);
-                tmem_wait_ld();
-                if (!m_ok) continue;
-                const int nb = n0 + c0;
-                if (nb >= g.N) continue;
-                float v[16];
+            const bool finish = !split_mode || (*(volatile int*)&last_split_flag != 0);
+            if (finish) {
+                if (split_mode) __threadfence();
+                EpiArgs e;
+                e.ybase = g.y + (long long)bz * g.y_bs;
+                e.rbase = g.residual ? g.residual + (long long)bz * g.y_bs : nullptr;
+                e.y_ms = g.y_ms; e.y_ns = g.y_ns; e.M = g.M;
+                e.lo = g.act == TT_ACT_NONE || g.act == TT_ACT_GELU_ERF ? -INFINITY : 0.f;
+                e.hi = g.act == TT_ACT_RELU6 ? 6.f : INFINITY;
+                e.gelu = g.act == TT_ACT_GELU_ERF;
+                e.vec = (g.vec_store & 1) != 0;
+                const bool transposed = g.y_ns == 1 && g.y_ms != 1;
+                const uint32_t stg = tiles_base + (uint32_t)gw * (uint32_t)kStageBytesPerWarp;   // pipeline buffers are idle now
+                const int m_first = m0 + quad * 32;
+                uint32_t r[32];
+                int c0 = half * 32;
+                if (!split_mode && c0 < g.tile_n) tmem_ld32(t_row + (uint32_t)c0, r);
+#pragma unroll 1
+                for (; c0 < g.tile_n; c0 += 64) {
+                    float v[32];
+                    const int nb = n0 + c0;
+                    const int cnt = min(g.N - nb, g.tile_n - c0);
+                    if (!split_mode) {
+                        // read-out is software-pipelined: the next block's tensor-memory load is in flight while
+                        // this block is biased, activated and stored
+                        tmem_wait_ld();
+                        if (threadIdx.x == 64 && c0 == 0) TT_STAMP(7);
 #pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
-                if (!to_partial) {
+                        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+                        if (c0 + 64 < g.tile_n) tmem_ld32(t_row + (uint32_t)(c0 + 64), r);
+                    } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int n = nb + j;
-                        if (n < g.N) {
-                            float t = v[j] + bias_m;
-                            if (g.bias_mode == 2) t += __ldg(g.bias + n);
-                            if (rrow) t += __ldg(rrow + (long long)n * ns);
-                            v[j] = apply_act(t, g.act);
+                        for (int j = 0; j < 32; ++j) v[j] = 0.f;
+                        if (m_ok && cnt > 0) {
+#pragma unroll 2
+                            for (int sp = 0; sp < g.split_k; ++sp) {
+                                const float* ps = pcol + (long long)sp * per_split + (long long)nb * g.M;
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    if (j < cnt) v[j] += __ldcg(ps + (long long)j * g.M);
+                            }
                         }
                     }
-                }
-                if (vec && nb + 16 <= g.N) {
+                    if (cnt <= 0) continue;              // warp-uniform
+                    if (g.bias_mode == 1) {
 #pragma unroll
-                    for (int j = 0; j < 16; j += 4)
-                        *reinterpret_cast<float4*>(yrow + nb + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                } else {
+                        for (int j = 0; j < 32; ++j) v[j] += bias_row;
+                    } else if (g.bias_mode == 2) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (nb + j < g.N) yrow[(long long)(nb + j) * ns] = v[j];
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 b = *reinterpret_cast<const float4*>(s_bias + c0 + j);
+                            v[j] += b.x; v[j + 1] += b.y; v[j + 2] += b.z; v[j + 3] += b.w;
+                        }
+                    }
+                    // full blocks take the unguarded path (16-byte accesses need the aligned layout when transposed)
+                    const bool full = cnt >= 32 && m_first + 32 <= g.M && (e.vec || !transposed);
+                    if (e.rbase == nullptr) {
+                        // no residual: activate here, once, outside the store loops
+                        if (e.gelu) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = 0.5f * v[j] * (1.f + erff(v[j] * 0.70710678118654752440f));
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = fminf(fmaxf(v[j], e.lo), e.hi);
+                        }
+                        if (full) epilogue_block<true, false>(v, e, m_first, nb, cnt, stg, lane, transposed);
+                        else epilogue_block<false, false>(v, e, m_first, nb, cnt, stg, lane, transposed);
+                    } else {
+                        if (full) epilogue_block<true, true>(v, e, m_first, nb, cnt, stg, lane, transposed);
+                        else epilogue_block<false, true>(v, e, m_first, nb, cnt, stg, lane, transposed);
+                    }
+                    if (threadIdx.x == 64 && c0 == 0) TT_STAMP(8);
                 }
             }
         }
     }
+    if (threadIdx.x == 64) TT_STAMP(5);
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -399,45 +713,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         tc_fence_after();
         tmem_dealloc(tmem_base, g.tmem_cols);
     }
-}
-
-// ------------------------------------------------------------------------------------------------------------
-// Split-K reduction + bias/activation epilogue (fixed summation order: bit-identical from run to run).
-// ------------------------------------------------------------------------------------------------------------
-__global__ void tt_splitk_reduce_kernel(const ReduceArgs a) {
-    const long long per = (long long)a.batch * a.M * a.N;
-    const int step = a.vec ? 4 : 1;
-    const long long total = per / step;
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-        const long long e = i * step;
-        const int n = (int)(e % a.N);
-        const long long bm = e / a.N;
-        const int m = (int)(bm % a.M);
-        const int b = (int)(bm / a.M);
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int s = 0; s < a.split_k; ++s) {
-            const float* p = a.partial + (long long)s * per + e;
-            if (a.vec) {
-                const float4 t = __ldg(reinterpret_cast<const float4*>(p));
-                acc[0] += t.x; acc[1] += t.y; acc[2] += t.z; acc[3] += t.w;
-            } else {
-                acc[0] += __ldg(p);
-            }
-        }
-        const long long ybase = (long long)b * a.y_bs + (long long)m * a.y_ms;
-        const float bm_ = a.bias_mode == 1 ? __ldg(a.bias + m) : 0.f;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            if (j < step) {
-                float t = acc[j] + bm_;
-                if (a.bias_mode == 2) t += __ldg(a.bias + n + j);
-                if (a.residual) t += __ldg(a.residual + ybase + (long long)(n + j) * a.y_ns);
-                acc[j] = apply_act(t, a.act);
-            }
-        }
-        if (a.vec) *reinterpret_cast<float4*>(a.y + ybase + n) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-        else a.y[ybase + (long long)n * a.y_ns] = acc[0];
-    }
+    if (threadIdx.x == 0) TT_STAMP(6);
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -552,8 +828,7 @@ __global__ void tt_softmax_kernel(const RowArgs a) {
 // ------------------------------------------------------------------------------------------------------------
 // Launchers (called from tt_device.cu)
 // ------------------------------------------------------------------------------------------------------------
-cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const ReduceArgs& red, const void* tmap_a,
-                        const void* tmap_b, cudaStream_t st) {
+cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, cudaStream_t st) {
     static int attr_set_for = -1;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -567,16 +842,7 @@ cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const ReduceA
     memcpy(&tb, tmap_b, sizeof tb);
     dim3 grid(I.grid_x, I.grid_y, I.grid_z);
     tt_gemm_tc_kernel<<<grid, kGemmThreads, I.smem_bytes, st>>>(ta, tb, g);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    if (g.split_k > 1) {
-        const long long total = (long long)red.batch * red.M * red.N / (red.vec ? 4 : 1);
-        long long blocks = (total + 255) / 256;
-        if (blocks > 148 * 8) blocks = 148 * 8;
-        tt_splitk_reduce_kernel<<<(int)blocks, 256, 0, st>>>(red);
-        e = cudaGetLastError();
-    }
-    return e;
+    return cudaGetLastError();
 }
 
 cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st) {
