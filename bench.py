@@ -243,8 +243,10 @@ def main():
     torch.cuda.synchronize()
     sampler = ClockSampler(local_rank)
     sampler.start()
+    torch.cuda.nvtx.range_push("tt_timed_region")      # lets a profiler restrict itself to the timed launches
     ms_total = timed_steps(args.steps, graph.replay)
     torch.cuda.synchronize()
+    torch.cuda.nvtx.range_pop()
     replicas.barrier()
     sampler.stop_flag = True
     sampler.join(timeout=2)

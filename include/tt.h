@@ -93,9 +93,11 @@ typedef struct tt_shapes {
  *   cache buffer / ComputeAt -> the accumulator lives in tensor memory and the bias/activation run on read-out;
  *                               `stages` shared-memory buffers decouple loading from the multiply
  *   Vectorize -> vec_width;   Unroll -> unroll / items_per_thread
- * GEMM_TC uses tile_m, tile_n, tile_k, stages, split_k, raster, mma_m_axis.
+ * GEMM_TC uses tile_m, tile_n, tile_k, stages, split_k, raster, mma_m_axis, slab_tiles.
  * DW_SIMT uses tile_m (channels per CTA), block_y x block_x (output rows x columns per CTA tile),
- *         items_per_thread (consecutive outputs along the width per thread), vec_width, threads.
+ *         items_per_thread (consecutive outputs along the width per thread), vec_width, threads, and unroll:
+ *         0 = shared-memory staged kernel; 1, 2, 4 = register-window kernel with that many output rows per thread
+ *         (3x3 and 5x5 filters with "same" padding, stride 1 or 2; strips of 4 columns).
  * ROW_SIMT uses block_x (threads cooperating on one row: 1..32, power of two), block_y (rows per CTA), vec_width.
  * origin_* say which kernel the record was tuned on (its "native" kernel, Section 3). */
 typedef struct tt_schedule_record {
@@ -108,7 +110,9 @@ typedef struct tt_schedule_record {
     int32_t block_x, block_y, items_per_thread, vec_width, unroll, threads;
     int32_t mma_m_axis;    /* GEMM_TC: which output axis rides the 128 accumulator rows: 0 library's choice by shape,
                               1 output rows (conv filters, dense/bmm rows m), 2 output columns (conv pixels, nn) */
-    int32_t reserved[3];
+    int32_t slab_tiles;    /* GEMM_TC, conv2d only: reduction tiles served by one staging of the input rows in shared
+                              memory (the cache buffer of the im2col operand); 0 = as many as fit */
+    int32_t reserved[2];
 } tt_schedule_record;
 
 typedef struct tt_tensors {
@@ -137,7 +141,7 @@ typedef struct tt_apply_info {
 } tt_apply_info;
 
 enum { TT_CHG_TILE_M = 1, TT_CHG_TILE_N = 2, TT_CHG_TILE_K = 4, TT_CHG_STAGES = 8, TT_CHG_SPLIT_K = 16,
-       TT_CHG_VEC = 32, TT_CHG_BLOCK = 64, TT_CHG_ITEMS = 128 };
+       TT_CHG_VEC = 32, TT_CHG_BLOCK = 64, TT_CHG_ITEMS = 128, TT_CHG_SLAB = 256 };
 
 /* Validity modes for mapping a record onto another shape (Section 4.1).
  *   TT_MODE_LEGALISE  reformulate: clamp/round tile sizes to the new extents and the hardware's legal set,

@@ -157,6 +157,7 @@ tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
         d.bias = w->sh.has_bias ? static_cast<const float*>(t->bias) : nullptr;
         d.y = static_cast<float*>(t->y);
         if ((reinterpret_cast<uintptr_t>(t->y) & 15u) != 0) d.vec = 1;
+        if ((reinterpret_cast<uintptr_t>(t->x) & 15u) != 0) d.vec_in = 0;
         e = launch_dw(p.info, d, st);
     } else {
         RowArgs r = p.row;
@@ -423,12 +424,13 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
     tt_schedule_record base;
     tt_default_schedule(w, &base);
     std::vector<tt_schedule_record> cand;
-    auto push = [&](const tt_schedule_record& r) {
+    auto push = [&](const tt_schedule_record& r) -> bool {
         // keep only records that are legal as written: a record that needs rounding duplicates another candidate
         tt_apply_info info;
-        if (tt_schedule_check(w, &r, TT_MODE_LEGALISE, 0, &info) != TT_OK) return;
-        if (info.changed & ~TT_CHG_TILE_M) return;
+        if (tt_schedule_check(w, &r, TT_MODE_LEGALISE, 0, &info) != TT_OK) return false;
+        if (info.changed & ~TT_CHG_TILE_M) return false;
         cand.push_back(info.legal);
+        return true;
     };
     const bool full = level > 0;
     if (w->family == TT_FAMILY_GEMM_TC) {
@@ -450,7 +452,20 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
         for (int tc : tcs) for (int by : bys) for (int bx : bxs) for (int it : its) for (int vw : {1, 4}) for (int th : {128, 256}) {
             tt_schedule_record r = base;
             r.tile_m = tc; r.block_y = by; r.block_x = bx; r.items_per_thread = it; r.vec_width = vw; r.threads = th;
+            r.unroll = 0;                               // staged kernel
             push(r);
+        }
+        // register-window kernel: rows per thread x CTA tile
+        const std::vector<int> wys = full ? std::vector<int>{1, 2, 4, 7, 8, 14, 16, 28, 56} : std::vector<int>{4, 8, 16};
+        const std::vector<int> wxs = full ? std::vector<int>{8, 16, 28, 32, 56, 64, 112} : std::vector<int>{16, 32, 64, 112};
+        for (int ro : {1, 2, 4}) for (int tc : tcs) for (int by : wys) for (int bx : wxs) for (int th : {64, 128, 256}) {
+            tt_schedule_record r = base;
+            r.tile_m = tc; r.block_y = by; r.block_x = bx; r.items_per_thread = 4; r.threads = th;
+            r.unroll = ro;
+            for (int vw : {4, 2, 1}) {                  // the widest store the output rows allow
+                r.vec_width = vw;
+                if (push(r)) break;
+            }
         }
     } else {
         for (int bx : {4, 8, 16, 32}) for (int by : {1, 2, 4, 8, 16}) for (int vw : {1, 2, 4}) {
@@ -491,3 +506,4 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
 }
 
 }  // extern "C"
+

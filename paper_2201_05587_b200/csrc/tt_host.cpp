@@ -78,6 +78,7 @@ size_t tensor_elems(const tt_workload* w, int which) {
 // ---- legalisation -------------------------------------------------------------------------------------------
 
 static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* rec, int mode, Plan* plan) {
+    tt_apply_info& I = plan->info;
     tt_schedule_record L = *rec;
     int changed = 0;
     const bool strict = mode == TT_MODE_STRICT;
@@ -123,25 +124,80 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     sk = (k_tiles + per_split - 1) / per_split;          // every split owns at least one reduction tile
     if (sk != rec->split_k) changed |= TT_CHG_SPLIT_K;
     L.split_k = sk;
+    // buffers beyond the reduction tiles of one CTA would never be filled
+    if (st > per_split) { st = per_split; changed |= TT_CHG_STAGES; L.stages = st; }
     if (strict && (changed & ~TT_CHG_TILE_M)) return TT_ERR_INVALID_SCHEDULE;
 
     const int atom_k = std::min(tk, 32), n_atoms = tk / atom_k, row_bytes = atom_k * 4;
     const unsigned a_stage = (unsigned)n_atoms * kHwTileM * row_bytes;
     const unsigned b_stage = (unsigned)n_atoms * tn * row_bytes;
-    // pipeline buffers, reused by the epilogue as a 32 x 36-float staging area per warp; then the im2col k-table
-    // (one word per reduction index of a CTA's K range); 1 KB of alignment slack
+    // Shared memory: pipeline buffers (reused by the epilogue as a 32 x 36-float staging area per warp), then for
+    // conv2d the k-table (one word per reduction index of a CTA's K range) and the slab of input rows from which
+    // the im2col operand is expanded; 1 KB of alignment slack.
+    // A slab row is an image row followed by `gap` zeros (the left/right padding of neighbouring rows share them).
+    // Per channel the slab holds, for each of the output rows a tile can span, the input rows its filter rows
+    // touch: consecutive rows when stride <= filter height, else `r` rows per output row.  A chunk holds the
+    // channels that `slab_tiles` consecutive reduction tiles touch; two buffers when there are several chunks.
+    const bool conv = w->op == TT_OP_CONV2D;
+    const long long ktab = conv ? (((long long)per_split * tk * 4 + 15) / 16) * 16 : 0;
+    int sl_tiles = 0, sl_nbuf = 0, sl_wp = 0, sl_gap = 0, sl_chpitch = 0, sl_in_rows = 0, sl_rstep = 1;
+    long long sl_buf_bytes = 0, chp = 0;
+    const int RS = conv ? s.r * s.s : 1;
+    if (conv) {
+        if (rec->slab_tiles < 0) return TT_ERR_INVALID_SCHEDULE;
+        if (strict && rec->slab_tiles > per_split) return TT_ERR_INVALID_SCHEDULE;
+        const int pix_rows = swap ? kHwTileM : tn;       // output pixels per tile of the im2col operand
+        const int out_rows = std::min(w->P, (pix_rows + 2 * w->Q - 2) / w->Q);
+        sl_rstep = std::min(s.stride_h, s.r);
+        sl_in_rows = s.stride_h <= s.r ? (out_rows - 1) * s.stride_h + s.r : out_rows * s.r;
+        sl_gap = round_up(std::max(1, std::max(s.pad_w, s.s - 1 - s.pad_w)), 4);
+        sl_wp = s.w + sl_gap;
+        chp = round_up(sl_in_rows * sl_wp, 4);
+        if (chp * (long long)s.c >= (1ll << 28) || s.w > 4095 || sl_in_rows > 4095) return TT_ERR_RESOURCE;
+        sl_chpitch = (int)chp;
+    }
+    auto chunk_bytes = [&](long long tiles) {
+        const long long ch = std::min<long long>(s.c, (tiles * tk + RS - 2) / RS + 1);
+        return ((ch * chp + sl_gap + 4) * 4 + 15) / 16 * 16;
+    };
+    long long smem = 0;
+    for (;;) {
+        const long long pipe_try = std::max<long long>((long long)st * (a_stage + b_stage), (long long)kGatherWarps * 32 * 36 * 4);
+        long long slab_total = 0;
+        bool fits = true;
+        if (conv) {
+            const long long budget = kDynSmemLimit - 1024 - pipe_try - ktab;
+            // largest chunk not above the request that fits (one buffer if it covers the CTA's whole K range)
+            int t = rec->slab_tiles == 0 ? per_split : std::min(rec->slab_tiles, per_split);
+            while (t >= 1 && (t >= per_split ? 1 : 2) * chunk_bytes(t) > budget) --t;
+            fits = t >= 1;
+            sl_tiles = std::max(t, 1);
+            sl_nbuf = sl_tiles >= per_split ? 1 : 2;
+            sl_buf_bytes = chunk_bytes(sl_tiles);
+            slab_total = sl_nbuf * sl_buf_bytes;
+        }
+        smem = pipe_try + ktab + slab_total + 1024;
+        if (fits && smem <= kDynSmemLimit) break;
+        // reformulate: a shallower pipeline leaves room (never in strict mode, never below one buffer)
+        if (strict || st <= 1) break;
+        --st;
+        changed |= TT_CHG_STAGES;
+    }
+    L.stages = st;
     const long long pipe = std::max<long long>((long long)st * (a_stage + b_stage), (long long)kGatherWarps * 32 * 36 * 4);
-    const long long ktab = w->op == TT_OP_CONV2D ? (long long)per_split * tk * 4 : 0;
-    const long long smem = pipe + ktab + 1024;
-    if (w->op == TT_OP_CONV2D) {
-        // table packing: element offsets below 2^26, tap indices below 63
-        if ((long long)s.c * s.h * s.w >= (1ll << 26) || s.r * s.s > 63) return TT_ERR_RESOURCE;
+    if (conv) {
+        if (rec->slab_tiles != 0 && sl_tiles != rec->slab_tiles) {
+            if (strict) return TT_ERR_INVALID_SCHEDULE;
+            changed |= TT_CHG_SLAB;
+        }
+        L.slab_tiles = rec->slab_tiles == 0 ? 0 : sl_tiles;
+    } else {
+        L.slab_tiles = 0;
     }
     int tmem_cols = std::max(32, pow2_ceil(tn));
     const int tiles_m = (M + kHwTileM - 1) / kHwTileM, tiles_n = (N + tn - 1) / tn;
     if ((long long)tiles_m * tiles_n > 0x7fffffffLL || sk > 65535 || B > 65535) return TT_ERR_RESOURCE;
 
-    tt_apply_info& I = plan->info;
     I = tt_apply_info{};
     I.legal = L;
     I.changed = changed;
@@ -165,6 +221,17 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     g.swz_mask = row_bytes == 128 ? 7 : (row_bytes == 64 ? 3 : 1);
     g.a_stage_bytes = a_stage; g.b_stage_bytes = b_stage;
     g.ktab_off = (unsigned)pipe;
+    g.slab_off = (unsigned)(pipe + ktab);
+    g.slab_buf_bytes = (unsigned)sl_buf_bytes; g.slab_nbuf = sl_nbuf; g.slab_tiles = sl_tiles;
+    g.slab_wp = sl_wp; g.slab_gap = sl_gap; g.slab_chpitch = sl_chpitch; g.slab_in_rows = sl_in_rows;
+    g.slab_rstep = sl_rstep;
+    g.magic_rstep = sl_rstep > 1 ? (unsigned)((0x100000000ull + sl_rstep - 1) / sl_rstep) : 0u;
+    g.slab_vec16 = (s.w % 4) == 0;
+    {
+        const unsigned wpieces = (unsigned)(g.slab_vec16 ? s.w / 4 : s.w);
+        g.magic_wpieces = wpieces > 1 ? (unsigned)((0x100000000ull + wpieces - 1) / wpieces) : 0u;
+        g.magic_in_rows = sl_in_rows > 1 ? (unsigned)((0x100000000ull + sl_in_rows - 1) / sl_in_rows) : 0u;
+    }
     g.tmem_cols = (unsigned)tmem_cols;
     // Instruction descriptor, kind::tf32: D = F32 (bits 4-5 = 1), A and B = TF32 (bits 7-9, 10-12 = 2), both
     // K-major (bits 15, 16 = 0), N >> 3 at bits 17-22, M >> 4 at bits 24-28.
@@ -222,6 +289,18 @@ static tt_status legalise_dw(const tt_workload* w, const tt_schedule_record* rec
     while (vec > 1 && (w->Q % vec) != 0) vec >>= 1;        // rows of y must stay vector-aligned
     int items = std::min(8, pow2_floor(rec->items_per_thread));
     items = std::max(items, vec);
+    // unroll >= 1 asks for the register-window kernel (that many output rows per thread: 1, 2 or 4), which exists
+    // for square 3x3 / 5x5 filters with "same" padding and stride 1 or 2 and works on strips of 4 columns;
+    // unroll == 0, or any other filter, takes the shared-memory staged kernel
+    const bool window_ok = s.r == s.s && (s.r == 3 || s.r == 5) && s.stride_h == s.stride_w &&
+                           (s.stride_h == 1 || s.stride_h == 2) && s.pad_h == s.r / 2 && s.pad_w == s.r / 2;
+    int window_rows = 0;
+    if (rec->unroll < 0) return TT_ERR_INVALID_SCHEDULE;
+    if (rec->unroll >= 1 && window_ok) {
+        window_rows = rec->unroll >= 4 ? 4 : (rec->unroll >= 2 ? 2 : 1);
+        items = 4;
+    }
+    L.unroll = window_rows;
     int bx = std::min(rec->block_x, round_up(w->Q, items));
     bx = round_up(bx, items);
     if (bx != rec->block_x || L.block_y != rec->block_y) changed |= TT_CHG_BLOCK;
@@ -230,7 +309,7 @@ static tt_status legalise_dw(const tt_workload* w, const tt_schedule_record* rec
     L.items_per_thread = items;
     if (vec != rec->vec_width) changed |= TT_CHG_VEC;
     L.vec_width = vec;
-    int th = std::min(1024, std::max(32, round_up(rec->threads, 32)));
+    int th = std::min(window_rows ? 256 : 1024, std::max(32, round_up(rec->threads, 32)));
     if (th != rec->threads) changed |= TT_CHG_BLOCK;
     L.threads = th;
     if (strict && changed) return TT_ERR_INVALID_SCHEDULE;
@@ -246,7 +325,9 @@ static tt_status legalise_dw(const tt_workload* w, const tt_schedule_record* rec
     d.tiles_c = (s.c + d.tile_c - 1) / d.tile_c;
     d.tiles_h = (w->P + d.tile_h - 1) / d.tile_h;
     d.tiles_w = (w->Q + d.tile_w - 1) / d.tile_w;
-    const long long smem = (long long)d.tile_c * ((long long)d.in_h * d.in_w + d.R * d.S + 1) * 4;
+    d.window_rows = window_rows;
+    d.vec_in = (s.w % 4) == 0;
+    const long long smem = window_rows ? 0 : (long long)d.tile_c * ((long long)d.in_h * d.in_w + d.R * d.S + 1) * 4;
     tt_apply_info& I = plan->info;
     I = tt_apply_info{};
     I.legal = L; I.changed = changed;
@@ -432,7 +513,7 @@ tt_status tt_default_schedule(const tt_workload* w, tt_schedule_record* out) {
     // One generic, shape-blind record per family: the counterpart of a compiler's default schedule.
     r.tile_m = 128; r.tile_n = 128; r.tile_k = 32; r.stages = 4; r.split_k = 1; r.raster = 0;
     r.block_x = 32; r.block_y = 4; r.items_per_thread = 1; r.vec_width = 1; r.unroll = 1; r.threads = 128;
-    if (w->family == TT_FAMILY_DW_SIMT) { r.tile_m = 1; r.block_x = 32; r.block_y = 8; }
+    if (w->family == TT_FAMILY_DW_SIMT) { r.tile_m = 1; r.block_x = 32; r.block_y = 8; r.items_per_thread = 4; r.unroll = 2; }
     if (w->family == TT_FAMILY_ROW_SIMT) { r.block_x = 32; r.block_y = 4; }
     *out = r;
     return TT_OK;

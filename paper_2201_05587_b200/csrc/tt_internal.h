@@ -45,6 +45,16 @@ struct GemmArgs {
     unsigned a_stage_bytes, b_stage_bytes, tx_bytes;
     unsigned ktab_off;                          // im2col k-table: byte offset from the aligned tile base
     int vec_store;                              // bit 0: y rows allow aligned float4 stores; bit 1: so does bias
+    // im2col slab: the input rows a CTA's pixels need, staged once in shared memory per chunk of reduction tiles
+    unsigned slab_off;                          // byte offset of the first slab buffer from the aligned tile base
+    unsigned slab_buf_bytes;                    // bytes per slab buffer (multiple of 16)
+    int slab_nbuf;                              // 1: the CTA's whole K range in one chunk; 2: double-buffered chunks
+    int slab_tiles;                             // reduction tiles per chunk
+    int slab_wp, slab_gap, slab_chpitch;        // row pitch (W + gap), zero gap, channel pitch, in elements
+    int slab_in_rows;                           // slab rows per channel (the most a tile can need)
+    int slab_rstep;                             // slab rows per output row: min(stride_h, r)
+    int slab_vec16;                             // rows copied 16 bytes at a time (W % 4 == 0 and x aligned)
+    unsigned magic_wpieces, magic_in_rows, magic_rstep;      // ceil(2^32 / d) for the exact small-range divisions of the slab loader
 };
 
 struct DwArgs {
@@ -52,6 +62,8 @@ struct DwArgs {
     int N, C, H, W, R, S, P, Q, sh, sw, ph, pw, act;
     int tile_c, tile_h, tile_w, in_h, in_w, items, vec;
     int tiles_c, tiles_h, tiles_w;
+    int window_rows;   // > 0: register-window kernel with this many output rows per thread; 0: staged kernel
+    int vec_in;        // input rows start on 16-byte boundaries (W % 4 == 0 and x aligned)
 };
 
 struct RowArgs {

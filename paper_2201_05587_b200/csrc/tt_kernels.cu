@@ -163,32 +163,145 @@ __device__ __forceinline__ uint32_t swz_off(uint32_t row, uint32_t kbyte, uint32
 }
 
 // ------------------------------------------------------------------------------------------------------------
-// Gather producers.  The 8 gather warps form 1, 2 or 4 groups; group g fills pipeline stages g, g + groups, ...
-// so that the global-memory latency of one stage overlaps the other groups' stages.  Within a stage a warp
-// takes (32-row block, 4-wide k chunk) tasks: lanes walk rows (coalesced loads), each lane assembles four
-// consecutive reduction indices of its row in registers and writes one 16-byte chunk into the swizzled K-major
-// tile.  Loads of four tasks are issued before the first store, so 16 loads per lane are in flight.
+// Operand producers that do not go through TMA.
+//
+// im2col operand of conv2d (rows = output pixels, k = (c, r, s), gathered from an NCHW image).  The input rows a
+// CTA's pixels need are staged ONCE per chunk of reduction tiles in a shared-memory slab by cp.async: per
+// channel, the rows [ih_lo, ih_lo + in_rows) one after the other, each followed by `gap` zeros, so that the
+// left/right padding of a row and rows outside the image read as zero without any test.  A pipeline stage is
+// then expanded from the slab: element (pixel, k) sits at rowoff[pixel] + koff[k], two table look-ups, and a
+// lane assembles four consecutive k of its pixel and writes one 16-byte chunk of the swizzled K-major tile.
+// Global memory is read once per CTA (not once per filter tap), and no load of the main loop waits on DRAM or L2.
+//
+// Strided views (the NN operand of batch_matmul) and K-contiguous operands with K % 4 != 0 are gathered from
+// global memory directly: the 8 gather warps form 1, 2 or 4 groups, group g fills stages g, g + groups, ...
 // ------------------------------------------------------------------------------------------------------------
-struct Im2col { int C, H, W, R, S, Q, sh, sw, ph, pw; };
-
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, float a, float b, float c, float d) {
     asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 __device__ __forceinline__ void st_shared_f32(uint32_t addr, float a) {
     asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(a) : "memory");
 }
+__device__ __forceinline__ void st_shared_u32(uint32_t addr, uint32_t a) {
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(a) : "memory");
+}
+__device__ __forceinline__ float ld_shared_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_shared_u32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint4 ld_shared_v4u(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// One stage of an operand whose rows are contiguous across lanes: IM2COL (rows = output pixels of an NCHW
-// image, k = (c, r, s)) or GATHER_ROWS (strided view with unit row stride).
-// IM2COL reads two shared-memory tables built once per CTA: ktab[k] = (element offset c*H*W + r*W + s) << 6 |
-// tap index r*S + s (63 for k beyond K), and rowinfo[row] = {ih0*W + iw0, in-bounds tap mask low, high, -} of the
-// row's output pixel (mask 0 for rows past the extent), so the inner loop holds neither a division nor a
-// bounds comparison: one table word per k (warp-uniform), one mask bit test and one add per element.
-template <int MODE>
+// All gather threads meet and learn whether every one of them is still healthy (named barrier 1).
+__device__ __forceinline__ bool gather_vote(bool ok) {
+    uint32_t all;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(all) : "r"((uint32_t)ok), "n"(kGatherThreads) : "memory");
+    return all != 0u;
+}
+
+// n / d for the small ranges of the slab loader: magic = ceil(2^32 / d) is exact while n * d < 2^32; d == 1 has magic 0.
+__device__ __forceinline__ int small_div(int n, unsigned magic) { return magic ? (int)__umulhi((unsigned)n, magic) : n; }
+
+// Stage the input rows of channels [c_first, c_first + nch) that this CTA's pixels need into one slab buffer.
+// Pieces (16 bytes when the rows allow it, else 4) are dealt round-robin to the gather threads; rows outside the
+// image or beyond the CTA's own range are skipped and keep the zeros written at kernel start.
+__device__ __forceinline__ void slab_load_chunk(const GemmArgs& g, const float* __restrict__ img, uint32_t buf, int c_first,
+                                                int nch, int ih_lo, int in_rows_cta, bool vec16, int gt) {
+    const int wpieces = vec16 ? g.W >> 2 : g.W;
+    const bool use_magic = vec16 == (g.slab_vec16 != 0);  // the host's magic number is for its own piece width
+    const int total = nch * g.slab_in_rows * wpieces;
+    for (int idx = gt; idx < total; idx += kGatherThreads) {
+        const int t1 = use_magic ? small_div(idx, g.magic_wpieces) : idx / wpieces;
+        const int pc = idx - t1 * wpieces;
+        const int cl = small_div(t1, g.magic_in_rows);
+        const int rl = t1 - cl * g.slab_in_rows;
+        // slab row -> image row: consecutive rows when stride <= filter height, else r rows per output row
+        int ih = ih_lo + rl;
+        if (g.sh > g.R) {
+            const int po = small_div(rl, g.magic_rstep);
+            ih = ih_lo + po * g.sh + (rl - po * g.slab_rstep);
+        }
+        if (rl >= in_rows_cta || (unsigned)ih >= (unsigned)g.H) continue;
+        const int col = vec16 ? pc << 2 : pc;
+        const float* src = img + ((long long)(c_first + cl) * g.H + ih) * g.W + col;
+        const uint32_t dst = buf + 4u * (uint32_t)(cl * g.slab_chpitch + rl * g.slab_wp + g.slab_gap + col);
+        if (vec16) cp_async_16(dst, src); else cp_async_4(dst, src);
+    }
+}
+
+// Expand one pipeline stage of the im2col operand from the slab.  A warp takes (32-row block, 4-wide k chunk)
+// tasks gw, gw + 8, ...; the loads of four tasks are issued before the first store.
+// rowoff_smem: per tile row, the byte offset of its pixel's window origin inside a channel of the slab;
+// ktab_smem: per reduction index of this tile, the byte offset of (channel, tap) relative to that origin.
+__device__ __forceinline__ void expand_stage(uint32_t tile_smem, int rows, uint32_t slab, uint32_t rowoff_smem,
+                                             uint32_t ktab_smem, int tile_k, int atom_k, int row_bytes, int swz_mask,
+                                             int gw, int lane) {
+    const int atom_shift = atom_k == 32 ? 5 : (atom_k == 16 ? 4 : 3);
+    const int shift = row_bytes == 128 ? 0 : (row_bytes == 64 ? 1 : 2);
+    const uint32_t atom_bytes = (uint32_t)rows * (uint32_t)row_bytes;
+    const int n_rb = (rows + 31) >> 5;
+    const int n_tasks = n_rb * (tile_k >> 2);
+    const uint32_t inv_rb = (65536u + (uint32_t)n_rb - 1u) / (uint32_t)n_rb;     // t / n_rb == (t * inv_rb) >> 16 for small t
+    constexpr int kBatch = 4;
+    for (int t0 = gw; t0 < n_tasks; t0 += kGatherWarps * kBatch) {
+        float val[kBatch][4];
+        uint32_t dst[kBatch];
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+            const int t = t0 + b * kGatherWarps;
+            const bool live = t < n_tasks;               // warp-uniform
+            const int tt = live ? t : 0;
+            const int ci = (int)(((uint32_t)tt * inv_rb) >> 16);
+            const int rb = tt - ci * n_rb;
+            const int kk = ci << 2;
+            const int row = rb * 32 + lane;
+            const bool in_tile = live && row < rows;
+            dst[b] = in_tile ? tile_smem + (uint32_t)(kk >> atom_shift) * atom_bytes + (uint32_t)row * (uint32_t)row_bytes +
+                                   ((uint32_t)((kk & (atom_k - 1)) << 2) ^ ((uint32_t)((row >> shift) & swz_mask) << 4))
+                             : 0xffffffffu;
+            const uint32_t origin = slab + ld_shared_u32(rowoff_smem + 4u * (uint32_t)(row < rows ? row : rows - 1));
+            const uint4 e = ld_shared_v4u(ktab_smem + 16u * (uint32_t)ci);       // same address in every lane
+            val[b][0] = ld_shared_f32(origin + e.x);
+            val[b][1] = ld_shared_f32(origin + e.y);
+            val[b][2] = ld_shared_f32(origin + e.z);
+            val[b][3] = ld_shared_f32(origin + e.w);
+        }
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b)
+            if (dst[b] != 0xffffffffu) st_shared_v4(dst[b], val[b][0], val[b][1], val[b][2], val[b][3]);
+    }
+}
+
+// One stage of a strided view whose rows are contiguous across lanes (unit row stride): lanes walk rows
+// (coalesced loads), each lane assembles four consecutive reduction indices of its row in registers and writes
+// one 16-byte chunk into the swizzled K-major tile.  Loads of eight tasks are issued before the first store.
 __device__ __forceinline__ void gather_rows_stage(uint32_t tile_smem, int rows, const float* __restrict__ src,
-                                                  long long rs, long long ks, const int4* rowinfo, const uint32_t* ktab,
-                                                  int row0, int row_extent, int k0, int K, int tile_k, int atom_k,
-                                                  int row_bytes, int swz_mask, int wig, int wpg, int lane) {
+                                                  long long rs, long long ks, int row0, int row_extent, int k0, int K,
+                                                  int tile_k, int atom_k, int row_bytes, int swz_mask, int wig, int wpg,
+                                                  int lane) {
     const int atom_shift = atom_k == 32 ? 5 : (atom_k == 16 ? 4 : 3);
     const int shift = row_bytes == 128 ? 0 : (row_bytes == 64 ? 1 : 2);
     const uint32_t atom_bytes = (uint32_t)rows * (uint32_t)row_bytes;
@@ -196,8 +309,8 @@ __device__ __forceinline__ void gather_rows_stage(uint32_t tile_smem, int rows, 
     const int n_ch = tile_k >> 2;
     const int my_ch = (n_ch - wig + wpg - 1) / wpg;      // chunks wig, wig + wpg, ... belong to this warp
     const int n_tasks = my_ch > 0 ? my_ch * n_rb : 0;    // task = (chunk, 32-row block)
-    const uint32_t inv_rb = (65536u + (uint32_t)n_rb - 1u) / (uint32_t)n_rb;     // t / n_rb == (t * inv_rb) >> 16 for small t
-    constexpr int kBatch = 8;                            // tasks whose loads are issued before the first store
+    const uint32_t inv_rb = (65536u + (uint32_t)n_rb - 1u) / (uint32_t)n_rb;
+    constexpr int kBatch = 8;
     for (int t0 = 0; t0 < n_tasks; t0 += kBatch) {
         float val[kBatch][4];
         uint32_t dst[kBatch];
@@ -214,25 +327,12 @@ __device__ __forceinline__ void gather_rows_stage(uint32_t tile_smem, int rows, 
             dst[b] = in_tile ? tile_smem + (uint32_t)(kk >> atom_shift) * atom_bytes + (uint32_t)row * (uint32_t)row_bytes +
                                    ((uint32_t)((kk & (atom_k - 1)) << 2) ^ ((uint32_t)((row >> shift) & swz_mask) << 4))
                              : 0xffffffffu;
-            if (MODE == OPM_IM2COL) {
-                const uint4 e = *reinterpret_cast<const uint4*>(ktab + kk);      // same address in every lane
-                const int4 info = rowinfo[row < rows ? row : 0];
-                const uint32_t ev[4] = {e.x, e.y, e.z, e.w};
+            const int grow = row0 + row;
+            const bool rv = in_tile && grow < row_extent;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t tap = ev[j] & 63u;
-                    const uint32_t word = tap < 32u ? (uint32_t)info.y : (uint32_t)info.z;
-                    const bool ok = in_tile && ((word >> (tap & 31u)) & 1u) != 0u;
-                    val[b][j] = ok ? __ldg(src + ((int)(ev[j] >> 6) + info.x)) : 0.f;
-                }
-            } else {
-                const int grow = row0 + row;
-                const bool rv = in_tile && grow < row_extent;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int k = k0 + kk + j;
-                    val[b][j] = (rv && k < K) ? __ldg(src + (long long)grow * rs + (long long)k * ks) : 0.f;
-                }
+            for (int j = 0; j < 4; ++j) {
+                const int k = k0 + kk + j;
+                val[b][j] = (rv && k < K) ? __ldg(src + (long long)grow * rs + (long long)k * ks) : 0.f;
             }
         }
 #pragma unroll
@@ -272,13 +372,11 @@ __device__ __forceinline__ void gather_k_stage(uint32_t tile_smem, int rows, con
 }
 
 __device__ __forceinline__ void gather_stage(int mode, uint32_t tile_smem, int rows, const float* __restrict__ src,
-                                             long long rs, long long ks, const int4* rowinfo, const uint32_t* ktab,
-                                             int row0, int row_extent, int k0, int K, int tile_k, int atom_k, int row_bytes,
-                                             int swz_mask, int wig, int wpg, int lane) {
-    if (mode == OPM_IM2COL)
-        gather_rows_stage<OPM_IM2COL>(tile_smem, rows, src, rs, ks, rowinfo, ktab, row0, row_extent, k0, K, tile_k, atom_k, row_bytes, swz_mask, wig, wpg, lane);
-    else if (mode == OPM_GATHER_ROWS)
-        gather_rows_stage<OPM_GATHER_ROWS>(tile_smem, rows, src, rs, ks, rowinfo, ktab, row0, row_extent, k0, K, tile_k, atom_k, row_bytes, swz_mask, wig, wpg, lane);
+                                             long long rs, long long ks, int row0, int row_extent, int k0, int K,
+                                             int tile_k, int atom_k, int row_bytes, int swz_mask, int wig, int wpg,
+                                             int lane) {
+    if (mode == OPM_GATHER_ROWS)
+        gather_rows_stage(tile_smem, rows, src, rs, ks, row0, row_extent, k0, K, tile_k, atom_k, row_bytes, swz_mask, wig, wpg, lane);
     else
         gather_k_stage(tile_smem, rows, src, rs, ks, row0, row_extent, k0, K, tile_k, atom_k, row_bytes, swz_mask, wig, wpg, lane);
 }
@@ -379,7 +477,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __shared__ int abort_flag;
     __shared__ int last_split_flag;
     __shared__ __align__(16) float s_bias[256];
-    __shared__ int4 s_rowinfo[256];
+    __shared__ int s_rowoff[256];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int* abortp = &abort_flag;
@@ -403,8 +501,10 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const uint32_t stage_bytes = g.a_stage_bytes + g.b_stage_bytes;
     const bool a_tma = g.a_mode == OPM_TMA, b_tma = g.b_mode == OPM_TMA;
     const bool any_tma = a_tma || b_tma, any_gather = !a_tma || !b_tma;
-    // gather groups: 4 groups of 2 warps from 4 stages up, 2 groups of 4 warps for 2-3 stages, else one group
-    const int n_groups = g.stages >= 4 ? 4 : (g.stages >= 2 ? 2 : 1);
+    const bool im2col = g.a_mode == OPM_IM2COL || g.b_mode == OPM_IM2COL;
+    // gather groups (global gathers only): 4 groups of 2 warps from 4 stages up, 2 groups of 4 warps for 2-3 stages,
+    // else one group; the im2col expansion keeps all eight warps on one stage
+    const int n_groups = im2col ? 1 : (g.stages >= 4 ? 4 : (g.stages >= 2 ? 2 : 1));
     const int wpg = kGatherWarps / n_groups;
 
     if (threadIdx.x == 0) {
@@ -517,46 +617,99 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         // bias is fetched now so that its latency hides behind the main loop
         if (g.bias_mode == 2 && gt < g.tile_n) s_bias[gt] = (n0 + gt < g.N) ? __ldg(g.bias + n0 + gt) : 0.f;
         const float bias_row = (g.bias_mode == 1 && m < g.M) ? __ldg(g.bias + m) : 0.f;
-        if (any_gather) {
-            const Im2col ic{g.C, g.H, g.W, g.R, g.S, g.Q, g.sh, g.sw, g.ph, g.pw};
+        if (im2col) {
+            // ---- conv2d: slab staging + expansion; all eight warps work on the same stage ----
+            const bool on_a = g.a_mode == OPM_IM2COL;
+            const int rows = on_a ? kHwTileM : g.tile_n, row0 = on_a ? m0 : n0, ext = on_a ? g.M : g.N;
+            const float* img = (on_a ? g.a : g.b) + (long long)bz * (on_a ? g.a_bs : g.b_bs);
+            const float* o_src = on_a ? g.b + (long long)bz * g.b_bs : g.a + (long long)bz * g.a_bs;   // the other operand
+            const bool o_gather = on_a ? !b_tma : !a_tma;
+            const uint32_t ktab = tiles_base + g.ktab_off;
+            const uint32_t slab0 = tiles_base + g.slab_off;
+            const uint32_t rowoff = smem_u32(s_rowoff);
+            const int RS = g.R * g.S, T = g.slab_tiles;
+            const int last = min(row0 + rows, ext) - 1;
+            const int p_first = row0 / g.Q, p_last = last / g.Q;
+            const int ih_lo = p_first * g.sh - g.ph;
+            const int in_rows_cta = (p_last - p_first) * g.slab_rstep + g.R;
+            const int kbeg = kt_begin * g.tile_k;
+            const bool vec16 = g.slab_vec16 && ((reinterpret_cast<uintptr_t>(img) & 15u) == 0);
+            // tables, built once per CTA: byte offset of each tile row's window origin inside a slab channel, and
+            // per reduction index the byte offset of (channel relative to its chunk's first channel, tap)
+            if (gt < rows) {
+                const int grow = min(row0 + gt, ext - 1);    // rows past the extent repeat the last pixel (never stored)
+                const int p = grow / g.Q, q = grow - p * g.Q;
+                s_rowoff[gt] = 4 * ((p - p_first) * g.slab_rstep * g.slab_wp + q * g.sw + (g.slab_gap - g.pw));
+            }
+            const int tk_shift = 31 - __clz(g.tile_k);
+            for (int i = gt; i < iters * g.tile_k; i += kGatherThreads) {
+                const int k = kbeg + i;
+                const int chunk = (i >> tk_shift) / T;
+                const int c_first = (kbeg + chunk * T * g.tile_k) / RS;
+                int ent = 0;                              // beyond K: any finite value will do, the filter side is zero
+                if (k < g.K) {
+                    const int c = k / RS, rem = k - c * RS, fr = rem / g.S, fs = rem - fr * g.S;
+                    ent = 4 * ((c - c_first) * g.slab_chpitch + fr * g.slab_wp + fs);
+                }
+                st_shared_u32(ktab + 4u * (uint32_t)i, (uint32_t)ent);
+            }
+            // zeros for the gaps and for rows outside the image; copies only ever land on in-image positions
+            const uint32_t slab_bytes = (uint32_t)g.slab_nbuf * g.slab_buf_bytes;
+            for (uint32_t o = (uint32_t)gt * 16u; o < slab_bytes; o += (uint32_t)kGatherThreads * 16u)
+                st_shared_v4(slab0 + o, 0.f, 0.f, 0.f, 0.f);
+            bool ok = gather_vote(true);                 // tables and zeros are in place before any copy lands
+            const int n_chunks = (iters + T - 1) / T;
+            auto chunk_load = [&](int j) {
+                const int k_lo = kbeg + j * T * g.tile_k;
+                const int k_hi = min(g.K, kbeg + min((j + 1) * T, iters) * g.tile_k);
+                if (k_hi > k_lo) {
+                    const int c_first = k_lo / RS, c_last = (k_hi - 1) / RS;
+                    slab_load_chunk(g, img, slab0 + (uint32_t)(j & 1) * g.slab_buf_bytes, c_first, c_last - c_first + 1, ih_lo,
+                                    in_rows_cta, vec16, gt);
+                }
+                cp_async_commit();
+            };
+            chunk_load(0);
+            if (n_chunks > 1) chunk_load(1);
+            const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+            uint32_t st = 0, ph = 0;
+            for (int j = 0; j < n_chunks; ++j) {
+                if (j + 1 < n_chunks) cp_async_wait<1>(); else cp_async_wait<0>();
+                ok = gather_vote(ok);                    // every thread's copies of chunk j are visible to all
+                if (!ok) break;
+                if (threadIdx.x == 64 && j == 0) TT_STAMP(15);
+                const uint32_t slab = slab0 + (uint32_t)(j & 1) * g.slab_buf_bytes;
+                const int it_end = min((j + 1) * T, iters);
+                for (int it = j * T; it < it_end; ++it) {
+                    if (ok && !mbar_wait(empty0 + st * 8u, ph ^ 1u, abortp, g.status, 3u)) ok = false;
+                    if (ok) {
+                        const uint32_t a_s = tiles_base + st * stage_bytes, b_s = a_s + g.a_stage_bytes;
+                        const uint32_t kt = ktab + 4u * (uint32_t)(it * g.tile_k);
+                        expand_stage(on_a ? a_s : b_s, rows, slab, rowoff, kt, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, gw, lane);
+                        if (o_gather) {
+                            const int k0 = (kt_begin + it) * g.tile_k;
+                            if (on_a) gather_stage(g.b_mode, b_s, g.tile_n, o_src, g.b_rs, g.b_ks, n0, g.N, k0, g.K, g.tile_k,
+                                                   g.atom_k, g.row_bytes, g.swz_mask, gw, kGatherWarps, lane);
+                            else gather_stage(g.a_mode, a_s, kHwTileM, o_src, g.a_rs, g.a_ks, m0, g.M, k0, g.K, g.tile_k,
+                                              g.atom_k, g.row_bytes, g.swz_mask, gw, kGatherWarps, lane);
+                        }
+                        fence_proxy_async_shared();      // generic-proxy stores -> visible to the tensor core's reads
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(full0 + st * 8u);
+                    }
+                    if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
+                }
+                if (j + 2 < n_chunks) {
+                    ok = gather_vote(ok);                // everyone is done reading this buffer
+                    if (!ok) break;
+                    chunk_load(j + 2);
+                }
+            }
+            cp_async_wait<0>();
+            if (threadIdx.x == 64) TT_STAMP(16);
+        } else if (any_gather) {
             const float* a_src = g.a + (long long)bz * g.a_bs;
             const float* b_src = g.b + (long long)bz * g.b_bs;
-            uint32_t* ktab = reinterpret_cast<uint32_t*>(smem_raw + (tiles_base - smem_u32(smem_raw)) + g.ktab_off);
-            if (g.a_mode == OPM_IM2COL || g.b_mode == OPM_IM2COL) {
-                // Tables of the im2col operand, built once per CTA.
-                // rowinfo: per tile row, where its pixel's receptive field starts and which filter taps fall
-                // inside the image (bit r*S + s); ktab: per reduction index of this CTA's K range, the element
-                // offset of (c, r, s) and its tap index.
-                const bool on_a = g.a_mode == OPM_IM2COL;
-                const int rows = on_a ? kHwTileM : g.tile_n, row0 = on_a ? m0 : n0, ext = on_a ? g.M : g.N;
-                if (gt < rows) {
-                    const int grow = row0 + gt;
-                    int4 info = make_int4(0, 0, 0, 0);
-                    if (grow < ext) {
-                        const int p = grow / ic.Q, q = grow - p * ic.Q;
-                        const int ih0 = p * ic.sh - ic.ph, iw0 = q * ic.sw - ic.pw;
-                        const int s_lo = max(0, -iw0), s_hi = min(ic.S, ic.W - iw0);      // taps s_lo .. s_hi-1 are in range
-                        const unsigned long long colmask = s_hi > s_lo ? (((1ull << s_hi) - 1ull) & ~((1ull << s_lo) - 1ull)) : 0ull;
-                        unsigned long long mask = 0ull;
-                        for (int fr = 0; fr < ic.R; ++fr)
-                            if ((unsigned)(ih0 + fr) < (unsigned)ic.H) mask |= colmask << (fr * ic.S);
-                        info.x = ih0 * ic.W + iw0; info.y = (int)(uint32_t)mask; info.z = (int)(uint32_t)(mask >> 32);
-                    }
-                    s_rowinfo[gt] = info;
-                }
-                const int RS = ic.R * ic.S, HW = ic.H * ic.W;
-                const int kbeg = kt_begin * g.tile_k;
-                for (int i = gt; i < iters * g.tile_k; i += kGatherThreads) {
-                    const int k = kbeg + i;
-                    uint32_t ent = 63u;                  // beyond K: a tap no mask ever enables
-                    if (k < g.K) {
-                        const int c = k / RS, rem = k - c * RS, fr = rem / ic.S, fs = rem - fr * ic.S;
-                        ent = ((uint32_t)(c * HW + fr * ic.W + fs) << 6) | (uint32_t)rem;
-                    }
-                    ktab[i] = ent;
-                }
-                asm volatile("bar.sync 1, %0;" ::"n"(kGatherThreads) : "memory");
-            }
             const int grp = gw / wpg, wig = gw - grp * wpg;
             const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
             int st = grp % g.stages;
@@ -565,17 +718,13 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (!mbar_wait(empty0 + (uint32_t)st * 8u, ph ^ 1u, abortp, g.status, 3u)) break;
                 const uint32_t a_s = tiles_base + (uint32_t)st * stage_bytes, b_s = a_s + g.a_stage_bytes;
                 const int k0 = (kt_begin + it) * g.tile_k;
-                if (threadIdx.x == 64 && it == 4) TT_STAMP(15);
-                const uint32_t* kt = ktab + (it * g.tile_k);
-                if (!a_tma) gather_stage(g.a_mode, a_s, kHwTileM, a_src, g.a_rs, g.a_ks, s_rowinfo, kt, m0, g.M, k0, g.K, g.tile_k,
+                if (!a_tma) gather_stage(g.a_mode, a_s, kHwTileM, a_src, g.a_rs, g.a_ks, m0, g.M, k0, g.K, g.tile_k,
                                          g.atom_k, g.row_bytes, g.swz_mask, wig, wpg, lane);
-                if (!b_tma) gather_stage(g.b_mode, b_s, g.tile_n, b_src, g.b_rs, g.b_ks, s_rowinfo, kt, n0, g.N, k0, g.K, g.tile_k,
+                if (!b_tma) gather_stage(g.b_mode, b_s, g.tile_n, b_src, g.b_rs, g.b_ks, n0, g.N, k0, g.K, g.tile_k,
                                          g.atom_k, g.row_bytes, g.swz_mask, wig, wpg, lane);
-                if (threadIdx.x == 64 && it == 4) TT_STAMP(16);
                 fence_proxy_async_shared();              // generic-proxy stores -> visible to the tensor core's reads
                 __syncwarp();
                 if (lane == 0) mbar_arrive(full0 + (uint32_t)st * 8u);
-                if (threadIdx.x == 64 && it == 4) TT_STAMP(17);
                 st += n_groups;
                 while (st >= g.stages) { st -= g.stages; ph ^= 1u; }
             }
@@ -791,6 +940,114 @@ __global__ void tt_dwconv_kernel(const DwArgs d) {
 }
 
 // ------------------------------------------------------------------------------------------------------------
+// DW_SIMT, register-window form (3x3 and 5x5 filters, stride 1 or 2).  A thread owns a strip of ROWS output rows
+// x 4 consecutive output columns of one channel.  It walks the (ROWS-1)*STRIDE + R input rows the strip needs
+// once: of each row it fetches 3*STRIDE + R values (aligned 16-byte loads for the columns under the strip when the
+// image rows allow it, 4-byte loads for the ragged edges; neighbouring strips' loads meet in L1) and feeds every
+// output row whose window contains that input row, so an input value is read once per strip and no shared
+// memory or barrier is involved.  Bound by HBM: the only DRAM traffic is x once, y once.
+// ------------------------------------------------------------------------------------------------------------
+template <int R, int STRIDE, int ROWS>
+__global__ void __launch_bounds__(256) tt_dwconv_window_kernel(const DwArgs d) {
+    constexpr int NCOL = 3 * STRIDE + R;                  // input columns under a 4-wide strip
+    constexpr int IN_ROWS = (ROWS - 1) * STRIDE + R;
+    constexpr int PAD = R / 2;                            // "same" padding: the launcher checks it
+    constexpr int NV = (NCOL - PAD) / 4;                  // aligned 16-byte groups per window row
+    const int n = blockIdx.y;
+    int t = blockIdx.x;
+    const int tw = t % d.tiles_w; t /= d.tiles_w;
+    const int th = t % d.tiles_h; t /= d.tiles_h;
+    const int c0 = t * d.tile_c, p0 = th * d.tile_h, q0 = tw * d.tile_w;
+    const int nc = min(d.tile_c, d.C - c0);
+    const int groups_w = d.tile_w >> 2;
+    const int groups_h = (d.tile_h + ROWS - 1) / ROWS;
+    const int work = nc * groups_h * groups_w;
+    for (int i = threadIdx.x; i < work; i += blockDim.x) {
+        const int gwi = i % groups_w;
+        const int rest = i / groups_w;
+        const int gh = rest % groups_h, cl = rest / groups_h;
+        const int p = p0 + gh * ROWS, q = q0 + gwi * 4;
+        if (p >= d.P || q >= d.Q || gh * ROWS >= d.tile_h) continue;
+        const int c = c0 + cl;
+        const float* __restrict__ xc = d.x + ((long long)n * d.C + c) * d.H * (long long)d.W;
+        const float* __restrict__ wc = d.w + (long long)c * (R * R);
+        float wv[R * R];
+#pragma unroll
+        for (int k = 0; k < R * R; ++k) wv[k] = __ldg(wc + k);
+        const float b = d.bias ? __ldg(d.bias + c) : 0.f;
+        float acc[ROWS][4];
+#pragma unroll
+        for (int ro = 0; ro < ROWS; ++ro)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[ro][j] = b;
+        const int ih0 = p * STRIDE - PAD, iw0 = q * STRIDE - PAD;
+#pragma unroll
+        for (int ri = 0; ri < IN_ROWS; ++ri) {
+            const int ih = ih0 + ri;
+            float v[NCOL];
+#pragma unroll
+            for (int j = 0; j < NCOL; ++j) v[j] = 0.f;
+            if ((unsigned)ih < (unsigned)d.H) {
+                const float* __restrict__ xr = xc + (long long)ih * d.W;
+                if (d.vec_in) {
+                    // window slots [PAD, PAD + 4*NV) lie under the strip and start on a 16-byte boundary; a group
+                    // of four columns is inside the row or outside it as a whole (W % 4 == 0)
+#pragma unroll
+                    for (int k = 0; k < NV; ++k) {
+                        const int col = iw0 + PAD + 4 * k;
+                        if (col < d.W) {
+                            const float4 f = __ldg(reinterpret_cast<const float4*>(xr + col));
+                            v[PAD + 4 * k] = f.x; v[PAD + 4 * k + 1] = f.y; v[PAD + 4 * k + 2] = f.z; v[PAD + 4 * k + 3] = f.w;
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < NCOL; ++j) {
+                        if (j >= PAD && j < PAD + 4 * NV) continue;
+                        const int col = iw0 + j;
+                        if ((unsigned)col < (unsigned)d.W) v[j] = __ldg(xr + col);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < NCOL; ++j) {
+                        const int col = iw0 + j;
+                        if ((unsigned)col < (unsigned)d.W) v[j] = __ldg(xr + col);
+                    }
+                }
+            }
+#pragma unroll
+            for (int ro = 0; ro < ROWS; ++ro) {
+                const int fr = ri - ro * STRIDE;              // compile-time after unrolling
+                if (fr >= 0 && fr < R) {
+#pragma unroll
+                    for (int fs = 0; fs < R; ++fs)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) acc[ro][j] = fmaf(v[j * STRIDE + fs], wv[fr * R + fs], acc[ro][j]);
+                }
+            }
+        }
+        float* __restrict__ yc = d.y + (((long long)n * d.C + c) * d.P + p) * (long long)d.Q + q;
+#pragma unroll
+        for (int ro = 0; ro < ROWS; ++ro) {
+            if (p + ro >= d.P || gh * ROWS + ro >= d.tile_h) break;
+            float o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) o[j] = apply_act(acc[ro][j], d.act);
+            float* yo = yc + (long long)ro * d.Q;
+            if (d.vec == 4 && q + 4 <= d.Q) {
+                *reinterpret_cast<float4*>(yo) = make_float4(o[0], o[1], o[2], o[3]);
+            } else if (d.vec == 2 && q + 4 <= d.Q) {
+                *reinterpret_cast<float2*>(yo) = make_float2(o[0], o[1]);
+                *reinterpret_cast<float2*>(yo + 2) = make_float2(o[2], o[3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (q + j < d.Q) yo[j] = o[j];
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------
 // ROW_SIMT: softmax(scale * x) per row; `lanes_per_row` threads of one warp share a row.
 // ------------------------------------------------------------------------------------------------------------
 __global__ void tt_softmax_kernel(const RowArgs a) {
@@ -855,6 +1112,17 @@ cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st)
         attr_set_for = dev;
     }
     dim3 grid(I.grid_x, I.grid_y, 1);
+    if (dw.window_rows > 0) {
+        // register-window kernels: one instantiation per (filter size, stride, output rows per thread)
+#define TT_DW_CASE(RR, SS, RO) \
+        if (dw.R == RR && dw.sh == SS && dw.window_rows == RO) { tt_dwconv_window_kernel<RR, SS, RO><<<grid, I.threads, 0, st>>>(dw); return cudaGetLastError(); }
+        TT_DW_CASE(3, 1, 1) TT_DW_CASE(3, 1, 2) TT_DW_CASE(3, 1, 4)
+        TT_DW_CASE(3, 2, 1) TT_DW_CASE(3, 2, 2) TT_DW_CASE(3, 2, 4)
+        TT_DW_CASE(5, 1, 1) TT_DW_CASE(5, 1, 2) TT_DW_CASE(5, 1, 4)
+        TT_DW_CASE(5, 2, 1) TT_DW_CASE(5, 2, 2) TT_DW_CASE(5, 2, 4)
+#undef TT_DW_CASE
+        return cudaErrorInvalidValue;
+    }
     tt_dwconv_kernel<<<grid, I.threads, I.smem_bytes, st>>>(dw);
     return cudaGetLastError();
 }

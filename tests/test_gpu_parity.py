@@ -46,13 +46,25 @@ GEMM_RECORDS = [
     tc(tile_n=128, tile_k=64, stages=3, split_k=2, mma_m_axis=2),
     tc(tile_n=32, tile_k=128, stages=2, split_k=1, raster=1, mma_m_axis=2),
     tc(tile_n=192, tile_k=16, stages=4, split_k=5, mma_m_axis=2),
+    # convolutions: the input rows are staged for 1, 2 or 3 reduction tiles at a time (double-buffered chunks)
+    tc(tile_n=64, tile_k=16, stages=3, slab_tiles=1, mma_m_axis=1),
+    tc(tile_n=128, tile_k=32, stages=2, slab_tiles=2, mma_m_axis=2),
+    tc(tile_n=32, tile_k=8, stages=4, split_k=2, slab_tiles=3, mma_m_axis=1),
 ]
 
 
 def check_all_records(spec, seed, records=GEMM_RECORDS):
     a = W.make_inputs(spec, seed)
     ref = util.oracle_ref(spec, a)
-    outs = [run_spec(spec, r, a, ref) for r in records]
+    # a record whose tiles (for a convolution: plus the staged input rows) exceed shared memory on this shape is an
+    # invalid pair, as in the evaluator; everything that applies must be right, and most records must apply
+    probe = spec.workload()
+    valid = [r for r in records if probe.check(r)[0] == B.TT_OK]
+    assert all(probe.check(r)[0] in (B.TT_OK, B.TT_ERR_RESOURCE) for r in records)
+    assert probe.check(probe.default_schedule())[0] == B.TT_OK
+    probe.close()
+    assert len(valid) >= len(records) - 2
+    outs = [run_spec(spec, r, a, ref) for r in valid]
     # a schedule changes speed, never semantics: every valid record gives the same output up to the order of the
     # fp32 additions (tile_k and split_k regroup them): sqrt(K) * 2^-24 is about 4e-6 at the largest K here
     for y in outs[1:]:
@@ -82,6 +94,11 @@ def test_dense_parity_all_records(spec):
     W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(2, 8, 9, 11, 12, 3, 3, 1, 1, True, B.TT_ACT_RELU, True), 1, "batch2_residual", "uniform"),
     W.Spec(B.TT_OP_CONV2D, B.make_shapes(n=1, c=6, h=10, w=12, k=9, r=3, s=2, stride_h=2, stride_w=1, pad_h=0, pad_w=1,
                                          has_bias=0, act=B.TT_ACT_NONE), 1, "asym_nobias", "uniform"),
+    W._conv(96, 9, 48, 3, 1, 1, name="conv3x3_96ch_chunks"),                # 864 reduction indices: many slab chunks
+    W._conv(40, 12, 24, 5, 1, 2, act=B.TT_ACT_RELU6, name="conv5x5_pad2"),
+    W._conv(32, 17, 16, 1, 3, 0, name="conv1x1s3"),                         # stride beyond the filter: rows are skipped
+    W.Spec(B.TT_OP_CONV2D, B.make_shapes(n=2, c=5, h=9, w=13, k=7, r=2, s=4, stride_h=3, stride_w=2, pad_h=1, pad_w=3,
+                                         has_bias=1, act=B.TT_ACT_RELU), 1, "asym_2x4_s3x2_p1x3", "uniform"),
 ], ids=lambda s: s.name)
 def test_conv_parity_all_records(spec):
     check_all_records(spec, seed=32)
@@ -154,10 +171,14 @@ def test_depthwise_parity_records(spec):
     a = W.make_inputs(spec, 34)
     ref = util.oracle_ref(spec, a)
     recs = [spec.workload().default_schedule()]
-    for tcn, by, bx, it, vw, th in ((4, 8, 32, 4, 4, 256), (16, 4, 16, 2, 2, 128), (1, 16, 64, 8, 4, 64), (32, 7, 7, 1, 1, 512),
-                                    (3, 5, 24, 8, 1, 96)):
+    # unroll 0: shared-memory staged kernel; 1, 2, 4: register-window kernel with that many output rows per thread
+    # (3x3 / 5x5 "same" filters; other filters fall back to the staged kernel)
+    for tcn, by, bx, it, vw, th, un in ((4, 8, 32, 4, 4, 256, 0), (16, 4, 16, 2, 2, 128, 0), (1, 16, 64, 8, 4, 64, 0),
+                                        (32, 7, 7, 1, 1, 512, 0), (3, 5, 24, 8, 1, 96, 0),
+                                        (4, 8, 32, 4, 4, 256, 1), (1, 16, 64, 8, 4, 64, 2), (2, 7, 12, 4, 4, 512, 4),
+                                        (8, 5, 8, 1, 1, 32, 4), (3, 6, 112, 4, 2, 96, 2)):
         recs.append(B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=tcn, block_y=by, block_x=bx, items_per_thread=it,
-                                  vec_width=vw, threads=th))
+                                  vec_width=vw, threads=th, unroll=un))
     outs = [run_spec(spec, r, a, ref) for r in recs]
     for y in outs[1:]:
         np.testing.assert_array_equal(y, outs[0])       # same fp32 operations in the same order: bit-identical

@@ -167,8 +167,19 @@ def test_legaliser_clamps_and_strict_mode_rejects():
     # resources: 8 stages of 128x256x128 do not fit shared memory
     fat = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=256, tile_k=128, stages=8, mma_m_axis=1)
     huge = W._dense(512, 4096, 4096).workload()
+    # reformulated: the pipeline is made shallower until it fits (one 192 KB stage); kept as written it is invalid
     st, info = huge.check(fat)
+    assert st == B.TT_OK and info.legal.stages == 1 and info.changed & B.TT_CHG_STAGES
+    st, info = huge.check(fat, mode=B.TT_MODE_STRICT)
     assert st == B.TT_ERR_RESOURCE and info.smem_bytes > 227 * 1024
+    # a 256-pixel x 128-channel tile of a 1x1 convolution: its input slab alone exceeds shared memory at any depth
+    wide = W._conv(256, 56, 64, 1, 1, 0).workload()
+    st, info = wide.check(B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=32, tile_k=128, stages=2, mma_m_axis=2))
+    assert st == B.TT_ERR_RESOURCE and info.smem_bytes > 227 * 1024
+    # the slab is part of the record: a request for more reduction tiles per staging than fit is lowered
+    conv = W._conv(512, 28, 512, 3, 1, 1).workload()
+    st, info = conv.check(B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=128, tile_k=32, stages=3, slab_tiles=64, mma_m_axis=1))
+    assert st == B.TT_OK and 1 <= info.legal.slab_tiles < 64 and info.changed & B.TT_CHG_SLAB
     # nonsense fields
     for kw in (dict(tile_n=0), dict(stages=0), dict(split_k=-1), dict(raster=5), dict(mma_m_axis=7)):
         assert wl.check(B.make_record(B.TT_FAMILY_GEMM_TC, **kw))[0] == B.TT_ERR_INVALID_SCHEDULE
