@@ -250,6 +250,27 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
                        size_t top_k, tt_schedule_record* out_records, float* out_us, size_t* n_out,
                        int32_t* n_tried);
 
+/* (No counterpart in the paper.)  dense+bias+activation under a split-K record for callers that cannot allocate
+ * device memory when they need the kernel: hosts whose memory pool already owns the whole device, loops that may
+ * not take the allocator's lock, plug-ins that are forbidden to allocate after start-up.  The partial sums of the
+ * splits, their arrival counters and the status word live in ONE fixed device array of TT_STATIC_SCRATCH_BYTES
+ * that belongs to the library image (each device that loads the library holds it until the process exits), so
+ * this call makes no cudaMalloc/cudaFree and calls no allocating routine.
+ *   x [m,kk], w [nn,kk], bias [nn] or NULL, y [m,nn]: DEVICE pointers, fp32, row-major, 16-byte aligned, owned by
+ *   the caller; `rec` is a GEMM_TC record (legalised as in tt_schedule_apply); act is a tt_act.
+ *   scratch_bytes_used (may be NULL) receives what the legalised record needs of the array.
+ * Errors: TT_ERR_RESOURCE when that exceeds TT_STATIC_SCRATCH_BYTES (lower split_k, or use tt_run, which
+ * allocates); the statuses of tt_schedule_apply for a bad record; TT_ERR_CUDA; TT_ERR_TIMEOUT from the kernel.
+ * The call launches on `cuda_stream` and synchronises it before returning.  The first call on a device looks up
+ * the array's address (with that device current); make that first call outside any stream capture.
+ * All calls share the array: it keeps the previous call's contents (the words that must start at zero are cleared
+ * on the stream before each launch), and two calls that overlap on the GPU race on it -- issue them one at a
+ * time per device. */
+#define TT_STATIC_SCRATCH_BYTES (8u << 20)
+tt_status tt_dense_static_scratch(const void* x, const void* w, const void* bias, void* y, int32_t m, int32_t nn,
+                                  int32_t kk, int32_t act, const tt_schedule_record* rec, void* cuda_stream,
+                                  int64_t* scratch_bytes_used);
+
 #ifdef __cplusplus
 }
 #endif

@@ -117,6 +117,8 @@ EXPORTS = {
                                C.c_size_t, C.POINTER(tt_tune_opts), C.c_void_p, C.POINTER(tt_tune_result)]),
     "tt_grid_tune": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(tt_timing_opts), i32, C.c_size_t,
                            C.POINTER(tt_schedule_record), C.POINTER(f32), C.POINTER(C.c_size_t), C.POINTER(i32)]),
+    "tt_dense_static_scratch": (i32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, i32, i32, i32, i32,
+                                      C.POINTER(tt_schedule_record), C.c_void_p, C.POINTER(C.c_int64)]),
 }
 
 _lib = None
@@ -322,6 +324,21 @@ class Workload:
             C.memmove(C.byref(r), C.byref(recs[i]), C.sizeof(r))
             out.append((r, float(us[i])))
         return out, tried.value
+
+
+TT_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def dense_static_scratch(x, w, bias, y, act, rec):
+    """tt_dense_static_scratch on torch CUDA tensors x [m,kk], w [nn,kk], bias [nn] or None, y [m,nn]: the dense
+    layer under `rec` with its split-K scratch in the library's fixed device array, for callers that cannot
+    allocate device memory.  Returns (tt_status, scratch bytes the record needs); never raises."""
+    m, kk = x.shape
+    nn = w.shape[0]
+    used = C.c_int64(0)
+    st = lib().tt_dense_static_scratch(_ptr(x), _ptr(w), _ptr(bias), _ptr(y), m, nn, kk, act, C.byref(rec), _stream(),
+                                       C.byref(used))
+    return st, used.value
 
 
 def transfer_tune(workloads, tensor_sets, pool, opts: tt_tune_opts | None = None):

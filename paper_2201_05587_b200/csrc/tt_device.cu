@@ -507,3 +507,90 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
 
 }  // extern "C"
 
+// ------------------------------------------------------------------------------------------------------------
+// Split-K dense layer for callers that must not allocate device memory.
+//
+// Some hosts of this library cannot call cudaMalloc at the point where they need a kernel: code running inside
+// a memory pool that owns the whole device, a real-time loop that may not take the allocator's lock, a plug-in
+// whose host application forbids allocations after start-up.  For them the split-K partial sums, the arrival
+// counters and the status word live in one fixed array that is part of the library image: every device that
+// loads the library carries it until the process exits.
+// ------------------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_tt_static_scratch[TT_STATIC_SCRATCH_BYTES];
+
+namespace tt {
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned char* g_scratch_addr[kMaxDevices] = {};
+
+// In host code the array's name only stands for the symbol; the device address is asked for once per device,
+// with that device current.
+tt_status static_scratch(unsigned char** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return TT_ERR_CUDA; }
+    if (!g_scratch_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_tt_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return TT_ERR_CUDA; }
+        g_scratch_addr[dev] = static_cast<unsigned char*>(p);
+    }
+    *out = g_scratch_addr[dev];
+    return TT_OK;
+}
+}  // namespace
+}  // namespace tt
+
+extern "C" tt_status tt_dense_static_scratch(const void* x, const void* w, const void* bias, void* y, int32_t m,
+                                             int32_t nn, int32_t kk, int32_t act, const tt_schedule_record* rec,
+                                             void* cuda_stream, int64_t* scratch_bytes_used) {
+    if (!x || !w || !y || !rec || m <= 0 || nn <= 0 || kk <= 0 || act < TT_ACT_NONE || act > TT_ACT_GELU_ERF)
+        return TT_ERR_INVALID_ARG;
+    if (!device_present()) return TT_ERR_CUDA;
+    // the kernel description, built in place (no handle is created)
+    tt_workload wl;
+    wl.op = TT_OP_DENSE;
+    std::memset(&wl.sh, 0, sizeof wl.sh);
+    wl.sh.batch = 1; wl.sh.m = m; wl.sh.nn = nn; wl.sh.kk = kk; wl.sh.trans_b = 1;
+    wl.sh.has_bias = bias != nullptr; wl.sh.act = act;
+    wl.family = TT_FAMILY_GEMM_TC;
+    wl.P = wl.Q = 0;
+    wl.view = tt_gemm_view{1, m, nn, kk, 2.0 * m * (double)nn * kk, 0.0};
+    Plan plan;
+    tt_status s = legalise(&wl, rec, TT_MODE_LEGALISE, 0, &plan);
+    if (s != TT_OK) return s;
+    // layout of the fixed array: status word | arrival counters | partial sums
+    const int64_t counters_bytes = ((int64_t)plan.info.grid_x * plan.info.grid_z * 4 + 255) / 256 * 256;
+    const int64_t need = 256 + counters_bytes + (plan.g.split_k > 1 ? plan.partial_bytes : 0);
+    if (scratch_bytes_used) *scratch_bytes_used = need;
+    if (need > (int64_t)TT_STATIC_SCRATCH_BYTES) return TT_ERR_RESOURCE;   // this record's partial sums do not fit
+    unsigned char* base = nullptr;
+    if ((s = static_scratch(&base)) != TT_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // the array keeps what the previous call left: the status word and the counters must start at zero
+    if (cudaMemsetAsync(base, 0, (size_t)(256 + counters_bytes), st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    GemmArgs g = plan.g;
+    const void* tens[2] = {x, w};
+    const void* a_ptr = tens[plan.a_tensor];
+    const void* b_ptr = tens[plan.b_tensor];
+    g.a = static_cast<const float*>(a_ptr);
+    g.b = static_cast<const float*>(b_ptr);
+    g.y = static_cast<float*>(y);
+    g.bias = static_cast<const float*>(bias);
+    g.residual = nullptr;
+    g.status = reinterpret_cast<unsigned*>(base);
+    g.counters = reinterpret_cast<unsigned*>(base + 256);
+    g.partial = reinterpret_cast<float*>(base + 256 + counters_bytes);
+    if ((reinterpret_cast<uintptr_t>(y) & 15u) != 0) g.vec_store = 0;
+    if (g.bias && (reinterpret_cast<uintptr_t>(g.bias) & 15u) == 0) g.vec_store |= 2;
+    TmapPair maps;
+    std::memset(&maps, 0, sizeof maps);
+    if (g.a_mode == OPM_TMA)
+        s = encode_operand(maps.a, g.a, g.K, g.M, g.batch, g.a_rs, g.a_bs, g.a_tma_batched != 0, g.atom_k, kHwTileM);
+    if (s == TT_OK && g.b_mode == OPM_TMA)
+        s = encode_operand(maps.b, g.b, g.K, g.N, g.batch, g.b_rs, g.b_bs, g.b_tma_batched != 0, g.atom_k, g.tile_n);
+    if (s != TT_OK) return s;
+    if (launch_gemm(plan.info, g, maps.a, maps.b, st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    unsigned v = 0;
+    if (cudaMemcpy(&v, base, 4, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    return v ? (tt_status)(v & 0xffu) : TT_OK;
+}
