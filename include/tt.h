@@ -93,7 +93,7 @@ typedef struct tt_shapes {
  *   cache buffer / ComputeAt -> the accumulator lives in tensor memory and the bias/activation run on read-out;
  *                               `stages` shared-memory buffers decouple loading from the multiply
  *   Vectorize -> vec_width;   Unroll -> unroll / items_per_thread
- * GEMM_TC uses tile_m, tile_n, tile_k, stages, split_k, raster, mma_m_axis, slab_tiles.
+ * GEMM_TC uses tile_m, tile_n, tile_k, stages, split_k, raster, mma_m_axis, slab_tiles, acc_split.
  * DW_SIMT uses tile_m (channels per CTA), block_y x block_x (output rows x columns per CTA tile),
  *         items_per_thread (consecutive outputs along the width per thread), vec_width, threads, and unroll:
  *         0 = shared-memory staged kernel; 1, 2, 4 = register-window kernel with that many output rows per thread
@@ -112,7 +112,11 @@ typedef struct tt_schedule_record {
                               1 output rows (conv filters, dense/bmm rows m), 2 output columns (conv pixels, nn) */
     int32_t slab_tiles;    /* GEMM_TC, conv2d only: reduction tiles served by one staging of the input rows in shared
                               memory (the cache buffer of the im2col operand); 0 = as many as fit */
-    int32_t reserved[2];
+    int32_t acc_split;     /* GEMM_TC: independent accumulators in tensor memory (1, 2, 4 or 8; 0 = 1) to which the
+                              8-wide reduction steps are dealt round-robin; they are added in fixed order on read-out.
+                              Consecutive multiply-accumulates into one accumulator wait for each other; into several,
+                              they overlap (the reduction-factoring of a schedule). */
+    int32_t reserved[1];
 } tt_schedule_record;
 
 typedef struct tt_tensors {
@@ -141,7 +145,7 @@ typedef struct tt_apply_info {
 } tt_apply_info;
 
 enum { TT_CHG_TILE_M = 1, TT_CHG_TILE_N = 2, TT_CHG_TILE_K = 4, TT_CHG_STAGES = 8, TT_CHG_SPLIT_K = 16,
-       TT_CHG_VEC = 32, TT_CHG_BLOCK = 64, TT_CHG_ITEMS = 128, TT_CHG_SLAB = 256 };
+       TT_CHG_VEC = 32, TT_CHG_BLOCK = 64, TT_CHG_ITEMS = 128, TT_CHG_SLAB = 256, TT_CHG_ACC = 512 };
 
 /* Validity modes for mapping a record onto another shape (Section 4.1).
  *   TT_MODE_LEGALISE  reformulate: clamp/round tile sizes to the new extents and the hardware's legal set,

@@ -13,6 +13,7 @@ namespace tt {
 cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, cudaStream_t st);
 cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st);
 cudaError_t launch_row(const tt_apply_info& I, const RowArgs& row, cudaStream_t st);
+cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits);
 
 namespace {
 
@@ -79,6 +80,12 @@ void release_device(tt_workload* w) {
 
 tt_status bind_device(tt_workload* w) {
     if (!device_present()) return TT_ERR_CUDA;
+    if (w->family == TT_FAMILY_GEMM_TC && w->plan.g.cluster) {
+        // a cluster whose CTAs cannot be resident together can never launch: an invalid pair, not a device error
+        int fits = 0;
+        if (gemm_cluster_fits(w->plan.info.smem_bytes, w->plan.g.cluster, &fits) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+        if (!fits) return TT_ERR_RESOURCE;
+    }
     const size_t need = (size_t)w->plan.info.workspace_bytes;
     if (need > w->workspace_bytes) {
         if (w->workspace) cudaFree(w->workspace);

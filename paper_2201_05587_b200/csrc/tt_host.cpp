@@ -124,6 +124,12 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     sk = (k_tiles + per_split - 1) / per_split;          // every split owns at least one reduction tile
     if (sk != rec->split_k) changed |= TT_CHG_SPLIT_K;
     L.split_k = sk;
+    // accumulators: a power of two, all of them inside the 512 columns of tensor memory, none left without a step
+    if (rec->acc_split < 0) return TT_ERR_INVALID_SCHEDULE;
+    int nacc = std::min(8, pow2_floor(std::max(1, rec->acc_split)));
+    while (nacc > 1 && (nacc * tn > 512 || (long long)nacc > (long long)per_split * (tk / 8))) nacc >>= 1;
+    if (nacc != std::max(1, rec->acc_split)) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_ACC; }
+    L.acc_split = nacc;
     // buffers beyond the reduction tiles of one CTA would never be filled
     if (st > per_split) { st = per_split; changed |= TT_CHG_STAGES; L.stages = st; }
     if (strict && (changed & ~TT_CHG_TILE_M)) return TT_ERR_INVALID_SCHEDULE;
@@ -138,6 +144,11 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     // Per channel the slab holds, for each of the output rows a tile can span, the input rows its filter rows
     // touch: consecutive rows when stride <= filter height, else `r` rows per output row.  A chunk holds the
     // channels that `slab_tiles` consecutive reduction tiles touch; two buffers when there are several chunks.
+    // split_k of 2..8: the splits of a tile form a thread-block cluster and reduce through distributed shared memory
+    // (each parks its 128 x tile_n partial tile in its pipeline buffers); beyond 8 the partial tiles go through a
+    // global workspace and the split that arrives last adds them up
+    const int cluster = (sk >= 2 && sk <= 8) ? sk : 0;
+    const long long min_pipe = std::max<long long>((long long)kGatherWarps * 32 * 36 * 4, cluster ? std::max<long long>((long long)tn * (kHwTileM + 4) * 4, (long long)kHwTileM * (tn + 4) * 4) : 0);
     const bool conv = w->op == TT_OP_CONV2D;
     const long long ktab = conv ? (((long long)per_split * tk * 4 + 15) / 16) * 16 : 0;
     int sl_tiles = 0, sl_nbuf = 0, sl_wp = 0, sl_gap = 0, sl_chpitch = 0, sl_in_rows = 0, sl_rstep = 1;
@@ -162,7 +173,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     };
     long long smem = 0;
     for (;;) {
-        const long long pipe_try = std::max<long long>((long long)st * (a_stage + b_stage), (long long)kGatherWarps * 32 * 36 * 4);
+        const long long pipe_try = std::max<long long>((long long)st * (a_stage + b_stage), min_pipe);
         long long slab_total = 0;
         bool fits = true;
         if (conv) {
@@ -184,7 +195,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
         changed |= TT_CHG_STAGES;
     }
     L.stages = st;
-    const long long pipe = std::max<long long>((long long)st * (a_stage + b_stage), (long long)kGatherWarps * 32 * 36 * 4);
+    const long long pipe = std::max<long long>((long long)st * (a_stage + b_stage), min_pipe);
     if (conv) {
         if (rec->slab_tiles != 0 && sl_tiles != rec->slab_tiles) {
             if (strict) return TT_ERR_INVALID_SCHEDULE;
@@ -194,7 +205,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     } else {
         L.slab_tiles = 0;
     }
-    int tmem_cols = std::max(32, pow2_ceil(tn));
+    int tmem_cols = std::max(32, pow2_ceil(nacc * tn));
     const int tiles_m = (M + kHwTileM - 1) / kHwTileM, tiles_n = (N + tn - 1) / tn;
     if ((long long)tiles_m * tiles_n > 0x7fffffffLL || sk > 65535 || B > 65535) return TT_ERR_RESOURCE;
 
@@ -206,8 +217,9 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     I.smem_bytes = (int)std::min<long long>(smem, 0x7fffffff);
     I.tmem_cols = tmem_cols;
     // split-K workspace: partial tiles, then one arrival counter per (batch, tile)
-    plan->partial_bytes = sk > 1 ? (((long long)sk * B * M * N * 4 + 255) / 256) * 256 : 0;
-    I.workspace_bytes = sk > 1 ? plan->partial_bytes + (int64_t)B * tiles_m * tiles_n * 4 : 0;
+    const bool ws = sk > 1 && cluster == 0;
+    plan->partial_bytes = ws ? (((long long)sk * B * M * N * 4 + 255) / 256) * 256 : 0;
+    I.workspace_bytes = ws ? plan->partial_bytes + (int64_t)B * tiles_m * tiles_n * 4 : 0;
     I.launches = 1;
     if (smem > kDynSmemLimit) return TT_ERR_RESOURCE;
 
@@ -233,6 +245,8 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
         g.magic_in_rows = sl_in_rows > 1 ? (unsigned)((0x100000000ull + sl_in_rows - 1) / sl_in_rows) : 0u;
     }
     g.tmem_cols = (unsigned)tmem_cols;
+    g.n_acc = nacc;
+    g.cluster = cluster;
     // Instruction descriptor, kind::tf32: D = F32 (bits 4-5 = 1), A and B = TF32 (bits 7-9, 10-12 = 2), both
     // K-major (bits 15, 16 = 0), N >> 3 at bits 17-22, M >> 4 at bits 24-28.
     g.idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(tn >> 3) << 17) | ((unsigned)(kHwTileM >> 4) << 24);
@@ -511,7 +525,7 @@ tt_status tt_default_schedule(const tt_workload* w, tt_schedule_record* out) {
     r.origin_op = w->op;
     r.origin = w->sh;
     // One generic, shape-blind record per family: the counterpart of a compiler's default schedule.
-    r.tile_m = 128; r.tile_n = 128; r.tile_k = 32; r.stages = 4; r.split_k = 1; r.raster = 0;
+    r.tile_m = 128; r.tile_n = 128; r.tile_k = 32; r.stages = 4; r.split_k = 1; r.raster = 0; r.acc_split = 1;
     r.block_x = 32; r.block_y = 4; r.items_per_thread = 1; r.vec_width = 1; r.unroll = 1; r.threads = 128;
     if (w->family == TT_FAMILY_DW_SIMT) { r.tile_m = 1; r.block_x = 32; r.block_y = 8; r.items_per_thread = 4; r.unroll = 2; }
     if (w->family == TT_FAMILY_ROW_SIMT) { r.block_x = 32; r.block_y = 4; }

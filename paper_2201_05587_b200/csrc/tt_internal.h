@@ -42,6 +42,8 @@ struct GemmArgs {
     unsigned* counters;                         // split-K arrival counters [batch][tiles], zero between launches
     unsigned* status;
     unsigned idesc, tmem_cols;
+    int cluster;                                // > 0: split-K over a thread-block cluster of this many CTAs (= split_k)
+    int n_acc;                                  // accumulators of tile_n columns each, reduction steps dealt round-robin
     unsigned a_stage_bytes, b_stage_bytes, tx_bytes;
     unsigned ktab_off;                          // im2col k-table: byte offset from the aligned tile base
     int vec_store;                              // bit 0: y rows allow aligned float4 stores; bit 1: so does bias

@@ -90,6 +90,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return mbar_wait_slow(bar, parity, abort_flag, status, where);
 }
 
+// One lane of a converged warp (the same lane every time): it issues the warp's asynchronous instructions.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0u;
+}
+
 __device__ __forceinline__ void fence_proxy_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -146,11 +157,25 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, int row_bytes) {
     return d;
 }
 
+// GELU in its erf form, 0.5 x (1 + erf(x / sqrt 2)).  erf through the rational approximation 7.1.26 of Abramowitz and
+// Stegun (absolute error below 1.5e-7, far inside what a TF32 product carries): a dozen instructions instead of
+// the library routine's, which matters in a read-out that is a long serial instruction stream per thread.
+__device__ __forceinline__ float gelu_erf(float x) {
+    const float z = fabsf(x) * 0.70710678118654752440f;
+    const float t = __fdividef(1.f, fmaf(0.3275911f, z, 1.f));
+    float poly = fmaf(1.061405429f, t, -1.453152027f);
+    poly = fmaf(poly, t, 1.421413741f);
+    poly = fmaf(poly, t, -0.284496736f);
+    poly = fmaf(poly, t, 0.254829592f);
+    const float erf_abs = 1.f - poly * t * __expf(-z * z);
+    return 0.5f * x * (1.f + copysignf(erf_abs, x));
+}
+
 __device__ __forceinline__ float apply_act(float v, int act) {
     switch (act) {
         case TT_ACT_RELU: return fmaxf(v, 0.f);
         case TT_ACT_RELU6: return fminf(fmaxf(v, 0.f), 6.f);
-        case TT_ACT_GELU_ERF: return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f));
+        case TT_ACT_GELU_ERF: return gelu_erf(v);
         default: return v;
     }
 }
@@ -210,6 +235,31 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
+// Thread-block cluster primitives (split-K over a cluster: the splits of one output tile are the CTAs of a cluster
+// and exchange their partial tiles through distributed shared memory).
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_peer(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float ld_peer_f32(uint32_t caddr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(caddr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_peer_v4(uint32_t caddr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(caddr) : "memory");
+    return v;
+}
+// A parked partial tile is laid out along the direction in which the output is contiguous, so that both the
+// remote 16-byte loads of the reduction and the global stores are contiguous across lanes:
+//   outputs contiguous along columns: [row][col], pitch tile_n + 4 floats;  along rows: [col][row], pitch 132 floats.
+constexpr int kRedColPitch = kHwTileM + 4;
+
 // All gather threads meet and learn whether every one of them is still healthy (named barrier 1).
 __device__ __forceinline__ bool gather_vote(bool ok) {
     uint32_t all;
@@ -264,6 +314,41 @@ __device__ __forceinline__ void expand_stage(uint32_t tile_smem, int rows, uint3
     const uint32_t atom_bytes = (uint32_t)rows * (uint32_t)row_bytes;
     const int n_rb = (rows + 31) >> 5;
     const int n_tasks = n_rb * (tile_k >> 2);
+    if ((kGatherWarps % n_rb) == 0) {
+        // 1, 2, 4 or 8 row blocks: a warp keeps one row block for the whole stage, so its pixel's window origin and
+        // the row part of the destination are loop-invariant; it takes every (8 / n_rb)-th chunk of four k
+        const int rb = gw % n_rb, step = kGatherWarps / n_rb, n_ch = tile_k >> 2;
+        const int row = rb * 32 + lane;
+        const bool in_tile = row < rows;
+        const uint32_t origin = slab + ld_shared_u32(rowoff_smem + 4u * (uint32_t)(in_tile ? row : rows - 1));
+        const uint32_t dst_row = tile_smem + (uint32_t)row * (uint32_t)row_bytes;
+        const uint32_t swz = (uint32_t)((row >> shift) & swz_mask) << 4;
+        constexpr int kB = 8;
+        for (int c0 = gw / n_rb; c0 < n_ch; c0 += step * kB) {
+            float val[kB][4];
+#pragma unroll
+            for (int b = 0; b < kB; ++b) {
+                const int ci = c0 + b * step;
+                if (ci < n_ch) {                         // warp-uniform
+                    const uint4 e = ld_shared_v4u(ktab_smem + 16u * (uint32_t)ci);   // same address in every lane
+                    val[b][0] = ld_shared_f32(origin + e.x);
+                    val[b][1] = ld_shared_f32(origin + e.y);
+                    val[b][2] = ld_shared_f32(origin + e.z);
+                    val[b][3] = ld_shared_f32(origin + e.w);
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < kB; ++b) {
+                const int ci = c0 + b * step;
+                if (ci < n_ch && in_tile) {
+                    const int kk = ci << 2;
+                    st_shared_v4(dst_row + (uint32_t)(kk >> atom_shift) * atom_bytes + ((uint32_t)((kk & (atom_k - 1)) << 2) ^ swz),
+                                 val[b][0], val[b][1], val[b][2], val[b][3]);
+                }
+            }
+        }
+        return;
+    }
     const uint32_t inv_rb = (65536u + (uint32_t)n_rb - 1u) / (uint32_t)n_rb;     // t / n_rb == (t * inv_rb) >> 16 for small t
     constexpr int kBatch = 4;
     for (int t0 = gw; t0 < n_tasks; t0 += kGatherWarps * kBatch) {
@@ -404,7 +489,7 @@ struct EpiArgs {
 };
 
 __device__ __forceinline__ float finish_one(float v, const EpiArgs& e) {
-    if (e.gelu) return 0.5f * v * (1.f + erff(v * 0.70710678118654752440f));     // uniform per kernel
+    if (e.gelu) return gelu_erf(v);              // uniform per kernel
     return fminf(fmaxf(v, e.lo), e.hi);
 }
 
@@ -479,7 +564,9 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __shared__ __align__(16) float s_bias[256];
     __shared__ int s_rowoff[256];
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the warp index is broadcast from lane 0 so that the compiler knows it is the same in all lanes of a warp and
+    // keeps the role loops (addresses, descriptors, counters) on the uniform datapath
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     volatile int* abortp = &abort_flag;
 #ifdef TT_PHASE_TIMERS
     if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
@@ -529,34 +616,45 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const uint32_t tmem_base = *(volatile uint32_t*)&tmem_slot;
     if (threadIdx.x == 0) TT_STAMP(1);
 
+    // Warps 0 and 1 run their loops with all 32 lanes: waits, counters and descriptor arithmetic stay
+    // warp-uniform, and one elected lane issues the asynchronous instructions.
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        if (lane == 0 && any_tma) {
+        if (any_tma) {
             int armed = 0;   // stages whose loads were issued
             uint32_t st = 0, ph = 0;
             const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
             const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes), b_atom = (uint32_t)(g.tile_n * g.row_bytes);
             const int a_bz = g.a_tma_batched ? bz : 0, b_bz = g.b_tma_batched ? bz : 0;
+            const bool leader = elect_one();             // this lane arms the barrier and issues every load
             int k0 = kt_begin * g.tile_k;
+            uint32_t a_stage = tiles_base, full_addr = full0, empty_addr = empty0;
             for (int it = 0; it < iters; ++it, k0 += g.tile_k) {
-                if (!mbar_wait(empty0 + st * 8u, ph ^ 1u, abortp, g.status, 1u)) break;
-                const uint32_t fb = full0 + st * 8u;
-                mbar_expect_tx(fb, g.tx_bytes);
-                const uint32_t a_s = tiles_base + st * stage_bytes, b_s = a_s + g.a_stage_bytes;
-                if (a_tma) {
+                const bool got = mbar_wait(empty_addr, ph ^ 1u, abortp, g.status, 1u);
+                if (!__all_sync(0xffffffffu, got)) break;
+                if (leader) {
+                    mbar_expect_tx(full_addr, g.tx_bytes);
+                    if (a_tma) {
+                        uint32_t dst = a_stage;
+                        int kc = k0;
 #pragma unroll 1
-                    for (int at = 0; at < g.n_atoms; ++at) tma_load_3d(a_s + at * a_atom, &tmap_a, fb, k0 + at * g.atom_k, m0, a_bz);
-                }
-                if (b_tma) {
+                        for (int at = 0; at < g.n_atoms; ++at, dst += a_atom, kc += g.atom_k) tma_load_3d(dst, &tmap_a, full_addr, kc, m0, a_bz);
+                    }
+                    if (b_tma) {
+                        uint32_t dst = a_stage + g.a_stage_bytes;
+                        int kc = k0;
 #pragma unroll 1
-                    for (int at = 0; at < g.n_atoms; ++at) tma_load_3d(b_s + at * b_atom, &tmap_b, fb, k0 + at * g.atom_k, n0, b_bz);
+                        for (int at = 0; at < g.n_atoms; ++at, dst += b_atom, kc += g.atom_k) tma_load_3d(dst, &tmap_b, full_addr, kc, n0, b_bz);
+                    }
                 }
+                __syncwarp();
                 armed = it + 1;
-                if (it == 5) TT_STAMP(10);
-                if (it == 6) TT_STAMP(11);
-                if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
+                if (lane == 0 && it == 5) TT_STAMP(10);
+                if (lane == 0 && it == 6) TT_STAMP(11);
+                a_stage += stage_bytes; full_addr += 8u; empty_addr += 8u;
+                if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; a_stage = tiles_base; full_addr = full0; empty_addr = empty0; }
             }
-            if (*abortp) {
+            if (*abortp && lane == 0) {
                 // let copies in flight land before shared memory is given back (bounded)
                 const int first = max(0, armed - g.stages);
                 for (int it = first; it < armed; ++it) {
@@ -566,10 +664,11 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                 }
             }
+            __syncwarp();
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+        {
             bool ok = true;
             uint32_t st = 0, ph = 0;
             const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
@@ -582,31 +681,61 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const uint32_t stage_step = stage_bytes >> 4;
             const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes) >> 4, b_atom = (uint32_t)(g.tile_n * g.row_bytes) >> 4;
             const int k8_per_atom = g.atom_k >> 3;
-            const int k8_shift = k8_per_atom == 4 ? 2 : (k8_per_atom == 2 ? 1 : 0);
-            const int n_mma = g.tile_k >> 3;
-            uint32_t accumulate = 0u;
+            const uint32_t a_next_atom = a_atom - 2u * (uint32_t)k8_per_atom, b_next_atom = b_atom - 2u * (uint32_t)k8_per_atom;
+            const bool leader = elect_one();             // this lane issues every multiply-accumulate and every commit
+            // accumulators: reduction steps are dealt round-robin; an accumulator's first step overwrites
+            uint32_t d_tmem = tmem_base;
+            const uint32_t d_end = tmem_base + (uint32_t)(g.n_acc * g.tile_n);
+            int fresh = g.n_acc;                         // accumulators not written yet
+            uint32_t a_stage = a_lo0, b_stage = b_lo0, full_addr = full0, empty_addr = empty0;
             for (int it = 0; it < iters; ++it) {
-                if (!mbar_wait(full0 + st * 8u, ph, abortp, g.status, 2u)) { ok = false; break; }
-                if (it == 0) TT_STAMP(2);
-                if (it == 5) TT_STAMP(12);
-                if (it == 6) TT_STAMP(13);
+                const bool got = mbar_wait(full_addr, ph, abortp, g.status, 2u);
+                if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+                if (lane == 0 && it == 0) TT_STAMP(2);
+                if (lane == 0 && it == 5) TT_STAMP(12);
+                if (lane == 0 && it == 6) TT_STAMP(13);
                 tc_fence_after();
-                const uint32_t a_lo = a_lo0 + st * stage_step, b_lo = b_lo0 + st * stage_step;
+                if (leader) {
+                    // descriptors step by 2 (32 bytes = 8 TF32 along K) inside a swizzle atom, then to the next atom
+                    uint32_t a_lo = a_stage, b_lo = b_stage;
+                    if (g.n_acc == 1) {
+                        // one accumulator: nothing to rotate
+                        uint32_t accumulate = it > 0 ? 1u : 0u;
+#pragma unroll 1
+                        for (int at = 0; at < g.n_atoms; ++at) {
 #pragma unroll 4
-                for (int i8 = 0; i8 < n_mma; ++i8) {
-                    const uint32_t at = (uint32_t)i8 >> k8_shift, k8 = (uint32_t)i8 & (uint32_t)(k8_per_atom - 1);
-                    // 8 TF32 = 32 bytes further along K inside the swizzle atom: start address + 2 (16-byte units)
-                    const uint64_t ad = ((uint64_t)d_hi << 32) | (uint64_t)(a_lo + at * a_atom + k8 * 2u);
-                    const uint64_t bd = ((uint64_t)d_hi << 32) | (uint64_t)(b_lo + at * b_atom + k8 * 2u);
-                    mma_tf32(tmem_base, ad, bd, g.idesc, accumulate);
-                    accumulate = 1u;
+                            for (int k8 = 0; k8 < k8_per_atom; ++k8) {
+                                mma_tf32(tmem_base, ((uint64_t)d_hi << 32) | (uint64_t)a_lo, ((uint64_t)d_hi << 32) | (uint64_t)b_lo, g.idesc,
+                                         accumulate);
+                                accumulate = 1u;
+                                a_lo += 2u; b_lo += 2u;
+                            }
+                            a_lo += a_next_atom; b_lo += b_next_atom;
+                        }
+                    } else
+#pragma unroll 1
+                    for (int at = 0; at < g.n_atoms; ++at) {
+#pragma unroll 4
+                        for (int k8 = 0; k8 < k8_per_atom; ++k8) {
+                            mma_tf32(d_tmem, ((uint64_t)d_hi << 32) | (uint64_t)a_lo, ((uint64_t)d_hi << 32) | (uint64_t)b_lo, g.idesc,
+                                     fresh > 0 ? 0u : 1u);
+                            a_lo += 2u; b_lo += 2u;
+                            if (fresh > 0) --fresh;
+                            d_tmem += (uint32_t)g.tile_n;
+                            if (d_tmem == d_end) d_tmem = tmem_base;
+                        }
+                        a_lo += a_next_atom; b_lo += b_next_atom;
+                    }
+                    mma_commit(empty_addr);              // stage reusable once these MMAs have read it
                 }
-                mma_commit(empty0 + st * 8u);            // stage reusable once these MMAs have read it
-                if (it == 5) TT_STAMP(14);
-                if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
+                __syncwarp();
+                if (lane == 0 && it == 5) TT_STAMP(14);
+                a_stage += stage_step; b_stage += stage_step; full_addr += 8u; empty_addr += 8u;
+                if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; a_stage = a_lo0; b_stage = b_lo0; full_addr = full0; empty_addr = empty0; }
             }
-            if (ok) mma_commit(smem_u32(&accum_bar));    // accumulator complete
-            TT_STAMP(3);
+            if (ok && leader) mma_commit(smem_u32(&accum_bar));    // accumulator complete
+            __syncwarp();
+            if (lane == 0) TT_STAMP(3);
         }
     } else {
         // ---------------- gather producers, then epilogue ----------------
@@ -658,6 +787,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             for (uint32_t o = (uint32_t)gt * 16u; o < slab_bytes; o += (uint32_t)kGatherThreads * 16u)
                 st_shared_v4(slab0 + o, 0.f, 0.f, 0.f, 0.f);
             bool ok = gather_vote(true);                 // tables and zeros are in place before any copy lands
+            if (threadIdx.x == 64) TT_STAMP(17);
             const int n_chunks = (iters + T - 1) / T;
             auto chunk_load = [&](int j) {
                 const int k_lo = kbeg + j * T * g.tile_k;
@@ -671,6 +801,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             };
             chunk_load(0);
             if (n_chunks > 1) chunk_load(1);
+            if (threadIdx.x == 64) TT_STAMP(18);
             const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
             uint32_t st = 0, ph = 0;
             for (int j = 0; j < n_chunks; ++j) {
@@ -747,11 +878,44 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int half = gw >> 2;
             const bool m_ok = m < g.M;
             const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16);
-            const bool split_mode = g.split_k > 1;
+            const bool split_mode = g.split_k > 1 && g.cluster == 0;   // splits beyond a cluster go through the workspace
+            // a split with fewer reduction steps than accumulators leaves the last ones unwritten
+            const int n_acc = min(g.n_acc, iters * (g.tile_k >> 3));
             // split-K workspace [split][batch][N][M]: a column of the tile is contiguous across lanes
             const long long per_split = (long long)g.batch * g.M * (long long)g.N;
             float* pcol = g.partial + (long long)bz * g.M * (long long)g.N + m;
-            if (split_mode) {
+            if (g.cluster) {
+                // split-K over a cluster: park this split's partial tile in its own shared memory (the pipeline
+                // buffers are idle now), column-major with a padded pitch; the reduction follows the cluster barrier
+#pragma unroll 1
+                for (int c0 = half * 32; c0 < g.tile_n; c0 += 64) {
+                    uint32_t r[32];
+                    tmem_ld32(t_row + (uint32_t)c0, r);
+                    tmem_wait_ld();
+#pragma unroll 1
+                    for (int j = 1; j < n_acc; ++j) {        // the other accumulators, in fixed order
+                        uint32_t t2[32];
+                        tmem_ld32(t_row + (uint32_t)(j * g.tile_n + c0), t2);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(t2[i]));
+                    }
+                    const int row = quad * 32 + lane;
+                    if (g.y_ns == 1) {
+                        const uint32_t dst = tiles_base + 4u * (uint32_t)(row * (g.tile_n + 4) + c0);
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            if (c0 + j < g.tile_n)           // tile_n is a multiple of 16: groups of four are whole
+                                st_shared_v4(dst + 4u * (uint32_t)j, __uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                             __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                    } else {
+                        const uint32_t dst = tiles_base + 4u * (uint32_t)(c0 * kRedColPitch + row);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (c0 + j < g.tile_n) st_shared_u32(dst + 4u * (uint32_t)(j * kRedColPitch), r[j]);
+                    }
+                }
+            } else if (split_mode) {
                 // 1. park this split's partial tile in the workspace
                 float* pmine = pcol + (long long)split * per_split;
 #pragma unroll 1
@@ -759,6 +923,14 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     uint32_t r[32];
                     tmem_ld32(t_row + (uint32_t)c0, r);
                     tmem_wait_ld();
+#pragma unroll 1
+                    for (int j = 1; j < n_acc; ++j) {        // the other accumulators, in fixed order
+                        uint32_t t2[32];
+                        tmem_ld32(t_row + (uint32_t)(j * g.tile_n + c0), t2);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(t2[i]));
+                    }
                     const int nb = n0 + c0;
                     const int cnt = min(g.N - nb, g.tile_n - c0);
                     if (!m_ok || cnt <= 0) continue;
@@ -778,7 +950,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 asm volatile("bar.sync 1, %0;" ::"n"(kGatherThreads) : "memory");
             }
-            const bool finish = !split_mode || (*(volatile int*)&last_split_flag != 0);
+            const bool finish = g.cluster == 0 && (!split_mode || (*(volatile int*)&last_split_flag != 0));
             if (finish) {
                 if (split_mode) __threadfence();
                 EpiArgs e;
@@ -807,6 +979,13 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         if (threadIdx.x == 64 && c0 == 0) TT_STAMP(7);
 #pragma unroll
                         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+#pragma unroll 1
+                        for (int a = 1; a < n_acc; ++a) {        // the other accumulators, in fixed order
+                            tmem_ld32(t_row + (uint32_t)(a * g.tile_n + c0), r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] += __uint_as_float(r[j]);
+                        }
                         if (c0 + 64 < g.tile_n) tmem_ld32(t_row + (uint32_t)(c0 + 64), r);
                     } else {
 #pragma unroll
@@ -838,7 +1017,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         // no residual: activate here, once, outside the store loops
                         if (e.gelu) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) v[j] = 0.5f * v[j] * (1.f + erff(v[j] * 0.70710678118654752440f));
+                            for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] = fminf(fmaxf(v[j], e.lo), e.hi);
@@ -853,6 +1032,77 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             }
         }
+    }
+    if (g.cluster) {
+        // ---------------- split-K over the cluster: reduce through distributed shared memory ----------------
+        // Every thread of every CTA of the cluster takes part in both barriers, also after a tripped wait.
+        if (threadIdx.x == 64) TT_STAMP(19);
+        cluster_sync_all();                              // all partial tiles are parked
+        if (threadIdx.x == 64) TT_STAMP(20);
+        if (warp >= 2) {
+            const int gw = warp - 2;
+            const int sk = g.split_k;
+            uint32_t peer[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) peer[q] = map_to_peer(tiles_base, (uint32_t)(q < sk ? q : 0));
+            float* ybase = g.y + (long long)bz * g.y_bs;
+            const float* rbase = g.residual ? g.residual + (long long)bz * g.y_bs : nullptr;
+            const float lo = g.act == TT_ACT_NONE || g.act == TT_ACT_GELU_ERF ? -INFINITY : 0.f;
+            const float hi = g.act == TT_ACT_RELU6 ? 6.f : INFINITY;
+            const bool gelu = g.act == TT_ACT_GELU_ERF;
+            // four outputs that are neighbours in memory: one 16-byte load per split (all issued before the first
+            // addition; partial sums are added in split order), the fused tail, one 16-byte store where alignment allows
+            const bool along_cols = g.y_ns == 1;
+            const long long lead = along_cols ? g.y_ms : g.y_ns;       // stride of the other output axis
+            const bool vec_ok = (lead & 3) == 0 && (g.y_bs & 3) == 0 && (reinterpret_cast<uintptr_t>(ybase) & 15u) == 0 &&
+                                (rbase == nullptr || (reinterpret_cast<uintptr_t>(rbase) & 15u) == 0);
+            auto finish4 = [&](uint32_t off, int mm, int nn, int valid) {
+                float4 p[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (q < sk) p[q] = ld_peer_v4(peer[q] + off);
+                float4 acc = p[0];
+#pragma unroll
+                for (int q = 1; q < 8; ++q)
+                    if (q < sk) { acc.x += p[q].x; acc.y += p[q].y; acc.z += p[q].z; acc.w += p[q].w; }
+                float v[4] = {acc.x, acc.y, acc.z, acc.w};
+                const long long o = (long long)mm * g.y_ms + (long long)nn * g.y_ns;   // the four are o, o+1, o+2, o+3
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (i < valid) {
+                        if (g.bias_mode == 1) v[i] += __ldg(g.bias + mm + (along_cols ? 0 : i));
+                        else if (g.bias_mode == 2) v[i] += __ldg(g.bias + nn + (along_cols ? i : 0));
+                        if (rbase) v[i] += __ldg(rbase + o + i);
+                        v[i] = gelu ? gelu_erf(v[i]) : fminf(fmaxf(v[i], lo), hi);
+                    }
+                }
+                if (valid == 4 && vec_ok) *reinterpret_cast<float4*>(ybase + o) = make_float4(v[0], v[1], v[2], v[3]);
+                else {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        if (i < valid) ybase[o + i] = v[i];
+                }
+            };
+            if (along_cols) {
+                // each CTA finishes a band of rows; a warp takes a row, its lanes walk the columns four at a time
+                const int per = (kHwTileM + sk - 1) / sk;
+                const int r_end = min(min(kHwTileM, (split + 1) * per), g.M - m0);
+                const int c_end = min(g.tile_n, g.N - n0);
+                for (int row = split * per + gw; row < r_end; row += kGatherWarps)
+                    for (int col = lane * 4; col < c_end; col += 128)
+                        finish4(4u * (uint32_t)(row * (g.tile_n + 4) + col), m0 + row, n0 + col, min(4, c_end - col));
+            } else {
+                // each CTA finishes a band of columns; a warp takes a column, its lanes walk the 128 rows four at a time
+                const int per = (g.tile_n + sk - 1) / sk;
+                const int c_end = min(min(g.tile_n, (split + 1) * per), g.N - n0);
+                const int r_end = min(kHwTileM, g.M - m0);
+                for (int col = split * per + gw; col < c_end; col += kGatherWarps)
+                    if (lane * 4 < r_end)
+                        finish4(4u * (uint32_t)(col * kRedColPitch + lane * 4), m0 + lane * 4, n0 + col, min(4, r_end - lane * 4));
+            }
+        }
+        if (threadIdx.x == 64) TT_STAMP(21);
+        cluster_sync_all();                              // nobody leaves while a peer may still read its tile
     }
     if (threadIdx.x == 64) TT_STAMP(5);
     tc_fence_before();
@@ -1098,8 +1348,35 @@ cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* t
     memcpy(&ta, tmap_a, sizeof ta);
     memcpy(&tb, tmap_b, sizeof tb);
     dim3 grid(I.grid_x, I.grid_y, I.grid_z);
+    if (g.cluster) {
+        // the splits of one output tile (grid.y) form a thread-block cluster
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = grid; cfg.blockDim = dim3(kGemmThreads, 1, 1); cfg.dynamicSmemBytes = (size_t)I.smem_bytes; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)g.cluster; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, tt_gemm_tc_kernel, ta, tb, g);
+    }
     tt_gemm_tc_kernel<<<grid, kGemmThreads, I.smem_bytes, st>>>(ta, tb, g);
     return cudaGetLastError();
+}
+
+// Can a cluster of `cluster` CTAs with this much shared memory each be resident at all?
+cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits) {
+    cudaError_t e = cudaFuncSetAttribute(tt_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemLimit);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(1, (unsigned)cluster, 1); cfg.blockDim = dim3(kGemmThreads, 1, 1); cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)cluster; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    e = cudaOccupancyMaxActiveClusters(&n, tt_gemm_tc_kernel, &cfg);
+    if (e != cudaSuccess) return e;
+    *fits = n > 0;
+    return cudaSuccess;
 }
 
 cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st) {

@@ -43,24 +43,25 @@ def _both_paths(spec, rec, seed):
 
 
 def test_static_scratch_matches_allocating_path_twice_in_a_row():
-    rec = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=64, tile_k=32, stages=3, split_k=6, mma_m_axis=1)
+    # more than 8 splits, so that the partial sums go through scratch memory (fewer reduce inside a cluster)
+    rec = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=64, tile_k=32, stages=3, split_k=12, mma_m_axis=1)
     _both_paths(W._dense(96, 1500, 200, act=B.TT_ACT_RELU, name="static_a"), rec, seed=41)
     # second call: other sizes and split count, the array still holds the first call's partial sums
-    rec2 = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=128, tile_k=64, stages=2, split_k=3, mma_m_axis=2)
-    _both_paths(W._dense(40, 700, 333, act=B.TT_ACT_NONE, name="static_b"), rec2, seed=42)
+    rec2 = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=128, tile_k=16, stages=2, split_k=11, mma_m_axis=2)
+    _both_paths(W._dense(40, 704, 333, act=B.TT_ACT_NONE, name="static_b"), rec2, seed=42)
     # and the first case again, after a differently shaped one
     _both_paths(W._dense(96, 1500, 200, act=B.TT_ACT_RELU, name="static_a"), rec, seed=43)
 
 
 def test_static_scratch_rejects_what_does_not_fit():
     import torch
-    # 2048 x 2048 outputs x 8 splits x 4 bytes = 128 MB of partial sums: far beyond the fixed array
+    # 2048 x 2048 outputs x 16 splits x 4 bytes = 256 MB of partial sums: far beyond the fixed array
     m = nn = 2048
     kk = 512
     x = torch.zeros(m, kk, device="cuda")
     w = torch.zeros(nn, kk, device="cuda")
     y = torch.zeros(m, nn, device="cuda")
-    rec = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=128, tile_k=32, stages=2, split_k=8, mma_m_axis=1)
+    rec = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=128, tile_k=32, stages=2, split_k=16, mma_m_axis=1)
     st, used = B.dense_static_scratch(x, w, None, y, B.TT_ACT_NONE, rec)
     assert st == B.TT_ERR_RESOURCE
     assert used > B.TT_STATIC_SCRATCH_BYTES
