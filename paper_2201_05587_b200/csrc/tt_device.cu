@@ -10,7 +10,8 @@
 
 namespace tt {
 
-cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, cudaStream_t st);
+cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, const void* tmap_x,
+                        cudaStream_t st);
 cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st);
 cudaError_t launch_row(const tt_apply_info& I, const RowArgs& row, cudaStream_t st);
 cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits);
@@ -65,6 +66,22 @@ tt_status encode_operand(void* out, const float* base, int K, int rows, int batc
     return r == CUDA_SUCCESS ? TT_OK : TT_ERR_CUDA;
 }
 
+// NCHW image -> 4-D tensor map (W, H, C, N) without swizzle; box = [W + gap, in_rows, box_ch, 1].  A load that
+// starts `gap` columns left of the image and at any (also negative) row gets zeros for everything outside.
+tt_status encode_image(void* out, const float* base, int W, int H, int C, int N, int box_w, int box_h, int box_c) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return TT_ERR_CUDA;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0) return TT_ERR_INVALID_ARG;
+    cuuint64_t dims[4] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)C, (cuuint64_t)N};
+    cuuint64_t strides[3] = {(cuuint64_t)W * 4, (cuuint64_t)W * H * 4, (cuuint64_t)W * H * C * 4};
+    cuuint32_t box[4] = {(cuuint32_t)box_w, (cuuint32_t)box_h, (cuuint32_t)box_c, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(base), dims,
+                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? TT_OK : TT_ERR_CUDA;
+}
+
 const void* pick(const tt_tensors* t, int which) { return which == 0 ? t->x : t->w; }
 
 }  // namespace
@@ -72,6 +89,8 @@ const void* pick(const tt_tensors* t, int which) { return which == 0 ? t->x : t-
 void release_device(tt_workload* w) {
     if (w->workspace) cudaFree(w->workspace);
     if (w->status_word) cudaFree(w->status_word);
+    if (w->ktab_dev) cudaFree(w->ktab_dev);
+    w->ktab_dev = nullptr; w->ktab_bytes = 0;
     for (int i = 0; i < 5; ++i) if (w->hbuf[i]) cudaFree(w->hbuf[i]);
     w->workspace = nullptr; w->workspace_bytes = 0; w->status_word = nullptr;
     for (int i = 0; i < 5; ++i) { w->hbuf[i] = nullptr; w->hbytes[i] = 0; }
@@ -102,6 +121,30 @@ tt_status bind_device(tt_workload* w) {
         if (cudaMalloc(reinterpret_cast<void**>(&w->status_word), 512) != cudaSuccess) { cudaGetLastError(); return TT_ERR_OOM; }
         if (cudaMemset(w->status_word, 0, 512) != cudaSuccess) return TT_ERR_CUDA;
     }
+    if (w->op == TT_OP_CONV2D) {
+        // reduction-index table of the applied record: byte offset of (c, r, s) inside the slab, channel counted
+        // from 0 (the kernel rebases it per chunk); indices past K point at the last channel, whose products meet
+        // zero-filled filter values
+        const GemmArgs& g = w->plan.g;
+        const int kpad = g.k_tiles * g.tile_k, RS = g.R * g.S;
+        std::vector<int> tab((size_t)kpad);
+        for (int k = 0; k < kpad; ++k) {
+            if (k < g.K) {
+                const int c = k / RS, rem = k - c * RS, fr = rem / g.S, fs = rem - fr * g.S;
+                tab[k] = 4 * (c * g.slab_chpitch + fr * g.slab_wp + fs);
+            } else {
+                tab[k] = 4 * ((g.C - 1) * g.slab_chpitch);
+            }
+        }
+        const size_t bytes = (size_t)kpad * 4;
+        if (bytes > w->ktab_bytes) {
+            if (w->ktab_dev) cudaFree(w->ktab_dev);
+            w->ktab_dev = nullptr; w->ktab_bytes = 0;
+            if (cudaMalloc(reinterpret_cast<void**>(&w->ktab_dev), bytes) != cudaSuccess) { cudaGetLastError(); return TT_ERR_OOM; }
+            w->ktab_bytes = bytes;
+        }
+        if (cudaMemcpy(w->ktab_dev, tab.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    }
     w->tmaps.clear();
     return TT_OK;
 }
@@ -123,6 +166,12 @@ static tt_status tensor_maps_for(tt_workload* w, const void* a_ptr, const void* 
         st = encode_operand(e.b, static_cast<const float*>(b_ptr), g.K, g.N, g.batch, g.b_rs, g.b_bs, g.b_tma_batched != 0,
                             g.atom_k, g.tile_n);
     if (st != TT_OK) return st;
+    if (g.slab_tma) {
+        const float* img = static_cast<const float*>(g.a_mode == OPM_IM2COL ? a_ptr : b_ptr);
+        if ((reinterpret_cast<uintptr_t>(img) & 15u) != 0) return TT_ERR_INVALID_ARG;   // images must be 16-byte aligned
+        st = encode_image(e.x, img, g.W, g.H, g.C, g.batch, g.slab_wp, g.slab_in_rows, g.slab_box_ch);
+        if (st != TT_OK) return st;
+    }
     if (w->tmaps.size() >= 4096) w->tmaps.clear();
     w->tmaps.push_back(e);
     *out = &w->tmaps.back();
@@ -157,7 +206,8 @@ tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
         if ((reinterpret_cast<uintptr_t>(t->y) & 15u) != 0 ||
             (g.residual && (reinterpret_cast<uintptr_t>(g.residual) & 15u) != 0)) g.vec_store = 0;
         if (g.bias && (reinterpret_cast<uintptr_t>(g.bias) & 15u) == 0) g.vec_store |= 2;
-        e = launch_gemm(p.info, g, maps->a, maps->b, st);
+        g.ktab_dev = w->ktab_dev;
+        e = launch_gemm(p.info, g, maps->a, maps->b, maps->x, st);
     } else if (w->family == TT_FAMILY_DW_SIMT) {
         DwArgs d = p.dw;
         d.x = static_cast<const float*>(t->x); d.w = static_cast<const float*>(t->w);
@@ -595,7 +645,7 @@ extern "C" tt_status tt_dense_static_scratch(const void* x, const void* w, const
     if (s == TT_OK && g.b_mode == OPM_TMA)
         s = encode_operand(maps.b, g.b, g.K, g.N, g.batch, g.b_rs, g.b_bs, g.b_tma_batched != 0, g.atom_k, g.tile_n);
     if (s != TT_OK) return s;
-    if (launch_gemm(plan.info, g, maps.a, maps.b, st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    if (launch_gemm(plan.info, g, maps.a, maps.b, maps.x, st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
     if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
     unsigned v = 0;
     if (cudaMemcpy(&v, base, 4, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }

@@ -150,7 +150,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     const int cluster = (sk >= 2 && sk <= 8) ? sk : 0;
     const long long min_pipe = std::max<long long>((long long)kGatherWarps * 32 * 36 * 4, cluster ? std::max<long long>((long long)tn * (kHwTileM + 4) * 4, (long long)kHwTileM * (tn + 4) * 4) : 0);
     const bool conv = w->op == TT_OP_CONV2D;
-    const long long ktab = conv ? (((long long)per_split * tk * 4 + 15) / 16) * 16 : 0;
+    const long long ktab = conv ? (((long long)per_split * tk * 4 + 127) / 128) * 128 : 0;
     int sl_tiles = 0, sl_nbuf = 0, sl_wp = 0, sl_gap = 0, sl_chpitch = 0, sl_in_rows = 0, sl_rstep = 1;
     long long sl_buf_bytes = 0, chp = 0;
     const int RS = conv ? s.r * s.s : 1;
@@ -167,9 +167,13 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
         if (chp * (long long)s.c >= (1ll << 28) || s.w > 4095 || sl_in_rows > 4095) return TT_ERR_RESOURCE;
         sl_chpitch = (int)chp;
     }
+    // TMA can stage the slab when image rows are 16-byte multiples and consecutive slab rows are consecutive image
+    // rows; a chunk is then one box of at most 256 channels
+    const bool slab_tma = conv && (s.w % 4) == 0 && s.stride_h <= s.r && sl_wp <= 256 && sl_in_rows <= 256;
+    auto chunk_channels = [&](long long tiles) { return std::min<long long>(s.c, (tiles * tk + RS - 2) / RS + 1); };
     auto chunk_bytes = [&](long long tiles) {
-        const long long ch = std::min<long long>(s.c, (tiles * tk + RS - 2) / RS + 1);
-        return ((ch * chp + sl_gap + 4) * 4 + 15) / 16 * 16;
+        // a tail of gap + 4 zeros follows the last row of the last channel
+        return ((chunk_channels(tiles) * chp + sl_gap + 4) * 4 + 127) / 128 * 128;
     };
     long long smem = 0;
     for (;;) {
@@ -180,7 +184,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
             const long long budget = kDynSmemLimit - 1024 - pipe_try - ktab;
             // largest chunk not above the request that fits (one buffer if it covers the CTA's whole K range)
             int t = rec->slab_tiles == 0 ? per_split : std::min(rec->slab_tiles, per_split);
-            while (t >= 1 && (t >= per_split ? 1 : 2) * chunk_bytes(t) > budget) --t;
+            while (t >= 1 && ((t >= per_split ? 1 : 2) * chunk_bytes(t) > budget || (slab_tma && chunk_channels(t) > 256))) --t;
             fits = t >= 1;
             sl_tiles = std::max(t, 1);
             sl_nbuf = sl_tiles >= per_split ? 1 : 2;
@@ -237,6 +241,11 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     g.slab_buf_bytes = (unsigned)sl_buf_bytes; g.slab_nbuf = sl_nbuf; g.slab_tiles = sl_tiles;
     g.slab_wp = sl_wp; g.slab_gap = sl_gap; g.slab_chpitch = sl_chpitch; g.slab_in_rows = sl_in_rows;
     g.slab_rstep = sl_rstep;
+    g.slab_tma = slab_tma ? 1 : 0;
+    if (slab_tma) {
+        g.slab_box_ch = (int)chunk_channels(sl_tiles);
+        g.slab_box_bytes = (unsigned)((long long)g.slab_box_ch * chp * 4);
+    }
     g.magic_rstep = sl_rstep > 1 ? (unsigned)((0x100000000ull + sl_rstep - 1) / sl_rstep) : 0u;
     g.slab_vec16 = (s.w % 4) == 0;
     {

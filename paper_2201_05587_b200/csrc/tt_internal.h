@@ -56,7 +56,13 @@ struct GemmArgs {
     int slab_in_rows;                           // slab rows per channel (the most a tile can need)
     int slab_rstep;                             // slab rows per output row: min(stride_h, r)
     int slab_vec16;                             // rows copied 16 bytes at a time (W % 4 == 0 and x aligned)
-    unsigned magic_wpieces, magic_in_rows, magic_rstep;      // ceil(2^32 / d) for the exact small-range divisions of the slab loader
+    unsigned magic_wpieces, magic_in_rows, magic_rstep;
+    // slab by TMA (rows 16-byte aligned, stride <= filter height): a chunk is one box [box_ch channels][in_rows][W + gap]
+    // starting `gap` columns left of the image, so the hardware's zero fill writes the gaps and the rows outside
+    int slab_tma;                               // 1: chunks arrive by TMA; 0: by cp.async from the gather warps
+    int slab_box_ch;                            // channels per box
+    unsigned slab_box_bytes;
+    const int* ktab_dev;                        // per reduction index: byte offset of (c, r, s) inside the slab (absolute channel)      // ceil(2^32 / d) for the exact small-range divisions of the slab loader
 };
 
 struct DwArgs {
@@ -91,6 +97,7 @@ struct TmapPair {
     const void* a_ptr; const void* b_ptr;
     alignas(64) unsigned char a[128];
     alignas(64) unsigned char b[128];
+    alignas(64) unsigned char x[128];   // conv2d: the image as a (W, H, C, N) tensor, for the slab
 };
 
 }  // namespace tt
@@ -103,6 +110,8 @@ struct tt_workload {
     tt_gemm_view view;
     tt::Plan plan;
     void* workspace = nullptr;   // device: split-K partials
+    int* ktab_dev = nullptr;     // device: conv2d reduction-index table of the applied record
+    size_t ktab_bytes = 0;
     size_t workspace_bytes = 0;
     unsigned* status_word = nullptr;  // device
     // device staging buffers of tt_run_host

@@ -112,6 +112,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* tmap, uint
         ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
 __device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
 }
@@ -553,11 +559,14 @@ __device__ __forceinline__ void epilogue_block(float (&v)[32], const EpiArgs& e,
 // warp 0 TMA producer, warp 1 MMA issuer + tensor-memory owner, warps 2-9 gather producers, then epilogue.
 // ------------------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kGemmThreads, 1)
-tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const GemmArgs g) {
+tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                  const __grid_constant__ CUtensorMap tmap_x, const GemmArgs g) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages];
     __shared__ uint64_t empty_bar[kMaxStages];
     __shared__ uint64_t accum_bar;
+    __shared__ uint64_t slab_full[2];     // a slab chunk has landed (TMA)
+    __shared__ uint64_t slab_empty[2];    // all gather warps are done with a slab buffer
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int last_split_flag;
@@ -589,6 +598,15 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const bool a_tma = g.a_mode == OPM_TMA, b_tma = g.b_mode == OPM_TMA;
     const bool any_tma = a_tma || b_tma, any_gather = !a_tma || !b_tma;
     const bool im2col = g.a_mode == OPM_IM2COL || g.b_mode == OPM_IM2COL;
+    const bool slab_tma = im2col && g.slab_tma != 0;
+    // im2col geometry of this CTA: first output row of its pixels, the image row its slab starts at, slab chunks
+    int ic_p_first = 0, ic_ih_lo = 0, ic_chunks = 0;
+    if (im2col) {
+        const int row0 = g.a_mode == OPM_IM2COL ? m0 : n0;
+        ic_p_first = row0 / g.Q;
+        ic_ih_lo = ic_p_first * g.sh - g.ph;
+        ic_chunks = (iters + g.slab_tiles - 1) / g.slab_tiles;
+    }
     // gather groups (global gathers only): 4 groups of 2 warps from 4 stages up, 2 groups of 4 warps for 2-3 stages,
     // else one group; the im2col expansion keeps all eight warps on one stage
     const int n_groups = im2col ? 1 : (g.stages >= 4 ? 4 : (g.stages >= 2 ? 2 : 1));
@@ -601,6 +619,10 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             mbar_init(smem_u32(&empty_bar[s]), 1u);
         }
         mbar_init(smem_u32(&accum_bar), 1u);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&slab_full[b]), 1u);
+            mbar_init(smem_u32(&slab_empty[b]), (uint32_t)kGatherWarps);
+        }
         abort_flag = 0;
         last_split_flag = 0;
         fence_mbar_init();
@@ -620,18 +642,47 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // warp-uniform, and one elected lane issues the asynchronous instructions.
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        if (any_tma) {
+        if (any_tma || slab_tma) {
             int armed = 0;   // stages whose loads were issued
             uint32_t st = 0, ph = 0;
             const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
             const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes), b_atom = (uint32_t)(g.tile_n * g.row_bytes);
             const int a_bz = g.a_tma_batched ? bz : 0, b_bz = g.b_tma_batched ? bz : 0;
-            const bool leader = elect_one();             // this lane arms the barrier and issues every load
+            const bool leader = elect_one();             // this lane arms the barriers and issues every load
             int k0 = kt_begin * g.tile_k;
             uint32_t a_stage = tiles_base, full_addr = full0, empty_addr = empty0;
+            // conv2d: slab chunk j (the input rows behind reduction tiles j*T .. j*T+T-1) goes to buffer j & 1 as one
+            // box that starts `gap` columns left of the image: the zero fill writes gaps and rows outside the image
+            const int RS = g.R * g.S, T = g.slab_tiles;
+            const uint32_t slab0 = tiles_base + g.slab_off;
+            int slab_issued = 0;
+            auto issue_chunk = [&](int j) {
+                const uint32_t bar = smem_u32(&slab_full[j & 1]);
+                mbar_expect_tx(bar, g.slab_box_bytes);
+                tma_load_4d(slab0 + (uint32_t)(j & 1) * g.slab_buf_bytes, &tmap_x, bar, -g.slab_gap, ic_ih_lo,
+                            (kt_begin * g.tile_k + j * T * g.tile_k) / RS, bz);
+            };
+            if (slab_tma) {
+                if (leader) { issue_chunk(0); if (ic_chunks > 1) issue_chunk(1); }
+                slab_issued = min(ic_chunks, 2);
+            }
+            int next_slab_it = slab_tma ? T : 0x7fffffff;    // chunk `slab_issued` is requested when chunk slab_issued-1 starts
+            bool ok = true;
             for (int it = 0; it < iters; ++it, k0 += g.tile_k) {
+                if (it == next_slab_it) {
+                    next_slab_it += T;
+                    if (slab_issued < ic_chunks) {
+                        // its buffer is free once the gather warps have left chunk slab_issued - 2
+                        const int j = slab_issued;
+                        const bool freed = mbar_wait(smem_u32(&slab_empty[j & 1]), (uint32_t)((j - 2) >> 1) & 1u, abortp, g.status, 5u);
+                        if (!__all_sync(0xffffffffu, freed)) { ok = false; break; }
+                        if (leader) issue_chunk(j);
+                        ++slab_issued;
+                    }
+                }
+                if (!any_tma) continue;
                 const bool got = mbar_wait(empty_addr, ph ^ 1u, abortp, g.status, 1u);
-                if (!__all_sync(0xffffffffu, got)) break;
+                if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 if (leader) {
                     mbar_expect_tx(full_addr, g.tx_bytes);
                     if (a_tma) {
@@ -654,12 +705,18 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 a_stage += stage_bytes; full_addr += 8u; empty_addr += 8u;
                 if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; a_stage = tiles_base; full_addr = full0; empty_addr = empty0; }
             }
-            if (*abortp && lane == 0) {
+            if ((!ok || *abortp) && lane == 0) {
                 // let copies in flight land before shared memory is given back (bounded)
                 const int first = max(0, armed - g.stages);
                 for (int it = first; it < armed; ++it) {
                     const unsigned long long t0 = global_timer_ns();
                     while (!mbar_try_wait(smem_u32(&full_bar[it % g.stages]), (uint32_t)(it / g.stages) & 1u)) {
+                        if (global_timer_ns() - t0 > 2000000ull) break;
+                    }
+                }
+                for (int j = max(0, slab_issued - 2); j < slab_issued; ++j) {
+                    const unsigned long long t0 = global_timer_ns();
+                    while (!mbar_try_wait(smem_u32(&slab_full[j & 1]), (uint32_t)(j >> 1) & 1u)) {
                         if (global_timer_ns() - t0 > 2000000ull) break;
                     }
                 }
@@ -758,38 +815,40 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const uint32_t rowoff = smem_u32(s_rowoff);
             const int RS = g.R * g.S, T = g.slab_tiles;
             const int last = min(row0 + rows, ext) - 1;
-            const int p_first = row0 / g.Q, p_last = last / g.Q;
-            const int ih_lo = p_first * g.sh - g.ph;
+            const int p_first = ic_p_first, p_last = last / g.Q;
+            const int ih_lo = ic_ih_lo;
             const int in_rows_cta = (p_last - p_first) * g.slab_rstep + g.R;
             const int kbeg = kt_begin * g.tile_k;
             const bool vec16 = g.slab_vec16 && ((reinterpret_cast<uintptr_t>(img) & 15u) == 0);
-            // tables, built once per CTA: byte offset of each tile row's window origin inside a slab channel, and
-            // per reduction index the byte offset of (channel relative to its chunk's first channel, tap)
+            // per tile row: byte offset of its pixel's window origin inside a slab channel
             if (gt < rows) {
                 const int grow = min(row0 + gt, ext - 1);    // rows past the extent repeat the last pixel (never stored)
                 const int p = grow / g.Q, q = grow - p * g.Q;
                 s_rowoff[gt] = 4 * ((p - p_first) * g.slab_rstep * g.slab_wp + q * g.sw + (g.slab_gap - g.pw));
             }
-            const int tk_shift = 31 - __clz(g.tile_k);
-            for (int i = gt; i < iters * g.tile_k; i += kGatherThreads) {
-                const int k = kbeg + i;
-                const int chunk = (i >> tk_shift) / T;
-                const int c_first = (kbeg + chunk * T * g.tile_k) / RS;
-                int ent = 0;                              // beyond K: any finite value will do, the filter side is zero
-                if (k < g.K) {
-                    const int c = k / RS, rem = k - c * RS, fr = rem / g.S, fs = rem - fr * g.S;
-                    ent = 4 * ((c - c_first) * g.slab_chpitch + fr * g.slab_wp + fs);
-                }
-                st_shared_u32(ktab + 4u * (uint32_t)i, (uint32_t)ent);
+            // per reduction index of this CTA: byte offset of (c, r, s) inside the slab, channel counted from 0
+            // (made by the host when the record was applied); four entries per copy
+            for (int i = gt * 4; i < iters * g.tile_k; i += kGatherThreads * 4)
+                cp_async_16(ktab + 4u * (uint32_t)i, g.ktab_dev + kbeg + i);
+            cp_async_commit();
+            // zeros that no copy ever writes: the tail behind each buffer's last row, and, when the gather warps stage
+            // the slab themselves, every gap and every row outside the image
+            if (slab_tma) {
+                const uint32_t tail = 4u * (uint32_t)(g.slab_box_ch * g.slab_chpitch);
+                for (int b = 0; b < g.slab_nbuf; ++b)
+                    for (uint32_t o = tail + (uint32_t)gt * 4u; o < g.slab_buf_bytes; o += (uint32_t)kGatherThreads * 4u)
+                        st_shared_u32(slab0 + (uint32_t)b * g.slab_buf_bytes + o, 0u);
+            } else {
+                const uint32_t slab_bytes = (uint32_t)g.slab_nbuf * g.slab_buf_bytes;
+                for (uint32_t o = (uint32_t)gt * 16u; o < slab_bytes; o += (uint32_t)kGatherThreads * 16u)
+                    st_shared_v4(slab0 + o, 0.f, 0.f, 0.f, 0.f);
             }
-            // zeros for the gaps and for rows outside the image; copies only ever land on in-image positions
-            const uint32_t slab_bytes = (uint32_t)g.slab_nbuf * g.slab_buf_bytes;
-            for (uint32_t o = (uint32_t)gt * 16u; o < slab_bytes; o += (uint32_t)kGatherThreads * 16u)
-                st_shared_v4(slab0 + o, 0.f, 0.f, 0.f, 0.f);
-            bool ok = gather_vote(true);                 // tables and zeros are in place before any copy lands
+            cp_async_wait<0>();
+            bool ok = gather_vote(true);                 // tables and zeros are in place
             if (threadIdx.x == 64) TT_STAMP(17);
-            const int n_chunks = (iters + T - 1) / T;
-            auto chunk_load = [&](int j) {
+            const int n_chunks = ic_chunks;
+            auto chunk_first_channel = [&](int j) { return (kbeg + j * T * g.tile_k) / RS; };
+            auto chunk_load = [&](int j) {               // the gather warps stage chunk j themselves (no TMA)
                 const int k_lo = kbeg + j * T * g.tile_k;
                 const int k_hi = min(g.K, kbeg + min((j + 1) * T, iters) * g.tile_k);
                 if (k_hi > k_lo) {
@@ -799,17 +858,24 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 cp_async_commit();
             };
-            chunk_load(0);
-            if (n_chunks > 1) chunk_load(1);
+            if (!slab_tma) {
+                chunk_load(0);
+                if (n_chunks > 1) chunk_load(1);
+            }
             if (threadIdx.x == 64) TT_STAMP(18);
             const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
             uint32_t st = 0, ph = 0;
             for (int j = 0; j < n_chunks; ++j) {
-                if (j + 1 < n_chunks) cp_async_wait<1>(); else cp_async_wait<0>();
-                ok = gather_vote(ok);                    // every thread's copies of chunk j are visible to all
-                if (!ok) break;
+                if (slab_tma) {
+                    if (ok && !mbar_wait(smem_u32(&slab_full[j & 1]), (uint32_t)(j >> 1) & 1u, abortp, g.status, 6u)) ok = false;
+                } else {
+                    if (j + 1 < n_chunks) cp_async_wait<1>(); else cp_async_wait<0>();
+                    ok = gather_vote(ok);                // every thread's copies of chunk j are visible to all
+                    if (!ok) break;
+                }
                 if (threadIdx.x == 64 && j == 0) TT_STAMP(15);
-                const uint32_t slab = slab0 + (uint32_t)(j & 1) * g.slab_buf_bytes;
+                // table offsets count channels from 0: rebase the buffer by the chunk's first channel
+                const uint32_t slab = slab0 + (uint32_t)(j & 1) * g.slab_buf_bytes - 4u * (uint32_t)(chunk_first_channel(j) * g.slab_chpitch);
                 const int it_end = min((j + 1) * T, iters);
                 for (int it = j * T; it < it_end; ++it) {
                     if (ok && !mbar_wait(empty0 + st * 8u, ph ^ 1u, abortp, g.status, 3u)) ok = false;
@@ -830,7 +896,11 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                     if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
                 }
-                if (j + 2 < n_chunks) {
+                if (slab_tma) {
+                    // this warp is done with the buffer: the producer may refill it
+                    __syncwarp();
+                    if (lane == 0 && j + 2 < n_chunks) mbar_arrive(smem_u32(&slab_empty[j & 1]));
+                } else if (j + 2 < n_chunks) {
                     ok = gather_vote(ok);                // everyone is done reading this buffer
                     if (!ok) break;
                     chunk_load(j + 2);
@@ -1056,22 +1126,20 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const long long lead = along_cols ? g.y_ms : g.y_ns;       // stride of the other output axis
             const bool vec_ok = (lead & 3) == 0 && (g.y_bs & 3) == 0 && (reinterpret_cast<uintptr_t>(ybase) & 15u) == 0 &&
                                 (rbase == nullptr || (reinterpret_cast<uintptr_t>(rbase) & 15u) == 0);
-            auto finish4 = [&](uint32_t off, int mm, int nn, int valid) {
-                float4 p[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    if (q < sk) p[q] = ld_peer_v4(peer[q] + off);
+            // sum over the splits, in split order
+            auto add_splits = [&](const float4 (&p)[8]) {
                 float4 acc = p[0];
 #pragma unroll
                 for (int q = 1; q < 8; ++q)
                     if (q < sk) { acc.x += p[q].x; acc.y += p[q].y; acc.z += p[q].z; acc.w += p[q].w; }
-                float v[4] = {acc.x, acc.y, acc.z, acc.w};
+                return acc;
+            };
+            auto tail4 = [&](float4 acc, float4 bias4, int mm, int nn, int valid) {
+                float v[4] = {acc.x + bias4.x, acc.y + bias4.y, acc.z + bias4.z, acc.w + bias4.w};
                 const long long o = (long long)mm * g.y_ms + (long long)nn * g.y_ns;   // the four are o, o+1, o+2, o+3
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (i < valid) {
-                        if (g.bias_mode == 1) v[i] += __ldg(g.bias + mm + (along_cols ? 0 : i));
-                        else if (g.bias_mode == 2) v[i] += __ldg(g.bias + nn + (along_cols ? i : 0));
                         if (rbase) v[i] += __ldg(rbase + o + i);
                         v[i] = gelu ? gelu_erf(v[i]) : fminf(fmaxf(v[i], lo), hi);
                     }
@@ -1083,22 +1151,60 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         if (i < valid) ybase[o + i] = v[i];
                 }
             };
+            // bias of four neighbouring outputs whose first is (mm, nn)
+            auto bias_of = [&](int mm, int nn, int valid) {
+                float b[4] = {0.f, 0.f, 0.f, 0.f};
+                if (g.bias_mode == 1) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) if (along_cols ? i == 0 : i < valid) b[i] = __ldg(g.bias + mm + (along_cols ? 0 : i));
+                    if (along_cols) b[1] = b[2] = b[3] = b[0];
+                } else if (g.bias_mode == 2) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) if (along_cols ? i < valid : i == 0) b[i] = __ldg(g.bias + nn + (along_cols ? i : 0));
+                    if (!along_cols) b[1] = b[2] = b[3] = b[0];
+                }
+                return make_float4(b[0], b[1], b[2], b[3]);
+            };
+            // two groups per step: their bias loads and all their remote loads are in flight together
+            auto finish_pair = [&](uint32_t off_a, int mm_a, int nn_a, int valid_a, bool has_b, uint32_t off_b, int mm_b, int nn_b, int valid_b) {
+                const float4 bias_a = bias_of(mm_a, nn_a, valid_a);
+                const float4 bias_b = has_b ? bias_of(mm_b, nn_b, valid_b) : make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 pa[8], pb[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (q < sk) pa[q] = ld_peer_v4(peer[q] + off_a);
+                if (has_b) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        if (q < sk) pb[q] = ld_peer_v4(peer[q] + off_b);
+                }
+                tail4(add_splits(pa), bias_a, mm_a, nn_a, valid_a);
+                if (has_b) tail4(add_splits(pb), bias_b, mm_b, nn_b, valid_b);
+            };
             if (along_cols) {
-                // each CTA finishes a band of rows; a warp takes a row, its lanes walk the columns four at a time
+                // each CTA finishes a band of rows; a warp takes two rows per step, its lanes walk the columns four at a time
                 const int per = (kHwTileM + sk - 1) / sk;
                 const int r_end = min(min(kHwTileM, (split + 1) * per), g.M - m0);
                 const int c_end = min(g.tile_n, g.N - n0);
-                for (int row = split * per + gw; row < r_end; row += kGatherWarps)
+                const int pitch = g.tile_n + 4;
+                for (int row = split * per + gw; row < r_end; row += 2 * kGatherWarps) {
+                    const int row_b = row + kGatherWarps;
                     for (int col = lane * 4; col < c_end; col += 128)
-                        finish4(4u * (uint32_t)(row * (g.tile_n + 4) + col), m0 + row, n0 + col, min(4, c_end - col));
+                        finish_pair(4u * (uint32_t)(row * pitch + col), m0 + row, n0 + col, min(4, c_end - col), row_b < r_end,
+                                    4u * (uint32_t)(row_b * pitch + col), m0 + row_b, n0 + col, min(4, c_end - col));
+                }
             } else {
-                // each CTA finishes a band of columns; a warp takes a column, its lanes walk the 128 rows four at a time
+                // each CTA finishes a band of columns; a warp takes two columns per step, its lanes walk the 128 rows
                 const int per = (g.tile_n + sk - 1) / sk;
                 const int c_end = min(min(g.tile_n, (split + 1) * per), g.N - n0);
                 const int r_end = min(kHwTileM, g.M - m0);
-                for (int col = split * per + gw; col < c_end; col += kGatherWarps)
+                for (int col = split * per + gw; col < c_end; col += 2 * kGatherWarps) {
+                    const int col_b = col + kGatherWarps;
                     if (lane * 4 < r_end)
-                        finish4(4u * (uint32_t)(col * kRedColPitch + lane * 4), m0 + lane * 4, n0 + col, min(4, r_end - lane * 4));
+                        finish_pair(4u * (uint32_t)(col * kRedColPitch + lane * 4), m0 + lane * 4, n0 + col, min(4, r_end - lane * 4),
+                                    col_b < c_end, 4u * (uint32_t)(col_b * kRedColPitch + lane * 4), m0 + lane * 4, n0 + col_b,
+                                    min(4, r_end - lane * 4));
+                }
             }
         }
         if (threadIdx.x == 64) TT_STAMP(21);
@@ -1335,7 +1441,8 @@ __global__ void tt_softmax_kernel(const RowArgs a) {
 // ------------------------------------------------------------------------------------------------------------
 // Launchers (called from tt_device.cu)
 // ------------------------------------------------------------------------------------------------------------
-cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, cudaStream_t st) {
+cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, const void* tmap_x,
+                        cudaStream_t st) {
     static int attr_set_for = -1;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -1344,9 +1451,10 @@ cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* t
         if (e != cudaSuccess) return e;
         attr_set_for = dev;
     }
-    CUtensorMap ta, tb;
+    CUtensorMap ta, tb, tx;
     memcpy(&ta, tmap_a, sizeof ta);
     memcpy(&tb, tmap_b, sizeof tb);
+    memcpy(&tx, tmap_x, sizeof tx);
     dim3 grid(I.grid_x, I.grid_y, I.grid_z);
     if (g.cluster) {
         // the splits of one output tile (grid.y) form a thread-block cluster
@@ -1356,9 +1464,9 @@ cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* t
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)g.cluster; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr; cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, tt_gemm_tc_kernel, ta, tb, g);
+        return cudaLaunchKernelEx(&cfg, tt_gemm_tc_kernel, ta, tb, tx, g);
     }
-    tt_gemm_tc_kernel<<<grid, kGemmThreads, I.smem_bytes, st>>>(ta, tb, g);
+    tt_gemm_tc_kernel<<<grid, kGemmThreads, I.smem_bytes, st>>>(ta, tb, tx, g);
     return cudaGetLastError();
 }
 
