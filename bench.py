@@ -24,6 +24,20 @@ METRIC = "TFLOP/s (model pass under transferred schedules)"
 UNIT = "TFLOP/s"
 
 
+# DRAM traffic of the dominant kernel per launch (dram__bytes_read.sum + dram__bytes_write.sum averaged over the
+# timed region's launches, one ncu pass; summary in profiles/bench_resnet18_launch_list.md), valid only for the
+# kernel source it was taken on: any later change of the kernel reports null until the counters are taken again.
+TRAFFIC_COUNTERS = {"model": "resnet18", "kernel_source_sha256_16": "e7cd53b47a258d68", "bytes_per_launch": 2.735e6}
+
+
+def kernel_source_hash():
+    import hashlib
+    path = os.path.join(ROOT, "paper_2201_05587_b200", "csrc", "tt_kernels.cu")
+    with open(path) as f:
+        body = "\n".join(line for line in f.read().splitlines() if "TT_STAMP" not in line)   # diagnostics-only lines
+    return hashlib.sha256(body.encode()).hexdigest()[:16]
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -140,6 +154,68 @@ def tf32_peak(torch):
     return 2.0 * n ** 3 / (best * 1e-3) / 1e12
 
 
+def saturating_points(B, W, torch, dev, peaks, tf32):
+    """The kernel families at sizes where a launch lasts long enough for its roofline to be reachable (NOT one of the
+    benchmark configurations: batch-1 kernels have roofline times below one launch).  Each family is timed under a
+    short list of records; the best is reported against its bound: tensor pipe (cuBLAS TF32 rate measured in this
+    run) for the contractions, measured HBM copy rate for depthwise and softmax."""
+    def conv(n, c, hw, k, r, pad):
+        return W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(n, c, hw, hw, k, r, r, 1, pad, True, B.TT_ACT_RELU), 1,
+                      f"conv{r}x{r}_n{n}_{c}x{hw}->{k}")
+    def dw(n, c, hw, stride):
+        sh = B.make_shapes(n=n, c=c, h=hw, w=hw, k=c, r=3, s=3, stride_h=stride, stride_w=stride, pad_h=1, pad_w=1,
+                           has_bias=1, act=B.TT_ACT_RELU6)
+        return W.Spec(B.TT_OP_DWCONV2D, sh, 1, f"dw3x3s{stride}_n{n}_{c}x{hw}")
+    tc = lambda **kw: B.make_record(B.TT_FAMILY_GEMM_TC, **kw)
+    dwr = lambda **kw: B.make_record(B.TT_FAMILY_DW_SIMT, **kw)
+    cases = [
+        (W._dense(4096, 4096, 4096), "tensor",
+         [tc(tile_n=256, tile_k=32, stages=4, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=4, mma_m_axis=2),
+          tc(tile_n=256, tile_k=64, stages=2, mma_m_axis=1)]),
+        (conv(32, 128, 28, 128, 3, 1), "tensor",
+         [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=128, tile_k=32, stages=3, mma_m_axis=2),
+          tc(tile_n=128, tile_k=64, stages=2, mma_m_axis=2)]),
+        (conv(32, 256, 56, 64, 1, 0), "hbm",
+         [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=2)]),
+        (dw(64, 144, 56, 1), "hbm",
+         [dwr(tile_m=4, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=2),
+          dwr(tile_m=16, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=128, unroll=2),
+          dwr(tile_m=4, block_y=16, block_x=56, items_per_thread=4, vec_width=4, threads=128, unroll=4)]),
+        (dw(32, 96, 112, 2), "hbm",
+         [dwr(tile_m=4, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=2),
+          dwr(tile_m=4, block_y=4, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=1)]),
+        (W.Spec(B.TT_OP_SOFTMAX, B.softmax_shapes(12 * 256, 128, 128, 0.125), 1, "softmax_3072x128x128", "bert"), "hbm",
+         [B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=8, block_y=8, vec_width=4),
+          B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=32, block_y=4, vec_width=4)]),
+    ]
+    o = B.tt_timing_opts()
+    o.warmup_batches, o.batches, o.min_batch_us, o.use_graph = 1, 3, 500, 0
+    out = []
+    for sp, bound, recs in cases:
+        a = W.make_inputs(sp, 7)
+        wl = sp.workload()
+        t, tt = W.device_tensors(sp, a, dev)
+        v = wl.gemm_view()
+        best = None
+        for r in recs:
+            st, info = wl.try_apply(r)
+            if st != B.TT_OK:
+                continue
+            us = wl.time(tt, o).median_us
+            if best is None or us < best[0]:
+                best = (us, info.legal.short())
+        wl.close()
+        del t, tt
+        if best is None:
+            continue
+        us, rec = best
+        row = {"kernel": sp.name, "record": rec, "us": us, "tflops": v.flops / us / 1e6, "gbs": v.bytes / us / 1e3,
+               "algorithmic_mbytes": v.bytes / 1e6, "bound": bound}
+        row["frac"] = (row["tflops"] / tf32) if bound == "tensor" and tf32 else row["gbs"] / peaks["hbm_gbs"]
+        out.append(row)
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -152,6 +228,7 @@ def main():
     ap.add_argument("--top-k", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--report", default="", help="write the per-kernel table (JSON) to this file")
+    ap.add_argument("--no-saturating", action="store_true", help="skip the saturating-size points of the kernel families")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
@@ -318,13 +395,16 @@ def main():
     else:
         roof = {"bound": "tensor", "achieved": gemm_flops / gemm_cold_us / 1e6, "peak": tf32, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = None
+    same_kernel = args.model == TRAFFIC_COUNTERS["model"] and kernel_source_hash() == TRAFFIC_COUNTERS["kernel_source_sha256_16"]
+    roof["traffic"] = TRAFFIC_COUNTERS["bytes_per_launch"] if same_kernel else None
+    roof["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum, timed region average)"
     roof.update({"kernel": "tt_gemm_tc_kernel", "peak_source": peaks["source"] + (" hbm copy" if roof["bound"] == "hbm" else " cuBLAS TF32 8192^3, this run"),
                  "launches_per_pass": gemm_launches, "avg_launch_us": gemm_cold_us / max(gemm_launches, 1),
                  "algorithmic_mbytes_per_pass": gemm_bytes / 1e6, "algorithmic_gflop_per_pass": gemm_flops / 1e9,
                  "tf32_peak_tflops_this_run": tf32, "tensor_frac": (gemm_flops / gemm_cold_us / 1e6) / tf32 if tf32 else None,
                  "l2": "cold (rotating tensor sets > 2x L2)"})
 
+    sat = saturating_points(B, W, torch, dev, peaks, tf32) if rank == 0 and not args.no_saturating else None
     line = None
     if rank == 0:
         cpu = None
@@ -350,6 +430,7 @@ def main():
             "model_latency_us": {"transferred_sum_standalone": lat_best, "default_sum_standalone": lat_default,
                                  "speedup_over_default": lat_default / lat_best if lat_best else None,
                                  "measured_pass_cold_l2": ms_per_step * 1e3},
+            "saturating_sizes_not_a_benchmark_config": sat,
             "search": {"pairs_timed": res["pairs_timed"], "pairs_invalid": res["pairs_invalid"],
                        "seconds": res["search_seconds"], "pool_records": len(pool), "pool_build_seconds": pool_seconds,
                        "pool_candidates_tried": n_tried},

@@ -492,9 +492,9 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
     const bool full = level > 0;
     if (w->family == TT_FAMILY_GEMM_TC) {
         const std::vector<int> tns = full ? std::vector<int>{16, 32, 48, 64, 96, 128, 192, 256} : std::vector<int>{32, 64, 128, 256};
-        const std::vector<int> tks = full ? std::vector<int>{8, 16, 32, 64, 128} : std::vector<int>{16, 32, 64};
-        const std::vector<int> sts = full ? std::vector<int>{2, 3, 4, 6} : std::vector<int>{2, 4};
-        const std::vector<int> sks = full ? std::vector<int>{1, 2, 3, 4, 6, 8, 12, 16, 24, 32} : std::vector<int>{1, 2, 4, 8, 16};
+        const std::vector<int> tks = full ? std::vector<int>{8, 16, 32, 64, 128} : std::vector<int>{32, 64, 128};
+        const std::vector<int> sts = full ? std::vector<int>{2, 3, 4, 6, 8} : std::vector<int>{2, 3, 4};
+        const std::vector<int> sks = full ? std::vector<int>{1, 2, 3, 4, 5, 6, 7, 8, 12, 16, 24, 32} : std::vector<int>{1, 2, 3, 4, 6, 8};
         const std::vector<int> ras = full ? std::vector<int>{0, 1} : std::vector<int>{0};
         for (int ax : {1, 2}) for (int tn : tns) for (int tk : tks) for (int sg : sts) for (int sk : sks) for (int ra : ras) {
             tt_schedule_record r = base;

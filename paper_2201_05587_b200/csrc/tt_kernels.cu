@@ -308,53 +308,90 @@ __device__ __forceinline__ void slab_load_chunk(const GemmArgs& g, const float* 
     }
 }
 
+// The chunks c0, c0 + step, ... of one tile row per lane, KB at a time, in three rounds without a branch between
+// loads: all table entries, all slab values, then the stores (chunks past the tile re-read the last one and are
+// not stored).
+template <int KB>
+__device__ __forceinline__ void expand_chunks(int c0, int step, int n_ch, uint32_t origin, uint32_t ktab_smem, uint32_t dst_row,
+                                              uint32_t swz, int atom_shift, int atom_k, uint32_t atom_bytes, bool in_tile) {
+    for (; c0 < n_ch; c0 += step * KB) {
+        uint4 e[KB];
+        float val[KB][4];
+#pragma unroll
+        for (int b = 0; b < KB; ++b)
+            e[b] = ld_shared_v4u(ktab_smem + 16u * (uint32_t)min(c0 + b * step, n_ch - 1));   // same address in every lane
+#pragma unroll
+        for (int b = 0; b < KB; ++b) {
+            val[b][0] = ld_shared_f32(origin + e[b].x);
+            val[b][1] = ld_shared_f32(origin + e[b].y);
+            val[b][2] = ld_shared_f32(origin + e[b].z);
+            val[b][3] = ld_shared_f32(origin + e[b].w);
+        }
+#pragma unroll
+        for (int b = 0; b < KB; ++b) {
+            const int ci = c0 + b * step;
+            if (ci < n_ch && in_tile) {
+                const int kk = ci << 2;
+                st_shared_v4(dst_row + (uint32_t)(kk >> atom_shift) * atom_bytes + ((uint32_t)((kk & (atom_k - 1)) << 2) ^ swz),
+                             val[b][0], val[b][1], val[b][2], val[b][3]);
+            }
+        }
+    }
+}
+
+// What a gather thread needs to expand its share of any stage, worked out once per kernel: which tile row it
+// serves, where that row's window starts in a slab channel, where the row lands in a K-major tile, which
+// chunks of four reduction indices it takes.
+struct ExpandPlan {
+    bool fast, in_tile;          // fast: 1, 2, 4 or 8 row blocks, so a warp keeps one row block for the whole kernel
+    uint32_t row_origin;         // byte offset of the row's window origin inside a slab channel
+    uint32_t dst_row, swz;       // byte offset of the row inside a tile; its swizzle term
+    int c0, step, n_ch, mine;    // first chunk, chunk stride, chunks per tile, chunks this warp takes
+    int atom_shift, atom_k;
+    uint32_t atom_bytes;
+};
+
+__device__ __forceinline__ ExpandPlan make_expand_plan(int rows, uint32_t rowoff_smem, int tile_k, int atom_k, int row_bytes,
+                                                       int swz_mask, int gw, int lane) {
+    ExpandPlan p;
+    const int n_rb = (rows + 31) >> 5;
+    p.fast = (kGatherWarps % n_rb) == 0;
+    p.atom_shift = atom_k == 32 ? 5 : (atom_k == 16 ? 4 : 3);
+    p.atom_k = atom_k;
+    p.atom_bytes = (uint32_t)rows * (uint32_t)row_bytes;
+    p.n_ch = tile_k >> 2;
+    const int shift = row_bytes == 128 ? 0 : (row_bytes == 64 ? 1 : 2);
+    const int rb = p.fast ? gw % n_rb : 0;
+    p.step = p.fast ? kGatherWarps / n_rb : 1;
+    p.c0 = p.fast ? gw / n_rb : 0;
+    p.mine = (p.n_ch - p.c0 + p.step - 1) / p.step;
+    const int row = rb * 32 + lane;
+    p.in_tile = row < rows;
+    p.row_origin = ld_shared_u32(rowoff_smem + 4u * (uint32_t)(p.in_tile ? row : rows - 1));
+    p.dst_row = (uint32_t)row * (uint32_t)row_bytes;
+    p.swz = (uint32_t)((row >> shift) & swz_mask) << 4;
+    return p;
+}
+
 // Expand one pipeline stage of the im2col operand from the slab.  A warp takes (32-row block, 4-wide k chunk)
 // tasks gw, gw + 8, ...; the loads of four tasks are issued before the first store.
 // rowoff_smem: per tile row, the byte offset of its pixel's window origin inside a channel of the slab;
 // ktab_smem: per reduction index of this tile, the byte offset of (channel, tap) relative to that origin.
-__device__ __forceinline__ void expand_stage(uint32_t tile_smem, int rows, uint32_t slab, uint32_t rowoff_smem,
+__device__ __forceinline__ void expand_stage(const ExpandPlan& xp, uint32_t tile_smem, int rows, uint32_t slab, uint32_t rowoff_smem,
                                              uint32_t ktab_smem, int tile_k, int atom_k, int row_bytes, int swz_mask,
                                              int gw, int lane) {
+    if (xp.fast) {
+        const uint32_t origin = slab + xp.row_origin, dst_row = tile_smem + xp.dst_row;
+        if (xp.mine <= 2) expand_chunks<2>(xp.c0, xp.step, xp.n_ch, origin, ktab_smem, dst_row, xp.swz, xp.atom_shift, xp.atom_k, xp.atom_bytes, xp.in_tile);
+        else if (xp.mine <= 4) expand_chunks<4>(xp.c0, xp.step, xp.n_ch, origin, ktab_smem, dst_row, xp.swz, xp.atom_shift, xp.atom_k, xp.atom_bytes, xp.in_tile);
+        else expand_chunks<8>(xp.c0, xp.step, xp.n_ch, origin, ktab_smem, dst_row, xp.swz, xp.atom_shift, xp.atom_k, xp.atom_bytes, xp.in_tile);
+        return;
+    }
     const int atom_shift = atom_k == 32 ? 5 : (atom_k == 16 ? 4 : 3);
     const int shift = row_bytes == 128 ? 0 : (row_bytes == 64 ? 1 : 2);
     const uint32_t atom_bytes = (uint32_t)rows * (uint32_t)row_bytes;
     const int n_rb = (rows + 31) >> 5;
     const int n_tasks = n_rb * (tile_k >> 2);
-    if ((kGatherWarps % n_rb) == 0) {
-        // 1, 2, 4 or 8 row blocks: a warp keeps one row block for the whole stage, so its pixel's window origin and
-        // the row part of the destination are loop-invariant; it takes every (8 / n_rb)-th chunk of four k
-        const int rb = gw % n_rb, step = kGatherWarps / n_rb, n_ch = tile_k >> 2;
-        const int row = rb * 32 + lane;
-        const bool in_tile = row < rows;
-        const uint32_t origin = slab + ld_shared_u32(rowoff_smem + 4u * (uint32_t)(in_tile ? row : rows - 1));
-        const uint32_t dst_row = tile_smem + (uint32_t)row * (uint32_t)row_bytes;
-        const uint32_t swz = (uint32_t)((row >> shift) & swz_mask) << 4;
-        constexpr int kB = 8;
-        for (int c0 = gw / n_rb; c0 < n_ch; c0 += step * kB) {
-            float val[kB][4];
-#pragma unroll
-            for (int b = 0; b < kB; ++b) {
-                const int ci = c0 + b * step;
-                if (ci < n_ch) {                         // warp-uniform
-                    const uint4 e = ld_shared_v4u(ktab_smem + 16u * (uint32_t)ci);   // same address in every lane
-                    val[b][0] = ld_shared_f32(origin + e.x);
-                    val[b][1] = ld_shared_f32(origin + e.y);
-                    val[b][2] = ld_shared_f32(origin + e.z);
-                    val[b][3] = ld_shared_f32(origin + e.w);
-                }
-            }
-#pragma unroll
-            for (int b = 0; b < kB; ++b) {
-                const int ci = c0 + b * step;
-                if (ci < n_ch && in_tile) {
-                    const int kk = ci << 2;
-                    st_shared_v4(dst_row + (uint32_t)(kk >> atom_shift) * atom_bytes + ((uint32_t)((kk & (atom_k - 1)) << 2) ^ swz),
-                                 val[b][0], val[b][1], val[b][2], val[b][3]);
-                }
-            }
-        }
-        return;
-    }
     const uint32_t inv_rb = (65536u + (uint32_t)n_rb - 1u) / (uint32_t)n_rb;     // t / n_rb == (t * inv_rb) >> 16 for small t
     constexpr int kBatch = 4;
     for (int t0 = gw; t0 < n_tasks; t0 += kGatherWarps * kBatch) {
@@ -843,10 +880,10 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 for (uint32_t o = (uint32_t)gt * 16u; o < slab_bytes; o += (uint32_t)kGatherThreads * 16u)
                     st_shared_v4(slab0 + o, 0.f, 0.f, 0.f, 0.f);
             }
-            cp_async_wait<0>();
-            bool ok = gather_vote(true);                 // tables and zeros are in place
+            bool ok = gather_vote(true);                 // row table and zeros are in place (the k-table may still be in flight)
             if (threadIdx.x == 64) TT_STAMP(17);
             const int n_chunks = ic_chunks;
+            const ExpandPlan xplan = make_expand_plan(rows, rowoff, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, gw, lane);   // after the vote: reads s_rowoff
             auto chunk_first_channel = [&](int j) { return (kbeg + j * T * g.tile_k) / RS; };
             auto chunk_load = [&](int j) {               // the gather warps stage chunk j themselves (no TMA)
                 const int k_lo = kbeg + j * T * g.tile_k;
@@ -868,6 +905,11 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             for (int j = 0; j < n_chunks; ++j) {
                 if (slab_tma) {
                     if (ok && !mbar_wait(smem_u32(&slab_full[j & 1]), (uint32_t)(j >> 1) & 1u, abortp, g.status, 6u)) ok = false;
+                    if (j == 0) {
+                        cp_async_wait<0>();              // the k-table copies of this thread ...
+                        ok = gather_vote(ok);            // ... and of every other gather thread have landed
+                        if (!ok) break;
+                    }
                 } else {
                     if (j + 1 < n_chunks) cp_async_wait<1>(); else cp_async_wait<0>();
                     ok = gather_vote(ok);                // every thread's copies of chunk j are visible to all
@@ -882,7 +924,9 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (ok) {
                         const uint32_t a_s = tiles_base + st * stage_bytes, b_s = a_s + g.a_stage_bytes;
                         const uint32_t kt = ktab + 4u * (uint32_t)(it * g.tile_k);
-                        expand_stage(on_a ? a_s : b_s, rows, slab, rowoff, kt, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, gw, lane);
+                        if (threadIdx.x == 64 && it == 5) TT_STAMP(22);
+                        expand_stage(xplan, on_a ? a_s : b_s, rows, slab, rowoff, kt, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, gw, lane);
+                        if (threadIdx.x == 64 && it == 5) TT_STAMP(23);
                         if (o_gather) {
                             const int k0 = (kt_begin + it) * g.tile_k;
                             if (on_a) gather_stage(g.b_mode, b_s, g.tile_n, o_src, g.b_rs, g.b_ks, n0, g.N, k0, g.K, g.tile_k,
@@ -893,7 +937,9 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         fence_proxy_async_shared();      // generic-proxy stores -> visible to the tensor core's reads
                         __syncwarp();
                         if (lane == 0) mbar_arrive(full0 + st * 8u);
+                        if (threadIdx.x == 64 && it == 5) TT_STAMP(24);
                     }
+                    if (threadIdx.x == 64 && it == 4) TT_STAMP(9);
                     if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
                 }
                 if (slab_tma) {

@@ -20,7 +20,7 @@ from . import workloads as W
 
 ACTS = {"none": B.TT_ACT_NONE, "relu": B.TT_ACT_RELU, "relu6": B.TT_ACT_RELU6, "gelu": B.TT_ACT_GELU_ERF}
 RECORD_FIELDS = ("tile_m", "tile_n", "tile_k", "stages", "split_k", "raster", "block_x", "block_y",
-                 "items_per_thread", "vec_width", "threads", "mma_m_axis")
+                 "items_per_thread", "vec_width", "threads", "unroll", "mma_m_axis", "slab_tiles", "acc_split")
 
 
 def build_spec(a) -> W.Spec:
@@ -52,6 +52,7 @@ def main(argv=None) -> int:
     ap.add_argument("--tune", type=int, default=-1, help="grid-tune at this level first and use the best record")
     ap.add_argument("--iters", type=int, default=3, help="plain launches after the timed batches")
     ap.add_argument("--seed", type=int, default=7)
+    ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of graph replays")
     a = ap.parse_args(argv)
 
     import torch
@@ -71,7 +72,9 @@ def main(argv=None) -> int:
         rec = best[0][0]
         print(f"grid tuner tried {tried} records")
     info = wl.apply(rec)
-    tm = wl.time(tt)
+    topts = B.tt_timing_opts()
+    topts.use_graph = 0 if a.no_graph else 1            # batches replayed as CUDA graphs: no CPU launch gaps
+    tm = wl.time(tt, topts)
     v = wl.gemm_view()
     print(f"{spec.name} {info.legal.short()} grid ({info.grid_x},{info.grid_y},{info.grid_z}) x {info.threads} threads, "
           f"smem {info.smem_bytes} B: median {tm.median_us:.2f} us, {v.flops / tm.median_us / 1e6:.1f} TFLOP/s, "
