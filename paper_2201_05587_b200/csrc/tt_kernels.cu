@@ -1350,7 +1350,7 @@ __global__ void tt_dwconv_kernel(const DwArgs d) {
 // memory or barrier is involved.  Bound by HBM: the only DRAM traffic is x once, y once.
 // ------------------------------------------------------------------------------------------------------------
 template <int R, int STRIDE, int ROWS>
-__global__ void __launch_bounds__(256) tt_dwconv_window_kernel(const DwArgs d) {
+__global__ void __launch_bounds__(256, 6) tt_dwconv_window_kernel(const DwArgs d) {
     constexpr int NCOL = 3 * STRIDE + R;                  // input columns under a 4-wide strip
     constexpr int IN_ROWS = (ROWS - 1) * STRIDE + R;
     constexpr int PAD = R / 2;                            // "same" padding: the launcher checks it
@@ -1484,6 +1484,48 @@ __global__ void tt_softmax_kernel(const RowArgs a) {
     }
 }
 
+// ROW_SIMT, register-resident form: every lane keeps its share of the row (up to NV 16-byte groups) in registers,
+// so x is read from memory once and each exponential is computed once.  Rows of up to lanes_per_row * 4 * NV columns
+// whose length is a multiple of 4 and whose pointers are 16-byte aligned; everything else takes the kernel above.
+template <int NV>
+__global__ void tt_softmax_cached_kernel(const RowArgs a) {
+    const int lpr = a.lanes_per_row;
+    const int sub = threadIdx.x % lpr;
+    const long long row = (long long)blockIdx.x * a.rows_per_cta + threadIdx.x / lpr;
+    const bool live = row < a.rows;
+    const float4* xr = reinterpret_cast<const float4*>(a.x + (live ? row : 0) * (long long)a.cols);
+    float4* yr = reinterpret_cast<float4*>(a.y + (live ? row : 0) * (long long)a.cols);
+    const int groups = a.cols >> 2;
+    float4 v[NV];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        const int gidx = sub + i * lpr;
+        if (live && gidx < groups) {
+            v[i] = __ldg(xr + gidx);
+            v[i].x *= a.scale; v[i].y *= a.scale; v[i].z *= a.scale; v[i].w *= a.scale;
+            mx = fmaxf(mx, fmaxf(fmaxf(v[i].x, v[i].y), fmaxf(v[i].z, v[i].w)));
+        }
+    }
+    for (int o = lpr >> 1; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        const int gidx = sub + i * lpr;
+        if (live && gidx < groups) {
+            v[i].x = expf(v[i].x - mx); v[i].y = expf(v[i].y - mx); v[i].z = expf(v[i].z - mx); v[i].w = expf(v[i].w - mx);
+            sum += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+        }
+    }
+    for (int o = lpr >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const float inv = 1.f / sum;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        const int gidx = sub + i * lpr;
+        if (live && gidx < groups) yr[gidx] = make_float4(v[i].x * inv, v[i].y * inv, v[i].z * inv, v[i].w * inv);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------------------
 // Launchers (called from tt_device.cu)
 // ------------------------------------------------------------------------------------------------------------
@@ -1559,6 +1601,15 @@ cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st)
 }
 
 cudaError_t launch_row(const tt_apply_info& I, const RowArgs& row, cudaStream_t st) {
+    // rows that fit the lanes' registers (and allow 16-byte accesses) are read once
+    const int per_lane = row.vec == 4 ? ((row.cols >> 2) + row.lanes_per_row - 1) / row.lanes_per_row : 0;
+    if (per_lane >= 1 && per_lane <= 8) {
+        if (per_lane == 1) tt_softmax_cached_kernel<1><<<I.grid_x, I.threads, 0, st>>>(row);
+        else if (per_lane == 2) tt_softmax_cached_kernel<2><<<I.grid_x, I.threads, 0, st>>>(row);
+        else if (per_lane <= 4) tt_softmax_cached_kernel<4><<<I.grid_x, I.threads, 0, st>>>(row);
+        else tt_softmax_cached_kernel<8><<<I.grid_x, I.threads, 0, st>>>(row);
+        return cudaGetLastError();
+    }
     tt_softmax_kernel<<<I.grid_x, I.threads, 0, st>>>(row);
     return cudaGetLastError();
 }
