@@ -374,8 +374,9 @@ tt_status tt_run(tt_workload* w, const tt_tensors* t, void* cuda_stream) { retur
 tt_status tt_debug_read_timers(tt_workload* w, unsigned long long* out50) {
     if (!w || !w->status_word || !out50) return TT_ERR_INVALID_ARG;
     cudaDeviceSynchronize();
-    return cudaMemcpy(out50, reinterpret_cast<char*>(w->status_word) + 16, 50 * 8, cudaMemcpyDeviceToHost) == cudaSuccess
-               ? TT_OK : TT_ERR_CUDA;
+    const bool ok = cudaMemcpy(out50, reinterpret_cast<char*>(w->status_word) + 16, 60 * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
+    cudaMemset(reinterpret_cast<char*>(w->status_word) + 16, 0, 60 * 8);      // the next launch starts from cleared stamps
+    return ok ? TT_OK : TT_ERR_CUDA;
 }
 #endif
 

@@ -618,7 +618,16 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
         g_tt_dbg = reinterpret_cast<unsigned long long*>(g.status) + 2;
 #endif
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel of the stream may begin its set-up
     if (threadIdx.x == 0) TT_STAMP(0);
+#ifdef TT_PHASE_TIMERS
+    // span of the whole grid: latest CTA start and latest CTA end (earliest start = ~min kept as max of the complement)
+    if (threadIdx.x == 0) {
+        unsigned long long* d = reinterpret_cast<unsigned long long*>(g.status) + 2;
+        atomicMax(d + 56, ~global_timer_ns());
+        atomicMax(d + 58, global_timer_ns());
+    }
+#endif
 
     // tile coordinates
     int tm, tn;
@@ -673,6 +682,11 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *(volatile uint32_t*)&tmem_slot;
+    // Programmatic dependent launch: everything above (barriers, tensor memory) touched no global memory and may
+    // run while the previous kernel of the stream is still draining; from here on its results are needed.  The
+    // kernel that follows this one was allowed to start its own set-up at this kernel's entry.  (Without the launch
+    // attribute both instructions do nothing.)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (threadIdx.x == 0) TT_STAMP(1);
 
     // Warps 0 and 1 run their loops with all 32 lanes: waits, counters and descriptor arithmetic stay
@@ -1265,6 +1279,9 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         tmem_dealloc(tmem_base, g.tmem_cols);
     }
     if (threadIdx.x == 0) TT_STAMP(6);
+#ifdef TT_PHASE_TIMERS
+    if (threadIdx.x == 0) atomicMax(reinterpret_cast<unsigned long long*>(g.status) + 2 + 57, global_timer_ns());
+#endif
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -1544,18 +1561,23 @@ cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* t
     memcpy(&tb, tmap_b, sizeof tb);
     memcpy(&tx, tmap_x, sizeof tx);
     dim3 grid(I.grid_x, I.grid_y, I.grid_z);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = dim3(kGemmThreads, 1, 1); cfg.dynamicSmemBytes = (size_t)I.smem_bytes; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    // the kernel's set-up may overlap the tail of the kernel before it in the stream (it waits before its first
+    // global access); captured into a graph this becomes a programmatic dependency edge
+    attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+    ++n_attr;
     if (g.cluster) {
         // the splits of one output tile (grid.y) form a thread-block cluster
-        cudaLaunchConfig_t cfg{};
-        cfg.gridDim = grid; cfg.blockDim = dim3(kGemmThreads, 1, 1); cfg.dynamicSmemBytes = (size_t)I.smem_bytes; cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)g.cluster; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, tt_gemm_tc_kernel, ta, tb, tx, g);
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = 1; attr[n_attr].val.clusterDim.y = (unsigned)g.cluster; attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
     }
-    tt_gemm_tc_kernel<<<grid, kGemmThreads, I.smem_bytes, st>>>(ta, tb, tx, g);
-    return cudaGetLastError();
+    cfg.attrs = attr; cfg.numAttrs = (unsigned)n_attr;
+    return cudaLaunchKernelEx(&cfg, tt_gemm_tc_kernel, ta, tb, tx, g);
 }
 
 // Can a cluster of `cluster` CTAs with this much shared memory each be resident at all?
