@@ -145,10 +145,14 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     // touch: consecutive rows when stride <= filter height, else `r` rows per output row.  A chunk holds the
     // channels that `slab_tiles` consecutive reduction tiles touch; two buffers when there are several chunks.
     // split_k of 2..8: the splits of a tile form a thread-block cluster and reduce through distributed shared memory
-    // (each parks its 128 x tile_n partial tile in its pipeline buffers); beyond 8 the partial tiles go through a
-    // global workspace and the split that arrives last adds them up
+    // (each sends the bands of its partial tile to the CTAs that finish them); beyond 8 the partial tiles go through
+    // a global workspace and the split that arrives last adds them up
     const int cluster = (sk >= 2 && sk <= 8) ? sk : 0;
-    const long long min_pipe = std::max<long long>((long long)kGatherWarps * 32 * 36 * 4, cluster ? std::max<long long>((long long)tn * (kHwTileM + 4) * 4, (long long)kHwTileM * (tn + 4) * 4) : 0);
+    const long long min_pipe = (long long)kGatherWarps * 32 * 36 * 4;
+    // cluster reduction area, apart from the pipeline buffers (peers write into it while this CTA may still be in its
+    // main loop): per source split, this CTA's band of the tile -- rows x (tile_n + 4) or columns x 132 floats
+    const long long red_bytes = cluster ? (4 * std::max<long long>((long long)sk * ((kHwTileM + sk - 1) / sk) * (tn + 4),
+                                                                    (long long)sk * ((tn + sk - 1) / sk) * (kHwTileM + 4)) + 127) / 128 * 128 : 0;
     const bool conv = w->op == TT_OP_CONV2D;
     const long long ktab = conv ? (((long long)per_split * tk * 4 + 127) / 128) * 128 : 0;
     int sl_tiles = 0, sl_nbuf = 0, sl_wp = 0, sl_gap = 0, sl_chpitch = 0, sl_in_rows = 0, sl_rstep = 1;
@@ -181,7 +185,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
         long long slab_total = 0;
         bool fits = true;
         if (conv) {
-            const long long budget = kDynSmemLimit - 1024 - pipe_try - ktab;
+            const long long budget = kDynSmemLimit - 1024 - pipe_try - ktab - red_bytes;
             // largest chunk not above the request that fits (one buffer if it covers the CTA's whole K range)
             int t = rec->slab_tiles == 0 ? per_split : std::min(rec->slab_tiles, per_split);
             while (t >= 1 && ((t >= per_split ? 1 : 2) * chunk_bytes(t) > budget || (slab_tma && chunk_channels(t) > 256))) --t;
@@ -191,7 +195,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
             sl_buf_bytes = chunk_bytes(sl_tiles);
             slab_total = sl_nbuf * sl_buf_bytes;
         }
-        smem = pipe_try + ktab + slab_total + 1024;
+        smem = pipe_try + ktab + slab_total + red_bytes + 1024;
         if (fits && smem <= kDynSmemLimit) break;
         // reformulate: a shallower pipeline leaves room (never in strict mode, never below one buffer)
         if (strict || st <= 1) break;
@@ -238,6 +242,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     g.a_stage_bytes = a_stage; g.b_stage_bytes = b_stage;
     g.ktab_off = (unsigned)pipe;
     g.slab_off = (unsigned)(pipe + ktab);
+    g.red_off = (unsigned)(pipe + ktab + (long long)sl_nbuf * sl_buf_bytes);
     g.slab_buf_bytes = (unsigned)sl_buf_bytes; g.slab_nbuf = sl_nbuf; g.slab_tiles = sl_tiles;
     g.slab_wp = sl_wp; g.slab_gap = sl_gap; g.slab_chpitch = sl_chpitch; g.slab_in_rows = sl_in_rows;
     g.slab_rstep = sl_rstep;

@@ -42,6 +42,7 @@ struct GemmArgs {
     unsigned* counters;                         // split-K arrival counters [batch][tiles], zero between launches
     unsigned* status;
     unsigned idesc, tmem_cols;
+    unsigned red_off;                           // cluster reduction area: byte offset from the aligned tile base
     int cluster;                                // > 0: split-K over a thread-block cluster of this many CTAs (= split_k)
     int n_acc;                                  // accumulators of tile_n columns each, reduction steps dealt round-robin
     unsigned a_stage_bytes, b_stage_bytes, tx_bytes;

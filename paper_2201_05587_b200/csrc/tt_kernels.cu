@@ -246,6 +246,8 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t map_to_peer(uint32_t saddr, uint32_t rank) {
     uint32_t r;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
@@ -256,14 +258,23 @@ __device__ __forceinline__ float ld_peer_f32(uint32_t caddr) {
     asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(caddr) : "memory");
     return v;
 }
-__device__ __forceinline__ float4 ld_peer_v4(uint32_t caddr) {
+__device__ __forceinline__ void st_peer_v4(uint32_t caddr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(caddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void st_peer_u32(uint32_t caddr, uint32_t a) {
+    asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(caddr), "r"(a) : "memory");
+}
+__device__ __forceinline__ float4 ld_shared_v4f(uint32_t addr) {
     float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(caddr) : "memory");
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
     return v;
 }
-// A parked partial tile is laid out along the direction in which the output is contiguous, so that both the
-// remote 16-byte loads of the reduction and the global stores are contiguous across lanes:
-//   outputs contiguous along columns: [row][col], pitch tile_n + 4 floats;  along rows: [col][row], pitch 132 floats.
+// Split-K over a cluster.  The output tile is cut into one band per CTA, along the direction in which the output is
+// NOT contiguous (bands of rows when outputs are contiguous along columns, bands of columns otherwise).  Every CTA
+// sends each band of its partial tile to the CTA that owns the band (remote shared-memory stores into a reduction
+// area that is not part of the pipeline buffers, so a fast peer cannot disturb a slower one's main loop); after one
+// cluster barrier every CTA adds up what it received, in split order, locally.  Area layout, per source split:
+//   bands of rows:    [row in band][col], pitch tile_n + 4 floats;   bands of columns: [col in band][row], pitch 132.
 constexpr int kRedColPitch = kHwTileM + 4;
 
 // All gather threads meet and learn whether every one of them is still healthy (named barrier 1).
@@ -619,6 +630,9 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         g_tt_dbg = reinterpret_cast<unsigned long long*>(g.status) + 2;
 #endif
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel of the stream may begin its set-up
+    // A CTA's shared memory may be written by a peer only once the CTA runs: every thread announces itself here and
+    // checks, much later and just before the first remote store could happen, that all peers have done the same.
+    if (g.cluster) cluster_arrive();
     if (threadIdx.x == 0) TT_STAMP(0);
 #ifdef TT_PHASE_TIMERS
     // span of the whole grid: latest CTA start and latest CTA end (earliest start = ~min kept as max of the complement)
@@ -774,6 +788,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
             __syncwarp();
         }
+        if (g.cluster) cluster_wait();
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         {
@@ -845,6 +860,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             __syncwarp();
             if (lane == 0) TT_STAMP(3);
         }
+        if (g.cluster) cluster_wait();
     } else {
         // ---------------- gather producers, then epilogue ----------------
         const int gw = warp - 2;
@@ -1003,6 +1019,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(all_acc) : "r"((uint32_t)have_acc), "n"(kGatherThreads) : "memory");
         if (threadIdx.x == 64) TT_STAMP(4);
+        if (g.cluster) cluster_wait();                   // every peer is running: its reduction area may be written
         if (all_acc) {
             tc_fence_after();
             const int half = gw >> 2;
@@ -1015,8 +1032,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const long long per_split = (long long)g.batch * g.M * (long long)g.N;
             float* pcol = g.partial + (long long)bz * g.M * (long long)g.N + m;
             if (g.cluster) {
-                // split-K over a cluster: park this split's partial tile in its own shared memory (the pipeline
-                // buffers are idle now), column-major with a padded pitch; the reduction follows the cluster barrier
+                // split-K over a cluster: send each band of this split's partial tile to the CTA that finishes it
 #pragma unroll 1
                 for (int c0 = half * 32; c0 < g.tile_n; c0 += 64) {
                     uint32_t r[32];
@@ -1031,18 +1047,30 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(t2[i]));
                     }
                     const int row = quad * 32 + lane;
+                    const uint32_t red = tiles_base + g.red_off;
                     if (g.y_ns == 1) {
-                        const uint32_t dst = tiles_base + 4u * (uint32_t)(row * (g.tile_n + 4) + c0);
+                        // bands of rows: this lane's row belongs to one CTA
+                        const int per = (kHwTileM + g.split_k - 1) / g.split_k;
+                        const int owner = row / per, rl = row - owner * per;
+                        const uint32_t dst = map_to_peer(red, (uint32_t)owner) + 4u * (uint32_t)((split * per + rl) * (g.tile_n + 4) + c0);
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
                             if (c0 + j < g.tile_n)           // tile_n is a multiple of 16: groups of four are whole
-                                st_shared_v4(dst + 4u * (uint32_t)j, __uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                                             __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                                st_peer_v4(dst + 4u * (uint32_t)j, r[j], r[j + 1], r[j + 2], r[j + 3]);
                     } else {
-                        const uint32_t dst = tiles_base + 4u * (uint32_t)(c0 * kRedColPitch + row);
+                        // bands of columns: column c0 + j belongs to CTA (c0 + j) / per; lanes (rows) are contiguous
+                        const int per = (g.tile_n + g.split_k - 1) / g.split_k;
+                        int owner = c0 / per, cl = c0 - owner * per;
+                        uint32_t dst = map_to_peer(red, (uint32_t)owner) + 4u * (uint32_t)((split * per + cl) * kRedColPitch + row);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (c0 + j < g.tile_n) st_shared_u32(dst + 4u * (uint32_t)(j * kRedColPitch), r[j]);
+                        for (int j = 0; j < 32; ++j) {
+                            if (c0 + j < g.tile_n) st_peer_u32(dst, r[j]);
+                            dst += 4u * (uint32_t)kRedColPitch;
+                            if (++cl == per) {               // next column starts the next CTA's band
+                                cl = 0; ++owner;
+                                dst = map_to_peer(red, (uint32_t)min(owner, g.split_k - 1)) + 4u * (uint32_t)(split * per * kRedColPitch + row);
+                            }
+                        }
                     }
                 }
             } else if (split_mode) {
@@ -1164,42 +1192,43 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
     }
     if (g.cluster) {
-        // ---------------- split-K over the cluster: reduce through distributed shared memory ----------------
-        // Every thread of every CTA of the cluster takes part in both barriers, also after a tripped wait.
+        // ---------------- split-K over the cluster: add up the bands the peers sent ----------------
+        // Every thread of every CTA of the cluster takes part in the barrier, also after a tripped wait.  After it
+        // nobody writes to or reads from another CTA's shared memory any more, so no second barrier is needed.
         if (threadIdx.x == 64) TT_STAMP(19);
-        cluster_sync_all();                              // all partial tiles are parked
+        cluster_sync_all();                              // all bands have arrived
         if (threadIdx.x == 64) TT_STAMP(20);
         if (warp >= 2) {
             const int gw = warp - 2;
             const int sk = g.split_k;
-            uint32_t peer[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) peer[q] = map_to_peer(tiles_base, (uint32_t)(q < sk ? q : 0));
+            const uint32_t red = tiles_base + g.red_off;
             float* ybase = g.y + (long long)bz * g.y_bs;
             const float* rbase = g.residual ? g.residual + (long long)bz * g.y_bs : nullptr;
             const float lo = g.act == TT_ACT_NONE || g.act == TT_ACT_GELU_ERF ? -INFINITY : 0.f;
             const float hi = g.act == TT_ACT_RELU6 ? 6.f : INFINITY;
             const bool gelu = g.act == TT_ACT_GELU_ERF;
-            // four outputs that are neighbours in memory: one 16-byte load per split (all issued before the first
-            // addition; partial sums are added in split order), the fused tail, one 16-byte store where alignment allows
             const bool along_cols = g.y_ns == 1;
             const long long lead = along_cols ? g.y_ms : g.y_ns;       // stride of the other output axis
             const bool vec_ok = (lead & 3) == 0 && (g.y_bs & 3) == 0 && (reinterpret_cast<uintptr_t>(ybase) & 15u) == 0 &&
                                 (rbase == nullptr || (reinterpret_cast<uintptr_t>(rbase) & 15u) == 0);
-            // sum over the splits, in split order
-            auto add_splits = [&](const float4 (&p)[8]) {
+            // four outputs that are neighbours in memory, first one (mm, nn): the partial sums of all splits (16 bytes
+            // each, `stride` bytes apart) are added in split order, then bias, residual, activation, one 16-byte store
+            auto finish4 = [&](uint32_t addr, uint32_t stride, int mm, int nn, int valid) {
+                float4 p[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (q < sk) p[q] = ld_shared_v4f(addr + (uint32_t)q * stride);
                 float4 acc = p[0];
 #pragma unroll
                 for (int q = 1; q < 8; ++q)
                     if (q < sk) { acc.x += p[q].x; acc.y += p[q].y; acc.z += p[q].z; acc.w += p[q].w; }
-                return acc;
-            };
-            auto tail4 = [&](float4 acc, float4 bias4, int mm, int nn, int valid) {
-                float v[4] = {acc.x + bias4.x, acc.y + bias4.y, acc.z + bias4.z, acc.w + bias4.w};
+                float v[4] = {acc.x, acc.y, acc.z, acc.w};
                 const long long o = (long long)mm * g.y_ms + (long long)nn * g.y_ns;   // the four are o, o+1, o+2, o+3
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (i < valid) {
+                        if (g.bias_mode == 1) v[i] += __ldg(g.bias + mm + (along_cols ? 0 : i));
+                        else if (g.bias_mode == 2) v[i] += __ldg(g.bias + nn + (along_cols ? i : 0));
                         if (rbase) v[i] += __ldg(rbase + o + i);
                         v[i] = gelu ? gelu_erf(v[i]) : fminf(fmaxf(v[i], lo), hi);
                     }
@@ -1211,64 +1240,28 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         if (i < valid) ybase[o + i] = v[i];
                 }
             };
-            // bias of four neighbouring outputs whose first is (mm, nn)
-            auto bias_of = [&](int mm, int nn, int valid) {
-                float b[4] = {0.f, 0.f, 0.f, 0.f};
-                if (g.bias_mode == 1) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) if (along_cols ? i == 0 : i < valid) b[i] = __ldg(g.bias + mm + (along_cols ? 0 : i));
-                    if (along_cols) b[1] = b[2] = b[3] = b[0];
-                } else if (g.bias_mode == 2) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) if (along_cols ? i < valid : i == 0) b[i] = __ldg(g.bias + nn + (along_cols ? i : 0));
-                    if (!along_cols) b[1] = b[2] = b[3] = b[0];
-                }
-                return make_float4(b[0], b[1], b[2], b[3]);
-            };
-            // two groups per step: their bias loads and all their remote loads are in flight together
-            auto finish_pair = [&](uint32_t off_a, int mm_a, int nn_a, int valid_a, bool has_b, uint32_t off_b, int mm_b, int nn_b, int valid_b) {
-                const float4 bias_a = bias_of(mm_a, nn_a, valid_a);
-                const float4 bias_b = has_b ? bias_of(mm_b, nn_b, valid_b) : make_float4(0.f, 0.f, 0.f, 0.f);
-                float4 pa[8], pb[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    if (q < sk) pa[q] = ld_peer_v4(peer[q] + off_a);
-                if (has_b) {
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        if (q < sk) pb[q] = ld_peer_v4(peer[q] + off_b);
-                }
-                tail4(add_splits(pa), bias_a, mm_a, nn_a, valid_a);
-                if (has_b) tail4(add_splits(pb), bias_b, mm_b, nn_b, valid_b);
-            };
             if (along_cols) {
-                // each CTA finishes a band of rows; a warp takes two rows per step, its lanes walk the columns four at a time
+                // this CTA's band of rows; a warp takes a row, its lanes walk the columns four at a time
                 const int per = (kHwTileM + sk - 1) / sk;
-                const int r_end = min(min(kHwTileM, (split + 1) * per), g.M - m0);
+                const int rows_here = min(min(kHwTileM, (split + 1) * per), g.M - m0) - split * per;
                 const int c_end = min(g.tile_n, g.N - n0);
                 const int pitch = g.tile_n + 4;
-                for (int row = split * per + gw; row < r_end; row += 2 * kGatherWarps) {
-                    const int row_b = row + kGatherWarps;
+                for (int rl = gw; rl < rows_here; rl += kGatherWarps)
                     for (int col = lane * 4; col < c_end; col += 128)
-                        finish_pair(4u * (uint32_t)(row * pitch + col), m0 + row, n0 + col, min(4, c_end - col), row_b < r_end,
-                                    4u * (uint32_t)(row_b * pitch + col), m0 + row_b, n0 + col, min(4, c_end - col));
-                }
+                        finish4(red + 4u * (uint32_t)(rl * pitch + col), 4u * (uint32_t)(per * pitch), m0 + split * per + rl, n0 + col,
+                                min(4, c_end - col));
             } else {
-                // each CTA finishes a band of columns; a warp takes two columns per step, its lanes walk the 128 rows
+                // this CTA's band of columns; a warp takes a column, its lanes walk the 128 rows four at a time
                 const int per = (g.tile_n + sk - 1) / sk;
-                const int c_end = min(min(g.tile_n, (split + 1) * per), g.N - n0);
+                const int cols_here = min(min(g.tile_n, (split + 1) * per), g.N - n0) - split * per;
                 const int r_end = min(kHwTileM, g.M - m0);
-                for (int col = split * per + gw; col < c_end; col += 2 * kGatherWarps) {
-                    const int col_b = col + kGatherWarps;
+                for (int cl = gw; cl < cols_here; cl += kGatherWarps)
                     if (lane * 4 < r_end)
-                        finish_pair(4u * (uint32_t)(col * kRedColPitch + lane * 4), m0 + lane * 4, n0 + col, min(4, r_end - lane * 4),
-                                    col_b < c_end, 4u * (uint32_t)(col_b * kRedColPitch + lane * 4), m0 + lane * 4, n0 + col_b,
-                                    min(4, r_end - lane * 4));
-                }
+                        finish4(red + 4u * (uint32_t)(cl * kRedColPitch + lane * 4), 4u * (uint32_t)(per * kRedColPitch), m0 + lane * 4,
+                                n0 + split * per + cl, min(4, r_end - lane * 4));
             }
         }
         if (threadIdx.x == 64) TT_STAMP(21);
-        cluster_sync_all();                              // nobody leaves while a peer may still read its tile
     }
     if (threadIdx.x == 64) TT_STAMP(5);
     tc_fence_before();
