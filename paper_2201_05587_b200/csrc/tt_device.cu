@@ -486,7 +486,8 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
         // keep only records that are legal as written: a record that needs rounding duplicates another candidate
         tt_apply_info info;
         if (tt_schedule_check(w, &r, TT_MODE_LEGALISE, 0, &info) != TT_OK) return false;
-        if (info.changed & ~TT_CHG_TILE_M) return false;
+        // (a pipeline made shallower to fit short reductions or shared memory is kept: exact duplicates are dropped below)
+        if (info.changed & ~(TT_CHG_TILE_M | TT_CHG_STAGES)) return false;
         cand.push_back(info.legal);
         return true;
     };
@@ -531,6 +532,11 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
             r.block_x = bx; r.block_y = by; r.vec_width = vw;
             push(r);
         }
+    }
+    if (cand.empty()) {
+        // nothing of the grid fits this shape as written: tune around the legalised default record
+        tt_apply_info info;
+        if (tt_schedule_check(w, &base, TT_MODE_LEGALISE, 0, &info) == TT_OK) cand.push_back(info.legal);
     }
     // drop exact duplicates (legalisation can map different inputs to one record)
     std::vector<tt_schedule_record> uniq;

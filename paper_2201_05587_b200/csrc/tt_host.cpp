@@ -542,7 +542,7 @@ tt_status tt_default_schedule(const tt_workload* w, tt_schedule_record* out) {
     r.tile_m = 128; r.tile_n = 128; r.tile_k = 32; r.stages = 4; r.split_k = 1; r.raster = 0; r.acc_split = 1;
     r.block_x = 32; r.block_y = 4; r.items_per_thread = 1; r.vec_width = 1; r.unroll = 1; r.threads = 128;
     if (w->family == TT_FAMILY_DW_SIMT) { r.tile_m = 1; r.block_x = 32; r.block_y = 8; r.items_per_thread = 4; r.unroll = 2; }
-    if (w->family == TT_FAMILY_ROW_SIMT) { r.block_x = 32; r.block_y = 4; }
+    if (w->family == TT_FAMILY_ROW_SIMT) { r.block_x = 8; r.block_y = 16; r.vec_width = 4; }
     *out = r;
     return TT_OK;
 }
