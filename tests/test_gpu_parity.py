@@ -100,6 +100,8 @@ def test_dense_parity_all_records(spec):
     W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(2, 8, 9, 11, 12, 3, 3, 1, 1, True, B.TT_ACT_RELU, True), 1, "batch2_residual", "uniform"),
     W.Spec(B.TT_OP_CONV2D, B.make_shapes(n=1, c=6, h=10, w=12, k=9, r=3, s=2, stride_h=2, stride_w=1, pad_h=0, pad_w=1,
                                          has_bias=0, act=B.TT_ACT_NONE), 1, "asym_nobias", "uniform"),
+    W._conv(20, 10, 40, 1, 1, 0, name="conv1x1_100px_20ch"),
+    W._conv(136, 12, 200, 1, 1, 0, act=B.TT_ACT_NONE, name="conv1x1_136ch"),
     W._conv(96, 9, 48, 3, 1, 1, name="conv3x3_96ch_chunks"),                # 864 reduction indices: many slab chunks
     W._conv(40, 12, 24, 5, 1, 2, act=B.TT_ACT_RELU6, name="conv5x5_pad2"),
     W._conv(32, 17, 16, 1, 3, 0, name="conv1x1s3"),                         # stride beyond the filter: rows are skipped
@@ -114,6 +116,7 @@ def test_conv_parity_all_records(spec):
     W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(12, 128, 128, 64, True), 1, "qk_nt", "bert"),
     W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(12, 128, 64, 128, False), 1, "pv_nn", "bert"),
     W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(3, 50, 70, 36, False), 1, "ragged_nn", "bert"),
+    W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(2, 45, 76, 52, False), 1, "ragged_nn_76", "bert"),
     W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(2, 33, 17, 10, True), 1, "ragged_nt_k10", "bert"),
 ], ids=lambda s: s.name)
 def test_batch_matmul_parity_all_records(spec):

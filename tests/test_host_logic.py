@@ -172,8 +172,8 @@ def test_legaliser_clamps_and_strict_mode_rejects():
     assert st == B.TT_OK and info.legal.stages == 1 and info.changed & B.TT_CHG_STAGES
     st, info = huge.check(fat, mode=B.TT_MODE_STRICT)
     assert st == B.TT_ERR_RESOURCE and info.smem_bytes > 227 * 1024
-    # a 256-pixel x 128-channel tile of a 1x1 convolution: its input slab alone exceeds shared memory at any depth
-    wide = W._conv(256, 56, 64, 1, 1, 0).workload()
+    # a 128-pixel x 128-channel tile of a strided 1x1 convolution: its input slab alone exceeds shared memory at any depth
+    wide = W._conv(256, 56, 512, 1, 2, 0).workload()
     st, info = wide.check(B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=32, tile_k=128, stages=2, mma_m_axis=2))
     assert st == B.TT_ERR_RESOURCE and info.smem_bytes > 227 * 1024
     # the slab is part of the record: a request for more reduction tiles per staging than fit is lowered
