@@ -312,3 +312,51 @@ def test_largest_dense_sampled_outputs():
     rows = [0, 1, 127, 128, 2047, 4000, 4095]
     sub = orc.dense(a["x"], a["w"][rows], a["bias"][rows], B.TT_ACT_RELU)
     assert util.rel_l2(y[:, rows], sub) <= util.TOL_TF32
+
+
+def test_chained_kernels_on_one_stream_see_each_others_results():
+    """Kernels are launched so that a kernel's set-up may overlap the tail of the one before it in the stream; every
+    global access still comes after the previous kernel has finished.  A chain in which each layer reads the output of
+    the layer before it (conv3x3 -> conv1x1/2 cluster split-K -> depthwise -> conv3x3 workspace split-K), launched back
+    to back without any synchronisation, several times over, must equal the same chain on the oracle."""
+    import torch
+    layers = [
+        (W._conv(16, 20, 32, 3, 1, 1), tc(tile_n=64, tile_k=32, stages=3, mma_m_axis=1)),
+        (W._conv(32, 20, 48, 1, 2, 0, act=B.TT_ACT_NONE), tc(tile_n=32, tile_k=8, stages=2, split_k=4, mma_m_axis=2)),
+        (W._dw(48, 10, 1), B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=4, block_y=4, block_x=8, items_per_thread=4, vec_width=2,
+                                          threads=64, unroll=2)),
+        (W._conv(48, 10, 24, 3, 1, 1, act=B.TT_ACT_RELU6), tc(tile_n=48, tile_k=16, stages=2, split_k=12, mma_m_axis=1)),
+    ]
+    arrays = [W.make_inputs(sp, 61, i) for i, (sp, _) in enumerate(layers)]
+    # oracle chain
+    x = arrays[0]["x"]
+    for (sp, _), a in zip(layers, arrays):
+        a = dict(a)
+        a["x"] = x
+        x = util.oracle_ref(sp, a)
+    ref = x
+    # device chain: layer i writes the buffer layer i + 1 reads
+    wls, tts, keep = [], [], []
+    first = cur = torch.from_numpy(arrays[0]["x"]).cuda()      # `first` keeps the chain's input alive
+    for (sp, rec), a in zip(layers, arrays):
+        wl = sp.workload()
+        wl.apply(rec)
+        t, _ = W.device_tensors(sp, a)
+        assert tuple(cur.shape) == tuple(t["x"].shape)
+        tts.append(B.tensors(cur, t["w"], t["bias"], None, t["y"]))
+        keep.append(t)
+        wls.append(wl)
+        cur = t["y"]
+    for _ in range(5):
+        for t in keep:
+            t["y"].fill_(float("nan"))
+        for wl, tt in zip(wls, tts):
+            wl.run(tt)
+        torch.cuda.synchronize()
+        y = cur.cpu().numpy()
+        assert not np.isnan(y).any()
+        assert util.rel_l2(y, ref) <= 3 * util.TOL_TF32      # three TF32 layers in a row
+    for wl in wls:
+        assert wl.status() == B.TT_OK
+        wl.close()
+    del first
