@@ -299,6 +299,28 @@ __device__ __forceinline__ void slab_load_chunk(const GemmArgs& g, const float* 
                                                 int nch, int ih_lo, int in_rows_cta, bool vec16, int gt) {
     const int wpieces = vec16 ? g.W >> 2 : g.W;
     const bool use_magic = vec16 == (g.slab_vec16 != 0);  // the host's magic number is for its own piece width
+    if (wpieces <= 16) {
+        // short rows (small images): one thread copies a whole row, so the row's address arithmetic is done once
+        const int n_rows = nch * g.slab_in_rows;
+        for (int row = gt; row < n_rows; row += kGatherThreads) {
+            const int cl = small_div(row, g.magic_in_rows);
+            const int rl = row - cl * g.slab_in_rows;
+            int ih = ih_lo + rl;
+            if (g.sh > g.R) {
+                const int po = small_div(rl, g.magic_rstep);
+                ih = ih_lo + po * g.sh + (rl - po * g.slab_rstep);
+            }
+            if (rl >= in_rows_cta || (unsigned)ih >= (unsigned)g.H) continue;
+            const float* src = img + ((long long)(c_first + cl) * g.H + ih) * g.W;
+            const uint32_t dst = buf + 4u * (uint32_t)(cl * g.slab_chpitch + rl * g.slab_wp + g.slab_gap);
+            if (vec16) {
+                for (int pc = 0; pc < wpieces; ++pc) cp_async_16(dst + 16u * (uint32_t)pc, src + 4 * pc);
+            } else {
+                for (int pc = 0; pc < wpieces; ++pc) cp_async_4(dst + 4u * (uint32_t)pc, src + pc);
+            }
+        }
+        return;
+    }
     const int total = nch * g.slab_in_rows * wpieces;
     for (int idx = gt; idx < total; idx += kGatherThreads) {
         const int t1 = use_magic ? small_div(idx, g.magic_wpieces) : idx / wpieces;
