@@ -517,9 +517,10 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
         // register-window kernel: rows per thread x CTA tile
         const std::vector<int> wys = full ? std::vector<int>{1, 2, 4, 7, 8, 14, 16, 28, 56} : std::vector<int>{4, 8, 16};
         const std::vector<int> wxs = full ? std::vector<int>{8, 16, 28, 32, 56, 64, 112} : std::vector<int>{16, 32, 64, 112};
-        for (int ro : {1, 2, 4}) for (int tc : tcs) for (int by : wys) for (int bx : wxs) for (int th : {64, 128, 256}) {
+        for (int it : {4, 8}) for (int ro : {1, 2, 4}) for (int tc : tcs) for (int by : wys) for (int bx : wxs) for (int th : {64, 128, 256}) {
+            if (it == 8 && ro == 4) continue;
             tt_schedule_record r = base;
-            r.tile_m = tc; r.block_y = by; r.block_x = bx; r.items_per_thread = 4; r.threads = th;
+            r.tile_m = tc; r.block_y = by; r.block_x = bx; r.items_per_thread = it; r.threads = th;
             r.unroll = ro;
             for (int vw : {4, 2, 1}) {                  // the widest store the output rows allow
                 r.vec_width = vw;

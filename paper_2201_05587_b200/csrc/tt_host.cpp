@@ -326,7 +326,8 @@ static tt_status legalise_dw(const tt_workload* w, const tt_schedule_record* rec
     if (rec->unroll < 0) return TT_ERR_INVALID_SCHEDULE;
     if (rec->unroll >= 1 && window_ok) {
         window_rows = rec->unroll >= 4 ? 4 : (rec->unroll >= 2 ? 2 : 1);
-        items = 4;
+        items = rec->items_per_thread >= 8 ? 8 : 4;      // strips of 4 or 8 columns; 8-wide strips are at most 2 rows tall
+        if (items == 8 && window_rows > 2) window_rows = 2;
     }
     L.unroll = window_rows;
     int bx = std::min(rec->block_x, round_up(w->Q, items));

@@ -1375,15 +1375,15 @@ __global__ void tt_dwconv_kernel(const DwArgs d) {
 
 // ------------------------------------------------------------------------------------------------------------
 // DW_SIMT, register-window form (3x3 and 5x5 filters, stride 1 or 2).  A thread owns a strip of ROWS output rows
-// x 4 consecutive output columns of one channel.  It walks the (ROWS-1)*STRIDE + R input rows the strip needs
+// x 4 or 8 consecutive output columns of one channel.  It walks the (ROWS-1)*STRIDE + R input rows the strip needs
 // once: of each row it fetches 3*STRIDE + R values (aligned 16-byte loads for the columns under the strip when the
 // image rows allow it, 4-byte loads for the ragged edges; neighbouring strips' loads meet in L1) and feeds every
 // output row whose window contains that input row, so an input value is read once per strip and no shared
 // memory or barrier is involved.  Bound by HBM: the only DRAM traffic is x once, y once.
 // ------------------------------------------------------------------------------------------------------------
-template <int R, int STRIDE, int ROWS>
-__global__ void __launch_bounds__(256, 6) tt_dwconv_window_kernel(const DwArgs d) {
-    constexpr int NCOL = 3 * STRIDE + R;                  // input columns under a 4-wide strip
+template <int R, int STRIDE, int ROWS, int WIDTH>
+__global__ void __launch_bounds__(256, WIDTH == 4 ? 6 : 4) tt_dwconv_window_kernel(const DwArgs d) {
+    constexpr int NCOL = (WIDTH - 1) * STRIDE + R;        // input columns under a WIDTH-wide strip
     constexpr int IN_ROWS = (ROWS - 1) * STRIDE + R;
     constexpr int PAD = R / 2;                            // "same" padding: the launcher checks it
     constexpr int NV = (NCOL - PAD) / 4;                  // aligned 16-byte groups per window row
@@ -1393,14 +1393,14 @@ __global__ void __launch_bounds__(256, 6) tt_dwconv_window_kernel(const DwArgs d
     const int th = t % d.tiles_h; t /= d.tiles_h;
     const int c0 = t * d.tile_c, p0 = th * d.tile_h, q0 = tw * d.tile_w;
     const int nc = min(d.tile_c, d.C - c0);
-    const int groups_w = d.tile_w >> 2;
+    const int groups_w = d.tile_w / WIDTH;
     const int groups_h = (d.tile_h + ROWS - 1) / ROWS;
     const int work = nc * groups_h * groups_w;
     for (int i = threadIdx.x; i < work; i += blockDim.x) {
         const int gwi = i % groups_w;
         const int rest = i / groups_w;
         const int gh = rest % groups_h, cl = rest / groups_h;
-        const int p = p0 + gh * ROWS, q = q0 + gwi * 4;
+        const int p = p0 + gh * ROWS, q = q0 + gwi * WIDTH;
         if (p >= d.P || q >= d.Q || gh * ROWS >= d.tile_h) continue;
         const int c = c0 + cl;
         const float* __restrict__ xc = d.x + ((long long)n * d.C + c) * d.H * (long long)d.W;
@@ -1409,11 +1409,11 @@ __global__ void __launch_bounds__(256, 6) tt_dwconv_window_kernel(const DwArgs d
 #pragma unroll
         for (int k = 0; k < R * R; ++k) wv[k] = __ldg(wc + k);
         const float b = d.bias ? __ldg(d.bias + c) : 0.f;
-        float acc[ROWS][4];
+        float acc[ROWS][WIDTH];
 #pragma unroll
         for (int ro = 0; ro < ROWS; ++ro)
 #pragma unroll
-            for (int j = 0; j < 4; ++j) acc[ro][j] = b;
+            for (int j = 0; j < WIDTH; ++j) acc[ro][j] = b;
         const int ih0 = p * STRIDE - PAD, iw0 = q * STRIDE - PAD;
 #pragma unroll
         for (int ri = 0; ri < IN_ROWS; ++ri) {
@@ -1455,7 +1455,7 @@ __global__ void __launch_bounds__(256, 6) tt_dwconv_window_kernel(const DwArgs d
 #pragma unroll
                     for (int fs = 0; fs < R; ++fs)
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) acc[ro][j] = fmaf(v[j * STRIDE + fs], wv[fr * R + fs], acc[ro][j]);
+                        for (int j = 0; j < WIDTH; ++j) acc[ro][j] = fmaf(v[j * STRIDE + fs], wv[fr * R + fs], acc[ro][j]);
                 }
             }
         }
@@ -1463,19 +1463,22 @@ __global__ void __launch_bounds__(256, 6) tt_dwconv_window_kernel(const DwArgs d
 #pragma unroll
         for (int ro = 0; ro < ROWS; ++ro) {
             if (p + ro >= d.P || gh * ROWS + ro >= d.tile_h) break;
-            float o[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) o[j] = apply_act(acc[ro][j], d.act);
             float* yo = yc + (long long)ro * d.Q;
-            if (d.vec == 4 && q + 4 <= d.Q) {
-                *reinterpret_cast<float4*>(yo) = make_float4(o[0], o[1], o[2], o[3]);
-            } else if (d.vec == 2 && q + 4 <= d.Q) {
-                *reinterpret_cast<float2*>(yo) = make_float2(o[0], o[1]);
-                *reinterpret_cast<float2*>(yo + 2) = make_float2(o[2], o[3]);
-            } else {
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if (q + j < d.Q) yo[j] = o[j];
+            for (int j0 = 0; j0 < WIDTH; j0 += 4) {
+                float o[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) o[j] = apply_act(acc[ro][j0 + j], d.act);
+                if (d.vec == 4 && q + j0 + 4 <= d.Q) {
+                    *reinterpret_cast<float4*>(yo + j0) = make_float4(o[0], o[1], o[2], o[3]);
+                } else if (d.vec == 2 && q + j0 + 4 <= d.Q) {
+                    *reinterpret_cast<float2*>(yo + j0) = make_float2(o[0], o[1]);
+                    *reinterpret_cast<float2*>(yo + j0 + 2) = make_float2(o[2], o[3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (q + j0 + j < d.Q) yo[j0 + j] = o[j];
+                }
             }
         }
     }
@@ -1624,12 +1627,14 @@ cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st)
     dim3 grid(I.grid_x, I.grid_y, 1);
     if (dw.window_rows > 0) {
         // register-window kernels: one instantiation per (filter size, stride, output rows per thread)
-#define TT_DW_CASE(RR, SS, RO) \
-        if (dw.R == RR && dw.sh == SS && dw.window_rows == RO) { tt_dwconv_window_kernel<RR, SS, RO><<<grid, I.threads, 0, st>>>(dw); return cudaGetLastError(); }
-        TT_DW_CASE(3, 1, 1) TT_DW_CASE(3, 1, 2) TT_DW_CASE(3, 1, 4)
-        TT_DW_CASE(3, 2, 1) TT_DW_CASE(3, 2, 2) TT_DW_CASE(3, 2, 4)
-        TT_DW_CASE(5, 1, 1) TT_DW_CASE(5, 1, 2) TT_DW_CASE(5, 1, 4)
-        TT_DW_CASE(5, 2, 1) TT_DW_CASE(5, 2, 2) TT_DW_CASE(5, 2, 4)
+#define TT_DW_CASE(RR, SS, RO, WD) \
+        if (dw.R == RR && dw.sh == SS && dw.window_rows == RO && dw.items == WD) { tt_dwconv_window_kernel<RR, SS, RO, WD><<<grid, I.threads, 0, st>>>(dw); return cudaGetLastError(); }
+        TT_DW_CASE(3, 1, 1, 4) TT_DW_CASE(3, 1, 2, 4) TT_DW_CASE(3, 1, 4, 4)
+        TT_DW_CASE(3, 2, 1, 4) TT_DW_CASE(3, 2, 2, 4) TT_DW_CASE(3, 2, 4, 4)
+        TT_DW_CASE(5, 1, 1, 4) TT_DW_CASE(5, 1, 2, 4) TT_DW_CASE(5, 1, 4, 4)
+        TT_DW_CASE(5, 2, 1, 4) TT_DW_CASE(5, 2, 2, 4) TT_DW_CASE(5, 2, 4, 4)
+        TT_DW_CASE(3, 1, 1, 8) TT_DW_CASE(3, 1, 2, 8) TT_DW_CASE(3, 2, 1, 8) TT_DW_CASE(3, 2, 2, 8)
+        TT_DW_CASE(5, 1, 1, 8) TT_DW_CASE(5, 1, 2, 8) TT_DW_CASE(5, 2, 1, 8) TT_DW_CASE(5, 2, 2, 8)
 #undef TT_DW_CASE
         return cudaErrorInvalidValue;
     }

@@ -185,7 +185,7 @@ def test_depthwise_parity_records(spec):
     for tcn, by, bx, it, vw, th, un in ((4, 8, 32, 4, 4, 256, 0), (16, 4, 16, 2, 2, 128, 0), (1, 16, 64, 8, 4, 64, 0),
                                         (32, 7, 7, 1, 1, 512, 0), (3, 5, 24, 8, 1, 96, 0),
                                         (4, 8, 32, 4, 4, 256, 1), (1, 16, 64, 8, 4, 64, 2), (2, 7, 12, 4, 4, 512, 4),
-                                        (8, 5, 8, 1, 1, 32, 4), (3, 6, 112, 4, 2, 96, 2)):
+                                        (8, 5, 8, 1, 1, 32, 4), (3, 6, 112, 4, 2, 96, 2), (2, 3, 16, 8, 4, 128, 1), (5, 9, 24, 8, 1, 64, 4)):
         recs.append(B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=tcn, block_y=by, block_x=bx, items_per_thread=it,
                                   vec_width=vw, threads=th, unroll=un))
     outs = [run_spec(spec, r, a, ref) for r in recs]
