@@ -891,6 +891,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         const int m = m0 + quad * 32 + lane;
         // bias is fetched now so that its latency hides behind the main loop
         if (g.bias_mode == 2 && gt < g.tile_n) s_bias[gt] = (n0 + gt < g.N) ? __ldg(g.bias + n0 + gt) : 0.f;
+        if (g.bias_mode == 1 && g.cluster && gt < kHwTileM) s_bias[gt] = (m0 + gt < g.M) ? __ldg(g.bias + m0 + gt) : 0.f;   // for the cluster reduction
         const float bias_row = (g.bias_mode == 1 && m < g.M) ? __ldg(g.bias + m) : 0.f;
         if (im2col) {
             // ---- conv2d: slab staging + expansion; all eight warps work on the same stage ----
@@ -1249,8 +1250,9 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     if (i < valid) {
-                        if (g.bias_mode == 1) v[i] += __ldg(g.bias + mm + (along_cols ? 0 : i));
-                        else if (g.bias_mode == 2) v[i] += __ldg(g.bias + nn + (along_cols ? i : 0));
+                        // the tile's bias values were staged in shared memory before the main loop
+                        if (g.bias_mode == 1) v[i] += s_bias[mm - m0 + (along_cols ? 0 : i)];
+                        else if (g.bias_mode == 2) v[i] += s_bias[nn - n0 + (along_cols ? i : 0)];
                         if (rbase) v[i] += __ldg(rbase + o + i);
                         v[i] = gelu ? gelu_erf(v[i]) : fminf(fmaxf(v[i], lo), hi);
                     }
