@@ -28,7 +28,7 @@
  *   - One handle must not be used from two threads at once.
  *   - A CUDA device must be present for everything except the pure host calls
  *     (tt_workload_create/key/class/gemm_view, tt_default_schedule, tt_schedule_check,
- *     tt_select, tt_model_latency, tt_split_check, tt_status_string); there is no
+ *     tt_select, tt_model_latency, tt_rank_pools, tt_split_check, tt_status_string); there is no
  *     CPU fallback: without a device the others return TT_ERR_CUDA.
  */
 #ifndef TT_H_
@@ -239,6 +239,14 @@ tt_status tt_select(const float* times_us, size_t n_wl, size_t n_cols, int32_t* 
 /* Pure host: sum_w use_count[w] * times_us[w, chosen[w]] (kernels assumed independent, Section 2). */
 tt_status tt_model_latency(const float* times_us, size_t n_wl, size_t n_cols, const int32_t* chosen,
                            const int32_t* use_count, double* latency_us);
+
+/* Pure host: the model-selection heuristic, Equation 1 of Section 4.4.  For a target model whose kernel classes
+ * take the shares class_share[c] (fractions of its untuned inference time) and n_models candidate models with
+ * class_kernels[t * n_classes + c] unique kernels of class c, scores[t] = sum_c class_share[c]^2 * sqrt(kernels of
+ * class c in t); order[] lists the candidates by decreasing score, ties keeping the lower index first.  scores may
+ * be NULL.  Shares can come from the default-record times of the evaluator's table. */
+tt_status tt_rank_pools(const double* class_share, size_t n_classes, const int32_t* class_kernels, size_t n_models,
+                        double* scores, int32_t* order);
 
 /* The evaluator of Section 4.3: every workload x every compatible pool record (plus the default), standalone, on
  * the workload's own tensors; invalid pairs are recorded, not fatal.  On return each workload is left with its

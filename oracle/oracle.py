@@ -12,16 +12,19 @@ the host-side definitions the paper fixes:
 * ``select`` — keep, per kernel, the fastest schedule that produced valid code
   (Section 4.3); invalid pairs carry a negative time as in Figure 4.
 * ``model_latency`` — sum of use count x chosen standalone time.
+* ``rank_pools`` — the model-selection heuristic, Equation 1 (Section 4.4).
 
 Parity pinning status: conv2d, dwconv2d, dense/batch_matmul, softmax, the
 activations, the split rules and ``select`` are pinned by closed forms, brute
-force and the paper's worked examples in ``tests/test_oracle_pins.py``.
+force and the paper's worked examples in ``tests/test_oracle_pins.py``;
+``rank_pools`` by Tables 2 and 3 of the paper (all ten top-3 rankings).
 The absolute kernel times and which schedule wins on a given kernel are
 "parity unpinned": the paper's per-kernel times exist only in a figure.
 """
 from __future__ import annotations
 
 import ctypes
+import math
 import os
 import subprocess
 
@@ -231,3 +234,21 @@ def model_latency(use_counts, times, chosen, n_sched: int) -> float:
     """Sum over kernels of use count x time of the chosen schedule."""
     t = np.asarray(times, dtype=np.float64).reshape(len(use_counts), n_sched)
     return float(sum(u * t[i, c] for i, (u, c) in enumerate(zip(use_counts, chosen)) if c >= 0))
+
+
+def rank_pools(target_share, candidate_counts):
+    """Equation 1 (model-selection heuristic): score of candidate model T for a target model with class shares P_c is
+    sum over the target's classes c of P_c^2 * sqrt(|W_Tc|), |W_Tc| = number of kernels of class c in T.
+
+    target_share: {class: share of untuned inference time, as a fraction};
+    candidate_counts: list of {class: number of kernels}, one per candidate.
+    Returns (scores, order): order lists candidate indices by decreasing score, ties keeping the lower index first."""
+    scores = []
+    for counts in candidate_counts:
+        s = 0.0
+        for cls, p in target_share.items():
+            n = counts.get(cls, 0)
+            s += (p * p) * math.sqrt(n)
+        scores.append(s)
+    order = sorted(range(len(scores)), key=lambda i: (-scores[i], i))
+    return scores, order

@@ -114,6 +114,8 @@ EXPORTS = {
     "tt_select": (i32, [C.POINTER(f32), C.c_size_t, C.c_size_t, C.POINTER(i32)]),
     "tt_model_latency": (i32, [C.POINTER(f32), C.c_size_t, C.c_size_t, C.POINTER(i32), C.POINTER(i32),
                                C.POINTER(C.c_double)]),
+    "tt_rank_pools": (i32, [C.POINTER(C.c_double), C.c_size_t, C.POINTER(i32), C.c_size_t, C.POINTER(C.c_double),
+                            C.POINTER(i32)]),
     "tt_transfer_tune": (i32, [C.POINTER(C.c_void_p), C.POINTER(tt_tensors), C.c_size_t, C.POINTER(tt_schedule_record),
                                C.c_size_t, C.POINTER(tt_tune_opts), C.c_void_p, C.POINTER(tt_tune_result)]),
     "tt_grid_tune": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(tt_timing_opts), i32, C.c_size_t,
@@ -215,6 +217,17 @@ def model_latency(times, n_wl, n_cols, chosen, use_count) -> float:
     out = C.c_double(0)
     _check(lib().tt_model_latency(arr, n_wl, n_cols, ch, uc, C.byref(out)), "tt_model_latency")
     return out.value
+
+
+def rank_pools(class_share, class_kernels):
+    """Equation 1: class_share[c] of the target model, class_kernels[t][c] of each candidate; returns (scores, order)."""
+    n_c, n_m = len(class_share), len(class_kernels)
+    sh = (C.c_double * n_c)(*[float(v) for v in class_share])
+    ck = (i32 * (n_c * max(n_m, 1)))(*[int(v) for row in class_kernels for v in row])
+    sc = (C.c_double * max(n_m, 1))()
+    od = (i32 * max(n_m, 1))()
+    _check(lib().tt_rank_pools(sh, n_c, ck, n_m, sc, od), "tt_rank_pools")
+    return list(sc)[:n_m], list(od)[:n_m]
 
 
 def _ptr(t):

@@ -592,6 +592,25 @@ tt_status tt_select(const float* times_us, size_t n_wl, size_t n_cols, int32_t* 
     return TT_OK;
 }
 
+tt_status tt_rank_pools(const double* class_share, size_t n_classes, const int32_t* class_kernels, size_t n_models,
+                        double* scores, int32_t* order) {
+    if (!class_share || !class_kernels || !order || n_classes == 0) return TT_ERR_INVALID_ARG;
+    std::vector<double> sc(n_models, 0.0);
+    for (size_t t = 0; t < n_models; ++t) {
+        double s = 0.0;
+        for (size_t c = 0; c < n_classes; ++c) {
+            const int32_t n = class_kernels[t * n_classes + c];
+            if (n < 0 || !(class_share[c] >= 0.0)) return TT_ERR_INVALID_ARG;
+            s += class_share[c] * class_share[c] * std::sqrt((double)n);
+        }
+        sc[t] = s;
+    }
+    for (size_t t = 0; t < n_models; ++t) order[t] = (int32_t)t;
+    std::stable_sort(order, order + n_models, [&](int32_t a, int32_t b) { return sc[a] > sc[b]; });
+    if (scores) for (size_t t = 0; t < n_models; ++t) scores[t] = sc[t];
+    return TT_OK;
+}
+
 tt_status tt_model_latency(const float* times_us, size_t n_wl, size_t n_cols, const int32_t* chosen,
                            const int32_t* use_count, double* latency_us) {
     if (!times_us || !chosen || !use_count || !latency_us) return TT_ERR_INVALID_ARG;

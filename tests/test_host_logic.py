@@ -221,3 +221,23 @@ def test_device_calls_fail_loudly_without_gpu():
     assert st == B.TT_ERR_CUDA                      # no CPU fallback
     t = B.tt_tensors()
     assert B.lib().tt_run(wl.handle, ctypes.byref(t), None) == B.TT_ERR_NOT_APPLIED
+
+
+def test_rank_pools_matches_the_oracle_on_the_papers_tables():
+    """tt_rank_pools (Equation 1) against the oracle on Table 2, target by target, and its argument checks."""
+    import test_oracle_pins as pins
+    feats, choices = pins._load_tables()
+    classes = sorted({c for f in feats.values() for c in f})
+    for target in feats:
+        cands = [m for m in feats if m != target]
+        share_d = {c: pct / 100.0 for c, (_, pct) in feats[target].items()}
+        counts_d = [{c: n for c, (n, _) in feats[m].items()} for m in cands]
+        want_scores, want_order = orc.rank_pools(share_d, counts_d)
+        share = [share_d.get(c, 0.0) for c in classes]
+        counts = [[cd.get(c, 0) for c in classes] for cd in counts_d]
+        scores, order = B.rank_pools(share, counts)
+        assert order == want_order
+        assert scores == pytest.approx(want_scores, rel=1e-12, abs=1e-15)
+        assert [cands[i] for i in order[:len(choices[target])]] == choices[target]
+    with pytest.raises(B.TTError):
+        B.rank_pools([0.5], [[-1]])

@@ -271,3 +271,52 @@ def test_select_hand_tables():
          2.0, -1.0, 1.5, 9.0]
     assert orc.select(t, 3, 4) == [1, -1, 2]
     assert orc.model_latency([2, 1, 3], t, [1, -1, 2], 4) == pytest.approx(2 * 3.0 + 3 * 1.5)
+
+
+def _load_tables():
+    """Tables 2 and 3 of the paper as stored under tests/golden/."""
+    feats = {}
+    with open(os.path.join(GOLDEN, "table2_model_features.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            mid, _name, cls, n, pct = line.split()
+            feats.setdefault(mid, {})[cls] = (int(n), int(pct))
+    choices = {}
+    with open(os.path.join(GOLDEN, "table3_heuristic_choices.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            t, c1, c2, c3 = line.split()
+            choices[t] = [c for c in (c1, c2, c3) if c != "-"]
+    return feats, choices
+
+
+def test_selection_heuristic_reproduces_the_papers_top3_choices():
+    """Equation 1 evaluated on Table 2 must rank the candidate models as Table 3 lists them (all ten targets)."""
+    feats, choices = _load_tables()
+    assert len(feats) == 10 and len(choices) == 10
+    for target, want in choices.items():
+        cands = [m for m in feats if m != target]
+        share = {c: pct / 100.0 for c, (_, pct) in feats[target].items()}
+        counts = [{c: n for c, (n, _) in feats[m].items()} for m in cands]
+        scores, order = orc.rank_pools(share, counts)
+        got = [cands[i] for i in order[:len(want)]]
+        assert got == want, (target, got, want, sorted(scores, reverse=True)[:4])
+        if len(want) == 1:        # BERT / MobileBERT: every other model scores zero
+            assert all(scores[i] == 0.0 for i in order[1:])
+    # a dropped square or square root changes the ranking somewhere: GoogLeNet's second and third choice differ by 2e-4
+    share = {c: pct / 100.0 for c, (_, pct) in feats["M7"].items()}
+    s_vgg = sum(share.get(c, 0) ** 2 * math.sqrt(n) for c, (n, _) in feats["M3"].items())
+    s_mnas = sum(share.get(c, 0) ** 2 * math.sqrt(n) for c, (n, _) in feats["M8"].items())
+    assert 0 < s_vgg - s_mnas < 1e-3
+
+
+def test_selection_heuristic_special_cases():
+    # one class, one candidate kernel: score = P^2
+    assert orc.rank_pools({"E": 0.5}, [{"E": 1}])[0] == [0.25]
+    # four times the kernels doubles the score; a class the target lacks adds nothing
+    s, order = orc.rank_pools({"E": 1.0}, [{"E": 4, "Z": 100}, {"E": 16}, {"Q": 9}])
+    assert s == [2.0, 4.0, 0.0] and order == [1, 0, 2]
+    # ties keep the lower index
+    assert orc.rank_pools({"A": 0.3}, [{"A": 2}, {"A": 2}])[1] == [0, 1]
