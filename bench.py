@@ -222,7 +222,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours")
-    ap.add_argument("--model", default="resnet18", choices=["resnet18", "resnet50", "mobilenet_v2", "bert_base"])
+    ap.add_argument("--model", default="resnet18", choices=["resnet18", "resnet50", "mobilenet_v2", "bert_base", "bert_base_256"])
+    ap.add_argument("--pool", default="", help="comma-separated models whose tuned records form the pool (default: the config's)")
     ap.add_argument("--seed", type=int, default=2)
     ap.add_argument("--tune-level", type=int, default=0)
     ap.add_argument("--top-k", type=int, default=2)
@@ -257,7 +258,8 @@ def main():
     topts.warmup_batches, topts.batches, topts.min_batch_us, topts.use_graph = 2, 5, 100, 1
     t0 = time.perf_counter()
     pool, n_tried = [], 0
-    for src in W.POOL_SOURCES[args.model]:
+    pool_sources = tuple(p for p in args.pool.split(",") if p) or W.POOL_SOURCES[args.model]
+    for src in pool_sources:
         for j, sp in enumerate(W.MODELS[src]()):
             a = W.make_inputs(sp, args.seed + 100, j)
             swl = sp.workload()
@@ -418,7 +420,7 @@ def main():
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "tf32",
             "data": "synthetic",
             "config": {"workload": f"{args.model}-shaped inference, batch 1, fp32 NCHW, {len(specs)} unique kernels / "
-                                   f"{sum(use)} per pass, pool from {','.join(W.POOL_SOURCES[args.model])}-shaped kernels",
+                                   f"{sum(use)} per pass, pool from {','.join(pool_sources)}-shaped kernels",
                        "l2": "flushed between steps (256 MB write)", "replay": "one CUDA graph per model pass",
                        "multi_gpu": "independent replicas"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bytes_up, "d2h_bytes_per_step": bytes_down,

@@ -178,9 +178,15 @@ def bert_base(seq=128, hidden=768, heads=12, ffn=3072, layers=12):
     ]
 
 
+def bert_base_256():
+    """The same encoder on 256 tokens: source or target of the sequence-length transfer of Section 5.4."""
+    return bert_base(seq=256)
+
+
 MODELS = {
     "single_conv": single_conv, "resnet18": resnet18, "resnet50": resnet50, "vgg16": vgg16,
     "mobilenet_v2": mobilenet_v2, "efficientnet_b0_like": efficientnet_b0_like, "bert_base": bert_base,
+    "bert_base_256": bert_base_256,
 }
 
 # target model -> models whose natively tuned records form its schedule pool
@@ -189,6 +195,7 @@ POOL_SOURCES = {
     "resnet50": ("resnet18", "vgg16"),
     "mobilenet_v2": ("resnet50", "efficientnet_b0_like"),
     "bert_base": ("resnet50", "mobilenet_v2"),
+    "bert_base_256": ("bert_base",),          # same model, other input size (Section 5.4)
 }
 
 
