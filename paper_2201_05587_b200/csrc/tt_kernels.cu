@@ -1,11 +1,13 @@
 // Device code of libtt for sm_100a: the schedule-parameterised kernel families.
 //
-//   GEMM_TC  tcgen05.mma kind::tf32, accumulator in tensor memory, operands staged in shared memory by TMA
-//            (K-major tensors) or by gather warps issuing cp.async (im2col of NCHW activations, strided views),
-//            `stages`-deep mbarrier pipeline, bias/activation fused into the accumulator read-out, split-K with
-//            an in-kernel reduction in fixed split order by the last-arriving CTA of each tile.
-//   DW_SIMT  depthwise convolution, shared-memory halo tile, fp32 FMA.
-//   ROW_SIMT row softmax with sub-warp shuffles.
+//   GEMM_TC  tcgen05.mma kind::tf32, accumulator in tensor memory, `stages`-deep mbarrier pipeline.  Operands reach
+//            shared memory by TMA (K-major tensors), by expansion from a slab of input rows that TMA (or cp.async)
+//            staged once per CTA (im2col of NCHW activations), or by gathers (strided views).  Bias/activation are
+//            fused into the accumulator read-out.  Split-K of 2..8 runs as a thread-block cluster that reduces
+//            through distributed shared memory; more splits go through a workspace and the last-arriving CTA adds
+//            them up, both in fixed split order.  Launched with programmatic stream serialization.
+//   DW_SIMT  depthwise convolution: a register-window kernel (3x3 / 5x5) and a shared-memory staged kernel, fp32 FMA.
+//   ROW_SIMT row softmax with sub-warp shuffles, register-resident rows when they fit.
 //
 // Every tile size, the pipeline depth, split-K and the tile order are run-time values taken from the applied
 // schedule record, so applying a record never recompiles anything.
