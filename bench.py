@@ -180,10 +180,12 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
         (dw(64, 144, 56, 1), "hbm",
          [dwr(tile_m=4, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=2),
           dwr(tile_m=16, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=128, unroll=2),
-          dwr(tile_m=4, block_y=16, block_x=56, items_per_thread=4, vec_width=4, threads=128, unroll=4)]),
+          dwr(tile_m=4, block_y=16, block_x=56, items_per_thread=4, vec_width=4, threads=128, unroll=4),
+          dwr(tile_m=8, block_y=56, block_x=56, items_per_thread=8, vec_width=4, threads=128, unroll=2)]),
         (dw(32, 96, 112, 2), "hbm",
          [dwr(tile_m=4, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=2),
-          dwr(tile_m=4, block_y=4, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=1)]),
+          dwr(tile_m=4, block_y=4, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=1),
+          dwr(tile_m=1, block_y=8, block_x=56, items_per_thread=4, vec_width=4, threads=64, unroll=2)]),
         (W.Spec(B.TT_OP_SOFTMAX, B.softmax_shapes(12 * 256, 128, 128, 0.125), 1, "softmax_3072x128x128", "bert"), "hbm",
          [B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=8, block_y=8, vec_width=4),
           B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=32, block_y=4, vec_width=4)]),

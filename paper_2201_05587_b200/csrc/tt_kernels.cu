@@ -137,6 +137,22 @@ __device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t adesc, uint64
         "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// All 8-wide reduction steps of one pipeline stage into one accumulator: ATOMS swizzle atoms of K8 steps each.
+// Inside an atom a step advances both descriptors by 2 (32 bytes); the next atom starts a_atom / b_atom later.
+template <int ATOMS, int K8>
+__device__ __forceinline__ void issue_steps(uint32_t d_tmem, uint32_t d_hi, uint32_t a_lo, uint32_t b_lo, uint32_t a_atom,
+                                            uint32_t b_atom, uint32_t idesc, uint32_t accumulate) {
+#pragma unroll
+    for (int at = 0; at < ATOMS; ++at) {
+#pragma unroll
+        for (int k8 = 0; k8 < K8; ++k8) {
+            mma_tf32(d_tmem, ((uint64_t)d_hi << 32) | (uint64_t)(a_lo + (uint32_t)at * a_atom + 2u * (uint32_t)k8),
+                     ((uint64_t)d_hi << 32) | (uint64_t)(b_lo + (uint32_t)at * b_atom + 2u * (uint32_t)k8), idesc,
+                     (at == 0 && k8 == 0) ? accumulate : 1u);
+        }
+    }
+}
+
 // Arrive on an mbarrier once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -846,19 +862,14 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     // descriptors step by 2 (32 bytes = 8 TF32 along K) inside a swizzle atom, then to the next atom
                     uint32_t a_lo = a_stage, b_lo = b_stage;
                     if (g.n_acc == 1) {
-                        // one accumulator: nothing to rotate
-                        uint32_t accumulate = it > 0 ? 1u : 0u;
-#pragma unroll 1
-                        for (int at = 0; at < g.n_atoms; ++at) {
-#pragma unroll 4
-                            for (int k8 = 0; k8 < k8_per_atom; ++k8) {
-                                mma_tf32(tmem_base, ((uint64_t)d_hi << 32) | (uint64_t)a_lo, ((uint64_t)d_hi << 32) | (uint64_t)b_lo, g.idesc,
-                                         accumulate);
-                                accumulate = 1u;
-                                a_lo += 2u; b_lo += 2u;
-                            }
-                            a_lo += a_next_atom; b_lo += b_next_atom;
-                        }
+                        // one accumulator: nothing to rotate.  The common tile_k values are unrolled completely, so
+                        // that an issue is two additions and the instruction.
+                        const uint32_t accumulate = it > 0 ? 1u : 0u;
+                        if (g.tile_k == 64) issue_steps<2, 4>(tmem_base, d_hi, a_lo, b_lo, a_atom, b_atom, g.idesc, accumulate);
+                        else if (g.tile_k == 32) issue_steps<1, 4>(tmem_base, d_hi, a_lo, b_lo, a_atom, b_atom, g.idesc, accumulate);
+                        else if (g.tile_k == 128) issue_steps<4, 4>(tmem_base, d_hi, a_lo, b_lo, a_atom, b_atom, g.idesc, accumulate);
+                        else if (g.tile_k == 16) issue_steps<1, 2>(tmem_base, d_hi, a_lo, b_lo, a_atom, b_atom, g.idesc, accumulate);
+                        else issue_steps<1, 1>(tmem_base, d_hi, a_lo, b_lo, a_atom, b_atom, g.idesc, accumulate);
                     } else
 #pragma unroll 1
                     for (int at = 0; at < g.n_atoms; ++at) {
