@@ -360,3 +360,44 @@ def test_chained_kernels_on_one_stream_see_each_others_results():
         assert wl.status() == B.TT_OK
         wl.close()
     del first
+
+
+def _sampled_filters_ok(spec, rec, seed):
+    a = W.make_inputs(spec, seed)
+    y = run_spec(spec, rec, a)
+    ks = sorted({0, spec.shapes.k // 2 + 1, spec.shapes.k - 1})
+    sub = orc.conv2d(a["x"], a["w"][ks], a["bias"][ks], (spec.shapes.stride_h,) * 2, (spec.shapes.pad_h,) * 2, spec.shapes.act)
+    assert util.rel_l2(y[:, ks], sub) <= util.TOL_TF32, (spec.name, rec.short())
+
+
+def test_vgg_shaped_pool_source_convs_sampled_filters():
+    """The widest images of the pool sources (224 x 224: the slab rows are 228 floats, chunks of a few channels) and a
+    512-channel layer whose reduction needs many slab chunks, checked on sampled filters."""
+    recs = [tc(tile_n=128, tile_k=32, stages=3, mma_m_axis=1),
+            tc(tile_n=256, tile_k=64, stages=2, slab_tiles=2, mma_m_axis=1),
+            tc(tile_n=64, tile_k=32, stages=2, split_k=3, mma_m_axis=2)]
+    for i, spec in enumerate([W._conv(3, 224, 64, 3, 1, 1), W._conv(64, 224, 64, 3, 1, 1), W._conv(512, 28, 512, 3, 1, 1)]):
+        for rec in recs:
+            _sampled_filters_ok(spec, rec, 70 + i)
+
+
+def test_batched_kernels_of_the_saturating_size_points():
+    """The batched shapes that bench.py times at saturating size, at a smaller batch, under the records it uses:
+    sampled filters for the convolutions, every output for depthwise and softmax."""
+    conv = W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(6, 128, 28, 28, 128, 3, 3, 1, 1, True, B.TT_ACT_RELU), 1, "conv3x3_n6_128x28")
+    _sampled_filters_ok(conv, tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), 80)
+    _sampled_filters_ok(conv, tc(tile_n=128, tile_k=64, stages=2, mma_m_axis=2), 80)
+    pw = W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(5, 256, 56, 56, 64, 1, 1, 1, 0, True, B.TT_ACT_RELU), 1, "conv1x1_n5_256x56")
+    _sampled_filters_ok(pw, tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), 81)
+    dw = W.Spec(B.TT_OP_DWCONV2D, B.make_shapes(n=3, c=144, h=56, w=56, k=144, r=3, s=3, stride_h=1, stride_w=1, pad_h=1,
+                                                  pad_w=1, has_bias=1, act=B.TT_ACT_RELU6), 1, "dw_n3_144x56")
+    a = W.make_inputs(dw, 82)
+    ref = util.oracle_ref(dw, a)
+    for rec in (B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=8, block_y=56, block_x=56, items_per_thread=8, vec_width=4,
+                              threads=128, unroll=2),
+                B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=4, block_y=16, block_x=56, items_per_thread=4, vec_width=4,
+                              threads=128, unroll=4)):
+        run_spec(dw, rec, a, ref)
+    sm = W.Spec(B.TT_OP_SOFTMAX, B.softmax_shapes(12 * 8, 128, 128, 0.125), 1, "softmax_96x128x128", "bert")
+    a = W.make_inputs(sm, 83)
+    run_spec(sm, B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=16, block_y=4, vec_width=4), a, util.oracle_ref(sm, a))
