@@ -712,6 +712,13 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const int n_groups = im2col ? 1 : (g.stages >= 4 ? 4 : (g.stages >= 2 ? 2 : 1));
     const int wpg = kGatherWarps / n_groups;
 
+    if (threadIdx.x == 32) {
+        // the tensor maps are fetched ahead of their first use (they are kernel parameters: nothing the previous
+        // kernel of the stream could still be writing)
+        if (g.a_mode == OPM_TMA) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
+        if (g.b_mode == OPM_TMA) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+        if (g.slab_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+    }
     if (threadIdx.x == 0) {
         const uint32_t full_count = (any_tma ? 1u : 0u) + (any_gather ? (uint32_t)wpg : 0u);
         for (int s = 0; s < g.stages; ++s) {
