@@ -93,7 +93,7 @@ typedef struct tt_shapes {
  *   cache buffer / ComputeAt -> the accumulator lives in tensor memory and the bias/activation run on read-out;
  *                               `stages` shared-memory buffers decouple loading from the multiply
  *   Vectorize -> vec_width;   Unroll -> unroll / items_per_thread
- * GEMM_TC uses tile_m, tile_n, tile_k, stages, split_k, raster, mma_m_axis, slab_tiles, acc_split.
+ * GEMM_TC uses tile_m, tile_n, tile_k, stages, split_k, raster, mma_m_axis, slab_tiles, acc_split, k_order.
  * DW_SIMT uses tile_m (channels per CTA), block_y x block_x (output rows x columns per CTA tile),
  *         items_per_thread (consecutive outputs along the width per thread), vec_width, threads, and unroll:
  *         0 = shared-memory staged kernel; 1, 2, 4 = register-window kernel with that many output rows per thread
@@ -116,7 +116,12 @@ typedef struct tt_schedule_record {
                               8-wide reduction steps are dealt round-robin; they are added in fixed order on read-out.
                               Consecutive multiply-accumulates into one accumulator wait for each other; into several,
                               they overlap (the reduction-factoring of a schedule). */
-    int32_t reserved[1];
+    int32_t k_order;       /* GEMM_TC, conv2d: order in which the reduction (c, r, s) is walked.  0 = as the filters are
+                              stored (channel-major; the im2col operand is expanded stage by stage).  1 = blocks of 32
+                              channels, tap by tap inside a block: the filters are re-packed into that order by a small
+                              kernel before each run, the input rows are transposed once per block into a pixel-major
+                              slab, and every tap's operand tile is a shifted view of that slab -- no expansion.
+                              Stride-1 convolutions with 16-byte image rows, filters on the 128 rows, split_k = 1. */
 } tt_schedule_record;
 
 typedef struct tt_tensors {
@@ -145,7 +150,7 @@ typedef struct tt_apply_info {
 } tt_apply_info;
 
 enum { TT_CHG_TILE_M = 1, TT_CHG_TILE_N = 2, TT_CHG_TILE_K = 4, TT_CHG_STAGES = 8, TT_CHG_SPLIT_K = 16,
-       TT_CHG_VEC = 32, TT_CHG_BLOCK = 64, TT_CHG_ITEMS = 128, TT_CHG_SLAB = 256, TT_CHG_ACC = 512 };
+       TT_CHG_VEC = 32, TT_CHG_BLOCK = 64, TT_CHG_ITEMS = 128, TT_CHG_SLAB = 256, TT_CHG_ACC = 512, TT_CHG_KORDER = 1024 };
 
 /* Validity modes for mapping a record onto another shape (Section 4.1).
  *   TT_MODE_LEGALISE  reformulate: clamp/round tile sizes to the new extents and the hardware's legal set,

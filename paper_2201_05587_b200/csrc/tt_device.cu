@@ -15,6 +15,7 @@ cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* t
 cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st);
 cudaError_t launch_row(const tt_apply_info& I, const RowArgs& row, cudaStream_t st);
 cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits);
+cudaError_t launch_repack(const float* w, float* out, int kout, int C, int RS, int CB, cudaStream_t st);
 
 namespace {
 
@@ -112,7 +113,7 @@ tt_status bind_device(tt_workload* w) {
         if (cudaMalloc(&w->workspace, need) != cudaSuccess) { cudaGetLastError(); return TT_ERR_OOM; }
         w->workspace_bytes = need;
     }
-    if (need > 0) {
+    if (need > 0 && !w->plan.repack) {
         // arrival counters start at zero; each launch leaves them at zero again
         const size_t off = (size_t)w->plan.partial_bytes;
         if (cudaMemset(static_cast<char*>(w->workspace) + off, 0, need - off) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
@@ -121,7 +122,7 @@ tt_status bind_device(tt_workload* w) {
         if (cudaMalloc(reinterpret_cast<void**>(&w->status_word), 512) != cudaSuccess) { cudaGetLastError(); return TT_ERR_OOM; }
         if (cudaMemset(w->status_word, 0, 512) != cudaSuccess) return TT_ERR_CUDA;
     }
-    if (w->op == TT_OP_CONV2D) {
+    if (w->op == TT_OP_CONV2D && !w->plan.g.tap_major) {
         // reduction-index table of the applied record: byte offset of (c, r, s) inside the slab, channel counted
         // from 0 (the kernel rebases it per chunk); indices past K point at the last channel, whose products meet
         // zero-filled filter values
@@ -192,6 +193,12 @@ tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
         GemmArgs g = p.g;
         const void* a_ptr = pick(t, p.a_tensor);
         const void* b_ptr = pick(t, p.b_tensor);
+        if (p.repack) {
+            // tap-major convolution: the filters are brought into [filter][32-channel block][tap][channel] order first
+            if (launch_repack(static_cast<const float*>(t->w), static_cast<float*>(w->workspace), g.M, g.C, g.R * g.S,
+                              p.repack_cb, st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+            a_ptr = w->workspace;
+        }
         const TmapPair* maps = nullptr;
         tt_status s = tensor_maps_for(w, a_ptr, b_ptr, &maps);
         if (s != TT_OK) return s;

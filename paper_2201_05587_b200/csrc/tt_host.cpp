@@ -77,7 +77,115 @@ size_t tensor_elems(const tt_workload* w, int which) {
 
 // ---- legalisation -------------------------------------------------------------------------------------------
 
+// conv2d with k_order = 1: the reduction walks blocks of 32 channels and, inside a block, tap by tap.  Filters are
+// re-packed into that order ([filter][block][tap][32 channels], zero-padded) before each run and arrive by TMA;
+// the output columns are padded-linear pixels n = p * (W + gap) + q', so that the operand tile of tap (r, s) is the
+// pixel-major slab read (r * (W + gap) + s) rows further down -- a view, no expansion.  Columns with q' >= Q are
+// computed and dropped.
+static bool tap_major_possible(const tt_workload* w) {
+    const tt_shapes& s = w->sh;
+    return w->op == TT_OP_CONV2D && s.stride_h == 1 && s.stride_w == 1 && (s.w % 4) == 0 && !s.has_residual &&
+           s.r * s.s <= 64 && (long long)w->P * w->Q > 1;
+}
+
+static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_record* rec, int mode, Plan* plan) {
+    tt_apply_info& I = plan->info;
+    const tt_shapes& s = w->sh;
+    const bool strict = mode == TT_MODE_STRICT;
+    tt_schedule_record L = *rec;
+    int changed = 0;
+    const int RS = s.r * s.s, CB = (s.c + 31) / 32;
+    const int gap = round_up(std::max(1, std::max(s.pad_w, s.s - 1 - s.pad_w)), 4), wp = s.w + gap;
+    if (wp > 256) return TT_ERR_RESOURCE;
+    const int M = s.k, B = s.n;
+    const long long Nl = (long long)w->P * wp;            // padded-linear output pixels
+    if (Nl > 0x7fffffffLL) return TT_ERR_RESOURCE;
+    const int N = (int)Nl, K = CB * RS * 32;
+    // fixed by the mode: filters on the 128 rows, 32-wide reduction tiles, no split-K, one accumulator
+    if (strict && (rec->mma_m_axis == 2 || rec->tile_k != 32 || rec->split_k != 1)) return TT_ERR_INVALID_SCHEDULE;
+    L.mma_m_axis = 1; L.tile_m = kHwTileM; L.tile_k = 32; L.split_k = 1; L.acc_split = 1; L.slab_tiles = 0; L.k_order = 1;
+    if (rec->tile_m != kHwTileM) changed |= TT_CHG_TILE_M;
+    if (rec->tile_k != 32) changed |= TT_CHG_TILE_K;
+    if (rec->split_k != 1) changed |= TT_CHG_SPLIT_K;
+    int tn = std::min(256, std::max(16, round_up(rec->tile_n, 16)));
+    tn = std::min(tn, round_up(N, 16));
+    if (tn != rec->tile_n) changed |= TT_CHG_TILE_N;
+    L.tile_n = tn;
+    const int k_tiles = CB * RS;
+    int st = std::min(std::min(kMaxStages, rec->stages), k_tiles);
+    if (st != rec->stages) changed |= TT_CHG_STAGES;
+    if (strict && (changed & ~TT_CHG_TILE_M)) return TT_ERR_INVALID_SCHEDULE;
+    // shared memory: filter stages | NCHW staging of a block (TMA box [32][in_rows][wp], two buffers) | pixel-major slab
+    // (two buffers of (in_rows * wp + reach) rows of 128 bytes)
+    const int out_rows = std::min(w->P, (tn + wp - 2) / wp + 1);
+    const int in_rows = out_rows - 1 + s.r;
+    if (in_rows > 256) return TT_ERR_RESOURCE;
+    const unsigned a_stage = kHwTileM * 128;
+    const long long s_buf = (((long long)32 * in_rows * wp) * 4 + 127) / 128 * 128;
+    // furthest row a tile's views can touch (all tile_n rows are read, also those of pixels past the image)
+    const long long pm_rows = (long long)((tn + wp - 2) / wp + s.r) * wp + s.s + gap + 8;
+    const long long pm_buf = pm_rows * 128;
+    const int nbuf = CB > 1 ? 2 : 1;
+    long long smem = 0;
+    const long long min_pipe = (long long)kGatherWarps * 32 * 36 * 4;
+    for (;;) {
+        const long long pipe = std::max<long long>((long long)st * a_stage, min_pipe);
+        smem = pipe + nbuf * s_buf + nbuf * pm_buf + 1024;
+        if (smem <= kDynSmemLimit || strict || st <= 1) break;
+        --st; changed |= TT_CHG_STAGES;
+    }
+    L.stages = st;
+    const long long pipe = std::max<long long>((long long)st * a_stage, min_pipe);
+    const int tiles_m = (M + kHwTileM - 1) / kHwTileM, tiles_n = (N + tn - 1) / tn;
+    I = tt_apply_info{};
+    I.legal = L; I.changed = changed;
+    I.grid_x = tiles_m * tiles_n; I.grid_y = 1; I.grid_z = B;
+    I.threads = kGemmThreads;
+    I.smem_bytes = (int)std::min<long long>(smem, 0x7fffffff);
+    I.tmem_cols = std::max(32, pow2_ceil(tn));
+    I.workspace_bytes = (int64_t)M * K * 4;              // the re-packed filters
+    I.launches = 2;
+    if (smem > kDynSmemLimit || (long long)tiles_m * tiles_n > 0x7fffffffLL || B > 65535) return TT_ERR_RESOURCE;
+    plan->swap_ab = false;
+    plan->gm = M; plan->gn = N; plan->gk = K; plan->gbatch = B;
+    plan->partial_bytes = 0;
+    plan->repack = true; plan->repack_cb = CB;
+    plan->a_tensor = 1; plan->b_tensor = 0;               // A: filters (re-packed), B: the image
+    GemmArgs& g = plan->g;
+    g = GemmArgs{};
+    g.M = M; g.N = N; g.K = K; g.batch = B;
+    g.tile_n = tn; g.tile_k = 32; g.stages = st;
+    g.k_tiles = k_tiles; g.k_tiles_per_split = k_tiles; g.split_k = 1;
+    g.tiles_m = tiles_m; g.tiles_n = tiles_n; g.raster = L.raster;
+    g.atom_k = 32; g.n_atoms = 1; g.row_bytes = 128; g.swz_mask = 7;
+    g.a_stage_bytes = a_stage; g.b_stage_bytes = 0; g.tx_bytes = a_stage;
+    g.tmem_cols = (unsigned)I.tmem_cols; g.n_acc = 1; g.cluster = 0;
+    g.idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(tn >> 3) << 17) | ((unsigned)(kHwTileM >> 4) << 24);
+    g.a_mode = OPM_TMA; g.a_rs = K; g.a_ks = 1; g.a_bs = 0; g.a_tma_batched = 0;
+    g.b_mode = OPM_IM2COL_T; g.b_rs = 0; g.b_ks = 0; g.b_bs = (long long)s.c * s.h * s.w; g.b_tma_batched = 1;
+    g.y_ms = (long long)w->P * w->Q; g.y_ns = 1; g.y_bs = (long long)s.k * w->P * w->Q;
+    g.bias_mode = s.has_bias ? 1 : 0;
+    g.act = s.act;
+    g.C = s.c; g.H = s.h; g.W = s.w; g.R = s.r; g.S = s.s; g.Q = w->Q; g.Pout = w->P;
+    g.sh = 1; g.sw = 1; g.ph = s.pad_h; g.pw = s.pad_w;
+    g.vec_store = 0;
+    g.tap_major = 1;
+    g.slab_tma = 1; g.slab_tiles = RS; g.slab_nbuf = nbuf;
+    g.slab_off = (unsigned)pipe; g.slab_buf_bytes = (unsigned)s_buf;
+    g.slab_wp = wp; g.slab_gap = gap; g.slab_chpitch = in_rows * wp; g.slab_in_rows = in_rows; g.slab_rstep = 1;
+    g.slab_box_ch = std::min(32, s.c);                   // (fewer than 32 channels: the rest of the staging buffer stays zero)
+    g.slab_box_bytes = (unsigned)((long long)g.slab_box_ch * in_rows * wp * 4);
+    g.slab_vec16 = 1;
+    g.pm_off = (unsigned)(pipe + nbuf * s_buf); g.pm_buf_bytes = (unsigned)pm_buf;
+    return TT_OK;
+}
+
 static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* rec, int mode, Plan* plan) {
+    if (rec->k_order < 0 || rec->k_order > 1) return TT_ERR_INVALID_SCHEDULE;
+    if (rec->k_order == 1) {
+        if (tap_major_possible(w)) return legalise_conv_tapmajor(w, rec, mode, plan);
+        if (mode == TT_MODE_STRICT) return TT_ERR_INVALID_SCHEDULE;       // no such reduction order on this kernel
+    }
     tt_apply_info& I = plan->info;
     tt_schedule_record L = *rec;
     int changed = 0;
@@ -91,6 +199,9 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     bool swap = rec->mma_m_axis == 2;
     if (rec->mma_m_axis == 0) swap = w->view.gm <= 64 && w->view.gn > w->view.gm;
     L.mma_m_axis = swap ? 2 : 1;
+    L.k_order = 0;
+    if (rec->k_order != 0) changed |= TT_CHG_KORDER;    // reformulated: the stored channel-major order
+    plan->repack = false;
     plan->swap_ab = swap;
     plan->gm = swap ? w->view.gn : w->view.gm;
     plan->gn = swap ? w->view.gm : w->view.gn;

@@ -20,7 +20,9 @@ enum OperandMode : int {
     OPM_TMA = 0,          // K-major 2-D/3-D tensor map, hardware swizzle
     OPM_GATHER_ROWS = 1,  // strided view, lanes walk rows (row stride 1): 16-byte swizzled stores
     OPM_GATHER_K = 2,     // strided view, lanes walk k (k stride 1): 4-byte swizzled stores
-    OPM_IM2COL = 3        // rows are output pixels, k = (c, r, s): gathered from NCHW
+    OPM_IM2COL = 3,       // rows are output pixels, k = (c, r, s): expanded from a slab of NCHW input rows
+    OPM_IM2COL_T = 4      // rows are padded-linear output pixels, k = (32-channel block, tap, channel): every tap's tile
+                          // is a shifted view of a pixel-major slab in shared memory (nothing is staged per tile)
 };
 
 // Device-side arguments of the GEMM_TC kernel (plain data, passed by value).
@@ -63,6 +65,9 @@ struct GemmArgs {
     int slab_tma;                               // 1: chunks arrive by TMA; 0: by cp.async from the gather warps
     int slab_box_ch;                            // channels per box
     unsigned slab_box_bytes;
+    unsigned pm_off, pm_buf_bytes;              // tap-major convolutions: the pixel-major slab buffers (two)
+    int tap_major;                              // 1: OPM_IM2COL_T on operand B
+    int Pout;                                   // output rows (padded-linear pixel -> (p, q'))
     const int* ktab_dev;                        // per reduction index: byte offset of (c, r, s) inside the slab (absolute channel)      // ceil(2^32 / d) for the exact small-range divisions of the slab loader
 };
 
@@ -90,6 +95,8 @@ struct Plan {
     int a_tensor = 0, b_tensor = 1;   // which caller tensor feeds operand A / B: 0 = x, 1 = w
     GemmArgs g{};
     long long partial_bytes = 0;      // counters start here inside the workspace
+    bool repack = false;              // tap-major convolution: filters are re-packed into the workspace before each run
+    int repack_cb = 0;                // 32-channel blocks
     DwArgs dw{};
     RowArgs row{};
 };

@@ -18,6 +18,7 @@
 #include <cuda.h>
 #include <cstdint>
 #include <cstring>
+#include <algorithm>
 #include "tt_internal.h"
 
 namespace tt {
@@ -580,6 +581,7 @@ constexpr int kStageBytesPerWarp = 32 * kStagePitch * 4;
 // ReLU, ReLU6 and "none" are one clamp with per-kernel bounds (no branch per element); GELU is a separate path.
 struct EpiArgs {
     float* ybase; const float* rbase; long long y_ms, y_ns; int M; float lo, hi; bool gelu, vec;
+    int lin_wp, lin_q, lin_p;   // lin_wp > 0: column n is the padded-linear pixel p * lin_wp + q', stored at p * lin_q + q' if q' < lin_q
 };
 
 __device__ __forceinline__ float finish_one(float v, const EpiArgs& e) {
@@ -615,6 +617,21 @@ __device__ __forceinline__ void epilogue_block(float (&v)[32], const EpiArgs& e,
                     t.z = finish_one(t.z + r4.z, e); t.w = finish_one(t.w + r4.w, e);
                 }
                 *reinterpret_cast<float4*>(e.ybase + o) = t;
+            } else if (e.lin_wp > 0) {
+                // tap-major convolution: drop the columns that fall into the gap between image rows
+                const float tv[4] = {t.x, t.y, t.z, t.w};
+                const bool row_ok = m < e.M;
+                const int n = nb + cc;
+                int p = n / e.lin_wp, q = n - p * e.lin_wp;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const bool ok = row_ok && cc + j < cnt && q < e.lin_q && p < e.lin_p;
+                    const long long oo = (long long)m * e.y_ms + (long long)p * e.lin_q + q;
+                    float out = tv[j];
+                    if (POST) out = finish_one(out + (ok ? __ldg(e.rbase + oo) : 0.f), e);
+                    if (ok) e.ybase[oo] = out;
+                    if (++q == e.lin_wp) { q = 0; ++p; }
+                }
             } else {
                 const float tv[4] = {t.x, t.y, t.z, t.w};
                 const bool row_ok = m < e.M;
@@ -655,6 +672,8 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __shared__ uint64_t accum_bar;
     __shared__ uint64_t slab_full[2];     // a slab chunk has landed (TMA)
     __shared__ uint64_t slab_empty[2];    // all gather warps are done with a slab buffer
+    __shared__ uint64_t pm_full[2];       // tap-major convolution: a pixel-major slab buffer has been written
+    __shared__ uint64_t pm_empty[2];      // ... and every multiply-accumulate that reads it has completed
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int last_split_flag;
@@ -698,13 +717,20 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const bool a_tma = g.a_mode == OPM_TMA, b_tma = g.b_mode == OPM_TMA;
     const bool any_tma = a_tma || b_tma, any_gather = !a_tma || !b_tma;
     const bool im2col = g.a_mode == OPM_IM2COL || g.b_mode == OPM_IM2COL;
-    const bool slab_tma = im2col && g.slab_tma != 0;
+    const bool tapm = g.tap_major != 0;               // conv2d, reduction walked by channel block and tap
+    const bool slab_tma = (im2col || tapm) && g.slab_tma != 0;
     // im2col geometry of this CTA: first output row of its pixels, the image row its slab starts at, slab chunks
     int ic_p_first = 0, ic_ih_lo = 0, ic_chunks = 0;
     if (im2col) {
         const int row0 = g.a_mode == OPM_IM2COL ? m0 : n0;
         ic_p_first = row0 / g.Q;
         ic_ih_lo = ic_p_first * g.sh - g.ph;
+        ic_chunks = (iters + g.slab_tiles - 1) / g.slab_tiles;
+    }
+    if (tapm) {
+        // the tile's columns are padded-linear pixels n = p * wp + q'
+        ic_p_first = n0 / g.slab_wp;
+        ic_ih_lo = ic_p_first - g.ph;
         ic_chunks = (iters + g.slab_tiles - 1) / g.slab_tiles;
     }
     // gather groups (global gathers only): 4 groups of 2 warps from 4 stages up, 2 groups of 4 warps for 2-3 stages,
@@ -720,7 +746,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         if (g.slab_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
     }
     if (threadIdx.x == 0) {
-        const uint32_t full_count = (any_tma ? 1u : 0u) + (any_gather ? (uint32_t)wpg : 0u);
+        const uint32_t full_count = tapm ? 1u : (any_tma ? 1u : 0u) + (any_gather ? (uint32_t)wpg : 0u);
         for (int s = 0; s < g.stages; ++s) {
             mbar_init(smem_u32(&full_bar[s]), full_count);
             mbar_init(smem_u32(&empty_bar[s]), 1u);
@@ -729,6 +755,8 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&slab_full[b]), 1u);
             mbar_init(smem_u32(&slab_empty[b]), (uint32_t)kGatherWarps);
+            mbar_init(smem_u32(&pm_full[b]), (uint32_t)kGatherWarps);
+            mbar_init(smem_u32(&pm_empty[b]), 1u);
         }
         abort_flag = 0;
         last_split_flag = 0;
@@ -858,6 +886,34 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const uint32_t d_end = tmem_base + (uint32_t)(g.n_acc * g.tile_n);
             int fresh = g.n_acc;                         // accumulators not written yet
             uint32_t a_stage = a_lo0, b_stage = b_lo0, full_addr = full0, empty_addr = empty0;
+            if (tapm) {
+                // Tap-major convolution: the B tile of reduction tile `it` = (channel block, tap (r, s)) is the
+                // pixel-major slab of that block read from row lin0 + r * wp + s on (128-byte rows, one per
+                // padded-linear pixel; the hardware swizzles on absolute addresses, so any start row works).
+                const uint32_t pm0 = tiles_base + g.pm_off;
+                const int RS = g.R * g.S;
+                const int lin0 = (n0 - ic_p_first * g.slab_wp) + g.slab_gap - g.pw;
+                int chunk = 0, tap = 0, fr = 0, fs = 0;
+                for (int it = 0; it < iters; ++it) {
+                    bool got = mbar_wait(full_addr, ph, abortp, g.status, 2u);                       // the filter tile
+                    if (tap == 0) got = mbar_wait(smem_u32(&pm_full[chunk & 1]), (uint32_t)(chunk >> 1) & 1u, abortp, g.status, 7u) && got;
+                    if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+                    if (lane == 0 && it == 0) TT_STAMP(2);
+                    tc_fence_after();
+                    if (leader) {
+                        const uint32_t row = (uint32_t)(lin0 + fr * g.slab_wp + fs);
+                        const uint32_t b_lo = d_lo + (((pm0 + (uint32_t)(chunk & 1) * g.pm_buf_bytes + row * 128u) & 0x3FFFFu) >> 4);
+                        issue_steps<1, 4>(tmem_base, d_hi, a_stage, b_lo, a_atom, b_atom, g.idesc, it > 0 ? 1u : 0u);
+                        mma_commit(empty_addr);                                                  // filter stage reusable
+                        if (tap == RS - 1) mma_commit(smem_u32(&pm_empty[chunk & 1]));             // slab buffer reusable
+                    }
+                    __syncwarp();
+                    if (++fs == g.S) { fs = 0; ++fr; }
+                    if (++tap == RS) { tap = 0; fr = 0; fs = 0; ++chunk; }
+                    a_stage += stage_step; full_addr += 8u; empty_addr += 8u;
+                    if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; a_stage = a_lo0; full_addr = full0; empty_addr = empty0; }
+                }
+            } else
             for (int it = 0; it < iters; ++it) {
                 const bool got = mbar_wait(full_addr, ph, abortp, g.status, 2u);
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
@@ -1027,6 +1083,57 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             }
             cp_async_wait<0>();
             if (threadIdx.x == 64) TT_STAMP(16);
+        } else if (tapm) {
+            // ---- conv2d, tap-major: transpose every 32-channel block of input rows, once, into a pixel-major slab ----
+            // staging buffer (TMA): [32 channels][in_rows][wp] floats; pixel-major slab: one 128-byte row per staged
+            // position (32 channels), 16-byte chunks swizzled by the row's absolute address like a TMA 128-byte tile.
+            const uint32_t st0 = tiles_base + g.slab_off, pm0 = tiles_base + g.pm_off;
+            const int npix = g.slab_in_rows * g.slab_wp;
+            // rows a view can touch beyond the transposed range must hold finite numbers: clear both buffers once
+            for (uint32_t o = (uint32_t)gt * 16u; o < (uint32_t)g.slab_nbuf * g.pm_buf_bytes; o += (uint32_t)kGatherThreads * 16u)
+                st_shared_v4(pm0 + o, 0.f, 0.f, 0.f, 0.f);
+            if (g.slab_box_ch < 32)                      // channels beyond the TMA box (which may already be landing) read as zero
+                for (int b = 0; b < g.slab_nbuf; ++b)
+                    for (uint32_t o = g.slab_box_bytes + (uint32_t)gt * 16u; o < g.slab_buf_bytes; o += (uint32_t)kGatherThreads * 16u)
+                        st_shared_v4(st0 + (uint32_t)b * g.slab_buf_bytes + o, 0.f, 0.f, 0.f, 0.f);
+            bool ok = gather_vote(true);
+            const uint32_t ch_bytes = 4u * (uint32_t)g.slab_chpitch;
+            for (int j = 0; j < ic_chunks; ++j) {
+                const int b = j & 1;
+                if (ok && !mbar_wait(smem_u32(&slab_full[b]), (uint32_t)(j >> 1) & 1u, abortp, g.status, 6u)) ok = false;
+                if (ok && j >= 2 && !mbar_wait(smem_u32(&pm_empty[b]), (uint32_t)((j - 2) >> 1) & 1u, abortp, g.status, 8u)) ok = false;
+                if (ok) {
+                    // warp gw moves channels 4 gw .. 4 gw + 3 of every staged position; lanes walk positions
+                    const uint32_t src = st0 + (uint32_t)b * g.slab_buf_bytes + (uint32_t)(4 * gw) * ch_bytes;
+                    const uint32_t dst = pm0 + (uint32_t)b * g.pm_buf_bytes;
+                    for (int p0 = lane; p0 < npix; p0 += 128) {
+                        float v[4][4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int pix = min(p0 + 32 * u, npix - 1);
+                            const uint32_t a = src + 4u * (uint32_t)pix;
+                            v[u][0] = ld_shared_f32(a);
+                            v[u][1] = ld_shared_f32(a + ch_bytes);
+                            v[u][2] = ld_shared_f32(a + 2u * ch_bytes);
+                            v[u][3] = ld_shared_f32(a + 3u * ch_bytes);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int pix = p0 + 32 * u;
+                            if (pix < npix) {
+                                const uint32_t rowa = dst + 128u * (uint32_t)pix;
+                                st_shared_v4(rowa + ((((uint32_t)gw) ^ ((rowa >> 7) & 7u)) << 4), v[u][0], v[u][1], v[u][2], v[u][3]);
+                            }
+                        }
+                    }
+                    fence_proxy_async_shared();          // generic-proxy stores -> visible to the tensor core's reads
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(smem_u32(&pm_full[b]));
+                        if (j + 2 < ic_chunks) mbar_arrive(smem_u32(&slab_empty[b]));   // the staging buffer may be refilled
+                    }
+                }
+            }
         } else if (any_gather) {
             const float* a_src = g.a + (long long)bz * g.a_bs;
             const float* b_src = g.b + (long long)bz * g.b_bs;
@@ -1162,6 +1269,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 e.hi = g.act == TT_ACT_RELU6 ? 6.f : INFINITY;
                 e.gelu = g.act == TT_ACT_GELU_ERF;
                 e.vec = (g.vec_store & 1) != 0;
+                e.lin_wp = tapm ? g.slab_wp : 0; e.lin_q = g.Q; e.lin_p = g.Pout;
                 const bool transposed = g.y_ns == 1 && g.y_ms != 1;
                 const uint32_t stg = tiles_base + (uint32_t)gw * (uint32_t)kStageBytesPerWarp;   // pipeline buffers are idle now
                 const int m_first = m0 + quad * 32;
@@ -1213,7 +1321,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         }
                     }
                     // full blocks take the unguarded path (16-byte accesses need the aligned layout when transposed)
-                    const bool full = cnt >= 32 && m_first + 32 <= g.M && (e.vec || !transposed);
+                    const bool full = !tapm && cnt >= 32 && m_first + 32 <= g.M && (e.vec || !transposed);
                     if (e.rbase == nullptr) {
                         // no residual: activate here, once, outside the store loops
                         if (e.gelu) {
@@ -1583,6 +1691,22 @@ __global__ void tt_softmax_cached_kernel(const RowArgs a) {
     }
 }
 
+// Filters [kout][C][RS] -> [kout][block of 32 channels][tap][channel in block], zero beyond C: the reduction order of the
+// tap-major convolution.  One thread per output element; reads walk the channels of a tap (stride RS), writes are
+// contiguous.
+__global__ void tt_repack_filters_kernel(const float* __restrict__ w, float* __restrict__ out, int kout, int C, int RS, int CB) {
+    const long long per_filter = (long long)CB * RS * 32;
+    const long long total = (long long)kout * per_filter;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long f = i / per_filter;
+        const int rem = (int)(i - f * per_filter);
+        const int ci = rem & 31, t2 = rem >> 5;
+        const int cb = t2 / RS, tap = t2 - cb * RS;
+        const int c = cb * 32 + ci;
+        out[i] = c < C ? __ldg(w + (f * C + c) * RS + tap) : 0.f;
+    }
+}
+
 // ------------------------------------------------------------------------------------------------------------
 // Launchers (called from tt_device.cu)
 // ------------------------------------------------------------------------------------------------------------
@@ -1635,6 +1759,13 @@ cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits) {
     if (e != cudaSuccess) return e;
     *fits = n > 0;
     return cudaSuccess;
+}
+
+cudaError_t launch_repack(const float* w, float* out, int kout, int C, int RS, int CB, cudaStream_t st) {
+    const long long total = (long long)kout * CB * RS * 32;
+    const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 8);
+    tt_repack_filters_kernel<<<blocks, 256, 0, st>>>(w, out, kout, C, RS, CB);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st) {
