@@ -494,7 +494,7 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
         tt_apply_info info;
         if (tt_schedule_check(w, &r, TT_MODE_LEGALISE, 0, &info) != TT_OK) return false;
         // (a pipeline made shallower to fit short reductions or shared memory is kept: exact duplicates are dropped below)
-        if (info.changed & ~(TT_CHG_TILE_M | TT_CHG_STAGES)) return false;
+        if (info.changed & ~(TT_CHG_TILE_M | TT_CHG_STAGES)) return false;      // (includes a reformulated reduction order)
         cand.push_back(info.legal);
         return true;
     };
@@ -509,6 +509,17 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
             tt_schedule_record r = base;
             r.mma_m_axis = ax; r.tile_m = kHwTileM; r.tile_n = tn; r.tile_k = tk; r.stages = sg; r.split_k = sk; r.raster = ra;
             push(r);
+        }
+        if (w->op == TT_OP_CONV2D) {
+            // the tap-major reduction order (records that ask for it on a kernel that has none are legalised back
+            // to the stored order and dropped here as duplicates-to-be)
+            for (int tn : full ? std::vector<int>{32, 64, 96, 128, 192, 256} : std::vector<int>{64, 128, 256})
+                for (int sg : full ? std::vector<int>{1, 2, 3, 4, 5, 6, 8} : std::vector<int>{2, 3, 5}) {
+                    tt_schedule_record r = base;
+                    r.mma_m_axis = 1; r.tile_m = kHwTileM; r.tile_n = tn; r.tile_k = 32; r.stages = sg; r.split_k = 1; r.raster = 0;
+                    r.k_order = 1;
+                    push(r);
+                }
         }
     } else if (w->family == TT_FAMILY_DW_SIMT) {
         const std::vector<int> tcs = full ? std::vector<int>{1, 2, 4, 8, 16, 32} : std::vector<int>{1, 4, 16};

@@ -84,8 +84,10 @@ size_t tensor_elems(const tt_workload* w, int which) {
 // computed and dropped.
 static bool tap_major_possible(const tt_workload* w) {
     const tt_shapes& s = w->sh;
+    const int gap = round_up(std::max(1, std::max(s.pad_w, s.s - 1 - s.pad_w)), 4);
+    // (an output row must fit a padded image row: the columns are numbered p * (W + gap) + q')
     return w->op == TT_OP_CONV2D && s.stride_h == 1 && s.stride_w == 1 && (s.w % 4) == 0 && !s.has_residual &&
-           s.r * s.s <= 64 && (long long)w->P * w->Q > 1;
+           s.r * s.s <= 64 && (long long)w->P * w->Q > 1 && w->Q <= s.w + gap;
 }
 
 static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_record* rec, int mode, Plan* plan) {
@@ -115,7 +117,7 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     int st = std::min(std::min(kMaxStages, rec->stages), k_tiles);
     if (st != rec->stages) changed |= TT_CHG_STAGES;
     if (strict && (changed & ~TT_CHG_TILE_M)) return TT_ERR_INVALID_SCHEDULE;
-    // shared memory: filter stages | NCHW staging of a block (TMA box [32][in_rows][wp], two buffers) | pixel-major slab
+    // shared memory: filter stages | NCHW staging of a block (TMA box [32][in_rows][wp], one buffer) | pixel-major slab
     // (two buffers of (in_rows * wp + reach) rows of 128 bytes)
     const int out_rows = std::min(w->P, (tn + wp - 2) / wp + 1);
     const int in_rows = out_rows - 1 + s.r;
@@ -130,7 +132,7 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     const long long min_pipe = (long long)kGatherWarps * 32 * 36 * 4;
     for (;;) {
         const long long pipe = std::max<long long>((long long)st * a_stage, min_pipe);
-        smem = pipe + nbuf * s_buf + nbuf * pm_buf + 1024;
+        smem = pipe + s_buf + nbuf * pm_buf + 1024;
         if (smem <= kDynSmemLimit || strict || st <= 1) break;
         --st; changed |= TT_CHG_STAGES;
     }
@@ -168,15 +170,15 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     g.act = s.act;
     g.C = s.c; g.H = s.h; g.W = s.w; g.R = s.r; g.S = s.s; g.Q = w->Q; g.Pout = w->P;
     g.sh = 1; g.sw = 1; g.ph = s.pad_h; g.pw = s.pad_w;
-    g.vec_store = 0;
+    g.vec_store = (w->Q % 4 == 0 && ((long long)w->P * w->Q) % 4 == 0) ? 1 : 0;   // a lane's four columns: one aligned 16-byte store
     g.tap_major = 1;
-    g.slab_tma = 1; g.slab_tiles = RS; g.slab_nbuf = nbuf;
+    g.slab_tma = 1; g.slab_tiles = RS; g.slab_nbuf = 1; g.pm_nbuf = nbuf;
     g.slab_off = (unsigned)pipe; g.slab_buf_bytes = (unsigned)s_buf;
     g.slab_wp = wp; g.slab_gap = gap; g.slab_chpitch = in_rows * wp; g.slab_in_rows = in_rows; g.slab_rstep = 1;
     g.slab_box_ch = std::min(32, s.c);                   // (fewer than 32 channels: the rest of the staging buffer stays zero)
     g.slab_box_bytes = (unsigned)((long long)g.slab_box_ch * in_rows * wp * 4);
     g.slab_vec16 = 1;
-    g.pm_off = (unsigned)(pipe + nbuf * s_buf); g.pm_buf_bytes = (unsigned)pm_buf;
+    g.pm_off = (unsigned)(pipe + s_buf); g.pm_buf_bytes = (unsigned)pm_buf;
     return TT_OK;
 }
 

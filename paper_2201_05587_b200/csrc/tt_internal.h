@@ -65,7 +65,7 @@ struct GemmArgs {
     int slab_tma;                               // 1: chunks arrive by TMA; 0: by cp.async from the gather warps
     int slab_box_ch;                            // channels per box
     unsigned slab_box_bytes;
-    unsigned pm_off, pm_buf_bytes;              // tap-major convolutions: the pixel-major slab buffers (two)
+    unsigned pm_off, pm_buf_bytes; int pm_nbuf; // tap-major convolutions: the pixel-major slab buffers (one or two)
     int tap_major;                              // 1: OPM_IM2COL_T on operand B
     int Pout;                                   // output rows (padded-linear pixel -> (p, q'))
     const int* ktab_dev;                        // per reduction index: byte offset of (c, r, s) inside the slab (absolute channel)      // ceil(2^32 / d) for the exact small-range divisions of the slab loader

@@ -602,6 +602,41 @@ __device__ __forceinline__ void epilogue_block(float (&v)[32], const EpiArgs& e,
         for (int j = 0; j < 32; j += 4) st_shared_v4(stg + (uint32_t)(lane * kStagePitch + j) * 4u, v[j], v[j + 1], v[j + 2], v[j + 3]);
         __syncwarp();
         const int cc = (lane & 7) * 4;
+        if (e.lin_wp > 0) {
+            // tap-major convolution: column n is the padded-linear pixel p * wp + q'.  A lane's four columns lie in one
+            // padded row (wp is a multiple of 4); when Q is one too, all four are outputs or all four fall into the gap.
+            const int n = nb + cc;
+            const int p = n / e.lin_wp, q = n - p * e.lin_wp;
+            const bool col_ok = cc < cnt && q < e.lin_q && p < e.lin_p;
+            const int nq = min(4, e.lin_q - q);          // outputs among the four (4 whenever Q is a multiple of 4)
+            const long long coff = (long long)p * e.lin_q + q;
+#pragma unroll
+            for (int itr = 0; itr < 8; ++itr) {
+                const int rr = itr * 4 + (lane >> 3);
+                const int m = m_first + rr;
+                float4 t;
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w)
+                             : "r"(stg + (uint32_t)(rr * kStagePitch + cc) * 4u));
+                if (col_ok && m < e.M) {
+                    const long long o = (long long)m * e.y_ms + coff;
+                    if (POST) {
+                        t.x = finish_one(t.x + __ldg(e.rbase + o), e);
+                        if (nq > 1) t.y = finish_one(t.y + __ldg(e.rbase + o + 1), e);
+                        if (nq > 2) t.z = finish_one(t.z + __ldg(e.rbase + o + 2), e);
+                        if (nq > 3) t.w = finish_one(t.w + __ldg(e.rbase + o + 3), e);
+                    }
+                    if (e.vec) *reinterpret_cast<float4*>(e.ybase + o) = t;      // (vec implies Q % 4 == 0)
+                    else {
+                        e.ybase[o] = t.x;
+                        if (nq > 1) e.ybase[o + 1] = t.y;
+                        if (nq > 2) e.ybase[o + 2] = t.z;
+                        if (nq > 3) e.ybase[o + 3] = t.w;
+                    }
+                }
+            }
+            __syncwarp();
+            return;
+        }
 #pragma unroll
         for (int itr = 0; itr < 8; ++itr) {
             const int rr = itr * 4 + (lane >> 3);
@@ -617,21 +652,6 @@ __device__ __forceinline__ void epilogue_block(float (&v)[32], const EpiArgs& e,
                     t.z = finish_one(t.z + r4.z, e); t.w = finish_one(t.w + r4.w, e);
                 }
                 *reinterpret_cast<float4*>(e.ybase + o) = t;
-            } else if (e.lin_wp > 0) {
-                // tap-major convolution: drop the columns that fall into the gap between image rows
-                const float tv[4] = {t.x, t.y, t.z, t.w};
-                const bool row_ok = m < e.M;
-                const int n = nb + cc;
-                int p = n / e.lin_wp, q = n - p * e.lin_wp;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const bool ok = row_ok && cc + j < cnt && q < e.lin_q && p < e.lin_p;
-                    const long long oo = (long long)m * e.y_ms + (long long)p * e.lin_q + q;
-                    float out = tv[j];
-                    if (POST) out = finish_one(out + (ok ? __ldg(e.rbase + oo) : 0.f), e);
-                    if (ok) e.ybase[oo] = out;
-                    if (++q == e.lin_wp) { q = 0; ++p; }
-                }
             } else {
                 const float tv[4] = {t.x, t.y, t.z, t.w};
                 const bool row_ok = m < e.M;
@@ -796,17 +816,20 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const int RS = g.R * g.S, T = g.slab_tiles;
             const uint32_t slab0 = tiles_base + g.slab_off;
             int slab_issued = 0;
+            // (the tap-major path has one staging buffer -- it is transposed away at once --, the other two)
+            const int sbufs = tapm ? 1 : 2;
             auto issue_chunk = [&](int j) {
-                const uint32_t bar = smem_u32(&slab_full[j & 1]);
+                const int b = tapm ? 0 : (j & 1);
+                const uint32_t bar = smem_u32(&slab_full[b]);
                 mbar_expect_tx(bar, g.slab_box_bytes);
-                tma_load_4d(slab0 + (uint32_t)(j & 1) * g.slab_buf_bytes, &tmap_x, bar, -g.slab_gap, ic_ih_lo,
+                tma_load_4d(slab0 + (uint32_t)b * g.slab_buf_bytes, &tmap_x, bar, -g.slab_gap, ic_ih_lo,
                             (kt_begin * g.tile_k + j * T * g.tile_k) / RS, bz);
             };
             if (slab_tma) {
-                if (leader) { issue_chunk(0); if (ic_chunks > 1) issue_chunk(1); }
-                slab_issued = min(ic_chunks, 2);
+                if (leader) { issue_chunk(0); if (sbufs > 1 && ic_chunks > 1) issue_chunk(1); }
+                slab_issued = min(ic_chunks, sbufs);
             }
-            int next_slab_it = slab_tma ? T : 0x7fffffff;    // chunk `slab_issued` is requested when chunk slab_issued-1 starts
+            int next_slab_it = slab_tma ? (slab_issued - 1) * T : 0x7fffffff;   // chunk `slab_issued` is requested when chunk slab_issued-1 starts
             bool ok = true;
             for (int it = 0; it < iters; ++it, k0 += g.tile_k) {
                 if (it == next_slab_it) {
@@ -814,7 +837,8 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (slab_issued < ic_chunks) {
                         // its buffer is free once the gather warps have left chunk slab_issued - 2
                         const int j = slab_issued;
-                        const bool freed = mbar_wait(smem_u32(&slab_empty[j & 1]), (uint32_t)((j - 2) >> 1) & 1u, abortp, g.status, 5u);
+                        const bool freed = tapm ? mbar_wait(smem_u32(&slab_empty[0]), (uint32_t)(j - 1) & 1u, abortp, g.status, 5u)
+                                                : mbar_wait(smem_u32(&slab_empty[j & 1]), (uint32_t)((j - 2) >> 1) & 1u, abortp, g.status, 5u);
                         if (!__all_sync(0xffffffffu, freed)) { ok = false; break; }
                         if (leader) issue_chunk(j);
                         ++slab_issued;
@@ -854,9 +878,9 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         if (global_timer_ns() - t0 > 2000000ull) break;
                     }
                 }
-                for (int j = max(0, slab_issued - 2); j < slab_issued; ++j) {
+                for (int j = max(0, slab_issued - sbufs); j < slab_issued; ++j) {
                     const unsigned long long t0 = global_timer_ns();
-                    while (!mbar_try_wait(smem_u32(&slab_full[j & 1]), (uint32_t)(j >> 1) & 1u)) {
+                    while (!mbar_try_wait(smem_u32(&slab_full[tapm ? 0 : (j & 1)]), (uint32_t)(tapm ? j : (j >> 1)) & 1u)) {
                         if (global_timer_ns() - t0 > 2000000ull) break;
                     }
                 }
@@ -899,6 +923,10 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (tap == 0) got = mbar_wait(smem_u32(&pm_full[chunk & 1]), (uint32_t)(chunk >> 1) & 1u, abortp, g.status, 7u) && got;
                     if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                     if (lane == 0 && it == 0) TT_STAMP(2);
+                    if (lane == 0 && it == 14) TT_STAMP(12);
+                    if (lane == 0 && it == 15) TT_STAMP(13);
+                    if (lane == 0 && it == 18) TT_STAMP(10);
+                    if (lane == 0 && it == 27) TT_STAMP(11);
                     tc_fence_after();
                     if (leader) {
                         const uint32_t row = (uint32_t)(lin0 + fr * g.slab_wp + fs);
@@ -1090,21 +1118,22 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const uint32_t st0 = tiles_base + g.slab_off, pm0 = tiles_base + g.pm_off;
             const int npix = g.slab_in_rows * g.slab_wp;
             // rows a view can touch beyond the transposed range must hold finite numbers: clear both buffers once
-            for (uint32_t o = (uint32_t)gt * 16u; o < (uint32_t)g.slab_nbuf * g.pm_buf_bytes; o += (uint32_t)kGatherThreads * 16u)
+            for (uint32_t o = (uint32_t)gt * 16u; o < (uint32_t)g.pm_nbuf * g.pm_buf_bytes; o += (uint32_t)kGatherThreads * 16u)
                 st_shared_v4(pm0 + o, 0.f, 0.f, 0.f, 0.f);
             if (g.slab_box_ch < 32)                      // channels beyond the TMA box (which may already be landing) read as zero
-                for (int b = 0; b < g.slab_nbuf; ++b)
-                    for (uint32_t o = g.slab_box_bytes + (uint32_t)gt * 16u; o < g.slab_buf_bytes; o += (uint32_t)kGatherThreads * 16u)
-                        st_shared_v4(st0 + (uint32_t)b * g.slab_buf_bytes + o, 0.f, 0.f, 0.f, 0.f);
+                for (uint32_t o = g.slab_box_bytes + (uint32_t)gt * 16u; o < g.slab_buf_bytes; o += (uint32_t)kGatherThreads * 16u)
+                    st_shared_v4(st0 + o, 0.f, 0.f, 0.f, 0.f);
             bool ok = gather_vote(true);
             const uint32_t ch_bytes = 4u * (uint32_t)g.slab_chpitch;
             for (int j = 0; j < ic_chunks; ++j) {
-                const int b = j & 1;
-                if (ok && !mbar_wait(smem_u32(&slab_full[b]), (uint32_t)(j >> 1) & 1u, abortp, g.status, 6u)) ok = false;
+                const int b = j & 1;                     // pixel-major buffer; the staging buffer is always the same one
+                if (ok && !mbar_wait(smem_u32(&slab_full[0]), (uint32_t)j & 1u, abortp, g.status, 6u)) ok = false;
+                if (threadIdx.x == 64 && j == 1) TT_STAMP(15);
+                if (threadIdx.x == 64 && j == 2) TT_STAMP(22);
                 if (ok && j >= 2 && !mbar_wait(smem_u32(&pm_empty[b]), (uint32_t)((j - 2) >> 1) & 1u, abortp, g.status, 8u)) ok = false;
                 if (ok) {
                     // warp gw moves channels 4 gw .. 4 gw + 3 of every staged position; lanes walk positions
-                    const uint32_t src = st0 + (uint32_t)b * g.slab_buf_bytes + (uint32_t)(4 * gw) * ch_bytes;
+                    const uint32_t src = st0 + (uint32_t)(4 * gw) * ch_bytes;
                     const uint32_t dst = pm0 + (uint32_t)b * g.pm_buf_bytes;
                     for (int p0 = lane; p0 < npix; p0 += 128) {
                         float v[4][4];
@@ -1128,9 +1157,11 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                     fence_proxy_async_shared();          // generic-proxy stores -> visible to the tensor core's reads
                     __syncwarp();
+                    if (threadIdx.x == 64 && j == 1) TT_STAMP(16);
+                    if (threadIdx.x == 64 && j == 2) TT_STAMP(23);
                     if (lane == 0) {
                         mbar_arrive(smem_u32(&pm_full[b]));
-                        if (j + 2 < ic_chunks) mbar_arrive(smem_u32(&slab_empty[b]));   // the staging buffer may be refilled
+                        if (j + 1 < ic_chunks) mbar_arrive(smem_u32(&slab_empty[0]));   // the staging buffer may be refilled
                     }
                 }
             }

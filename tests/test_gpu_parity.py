@@ -52,6 +52,10 @@ GEMM_RECORDS = [
     tc(tile_n=32, tile_k=8, stages=4, split_k=2, slab_tiles=3, mma_m_axis=1),
     # more than 8 splits: partial tiles through the global workspace (2..8 splits reduce inside a thread-block cluster)
     tc(tile_n=64, tile_k=16, stages=2, split_k=12, mma_m_axis=1),
+    # tap-major reduction order (stride-1 convolutions with 16-byte image rows; elsewhere legalised to the stored order)
+    tc(tile_n=128, tile_k=32, stages=3, k_order=1, mma_m_axis=1),
+    tc(tile_n=256, tile_k=64, stages=2, k_order=1, split_k=2, mma_m_axis=2),
+    tc(tile_n=48, tile_k=32, stages=1, k_order=1, raster=1, mma_m_axis=1),
     # several accumulators in tensor memory, reduction steps dealt round-robin, summed on read-out
     tc(tile_n=32, tile_k=32, stages=4, acc_split=4, mma_m_axis=1),
     tc(tile_n=48, tile_k=16, stages=3, acc_split=8, split_k=2, mma_m_axis=2),
@@ -69,7 +73,7 @@ def check_all_records(spec, seed, records=GEMM_RECORDS):
     assert all(probe.check(r)[0] in (B.TT_OK, B.TT_ERR_RESOURCE) for r in records)
     assert probe.check(probe.default_schedule())[0] == B.TT_OK
     probe.close()
-    assert len(valid) >= len(records) - 3
+    assert len(valid) >= len(records) - 4
     outs = [run_spec(spec, r, a, ref) for r in valid]
     # a schedule changes speed, never semantics: every valid record gives the same output up to the order of the
     # fp32 additions (tile_k and split_k regroup them): sqrt(K) * 2^-24 is about 4e-6 at the largest K here
@@ -100,6 +104,9 @@ def test_dense_parity_all_records(spec):
     W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(2, 8, 9, 11, 12, 3, 3, 1, 1, True, B.TT_ACT_RELU, True), 1, "batch2_residual", "uniform"),
     W.Spec(B.TT_OP_CONV2D, B.make_shapes(n=1, c=6, h=10, w=12, k=9, r=3, s=2, stride_h=2, stride_w=1, pad_h=0, pad_w=1,
                                          has_bias=0, act=B.TT_ACT_NONE), 1, "asym_nobias", "uniform"),
+    W._conv(20, 12, 40, 3, 1, 1, name="conv3x3_12x12_tap"),                 # rows of 48 bytes: the tap-major path applies
+    W._conv(72, 16, 136, 3, 1, 1, act=B.TT_ACT_NONE, name="conv3x3_72ch_tap"),   # 3 channel blocks (the last one partial), 2 filter tiles
+    W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(2, 33, 8, 20, 10, 5, 3, 1, 2, True, B.TT_ACT_RELU6), 1, "conv5x3_batch2_tap", "uniform"),
     W._conv(20, 10, 40, 1, 1, 0, name="conv1x1_100px_20ch"),
     W._conv(136, 12, 200, 1, 1, 0, act=B.TT_ACT_NONE, name="conv1x1_136ch"),
     W._conv(96, 9, 48, 3, 1, 1, name="conv3x3_96ch_chunks"),                # 864 reduction indices: many slab chunks

@@ -241,3 +241,23 @@ def test_rank_pools_matches_the_oracle_on_the_papers_tables():
         assert [cands[i] for i in order[:len(choices[target])]] == choices[target]
     with pytest.raises(B.TTError):
         B.rank_pools([0.5], [[-1]])
+
+
+def test_tap_major_reduction_order_is_legalised_per_kernel():
+    """k_order = 1 exists for stride-1 convolutions whose image rows are 16-byte multiples; elsewhere the record is
+    reformulated to the stored order (legalise) or invalid (strict)."""
+    rec = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=128, tile_k=32, stages=3, k_order=1, mma_m_axis=1)
+    st, info = W._conv(64, 28, 64, 3, 1, 1).workload().check(rec)
+    assert st == B.TT_OK and info.legal.k_order == 1 and info.launches == 2
+    assert info.workspace_bytes == 64 * 2 * 9 * 32 * 4        # re-packed filters: 2 blocks of 32 channels x 9 taps
+    assert info.grid_x == (28 * 32 + 127) // 128              # padded-linear pixels: 28 rows of 28 + 4
+    for sp in (W._conv(64, 56, 128, 3, 2, 1), W._conv(64, 14, 64, 3, 1, 1), W._dense(128, 768, 768)):
+        wl = sp.workload()
+        st, info = wl.check(rec)
+        assert st == B.TT_OK and info.legal.k_order == 0 and info.changed & B.TT_CHG_KORDER and info.launches == 1
+        assert wl.check(rec, mode=B.TT_MODE_STRICT)[0] == B.TT_ERR_INVALID_SCHEDULE
+    # the mode fixes tile_k, split_k and the row axis; other values are reformulated
+    odd = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=100, tile_k=64, stages=9, split_k=4, k_order=1, mma_m_axis=2)
+    st, info = W._conv(64, 28, 64, 3, 1, 1).workload().check(odd)
+    L = info.legal
+    assert st == B.TT_OK and (L.tile_n, L.tile_k, L.split_k, L.mma_m_axis, L.k_order) == (112, 32, 1, 1, 1) and L.stages <= 8
