@@ -176,6 +176,9 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=128, tile_k=32, stages=3, mma_m_axis=2),
           tc(tile_n=128, tile_k=64, stages=2, mma_m_axis=2),
           tc(tile_n=256, tile_k=32, stages=5, k_order=1, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=4, k_order=1, mma_m_axis=1)]),
+        (conv(32, 256, 28, 256, 3, 1), "tensor",
+         [tc(tile_n=256, tile_k=32, stages=5, k_order=1, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=4, k_order=1, mma_m_axis=1),
+          tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1)]),
         (conv(32, 256, 56, 64, 1, 0), "hbm",
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=2),
           tc(tile_n=256, tile_k=32, stages=4, k_order=1, mma_m_axis=1), tc(tile_n=128, tile_k=32, stages=4, k_order=1, mma_m_axis=1)]),

@@ -121,7 +121,8 @@ typedef struct tt_schedule_record {
                               channels, tap by tap inside a block: the filters are re-packed into that order by a small
                               kernel before each run, the input rows are transposed once per block into a pixel-major
                               slab, and every tap's operand tile is a shifted view of that slab -- no expansion.
-                              Stride-1 convolutions with 16-byte image rows, filters on the 128 rows, split_k = 1. */
+                              Stride-1 convolutions with 16-byte image rows, filters on the 128 rows, split_k = 1;
+                              tile_k = 32 * (taps per pipeline stage), the tap count a divisor of r*s, at most 128. */
 } tt_schedule_record;
 
 typedef struct tt_tensors {

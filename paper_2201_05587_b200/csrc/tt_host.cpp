@@ -103,17 +103,21 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     const long long Nl = (long long)w->P * wp;            // padded-linear output pixels
     if (Nl > 0x7fffffffLL) return TT_ERR_RESOURCE;
     const int N = (int)Nl, K = CB * RS * 32;
-    // fixed by the mode: filters on the 128 rows, 32-wide reduction tiles, no split-K, one accumulator
-    if (strict && (rec->mma_m_axis == 2 || rec->tile_k != 32 || rec->split_k != 1)) return TT_ERR_INVALID_SCHEDULE;
-    L.mma_m_axis = 1; L.tile_m = kHwTileM; L.tile_k = 32; L.split_k = 1; L.acc_split = 1; L.slab_tiles = 0; L.k_order = 1;
+    // fixed by the mode: filters on the 128 rows, no split-K, one accumulator; a reduction tile is `tps` taps of one
+    // 32-channel block (tile_k = 32 * tps, tps a divisor of the tap count, tile_k <= 128)
+    int tps = 1;
+    for (int d = 1; d <= 4; ++d) if (RS % d == 0 && 32 * d <= rec->tile_k) tps = d;
+    const int tk = 32 * tps;
+    if (strict && (rec->mma_m_axis == 2 || rec->tile_k != tk || rec->split_k != 1)) return TT_ERR_INVALID_SCHEDULE;
+    L.mma_m_axis = 1; L.tile_m = kHwTileM; L.tile_k = tk; L.split_k = 1; L.acc_split = 1; L.slab_tiles = 0; L.k_order = 1;
     if (rec->tile_m != kHwTileM) changed |= TT_CHG_TILE_M;
-    if (rec->tile_k != 32) changed |= TT_CHG_TILE_K;
+    if (rec->tile_k != tk) changed |= TT_CHG_TILE_K;
     if (rec->split_k != 1) changed |= TT_CHG_SPLIT_K;
     int tn = std::min(256, std::max(16, round_up(rec->tile_n, 16)));
     tn = std::min(tn, round_up(N, 16));
     if (tn != rec->tile_n) changed |= TT_CHG_TILE_N;
     L.tile_n = tn;
-    const int k_tiles = CB * RS;
+    const int k_tiles = CB * RS / tps;
     int st = std::min(std::min(kMaxStages, rec->stages), k_tiles);
     if (st != rec->stages) changed |= TT_CHG_STAGES;
     if (strict && (changed & ~TT_CHG_TILE_M)) return TT_ERR_INVALID_SCHEDULE;
@@ -122,7 +126,7 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     const int out_rows = std::min(w->P, (tn + wp - 2) / wp + 1);
     const int in_rows = out_rows - 1 + s.r;
     if (in_rows > 256) return TT_ERR_RESOURCE;
-    const unsigned a_stage = kHwTileM * 128;
+    const unsigned a_stage = (unsigned)tps * kHwTileM * 128;
     const long long s_buf = (((long long)32 * in_rows * wp) * 4 + 127) / 128 * 128;
     // furthest row a tile's views can touch (all tile_n rows are read, also those of pixels past the image)
     const long long pm_rows = (long long)((tn + wp - 2) / wp + s.r) * wp + s.s + gap + 8;
@@ -156,10 +160,10 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     GemmArgs& g = plan->g;
     g = GemmArgs{};
     g.M = M; g.N = N; g.K = K; g.batch = B;
-    g.tile_n = tn; g.tile_k = 32; g.stages = st;
+    g.tile_n = tn; g.tile_k = tk; g.stages = st;
     g.k_tiles = k_tiles; g.k_tiles_per_split = k_tiles; g.split_k = 1;
     g.tiles_m = tiles_m; g.tiles_n = tiles_n; g.raster = L.raster;
-    g.atom_k = 32; g.n_atoms = 1; g.row_bytes = 128; g.swz_mask = 7;
+    g.atom_k = 32; g.n_atoms = tps; g.row_bytes = 128; g.swz_mask = 7;
     g.a_stage_bytes = a_stage; g.b_stage_bytes = 0; g.tx_bytes = a_stage;
     g.tmem_cols = (unsigned)I.tmem_cols; g.n_acc = 1; g.cluster = 0;
     g.idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(tn >> 3) << 17) | ((unsigned)(kHwTileM >> 4) << 24);
@@ -172,7 +176,7 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     g.sh = 1; g.sw = 1; g.ph = s.pad_h; g.pw = s.pad_w;
     g.vec_store = (w->Q % 4 == 0 && ((long long)w->P * w->Q) % 4 == 0) ? 1 : 0;   // a lane's four columns: one aligned 16-byte store
     g.tap_major = 1;
-    g.slab_tma = 1; g.slab_tiles = RS; g.slab_nbuf = 1; g.pm_nbuf = nbuf;
+    g.slab_tma = 1; g.slab_tiles = RS / tps; g.slab_nbuf = 1; g.pm_nbuf = nbuf;
     g.slab_off = (unsigned)pipe; g.slab_buf_bytes = (unsigned)s_buf;
     g.slab_wp = wp; g.slab_gap = gap; g.slab_chpitch = in_rows * wp; g.slab_in_rows = in_rows; g.slab_rstep = 1;
     g.slab_box_ch = std::min(32, s.c);                   // (fewer than 32 channels: the rest of the staging buffer stays zero)

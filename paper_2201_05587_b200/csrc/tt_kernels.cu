@@ -929,15 +929,23 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (lane == 0 && it == 27) TT_STAMP(11);
                     tc_fence_after();
                     if (leader) {
-                        const uint32_t row = (uint32_t)(lin0 + fr * g.slab_wp + fs);
-                        const uint32_t b_lo = d_lo + (((pm0 + (uint32_t)(chunk & 1) * g.pm_buf_bytes + row * 128u) & 0x3FFFFu) >> 4);
-                        issue_steps<1, 4>(tmem_base, d_hi, a_stage, b_lo, a_atom, b_atom, g.idesc, it > 0 ? 1u : 0u);
+                        // the stage holds n_atoms taps of this channel block, one 128 x 32 filter atom each
+                        uint32_t a_lo = a_stage;
+                        int r2 = fr, s2 = fs;
+#pragma unroll 1
+                        for (int t = 0; t < g.n_atoms; ++t, a_lo += a_atom) {
+                            const uint32_t row = (uint32_t)(lin0 + r2 * g.slab_wp + s2);
+                            const uint32_t b_lo = d_lo + (((pm0 + (uint32_t)(chunk & 1) * g.pm_buf_bytes + row * 128u) & 0x3FFFFu) >> 4);
+                            issue_steps<1, 4>(tmem_base, d_hi, a_lo, b_lo, a_atom, b_atom, g.idesc, (it > 0 || t > 0) ? 1u : 0u);
+                            if (++s2 == g.S) { s2 = 0; ++r2; }
+                        }
                         mma_commit(empty_addr);                                                  // filter stage reusable
-                        if (tap == RS - 1) mma_commit(smem_u32(&pm_empty[chunk & 1]));             // slab buffer reusable
+                        if (tap + g.n_atoms == RS) mma_commit(smem_u32(&pm_empty[chunk & 1]));      // slab buffer reusable
                     }
                     __syncwarp();
-                    if (++fs == g.S) { fs = 0; ++fr; }
-                    if (++tap == RS) { tap = 0; fr = 0; fs = 0; ++chunk; }
+                    for (int t = 0; t < g.n_atoms; ++t) if (++fs == g.S) { fs = 0; ++fr; }
+                    tap += g.n_atoms;
+                    if (tap == RS) { tap = 0; fr = 0; fs = 0; ++chunk; }
                     a_stage += stage_step; full_addr += 8u; empty_addr += 8u;
                     if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; a_stage = a_lo0; full_addr = full0; empty_addr = empty0; }
                 }

@@ -56,6 +56,7 @@ GEMM_RECORDS = [
     tc(tile_n=128, tile_k=32, stages=3, k_order=1, mma_m_axis=1),
     tc(tile_n=256, tile_k=64, stages=2, k_order=1, split_k=2, mma_m_axis=2),
     tc(tile_n=48, tile_k=32, stages=1, k_order=1, raster=1, mma_m_axis=1),
+    tc(tile_n=64, tile_k=96, stages=2, k_order=1, mma_m_axis=1),            # three taps per pipeline stage where 3 divides r*s
     # several accumulators in tensor memory, reduction steps dealt round-robin, summed on read-out
     tc(tile_n=32, tile_k=32, stages=4, acc_split=4, mma_m_axis=1),
     tc(tile_n=48, tile_k=16, stages=3, acc_split=8, split_k=2, mma_m_axis=2),
