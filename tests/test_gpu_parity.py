@@ -409,3 +409,46 @@ def test_batched_kernels_of_the_saturating_size_points():
     sm = W.Spec(B.TT_OP_SOFTMAX, B.softmax_shapes(12 * 8, 128, 128, 0.125), 1, "softmax_96x128x128", "bert")
     a = W.make_inputs(sm, 83)
     run_spec(sm, B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=16, block_y=4, vec_width=4), a, util.oracle_ref(sm, a))
+
+
+def _random_records(family, n, seed):
+    """Seeded draws from the record space the tuner walks (and a little beyond it): any legal record, however ill
+    suited to the shape, must still compute the same kernel."""
+    import random
+    rng = random.Random(seed)
+    recs = []
+    for _ in range(n):
+        if family == B.TT_FAMILY_GEMM_TC:
+            recs.append(tc(tile_n=rng.choice([16, 32, 48, 64, 96, 128, 160, 192, 256]), tile_k=rng.choice([8, 16, 32, 64, 96, 128]),
+                           stages=rng.choice([1, 2, 3, 4, 6, 8]), split_k=rng.choice([1, 1, 2, 3, 4, 5, 8, 9, 16]),
+                           raster=rng.choice([0, 1]), mma_m_axis=rng.choice([0, 1, 2]), slab_tiles=rng.choice([0, 0, 1, 2, 5]),
+                           acc_split=rng.choice([1, 1, 2, 4, 8]), k_order=rng.choice([0, 0, 1])))
+        else:
+            recs.append(B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=rng.choice([1, 2, 4, 8, 16, 32]), block_y=rng.choice([1, 2, 4, 7, 8, 14, 28]),
+                                      block_x=rng.choice([4, 8, 16, 28, 32, 56]), items_per_thread=rng.choice([1, 2, 4, 8]),
+                                      vec_width=rng.choice([1, 2, 4]), threads=rng.choice([32, 64, 128, 256, 512]),
+                                      unroll=rng.choice([0, 1, 2, 4])))
+    return recs
+
+
+@pytest.mark.parametrize("spec,n", [
+    (W._conv(48, 20, 80, 3, 1, 1, name="rand_conv3x3"), 40),
+    (W._conv(40, 14, 72, 3, 2, 1, act=B.TT_ACT_RELU6, name="rand_conv3x3s2"), 25),
+    (W._dense(70, 300, 200, act=B.TT_ACT_GELU_ERF, name="rand_dense"), 25),
+    (W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(3, 40, 56, 48, False), 1, "rand_bmm_nn", "bert"), 15),
+    (W._dw(24, 28, 1), 25),
+], ids=lambda v: getattr(v, "name", str(v)))
+def test_a_schedule_changes_speed_never_semantics_random_records(spec, n):
+    a = W.make_inputs(spec, 90)
+    ref = util.oracle_ref(spec, a)
+    fam = B.TT_FAMILY_DW_SIMT if spec.op == B.TT_OP_DWCONV2D else B.TT_FAMILY_GEMM_TC
+    probe = spec.workload()
+    ran = 0
+    for rec in _random_records(fam, n, seed=sum(map(ord, spec.name))):
+        st, _ = probe.check(rec)
+        assert st in (B.TT_OK, B.TT_ERR_RESOURCE), (rec.short(), st)
+        if st == B.TT_OK:
+            run_spec(spec, rec, a, ref)
+            ran += 1
+    probe.close()
+    assert ran >= n * 2 // 3
