@@ -13,6 +13,7 @@ namespace tt {
 cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, const void* tmap_x,
                         cudaStream_t st);
 cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st);
+cudaError_t launch_dw_tma(const tt_apply_info& I, const DwArgs& dw, const void* tmap_x, cudaStream_t st);
 cudaError_t launch_row(const tt_apply_info& I, const RowArgs& row, cudaStream_t st);
 cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits);
 cudaError_t launch_repack(const float* w, float* out, int kout, int C, int RS, int CB, cudaStream_t st);
@@ -78,6 +79,21 @@ tt_status encode_image(void* out, const float* base, int W, int H, int C, int N,
     cuuint32_t box[4] = {(cuuint32_t)box_w, (cuuint32_t)box_h, (cuuint32_t)box_c, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = fn(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(base), dims,
+                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? TT_OK : TT_ERR_CUDA;
+}
+
+// Depthwise input as a 3-D tensor (W, H, planes = N * C), box = [box_w, in_h, tile_c], no swizzle.
+tt_status encode_planes(void* out, const float* base, int W, int H, long long planes, int box_w, int box_h, int box_c) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return TT_ERR_CUDA;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0) return TT_ERR_INVALID_ARG;
+    cuuint64_t dims[3] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)planes};
+    cuuint64_t strides[2] = {(cuuint64_t)W * 4, (cuuint64_t)W * H * 4};
+    cuuint32_t box[3] = {(cuuint32_t)box_w, (cuuint32_t)box_h, (cuuint32_t)box_c};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims,
                     strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? TT_OK : TT_ERR_CUDA;
@@ -222,6 +238,23 @@ tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
         d.y = static_cast<float*>(t->y);
         if ((reinterpret_cast<uintptr_t>(t->y) & 15u) != 0) d.vec = 1;
         if ((reinterpret_cast<uintptr_t>(t->x) & 15u) != 0) d.vec_in = 0;
+        if (d.tma_stages > 0) {
+            // the image's tensor map, cached per input pointer like the contraction's maps
+            const TmapPair* maps = nullptr;
+            for (const TmapPair& m : w->tmaps) if (m.a_ptr == t->x) { maps = &m; break; }
+            if (!maps) {
+                TmapPair m;
+                std::memset(&m, 0, sizeof m);
+                m.a_ptr = t->x;
+                tt_status s = encode_planes(m.x, d.x, d.W, d.H, (long long)d.N * d.C, d.box_w, d.in_h, d.tile_c);
+                if (s != TT_OK) return s;
+                if (w->tmaps.size() >= 4096) w->tmaps.clear();
+                w->tmaps.push_back(m);
+                maps = &w->tmaps.back();
+            }
+            d.status = w->status_word;
+            e = launch_dw_tma(p.info, d, maps->x, st);
+        } else
         e = launch_dw(p.info, d, st);
     } else {
         RowArgs r = p.row;

@@ -473,11 +473,47 @@ static tt_status legalise_dw(const tt_workload* w, const tt_schedule_record* rec
     d.tiles_w = (w->Q + d.tile_w - 1) / d.tile_w;
     d.window_rows = window_rows;
     d.vec_in = (s.w % 4) == 0;
-    const long long smem = window_rows ? 0 : (long long)d.tile_c * ((long long)d.in_h * d.in_w + d.R * d.S + 1) * 4;
+    long long smem = window_rows ? 0 : (long long)d.tile_c * ((long long)d.in_h * d.in_w + d.R * d.S + 1) * 4;
     tt_apply_info& I = plan->info;
     I = tt_apply_info{};
     I.legal = L; I.changed = changed;
-    const long long gx = (long long)d.tiles_w * d.tiles_h * d.tiles_c;
+    long long gx = (long long)d.tiles_w * d.tiles_h * d.tiles_c;
+    // raster = 1 (with a window-kernel filter and 16-byte image rows): the tiles' input boxes are staged by TMA in
+    // `stages` buffers, next to the filters and biases of their planes, and CTAs walk the tiles persistently
+    L.raster = 0;
+    if (rec->raster < 0 || rec->raster > 1) return TT_ERR_INVALID_SCHEDULE;
+    if (rec->raster == 1 && window_rows > 0 && (s.w % 4) == 0) {
+        const int st = d.sh, pad = d.pw;
+        const int ncol = (items - 1) * st + d.R, nld = (4 - pad + ncol + 3) / 4;      // 16-byte loads per window row
+        const int box_w = (d.tile_w - items) * st + 4 * nld;
+        // strips are window_rows tall: the box covers the rows of the last, possibly partial, strip too
+        const int in_h_box = (round_up(d.tile_h, window_rows) - 1) * d.sh + d.R;
+        const long long planes = (long long)s.n * s.c;
+        const long long box = (((long long)d.tile_c * in_h_box * box_w * 4) + 127) / 128 * 128;
+        const long long wstage = (((long long)d.tile_c * round_up(d.R * d.S + 1, 4) * 4) + 127) / 128 * 128;
+        const long long stage = box + wstage;
+        int stg = std::min(4, std::max(2, rec->stages));
+        while (stg > 2 && stg * stage + 128 > kDynSmemLimit) --stg;
+        if (box_w <= 256 && in_h_box <= 256 && d.tile_c <= 256 && stg * stage + 128 <= kDynSmemLimit && planes <= 0x7fffffffLL) {
+            d.in_h = in_h_box;
+            if (stg != rec->stages) { if (strict) return TT_ERR_INVALID_SCHEDULE; I.changed |= TT_CHG_STAGES; }
+            L.raster = 1; L.stages = stg;
+            d.tma_stages = stg; d.box_w = box_w; d.stage_bytes = (int)box; d.wstage_bytes = (int)wstage;
+            d.tiles_p = (int)((planes + d.tile_c - 1) / d.tile_c);
+            const long long total = (long long)d.tiles_p * d.tiles_h * d.tiles_w;
+            if (total > 0x7fffffffLL) return TT_ERR_RESOURCE;
+            d.total_tiles = (int)total;
+            smem = stg * stage + 128;
+            const long long per_sm = std::max<long long>(1, std::min<long long>(8, (228 * 1024) / (smem + 1024)));   // the launcher lowers it to what registers allow
+            gx = std::min<long long>(total, 148 * per_sm);
+            I.legal = L;
+            I.grid_x = (int)gx; I.grid_y = 1; I.grid_z = 1;
+            I.threads = th; I.smem_bytes = (int)smem; I.launches = 1;
+            return TT_OK;
+        }
+    }
+    if (rec->raster != 0) { if (strict) return TT_ERR_INVALID_SCHEDULE; I.changed |= TT_CHG_BLOCK; }
+    I.legal = L;
     I.grid_x = (int)std::min<long long>(gx, 0x7fffffff); I.grid_y = s.n; I.grid_z = 1;
     I.threads = th; I.smem_bytes = (int)std::min<long long>(smem, 0x7fffffff);
     I.launches = 1;

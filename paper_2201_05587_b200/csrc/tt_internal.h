@@ -78,6 +78,12 @@ struct DwArgs {
     int tiles_c, tiles_h, tiles_w;
     int window_rows;   // > 0: register-window kernel with this many output rows per thread; 0: staged kernel
     int vec_in;        // input rows start on 16-byte boundaries (W % 4 == 0 and x aligned)
+    // TMA-staged persistent kernel (record raster = 1): tiles of tile_c planes x tile_h x tile_w outputs, their input
+    // boxes [tile_c][in_h][box_w] land in `stages` shared-memory buffers by TMA (zero fill = padding)
+    int tma_stages;    // > 0 selects it
+    int box_w, stage_bytes, tiles_p, total_tiles;   // box width in floats (multiple of 4), bytes per buffer (multiple of 128)
+    int wstage_bytes;  // bytes per filter-and-bias buffer (one per box buffer, multiple of 128)
+    unsigned* status;  // the workload's status word (bounded waits)
 };
 
 struct RowArgs {

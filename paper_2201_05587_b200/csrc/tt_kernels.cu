@@ -682,8 +682,11 @@ __device__ __forceinline__ void epilogue_block(float (&v)[32], const EpiArgs& e,
 // ------------------------------------------------------------------------------------------------------------
 // GEMM_TC kernel.  grid = (tiles_m * tiles_n, split_k, batch), block = 320 threads:
 // warp 0 TMA producer, warp 1 MMA issuer + tensor-memory owner, warps 2-9 gather producers, then epilogue.
+// Two builds: MIN_CTAS = 1 (all registers), and MIN_CTAS = 2 (registers capped so that two CTAs share an SM when a
+// record's shared memory and tensor memory allow it: one CTA's set-up and read-out then overlap the other's main loop).
 // ------------------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kGemmThreads, 1)
+template <int MIN_CTAS>
+__global__ void __launch_bounds__(kGemmThreads, MIN_CTAS)
 tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                   const __grid_constant__ CUtensorMap tmap_x, const GemmArgs g) {
     extern __shared__ uint8_t smem_raw[];
@@ -1654,6 +1657,217 @@ __global__ void __launch_bounds__(256, WIDTH == 4 ? 6 : 4) tt_dwconv_window_kern
 }
 
 // ------------------------------------------------------------------------------------------------------------
+// DW_SIMT, TMA-staged persistent form (3x3 and 5x5 "same" filters, stride 1 or 2, image rows of 16-byte multiples).
+// The image is one 3-D tensor (W, H, planes = N * C).  A tile is tile_c consecutive planes x tile_h x tile_w
+// outputs; its input box [tile_c][in_h][box_w] starts 4 columns left of the tile (a 16-byte aligned coordinate) and
+// PAD rows above it, and the TMA zero fill supplies the padding, so the compute loop has no bounds test on inputs.
+// CTAs walk the tiles persistently with `stages` boxes in flight: no thread waits on a global load, which is what
+// limits the register-window kernel.  Threads work on ROWS x WIDTH strips exactly as there, reading the window rows
+// with aligned 16-byte shared-memory loads.  Same FMAs in the same order: bit-identical outputs.
+// The instruction stream per output is what bounds this kernel next to the memory system, so everything that does
+// not depend on the plane is hoisted: a thread keeps its strip position for the whole kernel, tile coordinates
+// advance by additions, and the filters and biases of a tile's planes are staged in shared memory (one buffer per
+// box buffer, [tile_c][WP] floats: filter, bias, padding) when the tile's box is requested.
+// ------------------------------------------------------------------------------------------------------------
+template <int R, int STRIDE, int ROWS, int WIDTH>
+__global__ void __launch_bounds__(256) tt_dwconv_tma_kernel(const __grid_constant__ CUtensorMap tmap_x, const DwArgs d) {
+    constexpr int NCOL = (WIDTH - 1) * STRIDE + R;
+    constexpr int IN_ROWS = (ROWS - 1) * STRIDE + R;
+    constexpr int PAD = R / 2;
+    constexpr int FIRST = 4 - PAD;                        // window slot 0 sits this many floats right of the strip's aligned base
+    constexpr int NLD = (FIRST + NCOL + 3) / 4;           // aligned 16-byte loads per window row
+    constexpr int WP = (R * R + 1 + 3) / 4 * 4;           // floats per plane in a weight buffer
+    extern __shared__ uint8_t dw_raw[];
+    __shared__ uint64_t full_bar[4];
+    __shared__ int abort_flag;
+    const uint32_t base = (smem_u32(dw_raw) + 127u) & ~127u;
+    const uint32_t wbase = base + (uint32_t)d.tma_stages * (uint32_t)d.stage_bytes;
+    volatile int* abortp = &abort_flag;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < d.tma_stages; ++s) mbar_init(smem_u32(&full_bar[s]), 1u);
+        abort_flag = 0;
+        fence_mbar_init();
+        fence_proxy_async_shared();
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
+    }
+    __syncthreads();
+    const int planes = d.N * d.C;
+    const int per_plane_tiles = d.tiles_h * d.tiles_w;
+    const int my_tiles = d.total_tiles > (int)blockIdx.x ? (d.total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    // Tile t = blockIdx.x + i * gridDim.x as (plane tile, row tile, column tile, first channel): decomposed once, then
+    // advanced by the decomposition of gridDim.x with carries -- no division per tile.
+    struct TilePos { int tp, th, tw, c0; };
+    int step_tp, step_th, step_tw, step_c;
+    {
+        const int gsz = (int)gridDim.x;
+        step_tp = gsz / per_plane_tiles;
+        const int rem = gsz - step_tp * per_plane_tiles;
+        step_th = rem / d.tiles_w; step_tw = rem - step_th * d.tiles_w;
+        step_c = (int)(((long long)step_tp * d.tile_c) % d.C);
+    }
+    const int tile_c_mod = d.tile_c % d.C;
+    auto first_pos = [&]() {
+        TilePos t;
+        const int b = (int)blockIdx.x;
+        t.tp = b / per_plane_tiles;
+        const int rem = b - t.tp * per_plane_tiles;
+        t.th = rem / d.tiles_w; t.tw = rem - t.th * d.tiles_w;
+        t.c0 = (int)(((long long)t.tp * d.tile_c) % d.C);
+        return t;
+    };
+    auto advance = [&](TilePos& t) {
+        t.tw += step_tw; t.th += step_th; t.tp += step_tp; t.c0 += step_c;
+        if (t.tw >= d.tiles_w) { t.tw -= d.tiles_w; ++t.th; }
+        if (t.th >= d.tiles_h) { t.th -= d.tiles_h; ++t.tp; t.c0 += tile_c_mod; }
+        while (t.c0 >= d.C) t.c0 -= d.C;
+    };
+    auto issue = [&](const TilePos& t, int s) {           // thread 0: request the input box of a tile into buffer s
+        const uint32_t bar = smem_u32(&full_bar[s]);
+        mbar_expect_tx(bar, (uint32_t)(d.tile_c * d.in_h * d.box_w * 4));
+        tma_load_3d(base + (uint32_t)s * (uint32_t)d.stage_bytes, &tmap_x, bar, t.tw * d.tile_w * STRIDE - 4,
+                    t.th * d.tile_h * STRIDE - PAD, t.tp * d.tile_c);
+    };
+    auto stage_weights = [&](const TilePos& t, int s) {   // all threads: the filters and biases of the tile's planes
+        const uint32_t dst = wbase + (uint32_t)s * (uint32_t)d.wstage_bytes;
+        const int pl0 = t.tp * d.tile_c;
+        for (int idx = (int)threadIdx.x; idx < d.tile_c * WP; idx += (int)blockDim.x) {
+            const int cl = idx / WP, k = idx - cl * WP;
+            int c = t.c0 + cl;                            // tile_c <= C: one subtraction wraps it
+            if (c >= d.C) c -= d.C;
+            float v = 0.f;
+            if (pl0 + cl < planes) {
+                if (k < R * R) v = __ldg(d.w + c * (R * R) + k);
+                else if (k == R * R && d.bias) v = __ldg(d.bias + c);
+            }
+            st_shared_f32(dst + 4u * (uint32_t)idx, v);
+        }
+    };
+    TilePos cur = first_pos(), nxt = cur;
+    {
+        const int pre = min(my_tiles, d.tma_stages);
+        for (int i = 0; i < pre; ++i) {
+            if (threadIdx.x == 0) issue(nxt, i);
+            stage_weights(nxt, i);
+            advance(nxt);
+        }
+    }
+    __syncthreads();                                      // the first weight buffers are in place
+    // a thread's strip position inside a plane is fixed for the whole kernel when a plane has at most blockDim strips
+    // (the thread then walks planes cl_f, cl_f + cpp, ...); otherwise it also walks strips
+    const int groups_w = d.tile_w / WIDTH;
+    const int groups_h = (d.tile_h + ROWS - 1) / ROWS;
+    const int spp = groups_h * groups_w;                  // strips per plane
+    const bool fixed_pos = spp <= (int)blockDim.x;
+    const int cpp = fixed_pos ? (int)blockDim.x / spp : 1;                  // planes per pass
+    const int cl_f = fixed_pos ? (int)threadIdx.x / spp : 0;
+    const int s_f = (int)threadIdx.x - cl_f * spp;
+    const int s_step = fixed_pos ? spp : (int)blockDim.x;                    // fixed: the strip loop runs once
+    const bool active = cl_f < cpp;
+    const int gh_f = s_f / groups_w, gwi_f = s_f - gh_f * groups_w;
+    const uint32_t plane_bytes = 4u * (uint32_t)(d.in_h * d.box_w);
+    const long long plane_out = (long long)d.P * d.Q;
+    const bool clamp = d.act == TT_ACT_RELU || d.act == TT_ACT_RELU6, gelu = d.act == TT_ACT_GELU_ERF;
+    const float hi = d.act == TT_ACT_RELU6 ? 6.f : INFINITY;
+    int s = 0;
+    uint32_t ph = 0;
+    for (int i = 0; i < my_tiles; ++i) {
+        // every thread waits for the box itself (all take the same decision: the same barrier and phase)
+        if (!mbar_wait(smem_u32(&full_bar[s]), ph, abortp, d.status, 9u)) break;
+        const int pl0 = cur.tp * d.tile_c, p0 = cur.th * d.tile_h, q0 = cur.tw * d.tile_w;
+        const int ncl = min(d.tile_c, planes - pl0);
+        const uint32_t stage = base + (uint32_t)s * (uint32_t)d.stage_bytes;
+        const uint32_t wst = wbase + (uint32_t)s * (uint32_t)d.wstage_bytes;
+        for (int sidx = s_f; active && sidx < spp; sidx += s_step) {
+            int gh = gh_f, gwi = gwi_f;
+            if (sidx != s_f) { gh = sidx / groups_w; gwi = sidx - gh * groups_w; }
+            const int p = p0 + gh * ROWS, q = q0 + gwi * WIDTH;
+            if (p >= d.P || q >= d.Q || gh * ROWS >= d.tile_h) continue;
+            const int nrows = min(ROWS, min(d.P - p, d.tile_h - gh * ROWS));
+            const bool whole = q + WIDTH <= d.Q;
+            // the strip's window rows: box row gh*ROWS*STRIDE + ri, from the aligned float WIDTH*gwi*STRIDE on
+            const uint32_t soff = stage + 4u * (uint32_t)((gh * ROWS * STRIDE) * d.box_w + WIDTH * gwi * STRIDE);
+            float* __restrict__ y0 = d.y + ((long long)pl0 * d.P + p) * (long long)d.Q + q;
+#pragma unroll 1
+            for (int cl = cl_f; cl < ncl; cl += cpp) {
+                float wv[WP];
+#pragma unroll
+                for (int k = 0; k < WP / 4; ++k) {
+                    const float4 f = ld_shared_v4f(wst + 4u * (uint32_t)(cl * WP + 4 * k));
+                    wv[4 * k] = f.x; wv[4 * k + 1] = f.y; wv[4 * k + 2] = f.z; wv[4 * k + 3] = f.w;
+                }
+                float acc[ROWS][WIDTH];
+#pragma unroll
+                for (int ro = 0; ro < ROWS; ++ro)
+#pragma unroll
+                    for (int j = 0; j < WIDTH; ++j) acc[ro][j] = wv[R * R];
+                const uint32_t row0 = soff + (uint32_t)cl * plane_bytes;
+#pragma unroll
+                for (int ri = 0; ri < IN_ROWS; ++ri) {
+                    float u[4 * NLD];
+#pragma unroll
+                    for (int k = 0; k < NLD; ++k) {
+                        const float4 f = ld_shared_v4f(row0 + 4u * (uint32_t)(ri * d.box_w + 4 * k));
+                        u[4 * k] = f.x; u[4 * k + 1] = f.y; u[4 * k + 2] = f.z; u[4 * k + 3] = f.w;
+                    }
+#pragma unroll
+                    for (int ro = 0; ro < ROWS; ++ro) {
+                        const int fr = ri - ro * STRIDE;          // compile-time after unrolling
+                        if (fr >= 0 && fr < R) {
+#pragma unroll
+                            for (int fs = 0; fs < R; ++fs)
+#pragma unroll
+                                for (int j = 0; j < WIDTH; ++j) acc[ro][j] = fmaf(u[FIRST + j * STRIDE + fs], wv[fr * R + fs], acc[ro][j]);
+                        }
+                    }
+                }
+                float* __restrict__ yc = y0 + (long long)cl * plane_out;
+#pragma unroll
+                for (int ro = 0; ro < ROWS; ++ro) {
+                    if (ro >= nrows) break;
+                    if (clamp) {
+#pragma unroll
+                        for (int j = 0; j < WIDTH; ++j) acc[ro][j] = fminf(fmaxf(acc[ro][j], 0.f), hi);
+                    } else if (gelu) {
+#pragma unroll
+                        for (int j = 0; j < WIDTH; ++j) acc[ro][j] = gelu_erf(acc[ro][j]);
+                    }
+                    float* yo = yc + (long long)ro * d.Q;
+                    if (whole && d.vec == 4) {
+#pragma unroll
+                        for (int j = 0; j < WIDTH; j += 4)
+                            *reinterpret_cast<float4*>(yo + j) = make_float4(acc[ro][j], acc[ro][j + 1], acc[ro][j + 2], acc[ro][j + 3]);
+                    } else if (whole && d.vec == 2) {
+#pragma unroll
+                        for (int j = 0; j < WIDTH; j += 2) *reinterpret_cast<float2*>(yo + j) = make_float2(acc[ro][j], acc[ro][j + 1]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < WIDTH; ++j)
+                            if (q + j < d.Q) yo[j] = acc[ro][j];
+                    }
+                }
+            }
+        }
+        __syncthreads();                                  // everyone is done with this box and its weight buffer
+        if (i + d.tma_stages < my_tiles) {
+            if (threadIdx.x == 0) issue(nxt, s);
+            stage_weights(nxt, s);                        // read again only after a later barrier (stages >= 2)
+            advance(nxt);
+        }
+        advance(cur);
+        if (++s == d.tma_stages) { s = 0; ph ^= 1u; }
+    }
+    // after a tripped wait: let the boxes still in flight land before the shared memory is given back (bounded)
+    if (threadIdx.x == 0 && *abortp) {
+        for (int b = 0; b < d.tma_stages; ++b) {
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(smem_u32(&full_bar[b]), 0u) && !mbar_try_wait(smem_u32(&full_bar[b]), 1u)) {
+                if (global_timer_ns() - t0 > 2000000ull) break;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------
 // ROW_SIMT: softmax(scale * x) per row; `lanes_per_row` threads of one warp share a row.
 // ------------------------------------------------------------------------------------------------------------
 __global__ void tt_softmax_kernel(const RowArgs a) {
@@ -1749,13 +1963,21 @@ __global__ void tt_repack_filters_kernel(const float* __restrict__ w, float* __r
 // ------------------------------------------------------------------------------------------------------------
 // Launchers (called from tt_device.cu)
 // ------------------------------------------------------------------------------------------------------------
+// Two CTAs fit one SM when each takes at most half of its shared memory (228 KB, of which 1 KB per CTA is the
+// system's, plus the kernel's static part) and half of its 512 tensor-memory columns.
+static bool gemm_two_per_sm(int smem_bytes, int tmem_cols) { return smem_bytes <= 112 * 1024 && tmem_cols <= 256; }
+
 cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, const void* tmap_x,
                         cudaStream_t st) {
     static int attr_set_for = -1;
     int dev = 0;
     cudaGetDevice(&dev);
     if (attr_set_for != dev) {
-        cudaError_t e = cudaFuncSetAttribute(tt_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemLimit);
+        cudaError_t e = cudaFuncSetAttribute(tt_gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemLimit);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(tt_gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemLimit);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(tt_gemm_tc_kernel<2>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_set_for = dev;
     }
@@ -1780,12 +2002,13 @@ cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* t
         ++n_attr;
     }
     cfg.attrs = attr; cfg.numAttrs = (unsigned)n_attr;
-    return cudaLaunchKernelEx(&cfg, tt_gemm_tc_kernel, ta, tb, tx, g);
+    if (gemm_two_per_sm(I.smem_bytes, g.tmem_cols)) return cudaLaunchKernelEx(&cfg, tt_gemm_tc_kernel<2>, ta, tb, tx, g);
+    return cudaLaunchKernelEx(&cfg, tt_gemm_tc_kernel<1>, ta, tb, tx, g);
 }
 
 // Can a cluster of `cluster` CTAs with this much shared memory each be resident at all?
 cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits) {
-    cudaError_t e = cudaFuncSetAttribute(tt_gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemLimit);
+    cudaError_t e = cudaFuncSetAttribute(tt_gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemLimit);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(1, (unsigned)cluster, 1); cfg.blockDim = dim3(kGemmThreads, 1, 1); cfg.dynamicSmemBytes = (size_t)smem_bytes;
@@ -1794,7 +2017,7 @@ cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits) {
     attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = (unsigned)cluster; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, tt_gemm_tc_kernel, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, tt_gemm_tc_kernel<1>, &cfg);   // the other build needs no more of anything
     if (e != cudaSuccess) return e;
     *fits = n > 0;
     return cudaSuccess;
@@ -1805,6 +2028,34 @@ cudaError_t launch_repack(const float* w, float* out, int kout, int C, int RS, i
     const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 8);
     tt_repack_filters_kernel<<<blocks, 256, 0, st>>>(w, out, kout, C, RS, CB);
     return cudaGetLastError();
+}
+
+cudaError_t launch_dw_tma(const tt_apply_info& I, const DwArgs& dw, const void* tmap_x, cudaStream_t st) {
+    CUtensorMap tx;
+    memcpy(&tx, tmap_x, sizeof tx);
+    dim3 grid(I.grid_x, 1, 1);
+    int sm_count = 148, dev_now = 0;
+    cudaGetDevice(&dev_now);
+    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev_now);
+#define TT_DWT_CASE(RR, SS, RO, WI) \
+    if (dw.R == RR && dw.sh == SS && dw.window_rows == RO && dw.items == WI) { \
+        static int attr_dev = -1; int dev = 0; cudaGetDevice(&dev); \
+        if (attr_dev != dev) { \
+            cudaError_t e = cudaFuncSetAttribute(tt_dwconv_tma_kernel<RR, SS, RO, WI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemLimit); \
+            if (e != cudaSuccess) return e; attr_dev = dev; } \
+        int occ = 0; \
+        cudaError_t eo = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, tt_dwconv_tma_kernel<RR, SS, RO, WI>, I.threads, (size_t)I.smem_bytes); \
+        if (eo != cudaSuccess) return eo; \
+        if (occ < 1) return cudaErrorLaunchOutOfResources; \
+        /* persistent CTAs: never more than are resident at once (registers may allow fewer than shared memory does) */ \
+        grid.x = (unsigned)std::min<long long>(grid.x, (long long)sm_count * occ); \
+        tt_dwconv_tma_kernel<RR, SS, RO, WI><<<grid, I.threads, I.smem_bytes, st>>>(tx, dw); return cudaGetLastError(); }
+    TT_DWT_CASE(3, 1, 1, 4) TT_DWT_CASE(3, 1, 2, 4) TT_DWT_CASE(3, 1, 4, 4) TT_DWT_CASE(3, 1, 1, 8) TT_DWT_CASE(3, 1, 2, 8)
+    TT_DWT_CASE(3, 2, 1, 4) TT_DWT_CASE(3, 2, 2, 4) TT_DWT_CASE(3, 2, 4, 4) TT_DWT_CASE(3, 2, 1, 8) TT_DWT_CASE(3, 2, 2, 8)
+    TT_DWT_CASE(5, 1, 1, 4) TT_DWT_CASE(5, 1, 2, 4) TT_DWT_CASE(5, 1, 4, 4) TT_DWT_CASE(5, 1, 1, 8) TT_DWT_CASE(5, 1, 2, 8)
+    TT_DWT_CASE(5, 2, 1, 4) TT_DWT_CASE(5, 2, 2, 4) TT_DWT_CASE(5, 2, 4, 4) TT_DWT_CASE(5, 2, 1, 8) TT_DWT_CASE(5, 2, 2, 8)
+#undef TT_DWT_CASE
+    return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st) {

@@ -196,6 +196,12 @@ def test_depthwise_parity_records(spec):
                                         (8, 5, 8, 1, 1, 32, 4), (3, 6, 112, 4, 2, 96, 2), (2, 3, 16, 8, 4, 128, 1), (5, 9, 24, 8, 1, 64, 4)):
         recs.append(B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=tcn, block_y=by, block_x=bx, items_per_thread=it,
                                   vec_width=vw, threads=th, unroll=un))
+    # raster = 1: input boxes staged by TMA, persistent CTAs (image rows of 16-byte multiples; elsewhere legalised away)
+    for tcn, by, bx, it, vw, th, un, st in ((4, 8, 32, 4, 4, 128, 2, 3), (1, 7, 16, 4, 4, 64, 4, 2), (16, 4, 8, 4, 2, 256, 1, 4),
+                                            (3, 5, 28, 4, 4, 96, 2, 2), (8, 6, 56, 8, 4, 256, 2, 2), (5, 3, 16, 8, 4, 32, 1, 3),
+                                            (32, 56, 56, 4, 4, 256, 1, 2)):
+        recs.append(B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=tcn, block_y=by, block_x=bx, items_per_thread=it, vec_width=vw,
+                                  threads=th, unroll=un, raster=1, stages=st))
     outs = [run_spec(spec, r, a, ref) for r in recs]
     for y in outs[1:]:
         np.testing.assert_array_equal(y, outs[0])       # same fp32 operations in the same order: bit-identical
@@ -427,7 +433,7 @@ def _random_records(family, n, seed):
             recs.append(B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=rng.choice([1, 2, 4, 8, 16, 32]), block_y=rng.choice([1, 2, 4, 7, 8, 14, 28]),
                                       block_x=rng.choice([4, 8, 16, 28, 32, 56]), items_per_thread=rng.choice([1, 2, 4, 8]),
                                       vec_width=rng.choice([1, 2, 4]), threads=rng.choice([32, 64, 128, 256, 512]),
-                                      unroll=rng.choice([0, 1, 2, 4])))
+                                      unroll=rng.choice([0, 1, 2, 4]), raster=rng.choice([0, 1]), stages=rng.choice([1, 2, 3, 4, 6])))
     return recs
 
 
