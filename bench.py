@@ -170,8 +170,8 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
     dwr = lambda **kw: B.make_record(B.TT_FAMILY_DW_SIMT, **kw)
     cases = [
         (W._dense(4096, 4096, 4096), "tensor",
-         [tc(tile_n=256, tile_k=32, stages=4, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=4, mma_m_axis=2),
-          tc(tile_n=256, tile_k=64, stages=2, mma_m_axis=1)]),
+         [tc(tile_n=256, tile_k=32, stages=4, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1),
+          tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=2)]),
         (conv(32, 128, 28, 128, 3, 1), "tensor",
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=128, tile_k=32, stages=3, mma_m_axis=2),
           tc(tile_n=128, tile_k=64, stages=2, mma_m_axis=2),
@@ -181,16 +181,20 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
           tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1)]),
         (conv(32, 256, 56, 64, 1, 0), "hbm",
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=2),
-          tc(tile_n=256, tile_k=32, stages=4, k_order=1, mma_m_axis=1), tc(tile_n=128, tile_k=32, stages=4, k_order=1, mma_m_axis=1)]),
+          tc(tile_n=64, tile_k=32, stages=2, mma_m_axis=2, slab_tiles=1), tc(tile_n=64, tile_k=32, stages=3, mma_m_axis=2, slab_tiles=1)]),
         (dw(64, 144, 56, 1), "hbm",
          [dwr(tile_m=4, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=2),
           dwr(tile_m=16, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=128, unroll=2),
           dwr(tile_m=4, block_y=16, block_x=56, items_per_thread=4, vec_width=4, threads=128, unroll=4),
-          dwr(tile_m=8, block_y=56, block_x=56, items_per_thread=8, vec_width=4, threads=128, unroll=2)]),
+          dwr(tile_m=8, block_y=56, block_x=56, items_per_thread=8, vec_width=4, threads=128, unroll=2),
+          dwr(tile_m=8, block_y=14, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=4, raster=1, stages=2),
+          dwr(tile_m=16, block_y=8, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=4, raster=1, stages=2)]),
         (dw(32, 96, 112, 2), "hbm",
          [dwr(tile_m=4, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=2),
           dwr(tile_m=4, block_y=4, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=1),
-          dwr(tile_m=1, block_y=8, block_x=56, items_per_thread=4, vec_width=4, threads=64, unroll=2)]),
+          dwr(tile_m=1, block_y=8, block_x=56, items_per_thread=4, vec_width=4, threads=64, unroll=2),
+          dwr(tile_m=4, block_y=8, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=2, raster=1, stages=2),
+          dwr(tile_m=8, block_y=4, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=2, raster=1, stages=2)]),
         (W.Spec(B.TT_OP_SOFTMAX, B.softmax_shapes(12 * 256, 128, 128, 0.125), 1, "softmax_3072x128x128", "bert"), "hbm",
          [B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=8, block_y=8, vec_width=4),
           B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=32, block_y=4, vec_width=4)]),

@@ -97,7 +97,9 @@ typedef struct tt_shapes {
  * DW_SIMT uses tile_m (channels per CTA), block_y x block_x (output rows x columns per CTA tile),
  *         items_per_thread (consecutive outputs along the width per thread), vec_width, threads, and unroll:
  *         0 = shared-memory staged kernel; 1, 2, 4 = register-window kernel with that many output rows per thread
- *         (3x3 and 5x5 filters with "same" padding, stride 1 or 2; strips of 4 columns).
+ *         (3x3 and 5x5 filters with "same" padding, stride 1 or 2; strips of 4 or 8 columns).  raster = 1 with
+ *         unroll >= 1 and image rows of 16-byte multiples: the same strips, but CTAs walk the tiles persistently and
+ *         a tile's input box and its planes' filters are staged in `stages` (2..4) shared-memory buffers by TMA.
  * ROW_SIMT uses block_x (threads cooperating on one row: 1..32, power of two), block_y (rows per CTA), vec_width.
  * origin_* say which kernel the record was tuned on (its "native" kernel, Section 3). */
 typedef struct tt_schedule_record {
@@ -267,6 +269,42 @@ tt_status tt_transfer_tune(tt_workload* const* model_workloads, const tt_tensors
 tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, const tt_timing_opts* o, int32_t level,
                        size_t top_k, tt_schedule_record* out_records, float* out_us, size_t* n_out,
                        int32_t* n_tried);
+
+/* Refining a transferred record (Section 7 names it as the next step: vary the parameters of schedules that were
+ * transfer-tuned from another model).  The neighbourhood of a record: every field its family uses is moved one rung
+ * down and one rung up its ladder of values (two-valued fields are toggled), one field at a time, in the order the
+ * fields are listed below; each candidate is legalised for `w`, and candidates that are invalid, that legalise back
+ * to the (legalised) start or that repeat an earlier neighbour are dropped.
+ *   GEMM_TC  tile_n {16,32,48,64,96,128,160,192,224,256}  tile_k {8,16,32,64,96,128}  stages {1..8}
+ *            split_k {1..8,12,16,24,32}  raster {0,1}  mma_m_axis {1,2}  slab_tiles {0,1,2,4,8}  acc_split {1,2,4,8}
+ *            k_order {0,1}
+ *   DW_SIMT  tile_m {1,2,4,8,16,32}  block_y {1,2,4,7,8,14,16,28,56}  block_x {8,16,28,32,56,64,112}
+ *            items_per_thread {1,2,4,8}  vec_width {1,2,4}  threads {32,...,512}  unroll {0,1,2,4}  raster {0,1}
+ *            stages {2,3,4}
+ *   ROW_SIMT block_x {1,...,32}  block_y {1,...,16}  vec_width {1,2,4}
+ * Pure host.  out[cap] receives the neighbours, *n_out their number (cap == 0: count only; more than cap:
+ * TT_ERR_RESOURCE).  At most two per field, so 18 entries always suffice. */
+tt_status tt_record_neighbours(const tt_workload* w, const tt_schedule_record* rec, tt_schedule_record* out, size_t cap,
+                               size_t* n_out);
+
+/* Time of one record in microseconds, negative when the record cannot run. */
+typedef float (*tt_time_fn)(void* user, const tt_schedule_record* rec);
+
+/* Greedy descent over that neighbourhood, pure host given the timing function: the start (legalised) is timed, then,
+ * up to max_rounds times, every neighbour of the current record that has not been timed before is timed and the
+ * fastest becomes the current record if it beats it by more than the fraction min_gain (ties keep the earlier
+ * neighbour); otherwise the search stops.  best/best_us receive the last current record and its time, start_us (may
+ * be NULL) the start's time, n_timed (may be NULL) the number of calls of time_us.  TT_ERR_INVALID_SCHEDULE when the
+ * start itself cannot run. */
+tt_status tt_refine_with(const tt_workload* w, const tt_schedule_record* start, tt_time_fn time_us, void* user,
+                         int32_t max_rounds, float min_gain, tt_schedule_record* best, float* best_us, float* start_us,
+                         int32_t* n_timed);
+
+/* The same on the device: a record's time is the median of tt_time under `o` on the tensors `t` (records that fail to
+ * apply or trip a wait count as unable to run).  On return the best record is applied to `w`. */
+tt_status tt_refine(tt_workload* w, const tt_tensors* t, void* cuda_stream, const tt_timing_opts* o,
+                    const tt_schedule_record* start, int32_t max_rounds, float min_gain, tt_schedule_record* best,
+                    float* best_us, float* start_us, int32_t* n_timed);
 
 /* (No counterpart in the paper.)  dense+bias+activation under a split-K record for callers that cannot allocate
  * device memory when they need the kernel: hosts whose memory pool already owns the whole device, loops that may

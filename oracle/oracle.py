@@ -13,11 +13,15 @@ the host-side definitions the paper fixes:
   (Section 4.3); invalid pairs carry a negative time as in Figure 4.
 * ``model_latency`` — sum of use count x chosen standalone time.
 * ``rank_pools`` — the model-selection heuristic, Equation 1 (Section 4.4).
+* ``ladder_steps`` / ``raw_neighbours`` / ``refine`` — varying the parameters of a
+  transferred schedule (Section 7, future work) as a greedy one-field-at-a-time descent.
 
 Parity pinning status: conv2d, dwconv2d, dense/batch_matmul, softmax, the
 activations, the split rules and ``select`` are pinned by closed forms, brute
 force and the paper's worked examples in ``tests/test_oracle_pins.py``;
 ``rank_pools`` by Tables 2 and 3 of the paper (all ten top-3 rankings).
+``refine`` is pinned by exhaustive search on small separable cost tables (on a
+separable convex cost a one-field descent must reach the global minimum).
 The absolute kernel times and which schedule wins on a given kernel are
 "parity unpinned": the paper's per-kernel times exist only in a figure.
 """
@@ -252,3 +256,71 @@ def rank_pools(target_share, candidate_counts):
         scores.append(s)
     order = sorted(range(len(scores)), key=lambda i: (-scores[i], i))
     return scores, order
+
+
+# ---- refining a transferred schedule (Section 7: "vary parameters from schedules transfer-tuned from another model") ----
+# The paper names the idea only; the reading taken here: each parameter has an ordered ladder of values, a step moves
+# one parameter to the next lower or next higher rung, and the search is a greedy descent over those steps.
+LADDERS = {
+    "gemm_tc": [("tile_n", [16, 32, 48, 64, 96, 128, 160, 192, 224, 256]), ("tile_k", [8, 16, 32, 64, 96, 128]),
+                ("stages", [1, 2, 3, 4, 5, 6, 7, 8]), ("split_k", [1, 2, 3, 4, 5, 6, 7, 8, 12, 16, 24, 32]),
+                ("raster", [0, 1]), ("mma_m_axis", [1, 2]), ("slab_tiles", [0, 1, 2, 4, 8]), ("acc_split", [1, 2, 4, 8]),
+                ("k_order", [0, 1])],
+    "dw_simt": [("tile_m", [1, 2, 4, 8, 16, 32]), ("block_y", [1, 2, 4, 7, 8, 14, 16, 28, 56]),
+                ("block_x", [8, 16, 28, 32, 56, 64, 112]), ("items_per_thread", [1, 2, 4, 8]), ("vec_width", [1, 2, 4]),
+                ("threads", [32, 64, 128, 256, 512]), ("unroll", [0, 1, 2, 4]), ("raster", [0, 1]), ("stages", [2, 3, 4])],
+    "row_simt": [("block_x", [1, 2, 4, 8, 16, 32]), ("block_y", [1, 2, 4, 8, 16]), ("vec_width", [1, 2, 4])],
+}
+
+
+def ladder_steps(value: int, ladder):
+    """The rungs next to `value`: the largest rung below it and the smallest above it (either may be missing;
+    `value` itself need not be a rung)."""
+    below = [r for r in ladder if r < value]
+    above = [r for r in ladder if r > value]
+    out = []
+    if below:
+        out.append(max(below))
+    if above:
+        out.append(min(above))
+    return out
+
+
+def raw_neighbours(record: dict, family: str):
+    """One-step variations of a schedule given as {parameter: value}: per parameter of the family, in ladder order,
+    the lower step then the upper step, everything else unchanged.  (Mapping a variation onto a kernel's legal
+    schedules, and dropping those that coincide, is the validity layer's job, not part of this definition.)"""
+    out = []
+    for name, ladder in LADDERS[family]:
+        for v in ladder_steps(record[name], ladder):
+            r = dict(record)
+            r[name] = v
+            out.append(r)
+    return out
+
+
+def refine(start, neighbours, time_us, max_rounds: int, min_gain: float = 0.0):
+    """Greedy descent: time the start; then, up to max_rounds times, time every neighbour of the current schedule
+    that was not timed before and move to the fastest one if it is faster than the current one by more than the
+    fraction min_gain (ties keep the earlier neighbour); stop otherwise.  `neighbours(s)` lists hashable schedules,
+    `time_us(s)` is negative for a schedule that cannot run.  Returns (best, best_us, start_us, number of timings)."""
+    cur, cur_us = start, time_us(start)
+    timed = 1
+    start_us = cur_us
+    if not cur_us >= 0:
+        raise ValueError("the start schedule cannot run")
+    seen = {start}
+    for _ in range(max_rounds):
+        pick, pick_us = None, cur_us
+        for nb in neighbours(cur):
+            if nb in seen:
+                continue
+            seen.add(nb)
+            us = time_us(nb)
+            timed += 1
+            if us >= 0 and us < pick_us:
+                pick, pick_us = nb, us
+        if pick is None or not pick_us < cur_us * (1.0 - min_gain):
+            break
+        cur, cur_us = pick, pick_us
+    return cur, cur_us, start_us, timed

@@ -53,7 +53,7 @@ class tt_schedule_record(C.Structure):
                     (f" acc{self.acc_split}" if self.acc_split > 1 else "") + (" tap" if self.k_order else "") + "]")
         if self.family == TT_FAMILY_DW_SIMT:
             return (f"dw[c{self.tile_m} {self.block_y}x{self.block_x} it{self.items_per_thread} "
-                    f"v{self.vec_width} t{self.threads} u{self.unroll}]")
+                    f"v{self.vec_width} t{self.threads} u{self.unroll}" + (f" tma st{self.stages}" if self.raster else "") + "]")
         return f"row[{self.block_x}x{self.block_y} v{self.vec_width}]"
 
 
@@ -119,6 +119,13 @@ EXPORTS = {
                                C.c_size_t, C.POINTER(tt_tune_opts), C.c_void_p, C.POINTER(tt_tune_result)]),
     "tt_grid_tune": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(tt_timing_opts), i32, C.c_size_t,
                            C.POINTER(tt_schedule_record), C.POINTER(f32), C.POINTER(C.c_size_t), C.POINTER(i32)]),
+    "tt_record_neighbours": (i32, [C.c_void_p, C.POINTER(tt_schedule_record), C.POINTER(tt_schedule_record), C.c_size_t,
+                                   C.POINTER(C.c_size_t)]),
+    "tt_refine_with": (i32, [C.c_void_p, C.POINTER(tt_schedule_record), C.c_void_p, C.c_void_p, i32, f32,
+                             C.POINTER(tt_schedule_record), C.POINTER(f32), C.POINTER(f32), C.POINTER(i32)]),
+    "tt_refine": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(tt_timing_opts),
+                        C.POINTER(tt_schedule_record), i32, f32, C.POINTER(tt_schedule_record), C.POINTER(f32),
+                        C.POINTER(f32), C.POINTER(i32)]),
     "tt_dense_static_scratch": (i32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, i32, i32, i32, i32,
                                       C.POINTER(tt_schedule_record), C.c_void_p, C.POINTER(C.c_int64)]),
 }
@@ -339,6 +346,39 @@ class Workload:
         return out, tried.value
 
 
+    def neighbours(self, rec):
+        """tt_record_neighbours: the legalised one-step neighbours of `rec` on this workload."""
+        out = (tt_schedule_record * 32)()
+        n = C.c_size_t()
+        _check(lib().tt_record_neighbours(self.handle, C.byref(rec), out, 32, C.byref(n)), f"tt_record_neighbours({self.name})")
+        res = []
+        for i in range(n.value):
+            r = tt_schedule_record()
+            C.memmove(C.byref(r), C.byref(out[i]), C.sizeof(r))
+            res.append(r)
+        return res
+
+    def refine_with(self, start, time_us, max_rounds=8, min_gain=0.0):
+        """tt_refine_with: greedy descent from `start` with a Python timing function rec -> microseconds (negative =
+        cannot run).  Returns (best record, best_us, start_us, calls of time_us)."""
+        def _cb(_user, rec_ptr):
+            return float(time_us(rec_ptr.contents))
+        cb = TIME_FN(_cb)
+        best, bus, sus, nt = tt_schedule_record(), f32(), f32(), i32()
+        _check(lib().tt_refine_with(self.handle, C.byref(start), C.cast(cb, C.c_void_p), None, max_rounds, min_gain,
+                                    C.byref(best), C.byref(bus), C.byref(sus), C.byref(nt)), f"tt_refine_with({self.name})")
+        return best, bus.value, sus.value, nt.value
+
+    def refine(self, t: tt_tensors, start, opts: tt_timing_opts | None = None, max_rounds=4, min_gain=0.02):
+        """tt_refine: the same with device times (median of tt_time); leaves the best record applied."""
+        best, bus, sus, nt = tt_schedule_record(), f32(), f32(), i32()
+        _check(lib().tt_refine(self.handle, C.byref(t), _stream(), C.byref(opts) if opts else None, C.byref(start),
+                               max_rounds, min_gain, C.byref(best), C.byref(bus), C.byref(sus), C.byref(nt)),
+               f"tt_refine({self.name})")
+        return best, bus.value, sus.value, nt.value
+
+
+TIME_FN = C.CFUNCTYPE(f32, C.c_void_p, C.POINTER(tt_schedule_record))
 TT_STATIC_SCRATCH_BYTES = 8 << 20
 
 

@@ -544,9 +544,17 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
             push(r);
         }
         if (w->op == TT_OP_CONV2D) {
+            // a slab that serves one reduction tile per staging: the smallest shared-memory footprint (two CTAs may
+            // then share an SM)
+            for (int ax : {1, 2}) for (int tn : full ? std::vector<int>{32, 64, 128, 256} : std::vector<int>{64, 128}) for (int sg : {2, 3}) {
+                tt_schedule_record r = base;
+                r.mma_m_axis = ax; r.tile_m = kHwTileM; r.tile_n = tn; r.tile_k = 32; r.stages = sg; r.split_k = 1; r.raster = 0;
+                r.slab_tiles = 1;
+                push(r);
+            }
             // the tap-major reduction order (records that ask for it on a kernel that has none are legalised back
             // to the stored order and dropped here as duplicates-to-be)
-            for (int tn : full ? std::vector<int>{32, 64, 96, 128, 192, 256} : std::vector<int>{64, 128, 256})
+            for (int tn : full ? std::vector<int>{32, 64, 96, 128, 160, 192, 224, 256} : std::vector<int>{64, 128, 224, 256})
                 for (int sg : full ? std::vector<int>{1, 2, 3, 4, 5, 6, 8} : std::vector<int>{2, 3, 5}) {
                     tt_schedule_record r = base;
                     r.mma_m_axis = 1; r.tile_m = kHwTileM; r.tile_n = tn; r.tile_k = 32; r.stages = sg; r.split_k = 1; r.raster = 0;
@@ -578,6 +586,22 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
                 if (push(r)) break;
             }
         }
+        // TMA-staged persistent kernel (raster = 1): strips of 4 or 8 columns, 1-4 rows; tiles span the image width
+        // where they can (a box then needs no columns of a neighbouring tile)
+        const std::vector<int> pcs = full ? std::vector<int>{1, 2, 4, 8, 16, 32} : std::vector<int>{2, 8, 16};
+        const std::vector<int> pys = full ? std::vector<int>{2, 4, 7, 8, 14, 16, 28, 56} : std::vector<int>{4, 8, 14};
+        const std::vector<int> pxs = full ? std::vector<int>{16, 28, 32, 56, 64, 112} : std::vector<int>{32, 56, 112};
+        for (int it : full ? std::vector<int>{4, 8} : std::vector<int>{4}) for (int ro : {2, 4}) for (int tc : pcs) for (int by : pys)
+            for (int bx : pxs) for (int sg : full ? std::vector<int>{2, 3, 4} : std::vector<int>{2, 3}) {
+                if (it == 8 && ro == 4) continue;
+                tt_schedule_record r = base;
+                r.tile_m = tc; r.block_y = by; r.block_x = bx; r.items_per_thread = it; r.threads = 256;
+                r.unroll = ro; r.raster = 1; r.stages = sg;
+                for (int vw : {4, 2, 1}) {
+                    r.vec_width = vw;
+                    if (push(r)) break;
+                }
+            }
     } else {
         for (int bx : {4, 8, 16, 32}) for (int by : {1, 2, 4, 8, 16}) for (int vw : {1, 2, 4}) {
             tt_schedule_record r = base;
@@ -619,6 +643,33 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
     *n_out = n;
     if (n > 0) return apply_impl(w, &out_records[0], TT_MODE_LEGALISE, 0, nullptr);
     return TT_ERR_INVALID_SCHEDULE;
+}
+
+namespace {
+struct RefineCtx { tt_workload* w; const tt_tensors* t; cudaStream_t st; const tt_timing_opts* o; tt_status fatal; };
+float refine_time(void* user, const tt_schedule_record* rec) {
+    RefineCtx* c = static_cast<RefineCtx*>(user);
+    if (c->fatal != TT_OK) return -1.f;
+    tt_status s = tt::apply_impl(c->w, rec, TT_MODE_LEGALISE, 0, nullptr);
+    if (s == TT_ERR_OOM || s == TT_ERR_CUDA) { c->fatal = s; return -1.f; }
+    if (s != TT_OK) return -1.f;
+    tt_timing tm{};
+    s = tt::time_applied(c->w, c->t, 1, c->st, c->o, &tm);
+    if (s == TT_ERR_OOM || s == TT_ERR_CUDA) { c->fatal = s; return -1.f; }
+    return s == TT_OK ? tm.median_us : -1.f;
+}
+}  // namespace
+
+tt_status tt_refine(tt_workload* w, const tt_tensors* t, void* cuda_stream, const tt_timing_opts* o,
+                    const tt_schedule_record* start, int32_t max_rounds, float min_gain, tt_schedule_record* best,
+                    float* best_us, float* start_us, int32_t* n_timed) {
+    if (!w || !t || !start || !best || !best_us) return TT_ERR_INVALID_ARG;
+    if (!device_present()) return TT_ERR_CUDA;
+    RefineCtx c{w, t, static_cast<cudaStream_t>(cuda_stream), o, TT_OK};
+    const tt_status s = tt_refine_with(w, start, refine_time, &c, max_rounds, min_gain, best, best_us, start_us, n_timed);
+    if (c.fatal != TT_OK) return c.fatal;
+    if (s != TT_OK) return s;
+    return tt::apply_impl(w, best, TT_MODE_LEGALISE, 0, nullptr);
 }
 
 }  // extern "C"

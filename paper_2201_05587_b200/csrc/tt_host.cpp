@@ -712,6 +712,118 @@ tt_status tt_schedule_check(const tt_workload* w, const tt_schedule_record* rec,
     return st;
 }
 
+// ---- refinement of a transferred record (Section 7, future work: "vary parameters from schedules transfer-tuned
+// from another model") ----
+namespace {
+struct FieldLadder { int32_t tt_schedule_record::*field; std::vector<int> steps; };   // two steps = a toggle when both differ
+
+const std::vector<FieldLadder>& ladders_of(uint32_t family) {
+    static const std::vector<FieldLadder> gemm = {
+        {&tt_schedule_record::tile_n, {16, 32, 48, 64, 96, 128, 160, 192, 224, 256}},
+        {&tt_schedule_record::tile_k, {8, 16, 32, 64, 96, 128}},
+        {&tt_schedule_record::stages, {1, 2, 3, 4, 5, 6, 7, 8}},
+        {&tt_schedule_record::split_k, {1, 2, 3, 4, 5, 6, 7, 8, 12, 16, 24, 32}},
+        {&tt_schedule_record::raster, {0, 1}},
+        {&tt_schedule_record::mma_m_axis, {1, 2}},
+        {&tt_schedule_record::slab_tiles, {0, 1, 2, 4, 8}},
+        {&tt_schedule_record::acc_split, {1, 2, 4, 8}},
+        {&tt_schedule_record::k_order, {0, 1}},
+    };
+    static const std::vector<FieldLadder> dw = {
+        {&tt_schedule_record::tile_m, {1, 2, 4, 8, 16, 32}},
+        {&tt_schedule_record::block_y, {1, 2, 4, 7, 8, 14, 16, 28, 56}},
+        {&tt_schedule_record::block_x, {8, 16, 28, 32, 56, 64, 112}},
+        {&tt_schedule_record::items_per_thread, {1, 2, 4, 8}},
+        {&tt_schedule_record::vec_width, {1, 2, 4}},
+        {&tt_schedule_record::threads, {32, 64, 128, 256, 512}},
+        {&tt_schedule_record::unroll, {0, 1, 2, 4}},
+        {&tt_schedule_record::raster, {0, 1}},
+        {&tt_schedule_record::stages, {2, 3, 4}},
+    };
+    static const std::vector<FieldLadder> row = {
+        {&tt_schedule_record::block_x, {1, 2, 4, 8, 16, 32}},
+        {&tt_schedule_record::block_y, {1, 2, 4, 8, 16}},
+        {&tt_schedule_record::vec_width, {1, 2, 4}},
+    };
+    return family == TT_FAMILY_GEMM_TC ? gemm : (family == TT_FAMILY_DW_SIMT ? dw : row);
+}
+}  // namespace
+
+tt_status tt_record_neighbours(const tt_workload* w, const tt_schedule_record* rec, tt_schedule_record* out, size_t cap,
+                               size_t* n_out) {
+    if (!w || !rec || !n_out || (cap > 0 && !out)) return TT_ERR_INVALID_ARG;
+    if (rec->version != TT_RECORD_VERSION || (int)rec->family != (int)w->family) return TT_ERR_INVALID_SCHEDULE;
+    // the start in its legalised form: a neighbour that legalises back to it is no neighbour
+    tt_apply_info start;
+    const tt_status s0 = tt_schedule_check(w, rec, TT_MODE_LEGALISE, 0, &start);
+    if (s0 != TT_OK) return s0;
+    std::vector<tt_schedule_record> found;
+    auto consider = [&](tt_schedule_record r) {
+        tt_apply_info info;
+        if (tt_schedule_check(w, &r, TT_MODE_LEGALISE, 0, &info) != TT_OK) return;
+        tt_schedule_record l = info.legal;
+        l.origin_op = rec->origin_op; l.origin = rec->origin;
+        tt_schedule_record s = start.legal;
+        s.origin_op = rec->origin_op; s.origin = rec->origin;
+        if (std::memcmp(&l, &s, sizeof l) == 0) return;
+        for (const auto& f : found) if (std::memcmp(&f, &l, sizeof l) == 0) return;
+        found.push_back(l);
+    };
+    for (const FieldLadder& fl : ladders_of(w->family)) {
+        const int v = start.legal.*(fl.field);
+        int below = INT32_MIN, above = INT32_MAX;       // nearest rungs on either side of v (v need not be a rung)
+        for (int step : fl.steps) {
+            if (step < v && step > below) below = step;
+            if (step > v && step < above) above = step;
+        }
+        if (below != INT32_MIN) { tt_schedule_record r = start.legal; r.*(fl.field) = below; consider(r); }
+        if (above != INT32_MAX) { tt_schedule_record r = start.legal; r.*(fl.field) = above; consider(r); }
+    }
+    *n_out = found.size();
+    if (found.size() > cap) return cap == 0 ? TT_OK : TT_ERR_RESOURCE;     // cap == 0: count only
+    for (size_t i = 0; i < found.size(); ++i) out[i] = found[i];
+    return TT_OK;
+}
+
+tt_status tt_refine_with(const tt_workload* w, const tt_schedule_record* start, tt_time_fn time_us, void* user,
+                         int32_t max_rounds, float min_gain, tt_schedule_record* best, float* best_us, float* start_us,
+                         int32_t* n_timed) {
+    if (!w || !start || !time_us || !best || !best_us || max_rounds < 0 || !(min_gain >= 0.f)) return TT_ERR_INVALID_ARG;
+    tt_apply_info info;
+    const tt_status s0 = tt_schedule_check(w, start, TT_MODE_LEGALISE, 0, &info);
+    if (s0 != TT_OK) return s0;
+    tt_schedule_record cur = info.legal;
+    cur.origin_op = start->origin_op; cur.origin = start->origin;
+    float cur_us = time_us(user, &cur);
+    int timed = 1;
+    if (start_us) *start_us = cur_us;
+    if (!(cur_us >= 0.f)) { if (n_timed) *n_timed = timed; return TT_ERR_INVALID_SCHEDULE; }
+    std::vector<tt_schedule_record> seen{cur};           // never time a record twice
+    for (int round = 0; round < max_rounds; ++round) {
+        size_t n = 0;
+        std::vector<tt_schedule_record> nb(32);
+        const tt_status sn = tt_record_neighbours(w, &cur, nb.data(), nb.size(), &n);
+        if (sn != TT_OK) return sn;
+        int pick = -1;
+        float pick_us = cur_us;
+        for (size_t i = 0; i < n; ++i) {
+            bool dup = false;
+            for (const auto& r : seen) if (std::memcmp(&r, &nb[i], sizeof r) == 0) { dup = true; break; }
+            if (dup) continue;
+            seen.push_back(nb[i]);
+            const float us = time_us(user, &nb[i]);
+            ++timed;
+            if (us >= 0.f && us < pick_us) { pick = (int)i; pick_us = us; }    // ties keep the earlier neighbour
+        }
+        // move only for a gain of more than min_gain (a fraction of the current time): noise does not walk the record
+        if (pick < 0 || !(pick_us < cur_us * (1.f - min_gain))) break;
+        cur = nb[(size_t)pick]; cur_us = pick_us;
+    }
+    *best = cur; *best_us = cur_us;
+    if (n_timed) *n_timed = timed;
+    return TT_OK;
+}
+
 tt_status tt_split_check(int64_t extent, const int64_t* factors, size_t n, int32_t reformulate, int32_t* valid) {
     if (!factors || !valid || n == 0 || extent <= 0) return TT_ERR_INVALID_ARG;
     if (reformulate) {

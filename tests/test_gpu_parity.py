@@ -277,6 +277,31 @@ def test_timing_and_grid_tuner_smoke():
     assert util.rel_l2(t["y"].cpu().numpy(), util.oracle_ref(spec, a)) <= util.TOL_TF32
 
 
+@pytest.mark.parametrize("spec,start", [
+    (W._conv(128, 28, 128, 3, 1, 1), tc(tile_n=32, tile_k=16, stages=2, split_k=1, mma_m_axis=2)),
+    (W._dw(96, 56, 1), B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=1, block_y=2, block_x=8, items_per_thread=1, vec_width=1,
+                                     threads=32, unroll=0)),
+], ids=lambda v: getattr(v, "name", None) or "start")
+def test_refining_a_transferred_record_never_loses_time_and_stays_correct(spec, start):
+    """tt_refine: greedy one-field-at-a-time descent from a (deliberately poor) transferred record.  The result is at
+    least as fast as the start by the search's own timings, is left applied, and computes what the oracle does."""
+    a = W.make_inputs(spec, 41)
+    wl = spec.workload()
+    t, tt = W.device_tensors(spec, a)
+    o = B.tt_timing_opts()
+    o.batches, o.warmup_batches, o.min_batch_us, o.use_graph = 5, 1, 100, 1
+    best, best_us, start_us, timed = wl.refine(tt, start, o, max_rounds=3, min_gain=0.02)
+    assert 0 < best_us <= start_us and timed >= 2
+    assert wl.check(best)[0] == B.TT_OK
+    if best_us < start_us:                          # a move was made: the record differs from the (legalised) start
+        assert best.as_dict() != wl.check(start)[1].legal.as_dict()
+    t["y"].fill_(float("nan"))
+    wl.run(tt)                                      # the best record is left applied
+    assert wl.status() == B.TT_OK
+    assert util.rel_l2(t["y"].cpu().numpy(), util.oracle_ref(spec, a)) <= util.tolerance(spec.op)
+    wl.close()
+
+
 def _model_parity(model, seed, recs):
     specs = W.MODELS[model]()
     for i, spec in enumerate(specs):

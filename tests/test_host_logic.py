@@ -3,6 +3,7 @@ import ctypes
 import os
 import re
 
+import numpy as np
 import pytest
 
 from oracle import oracle as orc
@@ -261,3 +262,107 @@ def test_tap_major_reduction_order_is_legalised_per_kernel():
     st, info = W._conv(64, 28, 64, 3, 1, 1).workload().check(odd)
     L = info.legal
     assert st == B.TT_OK and (L.tile_n, L.tile_k, L.split_k, L.mma_m_axis, L.k_order) == (112, 32, 1, 1, 1) and L.stages <= 8
+
+
+# ---- refinement of a transferred record: neighbourhood and greedy descent against the oracle's definitions ----
+_FAMILY_NAME = {B.TT_FAMILY_GEMM_TC: "gemm_tc", B.TT_FAMILY_DW_SIMT: "dw_simt", B.TT_FAMILY_ROW_SIMT: "row_simt"}
+
+
+def _rec_key(r):
+    return tuple(int(getattr(r, f)) for f in B.tt_schedule_record.FIELDS)
+
+
+def _legal_neighbours_by_definition(wl, rec):
+    """The oracle's raw one-step variations, mapped onto this workload by the validity layer (tt_schedule_check):
+    invalid ones, ones that coincide with the legalised start and repeats are dropped, order kept."""
+    st, info = wl.check(rec)
+    assert st == B.TT_OK
+    start = info.legal
+    fam = _FAMILY_NAME[int(start.family)]
+    out, seen = [], {_rec_key(start)}
+    for d in orc.raw_neighbours({f: int(getattr(start, f)) for f in B.tt_schedule_record.FIELDS}, fam):
+        r = B.make_record(int(start.family), **d)
+        st, info = wl.check(r)
+        if st != B.TT_OK or _rec_key(info.legal) in seen:
+            continue
+        seen.add(_rec_key(info.legal))
+        out.append(info.legal)
+    return out
+
+
+def _refine_cases():
+    r18 = W.resnet18()
+    mb = [s for s in W.mobilenet_v2() if s.op == B.TT_OP_DWCONV2D]
+    bert = W.bert_base()
+    cases = [(r18[1], B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=64, tile_k=32, stages=3, mma_m_axis=1)),
+             (r18[1], B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=256, tile_k=64, stages=4, split_k=8, mma_m_axis=2, k_order=1)),
+             (r18[-1], B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=16, tile_k=8, stages=1, split_k=3, mma_m_axis=1)),
+             (mb[0], B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=4, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=128, unroll=2)),
+             (mb[-1], B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=32, block_y=56, block_x=112, items_per_thread=8, vec_width=4, threads=512, unroll=4,
+                                    raster=1, stages=4)),
+             ([s for s in bert if s.op == B.TT_OP_SOFTMAX][0], B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=8, block_y=4, vec_width=2))]
+    return cases
+
+
+def test_record_neighbours_are_the_legalised_one_step_variations():
+    for spec, rec in _refine_cases():
+        wl = spec.workload()
+        got = wl.neighbours(rec)
+        want = _legal_neighbours_by_definition(wl, rec)
+        assert [_rec_key(r) for r in got] == [_rec_key(r) for r in want], spec.name
+        assert 0 < len(got) <= 18
+        _, info = wl.check(rec)
+        for r in got:                                    # each differs from the start, and is legal as written
+            assert _rec_key(r) != _rec_key(info.legal)
+            st, i2 = wl.check(r)
+            assert st == B.TT_OK and _rec_key(i2.legal) == _rec_key(r)
+        wl.close()
+
+
+def test_refine_with_follows_the_oracles_descent_on_synthetic_times():
+    import math
+    for spec, rec in _refine_cases():
+        wl = spec.workload()
+        # a deterministic, bumpy "time" per record: separable bowls plus a hash term, some records unable to run
+        def cost(key):
+            h = (hash(key) % 1000) / 1000.0
+            if int(h * 1000) % 7 == 0:
+                return -1.0
+            return float(np.float32(50.0 + sum(abs(math.log2(v + 1) - 3.0) * (i % 3 + 1) for i, v in enumerate(key)) + 3.0 * h))
+        _, info = wl.check(rec)
+        start_key = _rec_key(info.legal)
+        if cost(start_key) < 0:
+            wl.close()
+            continue
+        by_key = {}
+        def nb(key):
+            r = by_key.get(key) or info.legal
+            out = _legal_neighbours_by_definition(wl, r)
+            for x in out:
+                by_key[_rec_key(x)] = x
+            return [_rec_key(x) for x in out]
+        by_key[start_key] = info.legal
+        for rounds, gain in ((0, 0.0), (1, 0.0), (6, 0.0), (6, 0.03)):
+            want = orc.refine(start_key, nb, cost, rounds, gain)
+            best, best_us, start_us, timed = wl.refine_with(rec, lambda r: cost(_rec_key(r)), rounds, gain)
+            assert _rec_key(best) == want[0], (spec.name, rounds, gain)
+            assert best_us == pytest.approx(want[1]) and start_us == pytest.approx(want[2]) and timed == want[3]
+        wl.close()
+
+
+def test_refine_rejects_bad_arguments_and_needs_a_device_for_device_times():
+    spec, rec = _refine_cases()[0]
+    wl = spec.workload()
+    other = B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=8, block_y=4, vec_width=2)
+    with pytest.raises(B.TTError):
+        wl.neighbours(other)                             # a record of another family
+    with pytest.raises(B.TTError):
+        wl.refine_with(rec, lambda r: -1.0, 3, 0.0)      # the start itself cannot run
+    with pytest.raises(B.TTError):
+        wl.refine_with(rec, lambda r: 1.0, -1, 0.0)
+    import torch
+    if not torch.cuda.is_available():
+        t, best, us = B.tt_tensors(), B.tt_schedule_record(), ctypes.c_float()
+        assert B.lib().tt_refine(wl.handle, ctypes.byref(t), None, None, ctypes.byref(rec), 2, 0.0, ctypes.byref(best),
+                                 ctypes.byref(us), None, None) == B.TT_ERR_CUDA      # no CPU fallback
+    wl.close()

@@ -320,3 +320,71 @@ def test_selection_heuristic_special_cases():
     assert s == [2.0, 4.0, 0.0] and order == [1, 0, 2]
     # ties keep the lower index
     assert orc.rank_pools({"A": 0.3}, [{"A": 2}, {"A": 2}])[1] == [0, 1]
+
+
+# ---- refining a transferred schedule: greedy one-parameter-at-a-time descent (Section 7, future work) ----
+def test_ladder_steps_are_the_adjacent_rungs():
+    lad = [1, 2, 4, 7, 8, 14]
+    assert orc.ladder_steps(4, lad) == [2, 7]
+    assert orc.ladder_steps(1, lad) == [2]
+    assert orc.ladder_steps(14, lad) == [8]
+    assert orc.ladder_steps(5, lad) == [4, 7]            # a value between two rungs
+    assert orc.ladder_steps(100, lad) == [14] and orc.ladder_steps(0, lad) == [1]
+    assert orc.ladder_steps(0, [0, 1]) == [1] and orc.ladder_steps(1, [0, 1]) == [0]
+
+
+def test_raw_neighbours_change_exactly_one_parameter_by_one_rung():
+    rec = {"block_x": 8, "block_y": 4, "vec_width": 2}
+    nb = orc.raw_neighbours(rec, "row_simt")
+    assert nb == [{"block_x": 4, "block_y": 4, "vec_width": 2}, {"block_x": 16, "block_y": 4, "vec_width": 2},
+                  {"block_x": 8, "block_y": 2, "vec_width": 2}, {"block_x": 8, "block_y": 8, "vec_width": 2},
+                  {"block_x": 8, "block_y": 4, "vec_width": 1}, {"block_x": 8, "block_y": 4, "vec_width": 4}]
+    for fam in orc.LADDERS:
+        start = {name: lad[len(lad) // 2] for name, lad in orc.LADDERS[fam]}
+        for r in orc.raw_neighbours(start, fam):
+            changed = [k for k in r if r[k] != start[k]]
+            assert len(changed) == 1
+            lad = dict(orc.LADDERS[fam])[changed[0]]
+            assert abs(lad.index(r[changed[0]]) - lad.index(start[changed[0]])) == 1
+
+
+def _row_space():
+    lads = orc.LADDERS["row_simt"]
+    names = [n for n, _ in lads]
+    return names, [dict(zip(names, vals)) for vals in __import__("itertools").product(*[l for _, l in lads])]
+
+
+def test_refine_reaches_the_exhaustive_minimum_of_a_separable_convex_cost():
+    # cost = sum of per-parameter convex bowls: a one-parameter-at-a-time descent cannot get stuck, so it must end at
+    # the minimum that exhaustive search over the whole space finds
+    names, space = _row_space()
+    target = {"block_x": 16, "block_y": 2, "vec_width": 4}
+    cost = lambda d: 10.0 + sum((np.log2(d[k]) - np.log2(target[k])) ** 2 * (i + 1) for i, k in enumerate(names))
+    key = lambda d: tuple(d[k] for k in names)
+    unkey = lambda t: dict(zip(names, t))
+    best_exh = min(space, key=cost)
+    for start in ({"block_x": 1, "block_y": 16, "vec_width": 1}, {"block_x": 32, "block_y": 1, "vec_width": 2}, dict(target)):
+        best, best_us, start_us, timed = orc.refine(key(start), lambda s: [key(r) for r in orc.raw_neighbours(unkey(s), "row_simt")],
+                                                    lambda s: cost(unkey(s)), max_rounds=50)
+        assert unkey(best) == best_exh == target
+        assert best_us == pytest.approx(10.0) and start_us == pytest.approx(cost(start))
+        assert timed <= len(space)                       # nothing is timed twice
+    # from the optimum: one round, every neighbour timed once, no move
+    _, _, _, timed = orc.refine(key(target), lambda s: [key(r) for r in orc.raw_neighbours(unkey(s), "row_simt")],
+                                lambda s: cost(unkey(s)), max_rounds=50)
+    assert timed == 1 + len(orc.raw_neighbours(target, "row_simt"))
+
+
+def test_refine_round_limit_gain_threshold_invalid_and_ties():
+    chain = {0: [1], 1: [2], 2: [3], 3: []}
+    t = {0: 10.0, 1: 9.0, 2: 8.0, 3: 7.0}
+    assert orc.refine(0, chain.__getitem__, t.__getitem__, max_rounds=2)[0] == 2           # two moves, no more
+    assert orc.refine(0, chain.__getitem__, t.__getitem__, max_rounds=0) == (0, 10.0, 10.0, 1)
+    t2 = {0: 10.0, 1: 8.5, 2: 8.0, 3: 1.0}
+    assert orc.refine(0, chain.__getitem__, t2.__getitem__, max_rounds=9, min_gain=0.10)[0] == 1   # 15 % moves, the next 5.9 % does not
+    assert orc.refine(0, chain.__getitem__, t.__getitem__, max_rounds=9, min_gain=0.10)[0] == 0    # a gain must EXCEED the threshold
+    # a neighbour that cannot run (negative time) is never chosen, however "fast"; ties keep the earlier neighbour
+    star = {0: [1, 2, 3], 1: [], 2: [], 3: []}
+    assert orc.refine(0, star.__getitem__, {0: 5.0, 1: -1.0, 2: 4.0, 3: 4.0}.__getitem__, 3)[0] == 2
+    with pytest.raises(ValueError):
+        orc.refine(0, star.__getitem__, {0: -1.0, 1: 1.0, 2: 1.0, 3: 1.0}.__getitem__, 3)
