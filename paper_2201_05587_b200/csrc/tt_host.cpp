@@ -201,7 +201,8 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
         return TT_ERR_INVALID_SCHEDULE;
     // Which output axis becomes the accumulator's 128 rows.  Left to the library (0), the shorter-than-a-tile
     // axis goes to the MMA's N side, where 16..256 columns are legal.
-    const tt_shapes& s = w->sh;
+    tt_shapes s = w->sh;                                  // a copy: a pointwise convolution is re-viewed below
+    int P = w->P, Q = w->Q;
     bool swap = rec->mma_m_axis == 2;
     if (rec->mma_m_axis == 0) swap = w->view.gm <= 64 && w->view.gn > w->view.gm;
     L.mma_m_axis = swap ? 2 : 1;
@@ -279,7 +280,20 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
         if (rec->slab_tiles < 0) return TT_ERR_INVALID_SCHEDULE;
         if (strict && rec->slab_tiles > per_split) return TT_ERR_INVALID_SCHEDULE;
         const int pix_rows = swap ? kHwTileM : tn;       // output pixels per tile of the im2col operand
-        const int out_rows = std::min(w->P, (pix_rows + 2 * w->Q - 2) / w->Q);
+        // A pointwise convolution (1x1, stride 1, no padding) sees no neighbourhood: its H x W pixels are one run of
+        // H*W values per channel, and any H' x W' with the same product is the same kernel.  Rows of W' pixels with
+        // W' the largest multiple of 4 that divides both H*W and the tile's pixel count make every tile a whole
+        // number of rows, so a slab chunk holds exactly the tile's pixels (the image's own rows would add up to a
+        // row on either side: 224 staged pixels for 128 at 56 x 56).
+        bool whole_rows = false;
+        if (s.r == 1 && s.s == 1 && s.stride_h == 1 && s.stride_w == 1 && s.pad_h == 0 && s.pad_w == 0) {
+            const long long hw = (long long)s.h * s.w;
+            int best = 0;
+            for (int d = 16; d <= 248 && d <= pix_rows; d += 4)
+                if (hw % d == 0 && pix_rows % d == 0) best = d;
+            if (best > 0) { s.w = best; s.h = (int)(hw / best); P = s.h; Q = s.w; whole_rows = true; }
+        }
+        const int out_rows = whole_rows ? std::min(P, pix_rows / Q) : std::min(P, (pix_rows + 2 * Q - 2) / Q);
         sl_rstep = std::min(s.stride_h, s.r);
         sl_in_rows = s.stride_h <= s.r ? (out_rows - 1) * s.stride_h + s.r : out_rows * s.r;
         sl_gap = round_up(std::max(1, std::max(s.pad_w, s.s - 1 - s.pad_w)), 4);
@@ -389,7 +403,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     if (w->op == TT_OP_CONV2D) {
         U = {k4 ? OPM_TMA : OPM_GATHER_K, K, 1, 0, 0};                         // filters [k][c*r*s], shared by images
         V = {OPM_IM2COL, 0, 0, (long long)s.c * s.h * s.w, 1};                 // pixels x (c,r,s) gathered from NCHW
-        y_is = (long long)w->P * w->Q; y_js = 1; y_bs = (long long)s.k * w->P * w->Q; bias_on = 1;
+        y_is = (long long)P * Q; y_js = 1; y_bs = (long long)s.k * P * Q; bias_on = 1;
     } else if (w->op == TT_OP_DENSE) {
         U = {k4 ? OPM_TMA : OPM_GATHER_K, K, 1, 0, 0};
         V = {k4 ? OPM_TMA : OPM_GATHER_K, K, 1, 0, 0};
@@ -410,7 +424,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     g.y_ms = swap ? y_js : y_is; g.y_ns = swap ? y_is : y_js; g.y_bs = y_bs;
     g.bias_mode = s.has_bias ? (swap ? 3 - bias_on : bias_on) : 0;
     g.act = s.act;
-    g.C = s.c; g.H = s.h; g.W = s.w; g.R = s.r; g.S = s.s; g.Q = w->Q;
+    g.C = s.c; g.H = s.h; g.W = s.w; g.R = s.r; g.S = s.s; g.Q = Q;
     g.sh = s.stride_h; g.sw = s.stride_w; g.ph = s.pad_h; g.pw = s.pad_w;
     g.tx_bytes = (A.mode == OPM_TMA ? a_stage : 0) + (Bo.mode == OPM_TMA ? b_stage : 0);
     g.vec_store = (g.y_ns == 1 && g.y_ms % 4 == 0 && g.y_bs % 4 == 0) ? 1 : 0;
