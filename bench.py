@@ -27,7 +27,7 @@ UNIT = "TFLOP/s"
 # DRAM traffic of the dominant kernel per launch (dram__bytes_read.sum + dram__bytes_write.sum averaged over the
 # timed region's launches, one ncu pass; its summary is kept under profiles/), valid only for the
 # kernel source it was taken on: any later change of the kernel reports null until the counters are taken again.
-TRAFFIC_COUNTERS = {"model": "resnet18", "kernel_source_sha256_16": "610ef33186034c34", "bytes_per_launch": 2.735e6}
+TRAFFIC_COUNTERS = {"model": "resnet18", "kernel_source_sha256_16": "e851abb110f2b72c", "bytes_per_launch": 2.734e6}
 
 
 def kernel_source_hash():
@@ -175,10 +175,14 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
         (conv(32, 128, 28, 128, 3, 1), "tensor",
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=128, tile_k=32, stages=3, mma_m_axis=2),
           tc(tile_n=128, tile_k=64, stages=2, mma_m_axis=2),
-          tc(tile_n=256, tile_k=32, stages=5, k_order=1, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=4, k_order=1, mma_m_axis=1)]),
+          tc(tile_n=256, tile_k=32, stages=5, k_order=1, mma_m_axis=1), tc(tile_n=224, tile_k=96, stages=2, k_order=1, mma_m_axis=1)]),
         (conv(32, 256, 28, 256, 3, 1), "tensor",
-         [tc(tile_n=256, tile_k=32, stages=5, k_order=1, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=4, k_order=1, mma_m_axis=1),
+         [tc(tile_n=256, tile_k=32, stages=5, k_order=1, mma_m_axis=1), tc(tile_n=224, tile_k=96, stages=2, k_order=1, mma_m_axis=1),
           tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1)]),
+        # the same layer at batch 37: 8 tiles x 37 images = 296 CTAs = exactly two per SM-slot wave of 148 (batch 32
+        # leaves the second wave 27 % empty)
+        (conv(37, 256, 28, 256, 3, 1), "tensor",
+         [tc(tile_n=224, tile_k=96, stages=2, k_order=1, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=5, k_order=1, mma_m_axis=1)]),
         (conv(32, 256, 56, 64, 1, 0), "hbm",
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=2),
           tc(tile_n=64, tile_k=32, stages=2, mma_m_axis=2, slab_tiles=1), tc(tile_n=64, tile_k=32, stages=3, mma_m_axis=2, slab_tiles=1)]),
@@ -422,9 +426,15 @@ def main():
     if rank == 0:
         cpu = None
         if not args.no_cpu_baseline:
-            f, s, used, names = cpu_baseline_oracle(specs, arrays, 20.0)
+            # the whole pass costs the oracle a fraction of a second: repeat it until about ten seconds have been timed
+            f = s = 0.0
+            rounds = 0
+            while s < 10.0 and rounds < 1000:
+                f1, s1, used, names = cpu_baseline_oracle(specs, arrays, 20.0)
+                f += f1; s += s1; rounds += 1
             cpu = {"value": f / s / 1e12, "unit": UNIT, "cores": used, "kind": "oracle",
-                   "sample": f"{len(names)} of {len(specs)} unique kernels once each ({f / 1e9:.2f} GFLOP in {s:.1f} s)"}
+                   "sample": f"{len(names)} of {len(specs)} unique kernels once each per round, {rounds} rounds "
+                             f"({f / 1e9:.1f} GFLOP in {s:.1f} s)"}
         clocks = sampler.summary()
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
