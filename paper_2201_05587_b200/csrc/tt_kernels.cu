@@ -5,8 +5,10 @@
 //            staged once per CTA (im2col of NCHW activations), or by gathers (strided views).  Bias/activation are
 //            fused into the accumulator read-out.  Split-K of 2..8 runs as a thread-block cluster that reduces
 //            through distributed shared memory; more splits go through a workspace and the last-arriving CTA adds
-//            them up, both in fixed split order.  Launched with programmatic stream serialization.
-//   DW_SIMT  depthwise convolution: a register-window kernel (3x3 / 5x5) and a shared-memory staged kernel, fp32 FMA.
+//            them up, both in fixed split order.  Launched with programmatic stream serialization.  Built twice:
+//            with all registers (one CTA per SM) and capped so that two CTAs share an SM on large grids.
+//   DW_SIMT  depthwise convolution, fp32 FMA: a persistent kernel whose tiles' input boxes arrive by TMA (3x3 / 5x5,
+//            16-byte image rows), a register-window kernel (3x3 / 5x5) and a shared-memory staged kernel.
 //   ROW_SIMT row softmax with sub-warp shuffles, register-resident rows when they fit.
 //
 // Every tile size, the pipeline depth, split-K and the tile order are run-time values taken from the applied
