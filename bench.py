@@ -162,10 +162,10 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
     def conv(n, c, hw, k, r, pad):
         return W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(n, c, hw, hw, k, r, r, 1, pad, True, B.TT_ACT_RELU), 1,
                       f"conv{r}x{r}_n{n}_{c}x{hw}->{k}")
-    def dw(n, c, hw, stride):
-        sh = B.make_shapes(n=n, c=c, h=hw, w=hw, k=c, r=3, s=3, stride_h=stride, stride_w=stride, pad_h=1, pad_w=1,
+    def dw(n, c, hw, stride, r=3):
+        sh = B.make_shapes(n=n, c=c, h=hw, w=hw, k=c, r=r, s=r, stride_h=stride, stride_w=stride, pad_h=r // 2, pad_w=r // 2,
                            has_bias=1, act=B.TT_ACT_RELU6)
-        return W.Spec(B.TT_OP_DWCONV2D, sh, 1, f"dw3x3s{stride}_n{n}_{c}x{hw}")
+        return W.Spec(B.TT_OP_DWCONV2D, sh, 1, f"dw{r}x{r}s{stride}_n{n}_{c}x{hw}")
     tc = lambda **kw: B.make_record(B.TT_FAMILY_GEMM_TC, **kw)
     dwr = lambda **kw: B.make_record(B.TT_FAMILY_DW_SIMT, **kw)
     cases = [
@@ -199,6 +199,11 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
           dwr(tile_m=1, block_y=8, block_x=56, items_per_thread=4, vec_width=4, threads=64, unroll=2),
           dwr(tile_m=4, block_y=8, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=2, raster=1, stages=2),
           dwr(tile_m=8, block_y=4, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=2, raster=1, stages=2)]),
+        (dw(256, 240, 28, 1, r=5), "hbm",      # an EfficientNet-B0-shaped 5x5 layer
+         [dwr(tile_m=4, block_y=14, block_x=28, items_per_thread=4, vec_width=4, threads=128, unroll=2),
+          dwr(tile_m=16, block_y=14, block_x=28, items_per_thread=4, vec_width=4, threads=256, unroll=2, raster=1, stages=2),
+          dwr(tile_m=8, block_y=28, block_x=28, items_per_thread=4, vec_width=4, threads=256, unroll=4, raster=1, stages=2),
+          dwr(tile_m=16, block_y=28, block_x=28, items_per_thread=4, vec_width=4, threads=256, unroll=2, raster=1, stages=2)]),
         (W.Spec(B.TT_OP_SOFTMAX, B.softmax_shapes(12 * 256, 128, 128, 0.125), 1, "softmax_3072x128x128", "bert"), "hbm",
          [B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=8, block_y=8, vec_width=4),
           B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=32, block_y=4, vec_width=4)]),

@@ -110,6 +110,12 @@ def test_dense_parity_all_records(spec):
     W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(2, 33, 8, 20, 10, 5, 3, 1, 2, True, B.TT_ACT_RELU6), 1, "conv5x3_batch2_tap", "uniform"),
     W._conv(20, 10, 40, 1, 1, 0, name="conv1x1_100px_20ch"),
     W._conv(136, 12, 200, 1, 1, 0, act=B.TT_ACT_NONE, name="conv1x1_136ch"),
+    # pointwise layers whose pixels are re-viewed as rows that tile the CTA exactly: 400 = 16 x 25, 784 = 16 x 49,
+    # 3136 = 64 x 49 (batch 3, a partial last tile, a residual), and one whose pixel count has no such divisor
+    W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(3, 40, 20, 20, 24, 1, 1, 1, 0, True, B.TT_ACT_RELU, True), 1, "conv1x1_400px_batch3_residual", "uniform"),
+    W._conv(64, 28, 80, 1, 1, 0, act=B.TT_ACT_RELU6, name="conv1x1_784px"),
+    W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(2, 24, 56, 56, 40, 1, 1, 1, 0, True, B.TT_ACT_NONE), 1, "conv1x1_3136px_batch2", "uniform"),
+    W._conv(48, 18, 32, 1, 1, 0, name="conv1x1_324px_no_row_view"),
     W._conv(96, 9, 48, 3, 1, 1, name="conv3x3_96ch_chunks"),                # 864 reduction indices: many slab chunks
     W._conv(40, 12, 24, 5, 1, 2, act=B.TT_ACT_RELU6, name="conv5x5_pad2"),
     W._conv(32, 17, 16, 1, 3, 0, name="conv1x1s3"),                         # stride beyond the filter: rows are skipped
