@@ -192,7 +192,7 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
           dwr(tile_m=4, block_y=16, block_x=56, items_per_thread=4, vec_width=4, threads=128, unroll=4),
           dwr(tile_m=8, block_y=56, block_x=56, items_per_thread=8, vec_width=4, threads=128, unroll=2),
           dwr(tile_m=8, block_y=14, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=4, raster=1, stages=2),
-          dwr(tile_m=16, block_y=8, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=4, raster=1, stages=2)]),
+          dwr(tile_m=4, block_y=28, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=4, raster=1, stages=2)]),
         (dw(32, 96, 112, 2), "hbm",
          [dwr(tile_m=4, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=2),
           dwr(tile_m=4, block_y=4, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=1),

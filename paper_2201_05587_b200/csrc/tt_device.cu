@@ -588,8 +588,8 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
         }
         // TMA-staged persistent kernel (raster = 1): strips of 4 or 8 columns, 1-4 rows; tiles span the image width
         // where they can (a box then needs no columns of a neighbouring tile)
-        const std::vector<int> pcs = full ? std::vector<int>{1, 2, 4, 8, 16, 32} : std::vector<int>{2, 8, 16};
-        const std::vector<int> pys = full ? std::vector<int>{2, 4, 7, 8, 14, 16, 28, 56} : std::vector<int>{4, 8, 14};
+        const std::vector<int> pcs = full ? std::vector<int>{1, 2, 4, 8, 16, 32} : std::vector<int>{2, 4, 8, 16};
+        const std::vector<int> pys = full ? std::vector<int>{2, 4, 7, 8, 14, 16, 28, 56} : std::vector<int>{4, 8, 14, 28};
         const std::vector<int> pxs = full ? std::vector<int>{16, 28, 32, 56, 64, 112} : std::vector<int>{32, 56, 112};
         for (int it : full ? std::vector<int>{4, 8} : std::vector<int>{4}) for (int ro : {2, 4}) for (int tc : pcs) for (int by : pys)
             for (int bx : pxs) for (int sg : full ? std::vector<int>{2, 3, 4} : std::vector<int>{2, 3}) {
