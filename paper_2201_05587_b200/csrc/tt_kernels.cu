@@ -21,6 +21,7 @@
 #include <cstdint>
 #include <cstring>
 #include <algorithm>
+#include <utility>
 #include "tt_internal.h"
 
 namespace tt {
@@ -94,6 +95,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;         // the common case costs one instruction
     return mbar_wait_slow(bar, parity, abort_flag, status, where);
 }
+
+// Programmatic dependent launch.  A kernel launched with programmatic stream serialization may become resident while
+// its predecessor in the stream is still running; it must wait here before its first access to global memory.  The
+// kernel after it is allowed to do the same from this kernel's entry on.  (Without the launch attribute both
+// instructions do nothing.)
+__device__ __forceinline__ void pdl_allow_next() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_prev() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // One lane of a converged warp (the same lane every time): it issues the warp's asynchronous instructions.
 __device__ __forceinline__ bool elect_one() {
@@ -1479,6 +1487,8 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 // consecutive outputs along the width and stores them with vec-wide stores.
 // ------------------------------------------------------------------------------------------------------------
 __global__ void tt_dwconv_kernel(const DwArgs d) {
+    pdl_allow_next();
+    pdl_wait_prev();
     extern __shared__ float dsm[];
     const int n = blockIdx.y;
     int t = blockIdx.x;
@@ -1561,6 +1571,8 @@ __global__ void __launch_bounds__(256, WIDTH == 4 ? 6 : 4) tt_dwconv_window_kern
     constexpr int IN_ROWS = (ROWS - 1) * STRIDE + R;
     constexpr int PAD = R / 2;                            // "same" padding: the launcher checks it
     constexpr int NV = (NCOL - PAD) / 4;                  // aligned 16-byte groups per window row
+    pdl_allow_next();
+    pdl_wait_prev();
     const int n = blockIdx.y;
     int t = blockIdx.x;
     const int tw = t % d.tiles_w; t /= d.tiles_w;
@@ -1685,6 +1697,7 @@ __global__ void __launch_bounds__(256) tt_dwconv_tma_kernel(const __grid_constan
     const uint32_t base = (smem_u32(dw_raw) + 127u) & ~127u;
     const uint32_t wbase = base + (uint32_t)d.tma_stages * (uint32_t)d.stage_bytes;
     volatile int* abortp = &abort_flag;
+    pdl_allow_next();
     if (threadIdx.x == 0) {
         for (int s = 0; s < d.tma_stages; ++s) mbar_init(smem_u32(&full_bar[s]), 1u);
         abort_flag = 0;
@@ -1693,6 +1706,7 @@ __global__ void __launch_bounds__(256) tt_dwconv_tma_kernel(const __grid_constan
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
     }
     __syncthreads();
+    pdl_wait_prev();                                      // the set-up above touched no global memory
     const int planes = d.N * d.C;
     const int per_plane_tiles = d.tiles_h * d.tiles_w;
     const int my_tiles = d.total_tiles > (int)blockIdx.x ? (d.total_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
@@ -1873,6 +1887,8 @@ __global__ void __launch_bounds__(256) tt_dwconv_tma_kernel(const __grid_constan
 // ROW_SIMT: softmax(scale * x) per row; `lanes_per_row` threads of one warp share a row.
 // ------------------------------------------------------------------------------------------------------------
 __global__ void tt_softmax_kernel(const RowArgs a) {
+    pdl_allow_next();
+    pdl_wait_prev();
     const int lpr = a.lanes_per_row;
     const int sub = threadIdx.x % lpr;
     const long long row = (long long)blockIdx.x * a.rows_per_cta + threadIdx.x / lpr;
@@ -1909,6 +1925,8 @@ __global__ void tt_softmax_kernel(const RowArgs a) {
 // whose length is a multiple of 4 and whose pointers are 16-byte aligned; everything else takes the kernel above.
 template <int NV>
 __global__ void tt_softmax_cached_kernel(const RowArgs a) {
+    pdl_allow_next();
+    pdl_wait_prev();
     const int lpr = a.lanes_per_row;
     const int sub = threadIdx.x % lpr;
     const long long row = (long long)blockIdx.x * a.rows_per_cta + threadIdx.x / lpr;
@@ -2034,6 +2052,19 @@ cudaError_t launch_repack(const float* w, float* out, int kout, int C, int RS, i
     return cudaGetLastError();
 }
 
+// Launch with programmatic stream serialization (the kernels wait before their first global access): in a stream or
+// a captured graph the kernel's launch latency and set-up hide behind its predecessor's tail.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_serialized(void (*kern)(KArgs...), dim3 grid, unsigned threads, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = dim3(threads, 1, 1); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 cudaError_t launch_dw_tma(const tt_apply_info& I, const DwArgs& dw, const void* tmap_x, cudaStream_t st) {
     CUtensorMap tx;
     memcpy(&tx, tmap_x, sizeof tx);
@@ -2053,7 +2084,7 @@ cudaError_t launch_dw_tma(const tt_apply_info& I, const DwArgs& dw, const void* 
         if (occ < 1) return cudaErrorLaunchOutOfResources; \
         /* persistent CTAs: never more than are resident at once (registers may allow fewer than shared memory does) */ \
         grid.x = (unsigned)std::min<long long>(grid.x, (long long)sm_count * occ); \
-        tt_dwconv_tma_kernel<RR, SS, RO, WI><<<grid, I.threads, I.smem_bytes, st>>>(tx, dw); return cudaGetLastError(); }
+        return launch_serialized(tt_dwconv_tma_kernel<RR, SS, RO, WI>, grid, (unsigned)I.threads, (size_t)I.smem_bytes, st, tx, dw); }
     TT_DWT_CASE(3, 1, 1, 4) TT_DWT_CASE(3, 1, 2, 4) TT_DWT_CASE(3, 1, 4, 4) TT_DWT_CASE(3, 1, 1, 8) TT_DWT_CASE(3, 1, 2, 8)
     TT_DWT_CASE(3, 2, 1, 4) TT_DWT_CASE(3, 2, 2, 4) TT_DWT_CASE(3, 2, 4, 4) TT_DWT_CASE(3, 2, 1, 8) TT_DWT_CASE(3, 2, 2, 8)
     TT_DWT_CASE(5, 1, 1, 4) TT_DWT_CASE(5, 1, 2, 4) TT_DWT_CASE(5, 1, 4, 4) TT_DWT_CASE(5, 1, 1, 8) TT_DWT_CASE(5, 1, 2, 8)
@@ -2075,7 +2106,7 @@ cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st)
     if (dw.window_rows > 0) {
         // register-window kernels: one instantiation per (filter size, stride, output rows per thread)
 #define TT_DW_CASE(RR, SS, RO, WD) \
-        if (dw.R == RR && dw.sh == SS && dw.window_rows == RO && dw.items == WD) { tt_dwconv_window_kernel<RR, SS, RO, WD><<<grid, I.threads, 0, st>>>(dw); return cudaGetLastError(); }
+        if (dw.R == RR && dw.sh == SS && dw.window_rows == RO && dw.items == WD) return launch_serialized(tt_dwconv_window_kernel<RR, SS, RO, WD>, grid, (unsigned)I.threads, 0, st, dw);
         TT_DW_CASE(3, 1, 1, 4) TT_DW_CASE(3, 1, 2, 4) TT_DW_CASE(3, 1, 4, 4)
         TT_DW_CASE(3, 2, 1, 4) TT_DW_CASE(3, 2, 2, 4) TT_DW_CASE(3, 2, 4, 4)
         TT_DW_CASE(5, 1, 1, 4) TT_DW_CASE(5, 1, 2, 4) TT_DW_CASE(5, 1, 4, 4)
@@ -2085,22 +2116,20 @@ cudaError_t launch_dw(const tt_apply_info& I, const DwArgs& dw, cudaStream_t st)
 #undef TT_DW_CASE
         return cudaErrorInvalidValue;
     }
-    tt_dwconv_kernel<<<grid, I.threads, I.smem_bytes, st>>>(dw);
-    return cudaGetLastError();
+    return launch_serialized(tt_dwconv_kernel, grid, (unsigned)I.threads, (size_t)I.smem_bytes, st, dw);
 }
 
 cudaError_t launch_row(const tt_apply_info& I, const RowArgs& row, cudaStream_t st) {
     // rows that fit the lanes' registers (and allow 16-byte accesses) are read once
     const int per_lane = row.vec == 4 ? ((row.cols >> 2) + row.lanes_per_row - 1) / row.lanes_per_row : 0;
     if (per_lane >= 1 && per_lane <= 8) {
-        if (per_lane == 1) tt_softmax_cached_kernel<1><<<I.grid_x, I.threads, 0, st>>>(row);
-        else if (per_lane == 2) tt_softmax_cached_kernel<2><<<I.grid_x, I.threads, 0, st>>>(row);
-        else if (per_lane <= 4) tt_softmax_cached_kernel<4><<<I.grid_x, I.threads, 0, st>>>(row);
-        else tt_softmax_cached_kernel<8><<<I.grid_x, I.threads, 0, st>>>(row);
-        return cudaGetLastError();
+        const dim3 grid(I.grid_x, 1, 1);
+        if (per_lane == 1) return launch_serialized(tt_softmax_cached_kernel<1>, grid, (unsigned)I.threads, 0, st, row);
+        if (per_lane == 2) return launch_serialized(tt_softmax_cached_kernel<2>, grid, (unsigned)I.threads, 0, st, row);
+        if (per_lane <= 4) return launch_serialized(tt_softmax_cached_kernel<4>, grid, (unsigned)I.threads, 0, st, row);
+        return launch_serialized(tt_softmax_cached_kernel<8>, grid, (unsigned)I.threads, 0, st, row);
     }
-    tt_softmax_kernel<<<I.grid_x, I.threads, 0, st>>>(row);
-    return cudaGetLastError();
+    return launch_serialized(tt_softmax_kernel, dim3(I.grid_x, 1, 1), (unsigned)I.threads, 0, st, row);
 }
 
 }  // namespace tt
