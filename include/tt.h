@@ -232,6 +232,13 @@ tt_status tt_run(tt_workload* w, const tt_tensors* t, void* cuda_stream);
 /* The same with HOST pointers: copies x, w, bias, residual to library-owned device buffers, runs, copies y back,
  * synchronises.  bytes_h2d/bytes_d2h (may be NULL) receive the bytes copied. */
 tt_status tt_run_host(tt_workload* w, const tt_tensors* host, void* cuda_stream, int64_t* bytes_h2d, int64_t* bytes_d2h);
+/* The same without the final synchronisation: the copies and the kernel are only enqueued on `cuda_stream`, so calls
+ * for DIFFERENT workloads on different streams overlap their transfers (both directions) and kernels.  The host
+ * buffers must be page-locked for the copies to be asynchronous and must stay untouched until the stream has been
+ * synchronised; y and the device status are valid after tt_workload_status(w, cuda_stream) (or any synchronisation
+ * of that stream).  A workload owns one set of device staging buffers: enqueue its calls on one stream at a time. */
+tt_status tt_run_host_async(tt_workload* w, const tt_tensors* host, void* cuda_stream, int64_t* bytes_h2d,
+                            int64_t* bytes_d2h);
 /* Read and clear the device status word of the last runs (TT_OK or TT_ERR_TIMEOUT); synchronises the stream. */
 tt_status tt_workload_status(tt_workload* w, void* cuda_stream);
 

@@ -107,6 +107,7 @@ EXPORTS = {
     "tt_split_check": (i32, [C.c_int64, C.POINTER(C.c_int64), C.c_size_t, i32, C.POINTER(i32)]),
     "tt_run": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p]),
     "tt_run_host": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
+    "tt_run_host_async": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "tt_workload_status": (i32, [C.c_void_p, C.c_void_p]),
     "tt_time": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_size_t, C.c_void_p, C.POINTER(tt_timing_opts),
                       C.POINTER(tt_timing)]),
@@ -319,8 +320,17 @@ class Workload:
                f"tt_run_host({self.name})")
         return up.value, down.value
 
-    def status(self) -> int:
-        return lib().tt_workload_status(self.handle, _stream())
+    def run_host_async(self, t: tt_tensors, stream=None):
+        """tt_run_host_async on `stream` (a torch.cuda.Stream; default: the current one): enqueues only."""
+        up, down = C.c_int64(), C.c_int64()
+        sp = _stream() if stream is None else C.c_void_p(stream.cuda_stream)
+        _check(lib().tt_run_host_async(self.handle, C.byref(t), sp, C.byref(up), C.byref(down)),
+               f"tt_run_host_async({self.name})")
+        return up.value, down.value
+
+    def status(self, stream=None) -> int:
+        sp = _stream() if stream is None else C.c_void_p(stream.cuda_stream)
+        return lib().tt_workload_status(self.handle, sp)
 
     def time(self, sets, opts: tt_timing_opts | None = None) -> tt_timing:
         if isinstance(sets, tt_tensors):

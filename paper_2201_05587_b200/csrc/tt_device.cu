@@ -425,7 +425,8 @@ tt_status tt_workload_status(tt_workload* w, void* cuda_stream) {
     return read_status(w, static_cast<cudaStream_t>(cuda_stream));
 }
 
-tt_status tt_run_host(tt_workload* w, const tt_tensors* host, void* cuda_stream, int64_t* bytes_h2d, int64_t* bytes_d2h) {
+static tt_status run_host_impl(tt_workload* w, const tt_tensors* host, void* cuda_stream, int64_t* bytes_h2d, int64_t* bytes_d2h,
+                               bool synchronise) {
     if (!w || !host) return TT_ERR_INVALID_ARG;
     if (!w->plan.applied) return TT_ERR_NOT_APPLIED;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -452,10 +453,18 @@ tt_status tt_run_host(tt_workload* w, const tt_tensors* host, void* cuda_stream,
     if (s != TT_OK) return s;
     const size_t ybytes = tensor_elems(w, 4) * 4;
     if (cudaMemcpyAsync(host->y, w->hbuf[4], ybytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
-    s = read_status(w, st);
+    if (synchronise) s = read_status(w, st);
     if (bytes_h2d) *bytes_h2d = up;
     if (bytes_d2h) *bytes_d2h = (int64_t)ybytes;
     return s;
+}
+
+tt_status tt_run_host(tt_workload* w, const tt_tensors* host, void* cuda_stream, int64_t* bytes_h2d, int64_t* bytes_d2h) {
+    return run_host_impl(w, host, cuda_stream, bytes_h2d, bytes_d2h, true);
+}
+
+tt_status tt_run_host_async(tt_workload* w, const tt_tensors* host, void* cuda_stream, int64_t* bytes_h2d, int64_t* bytes_d2h) {
+    return run_host_impl(w, host, cuda_stream, bytes_h2d, bytes_d2h, false);
 }
 
 tt_status tt_time(tt_workload* w, const tt_tensors* sets, size_t n_sets, void* cuda_stream, const tt_timing_opts* o,

@@ -262,6 +262,31 @@ def test_run_host_matches_oracle():
     assert util.rel_l2(y.numpy(), util.oracle_ref(spec, a)) <= util.TOL_TF32
 
 
+def test_run_host_async_on_several_streams_matches_oracle():
+    """tt_run_host_async: several workloads enqueued on different streams (each workload always on its own), twice
+    each, nothing synchronised in between; after tt_workload_status every output equals the oracle's."""
+    import torch
+    specs = [W._conv(16, 14, 32, 3, 1, 1), W._dw(24, 28, 1), W._dense(8, 96, 40), W._conv(32, 14, 64, 1, 1, 0)]
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    jobs = []
+    for i, spec in enumerate(specs):
+        a = W.make_inputs(spec, 60 + i)
+        wl = spec.workload()
+        wl.apply(wl.default_schedule())
+        host = {k: (None if v is None else torch.from_numpy(v).pin_memory()) for k, v in a.items()}
+        y = torch.full(W.tensor_shapes(spec)[4], float("nan"), dtype=torch.float32).pin_memory()
+        jobs.append((spec, a, wl, host, y, streams[i % len(streams)]))
+    torch.cuda.synchronize()
+    for _ in range(2):
+        for spec, a, wl, host, y, st in jobs:
+            up, down = wl.run_host_async(B.tensors(host["x"], host["w"], host["bias"], None, y), st)
+            assert down == 4 * y.numel() and up > 0
+    for spec, a, wl, host, y, st in jobs:
+        assert wl.status(st) == B.TT_OK                  # synchronises that workload's stream
+        assert util.rel_l2(y.numpy(), util.oracle_ref(spec, a)) <= util.tolerance(spec.op), spec.name
+        wl.close()
+
+
 def test_timing_and_grid_tuner_smoke():
     spec = W._conv(32, 14, 64, 3, 1, 1)
     a = W.make_inputs(spec, 39)
