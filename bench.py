@@ -186,6 +186,14 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
         (conv(32, 256, 56, 64, 1, 0), "hbm",
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=2),
           tc(tile_n=64, tile_k=32, stages=2, mma_m_axis=2, slab_tiles=1), tc(tile_n=64, tile_k=32, stages=3, mma_m_axis=2, slab_tiles=1)]),
+        # batch_matmul at BERT-base head shapes, 3072 = 12 heads x 256 sequences: scores (NT) and context (NN)
+        (W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(3072, 128, 128, 64, True), 1, "bmm_nt_3072x128x128x64", "bert"), "hbm",
+         [tc(tile_n=128, tile_k=64, stages=1, mma_m_axis=1), tc(tile_n=128, tile_k=64, stages=1, mma_m_axis=2),
+          tc(tile_n=128, tile_k=32, stages=2, mma_m_axis=1)]),
+        (W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(3072, 128, 64, 128, False), 1, "bmm_nn_3072x128x64x128", "bert"), "hbm",
+         [tc(tile_n=64, tile_k=128, stages=1, mma_m_axis=1), tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=1)]),
+        (W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(64, 1024, 1024, 1024, True), 1, "bmm_nt_64x1024x1024x1024", "bert"), "tensor",
+         [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=4, mma_m_axis=1)]),
         (dw(64, 144, 56, 1), "hbm",
          [dwr(tile_m=4, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=2),
           dwr(tile_m=16, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=128, unroll=2),
