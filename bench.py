@@ -53,25 +53,32 @@ class ClockSampler(threading.Thread):
     def __init__(self, index):
         super().__init__(daemon=True)
         self.index, self.samples, self.reasons, self.max_mhz, self.stop_flag = index, [], set(), None, False
-
-    def run(self):
-        try:
+        self.nv = self.h = None
+        try:                                             # NVML is opened here, before the timed region starts
             import pynvml as nv
             nv.nvmlInit()
-            h = nv.nvmlDeviceGetHandleByIndex(self.index)
-            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            self.nv, self.h = nv, nv.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(self.h, nv.NVML_CLOCK_SM)
+        except Exception as e:  # NVML missing: report that, do not fail the bench
+            self.reasons.add(f"nvml_unavailable:{type(e).__name__}")
+
+    def run(self):
+        nv, h = self.nv, self.h
+        if nv is None:
+            return
+        try:
             names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
                      nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
                      nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
                      nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
-            while not self.stop_flag:
+            while not self.stop_flag:                    # the timed region lasts a few milliseconds: sample densely
                 self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
                 mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
                 for bit, name in names.items():
                     if mask & bit:
                         self.reasons.add(name)
-                time.sleep(0.05)
-        except Exception as e:  # NVML missing: report that, do not fail the bench
+                time.sleep(0.0005)
+        except Exception as e:
             self.reasons.add(f"nvml_unavailable:{type(e).__name__}")
 
     def summary(self):
@@ -247,7 +254,7 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--model", default="resnet18", choices=["resnet18", "resnet50", "mobilenet_v2", "bert_base", "bert_base_256"])
@@ -355,8 +362,6 @@ def main():
     torch.cuda.synchronize()
     torch.cuda.nvtx.range_pop()
     replicas.barrier()
-    sampler.stop_flag = True
-    sampler.join(timeout=2)
     for w in wls:
         st = w.status()
         if st != B.TT_OK:
@@ -397,6 +402,8 @@ def main():
     e2e_ms = timed_steps(e2e_steps, e2e_pass)
     replicas.barrier()
     e2e_value, _ = replicas.aggregate(flops_pass * e2e_steps / 1e12, e2e_ms * 1e-3, dev)
+    sampler.stop_flag = True                             # clocks were sampled over both timed regions (device-resident and end to end)
+    sampler.join(timeout=2)
     for i, (w, (h, ht)) in enumerate(zip(wls, host_sets)):
         st = w.status(side[i % len(side)])
         if st != B.TT_OK:
