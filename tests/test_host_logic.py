@@ -366,3 +366,51 @@ def test_refine_rejects_bad_arguments_and_needs_a_device_for_device_times():
         assert B.lib().tt_refine(wl.handle, ctypes.byref(t), None, None, ctypes.byref(rec), 2, 0.0, ctypes.byref(best),
                                  ctypes.byref(us), None, None) == B.TT_ERR_CUDA      # no CPU fallback
     wl.close()
+
+
+def test_depthwise_tma_records_are_legalised_by_shape():
+    """raster = 1 names the TMA-staged persistent depthwise kernel: kept where image rows are 16-byte multiples and the
+    filter is one the window kernels cover, with 2..4 staging buffers that fit shared memory; legalised away elsewhere
+    (strict mode: invalid)."""
+    rec = B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=8, block_y=14, block_x=56, items_per_thread=4, vec_width=4, threads=256,
+                        unroll=2, raster=1, stages=3)
+    ok = W._dw(144, 56, 1).workload()                     # 56-pixel rows: 224 bytes
+    st, info = ok.check(rec)
+    assert st == B.TT_OK and info.legal.raster == 1 and info.legal.stages == 3 and info.grid_y == 1
+    assert 0 < info.smem_bytes <= 227 * 1024 and info.grid_x <= 148 * 8
+    assert ok.check(rec, mode=B.TT_MODE_STRICT)[0] == B.TT_OK
+    deep = B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=8, block_y=14, block_x=56, items_per_thread=4, vec_width=4, threads=256,
+                         unroll=2, raster=1, stages=9)
+    st, info = ok.check(deep)
+    assert st == B.TT_OK and info.legal.raster == 1 and info.legal.stages == 4 and info.changed & B.TT_CHG_STAGES
+    assert ok.check(deep, mode=B.TT_MODE_STRICT)[0] == B.TT_ERR_INVALID_SCHEDULE
+    odd = W._dw(96, 14, 1).workload()                     # 14-pixel rows: 56 bytes, no aligned TMA rows
+    st, info = odd.check(rec)
+    assert st == B.TT_OK and info.legal.raster == 0 and info.changed & B.TT_CHG_BLOCK
+    assert odd.check(rec, mode=B.TT_MODE_STRICT)[0] == B.TT_ERR_INVALID_SCHEDULE
+    staged = B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=8, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=256,
+                           unroll=0, raster=1, stages=2)  # unroll 0 asks for the staged kernel: no TMA form of it
+    st, info = ok.check(staged)
+    assert st == B.TT_OK and info.legal.raster == 0
+    bad = B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=8, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=256,
+                        unroll=2, raster=2, stages=2)
+    assert ok.check(bad)[0] == B.TT_ERR_INVALID_SCHEDULE
+    for w in (ok, odd):
+        w.close()
+
+
+def test_pointwise_convolutions_take_the_whole_row_view():
+    """A 1x1, stride-1, unpadded convolution is legalised on rows that tile the CTA's pixels exactly: less shared
+    memory than the same record needs on a 3x3 layer's slab geometry would suggest, and never more than the image-row
+    view of a layer whose pixel count has no suitable divisor."""
+    rec = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=64, tile_k=32, stages=2, mma_m_axis=2, slab_tiles=1)
+    pw = W._conv(256, 56, 64, 1, 1, 0).workload()         # 3136 pixels = 49 rows of 64
+    st, info = pw.check(rec)
+    assert st == B.TT_OK and info.smem_bytes <= 90 * 1024
+    strided = W._conv(256, 56, 64, 1, 2, 0).workload()    # stride 2: the image's own rows
+    st2, info2 = strided.check(rec)
+    assert st2 == B.TT_OK
+    v = pw.gemm_view()
+    assert (v.gm, v.gn, v.gk) == (64, 3136, 256)          # the view changes nothing the caller sees
+    for w in (pw, strided):
+        w.close()
