@@ -109,6 +109,12 @@ def cpu_baseline_oracle(specs, arrays, budget_s, threads=0):
     return flops, secs, used, names
 
 
+def workload_name(model, specs, pool_sources):
+    """The workload both arms report: model shape, kernel counts and where the schedule pool comes from."""
+    return (f"{model}-shaped inference, batch 1, fp32 NCHW, {len(specs)} unique kernels / "
+            f"{sum(sp.use_count for sp in specs)} per pass, pool from {','.join(pool_sources)}-shaped kernels")
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle, rank 0 only, on bounded samples of the same workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -131,7 +137,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": secs / max(args.steps, 1) * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"{args.model}-shaped inference, batch 1, fp32, pool from {','.join(W.POOL_SOURCES[args.model])}"},
+            "config": {"workload": workload_name(args.model, specs, tuple(p for p in args.pool.split(",") if p) or W.POOL_SOURCES[args.model])},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -476,8 +482,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "tf32",
             "data": "synthetic",
-            "config": {"workload": f"{args.model}-shaped inference, batch 1, fp32 NCHW, {len(specs)} unique kernels / "
-                                   f"{sum(use)} per pass, pool from {','.join(pool_sources)}-shaped kernels",
+            "config": {"workload": workload_name(args.model, specs, pool_sources),
                        "l2": "flushed between steps (256 MB write)", "replay": "one CUDA graph per model pass",
                        "multi_gpu": "independent replicas"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bytes_up, "d2h_bytes_per_step": bytes_down,
