@@ -136,17 +136,60 @@ def test_conv_linearity_and_residual():
     np.testing.assert_allclose(yr, np.maximum(ya + res, 0).astype(np.float32), atol=1e-6)
 
 
-@pytest.mark.parametrize("stride", [1, 2])
-def test_depthwise_equals_block_diagonal_full_conv(stride):
+def test_conv_residual_with_stride_and_asymmetric_padding():
+    """The residual has the OUTPUT's shape and is added before the activation, also when stride > 1 and the two
+    paddings differ (an index error between the strided output and the residual shows here, not at stride 1)."""
+    x = inputs.uniform((2, 3, 9, 7), 24, 0)
+    w = inputs.uniform((4, 3, 3, 2), 24, 1)
+    b = inputs.uniform((4,), 24, 2)
+    for stride, pad in (((2, 2), (1, 1)), ((2, 1), (0, 1)), ((1, 2), (2, 0))):
+        pre = im2col_conv(x, w, b, stride, pad)
+        res = inputs.uniform(pre.shape, 24, 3)
+        y = orc.conv2d(x, w, b, stride=stride, pad=pad, residual=res, act=orc.ACT_RELU)
+        np.testing.assert_allclose(y, np.maximum(pre + res, 0).astype(np.float32), rtol=0, atol=1e-6)
+
+
+def window_products_dw(x, w, bias, stride, pad):
+    """Depthwise convolution through a formulation that shares nothing with the loops of the oracle: explicit zero
+    padding, then one strided view of the padded image per filter tap, multiplied by that tap and summed in fp64."""
+    x = x.astype(np.float64)
+    n, c, h, wd = x.shape
+    r, s = w.shape[2], w.shape[3]
+    xp = np.zeros((n, c, h + 2 * pad[0], wd + 2 * pad[1]))
+    xp[:, :, pad[0]:pad[0] + h, pad[1]:pad[1] + wd] = x
+    p = (h + 2 * pad[0] - r) // stride[0] + 1
+    q = (wd + 2 * pad[1] - s) // stride[1] + 1
+    y = np.zeros((n, c, p, q))
+    for ri in range(r):
+        for si in range(s):
+            view = xp[:, :, ri:ri + stride[0] * (p - 1) + 1:stride[0], si:si + stride[1] * (q - 1) + 1:stride[1]]
+            y += view * w[:, 0, ri, si].astype(np.float64)[None, :, None, None]
+    if bias is not None:
+        y += bias.astype(np.float64)[None, :, None, None]
+    return y
+
+
+@pytest.mark.parametrize("stride", [(1, 1), (2, 2), (1, 2), (2, 1)])
+@pytest.mark.parametrize("pad", [(1, 1), (1, 0), (0, 2), (2, 2)])
+@pytest.mark.parametrize("rs", [(3, 3), (5, 5), (3, 5)])
+def test_depthwise_brute_force_and_block_diagonal_full_conv(stride, pad, rs):
+    """Depthwise against (a) the tap-by-tap window products above and (b) the full convolution with block-diagonal
+    weights, over asymmetric strides, paddings and filters: a swapped stride or padding axis, or a slip that only a
+    5-wide filter shows, fails here."""
     c = 4
-    x = inputs.uniform((2, c, 7, 6), 19, 0)
-    w = inputs.uniform((c, 1, 3, 3), 19, 1)
+    x = inputs.uniform((2, c, 9, 8), 19, 0)
+    w = inputs.uniform((c, 1) + rs, 19, 1)
     b = inputs.uniform((c,), 19, 2)
-    y = orc.dwconv2d(x, w, b, stride=(stride, stride), pad=(1, 1), act=orc.ACT_RELU6)
-    full = np.zeros((c, c, 3, 3), np.float32)
+    if 9 + 2 * pad[0] < rs[0] or 8 + 2 * pad[1] < rs[1]:
+        pytest.skip("filter larger than padded input")
+    y = orc.dwconv2d(x, w, b, stride=stride, pad=pad, act=orc.ACT_RELU6)
+    pre = window_products_dw(x, w, b, stride, pad)
+    assert y.shape == pre.shape
+    np.testing.assert_allclose(y, np.clip(pre, 0.0, 6.0).astype(np.float32), rtol=0, atol=1e-6)
+    full = np.zeros((c, c) + rs, np.float32)
     for i in range(c):
         full[i, i] = w[i, 0]
-    ref = orc.conv2d(x, full, b, stride=(stride, stride), pad=(1, 1), act=orc.ACT_RELU6)
+    ref = orc.conv2d(x, full, b, stride=stride, pad=pad, act=orc.ACT_RELU6)
     np.testing.assert_array_equal(y, ref)
 
 
