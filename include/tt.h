@@ -153,7 +153,8 @@ typedef struct tt_apply_info {
 } tt_apply_info;
 
 enum { TT_CHG_TILE_M = 1, TT_CHG_TILE_N = 2, TT_CHG_TILE_K = 4, TT_CHG_STAGES = 8, TT_CHG_SPLIT_K = 16,
-       TT_CHG_VEC = 32, TT_CHG_BLOCK = 64, TT_CHG_ITEMS = 128, TT_CHG_SLAB = 256, TT_CHG_ACC = 512, TT_CHG_KORDER = 1024 };
+       TT_CHG_VEC = 32, TT_CHG_BLOCK = 64, TT_CHG_ITEMS = 128, TT_CHG_SLAB = 256, TT_CHG_ACC = 512, TT_CHG_KORDER = 1024,
+       TT_CHG_FORM = 2048   /* the record named a kernel form this shape does not have (DW_SIMT unroll / raster) */ };
 
 /* Validity modes for mapping a record onto another shape (Section 4.1).
  *   TT_MODE_LEGALISE  reformulate: clamp/round tile sizes to the new extents and the hardware's legal set,
@@ -239,8 +240,20 @@ tt_status tt_run_host(tt_workload* w, const tt_tensors* host, void* cuda_stream,
  * of that stream).  A workload owns one set of device staging buffers: enqueue its calls on one stream at a time. */
 tt_status tt_run_host_async(tt_workload* w, const tt_tensors* host, void* cuda_stream, int64_t* bytes_h2d,
                             int64_t* bytes_d2h);
-/* Read and clear the device status word of the last runs (TT_OK or TT_ERR_TIMEOUT); synchronises the stream. */
+/* Read and clear the device status word of the last runs (TT_OK or TT_ERR_TIMEOUT); synchronises the stream.
+ * After a TT_ERR_TIMEOUT the split-K arrival counters of the applied record are cleared too, so the next run starts
+ * from a clean workspace (an invalid pair is a result of the search, which then goes on: Section 4.3). */
 tt_status tt_workload_status(tt_workload* w, void* cuda_stream);
+/* Every wait inside a kernel (on a copy, on a pipeline buffer, on the accumulator) gives up after this many
+ * nanoseconds: the kernel then records TT_ERR_TIMEOUT in the status word, lets its copies land, releases its tensor
+ * memory and returns, and the context stays usable.  Default: one second.  Takes effect with the next run. */
+tt_status tt_workload_set_wait_limit(tt_workload* w, uint64_t nanoseconds);
+/* Test facility for that path.  With extra_bytes > 0 (a multiple of 16) the barrier of the first pipeline stage of a
+ * GEMM_TC kernel whose operands arrive by TMA is told to expect extra_bytes more than its copies deliver (in the CTAs
+ * of the first reduction split only, so that a split-K record is left half finished): every copy still lands, only
+ * the barrier never completes, so the wait on it runs into the limit above.  0 switches it off.
+ * Nothing traps and nothing waits without a limit. */
+tt_status tt_workload_test_stall(tt_workload* w, uint32_t extra_bytes);
 
 /* Time the applied record: warm-up batches, then `batches` batches of back-to-back launches between two CUDA
  * events.  `sets` holds n_sets tensor sets used round-robin (n_sets > 1 with a footprint beyond L2 gives cold-cache
@@ -323,9 +336,12 @@ tt_status tt_refine(tt_workload* w, const tt_tensors* t, void* cuda_stream, cons
  *   the caller; `rec` is a GEMM_TC record (legalised as in tt_schedule_apply); act is a tt_act.
  *   scratch_bytes_used (may be NULL) receives what the legalised record needs of the array.
  * Errors: TT_ERR_RESOURCE when that exceeds TT_STATIC_SCRATCH_BYTES (lower split_k, or use tt_run, which
- * allocates); the statuses of tt_schedule_apply for a bad record; TT_ERR_CUDA; TT_ERR_TIMEOUT from the kernel.
- * The call launches on `cuda_stream` and synchronises it before returning.  The first call on a device looks up
- * the array's address (with that device current); make that first call outside any stream capture.
+ * allocates) or when the record's split-K cluster cannot be resident; the statuses of tt_schedule_apply for a bad
+ * record; TT_ERR_CUDA; TT_ERR_TIMEOUT from the kernel.
+ * The call launches on `cuda_stream`, synchronises it and reads the status word back before returning, so it cannot
+ * be part of a stream capture.  The first call on a device loads the library's device image (which is when the
+ * driver sets the array aside) and looks up the array's address, with that device current: make that first call at
+ * start-up, before the application declares its allocation phase over.
  * All calls share the array: it keeps the previous call's contents (the words that must start at zero are cleared
  * on the stream before each launch), and two calls that overlap on the GPU race on it -- issue them one at a
  * time per device. */

@@ -258,7 +258,7 @@ def rank_pools(target_share, candidate_counts):
     return scores, order
 
 
-# ---- refining a transferred schedule (Section 7: "vary parameters from schedules transfer-tuned from another model") ----
+# ---- refining a transferred schedule (named as future work in Section 7): local search over a record's fields ----
 # The paper names the idea only; the reading taken here: each parameter has an ordered ladder of values, a step moves
 # one parameter to the next lower or next higher rung, and the search is a greedy descent over those steps.
 LADDERS = {

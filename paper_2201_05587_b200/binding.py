@@ -21,8 +21,8 @@ TT_ACT_NONE, TT_ACT_RELU, TT_ACT_RELU6, TT_ACT_GELU_ERF = range(4)
 TT_FAMILY_GEMM_TC, TT_FAMILY_DW_SIMT, TT_FAMILY_ROW_SIMT = range(3)
 TT_MODE_LEGALISE, TT_MODE_STRICT = 0, 1
 TT_RECORD_VERSION = 1
-TT_CHG_TILE_M, TT_CHG_TILE_N, TT_CHG_TILE_K, TT_CHG_STAGES, TT_CHG_SPLIT_K, TT_CHG_VEC, TT_CHG_BLOCK, TT_CHG_ITEMS, TT_CHG_SLAB, TT_CHG_ACC, TT_CHG_KORDER = \
-    1, 2, 4, 8, 16, 32, 64, 128, 256, 512, 1024
+TT_CHG_TILE_M, TT_CHG_TILE_N, TT_CHG_TILE_K, TT_CHG_STAGES, TT_CHG_SPLIT_K, TT_CHG_VEC, TT_CHG_BLOCK, TT_CHG_ITEMS, TT_CHG_SLAB, TT_CHG_ACC, TT_CHG_KORDER, TT_CHG_FORM = \
+    1, 2, 4, 8, 16, 32, 64, 128, 256, 512, 1024, 2048
 
 i32, u32, f32 = C.c_int32, C.c_uint32, C.c_float
 
@@ -109,6 +109,8 @@ EXPORTS = {
     "tt_run_host": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "tt_run_host_async": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "tt_workload_status": (i32, [C.c_void_p, C.c_void_p]),
+    "tt_workload_set_wait_limit": (i32, [C.c_void_p, C.c_uint64]),
+    "tt_workload_test_stall": (i32, [C.c_void_p, C.c_uint32]),
     "tt_time": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_size_t, C.c_void_p, C.POINTER(tt_timing_opts),
                       C.POINTER(tt_timing)]),
     "tt_select": (i32, [C.POINTER(f32), C.c_size_t, C.c_size_t, C.POINTER(i32)]),
@@ -331,6 +333,12 @@ class Workload:
     def status(self, stream=None) -> int:
         sp = _stream() if stream is None else C.c_void_p(stream.cuda_stream)
         return lib().tt_workload_status(self.handle, sp)
+
+    def set_wait_limit(self, nanoseconds: int):
+        _check(lib().tt_workload_set_wait_limit(self.handle, int(nanoseconds)), "tt_workload_set_wait_limit")
+
+    def test_stall(self, extra_bytes: int):
+        _check(lib().tt_workload_test_stall(self.handle, int(extra_bytes)), "tt_workload_test_stall")
 
     def time(self, sets, opts: tt_timing_opts | None = None) -> tt_timing:
         if isinstance(sets, tt_tensors):

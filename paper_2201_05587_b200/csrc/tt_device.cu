@@ -230,6 +230,8 @@ tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
             (g.residual && (reinterpret_cast<uintptr_t>(g.residual) & 15u) != 0)) g.vec_store = 0;
         if (g.bias && (reinterpret_cast<uintptr_t>(g.bias) & 15u) == 0) g.vec_store |= 2;
         g.ktab_dev = w->ktab_dev;
+        g.wait_ns = w->wait_ns;
+        g.extra_tx = w->extra_tx;
         e = launch_gemm(p.info, g, maps->a, maps->b, maps->x, st);
     } else if (w->family == TT_FAMILY_DW_SIMT) {
         DwArgs d = p.dw;
@@ -253,6 +255,7 @@ tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
                 maps = &w->tmaps.back();
             }
             d.status = w->status_word;
+            d.wait_ns = w->wait_ns;
             e = launch_dw_tma(p.info, d, maps->x, st);
         } else
         e = launch_dw(p.info, d, st);
@@ -273,6 +276,11 @@ static tt_status read_status(tt_workload* w, cudaStream_t st) {
     if (cudaMemcpy(&v, w->status_word, 4, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
     if (v != 0) {
         cudaMemset(w->status_word, 0, 4);
+        // A CTA that gave up never reported at its tile's arrival counter: the counters of a workspace split-K record
+        // are no longer all zero, and the next run would finish tiles from incomplete partial sums.  Clear them.
+        const Plan& p = w->plan;
+        if (w->family == TT_FAMILY_GEMM_TC && w->workspace && !p.repack && p.info.workspace_bytes > p.partial_bytes)
+            cudaMemset(static_cast<char*>(w->workspace) + p.partial_bytes, 0, (size_t)(p.info.workspace_bytes - p.partial_bytes));
         return (tt_status)(v & 0xffu);
     }
     return TT_OK;
@@ -409,16 +417,18 @@ tt_status tt_schedule_apply_ex(tt_workload* w, const tt_schedule_record* rec, in
 
 tt_status tt_run(tt_workload* w, const tt_tensors* t, void* cuda_stream) { return launch(w, t, cuda_stream); }
 
-#ifdef TT_PHASE_TIMERS
-// Diagnostic build only: copy the 10 phase stamps (global timer ns, SM clock) of the last GEMM launch.
-tt_status tt_debug_read_timers(tt_workload* w, unsigned long long* out50) {
-    if (!w || !w->status_word || !out50) return TT_ERR_INVALID_ARG;
-    cudaDeviceSynchronize();
-    const bool ok = cudaMemcpy(out50, reinterpret_cast<char*>(w->status_word) + 16, 60 * 8, cudaMemcpyDeviceToHost) == cudaSuccess;
-    cudaMemset(reinterpret_cast<char*>(w->status_word) + 16, 0, 60 * 8);      // the next launch starts from cleared stamps
-    return ok ? TT_OK : TT_ERR_CUDA;
+
+tt_status tt_workload_set_wait_limit(tt_workload* w, uint64_t nanoseconds) {
+    if (!w || nanoseconds == 0) return TT_ERR_INVALID_ARG;
+    w->wait_ns = nanoseconds;
+    return TT_OK;
 }
-#endif
+
+tt_status tt_workload_test_stall(tt_workload* w, uint32_t extra_bytes) {
+    if (!w || (extra_bytes & 15u)) return TT_ERR_INVALID_ARG;
+    w->extra_tx = extra_bytes;
+    return TT_OK;
+}
 
 tt_status tt_workload_status(tt_workload* w, void* cuda_stream) {
     if (!w) return TT_ERR_INVALID_ARG;
@@ -697,6 +707,7 @@ static __device__ __align__(256) unsigned char g_tt_static_scratch[TT_STATIC_SCR
 namespace tt {
 namespace {
 constexpr int kMaxDevices = 64;
+constexpr int64_t kStaticStatusBytes = 512;   // the status area, sized like the one tt_schedule_apply allocates
 unsigned char* g_scratch_addr[kMaxDevices] = {};
 
 // In host code the array's name only stands for the symbol; the device address is asked for once per device,
@@ -735,14 +746,20 @@ extern "C" tt_status tt_dense_static_scratch(const void* x, const void* w, const
     if (s != TT_OK) return s;
     // layout of the fixed array: status word | arrival counters | partial sums
     const int64_t counters_bytes = ((int64_t)plan.info.grid_x * plan.info.grid_z * 4 + 255) / 256 * 256;
-    const int64_t need = 256 + counters_bytes + (plan.g.split_k > 1 ? plan.partial_bytes : 0);
+    const int64_t need = kStaticStatusBytes + counters_bytes + (plan.g.split_k > 1 ? plan.partial_bytes : 0);
     if (scratch_bytes_used) *scratch_bytes_used = need;
     if (need > (int64_t)TT_STATIC_SCRATCH_BYTES) return TT_ERR_RESOURCE;   // this record's partial sums do not fit
+    if (plan.g.cluster) {
+        // as in tt_schedule_apply: a split-K cluster whose CTAs cannot be resident together is an invalid pair
+        int fits = 0;
+        if (gemm_cluster_fits(plan.info.smem_bytes, plan.g.cluster, &fits) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+        if (!fits) return TT_ERR_RESOURCE;
+    }
     unsigned char* base = nullptr;
     if ((s = static_scratch(&base)) != TT_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     // the array keeps what the previous call left: the status word and the counters must start at zero
-    if (cudaMemsetAsync(base, 0, (size_t)(256 + counters_bytes), st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+    if (cudaMemsetAsync(base, 0, (size_t)(kStaticStatusBytes + counters_bytes), st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
     GemmArgs g = plan.g;
     const void* tens[2] = {x, w};
     const void* a_ptr = tens[plan.a_tensor];
@@ -753,8 +770,10 @@ extern "C" tt_status tt_dense_static_scratch(const void* x, const void* w, const
     g.bias = static_cast<const float*>(bias);
     g.residual = nullptr;
     g.status = reinterpret_cast<unsigned*>(base);
-    g.counters = reinterpret_cast<unsigned*>(base + 256);
-    g.partial = reinterpret_cast<float*>(base + 256 + counters_bytes);
+    g.counters = reinterpret_cast<unsigned*>(base + kStaticStatusBytes);
+    g.partial = reinterpret_cast<float*>(base + kStaticStatusBytes + counters_bytes);
+    g.wait_ns = 1000000000ull;
+    g.extra_tx = 0;
     if ((reinterpret_cast<uintptr_t>(y) & 15u) != 0) g.vec_store = 0;
     if (g.bias && (reinterpret_cast<uintptr_t>(g.bias) & 15u) == 0) g.vec_store |= 2;
     TmapPair maps;

@@ -461,6 +461,9 @@ static tt_status legalise_dw(const tt_workload* w, const tt_schedule_record* rec
         if (items == 8 && window_rows > 2) window_rows = 2;
     }
     L.unroll = window_rows;
+    // a record that names the register-window form (or a strip height it does not have) on a filter without one runs
+    // another kernel form than it was written for: a reformulation, invalid when nothing may be reformulated
+    if (window_rows != rec->unroll) changed |= TT_CHG_FORM;
     int bx = std::min(rec->block_x, round_up(w->Q, items));
     bx = round_up(bx, items);
     if (bx != rec->block_x || L.block_y != rec->block_y) changed |= TT_CHG_BLOCK;
@@ -526,7 +529,7 @@ static tt_status legalise_dw(const tt_workload* w, const tt_schedule_record* rec
             return TT_OK;
         }
     }
-    if (rec->raster != 0) { if (strict) return TT_ERR_INVALID_SCHEDULE; I.changed |= TT_CHG_BLOCK; }
+    if (rec->raster != 0) { if (strict) return TT_ERR_INVALID_SCHEDULE; I.changed |= TT_CHG_FORM; }
     I.legal = L;
     I.grid_x = (int)std::min<long long>(gx, 0x7fffffff); I.grid_y = s.n; I.grid_z = 1;
     I.threads = th; I.smem_bytes = (int)std::min<long long>(smem, 0x7fffffff);
@@ -726,8 +729,8 @@ tt_status tt_schedule_check(const tt_workload* w, const tt_schedule_record* rec,
     return st;
 }
 
-// ---- refinement of a transferred record (Section 7, future work: "vary parameters from schedules transfer-tuned
-// from another model") ----
+// ---- refinement of a transferred record (named as future work in Section 7): a local search over the fields of a
+// record that another model's tuning produced ----
 namespace {
 struct FieldLadder { int32_t tt_schedule_record::*field; std::vector<int> steps; };   // two steps = a toggle when both differ
 

@@ -68,7 +68,9 @@ struct GemmArgs {
     unsigned pm_off, pm_buf_bytes; int pm_nbuf; // tap-major convolutions: the pixel-major slab buffers (one or two)
     int tap_major;                              // 1: OPM_IM2COL_T on operand B
     int Pout;                                   // output rows (padded-linear pixel -> (p, q'))
-    const int* ktab_dev;                        // per reduction index: byte offset of (c, r, s) inside the slab (absolute channel)      // ceil(2^32 / d) for the exact small-range divisions of the slab loader
+    const int* ktab_dev;                        // per reduction index: byte offset of (c, r, s) inside the slab (absolute channel)
+    unsigned long long wait_ns;                 // limit of every bounded wait inside the kernel
+    unsigned extra_tx;                          // test facility: bytes added to what the first stage's barrier expects
 };
 
 struct DwArgs {
@@ -84,6 +86,7 @@ struct DwArgs {
     int box_w, stage_bytes, tiles_p, total_tiles;   // box width in floats (multiple of 4), bytes per buffer (multiple of 128)
     int wstage_bytes;  // bytes per filter-and-bias buffer (one per box buffer, multiple of 128)
     unsigned* status;  // the workload's status word (bounded waits)
+    unsigned long long wait_ns;   // limit of every bounded wait inside the kernel
 };
 
 struct RowArgs {
@@ -128,6 +131,8 @@ struct tt_workload {
     size_t ktab_bytes = 0;
     size_t workspace_bytes = 0;
     unsigned* status_word = nullptr;  // device
+    unsigned long long wait_ns = 1000000000ull;   // one second per wait inside a kernel, then the kernel gives up
+    unsigned extra_tx = 0;            // test facility (tt_workload_test_stall)
     // device staging buffers of tt_run_host
     void* hbuf[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     size_t hbytes[5] = {0, 0, 0, 0, 0};

@@ -55,33 +55,18 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     return t;
 }
 
-constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second per wait, then give up
 
-// Diagnostic build only (-DTT_PHASE_TIMERS): CTA (0,0,0) stamps the global timer and the SM clock at the phase
-// boundaries of the GEMM kernel into the 64-bit slots that follow the status word.
-#ifdef TT_PHASE_TIMERS
-__device__ unsigned long long* g_tt_dbg = nullptr;       // set by CTA (0,0,0) before its first barrier
-__device__ __forceinline__ void tt_stamp(int slot) {
-    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && g_tt_dbg) {
-        g_tt_dbg[2 * slot] = global_timer_ns();
-        g_tt_dbg[2 * slot + 1] = (unsigned long long)clock64();
-    }
-}
-#define TT_STAMP(slot) tt_stamp(slot)
-#else
-#define TT_STAMP(slot) do { } while (0)
-#endif
 
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one expired).
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
-                                            unsigned where) {
+                                            unsigned where, unsigned long long limit_ns) {
     const unsigned long long t0 = global_timer_ns();
     unsigned spins = 0;
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 31u) == 0u) {
             if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
+            if (global_timer_ns() - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicCAS(status, 0u, (unsigned)TT_ERR_TIMEOUT | (where << 8));
                 return false;
@@ -91,9 +76,9 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
 }
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
-                                          unsigned where) {
+                                          unsigned where, unsigned long long limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;         // the common case costs one instruction
-    return mbar_wait_slow(bar, parity, abort_flag, status, where);
+    return mbar_wait_slow(bar, parity, abort_flag, status, where, limit_ns);
 }
 
 // Programmatic dependent launch.  A kernel launched with programmatic stream serialization may become resident while
@@ -717,23 +702,10 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // keeps the role loops (addresses, descriptors, counters) on the uniform datapath
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     volatile int* abortp = &abort_flag;
-#ifdef TT_PHASE_TIMERS
-    if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
-        g_tt_dbg = reinterpret_cast<unsigned long long*>(g.status) + 2;
-#endif
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel of the stream may begin its set-up
     // A CTA's shared memory may be written by a peer only once the CTA runs: every thread announces itself here and
     // checks, much later and just before the first remote store could happen, that all peers have done the same.
     if (g.cluster) cluster_arrive();
-    if (threadIdx.x == 0) TT_STAMP(0);
-#ifdef TT_PHASE_TIMERS
-    // span of the whole grid: latest CTA start and latest CTA end (earliest start = ~min kept as max of the complement)
-    if (threadIdx.x == 0) {
-        unsigned long long* d = reinterpret_cast<unsigned long long*>(g.status) + 2;
-        atomicMax(d + 56, ~global_timer_ns());
-        atomicMax(d + 58, global_timer_ns());
-    }
-#endif
 
     // tile coordinates
     int tm, tn;
@@ -809,7 +781,6 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // kernel that follows this one was allowed to start its own set-up at this kernel's entry.  (Without the launch
     // attribute both instructions do nothing.)
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (threadIdx.x == 0) TT_STAMP(1);
 
     // Warps 0 and 1 run their loops with all 32 lanes: waits, counters and descriptor arithmetic stay
     // warp-uniform, and one elected lane issues the asynchronous instructions.
@@ -850,18 +821,19 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (slab_issued < ic_chunks) {
                         // its buffer is free once the gather warps have left chunk slab_issued - 2
                         const int j = slab_issued;
-                        const bool freed = tapm ? mbar_wait(smem_u32(&slab_empty[0]), (uint32_t)(j - 1) & 1u, abortp, g.status, 5u)
-                                                : mbar_wait(smem_u32(&slab_empty[j & 1]), (uint32_t)((j - 2) >> 1) & 1u, abortp, g.status, 5u);
+                        const bool freed = tapm ? mbar_wait(smem_u32(&slab_empty[0]), (uint32_t)(j - 1) & 1u, abortp, g.status, 5u, g.wait_ns)
+                                                : mbar_wait(smem_u32(&slab_empty[j & 1]), (uint32_t)((j - 2) >> 1) & 1u, abortp, g.status, 5u, g.wait_ns);
                         if (!__all_sync(0xffffffffu, freed)) { ok = false; break; }
                         if (leader) issue_chunk(j);
                         ++slab_issued;
                     }
                 }
                 if (!any_tma) continue;
-                const bool got = mbar_wait(empty_addr, ph ^ 1u, abortp, g.status, 1u);
+                const bool got = mbar_wait(empty_addr, ph ^ 1u, abortp, g.status, 1u, g.wait_ns);
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 if (leader) {
-                    mbar_expect_tx(full_addr, g.tx_bytes);
+                    // (test facility: split 0 may be told to expect more than arrives, see tt_workload_test_stall)
+                    mbar_expect_tx(full_addr, g.tx_bytes + ((it == 0 && split == 0) ? g.extra_tx : 0u));
                     if (a_tma) {
                         uint32_t dst = a_stage;
                         int kc = k0;
@@ -877,8 +849,6 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
                 __syncwarp();
                 armed = it + 1;
-                if (lane == 0 && it == 5) TT_STAMP(10);
-                if (lane == 0 && it == 6) TT_STAMP(11);
                 a_stage += stage_bytes; full_addr += 8u; empty_addr += 8u;
                 if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; a_stage = tiles_base; full_addr = full0; empty_addr = empty0; }
             }
@@ -932,14 +902,9 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 const int lin0 = (n0 - ic_p_first * g.slab_wp) + g.slab_gap - g.pw;
                 int chunk = 0, tap = 0, fr = 0, fs = 0;
                 for (int it = 0; it < iters; ++it) {
-                    bool got = mbar_wait(full_addr, ph, abortp, g.status, 2u);                       // the filter tile
-                    if (tap == 0) got = mbar_wait(smem_u32(&pm_full[chunk & 1]), (uint32_t)(chunk >> 1) & 1u, abortp, g.status, 7u) && got;
+                    bool got = mbar_wait(full_addr, ph, abortp, g.status, 2u, g.wait_ns);                       // the filter tile
+                    if (tap == 0) got = mbar_wait(smem_u32(&pm_full[chunk & 1]), (uint32_t)(chunk >> 1) & 1u, abortp, g.status, 7u, g.wait_ns) && got;
                     if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-                    if (lane == 0 && it == 0) TT_STAMP(2);
-                    if (lane == 0 && it == 14) TT_STAMP(12);
-                    if (lane == 0 && it == 15) TT_STAMP(13);
-                    if (lane == 0 && it == 18) TT_STAMP(10);
-                    if (lane == 0 && it == 27) TT_STAMP(11);
                     tc_fence_after();
                     if (leader) {
                         // the stage holds n_atoms taps of this channel block, one 128 x 32 filter atom each
@@ -964,11 +929,8 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             } else
             for (int it = 0; it < iters; ++it) {
-                const bool got = mbar_wait(full_addr, ph, abortp, g.status, 2u);
+                const bool got = mbar_wait(full_addr, ph, abortp, g.status, 2u, g.wait_ns);
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-                if (lane == 0 && it == 0) TT_STAMP(2);
-                if (lane == 0 && it == 5) TT_STAMP(12);
-                if (lane == 0 && it == 6) TT_STAMP(13);
                 tc_fence_after();
                 if (leader) {
                     // descriptors step by 2 (32 bytes = 8 TF32 along K) inside a swizzle atom, then to the next atom
@@ -999,13 +961,11 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     mma_commit(empty_addr);              // stage reusable once these MMAs have read it
                 }
                 __syncwarp();
-                if (lane == 0 && it == 5) TT_STAMP(14);
                 a_stage += stage_step; b_stage += stage_step; full_addr += 8u; empty_addr += 8u;
                 if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; a_stage = a_lo0; b_stage = b_lo0; full_addr = full0; empty_addr = empty0; }
             }
             if (ok && leader) mma_commit(smem_u32(&accum_bar));    // accumulator complete
             __syncwarp();
-            if (lane == 0) TT_STAMP(3);
         }
         if (g.cluster) cluster_wait();
     } else {
@@ -1059,7 +1019,6 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     st_shared_v4(slab0 + o, 0.f, 0.f, 0.f, 0.f);
             }
             bool ok = gather_vote(true);                 // row table and zeros are in place (the k-table may still be in flight)
-            if (threadIdx.x == 64) TT_STAMP(17);
             const int n_chunks = ic_chunks;
             const ExpandPlan xplan = make_expand_plan(rows, rowoff, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, gw, lane);   // after the vote: reads s_rowoff
             auto chunk_first_channel = [&](int j) { return (kbeg + j * T * g.tile_k) / RS; };
@@ -1077,12 +1036,11 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 chunk_load(0);
                 if (n_chunks > 1) chunk_load(1);
             }
-            if (threadIdx.x == 64) TT_STAMP(18);
             const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
             uint32_t st = 0, ph = 0;
             for (int j = 0; j < n_chunks; ++j) {
                 if (slab_tma) {
-                    if (ok && !mbar_wait(smem_u32(&slab_full[j & 1]), (uint32_t)(j >> 1) & 1u, abortp, g.status, 6u)) ok = false;
+                    if (ok && !mbar_wait(smem_u32(&slab_full[j & 1]), (uint32_t)(j >> 1) & 1u, abortp, g.status, 6u, g.wait_ns)) ok = false;
                     if (j == 0) {
                         cp_async_wait<0>();              // the k-table copies of this thread ...
                         ok = gather_vote(ok);            // ... and of every other gather thread have landed
@@ -1093,18 +1051,15 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     ok = gather_vote(ok);                // every thread's copies of chunk j are visible to all
                     if (!ok) break;
                 }
-                if (threadIdx.x == 64 && j == 0) TT_STAMP(15);
                 // table offsets count channels from 0: rebase the buffer by the chunk's first channel
                 const uint32_t slab = slab0 + (uint32_t)(j & 1) * g.slab_buf_bytes - 4u * (uint32_t)(chunk_first_channel(j) * g.slab_chpitch);
                 const int it_end = min((j + 1) * T, iters);
                 for (int it = j * T; it < it_end; ++it) {
-                    if (ok && !mbar_wait(empty0 + st * 8u, ph ^ 1u, abortp, g.status, 3u)) ok = false;
+                    if (ok && !mbar_wait(empty0 + st * 8u, ph ^ 1u, abortp, g.status, 3u, g.wait_ns)) ok = false;
                     if (ok) {
                         const uint32_t a_s = tiles_base + st * stage_bytes, b_s = a_s + g.a_stage_bytes;
                         const uint32_t kt = ktab + 4u * (uint32_t)(it * g.tile_k);
-                        if (threadIdx.x == 64 && it == 5) TT_STAMP(22);
                         expand_stage(xplan, on_a ? a_s : b_s, rows, slab, rowoff, kt, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, gw, lane);
-                        if (threadIdx.x == 64 && it == 5) TT_STAMP(23);
                         if (o_gather) {
                             const int k0 = (kt_begin + it) * g.tile_k;
                             if (on_a) gather_stage(g.b_mode, b_s, g.tile_n, o_src, g.b_rs, g.b_ks, n0, g.N, k0, g.K, g.tile_k,
@@ -1115,9 +1070,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         fence_proxy_async_shared();      // generic-proxy stores -> visible to the tensor core's reads
                         __syncwarp();
                         if (lane == 0) mbar_arrive(full0 + st * 8u);
-                        if (threadIdx.x == 64 && it == 5) TT_STAMP(24);
                     }
-                    if (threadIdx.x == 64 && it == 4) TT_STAMP(9);
                     if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
                 }
                 if (slab_tma) {
@@ -1131,7 +1084,6 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             }
             cp_async_wait<0>();
-            if (threadIdx.x == 64) TT_STAMP(16);
         } else if (tapm) {
             // ---- conv2d, tap-major: transpose every 32-channel block of input rows, once, into a pixel-major slab ----
             // staging buffer (TMA): [32 channels][in_rows][wp] floats; pixel-major slab: one 128-byte row per staged
@@ -1148,10 +1100,8 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const uint32_t ch_bytes = 4u * (uint32_t)g.slab_chpitch;
             for (int j = 0; j < ic_chunks; ++j) {
                 const int b = j & 1;                     // pixel-major buffer; the staging buffer is always the same one
-                if (ok && !mbar_wait(smem_u32(&slab_full[0]), (uint32_t)j & 1u, abortp, g.status, 6u)) ok = false;
-                if (threadIdx.x == 64 && j == 1) TT_STAMP(15);
-                if (threadIdx.x == 64 && j == 2) TT_STAMP(22);
-                if (ok && j >= 2 && !mbar_wait(smem_u32(&pm_empty[b]), (uint32_t)((j - 2) >> 1) & 1u, abortp, g.status, 8u)) ok = false;
+                if (ok && !mbar_wait(smem_u32(&slab_full[0]), (uint32_t)j & 1u, abortp, g.status, 6u, g.wait_ns)) ok = false;
+                if (ok && j >= 2 && !mbar_wait(smem_u32(&pm_empty[b]), (uint32_t)((j - 2) >> 1) & 1u, abortp, g.status, 8u, g.wait_ns)) ok = false;
                 if (ok) {
                     // warp gw moves channels 4 gw .. 4 gw + 3 of every staged position; lanes walk positions
                     const uint32_t src = st0 + (uint32_t)(4 * gw) * ch_bytes;
@@ -1178,8 +1128,6 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                     fence_proxy_async_shared();          // generic-proxy stores -> visible to the tensor core's reads
                     __syncwarp();
-                    if (threadIdx.x == 64 && j == 1) TT_STAMP(16);
-                    if (threadIdx.x == 64 && j == 2) TT_STAMP(23);
                     if (lane == 0) {
                         mbar_arrive(smem_u32(&pm_full[b]));
                         if (j + 1 < ic_chunks) mbar_arrive(smem_u32(&slab_empty[0]));   // the staging buffer may be refilled
@@ -1194,7 +1142,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             int st = grp % g.stages;
             uint32_t ph = (uint32_t)(grp / g.stages) & 1u;
             for (int it = grp; it < iters; it += n_groups) {
-                if (!mbar_wait(empty0 + (uint32_t)st * 8u, ph ^ 1u, abortp, g.status, 3u)) break;
+                if (!mbar_wait(empty0 + (uint32_t)st * 8u, ph ^ 1u, abortp, g.status, 3u, g.wait_ns)) break;
                 const uint32_t a_s = tiles_base + (uint32_t)st * stage_bytes, b_s = a_s + g.a_stage_bytes;
                 const int k0 = (kt_begin + it) * g.tile_k;
                 if (!a_tma) gather_stage(g.a_mode, a_s, kHwTileM, a_src, g.a_rs, g.a_ks, m0, g.M, k0, g.K, g.tile_k,
@@ -1210,7 +1158,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         // epilogue: warp w owns tensor-memory lanes 32*(w % 4) .. +31; the two warps of a lane quadrant take
         // alternate 32-column blocks
-        const bool have_acc = mbar_wait(smem_u32(&accum_bar), 0u, abortp, g.status, 4u);
+        const bool have_acc = mbar_wait(smem_u32(&accum_bar), 0u, abortp, g.status, 4u, g.wait_ns);
         // every epilogue thread takes the same decision (named barrier 1 over the epilogue threads); the barrier
         // also orders the bias staging above against its readers below
         uint32_t all_acc;
@@ -1220,7 +1168,6 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             "bar.red.and.pred p, 1, %2, q;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(all_acc) : "r"((uint32_t)have_acc), "n"(kGatherThreads) : "memory");
-        if (threadIdx.x == 64) TT_STAMP(4);
         if (g.cluster) cluster_wait();                   // every peer is running: its reduction area may be written
         if (all_acc) {
             tc_fence_after();
@@ -1337,7 +1284,6 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         // read-out is software-pipelined: the next block's tensor-memory load is in flight while
                         // this block is biased, activated and stored
                         tmem_wait_ld();
-                        if (threadIdx.x == 64 && c0 == 0) TT_STAMP(7);
 #pragma unroll
                         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
 #pragma unroll 1
@@ -1389,7 +1335,6 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         if (full) epilogue_block<true, true>(v, e, m_first, nb, cnt, stg, lane, transposed);
                         else epilogue_block<false, true>(v, e, m_first, nb, cnt, stg, lane, transposed);
                     }
-                    if (threadIdx.x == 64 && c0 == 0) TT_STAMP(8);
                 }
             }
         }
@@ -1398,9 +1343,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         // ---------------- split-K over the cluster: add up the bands the peers sent ----------------
         // Every thread of every CTA of the cluster takes part in the barrier, also after a tripped wait.  After it
         // nobody writes to or reads from another CTA's shared memory any more, so no second barrier is needed.
-        if (threadIdx.x == 64) TT_STAMP(19);
         cluster_sync_all();                              // all bands have arrived
-        if (threadIdx.x == 64) TT_STAMP(20);
         if (warp >= 2) {
             const int gw = warp - 2;
             const int sk = g.split_k;
@@ -1465,9 +1408,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                 n0 + split * per + cl, min(4, r_end - lane * 4));
             }
         }
-        if (threadIdx.x == 64) TT_STAMP(21);
     }
-    if (threadIdx.x == 64) TT_STAMP(5);
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -1475,10 +1416,6 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         tc_fence_after();
         tmem_dealloc(tmem_base, g.tmem_cols);
     }
-    if (threadIdx.x == 0) TT_STAMP(6);
-#ifdef TT_PHASE_TIMERS
-    if (threadIdx.x == 0) atomicMax(reinterpret_cast<unsigned long long*>(g.status) + 2 + 57, global_timer_ns());
-#endif
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -1788,7 +1725,7 @@ __global__ void __launch_bounds__(256) tt_dwconv_tma_kernel(const __grid_constan
     uint32_t ph = 0;
     for (int i = 0; i < my_tiles; ++i) {
         // every thread waits for the box itself (all take the same decision: the same barrier and phase)
-        if (!mbar_wait(smem_u32(&full_bar[s]), ph, abortp, d.status, 9u)) break;
+        if (!mbar_wait(smem_u32(&full_bar[s]), ph, abortp, d.status, 9u, d.wait_ns)) break;
         const int pl0 = cur.tp * d.tile_c, p0 = cur.th * d.tile_h, q0 = cur.tw * d.tile_w;
         const int ncl = min(d.tile_c, planes - pl0);
         const uint32_t stage = base + (uint32_t)s * (uint32_t)d.stage_bytes;

@@ -414,3 +414,32 @@ def test_pointwise_convolutions_take_the_whole_row_view():
     assert (v.gm, v.gn, v.gk) == (64, 3136, 256)          # the view changes nothing the caller sees
     for w in (pw, strided):
         w.close()
+
+
+def test_depthwise_record_naming_a_kernel_form_the_shape_lacks_is_a_reformulation():
+    """A register-window (unroll >= 1) or TMA-staged (raster = 1) depthwise record on a filter that has no such kernel
+    runs the staged kernel instead: legalise mode says so in `changed`, strict mode rejects the record (a primitive
+    that does not fit the loop nest is invalid code, Sections 4.1 and 4.2)."""
+    dw7 = B.Workload(B.TT_OP_DWCONV2D, B.make_shapes(n=1, c=8, h=20, w=20, k=8, r=7, s=7, stride_h=1, stride_w=1, pad_h=3,
+                                                     pad_w=3, has_bias=1, act=B.TT_ACT_RELU), "dw7x7")
+    dw3s3 = B.Workload(B.TT_OP_DWCONV2D, B.make_shapes(n=1, c=8, h=20, w=20, k=8, r=3, s=3, stride_h=3, stride_w=3, pad_h=1,
+                                                       pad_w=1, has_bias=1, act=B.TT_ACT_RELU), "dw3x3s3")
+    dw3 = B.Workload(B.TT_OP_DWCONV2D, B.make_shapes(n=1, c=8, h=20, w=20, k=8, r=3, s=3, stride_h=1, stride_w=1, pad_h=1,
+                                                     pad_w=1, has_bias=1, act=B.TT_ACT_RELU), "dw3x3")
+    win = B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=4, block_y=4, block_x=20, items_per_thread=4, vec_width=4, threads=128, unroll=2)
+    for wl in (dw7, dw3s3):
+        st, info = wl.check(win)
+        assert st == B.TT_OK and info.legal.unroll == 0 and info.changed & B.TT_CHG_FORM
+        assert wl.check(win, mode=B.TT_MODE_STRICT)[0] == B.TT_ERR_INVALID_SCHEDULE
+    st, info = dw3.check(win)
+    assert st == B.TT_OK and info.legal.unroll == 2 and not info.changed & B.TT_CHG_FORM
+    assert dw3.check(win, mode=B.TT_MODE_STRICT)[0] == B.TT_OK
+    three = B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=4, block_y=4, block_x=20, items_per_thread=4, vec_width=4, threads=128, unroll=3)
+    st, info = dw3.check(three)
+    assert st == B.TT_OK and info.legal.unroll == 2 and info.changed & B.TT_CHG_FORM
+    assert dw3.check(three, mode=B.TT_MODE_STRICT)[0] == B.TT_ERR_INVALID_SCHEDULE
+    tma = B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=4, block_y=4, block_x=20, items_per_thread=4, vec_width=4, threads=256,
+                        unroll=2, raster=1, stages=2)
+    st, info = dw7.check(tma)
+    assert st == B.TT_OK and info.legal.raster == 0 and info.changed & B.TT_CHG_FORM
+    assert dw3.check(tma)[1].legal.raster == 1

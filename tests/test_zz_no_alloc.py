@@ -53,6 +53,28 @@ def test_static_scratch_matches_allocating_path_twice_in_a_row():
     _both_paths(W._dense(96, 1500, 200, act=B.TT_ACT_RELU, name="static_a"), rec, seed=43)
 
 
+def test_static_scratch_cluster_split_and_no_allocation_between_calls():
+    """Two to eight splits reduce inside a thread-block cluster: the fixed array then only holds the status word and
+    the counters.  And the point of the entry point: the device's free memory is the same before and after calls
+    (the first call on a device may load the library's image; the later ones must not change anything)."""
+    import torch
+    rec4 = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=64, tile_k=32, stages=3, split_k=4, mma_m_axis=1)
+    _both_paths(W._dense(96, 1500, 200, act=B.TT_ACT_RELU, name="static_cluster4"), rec4, seed=44)
+    spec = W._dense(64, 1024, 256, act=B.TT_ACT_NONE, name="static_free_mem")
+    a = W.make_inputs(spec, 45)
+    t, _ = W.device_tensors(spec, a)
+    y = torch.empty_like(t["y"])
+    rec12 = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=64, tile_k=32, stages=3, split_k=12, mma_m_axis=1)
+    assert B.dense_static_scratch(t["x"], t["w"], t["bias"], y, spec.shapes.act, rec12)[0] == B.TT_OK
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for rec in (rec12, rec4, rec12):
+        assert B.dense_static_scratch(t["x"], t["w"], t["bias"], y, spec.shapes.act, rec)[0] == B.TT_OK
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert util.rel_l2(y.cpu().numpy(), util.oracle_ref(spec, a)) <= util.TOL_TF32
+
+
 def test_static_scratch_rejects_what_does_not_fit():
     import torch
     # 2048 x 2048 outputs x 16 splits x 4 bytes = 256 MB of partial sums: far beyond the fixed array
