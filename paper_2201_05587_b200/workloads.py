@@ -1,13 +1,21 @@
-"""Workload inventories shaped like the paper's models, and seeded inputs for them.
+"""Workload inventories shaped like the paper's models, their data-flow chains, and seeded inputs for them.
 
 The paper evaluates ImageNet CNNs and BERT (Section 5.1); a schedule depends only on
 the operator and the data sizes of a kernel (Section 2), never on weight values, so
 each model is represented by the list of its unique kernels (operator, sizes, use
 count) with synthetic tensors.  No dataset item or trained weight is involved.
 
-Kernel classes follow Table 1: conv2d_add (class A: 1x1 stride-2 downsample, no
-activation), conv2d_bias_relu (class E), dense_add (class D).  Residual-add variants
-(class F/G/K) share the shape of their class-E sibling and are counted with it.
+Kernel classes follow Tables 1 and 2: conv2d_add (class A: 1x1 downsample or projection,
+no activation), conv2d_bias_relu (class E), conv2d_bias_add_relu (classes F and G: the
+last convolution of a residual block, skip tensor added before the ReLU),
+conv2d_bias_add (class K: MobileNetV2 projection with a skip), depthwise (class L),
+dense_add (class D).  A model is written down once, as the ordered list of its layers
+with their wiring (which layer's output each layer reads, which one it adds as a
+skip); the unique-kernel inventory and its use counts are derived from that list, so
+the two always agree.  Pooling, layer normalisation and the reshapes between
+attention heads are outside the hot path (about 0 % of inference time, Table 2): where one
+would sit the chain reads a seeded tensor of the right shape (pools) or reinterprets
+the producer's buffer (head reshapes), and says so in the step.
 """
 from __future__ import annotations
 
@@ -30,9 +38,9 @@ class Spec:
         return B.Workload(self.op, self.shapes, self.name, self.use_count)
 
 
-def _conv(c, hw, k, r, stride, pad, act=B.TT_ACT_RELU, use=1, name=None, bias=True):
-    nm = name or f"conv{r}x{r}s{stride}_{c}x{hw}->{k}"
-    return Spec(B.TT_OP_CONV2D, B.conv2d_shapes(1, c, hw, hw, k, r, r, stride, pad, bias, act), use, nm)
+def _conv(c, hw, k, r, stride, pad, act=B.TT_ACT_RELU, use=1, name=None, bias=True, residual=False):
+    nm = name or f"conv{r}x{r}s{stride}_{c}x{hw}->{k}" + ("+res" if residual else "")
+    return Spec(B.TT_OP_CONV2D, B.conv2d_shapes(1, c, hw, hw, k, r, r, stride, pad, bias, act, residual), use, nm)
 
 
 def _dw(c, hw, stride, r=3, act=B.TT_ACT_RELU6, use=1):
@@ -53,8 +61,48 @@ def _dedup(specs):
         if key in seen:
             seen[key].use_count += sp.use_count
         else:
-            seen[key] = sp
+            seen[key] = Spec(sp.op, sp.shapes, sp.use_count, sp.name, sp.init)
     return list(seen.values())
+
+
+class Step:
+    """One node of a model in execution order: a layer (spec is its kernel), or, with spec None, a seeded tensor of
+    `shape` that enters the chain from outside the hot path (the model's input, or the stand-in for the output of an
+    operator that is not part of it, named in `note`).  x / res / w_from: index of the node whose buffer this layer
+    reads as its input / adds as its skip tensor / (batch_matmul) takes as second operand.  A producer's buffer is
+    read with the consumer's shape (same number of elements): that is how the head reshapes of the attention block
+    are represented."""
+
+    def __init__(self, spec, x=None, res=None, note="", shape=None):
+        self.spec, self.x, self.res, self.note, self.shape = spec, x, res, note, shape
+        self.w_from = None        # batch_matmul only; None = the layer's own seeded second operand
+        self.kernel = -1          # index into the unique-kernel inventory, filled by Net.finish
+
+    def out_shape(self):
+        return tuple(self.shape) if self.spec is None else tuple(tensor_shapes(self.spec)[4])
+
+
+class Net:
+    """A model as an ordered list of wired nodes; the inventory of unique kernels is derived from it."""
+
+    def __init__(self):
+        self.steps = []
+
+    def external(self, shape, note):
+        self.steps.append(Step(None, shape=tuple(shape), note=note))
+        return len(self.steps) - 1
+
+    def add(self, spec, x, res=None, note=""):
+        self.steps.append(Step(spec, x, res, note))
+        return len(self.steps) - 1
+
+    def finish(self):
+        specs = _dedup([st.spec for st in self.steps if st.spec is not None])
+        index = {(sp.op, bytes(sp.shapes)): i for i, sp in enumerate(specs)}
+        for st in self.steps:
+            if st.spec is not None:
+                st.kernel = index[(st.spec.op, bytes(st.spec.shapes))]
+        return specs, self.steps
 
 
 def single_conv():
@@ -75,41 +123,57 @@ def single_conv_pool():
     return recs
 
 
-def resnet18():
-    """Table 1 (classes A, E+F merged per shape, D): 12 unique kernels."""
-    specs = [_conv(3, 224, 64, 7, 2, 3, name="stem7x7s2_3x224->64")]
+def resnet18_net():
+    """Table 1: classes A (3 kernels), E (8), F (4), D (1) = 16 unique kernels, 21 uses."""
+    net = Net()
+    net.add(_conv(3, 224, 64, 7, 2, 3, name="stem7x7s2_3x224->64"), x=net.external((1, 3, 224, 224), "the image"))
+    cur = net.external((1, 64, 56, 56), "stands in for the max-pool's output")
     ch, hw = 64, 56
     for stage, k in enumerate((64, 128, 256, 512)):
-        if stage > 0:
-            specs.append(_conv(ch, hw, k, 3, 2, 1))                                     # first 3x3, strided
-            specs.append(_conv(ch, hw, k, 1, 2, 0, act=B.TT_ACT_NONE))                  # downsample (class A)
-            hw //= 2
-            specs.append(_conv(k, hw, k, 3, 1, 1, use=3))
-        else:
-            specs.append(_conv(ch, hw, k, 3, 1, 1, use=4))
-        ch = k
-    specs.append(_dense(1, 512, 1000))
-    return _dedup(specs)
+        for block in range(2):
+            if stage > 0 and block == 0:
+                c1 = net.add(_conv(ch, hw, k, 3, 2, 1), x=cur)                                   # first 3x3, strided
+                skip = net.add(_conv(ch, hw, k, 1, 2, 0, act=B.TT_ACT_NONE), x=cur)               # downsample (class A)
+                hw //= 2
+            else:
+                c1 = net.add(_conv(k, hw, k, 3, 1, 1), x=cur)
+                skip = cur
+            cur = net.add(_conv(k, hw, k, 3, 1, 1, residual=True), x=c1, res=skip)               # class F
+            ch = k
+    net.add(_dense(1, 512, 1000), x=net.external((1, 512), "stands in for the global average pool's output"))
+    return net.finish()
 
 
-def resnet50():
-    """Bottleneck 1x1 / 3x3 / 1x1 kernels (stride on the 3x3), 1x1 downsamples, the 2048->1000 dense layer."""
-    specs = [_conv(3, 224, 64, 7, 2, 3, name="stem7x7s2_3x224->64")]
+def resnet50_net():
+    """Bottleneck 1x1 / 3x3 / 1x1 kernels (stride on the 3x3; the expanding 1x1 adds the skip: class G), 1x1
+    downsamples (class A), the 2048->1000 dense layer.  Table 2: E 16, G 4, A 4, D 1."""
+    net = Net()
+    net.add(_conv(3, 224, 64, 7, 2, 3, name="stem7x7s2_3x224->64"), x=net.external((1, 3, 224, 224), "the image"))
+    cur = net.external((1, 64, 56, 56), "stands in for the max-pool's output")
     in_ch, hw = 64, 56
     for stage, (mid, blocks) in enumerate(((64, 3), (128, 4), (256, 6), (512, 3))):
         out_ch = mid * 4
         stride = 1 if stage == 0 else 2
         for b in range(blocks):
             s = stride if b == 0 else 1
-            specs.append(_conv(in_ch, hw, mid, 1, 1, 0))                                # reduce
-            specs.append(_conv(mid, hw, mid, 3, s, 1))                                  # 3x3
+            r1 = net.add(_conv(in_ch, hw, mid, 1, 1, 0), x=cur)                                  # reduce
+            m3 = net.add(_conv(mid, hw, mid, 3, s, 1), x=r1)                                     # 3x3
+            skip = cur
             if b == 0:
-                specs.append(_conv(in_ch, hw, out_ch, 1, s, 0, act=B.TT_ACT_NONE))      # downsample
+                skip = net.add(_conv(in_ch, hw, out_ch, 1, s, 0, act=B.TT_ACT_NONE), x=cur)      # downsample
             hw2 = hw // s
-            specs.append(_conv(mid, hw2, out_ch, 1, 1, 0))                              # expand (+residual in-model)
+            cur = net.add(_conv(mid, hw2, out_ch, 1, 1, 0, residual=True), x=m3, res=skip)       # expand + skip
             in_ch, hw = out_ch, hw2
-    specs.append(_dense(1, 2048, 1000))
-    return _dedup(specs)
+    net.add(_dense(1, 2048, 1000), x=net.external((1, 2048), "stands in for the global average pool's output"))
+    return net.finish()
+
+
+def resnet18():
+    return resnet18_net()[0]
+
+
+def resnet50():
+    return resnet50_net()[0]
 
 
 def vgg16():
@@ -127,22 +191,32 @@ def vgg16():
 _MBV2 = ((1, 16, 1, 1), (6, 24, 2, 2), (6, 32, 3, 2), (6, 64, 4, 2), (6, 96, 3, 1), (6, 160, 3, 2), (6, 320, 1, 1))
 
 
-def mobilenet_v2():
-    specs = [_conv(3, 224, 32, 3, 2, 1, act=B.TT_ACT_RELU6, name="stem3x3s2_3x224->32")]
+def mobilenet_v2_net():
+    """Table 2: J 8 (stem, six expansions, last 1x1: +ReLU6), L 10 (depthwise), A 7 (projection), K 5 (projection that
+    adds the block's input), D 1."""
+    net = Net()
+    cur = net.add(_conv(3, 224, 32, 3, 2, 1, act=B.TT_ACT_RELU6, name="stem3x3s2_3x224->32"),
+                  x=net.external((1, 3, 224, 224), "the image"))
     ch, hw = 32, 112
     for t, c, n, s in _MBV2:
         for i in range(n):
             stride = s if i == 0 else 1
             hid = ch * t
+            h = cur
             if t != 1:
-                specs.append(_conv(ch, hw, hid, 1, 1, 0, act=B.TT_ACT_RELU6))           # expand
-            specs.append(_dw(hid, hw, stride))
+                h = net.add(_conv(ch, hw, hid, 1, 1, 0, act=B.TT_ACT_RELU6), x=cur)              # expand
+            d = net.add(_dw(hid, hw, stride), x=h)
             hw //= stride
-            specs.append(_conv(hid, hw, c, 1, 1, 0, act=B.TT_ACT_NONE))                 # project
+            skip = stride == 1 and ch == c
+            cur = net.add(_conv(hid, hw, c, 1, 1, 0, act=B.TT_ACT_NONE, residual=skip), x=d, res=cur if skip else None)
             ch = c
-    specs.append(_conv(320, 7, 1280, 1, 1, 0, act=B.TT_ACT_RELU6))
-    specs.append(_dense(1, 1280, 1000))
-    return _dedup(specs)
+    net.add(_conv(320, 7, 1280, 1, 1, 0, act=B.TT_ACT_RELU6), x=cur)
+    net.add(_dense(1, 1280, 1000), x=net.external((1, 1280), "stands in for the global average pool's output"))
+    return net.finish()
+
+
+def mobilenet_v2():
+    return mobilenet_v2_net()[0]
 
 
 def efficientnet_b0_like():
@@ -166,16 +240,34 @@ def efficientnet_b0_like():
     return _dedup(specs)
 
 
-def bert_base(seq=128, hidden=768, heads=12, ffn=3072, layers=12):
+def bert_base_net(seq=128, hidden=768, heads=12, ffn=3072, layers=12):
+    """Encoder layers as the hot path sees them: three projections of the layer input, scores, softmax, context,
+    output projection, the two feed-forward layers.  The reshapes between [seq, hidden] and [heads, seq, hidden/heads]
+    are layout shuffles outside the hot path: a consumer reads the producer's buffer with its own shape.  Layer
+    normalisation and the skip additions around it are separate, negligible kernel classes (Table 2: 0 %)."""
     d = hidden // heads
-    return [
-        _dense(seq, hidden, hidden, use=4 * layers, init="bert", name=f"dense_{seq}x{hidden}->{hidden}"),
-        _dense(seq, hidden, ffn, act=B.TT_ACT_GELU_ERF, use=layers, init="bert", name=f"dense_gelu_{seq}x{hidden}->{ffn}"),
-        _dense(seq, ffn, hidden, use=layers, init="bert", name=f"dense_{seq}x{ffn}->{hidden}"),
-        Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(heads, seq, seq, d, True), layers, "bmm_qk_nt", "bert"),
-        Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(heads, seq, d, seq, False), layers, "bmm_pv_nn", "bert"),
-        Spec(B.TT_OP_SOFTMAX, B.softmax_shapes(heads, seq, seq, 1.0 / math.sqrt(d)), layers, "softmax", "bert"),
-    ]
+    proj = lambda: _dense(seq, hidden, hidden, init="bert", name=f"dense_{seq}x{hidden}->{hidden}")
+    net = Net()
+    cur = net.external((seq, hidden), "the embedded tokens")
+    for _ in range(layers):
+        q = net.add(proj(), x=cur)
+        k = net.add(proj(), x=cur)
+        v = net.add(proj(), x=cur)
+        sc = net.add(Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(heads, seq, seq, d, True), 1, "bmm_qk_nt", "bert"), x=q, res=None,
+                     note="w = the key projection's buffer")
+        net.steps[sc].w_from = k
+        pr = net.add(Spec(B.TT_OP_SOFTMAX, B.softmax_shapes(heads, seq, seq, 1.0 / math.sqrt(d)), 1, "softmax", "bert"), x=sc)
+        cx = net.add(Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(heads, seq, d, seq, False), 1, "bmm_pv_nn", "bert"), x=pr,
+                     note="w = the value projection's buffer")
+        net.steps[cx].w_from = v
+        o = net.add(proj(), x=cx)
+        f1 = net.add(_dense(seq, hidden, ffn, act=B.TT_ACT_GELU_ERF, init="bert", name=f"dense_gelu_{seq}x{hidden}->{ffn}"), x=o)
+        cur = net.add(_dense(seq, ffn, hidden, init="bert", name=f"dense_{seq}x{ffn}->{hidden}"), x=f1)
+    return net.finish()
+
+
+def bert_base(seq=128):
+    return bert_base_net(seq=seq)[0]
 
 
 def bert_base_256():
@@ -187,6 +279,12 @@ MODELS = {
     "single_conv": single_conv, "resnet18": resnet18, "resnet50": resnet50, "vgg16": vgg16,
     "mobilenet_v2": mobilenet_v2, "efficientnet_b0_like": efficientnet_b0_like, "bert_base": bert_base,
     "bert_base_256": bert_base_256,
+}
+
+# model -> (unique kernels, wired layers in execution order)
+CHAINS = {
+    "resnet18": resnet18_net, "resnet50": resnet50_net, "mobilenet_v2": mobilenet_v2_net, "bert_base": bert_base_net,
+    "bert_base_256": lambda: bert_base_net(seq=256),
 }
 
 # target model -> models whose natively tuned records form its schedule pool
@@ -259,3 +357,46 @@ def device_tensors(spec: Spec, arrays, device="cuda"):
     t = {k: (None if v is None else torch.from_numpy(v).to(device)) for k, v in arrays.items()}
     t["y"] = torch.empty(tensor_shapes(spec)[4], dtype=torch.float32, device=device)
     return t, B.tensors(t["x"], t["w"], t["bias"], t["residual"], t["y"])
+
+
+def make_chain_inputs(steps, seed: int, init="he"):
+    """Seeded numpy tensors for every node of a chain: a layer's own weights and bias (and second batch_matmul
+    operand where that is not wired), an external node's tensor ("x": U[-1,1], or N(0,1) for init "bert")."""
+    out = []
+    for i, st in enumerate(steps):
+        if st.spec is None:
+            x = inputs.normal(st.shape, seed, 8 * (1000 + i)) if init == "bert" else inputs.uniform(st.shape, seed, 8 * (1000 + i))
+            out.append({"x": x, "w": None, "bias": None, "residual": None})
+            continue
+        a = make_inputs(st.spec, seed, 1000 + i)
+        a["x"] = None
+        if st.w_from is not None:
+            a["w"] = None
+        a["residual"] = None
+        out.append(a)
+    return out
+
+
+def chain_device_tensors(steps, arrays, device="cuda"):
+    """Wire a chain on the device: every layer writes its own output buffer, and reads its input, skip tensor and
+    (batch_matmul) second operand from the buffers of the nodes that produce them, viewed with its own shapes.
+    Returns (per-node dicts of torch tensors, with the node's buffer under "y"; per-node tt_tensors, None for
+    external nodes)."""
+    import torch
+    bufs, tts = [], []
+    for st, a in zip(steps, arrays):
+        if st.spec is None:
+            bufs.append({"y": torch.from_numpy(a["x"]).to(device)})
+            tts.append(None)
+            continue
+        xs, ws, bs, rs, ys = tensor_shapes(st.spec)
+        t = {k: (None if v is None else torch.from_numpy(v).to(device)) for k, v in a.items()}
+        t["x"] = bufs[st.x]["y"].view(xs)
+        if st.w_from is not None:
+            t["w"] = bufs[st.w_from]["y"].view(ws)
+        if st.res is not None:
+            t["residual"] = bufs[st.res]["y"].view(rs)
+        t["y"] = torch.empty(ys, dtype=torch.float32, device=device)
+        bufs.append(t)
+        tts.append(B.tensors(t["x"], t["w"], t["bias"], t["residual"], t["y"]))
+    return bufs, tts

@@ -649,3 +649,59 @@ def test_bounded_wait_expires_reports_timeout_and_the_workload_recovers():
         assert wl.status() == B.TT_OK
         assert util.rel_l2(t["y"].cpu().numpy(), ref) <= util.TOL_TF32
         wl.close()
+
+
+def _tf32_depth(steps):
+    """Per node: the number of TF32 layers on the longest path that leads to it (each may add the TF32 tolerance)."""
+    depth = []
+    for st in steps:
+        if st.spec is None:
+            depth.append(0)
+            continue
+        d = max([depth[i] for i in (st.x, st.res, st.w_from) if i is not None])
+        depth.append(d + (1 if st.spec.op in (B.TT_OP_CONV2D, B.TT_OP_DENSE, B.TT_OP_BATCH_MATMUL) else 0))
+    return depth
+
+
+@pytest.mark.parametrize("model,make,seed", [
+    ("resnet18", W.resnet18_net, 2),
+    ("mobilenet_v2", W.mobilenet_v2_net, 4),
+    ("resnet50", W.resnet50_net, 3),
+    ("bert_base_2_layers", lambda: W.bert_base_net(layers=2), 5),
+], ids=lambda v: v if isinstance(v, str) else "")
+def test_data_chained_model_pass_matches_the_oracle_chain(model, make, seed):
+    """The whole model as a chain: every layer reads the buffer its producer wrote (and the skip tensor of its block),
+    all launched back to back on one stream without synchronisation, three passes.  Every layer's output is compared
+    with the same chain on the oracle; a layer k TF32 layers deep may be off by k times the TF32 tolerance.  Run once
+    under the default records and once under a record that uses cluster split-K and the other accumulator axis."""
+    import torch
+    specs, steps = make()
+    arrays = W.make_chain_inputs(steps, seed, init="bert" if model.startswith("bert") else "he")
+    refs = util.oracle_chain(steps, arrays)
+    depth = _tf32_depth(steps)
+    alt = tc(tile_n=64, tile_k=32, stages=3, split_k=2, mma_m_axis=2)
+    for use_alt in (False, True):
+        wls = [sp.workload() for sp in specs]
+        for wl in wls:
+            rec = alt if use_alt and wl.family() == B.TT_FAMILY_GEMM_TC else wl.default_schedule()
+            wl.apply(rec)
+        bufs, tts = W.chain_device_tensors(steps, arrays)
+        for _ in range(3):
+            for st, b in zip(steps, bufs):
+                if st.spec is not None:
+                    b["y"].fill_(float("nan"))
+            for st, tt in zip(steps, tts):
+                if st.spec is not None:
+                    wls[st.kernel].run(tt)
+            torch.cuda.synchronize()
+        for wl in wls:
+            assert wl.status() == B.TT_OK
+        for i, (st, b, ref, d) in enumerate(zip(steps, bufs, refs, depth)):
+            if st.spec is None:
+                continue
+            y = b["y"].cpu().numpy()
+            assert not np.isnan(y).any(), (model, i, st.spec.name)
+            tol = max(d, 1) * util.TOL_TF32 if d else util.TOL_FP32
+            assert util.rel_l2(y, ref) <= tol, (model, i, st.spec.name, d, util.rel_l2(y, ref))
+        for wl in wls:
+            wl.close()

@@ -68,12 +68,8 @@ def test_resnet18_inventory_matches_table1():
                 i, cls, ic, ihw, oc, ohw, use = line.split()
                 rows.append((cls, int(ic), int(ihw), int(oc), int(ohw), int(use)))
     specs = W.resnet18()
-    assert len(specs) == 12
-    # merge the table's E and F rows per shape (residual variants share the shape), keep A and D
-    want = {}
-    for cls, ic, ihw, oc, ohw, use in rows:
-        kind = "A" if cls == "A" else ("D" if cls == "D" else "E")
-        want[(kind, ic, ihw, oc, ohw)] = want.get((kind, ic, ihw, oc, ohw), 0) + use
+    assert len(specs) == 16                               # A 3, E 8, F 4, D 1
+    want = {(cls, ic, ihw, oc, ohw): use for cls, ic, ihw, oc, ohw, use in rows}
     got = {}
     for sp in specs:
         s = sp.shapes
@@ -81,10 +77,38 @@ def test_resnet18_inventory_matches_table1():
             got[("D", s.kk, 1, s.nn, 1)] = sp.use_count
         else:
             p = (s.h + 2 * s.pad_h - s.r) // s.stride_h + 1
-            kind = "A" if (s.r == 1 and s.act == B.TT_ACT_NONE) else "E"
+            kind = "A" if (s.r == 1 and s.act == B.TT_ACT_NONE) else ("F" if s.has_residual else "E")
             got[(kind, s.c, s.h, s.k, p)] = sp.use_count
     assert got == want
     assert sum(sp.use_count for sp in specs) == 21          # 20 convolutions + 1 dense
+    # the residual variants are kernels of their own class and workload ID, although they share their sibling's sizes
+    e = [sp for sp in specs if sp.shapes.c == 64 and sp.shapes.k == 64 and sp.shapes.r == 3]
+    assert len(e) == 2 and e[0].workload().kernel_class() != e[1].workload().kernel_class()
+    assert e[0].workload().key() != e[1].workload().key()
+
+
+def test_chains_are_consistent_with_their_inventories():
+    """A model is written once as wired layers; the inventory is derived from it.  Every wire connects buffers of the
+    same element count, every skip tensor has the consumer's output shape, and the use counts are the layer counts."""
+    for name, make in W.CHAINS.items():
+        specs, steps = make()
+        assert [sp.use_count for sp in specs] == [sum(1 for st in steps if st.kernel == i) for i in range(len(specs))], name
+        for i, st in enumerate(steps):
+            if st.spec is None:
+                assert st.shape and st.note, (name, i)
+                continue
+            xs, ws, bs, rs, ys = W.tensor_shapes(st.spec)
+            assert bytes(specs[st.kernel].shapes) == bytes(st.spec.shapes)
+            assert 0 <= st.x < i and np.prod(steps[st.x].out_shape()) == np.prod(xs), (name, i)
+            if st.w_from is not None:
+                assert 0 <= st.w_from < i and np.prod(steps[st.w_from].out_shape()) == np.prod(ws), (name, i)
+            assert (st.res is not None) == bool(st.spec.shapes.has_residual), (name, i)
+            if st.res is not None:
+                assert 0 <= st.res < i and steps[st.res].out_shape() == tuple(ys), (name, i)
+    # the ResNet-18-shaped chain: a block's second convolution adds the block's input, or its 1x1 downsample
+    specs, steps = W.resnet18_net()
+    f = [st for st in steps if st.spec is not None and st.spec.shapes.has_residual]
+    assert len(f) == 8 and sum(1 for st in f if steps[st.res].spec is not None and steps[st.res].spec.shapes.r == 1) == 3
 
 
 def test_unique_kernel_counts_of_table2():
@@ -92,7 +116,8 @@ def test_unique_kernel_counts_of_table2():
     r50 = W.resnet50()
     convs = [s for s in r50 if s.op == B.TT_OP_CONV2D]
     down = [s for s in convs if s.shapes.act == B.TT_ACT_NONE]
-    assert len(down) == 4 and len(convs) - len(down) == 20 and len(r50) == 25    # 16 (E) + 4 (G) share code here
+    g = [s for s in convs if s.shapes.has_residual]
+    assert len(down) == 4 and len(g) == 4 and len(convs) - len(down) - len(g) == 16 and len(r50) == 25    # A, G, E
     vgg = W.vgg16()
     assert len([s for s in vgg if s.op == B.TT_OP_CONV2D]) == 9 and len(vgg) == 12
     mb = W.mobilenet_v2()
@@ -100,6 +125,7 @@ def test_unique_kernel_counts_of_table2():
     proj = [s for s in mb if s.op == B.TT_OP_CONV2D and s.shapes.act == B.TT_ACT_NONE]
     relu6 = [s for s in mb if s.op == B.TT_OP_CONV2D and s.shapes.act == B.TT_ACT_RELU6]
     assert (len(dw), len(proj), len(relu6)) == (10, 12, 8)
+    assert len([s for s in proj if s.shapes.has_residual]) == 5                 # class K; the other 7 are class A
     bert = W.bert_base()
     assert len([s for s in bert if s.op == B.TT_OP_DENSE]) == 3
     assert len([s for s in bert if s.op == B.TT_OP_BATCH_MATMUL]) == 2
@@ -208,7 +234,7 @@ def test_simt_legalisers():
     L = info.legal
     assert L.tile_m == 96 and L.block_y == 7 and L.vec_width == 1 and L.block_x % L.items_per_thread == 0
     assert dw.check(r, mode=B.TT_MODE_STRICT)[0] == B.TT_ERR_INVALID_SCHEDULE
-    sm = W.bert_base()[5].workload()
+    sm = [s for s in W.bert_base() if s.op == B.TT_OP_SOFTMAX][0].workload()
     st, info = sm.check(B.make_record(B.TT_FAMILY_ROW_SIMT, block_x=24, block_y=3, vec_width=4))
     assert st == B.TT_OK and info.legal.block_x == 16 and info.threads % 32 == 0 and info.legal.vec_width == 4
 
