@@ -1,18 +1,23 @@
 #!/usr/bin/env python
 """Benchmark of the transfer-tuning hot path on B200.
 
-One step = one pass over every kernel of the target model (use counts included), each run under the record the
-evaluator selected from a pool tuned on *other* models.  Before the timed region the pool is built (native grid
-tuning of the source models' kernels) and the evaluator runs every (kernel, record) pair; both are reported but
-not part of a step.  Prints ONE JSON line.
+One step = one data-chained pass over every layer of the target model (each layer reads the buffer its producer
+wrote; every layer has its own weights), each kernel under the record the evaluator selected from a pool tuned on
+*other* models, replayed as one CUDA graph with the L2 flushed between steps.  The headline is the largest
+configuration (BERT-base-shaped encoder, 128 tokens); `per_config` carries the same measurements for all five
+configurations and for the two sequence-length transfers.  Before the timed region the pools are loaded (or built by
+native grid tuning and saved) and the evaluator runs every (kernel, record) pair; both are reported, neither is part
+of a step.  Prints ONE JSON line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--model resnet18] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--only CONFIG] [--retune]
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -22,20 +27,48 @@ sys.path.insert(0, ROOT)
 
 METRIC = "TFLOP/s (model pass under transferred schedules)"
 UNIT = "TFLOP/s"
+POOL_DIR = os.path.join(ROOT, "paper_2201_05587_b200", "pools")
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "gemm_tc_traffic_bert_base.txt")
 
-
-# DRAM traffic of the dominant kernel per launch (dram__bytes_read.sum + dram__bytes_write.sum averaged over the
-# timed region's launches, one ncu pass; its summary is kept under profiles/), valid only for the
-# kernel source it was taken on: any later change of the kernel reports null until the counters are taken again.
-TRAFFIC_COUNTERS = {"model": "resnet18", "kernel_source_sha256_16": "4c28b7a4541da946", "bytes_per_launch": 2.736e6}
+# name -> (target model, pool sources); the first five are the benchmark configurations, in their order
+CONFIGS = [
+    ("config1_single_conv", "single_conv", ()),
+    ("config2_resnet18", "resnet18", ("resnet50",)),
+    ("config3_resnet50", "resnet50", ("resnet18", "vgg16")),
+    ("config4_mobilenet_v2", "mobilenet_v2", ("resnet50", "efficientnet_b0_like")),
+    ("config5_bert_base", "bert_base", ("resnet50", "mobilenet_v2")),
+    ("seq_transfer_128_to_256", "bert_base_256", ("bert_base",)),
+    ("seq_transfer_256_to_128", "bert_base", ("bert_base_256",)),
+]
+HEADLINE = "config5_bert_base"
+SEEDS = {"single_conv": 1, "resnet18": 2, "resnet50": 3, "mobilenet_v2": 4, "bert_base": 5, "bert_base_256": 5}
+CLASS_OF_OP = {0: "conv2d", 1: "depthwise", 2: "dense", 3: "batch_matmul", 4: "softmax"}
 
 
 def kernel_source_hash():
     import hashlib
-    path = os.path.join(ROOT, "paper_2201_05587_b200", "csrc", "tt_kernels.cu")
-    with open(path) as f:
-        body = "\n".join(line for line in f.read().splitlines() if "TT_STAMP" not in line)   # diagnostics-only lines
-    return hashlib.sha256(body.encode()).hexdigest()[:16]
+    h = hashlib.sha256()
+    for name in ("tt_kernels.cu", "tt_internal.h"):
+        with open(os.path.join(ROOT, "paper_2201_05587_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def traffic_per_launch():
+    """DRAM bytes per launch of the dominant kernel from the ncu capture summarised under profiles/ -- valid only for
+    the kernel source it was taken on: after any later change of the kernel this is None until the counters are retaken."""
+    try:
+        kv = {}
+        with open(TRAFFIC_FILE) as f:
+            for line in f:
+                if "=" in line and not line.startswith("#"):
+                    k, v = line.split("=", 1)
+                    kv[k.strip()] = v.strip()
+        if kv.get("kernel_source_sha256_16") == kernel_source_hash():
+            return float(kv["dram_bytes_per_launch"])
+    except (OSError, KeyError, ValueError):
+        pass
+    return None
 
 
 def measured_peaks():
@@ -45,6 +78,37 @@ def measured_peaks():
             d = json.load(f)
         return {"hbm_gbs": d.get("hbm_gbs", 6650.0), "bf16_tflops": d.get("bf16_tflops", 1590.0), "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+def algorithmic_work(spec):
+    """(flops, bytes) of one launch from the shapes alone: 2*M*N*K (depthwise: 2*outputs*taps; softmax: 5 per element);
+    4 bytes for every element of every tensor, each tensor once."""
+    from paper_2201_05587_b200 import workloads as W
+    s = spec.shapes
+    xs, ws, bs, rs, ys = W.tensor_shapes(spec)
+    n_el = lambda sh: 0 if sh is None else int(__import__("numpy").prod(sh))
+    by = 4.0 * (n_el(xs) + n_el(ws) + n_el(bs) + n_el(rs) + n_el(ys))
+    if spec.op == 0:
+        fl = 2.0 * n_el(ys) * s.c * s.r * s.s
+    elif spec.op == 1:
+        fl = 2.0 * n_el(ys) * s.r * s.s
+    elif spec.op in (2, 3):
+        fl = 2.0 * n_el(ys) * s.kk
+    else:
+        fl = 5.0 * n_el(ys)
+    return fl, by
+
+
+def workload_name(model, specs, pool_sources):
+    """The workload both arms report: model shape, kernel counts and where the schedule pool comes from."""
+    src = ",".join(pool_sources) if pool_sources else "the configuration's four fixed records"
+    return (f"{model}-shaped inference, batch 1, fp32, {len(specs)} unique kernels / "
+            f"{sum(sp.use_count for sp in specs)} layers per pass, pool from {src}")
+
+
+def config_dict(model, specs, pool_sources):
+    return {"workload": workload_name(model, specs, pool_sources), "l2": "flushed between steps (256 MB write)",
+            "replay": "one CUDA graph per data-chained model pass", "multi_gpu": "independent replicas"}
 
 
 class ClockSampler(threading.Thread):
@@ -92,16 +156,15 @@ def cpu_baseline_oracle(specs, arrays, budget_s, threads=0):
     from oracle import oracle as orc
     orc.build()
     flops, secs, used, names = 0.0, 0.0, 1, []
-    order = sorted(range(len(specs)), key=lambda i: -specs[i].workload().gemm_view().flops)
-    for i in order:
-        v = specs[i].workload().gemm_view()
-        est = v.flops / 2.0e9
+    work = [algorithmic_work(sp)[0] for sp in specs]
+    for i in sorted(range(len(specs)), key=lambda i: -work[i]):
+        est = work[i] / 2.0e9
         if secs > 0 and secs + est > budget_s:
             continue
         t0 = time.perf_counter()
         orc.reference(specs[i].op, specs[i].shapes, arrays[i], threads=threads)
         secs += time.perf_counter() - t0
-        flops += v.flops
+        flops += work[i]
         names.append(specs[i].name)
         if secs > budget_s:
             break
@@ -109,20 +172,23 @@ def cpu_baseline_oracle(specs, arrays, budget_s, threads=0):
     return flops, secs, used, names
 
 
-def workload_name(model, specs, pool_sources):
-    """The workload both arms report: model shape, kernel counts and where the schedule pool comes from."""
-    return (f"{model}-shaped inference, batch 1, fp32 NCHW, {len(specs)} unique kernels / "
-            f"{sum(sp.use_count for sp in specs)} per pass, pool from {','.join(pool_sources)}-shaped kernels")
+def headline_model_and_sources(args):
+    from paper_2201_05587_b200 import workloads as W
+    name = args.only or HEADLINE
+    for cname, model, sources in CONFIGS:
+        if cname == name:
+            return cname, model, sources
+    raise SystemExit(f"unknown configuration {name}; choose from {[c[0] for c in CONFIGS]}")
 
 
 def run_reference(args):
     """--impl reference: the CPU oracle, rank 0 only, on bounded samples of the same workload."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return 0
     from paper_2201_05587_b200 import workloads as W
-    specs = W.MODELS[args.model]()
-    arrays = [W.make_inputs(sp, args.seed, i) for i, sp in enumerate(specs)]
+    _, model, sources = headline_model_and_sources(args)
+    specs = W.MODELS[model]()
+    arrays = [W.make_inputs(sp, SEEDS[model], i) for i, sp in enumerate(specs)]
     total = args.steps + args.warmup
     per_step = max(1.0, 150.0 / max(total, 1))
     flops = secs = 0.0
@@ -137,7 +203,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": secs / max(args.steps, 1) * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": workload_name(args.model, specs, tuple(p for p in args.pool.split(",") if p) or W.POOL_SOURCES[args.model])},
+            "config": config_dict(model, specs, sources),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -145,33 +211,265 @@ def run_reference(args):
     return 0
 
 
-def tf32_peak(torch):
-    """cuBLAS TF32 matmul 8192^3, best of 10: the tensor-pipe denominator for this path (library call, not the product)."""
+def tf32_cublas_rate(torch):
+    """cuBLAS TF32 matmul 8192^3, median of 15 after warm-up: a library's achieved rate, reported beside the
+    tensor-pipe denominator (half of the measured BF16 rate), never used as the denominator itself."""
     old = torch.backends.cuda.matmul.allow_tf32
     torch.backends.cuda.matmul.allow_tf32 = True
     n = 8192
     a = torch.randn(n, n, device="cuda")
     b = torch.randn(n, n, device="cuda")
-    for _ in range(3):
+    for _ in range(5):
         a @ b
-    best = 1e9
-    for _ in range(10):
+    times = []
+    for _ in range(15):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         a @ b
         e1.record()
         e1.synchronize()
-        best = min(best, e0.elapsed_time(e1))
+        times.append(e0.elapsed_time(e1))
     torch.backends.cuda.matmul.allow_tf32 = old
     del a, b
-    return 2.0 * n ** 3 / (best * 1e-3) / 1e12
+    times.sort()
+    return 2.0 * n ** 3 / (times[len(times) // 2] * 1e-3) / 1e12
 
 
-def saturating_points(B, W, torch, dev, peaks, tf32):
+class Bench:
+    """Shared state of one bench process: device, peaks, the pool store."""
+
+    def __init__(self, args, torch, B, W, dev):
+        self.args, self.torch, self.B, self.W, self.dev = args, torch, B, W, dev
+        self.peaks = measured_peaks()
+        self.tensor_peak = self.peaks["bf16_tflops"] / 2.0        # TF32 issues at half the BF16 rate
+        self.pools, self.pool_how, self.pool_seconds, self.pool_tried = {}, {}, 0.0, 0
+        self.flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)          # larger than the 126 MB L2
+        self.tune_opts = B.tt_timing_opts()
+        self.tune_opts.warmup_batches, self.tune_opts.batches, self.tune_opts.min_batch_us, self.tune_opts.use_graph = 2, 5, 100, 1
+
+    # ---- pools: natively tuned records of a source model, kept as a text file --------------------------------
+    def pool_of(self, model):
+        B, W = self.B, self.W
+        if model in self.pools:
+            return self.pools[model]
+        path = os.path.join(POOL_DIR, f"{model}.txt")
+        if not self.args.retune and os.path.exists(path):
+            try:
+                recs, _ = B.pool_load(path)
+                self.pools[model], self.pool_how[model] = recs, "loaded"
+                return recs
+            except B.TTError:
+                pass                                     # written for another record version: tune again
+        t0 = time.perf_counter()
+        recs, us = [], []
+        for j, sp in enumerate(W.MODELS[model]()):
+            a = W.make_inputs(sp, SEEDS.get(model, 7) + 100, j)
+            swl = sp.workload()
+            keep, stt = W.device_tensors(sp, a, self.dev)
+            best, tried = swl.grid_tune(stt, self.tune_opts, level=self.args.tune_level, top_k=self.args.top_k)
+            self.pool_tried += tried
+            recs += [r for r, _ in best]
+            us += [u for _, u in best]
+            swl.close()
+            del keep
+        self.pool_seconds += time.perf_counter() - t0
+        try:
+            os.makedirs(POOL_DIR, exist_ok=True)
+            B.pool_save(path, recs, us)
+        except (OSError, B.TTError):
+            pass
+        self.pools[model], self.pool_how[model] = recs, "tuned"
+        return recs
+
+    def timed_steps(self, n, body, flush=True):
+        torch = self.torch
+        ms = 0.0
+        for _ in range(n):
+            if flush:
+                self.flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            body()
+            e1.record()
+            e1.synchronize()
+            ms += e0.elapsed_time(e1)
+        return ms
+
+    def capture(self, body):
+        torch = self.torch
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            body()
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            body()
+        return graph
+
+    def cold_sets(self, spec, arrays, max_sets=2048):
+        """Tensor sets carved out of one arena whose total footprint exceeds twice the L2, so that a launch that walks
+        them round-robin never finds its operands cached."""
+        torch, B, W = self.torch, self.B, self.W
+        shapes = W.tensor_shapes(spec)
+        names = ("x", "w", "bias", "residual")
+        parts, offs, off = [], {}, 0
+        for nm, sh in zip(names + ("y",), shapes):
+            if sh is None:
+                continue
+            n = 1
+            for d in sh:
+                n *= d
+            padded = (n + 63) // 64 * 64                                      # 256-byte granules
+            src = torch.zeros(padded, dtype=torch.float32, device=self.dev)
+            if nm != "y":
+                src[:n] = torch.from_numpy(arrays[nm]).to(self.dev).reshape(-1)
+            parts.append(src)
+            offs[nm] = (off, n, sh)
+            off += padded
+        row = torch.cat(parts)
+        n_sets = int(min(max_sets, max(2, (2 * 126e6) // (4 * off) + 1)))
+        arena = row.repeat(n_sets, 1)
+        sets = []
+        for i in range(n_sets):
+            v = {nm: arena[i, o:o + n].view(sh) for nm, (o, n, sh) in offs.items()}
+            sets.append(B.tensors(v["x"], v.get("w"), v.get("bias"), v.get("residual"), v["y"]))
+        return arena, sets
+
+    # ---- one configuration ---------------------------------------------------------------------------------------
+    def run_config(self, cname, model, sources, headline, steps, warmup):
+        torch, B, W, dev, args = self.torch, self.B, self.W, self.dev, self.args
+        seed = SEEDS[model]
+        specs = W.MODELS[model]()
+        arrays = [W.make_inputs(sp, seed, i) for i, sp in enumerate(specs)]
+        wls = [sp.workload() for sp in specs]
+        dev_t, tts = zip(*[W.device_tensors(sp, a, dev) for sp, a in zip(specs, arrays)])
+        pool = W.single_conv_pool() if model == "single_conv" else [r for src in sources for r in self.pool_of(src)]
+
+        # the evaluator: every kernel x every pool record (+ default)
+        o = B.tt_tune_opts()
+        o.include_default = 1
+        o.timing.warmup_batches, o.timing.batches, o.timing.min_batch_us, o.timing.use_graph = 3, 10, 200, 1
+        res = B.transfer_tune(list(wls), list(tts), pool, o)
+        n_cols = len(pool) + 1
+        chosen = res["chosen"]
+        use = [sp.use_count for sp in specs]
+        flat = [v for row in res["times_us"] for v in row]
+        lat_best = B.model_latency(flat, len(wls), n_cols, chosen, use)
+        lat_default = B.model_latency(flat, len(wls), n_cols, [0] * len(wls), use)
+        work = [algorithmic_work(sp) for sp in specs]
+        flops_pass = sum(f * u for (f, _), u in zip(work, use))
+        bytes_pass = sum(b * u for (_, b), u in zip(work, use))
+        best_recs = [w.default_schedule() if c == 0 else pool[c - 1] for w, c in zip(wls, chosen)]
+        infos = [w.check(r)[1] for w, r in zip(wls, best_recs)]
+        launches_pass = sum(i.launches * u for i, u in zip(infos, use))
+
+        out = {"model": model, "pool_sources": list(sources), "unique_kernels": len(specs), "layers_per_pass": sum(use),
+               "gflop_per_pass": flops_pass / 1e9, "algorithmic_mbytes_per_pass": bytes_pass / 1e6,
+               "sum_standalone_us": {"transferred": lat_best, "default": lat_default,
+                                     "speedup_over_default": lat_default / lat_best if lat_best else None},
+               "search": {"pairs_timed": res["pairs_timed"], "pairs_invalid": res["pairs_invalid"],
+                          "seconds": res["search_seconds"], "pool_records": len(pool)}}
+
+        # the data-chained pass (config 1 is a single kernel: its pass is that kernel)
+        if model in W.CHAINS:
+            _, steps_ = W.CHAINS[model]()
+            ch_arrays = W.make_chain_inputs(steps_, seed, init="bert" if model.startswith("bert") else "he")
+            bufs, ch_tts = W.chain_device_tensors(steps_, ch_arrays, dev)
+            order = [(st.kernel, tt) for st, tt in zip(steps_, ch_tts) if st.spec is not None]
+            del ch_arrays
+        else:
+            bufs, order = None, [(i, tt) for i, (tt, u) in enumerate(zip(tts, use)) for _ in range(u)]
+
+        def chained_pass():
+            for k, tt in order:
+                wls[k].run(tt)
+
+        def independent_pass():
+            for w, t, u in zip(wls, tts, use):
+                for _ in range(u):
+                    w.run(t)
+
+        n_side = max(5, min(steps, 30))
+        graph = self.capture(chained_pass)
+        self.timed_steps(warmup, graph.replay)
+        clocks = None
+        if headline:
+            from paper_2201_05587_b200 import replicas
+            replicas.barrier()
+            torch.cuda.synchronize()
+            sampler = ClockSampler(torch.cuda.current_device())
+            sampler.start()
+            torch.cuda.nvtx.range_push("tt_timed_region")      # lets a profiler restrict itself to the timed launches
+            ms_total = self.timed_steps(steps, graph.replay)
+            torch.cuda.synchronize()
+            torch.cuda.nvtx.range_pop()
+            replicas.barrier()
+            out["_ms_total"], out["_sampler"] = ms_total, sampler
+            chained_cold = ms_total / steps * 1e3
+        else:
+            chained_cold = self.timed_steps(n_side, graph.replay) / n_side * 1e3
+        chained_warm = self.timed_steps(n_side, graph.replay, flush=False) / n_side * 1e3
+        gi = self.capture(independent_pass)
+        self.timed_steps(3, gi.replay)
+        indep_cold = self.timed_steps(n_side, gi.replay) / n_side * 1e3
+        del gi
+        for w in wls:
+            st = w.status()
+            if st != B.TT_OK:
+                raise SystemExit(f"device status {st} after the timed region of {cname}")
+        out["pass_us"] = {"chained_cold_l2": chained_cold, "chained_warm_l2": chained_warm,
+                          "independent_kernels_cold_l2": indep_cold, "tflops_chained_cold_l2": flops_pass / chained_cold / 1e6}
+
+        # per kernel: cold-L2 standalone time and launch floor under the chosen record; per class: roofline fractions
+        cold = B.tt_timing_opts()
+        cold.warmup_batches, cold.batches, cold.min_batch_us, cold.use_graph = 2, 5, 200, 1
+        floor = B.tt_timing_opts()
+        floor.warmup_batches, floor.batches, floor.min_batch_us, floor.use_graph, floor.floor = 2, 5, 100, 1, 1
+        rows, classes = [], {}
+        hbm, tpk = self.peaks["hbm_gbs"], self.tensor_peak
+        for i, (sp, w, a) in enumerate(zip(specs, wls, arrays)):
+            arena, sets = self.cold_sets(sp, a)
+            tm = w.time(sets, cold)
+            fl = w.time(sets[:1], floor)
+            del arena, sets
+            f, b = work[i]
+            t_hbm, t_tensor = b / hbm / 1e3, (f / tpk / 1e6 if sp.op in (0, 2, 3) else 0.0)
+            t_roof = max(t_hbm, t_tensor)
+            rows.append({"kernel": sp.name, "class": CLASS_OF_OP[sp.op], "use": sp.use_count, "mflop": f / 1e6, "mbytes": b / 1e6,
+                         "record": infos[i].legal.short(), "grid": [infos[i].grid_x, infos[i].grid_y, infos[i].grid_z],
+                         "warm_us": res["best_us"][i], "default_us": res["times_us"][i][0], "cold_us": tm.median_us,
+                         "floor_us": fl.median_us, "roofline_us": t_roof, "bound": "hbm" if t_hbm >= t_tensor else "tensor",
+                         "valid_records": sum(1 for s in res["status"][i] if s == 0), "chosen_column": chosen[i]})
+            c = classes.setdefault(CLASS_OF_OP[sp.op], {"kernels": 0, "launches": 0, "flops": 0.0, "bytes": 0.0, "cold_us": 0.0,
+                                                        "roof_us": 0.0, "roof_or_floor_us": 0.0, "floor_us": 0.0})
+            u = sp.use_count
+            c["kernels"] += 1
+            c["launches"] += infos[i].launches * u
+            c["flops"] += f * u
+            c["bytes"] += b * u
+            c["cold_us"] += tm.median_us * u
+            c["floor_us"] += fl.median_us * u
+            c["roof_us"] += t_roof * u
+            c["roof_or_floor_us"] += max(t_roof, fl.median_us) * u
+        per_class = {}
+        for name, c in classes.items():
+            per_class[name] = {"unique_kernels": c["kernels"], "launches_per_pass": c["launches"],
+                               "tflops_cold_l2": c["flops"] / c["cold_us"] / 1e6, "gbs_cold_l2": c["bytes"] / c["cold_us"] / 1e3,
+                               "frac_of_roofline": c["roof_us"] / c["cold_us"],
+                               "frac_of_max_roofline_launch_floor": c["roof_or_floor_us"] / c["cold_us"],
+                               "sum_cold_us": c["cold_us"], "sum_launch_floor_us": c["floor_us"]}
+        out["per_class_cold_l2"] = per_class
+        out["_rows"], out["_classes"] = rows, classes
+        out["_ctx"] = (specs, arrays, wls, tts, dev_t, use, flops_pass, launches_pass, bufs, order, graph)
+        return out
+
+
+def saturating_points(bench):
     """The kernel families at sizes where a launch lasts long enough for its roofline to be reachable (NOT one of the
     benchmark configurations: batch-1 kernels have roofline times below one launch).  Each family is timed under a
-    short list of records; the best is reported against its bound: tensor pipe (cuBLAS TF32 rate measured in this
-    run) for the contractions, measured HBM copy rate for depthwise and softmax."""
+    short list of records; the best is reported against its bound: the tensor pipe (half the measured BF16 rate; the
+    cuBLAS TF32 rate of this run is given beside it) for the contractions, the measured HBM copy rate otherwise."""
+    B, W, dev = bench.B, bench.W, bench.dev
     def conv(n, c, hw, k, r, pad):
         return W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(n, c, hw, hw, k, r, r, 1, pad, True, B.TT_ACT_RELU), 1,
                       f"conv{r}x{r}_n{n}_{c}x{hw}->{k}")
@@ -192,8 +490,7 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
         (conv(32, 256, 28, 256, 3, 1), "tensor",
          [tc(tile_n=256, tile_k=32, stages=5, k_order=1, mma_m_axis=1), tc(tile_n=224, tile_k=96, stages=2, k_order=1, mma_m_axis=1),
           tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1)]),
-        # the same layer at batch 37: 8 tiles x 37 images = 296 CTAs = exactly two per SM-slot wave of 148 (batch 32
-        # leaves the second wave 27 % empty)
+        # the same layer at batch 37: 8 tiles x 37 images = 296 CTAs = exactly two waves of 148
         (conv(37, 256, 28, 256, 3, 1), "tensor",
          [tc(tile_n=224, tile_k=96, stages=2, k_order=1, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=5, k_order=1, mma_m_axis=1)]),
         (conv(32, 256, 56, 64, 1, 0), "hbm",
@@ -208,16 +505,11 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
         (W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(64, 1024, 1024, 1024, True), 1, "bmm_nt_64x1024x1024x1024", "bert"), "tensor",
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=4, mma_m_axis=1)]),
         (dw(64, 144, 56, 1), "hbm",
-         [dwr(tile_m=4, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=2),
-          dwr(tile_m=16, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=128, unroll=2),
-          dwr(tile_m=4, block_y=16, block_x=56, items_per_thread=4, vec_width=4, threads=128, unroll=4),
-          dwr(tile_m=8, block_y=56, block_x=56, items_per_thread=8, vec_width=4, threads=128, unroll=2),
+         [dwr(tile_m=4, block_y=16, block_x=56, items_per_thread=4, vec_width=4, threads=128, unroll=4),
           dwr(tile_m=8, block_y=14, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=4, raster=1, stages=2),
           dwr(tile_m=4, block_y=28, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=4, raster=1, stages=2)]),
         (dw(32, 96, 112, 2), "hbm",
          [dwr(tile_m=4, block_y=8, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=2),
-          dwr(tile_m=4, block_y=4, block_x=32, items_per_thread=4, vec_width=4, threads=64, unroll=1),
-          dwr(tile_m=1, block_y=8, block_x=56, items_per_thread=4, vec_width=4, threads=64, unroll=2),
           dwr(tile_m=4, block_y=8, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=2, raster=1, stages=2),
           dwr(tile_m=8, block_y=4, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=2, raster=1, stages=2)]),
         (dw(256, 240, 28, 1, r=5), "hbm",      # an EfficientNet-B0-shaped 5x5 layer
@@ -236,7 +528,7 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
         a = W.make_inputs(sp, 7)
         wl = sp.workload()
         t, tt = W.device_tensors(sp, a, dev)
-        v = wl.gemm_view()
+        f, b = algorithmic_work(sp)
         best = None
         for r in recs:
             st, info = wl.try_apply(r)
@@ -250,11 +542,23 @@ def saturating_points(B, W, torch, dev, peaks, tf32):
         if best is None:
             continue
         us, rec = best
-        row = {"kernel": sp.name, "record": rec, "us": us, "tflops": v.flops / us / 1e6, "gbs": v.bytes / us / 1e3,
-               "algorithmic_mbytes": v.bytes / 1e6, "bound": bound}
-        row["frac"] = (row["tflops"] / tf32) if bound == "tensor" and tf32 else row["gbs"] / peaks["hbm_gbs"]
+        row = {"kernel": sp.name, "record": rec, "us": us, "tflops": f / us / 1e6, "gbs": b / us / 1e3,
+               "algorithmic_mbytes": b / 1e6, "bound": bound}
+        if bound == "tensor":
+            row["frac"] = row["tflops"] / bench.tensor_peak
+            row["frac_of_cublas_tf32_this_run"] = row["tflops"] / bench.cublas_tf32 if bench.cublas_tf32 else None
+        else:
+            row["frac"] = row["gbs"] / bench.peaks["hbm_gbs"]
         out.append(row)
     return out
+
+
+def free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    p = s.getsockname()[1]
+    s.close()
+    return p
 
 
 def main():
@@ -263,16 +567,20 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours")
-    ap.add_argument("--model", default="resnet18", choices=["resnet18", "resnet50", "mobilenet_v2", "bert_base", "bert_base_256"])
-    ap.add_argument("--pool", default="", help="comma-separated models whose tuned records form the pool (default: the config's)")
-    ap.add_argument("--seed", type=int, default=2)
+    ap.add_argument("--only", default="", help="run this configuration alone, as the headline (e.g. config2_resnet18)")
+    ap.add_argument("--retune", action="store_true", help="ignore the pool files and tune the source models again")
     ap.add_argument("--tune-level", type=int, default=0)
     ap.add_argument("--top-k", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--report", default="", help="write the per-kernel table (JSON) to this file")
+    ap.add_argument("--report", default="", help="write the per-kernel tables (JSON) to this file")
     ap.add_argument("--no-saturating", action="store_true", help="skip the saturating-size points of the kernel families")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    if args.gpus > 1 and "RANK" not in os.environ:
+        # started by hand for N GPUs: become N replica processes, one per GPU
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+        return subprocess.call(cmd)
     if args.impl == "reference":
         return run_reference(args)
 
@@ -287,91 +595,13 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     B.lib()
-    peaks = measured_peaks()
+    bench = Bench(args, torch, B, W, dev)
+    bench.cublas_tf32 = tf32_cublas_rate(torch) if rank == 0 else 0.0
 
-    # ---- target model, pool sources, tensors -------------------------------------------------------------
-    specs = W.MODELS[args.model]()
-    arrays = [W.make_inputs(sp, args.seed, i) for i, sp in enumerate(specs)]
-    wls = [sp.workload() for sp in specs]
-    dev_t, tts = zip(*[W.device_tensors(sp, a, dev) for sp, a in zip(specs, arrays)])
-
-    topts = B.tt_timing_opts()
-    topts.warmup_batches, topts.batches, topts.min_batch_us, topts.use_graph = 2, 5, 100, 1
-    t0 = time.perf_counter()
-    pool, n_tried = [], 0
-    pool_sources = tuple(p for p in args.pool.split(",") if p) or W.POOL_SOURCES[args.model]
-    for src in pool_sources:
-        for j, sp in enumerate(W.MODELS[src]()):
-            a = W.make_inputs(sp, args.seed + 100, j)
-            swl = sp.workload()
-            _, stt = W.device_tensors(sp, a, dev)
-            best, tried = swl.grid_tune(stt, topts, level=args.tune_level, top_k=args.top_k)
-            n_tried += tried
-            pool += [r for r, _ in best]
-            swl.close()
-    pool_seconds = time.perf_counter() - t0
-
-    # ---- the evaluator: every kernel x every pool record (+ default) -------------------------------------
-    o = B.tt_tune_opts()
-    o.include_default = 1
-    o.timing.warmup_batches, o.timing.batches, o.timing.min_batch_us, o.timing.use_graph = 3, 10, 200, 1
-    res = B.transfer_tune(list(wls), list(tts), pool, o)
-    n_cols = len(pool) + 1
-    chosen = res["chosen"]
-    use = [sp.use_count for sp in specs]
-    flat = [v for row in res["times_us"] for v in row]
-    lat_best = B.model_latency(flat, len(wls), n_cols, chosen, use)
-    lat_default = B.model_latency(flat, len(wls), n_cols, [0] * len(wls), use)
-
-    views = [w.gemm_view() for w in wls]
-    flops_pass = sum(v.flops * u for v, u in zip(views, use))
-    bytes_pass = sum(v.bytes * u for v, u in zip(views, use))
-    launches_pass = 0
-    for w, u, c in zip(wls, use, chosen):
-        rec = w.default_schedule() if c == 0 else pool[c - 1]
-        launches_pass += w.check(rec)[1].launches * u
-
-    # ---- one model pass as a CUDA graph --------------------------------------------------------------------
-    def model_pass():
-        for w, t, u in zip(wls, tts, use):
-            for _ in range(u):
-                w.run(t)
-
-    side = torch.cuda.Stream()
-    with torch.cuda.stream(side):
-        model_pass()
-    side.synchronize()
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph, stream=side):
-        model_pass()
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)          # larger than the 126 MB L2
-
-    def timed_steps(n, body):
-        ms = 0.0
-        for _ in range(n):
-            flush.fill_(1)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            body()
-            e1.record()
-            e1.synchronize()
-            ms += e0.elapsed_time(e1)
-        return ms
-
-    timed_steps(args.warmup, graph.replay)
-    replicas.barrier()
-    torch.cuda.synchronize()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    torch.cuda.nvtx.range_push("tt_timed_region")      # lets a profiler restrict itself to the timed launches
-    ms_total = timed_steps(args.steps, graph.replay)
-    torch.cuda.synchronize()
-    torch.cuda.nvtx.range_pop()
-    replicas.barrier()
-    for w in wls:
-        st = w.status()
-        if st != B.TT_OK:
-            raise SystemExit(f"device status {st} after the timed region")
+    head_name, head_model, head_sources = headline_model_and_sources(args)
+    head = bench.run_config(head_name, head_model, head_sources, True, args.steps, args.warmup)
+    specs, arrays, wls, tts, dev_t, use, flops_pass, launches_pass, bufs, order, graph = head.pop("_ctx")
+    ms_total, sampler = head.pop("_ms_total"), head.pop("_sampler")
     value, slowest_s = replicas.aggregate(flops_pass * args.steps / 1e12, ms_total * 1e-3, dev)
     ms_per_step = slowest_s * 1e3 / args.steps
 
@@ -383,7 +613,7 @@ def main():
         host_sets.append((h, B.tensors(h["x"], h["w"], h["bias"], h["residual"], h["y"])))
     bytes_up = bytes_down = 0
 
-    # Every kernel's inputs go up and its output comes down every time it runs.  The calls are enqueued on three
+    # Every layer's inputs go up and its output comes down every time it runs.  The calls are enqueued on three
     # streams (a workload always on the same one: it owns one set of device staging buffers), so that one kernel's
     # upload, another's compute and a third's download overlap; the pass ends when all three streams have drained.
     side = [torch.cuda.Stream(device=dev) for _ in range(3)]
@@ -394,18 +624,17 @@ def main():
         cur = torch.cuda.current_stream()
         for s_ in side:
             s_.wait_stream(cur)
-        for i, (w, (h, ht), u) in enumerate(zip(wls, host_sets, use)):
-            for _ in range(u):
-                up, down = w.run_host_async(ht, side[i % len(side)])
-                bytes_up += up
-                bytes_down += down
+        for k, _ in order:
+            up, down = wls[k].run_host_async(host_sets[k][1], side[k % len(side)])
+            bytes_up += up
+            bytes_down += down
         for s_ in side:
             cur.wait_stream(s_)
 
-    timed_steps(3, e2e_pass)
+    bench.timed_steps(3, e2e_pass)
     e2e_steps = max(3, min(args.steps, 10))
     replicas.barrier()
-    e2e_ms = timed_steps(e2e_steps, e2e_pass)
+    e2e_ms = bench.timed_steps(e2e_steps, e2e_pass)
     replicas.barrier()
     e2e_value, _ = replicas.aggregate(flops_pass * e2e_steps / 1e12, e2e_ms * 1e-3, dev)
     sampler.stop_flag = True                             # clocks were sampled over both timed regions (device-resident and end to end)
@@ -416,92 +645,87 @@ def main():
             raise SystemExit(f"device status {st} after the end-to-end region")
         if not bool(torch.isfinite(h["y"]).all()):
             raise SystemExit("end-to-end pass left a host output unwritten")
+    del host_sets
 
-    # ---- roofline of the dominant kernel family (live, standalone, cold L2) ------------------------------
-    # Rotating tensor sets whose footprint exceeds twice the L2 make every launch miss; times are CUDA events
-    # around batches of launches on the launching stream.
-    rows = []
-    cold = B.tt_timing_opts()
-    cold.warmup_batches, cold.batches, cold.min_batch_us, cold.use_graph = 2, 5, 200, 1
-    gemm_flops = gemm_bytes = gemm_cold_us = gemm_launches = 0.0
-    tf32 = tf32_peak(torch) if rank == 0 else 0.0
-    for i, (sp, w, v, a) in enumerate(zip(specs, wls, views, arrays)):
-        n_sets = int(min(1024, max(2, (2 * 126e6) // max(v.bytes, 1) + 1)))
-        sets, keep = [], []
-        for _ in range(n_sets):
-            t, tt = W.device_tensors(sp, a, dev)
-            keep.append(t)
-            sets.append(tt)
-        tm = w.time(sets, cold)
-        warm = res["best_us"][i]
-        rec = w.default_schedule() if chosen[i] == 0 else pool[chosen[i] - 1]
-        info = w.check(rec)[1]
-        rows.append({"kernel": sp.name, "use": sp.use_count, "mflop": v.flops / 1e6, "mbytes": v.bytes / 1e6,
-                     "record": info.legal.short(), "grid": [info.grid_x, info.grid_y, info.grid_z],
-                     "warm_us": warm, "default_us": res["times_us"][i][0], "cold_us": tm.median_us,
-                     "tflops_warm": v.flops / warm / 1e6, "gbs_cold": v.bytes / tm.median_us / 1e3,
-                     "valid_records": sum(1 for s in res["status"][i] if s == 0), "origin": chosen[i]})
-        if w.family() == B.TT_FAMILY_GEMM_TC:
-            gemm_flops += v.flops * sp.use_count
-            gemm_bytes += v.bytes * sp.use_count
-            gemm_cold_us += tm.median_us * sp.use_count
-            gemm_launches += info.launches * sp.use_count
-        del keep, sets
-    ai = gemm_flops / max(gemm_bytes, 1)
-    ridge = tf32 * 1e12 / (peaks["hbm_gbs"] * 1e9) if tf32 else 107.0
+    # ---- roofline of the dominant kernel family over the headline pass (live, standalone, cold L2) ---------------
+    classes = head.pop("_classes")
+    rows_by_config = {head_name: head.pop("_rows")}
+    gemm = {"flops": 0.0, "bytes": 0.0, "cold_us": 0.0, "launches": 0, "floor_us": 0.0}
+    for name in ("conv2d", "dense", "batch_matmul"):
+        if name in classes:
+            for k in gemm:
+                gemm[k] += classes[name][k]
+    peaks = bench.peaks
+    ai = gemm["flops"] / max(gemm["bytes"], 1)
+    ridge = bench.tensor_peak * 1e12 / (peaks["hbm_gbs"] * 1e9)
     if ai < ridge:
-        roof = {"bound": "hbm", "achieved": gemm_bytes / gemm_cold_us / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        roof = {"bound": "hbm", "achieved": gemm["bytes"] / gemm["cold_us"] / 1e3, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     else:
-        roof = {"bound": "tensor", "achieved": gemm_flops / gemm_cold_us / 1e6, "peak": tf32, "unit": "TFLOP/s"}
+        roof = {"bound": "tensor", "achieved": gemm["flops"] / gemm["cold_us"] / 1e6, "peak": bench.tensor_peak, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    same_kernel = args.model == TRAFFIC_COUNTERS["model"] and kernel_source_hash() == TRAFFIC_COUNTERS["kernel_source_sha256_16"]
-    roof["traffic"] = TRAFFIC_COUNTERS["bytes_per_launch"] if same_kernel else None
+    roof["traffic"] = traffic_per_launch()
     roof["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum, timed region average)"
-    roof.update({"kernel": "tt_gemm_tc_kernel", "peak_source": peaks["source"] + (" hbm copy" if roof["bound"] == "hbm" else " cuBLAS TF32 8192^3, this run"),
-                 "launches_per_pass": gemm_launches, "avg_launch_us": gemm_cold_us / max(gemm_launches, 1),
-                 "algorithmic_mbytes_per_pass": gemm_bytes / 1e6, "algorithmic_gflop_per_pass": gemm_flops / 1e9,
-                 "tf32_peak_tflops_this_run": tf32, "tensor_frac": (gemm_flops / gemm_cold_us / 1e6) / tf32 if tf32 else None,
+    roof.update({"kernel": "tt_gemm_tc_kernel",
+                 "peak_source": peaks["source"] + (" hbm copy" if roof["bound"] == "hbm" else " bf16 burst / 2 (TF32 issues at half the BF16 rate)"),
+                 "launches_per_pass": gemm["launches"], "avg_launch_us": gemm["cold_us"] / max(gemm["launches"], 1),
+                 "avg_launch_floor_us": gemm["floor_us"] / max(gemm["launches"], 1),
+                 "algorithmic_mbytes_per_pass": gemm["bytes"] / 1e6, "algorithmic_gflop_per_pass": gemm["flops"] / 1e9,
+                 "tensor_peak_tflops": bench.tensor_peak, "cublas_tf32_tflops_this_run": bench.cublas_tf32,
+                 "tensor_frac": (gemm["flops"] / gemm["cold_us"] / 1e6) / bench.tensor_peak,
                  "l2": "cold (rotating tensor sets > 2x L2)"})
 
-    sat = saturating_points(B, W, torch, dev, peaks, tf32) if rank == 0 and not args.no_saturating else None
-    line = None
+    cpu = None
+    if rank == 0 and not args.no_cpu_baseline:
+        # the whole pass costs the oracle a fraction of a second: repeat it until about ten seconds have been timed
+        f = s = 0.0
+        rounds = 0
+        while s < 10.0 and rounds < 1000:
+            f1, s1, used, names = cpu_baseline_oracle(specs, arrays, 20.0)
+            f += f1; s += s1; rounds += 1
+        cpu = {"value": f / s / 1e12, "unit": UNIT, "cores": used, "kind": "oracle",
+               "sample": f"{len(names)} of {len(specs)} unique kernels once each per round, {rounds} rounds "
+                         f"({f / 1e9:.1f} GFLOP in {s:.1f} s)"}
+    for w in wls:
+        w.close()
+    del graph, bufs, order, tts, dev_t, wls
+
+    # ---- the other configurations (one process only: they are measurements, not part of the scaling run) -----------
+    per_config = {head_name: head}
+    if world == 1 and not args.only:
+        for cname, model, sources in CONFIGS:
+            if cname == head_name:
+                continue
+            c = bench.run_config(cname, model, sources, False, 20, 3)
+            ctx = c.pop("_ctx")
+            for w in ctx[2]:
+                w.close()
+            del ctx
+            c.pop("_classes")
+            rows_by_config[cname] = c.pop("_rows")
+            per_config[cname] = c
+            torch.cuda.empty_cache()
+    sat = saturating_points(bench) if rank == 0 and not args.no_saturating and world == 1 else None
+
     if rank == 0:
-        cpu = None
-        if not args.no_cpu_baseline:
-            # the whole pass costs the oracle a fraction of a second: repeat it until about ten seconds have been timed
-            f = s = 0.0
-            rounds = 0
-            while s < 10.0 and rounds < 1000:
-                f1, s1, used, names = cpu_baseline_oracle(specs, arrays, 20.0)
-                f += f1; s += s1; rounds += 1
-            cpu = {"value": f / s / 1e12, "unit": UNIT, "cores": used, "kind": "oracle",
-                   "sample": f"{len(names)} of {len(specs)} unique kernels once each per round, {rounds} rounds "
-                             f"({f / 1e9:.1f} GFLOP in {s:.1f} s)"}
-        clocks = sampler.summary()
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "tf32",
             "data": "synthetic",
-            "config": {"workload": workload_name(args.model, specs, pool_sources),
-                       "l2": "flushed between steps (256 MB write)", "replay": "one CUDA graph per model pass",
-                       "multi_gpu": "independent replicas"},
+            "config": config_dict(head_model, specs, head_sources),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bytes_up, "d2h_bytes_per_step": bytes_down,
                     "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
             "gpu_launches": int(launches_pass * args.steps),
-            "clocks": clocks,
+            "clocks": sampler.summary(),
             "roofline": roof,
             "cpu_baseline": cpu,
-            "model_latency_us": {"transferred_sum_standalone": lat_best, "default_sum_standalone": lat_default,
-                                 "speedup_over_default": lat_default / lat_best if lat_best else None,
-                                 "measured_pass_cold_l2": ms_per_step * 1e3},
+            "per_config": per_config,
             "saturating_sizes_not_a_benchmark_config": sat,
-            "search": {"pairs_timed": res["pairs_timed"], "pairs_invalid": res["pairs_invalid"],
-                       "seconds": res["search_seconds"], "pool_records": len(pool), "pool_build_seconds": pool_seconds,
-                       "pool_candidates_tried": n_tried},
+            "pools": {"how": bench.pool_how, "build_seconds": bench.pool_seconds, "candidates_tried": bench.pool_tried,
+                      "directory": os.path.relpath(POOL_DIR, ROOT)},
         }
         if args.report:
             with open(args.report, "w") as fh:
-                json.dump({"line": line, "kernels": rows}, fh, indent=1)
+                json.dump({"line": line, "kernels": rows_by_config}, fh, indent=1)
         print(json.dumps(line))
     replicas.finalize()
     return 0

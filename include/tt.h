@@ -170,7 +170,10 @@ typedef struct tt_timing_opts {
     int32_t min_batch_us;     /* each batch repeats the launch until it lasts at least this long; default 200 */
     int32_t max_repeats;      /* cap on launches per batch; default 4096 */
     int32_t use_graph;        /* 1: replay each batch as a CUDA graph (no CPU launch gaps) */
-    int32_t reserved[3];
+    int32_t floor;            /* 1: time, instead of the kernel, an empty kernel launched the same way (same grid, block
+                                 size, shared memory, cluster shape, dependent launch): what a launch of this record costs
+                                 before it does any work */
+    int32_t reserved[2];
 } tt_timing_opts;
 
 typedef struct tt_timing {
@@ -289,6 +292,17 @@ tt_status tt_transfer_tune(tt_workload* const* model_workloads, const tt_tensors
 tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, const tt_timing_opts* o, int32_t level,
                        size_t top_k, tt_schedule_record* out_records, float* out_us, size_t* n_out,
                        int32_t* n_tried);
+
+/* Schedules persist as records keyed by the kernel they were tuned on (Section 2: tuned schedules are kept in a log and
+ * looked up by workload ID).  A pool file is text, one record per line, "field=value" pairs separated by blanks
+ * (version, family, origin_op, origin=<the nineteen integers of tt_shapes, comma-separated, then scale>, every
+ * record field by name, us=<the time it was tuned to, microseconds>); lines that start with '#' are comments.
+ * Pure host.  tt_pool_save overwrites `path`; us may be NULL (written as -1).  tt_pool_load reads at most `cap`
+ * records into out/us (us may be NULL), sets *n_out to the number of records in the file (more than cap:
+ * TT_ERR_RESOURCE, nothing beyond cap is written); cap == 0 counts only.  A line that cannot be parsed, names an
+ * unknown field or carries another record version: TT_ERR_INVALID_ARG.  A missing file: TT_ERR_INVALID_ARG. */
+tt_status tt_pool_save(const char* path, const tt_schedule_record* records, const float* us, size_t n);
+tt_status tt_pool_load(const char* path, tt_schedule_record* out, float* us, size_t cap, size_t* n_out);
 
 /* Refining a transferred record (Section 7 names it as the next step: vary the parameters of schedules that were
  * transfer-tuned from another model).  The neighbourhood of a record: every field its family uses is moved one rung

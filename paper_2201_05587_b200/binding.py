@@ -73,7 +73,7 @@ class tt_apply_info(C.Structure):
 
 class tt_timing_opts(C.Structure):
     _fields_ = [("warmup_batches", i32), ("batches", i32), ("min_batch_us", i32), ("max_repeats", i32),
-                ("use_graph", i32), ("reserved", i32 * 3)]
+                ("use_graph", i32), ("floor", i32), ("reserved", i32 * 2)]
 
 
 class tt_timing(C.Structure):
@@ -129,6 +129,8 @@ EXPORTS = {
     "tt_refine": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(tt_timing_opts),
                         C.POINTER(tt_schedule_record), i32, f32, C.POINTER(tt_schedule_record), C.POINTER(f32),
                         C.POINTER(f32), C.POINTER(i32)]),
+    "tt_pool_save": (i32, [C.c_char_p, C.POINTER(tt_schedule_record), C.POINTER(f32), C.c_size_t]),
+    "tt_pool_load": (i32, [C.c_char_p, C.POINTER(tt_schedule_record), C.POINTER(f32), C.c_size_t, C.POINTER(C.c_size_t)]),
     "tt_dense_static_scratch": (i32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, i32, i32, i32, i32,
                                       C.POINTER(tt_schedule_record), C.c_void_p, C.POINTER(C.c_int64)]),
 }
@@ -237,6 +239,29 @@ def rank_pools(class_share, class_kernels):
     od = (i32 * max(n_m, 1))()
     _check(lib().tt_rank_pools(sh, n_c, ck, n_m, sc, od), "tt_rank_pools")
     return list(sc)[:n_m], list(od)[:n_m]
+
+
+def pool_save(path, records, us=None):
+    """tt_pool_save: write records (and the times they were tuned to) as a text pool file."""
+    n = len(records)
+    arr = (tt_schedule_record * max(n, 1))(*records)
+    uarr = (f32 * max(n, 1))(*[float(v) for v in us]) if us is not None else None
+    _check(lib().tt_pool_save(os.fsencode(path), arr, uarr, n), f"tt_pool_save({path})")
+
+
+def pool_load(path):
+    """tt_pool_load: returns (records, times in microseconds)."""
+    n = C.c_size_t()
+    _check(lib().tt_pool_load(os.fsencode(path), None, None, 0, C.byref(n)), f"tt_pool_load({path})")
+    arr = (tt_schedule_record * max(n.value, 1))()
+    uarr = (f32 * max(n.value, 1))()
+    _check(lib().tt_pool_load(os.fsencode(path), arr, uarr, n.value, C.byref(n)), f"tt_pool_load({path})")
+    out = []
+    for i in range(n.value):
+        r = tt_schedule_record()
+        C.memmove(C.byref(r), C.byref(arr[i]), C.sizeof(r))
+        out.append(r)
+    return out, [float(uarr[i]) for i in range(n.value)]
 
 
 def _ptr(t):

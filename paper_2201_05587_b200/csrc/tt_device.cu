@@ -17,6 +17,7 @@ cudaError_t launch_dw_tma(const tt_apply_info& I, const DwArgs& dw, const void* 
 cudaError_t launch_row(const tt_apply_info& I, const RowArgs& row, cudaStream_t st);
 cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits);
 cudaError_t launch_repack(const float* w, float* out, int kout, int C, int RS, int CB, cudaStream_t st);
+cudaError_t launch_floor(const tt_apply_info& I, int cluster, cudaStream_t st);
 
 namespace {
 
@@ -323,6 +324,15 @@ static tt_status time_applied(tt_workload* w, const tt_tensors* sets, size_t n_s
     auto fail = [&](tt_status s) { rc = s; };
     auto run_n = [&](int n, cudaStream_t s) -> tt_status {
         for (int i = 0; i < n; ++i) {
+            if (o.floor) {
+                // the launch floor of the applied record: an empty kernel with the same launch shape
+                for (int l = 0; l < w->plan.info.launches; ++l)
+                    if (launch_floor(w->plan.info, w->family == TT_FAMILY_GEMM_TC ? w->plan.g.cluster : 0, s) != cudaSuccess) {
+                        cudaGetLastError();
+                        return TT_ERR_CUDA;
+                    }
+                continue;
+            }
             tt_status r = launch(w, &sets[next], s);
             next = (next + 1) % n_sets;
             if (r != TT_OK) return r;

@@ -2,7 +2,10 @@
 // legalisation / validity layer, the selector.  Nothing here touches the device.
 #include <algorithm>
 #include <cmath>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
+#include <string>
 #include <new>
 #include "tt_internal.h"
 
@@ -839,6 +842,96 @@ tt_status tt_refine_with(const tt_workload* w, const tt_schedule_record* start, 
     *best = cur; *best_us = cur_us;
     if (n_timed) *n_timed = timed;
     return TT_OK;
+}
+
+// ---- pool files ---------------------------------------------------------------------------------------------------
+namespace {
+struct RecField { const char* name; int32_t tt_schedule_record::*field; };
+const RecField kRecFields[] = {
+    {"tile_m", &tt_schedule_record::tile_m}, {"tile_n", &tt_schedule_record::tile_n}, {"tile_k", &tt_schedule_record::tile_k},
+    {"stages", &tt_schedule_record::stages}, {"split_k", &tt_schedule_record::split_k}, {"raster", &tt_schedule_record::raster},
+    {"block_x", &tt_schedule_record::block_x}, {"block_y", &tt_schedule_record::block_y},
+    {"items_per_thread", &tt_schedule_record::items_per_thread}, {"vec_width", &tt_schedule_record::vec_width},
+    {"unroll", &tt_schedule_record::unroll}, {"threads", &tt_schedule_record::threads},
+    {"mma_m_axis", &tt_schedule_record::mma_m_axis}, {"slab_tiles", &tt_schedule_record::slab_tiles},
+    {"acc_split", &tt_schedule_record::acc_split}, {"k_order", &tt_schedule_record::k_order},
+};
+int32_t* shape_ints(tt_shapes& s, int i) {
+    int32_t* f[] = {&s.n, &s.c, &s.h, &s.w, &s.k, &s.r, &s.s, &s.stride_h, &s.stride_w, &s.pad_h, &s.pad_w,
+                    &s.batch, &s.m, &s.nn, &s.kk, &s.trans_b, &s.has_bias, &s.has_residual, &s.act};
+    return f[i];
+}
+constexpr int kShapeInts = 19;
+}  // namespace
+
+tt_status tt_pool_save(const char* path, const tt_schedule_record* records, const float* us, size_t n) {
+    if (!path || (n && !records)) return TT_ERR_INVALID_ARG;
+    FILE* f = std::fopen(path, "w");
+    if (!f) return TT_ERR_INVALID_ARG;
+    std::fprintf(f, "# schedule pool: one record per line, field=value\n");
+    for (size_t i = 0; i < n; ++i) {
+        tt_schedule_record r = records[i];
+        std::fprintf(f, "version=%u family=%u origin_op=%d origin=", r.version, r.family, r.origin_op);
+        for (int j = 0; j < kShapeInts; ++j) std::fprintf(f, "%d,", *shape_ints(r.origin, j));
+        std::fprintf(f, "%.9g", (double)r.origin.scale);
+        for (const RecField& rf : kRecFields) std::fprintf(f, " %s=%d", rf.name, r.*(rf.field));
+        std::fprintf(f, " us=%.6g\n", us ? (double)us[i] : -1.0);
+    }
+    const bool ok = std::fclose(f) == 0;
+    return ok ? TT_OK : TT_ERR_INVALID_ARG;
+}
+
+tt_status tt_pool_load(const char* path, tt_schedule_record* out, float* us, size_t cap, size_t* n_out) {
+    if (!path || !n_out || (cap && !out)) return TT_ERR_INVALID_ARG;
+    FILE* f = std::fopen(path, "r");
+    if (!f) return TT_ERR_INVALID_ARG;
+    size_t n = 0;
+    tt_status rc = TT_OK;
+    char line[2048];
+    while (rc == TT_OK && std::fgets(line, sizeof line, f)) {
+        char* p = line;
+        while (*p == ' ' || *p == '\t') ++p;
+        if (*p == '#' || *p == '\n' || *p == '\r' || *p == 0) continue;
+        tt_schedule_record r;
+        std::memset(&r, 0, sizeof r);
+        float t = -1.f;
+        bool have_version = false;
+        for (char* tok = std::strtok(p, " \t\r\n"); tok && rc == TT_OK; tok = std::strtok(nullptr, " \t\r\n")) {
+            char* eq = std::strchr(tok, '=');
+            if (!eq) { rc = TT_ERR_INVALID_ARG; break; }
+            *eq = 0;
+            const std::string key(tok);
+            const char* val = eq + 1;
+            char* end = nullptr;
+            if (key == "version") { r.version = (uint32_t)std::strtoul(val, &end, 10); have_version = true; }
+            else if (key == "family") r.family = (uint32_t)std::strtoul(val, &end, 10);
+            else if (key == "origin_op") r.origin_op = (int32_t)std::strtol(val, &end, 10);
+            else if (key == "us") t = std::strtof(val, &end);
+            else if (key == "origin") {
+                const char* q = val;
+                for (int j = 0; j < kShapeInts && rc == TT_OK; ++j) {
+                    *shape_ints(r.origin, j) = (int32_t)std::strtol(q, &end, 10);
+                    if (end == q || *end != ',') rc = TT_ERR_INVALID_ARG;
+                    q = end + 1;
+                }
+                if (rc == TT_OK) { r.origin.scale = std::strtof(q, &end); if (end == q) rc = TT_ERR_INVALID_ARG; }
+            } else {
+                bool found = false;
+                for (const RecField& rf : kRecFields)
+                    if (key == rf.name) { r.*(rf.field) = (int32_t)std::strtol(val, &end, 10); found = true; break; }
+                if (!found) rc = TT_ERR_INVALID_ARG;
+            }
+            if (rc == TT_OK && (end == val || (end && *end != 0))) rc = TT_ERR_INVALID_ARG;
+        }
+        if (rc != TT_OK) break;
+        if (!have_version || r.version != TT_RECORD_VERSION) { rc = TT_ERR_INVALID_ARG; break; }
+        if (n < cap) { out[n] = r; if (us) us[n] = t; }
+        ++n;
+    }
+    std::fclose(f);
+    *n_out = n;
+    if (rc != TT_OK) return rc;
+    return (cap && n > cap) ? TT_ERR_RESOURCE : TT_OK;
 }
 
 tt_status tt_split_check(int64_t extent, const int64_t* factors, size_t n, int32_t reformulate, int32_t* valid) {

@@ -1917,6 +1917,13 @@ __global__ void tt_repack_filters_kernel(const float* __restrict__ w, float* __r
     }
 }
 
+// A kernel that does nothing, for the launch floor: launched with a record's grid, block size, shared memory,
+// cluster shape and dependent-launch attribute, its time is what a launch of that record costs before any work.
+__global__ void tt_floor_kernel() {
+    pdl_allow_next();
+    pdl_wait_prev();
+}
+
 // ------------------------------------------------------------------------------------------------------------
 // Launchers (called from tt_device.cu)
 // ------------------------------------------------------------------------------------------------------------
@@ -1980,6 +1987,32 @@ cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits) {
     if (e != cudaSuccess) return e;
     *fits = n > 0;
     return cudaSuccess;
+}
+
+cudaError_t launch_floor(const tt_apply_info& I, int cluster, cudaStream_t st) {
+    static int attr_set_for = -1;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (attr_set_for != dev) {
+        cudaError_t e = cudaFuncSetAttribute(tt_floor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemLimit);
+        if (e != cudaSuccess) return e;
+        attr_set_for = dev;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(I.grid_x, I.grid_y, I.grid_z); cfg.blockDim = dim3(I.threads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)I.smem_bytes; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+    ++n_attr;
+    if (cluster) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = 1; attr[n_attr].val.clusterDim.y = (unsigned)cluster; attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
+    cfg.attrs = attr; cfg.numAttrs = (unsigned)n_attr;
+    return cudaLaunchKernelEx(&cfg, tt_floor_kernel);
 }
 
 cudaError_t launch_repack(const float* w, float* out, int kout, int C, int RS, int CB, cudaStream_t st) {

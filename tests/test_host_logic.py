@@ -469,3 +469,42 @@ def test_depthwise_record_naming_a_kernel_form_the_shape_lacks_is_a_reformulatio
     st, info = dw7.check(tma)
     assert st == B.TT_OK and info.legal.raster == 0 and info.changed & B.TT_CHG_FORM
     assert dw3.check(tma)[1].legal.raster == 1
+
+
+def test_pool_file_round_trip_and_rejections(tmp_path):
+    """Schedules persist as records keyed by the kernel they were tuned on (Section 2): a pool written as text reads
+    back bit for bit; a damaged line, an unknown field or another record version is refused, not guessed at."""
+    recs = W.single_conv_pool()
+    recs[2].origin.scale = 0.125
+    recs.append(B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=8, block_y=14, block_x=28, items_per_thread=4, vec_width=4, threads=256,
+                              unroll=2, raster=1, stages=2))
+    path = str(tmp_path / "pool.txt")
+    B.pool_save(path, recs, [1.5, 2.25, -1.0, 7.0, 40.5])
+    back, us = B.pool_load(path)
+    assert us == [1.5, 2.25, -1.0, 7.0, 40.5]
+    assert [bytes(r) for r in back] == [bytes(r) for r in recs]
+    B.pool_save(path, [], None)
+    assert B.pool_load(path) == ([], [])
+    good = open(str(tmp_path / "pool.txt")).read()
+    B.pool_save(path, recs[:1], None)
+    line = [l for l in open(path).read().splitlines() if not l.startswith("#")][0]
+    assert "us=-1" in line
+    for bad in (line.replace("tile_n=", "tile_q="), line.replace("version=1", "version=99"), line.replace("stages=2", "stages=two"),
+                line.replace("origin=1,", "origin=1;")):
+        with open(path, "w") as f:
+            f.write(bad + "\n")
+        n = ctypes.c_size_t()
+        assert B.lib().tt_pool_load(path.encode(), None, None, 0, ctypes.byref(n)) == B.TT_ERR_INVALID_ARG, bad
+    n = ctypes.c_size_t()
+    assert B.lib().tt_pool_load(str(tmp_path / "missing.txt").encode(), None, None, 0, ctypes.byref(n)) == B.TT_ERR_INVALID_ARG
+    del good
+
+
+def test_bench_counts_algorithmic_work_like_the_library():
+    """bench.py's reference arm counts flops and bytes from the shapes alone; they are the library's gemm view."""
+    import bench
+    for model in ("resnet18", "mobilenet_v2", "bert_base"):
+        for sp in W.MODELS[model]():
+            v = sp.workload().gemm_view()
+            f, b = bench.algorithmic_work(sp)
+            assert f == pytest.approx(v.flops) and b == pytest.approx(v.bytes), sp.name
