@@ -83,7 +83,7 @@ typedef struct tt_shapes {
     float scale;                                                   /* softmax only */
 } tt_shapes;
 
-#define TT_RECORD_VERSION 1u
+#define TT_RECORD_VERSION 2u
 
 /* A schedule record.  Correspondence with the primitives listed under Algorithm 1:
  *   Split     -> tile_m, tile_n, tile_k (CTA tile of the output and of the reduction), split_k
@@ -93,7 +93,8 @@ typedef struct tt_shapes {
  *   cache buffer / ComputeAt -> the accumulator lives in tensor memory and the bias/activation run on read-out;
  *                               `stages` shared-memory buffers decouple loading from the multiply
  *   Vectorize -> vec_width;   Unroll -> unroll / items_per_thread
- * GEMM_TC uses tile_m, tile_n, tile_k, stages, split_k, raster, mma_m_axis, slab_tiles, acc_split, k_order.
+ * GEMM_TC uses tile_m, tile_n, tile_k, stages, split_k, raster, mma_m_axis, slab_tiles, acc_split, k_order, persistent,
+ *         cta_group, ctas_per_sm, warp_layout.
  * DW_SIMT uses tile_m (channels per CTA), block_y x block_x (output rows x columns per CTA tile),
  *         items_per_thread (consecutive outputs along the width per thread), vec_width, threads, and unroll:
  *         0 = shared-memory staged kernel; 1, 2, 4 = register-window kernel with that many output rows per thread
@@ -125,6 +126,23 @@ typedef struct tt_schedule_record {
                               slab, and every tap's operand tile is a shifted view of that slab -- no expansion.
                               Stride-1 convolutions with 16-byte image rows, filters on the 128 rows, split_k = 1;
                               tile_k = 32 * (taps per pipeline stage), the tap count a divisor of r*s, at most 128. */
+    int32_t persistent;    /* GEMM_TC: 1 = the grid is one CTA (or CTA pair) per SM and every CTA walks output tiles; the
+                              operand pipeline runs on across tiles and two accumulators in tensor memory alternate, so a
+                              tile is read out (bias, activation, stores) while the next one is accumulated.  Needs
+                              split_k = 1 and operands that TMA can fetch: dense and batch_matmul with 16-byte rows, 1x1
+                              stride-1 unpadded convolutions with h*w and c multiples of 4 (an operand whose row index is
+                              the contiguous one -- the image, the second operand of an NN batch_matmul -- is staged as
+                              [tile_k][rows] boxes and transposed in shared memory).  Elsewhere legalised to 0. */
+    int32_t cta_group;     /* GEMM_TC, persistent: 2 = two CTAs of a cluster share a 256-row tile; each loads its own rows of
+                              the first operand and HALF of the second operand's rows, the multiply-accumulate runs across
+                              both SMs (tcgen05 cta_group::2).  K-major operands only, tile_n >= 32.  0 or 1 = one CTA. */
+    int32_t ctas_per_sm;   /* GEMM_TC, not persistent: 2 = the register-capped build of the kernel, so that two CTAs share an
+                              SM when the record needs at most 112 KB of shared memory and 256 tensor-memory columns (one
+                              CTA's set-up and read-out overlap the other's main loop); 1 = all registers, one CTA per SM;
+                              0 = the library's choice by grid size (2 when the grid has more than two CTAs per SM). */
+    int32_t warp_layout;   /* GEMM_TC: warps by role.  0 = the only layout of each kernel form: 1 TMA + 1 MMA + 8 operand
+                              producers that then read out (320 threads), or, persistent, 1 TMA + 1 MMA + 4 transposers + 4
+                              read-out warps.  Reserved for further layouts; any other value is invalid. */
 } tt_schedule_record;
 
 typedef struct tt_tensors {
@@ -243,6 +261,12 @@ tt_status tt_run_host(tt_workload* w, const tt_tensors* host, void* cuda_stream,
  * of that stream).  A workload owns one set of device staging buffers: enqueue its calls on one stream at a time. */
 tt_status tt_run_host_async(tt_workload* w, const tt_tensors* host, void* cuda_stream, int64_t* bytes_h2d,
                             int64_t* bytes_d2h);
+/* A promise by the caller, off by default: the w and bias tensors passed to tt_run for this workload are constants
+ * (the parameters of an inference pass) -- no kernel enqueued directly in front of the run on the same stream writes
+ * them.  A dense or conv2d kernel then requests the first tiles of w BEFORE it waits for the kernel in front of it
+ * (kernels are launched with programmatic stream serialization), so the weights stream in while that kernel is still
+ * running.  Results are unchanged as long as the promise holds.  batch_matmul operands are never treated this way. */
+tt_status tt_workload_set_constant_weights(tt_workload* w, int32_t on);
 /* Read and clear the device status word of the last runs (TT_OK or TT_ERR_TIMEOUT); synchronises the stream.
  * After a TT_ERR_TIMEOUT the split-K arrival counters of the applied record are cleared too, so the next run starts
  * from a clean workspace (an invalid pair is a result of the search, which then goes on: Section 4.3). */
@@ -311,13 +335,13 @@ tt_status tt_pool_load(const char* path, tt_schedule_record* out, float* us, siz
  * to the (legalised) start or that repeat an earlier neighbour are dropped.
  *   GEMM_TC  tile_n {16,32,48,64,96,128,160,192,224,256}  tile_k {8,16,32,64,96,128}  stages {1..8}
  *            split_k {1..8,12,16,24,32}  raster {0,1}  mma_m_axis {1,2}  slab_tiles {0,1,2,4,8}  acc_split {1,2,4,8}
- *            k_order {0,1}
+ *            k_order {0,1}  persistent {0,1}  cta_group {1,2}  ctas_per_sm {1,2}
  *   DW_SIMT  tile_m {1,2,4,8,16,32}  block_y {1,2,4,7,8,14,16,28,56}  block_x {8,16,28,32,56,64,112}
  *            items_per_thread {1,2,4,8}  vec_width {1,2,4}  threads {32,...,512}  unroll {0,1,2,4}  raster {0,1}
  *            stages {2,3,4}
  *   ROW_SIMT block_x {1,...,32}  block_y {1,...,16}  vec_width {1,2,4}
  * Pure host.  out[cap] receives the neighbours, *n_out their number (cap == 0: count only; more than cap:
- * TT_ERR_RESOURCE).  At most two per field, so 18 entries always suffice. */
+ * TT_ERR_RESOURCE).  At most two per field, so 24 entries always suffice. */
 tt_status tt_record_neighbours(const tt_workload* w, const tt_schedule_record* rec, tt_schedule_record* out, size_t cap,
                                size_t* n_out);
 

@@ -265,7 +265,7 @@ LADDERS = {
     "gemm_tc": [("tile_n", [16, 32, 48, 64, 96, 128, 160, 192, 224, 256]), ("tile_k", [8, 16, 32, 64, 96, 128]),
                 ("stages", [1, 2, 3, 4, 5, 6, 7, 8]), ("split_k", [1, 2, 3, 4, 5, 6, 7, 8, 12, 16, 24, 32]),
                 ("raster", [0, 1]), ("mma_m_axis", [1, 2]), ("slab_tiles", [0, 1, 2, 4, 8]), ("acc_split", [1, 2, 4, 8]),
-                ("k_order", [0, 1])],
+                ("k_order", [0, 1]), ("persistent", [0, 1]), ("cta_group", [1, 2]), ("ctas_per_sm", [1, 2])],
     "dw_simt": [("tile_m", [1, 2, 4, 8, 16, 32]), ("block_y", [1, 2, 4, 7, 8, 14, 16, 28, 56]),
                 ("block_x", [8, 16, 28, 32, 56, 64, 112]), ("items_per_thread", [1, 2, 4, 8]), ("vec_width", [1, 2, 4]),
                 ("threads", [32, 64, 128, 256, 512]), ("unroll", [0, 1, 2, 4]), ("raster", [0, 1]), ("stages", [2, 3, 4])],

@@ -20,7 +20,7 @@ TT_OP_CONV2D, TT_OP_DWCONV2D, TT_OP_DENSE, TT_OP_BATCH_MATMUL, TT_OP_SOFTMAX = r
 TT_ACT_NONE, TT_ACT_RELU, TT_ACT_RELU6, TT_ACT_GELU_ERF = range(4)
 TT_FAMILY_GEMM_TC, TT_FAMILY_DW_SIMT, TT_FAMILY_ROW_SIMT = range(3)
 TT_MODE_LEGALISE, TT_MODE_STRICT = 0, 1
-TT_RECORD_VERSION = 1
+TT_RECORD_VERSION = 2
 TT_CHG_TILE_M, TT_CHG_TILE_N, TT_CHG_TILE_K, TT_CHG_STAGES, TT_CHG_SPLIT_K, TT_CHG_VEC, TT_CHG_BLOCK, TT_CHG_ITEMS, TT_CHG_SLAB, TT_CHG_ACC, TT_CHG_KORDER, TT_CHG_FORM = \
     1, 2, 4, 8, 16, 32, 64, 128, 256, 512, 1024, 2048
 
@@ -36,10 +36,12 @@ class tt_shapes(C.Structure):
 class tt_schedule_record(C.Structure):
     _fields_ = [("version", u32), ("family", u32), ("origin_op", i32), ("origin", tt_shapes)] + \
                [(n, i32) for n in ("tile_m", "tile_n", "tile_k", "stages", "split_k", "raster", "block_x", "block_y",
-                                   "items_per_thread", "vec_width", "unroll", "threads", "mma_m_axis", "slab_tiles", "acc_split", "k_order")]
+                                   "items_per_thread", "vec_width", "unroll", "threads", "mma_m_axis", "slab_tiles", "acc_split", "k_order",
+                                   "persistent", "cta_group", "ctas_per_sm", "warp_layout")]
 
     FIELDS = ("tile_m", "tile_n", "tile_k", "stages", "split_k", "raster", "block_x", "block_y",
-              "items_per_thread", "vec_width", "unroll", "threads", "mma_m_axis", "slab_tiles", "acc_split", "k_order")
+              "items_per_thread", "vec_width", "unroll", "threads", "mma_m_axis", "slab_tiles", "acc_split", "k_order",
+              "persistent", "cta_group", "ctas_per_sm", "warp_layout")
 
     def as_dict(self):
         d = {"family": int(self.family), "origin_op": int(self.origin_op)}
@@ -50,7 +52,9 @@ class tt_schedule_record(C.Structure):
         if self.family == TT_FAMILY_GEMM_TC:
             return (f"tc[{self.tile_m}x{self.tile_n}x{self.tile_k} st{self.stages} sk{self.split_k} "
                     f"r{self.raster} ax{self.mma_m_axis}" + (f" sl{self.slab_tiles}" if self.slab_tiles else "") +
-                    (f" acc{self.acc_split}" if self.acc_split > 1 else "") + (" tap" if self.k_order else "") + "]")
+                    (f" acc{self.acc_split}" if self.acc_split > 1 else "") + (" tap" if self.k_order else "") +
+                    (" ps" if self.persistent else "") + (" cg2" if self.cta_group == 2 else "") +
+                    (" 2/sm" if self.ctas_per_sm == 2 else "") + "]")
         if self.family == TT_FAMILY_DW_SIMT:
             return (f"dw[c{self.tile_m} {self.block_y}x{self.block_x} it{self.items_per_thread} "
                     f"v{self.vec_width} t{self.threads} u{self.unroll}" + (f" tma st{self.stages}" if self.raster else "") + "]")
@@ -109,6 +113,7 @@ EXPORTS = {
     "tt_run_host": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "tt_run_host_async": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "tt_workload_status": (i32, [C.c_void_p, C.c_void_p]),
+    "tt_workload_set_constant_weights": (i32, [C.c_void_p, i32]),
     "tt_workload_set_wait_limit": (i32, [C.c_void_p, C.c_uint64]),
     "tt_workload_test_stall": (i32, [C.c_void_p, C.c_uint32]),
     "tt_time": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_size_t, C.c_void_p, C.POINTER(tt_timing_opts),
@@ -200,7 +205,8 @@ def make_record(family, **kw) -> tt_schedule_record:
     r.version = TT_RECORD_VERSION
     r.family = family
     defaults = dict(tile_m=128, tile_n=128, tile_k=32, stages=4, split_k=1, raster=0, block_x=32, block_y=4,
-                    items_per_thread=1, vec_width=1, unroll=1, threads=128, mma_m_axis=0, slab_tiles=0, acc_split=1, k_order=0)
+                    items_per_thread=1, vec_width=1, unroll=1, threads=128, mma_m_axis=0, slab_tiles=0, acc_split=1, k_order=0,
+                    persistent=0, cta_group=1, ctas_per_sm=0, warp_layout=0)
     defaults.update(kw)
     for k, v in defaults.items():
         setattr(r, k, v)
@@ -358,6 +364,9 @@ class Workload:
     def status(self, stream=None) -> int:
         sp = _stream() if stream is None else C.c_void_p(stream.cuda_stream)
         return lib().tt_workload_status(self.handle, sp)
+
+    def set_constant_weights(self, on: bool = True):
+        _check(lib().tt_workload_set_constant_weights(self.handle, int(bool(on))), "tt_workload_set_constant_weights")
 
     def set_wait_limit(self, nanoseconds: int):
         _check(lib().tt_workload_set_wait_limit(self.handle, int(nanoseconds)), "tt_workload_set_wait_limit")

@@ -18,6 +18,7 @@ cudaError_t launch_row(const tt_apply_info& I, const RowArgs& row, cudaStream_t 
 cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits);
 cudaError_t launch_repack(const float* w, float* out, int kout, int C, int RS, int CB, cudaStream_t st);
 cudaError_t launch_floor(const tt_apply_info& I, int cluster, cudaStream_t st);
+cudaError_t launch_gemm_ps(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, cudaStream_t st);
 
 namespace {
 
@@ -66,6 +67,24 @@ tt_status encode_operand(void* out, const float* base, int K, int rows, int batc
     CUresult r = fn(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base),
                     dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? TT_OK : TT_ERR_CUDA;
+}
+
+// Row-contiguous operand [batch][K][rows] (element (row, k) at k * ks + row) -> 3-D tensor map without swizzle,
+// box = [box_rows, box_k, 1]: the staging boxes of the persistent kernel.
+tt_status encode_operand_mn(void* out, const float* base, int rows, int K, int batch, long long ks, long long bs, bool batched,
+                            int box_rows, int box_k) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return TT_ERR_CUDA;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) != 0) return TT_ERR_INVALID_ARG;
+    const cuuint64_t nb = batched ? (cuuint64_t)batch : 1;
+    cuuint64_t dims[3] = {(cuuint64_t)rows, (cuuint64_t)K, nb};
+    cuuint64_t strides[2] = {(cuuint64_t)ks * 4, (cuuint64_t)(batched ? bs : (long long)K * ks) * 4};
+    cuuint32_t box[3] = {(cuuint32_t)box_rows, (cuuint32_t)box_k, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims,
+                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? TT_OK : TT_ERR_CUDA;
 }
 
@@ -139,7 +158,7 @@ tt_status bind_device(tt_workload* w) {
         if (cudaMalloc(reinterpret_cast<void**>(&w->status_word), 512) != cudaSuccess) { cudaGetLastError(); return TT_ERR_OOM; }
         if (cudaMemset(w->status_word, 0, 512) != cudaSuccess) return TT_ERR_CUDA;
     }
-    if (w->op == TT_OP_CONV2D && !w->plan.g.tap_major) {
+    if (w->op == TT_OP_CONV2D && !w->plan.g.tap_major && !w->plan.g.persistent) {
         // reduction-index table of the applied record: byte offset of (c, r, s) inside the slab, channel counted
         // from 0 (the kernel rebases it per chunk); indices past K point at the last channel, whose products meet
         // zero-filled filter values
@@ -182,7 +201,15 @@ static tt_status tensor_maps_for(tt_workload* w, const void* a_ptr, const void* 
     if (st != TT_OK) return st;
     if (g.b_mode == OPM_TMA)
         st = encode_operand(e.b, static_cast<const float*>(b_ptr), g.K, g.N, g.batch, g.b_rs, g.b_bs, g.b_tma_batched != 0,
-                            g.atom_k, g.tile_n);
+                            g.atom_k, g.b_rows_cta);
+    if (st != TT_OK) return st;
+    if (g.a_mode == OPM_TMA_MN)
+        st = encode_operand_mn(e.a, static_cast<const float*>(a_ptr), g.M, g.K, g.batch, g.a_ks, g.a_bs, g.a_tma_batched != 0,
+                               kHwTileM, g.tile_k);
+    if (st != TT_OK) return st;
+    if (g.b_mode == OPM_TMA_MN)
+        st = encode_operand_mn(e.b, static_cast<const float*>(b_ptr), g.N, g.K, g.batch, g.b_ks, g.b_bs, g.b_tma_batched != 0,
+                               g.b_rows_cta, g.tile_k);
     if (st != TT_OK) return st;
     if (g.slab_tma) {
         const float* img = static_cast<const float*>(g.a_mode == OPM_IM2COL ? a_ptr : b_ptr);
@@ -233,7 +260,12 @@ tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
         g.ktab_dev = w->ktab_dev;
         g.wait_ns = w->wait_ns;
         g.extra_tx = w->extra_tx;
-        e = launch_gemm(p.info, g, maps->a, maps->b, maps->x, st);
+        g.w_operand = 0;
+        if (w->constant_weights && !p.repack && (w->op == TT_OP_DENSE || w->op == TT_OP_CONV2D)) {
+            if (p.a_tensor == 1 && g.a_mode == OPM_TMA) g.w_operand = 1;
+            else if (p.b_tensor == 1 && g.b_mode == OPM_TMA) g.w_operand = 2;
+        }
+        e = g.persistent ? launch_gemm_ps(p.info, g, maps->a, maps->b, st) : launch_gemm(p.info, g, maps->a, maps->b, maps->x, st);
     } else if (w->family == TT_FAMILY_DW_SIMT) {
         DwArgs d = p.dw;
         d.x = static_cast<const float*>(t->x); d.w = static_cast<const float*>(t->w);
@@ -427,6 +459,12 @@ tt_status tt_schedule_apply_ex(tt_workload* w, const tt_schedule_record* rec, in
 
 tt_status tt_run(tt_workload* w, const tt_tensors* t, void* cuda_stream) { return launch(w, t, cuda_stream); }
 
+
+tt_status tt_workload_set_constant_weights(tt_workload* w, int32_t on) {
+    if (!w) return TT_ERR_INVALID_ARG;
+    w->constant_weights = on != 0;
+    return TT_OK;
+}
 
 tt_status tt_workload_set_wait_limit(tt_workload* w, uint64_t nanoseconds) {
     if (!w || nanoseconds == 0) return TT_ERR_INVALID_ARG;
@@ -752,7 +790,9 @@ extern "C" tt_status tt_dense_static_scratch(const void* x, const void* w, const
     wl.P = wl.Q = 0;
     wl.view = tt_gemm_view{1, m, nn, kk, 2.0 * m * (double)nn * kk, 0.0};
     Plan plan;
-    tt_status s = legalise(&wl, rec, TT_MODE_LEGALISE, 0, &plan);
+    tt_schedule_record r1 = *rec;
+    r1.persistent = 0; r1.cta_group = 1;        // the one-tile-per-CTA form: the persistent one has no split-K, hence no scratch
+    tt_status s = legalise(&wl, &r1, TT_MODE_LEGALISE, 0, &plan);
     if (s != TT_OK) return s;
     // layout of the fixed array: status word | arrival counters | partial sums
     const int64_t counters_bytes = ((int64_t)plan.info.grid_x * plan.info.grid_z * 4 + 255) / 256 * 256;
@@ -784,6 +824,7 @@ extern "C" tt_status tt_dense_static_scratch(const void* x, const void* w, const
     g.partial = reinterpret_cast<float*>(base + kStaticStatusBytes + counters_bytes);
     g.wait_ns = 1000000000ull;
     g.extra_tx = 0;
+    g.w_operand = 0;
     if ((reinterpret_cast<uintptr_t>(y) & 15u) != 0) g.vec_store = 0;
     if (g.bias && (reinterpret_cast<uintptr_t>(g.bias) & 15u) == 0) g.vec_store |= 2;
     TmapPair maps;

@@ -113,6 +113,12 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     const int tk = 32 * tps;
     if (strict && (rec->mma_m_axis == 2 || rec->tile_k != tk || rec->split_k != 1)) return TT_ERR_INVALID_SCHEDULE;
     L.mma_m_axis = 1; L.tile_m = kHwTileM; L.tile_k = tk; L.split_k = 1; L.acc_split = 1; L.slab_tiles = 0; L.k_order = 1;
+    if (rec->persistent < 0 || rec->persistent > 1 || rec->cta_group < 0 || rec->cta_group > 2 || rec->ctas_per_sm < 0 ||
+        rec->ctas_per_sm > 2 || rec->warp_layout != 0)
+        return TT_ERR_INVALID_SCHEDULE;
+    // this reduction order exists in the one-tile-per-CTA kernel only
+    L.persistent = 0; L.cta_group = 1;
+    if (rec->persistent != 0 || rec->cta_group == 2) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_FORM; }
     if (rec->tile_m != kHwTileM) changed |= TT_CHG_TILE_M;
     if (rec->tile_k != tk) changed |= TT_CHG_TILE_K;
     if (rec->split_k != 1) changed |= TT_CHG_SPLIT_K;
@@ -146,12 +152,21 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     L.stages = st;
     const long long pipe = std::max<long long>((long long)st * a_stage, min_pipe);
     const int tiles_m = (M + kHwTileM - 1) / kHwTileM, tiles_n = (N + tn - 1) / tn;
+    const int tmem_cols_t = std::max(32, pow2_ceil(tn));
+    {
+        // which build: two CTAs per SM need half the shared memory and half the tensor memory each
+        const bool fits2 = smem <= 112 * 1024 && tmem_cols_t <= 256;
+        const long long ctas = (long long)tiles_m * tiles_n * B;
+        int cps = rec->ctas_per_sm == 0 ? ((ctas > 2 * 148 && fits2) ? 2 : 1) : rec->ctas_per_sm;
+        if (cps == 2 && !fits2) { if (strict) return TT_ERR_INVALID_SCHEDULE; cps = 1; changed |= TT_CHG_FORM; }
+        L.ctas_per_sm = cps;
+    }
     I = tt_apply_info{};
     I.legal = L; I.changed = changed;
     I.grid_x = tiles_m * tiles_n; I.grid_y = 1; I.grid_z = B;
     I.threads = kGemmThreads;
     I.smem_bytes = (int)std::min<long long>(smem, 0x7fffffff);
-    I.tmem_cols = std::max(32, pow2_ceil(tn));
+    I.tmem_cols = tmem_cols_t;
     I.workspace_bytes = (int64_t)M * K * 4;              // the re-packed filters
     I.launches = 2;
     if (smem > kDynSmemLimit || (long long)tiles_m * tiles_n > 0x7fffffffLL || B > 65535) return TT_ERR_RESOURCE;
@@ -179,6 +194,8 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     g.sh = 1; g.sw = 1; g.ph = s.pad_h; g.pw = s.pad_w;
     g.vec_store = (w->Q % 4 == 0 && ((long long)w->P * w->Q) % 4 == 0) ? 1 : 0;   // a lane's four columns: one aligned 16-byte store
     g.tap_major = 1;
+    g.two_per_sm = L.ctas_per_sm == 2;
+    g.b_rows_cta = tn; g.cta_group = 1;
     g.slab_tma = 1; g.slab_tiles = RS / tps; g.slab_nbuf = 1; g.pm_nbuf = nbuf;
     g.slab_off = (unsigned)pipe; g.slab_buf_bytes = (unsigned)s_buf;
     g.slab_wp = wp; g.slab_gap = gap; g.slab_chpitch = in_rows * wp; g.slab_in_rows = in_rows; g.slab_rstep = 1;
@@ -200,7 +217,9 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     int changed = 0;
     const bool strict = mode == TT_MODE_STRICT;
     if (rec->tile_m <= 0 || rec->tile_n <= 0 || rec->tile_k <= 0 || rec->stages <= 0 || rec->split_k <= 0 ||
-        rec->raster < 0 || rec->raster > 1 || rec->mma_m_axis < 0 || rec->mma_m_axis > 2)
+        rec->raster < 0 || rec->raster > 1 || rec->mma_m_axis < 0 || rec->mma_m_axis > 2 || rec->persistent < 0 ||
+        rec->persistent > 1 || rec->cta_group < 0 || rec->cta_group > 2 || rec->ctas_per_sm < 0 || rec->ctas_per_sm > 2 ||
+        rec->warp_layout != 0)
         return TT_ERR_INVALID_SCHEDULE;
     // Which output axis becomes the accumulator's 128 rows.  Left to the library (0), the shorter-than-a-tile
     // axis goes to the MMA's N side, where 16..256 columns are legal.
@@ -236,7 +255,25 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     if (st != rec->stages) changed |= TT_CHG_STAGES;
     L.stages = st;
     const int k_tiles = (K + tk - 1) / tk;
-    int sk = rec->split_k;
+    // The persistent form: both operands must be reachable by TMA -- K-major with 16-byte rows, or row-contiguous (the
+    // image of a pointwise convolution, the second operand of an NN batch_matmul) with 16-byte row pitch.
+    bool persistent = rec->persistent == 1;
+    {
+        const tt_shapes& o = w->sh;
+        bool can = (K % 4) == 0;
+        if (w->op == TT_OP_CONV2D)
+            can = can && o.r == 1 && o.s == 1 && o.stride_h == 1 && o.stride_w == 1 && o.pad_h == 0 && o.pad_w == 0 &&
+                  ((long long)o.h * o.w) % 4 == 0;
+        else if (w->op == TT_OP_BATCH_MATMUL && !o.trans_b)
+            can = can && (o.nn % 4) == 0;
+        if (persistent && !can) { if (strict) return TT_ERR_INVALID_SCHEDULE; persistent = false; changed |= TT_CHG_FORM; }
+    }
+    const bool mn_operand = persistent && (w->op == TT_OP_CONV2D || (w->op == TT_OP_BATCH_MATMUL && !w->sh.trans_b));
+    int cg = rec->cta_group == 2 ? 2 : 1;
+    if (cg == 2 && (!persistent || mn_operand || tn < 32)) { if (strict) return TT_ERR_INVALID_SCHEDULE; cg = 1; changed |= TT_CHG_FORM; }
+    L.persistent = persistent ? 1 : 0;
+    L.cta_group = cg;
+    int sk = persistent ? 1 : rec->split_k;
     if (sk > k_tiles) {
         if (strict) return TT_ERR_INVALID_SCHEDULE;
         sk = k_tiles;
@@ -247,17 +284,99 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     L.split_k = sk;
     // accumulators: a power of two, all of them inside the 512 columns of tensor memory, none left without a step
     if (rec->acc_split < 0) return TT_ERR_INVALID_SCHEDULE;
-    int nacc = std::min(8, pow2_floor(std::max(1, rec->acc_split)));
+    int nacc = persistent ? 1 : std::min(8, pow2_floor(std::max(1, rec->acc_split)));
     while (nacc > 1 && (nacc * tn > 512 || (long long)nacc > (long long)per_split * (tk / 8))) nacc >>= 1;
     if (nacc != std::max(1, rec->acc_split)) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_ACC; }
     L.acc_split = nacc;
     // buffers beyond the reduction tiles of one CTA would never be filled
-    if (st > per_split) { st = per_split; changed |= TT_CHG_STAGES; L.stages = st; }
+    // (the persistent form's pipeline runs on across tiles: there the depth is bounded by shared memory alone)
+    if (!persistent && st > per_split) { st = per_split; changed |= TT_CHG_STAGES; L.stages = st; }
     if (strict && (changed & ~TT_CHG_TILE_M)) return TT_ERR_INVALID_SCHEDULE;
 
     const int atom_k = std::min(tk, 32), n_atoms = tk / atom_k, row_bytes = atom_k * 4;
     const unsigned a_stage = (unsigned)n_atoms * kHwTileM * row_bytes;
-    const unsigned b_stage = (unsigned)n_atoms * tn * row_bytes;
+    const unsigned b_stage = (unsigned)n_atoms * (tn / cg) * row_bytes;
+    if (persistent) {
+        // ---- the persistent form: its own shared-memory plan, grid and arguments ----
+        const tt_shapes& o = w->sh;
+        const bool conv1 = w->op == TT_OP_CONV2D, nn = w->op == TT_OP_BATCH_MATMUL && !o.trans_b;
+        // logical operands U (rows i of the output) and V (columns j): which of them is row-contiguous
+        const bool u_mn = false, v_mn = conv1 || nn;
+        const bool a_mn = swap ? v_mn : u_mn, b_mn = swap ? u_mn : v_mn;
+        const unsigned stg_a = a_mn ? (unsigned)(tk * kHwTileM * 4) : 0u, stg_b = b_mn ? (unsigned)(tk * tn * 4) : 0u;
+        const long long epi = 4ll * 32 * 36 * 4;
+        long long smem_p = 0;
+        for (;;) {
+            smem_p = (long long)st * (a_stage + b_stage + stg_a + stg_b) + epi + 1024;
+            if (smem_p <= kDynSmemLimit || strict || st <= 1) break;
+            --st; changed |= TT_CHG_STAGES;
+        }
+        L.stages = st; L.split_k = 1; L.acc_split = 1; L.slab_tiles = 0; L.ctas_per_sm = 1;
+        if (rec->ctas_per_sm == 2) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_FORM; }
+        if (strict && (changed & ~TT_CHG_TILE_M)) return TT_ERR_INVALID_SCHEDULE;
+        const int rows_m = kHwTileM * cg;
+        const int tiles_m = (M + rows_m - 1) / rows_m, tiles_n = (N + tn - 1) / tn;
+        const long long units = (long long)tiles_m * tiles_n * B;
+        if (units > 0x7fffffffLL) return TT_ERR_RESOURCE;
+        I = tt_apply_info{};
+        I.legal = L; I.changed = changed;
+        I.grid_x = (int)std::min<long long>(units, 148 / cg) * cg; I.grid_y = 1; I.grid_z = 1;   // the launcher clamps to the device's SM count
+        I.threads = kGemmThreads;
+        // one CTA per SM: ask for more than half of an SM's shared memory
+        I.smem_bytes = (int)std::max<long long>(smem_p, 116 * 1024);
+        I.tmem_cols = std::max(32, pow2_ceil(2 * tn));
+        I.workspace_bytes = 0; I.launches = 1;
+        plan->partial_bytes = 0;
+        if (smem_p > kDynSmemLimit) return TT_ERR_RESOURCE;
+        GemmArgs& g = plan->g;
+        g = GemmArgs{};
+        g.M = M; g.N = N; g.K = K; g.batch = B;
+        g.tile_n = tn; g.tile_k = tk; g.stages = st;
+        g.k_tiles = k_tiles; g.k_tiles_per_split = k_tiles; g.split_k = 1;
+        g.tiles_m = tiles_m; g.tiles_n = tiles_n; g.raster = L.raster;
+        g.atom_k = atom_k; g.n_atoms = n_atoms; g.row_bytes = row_bytes;
+        g.swz_mask = row_bytes == 128 ? 7 : (row_bytes == 64 ? 3 : 1);
+        g.a_stage_bytes = a_stage; g.b_stage_bytes = b_stage;
+        g.tmem_cols = (unsigned)I.tmem_cols; g.n_acc = 1; g.cluster = 0;
+        g.idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(tn >> 3) << 17) | ((unsigned)(rows_m >> 4) << 24);
+        g.persistent = 1; g.cta_group = cg; g.total_tiles = (int)units;
+        g.a_mn = a_mn; g.b_mn = b_mn; g.b_rows_cta = tn / cg;
+        g.a_stg_off = (unsigned)((long long)st * (a_stage + b_stage));
+        g.b_stg_off = g.a_stg_off + (unsigned)st * stg_a;
+        g.stg_a_bytes = stg_a; g.stg_b_bytes = stg_b;
+        g.epi_off = g.b_stg_off + (unsigned)st * stg_b;
+        struct Opnd { int mode; long long rs, ks, bs; int batched; } U{}, V{};
+        long long y_is, y_js, y_bs;
+        int bias_on;
+        if (conv1) {
+            const long long hw = (long long)o.h * o.w;
+            U = {OPM_TMA, K, 1, 0, 0};                              // filters [k][c]
+            V = {OPM_TMA_MN, 1, hw, (long long)o.c * hw, 1};        // image: pixel index contiguous, channels hw apart
+            y_is = hw; y_js = 1; y_bs = (long long)o.k * hw; bias_on = 1;
+        } else if (w->op == TT_OP_DENSE) {
+            U = {OPM_TMA, K, 1, 0, 0};
+            V = {OPM_TMA, K, 1, 0, 0};
+            y_is = o.nn; y_js = 1; y_bs = 0; bias_on = 2;
+        } else {
+            U = {OPM_TMA, K, 1, (long long)o.m * K, 1};
+            if (o.trans_b) V = {OPM_TMA, K, 1, (long long)o.nn * K, 1};
+            else V = {OPM_TMA_MN, 1, o.nn, (long long)o.nn * K, 1};
+            y_is = o.nn; y_js = 1; y_bs = (long long)o.m * o.nn; bias_on = 2;
+        }
+        const int u_tensor = conv1 ? 1 : 0;
+        plan->a_tensor = swap ? 1 - u_tensor : u_tensor;
+        plan->b_tensor = 1 - plan->a_tensor;
+        const Opnd& A = swap ? V : U;
+        const Opnd& Bo = swap ? U : V;
+        g.a_mode = A.mode; g.a_rs = A.rs; g.a_ks = A.ks; g.a_bs = A.bs; g.a_tma_batched = A.batched;
+        g.b_mode = Bo.mode; g.b_rs = Bo.rs; g.b_ks = Bo.ks; g.b_bs = Bo.bs; g.b_tma_batched = Bo.batched;
+        g.y_ms = swap ? y_js : y_is; g.y_ns = swap ? y_is : y_js; g.y_bs = y_bs;
+        g.bias_mode = o.has_bias ? (swap ? 3 - bias_on : bias_on) : 0;
+        g.act = o.act;
+        g.tx_bytes = (a_mn ? 0 : a_stage) + (b_mn ? 0 : b_stage);
+        g.vec_store = (g.y_ns == 1 && g.y_ms % 4 == 0 && g.y_bs % 4 == 0) ? 1 : 0;
+        return TT_OK;
+    }
     // Shared memory: pipeline buffers (reused by the epilogue as a 32 x 36-float staging area per warp), then for
     // conv2d the k-table (one word per reduction index of a CTA's K range) and the slab of input rows from which
     // the im2col operand is expanded; 1 KB of alignment slack.
@@ -351,6 +470,14 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     const int tiles_m = (M + kHwTileM - 1) / kHwTileM, tiles_n = (N + tn - 1) / tn;
     if ((long long)tiles_m * tiles_n > 0x7fffffffLL || sk > 65535 || B > 65535) return TT_ERR_RESOURCE;
 
+    {
+        // which build: two CTAs per SM need half the shared memory and half the tensor memory each
+        const bool fits2 = smem <= 112 * 1024 && tmem_cols <= 256;
+        const long long ctas = (long long)tiles_m * tiles_n * sk * B;
+        int cps = rec->ctas_per_sm == 0 ? ((ctas > 2 * 148 && fits2) ? 2 : 1) : rec->ctas_per_sm;
+        if (cps == 2 && !fits2) { if (strict) return TT_ERR_INVALID_SCHEDULE; cps = 1; changed |= TT_CHG_FORM; }
+        L.ctas_per_sm = cps;
+    }
     I = tt_apply_info{};
     I.legal = L;
     I.changed = changed;
@@ -395,6 +522,8 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     g.tmem_cols = (unsigned)tmem_cols;
     g.n_acc = nacc;
     g.cluster = cluster;
+    g.two_per_sm = L.ctas_per_sm == 2;
+    g.b_rows_cta = tn; g.cta_group = 1;
     // Instruction descriptor, kind::tf32: D = F32 (bits 4-5 = 1), A and B = TF32 (bits 7-9, 10-12 = 2), both
     // K-major (bits 15, 16 = 0), N >> 3 at bits 17-22, M >> 4 at bits 24-28.
     g.idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(tn >> 3) << 17) | ((unsigned)(kHwTileM >> 4) << 24);
@@ -714,6 +843,7 @@ tt_status tt_default_schedule(const tt_workload* w, tt_schedule_record* out) {
     r.origin = w->sh;
     // One generic, shape-blind record per family: the counterpart of a compiler's default schedule.
     r.tile_m = 128; r.tile_n = 128; r.tile_k = 32; r.stages = 4; r.split_k = 1; r.raster = 0; r.acc_split = 1;
+    r.cta_group = 1;
     r.block_x = 32; r.block_y = 4; r.items_per_thread = 1; r.vec_width = 1; r.unroll = 1; r.threads = 128;
     if (w->family == TT_FAMILY_DW_SIMT) { r.tile_m = 1; r.block_x = 32; r.block_y = 8; r.items_per_thread = 4; r.unroll = 2; }
     if (w->family == TT_FAMILY_ROW_SIMT) { r.block_x = 8; r.block_y = 16; r.vec_width = 4; }
@@ -748,6 +878,9 @@ const std::vector<FieldLadder>& ladders_of(uint32_t family) {
         {&tt_schedule_record::slab_tiles, {0, 1, 2, 4, 8}},
         {&tt_schedule_record::acc_split, {1, 2, 4, 8}},
         {&tt_schedule_record::k_order, {0, 1}},
+        {&tt_schedule_record::persistent, {0, 1}},
+        {&tt_schedule_record::cta_group, {1, 2}},
+        {&tt_schedule_record::ctas_per_sm, {1, 2}},
     };
     static const std::vector<FieldLadder> dw = {
         {&tt_schedule_record::tile_m, {1, 2, 4, 8, 16, 32}},
@@ -855,6 +988,8 @@ const RecField kRecFields[] = {
     {"unroll", &tt_schedule_record::unroll}, {"threads", &tt_schedule_record::threads},
     {"mma_m_axis", &tt_schedule_record::mma_m_axis}, {"slab_tiles", &tt_schedule_record::slab_tiles},
     {"acc_split", &tt_schedule_record::acc_split}, {"k_order", &tt_schedule_record::k_order},
+    {"persistent", &tt_schedule_record::persistent}, {"cta_group", &tt_schedule_record::cta_group},
+    {"ctas_per_sm", &tt_schedule_record::ctas_per_sm}, {"warp_layout", &tt_schedule_record::warp_layout},
 };
 int32_t* shape_ints(tt_shapes& s, int i) {
     int32_t* f[] = {&s.n, &s.c, &s.h, &s.w, &s.k, &s.r, &s.s, &s.stride_h, &s.stride_w, &s.pad_h, &s.pad_w,

@@ -21,8 +21,10 @@ enum OperandMode : int {
     OPM_GATHER_ROWS = 1,  // strided view, lanes walk rows (row stride 1): 16-byte swizzled stores
     OPM_GATHER_K = 2,     // strided view, lanes walk k (k stride 1): 4-byte swizzled stores
     OPM_IM2COL = 3,       // rows are output pixels, k = (c, r, s): expanded from a slab of NCHW input rows
-    OPM_IM2COL_T = 4      // rows are padded-linear output pixels, k = (32-channel block, tap, channel): every tap's tile
+    OPM_IM2COL_T = 4,     // rows are padded-linear output pixels, k = (32-channel block, tap, channel): every tap's tile
                           // is a shifted view of a pixel-major slab in shared memory (nothing is staged per tile)
+    OPM_TMA_MN = 5        // persistent kernel: the row index is the contiguous one in memory; [tile_k][rows] boxes arrive by
+                          // TMA in a staging ring and are transposed into the K-major stage by four warps
 };
 
 // Device-side arguments of the GEMM_TC kernel (plain data, passed by value).
@@ -71,6 +73,17 @@ struct GemmArgs {
     const int* ktab_dev;                        // per reduction index: byte offset of (c, r, s) inside the slab (absolute channel)
     unsigned long long wait_ns;                 // limit of every bounded wait inside the kernel
     unsigned extra_tx;                          // test facility: bytes added to what the first stage's barrier expects
+    int w_operand;                              // 1 / 2: operand A / B is constant (weights the caller promised nobody is
+                                                // writing): its first stages are requested before the wait on the kernel in front
+    int two_per_sm;                             // the register-capped build, so that two CTAs share an SM
+    // persistent kernel (record field persistent = 1)
+    int persistent, cta_group;
+    int total_tiles;                            // tiles_m * tiles_n * batch; tiles_m counts 128 * cta_group rows
+    int a_mn, b_mn;                             // operand arrives as [tile_k][rows] boxes and is transposed in shared memory
+    int b_rows_cta;                             // rows of operand B one CTA loads: tile_n / cta_group
+    unsigned a_stg_off, b_stg_off;              // staging rings: byte offsets from the aligned tile base
+    unsigned stg_a_bytes, stg_b_bytes;          // ... and bytes per stage
+    unsigned epi_off;                           // read-out staging area (one 32 x 36-float block per read-out warp)
 };
 
 struct DwArgs {
@@ -133,6 +146,7 @@ struct tt_workload {
     unsigned* status_word = nullptr;  // device
     unsigned long long wait_ns = 1000000000ull;   // one second per wait inside a kernel, then the kernel gives up
     unsigned extra_tx = 0;            // test facility (tt_workload_test_stall)
+    bool constant_weights = false;    // the caller's promise of tt_workload_set_constant_weights
     // device staging buffers of tt_run_host
     void* hbuf[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     size_t hbytes[5] = {0, 0, 0, 0, 0};

@@ -37,6 +37,10 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// Raise the byte count the barrier's current phase expects, without arriving on it.
+__device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -780,19 +784,43 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     // run while the previous kernel of the stream is still draining; from here on its results are needed.  The
     // kernel that follows this one was allowed to start its own set-up at this kernel's entry.  (Without the launch
     // attribute both instructions do nothing.)
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // (The TMA warp waits a little later: it first requests the constant operand's first stages, see below.)
+    if (warp != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // Warps 0 and 1 run their loops with all 32 lanes: waits, counters and descriptor arithmetic stay
     // warp-uniform, and one elected lane issues the asynchronous instructions.
     if (warp == 0) {
         // ---------------- TMA producer ----------------
+        const bool leader = elect_one();                 // this lane arms the barriers and issues every load
+        const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes), b_atom = (uint32_t)(g.tile_n * g.row_bytes);
+        const int a_bz = g.a_tma_batched ? bz : 0, b_bz = g.b_tma_batched ? bz : 0;
+        // Constant operand (the caller promised that the weights are not written by the kernel in front of this one): its
+        // tiles for the first pipeline stages are requested before the wait on that kernel, so they stream in while
+        // it is still running.  The barrier only learns of the bytes here; the arrival comes with the stage's other operand.
+        int n_pref = 0;
+        if (g.w_operand) {
+            n_pref = min(g.stages, iters);
+            if (leader) {
+                int kc0 = kt_begin * g.tile_k;
+                for (int it = 0; it < n_pref; ++it, kc0 += g.tile_k) {
+                    const uint32_t bar = smem_u32(&full_bar[it]);
+                    uint32_t dst = tiles_base + (uint32_t)it * stage_bytes + (g.w_operand == 2 ? g.a_stage_bytes : 0u);
+                    mbar_expect_tx_only(bar, g.w_operand == 2 ? g.b_stage_bytes : g.a_stage_bytes);
+                    int kc = kc0;
+#pragma unroll 1
+                    for (int at = 0; at < g.n_atoms; ++at, kc += g.atom_k) {
+                        if (g.w_operand == 1) { tma_load_3d(dst, &tmap_a, bar, kc, m0, a_bz); dst += a_atom; }
+                        else { tma_load_3d(dst, &tmap_b, bar, kc, n0, b_bz); dst += b_atom; }
+                    }
+                }
+            }
+            __syncwarp();
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         if (any_tma || slab_tma) {
-            int armed = 0;   // stages whose loads were issued
+            int armed = n_pref;   // stages whose loads were issued
             uint32_t st = 0, ph = 0;
             const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
-            const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes), b_atom = (uint32_t)(g.tile_n * g.row_bytes);
-            const int a_bz = g.a_tma_batched ? bz : 0, b_bz = g.b_tma_batched ? bz : 0;
-            const bool leader = elect_one();             // this lane arms the barriers and issues every load
             int k0 = kt_begin * g.tile_k;
             uint32_t a_stage = tiles_base, full_addr = full0, empty_addr = empty0;
             // conv2d: slab chunk j (the input rows behind reduction tiles j*T .. j*T+T-1) goes to buffer j & 1 as one
@@ -833,14 +861,16 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 if (leader) {
                     // (test facility: split 0 may be told to expect more than arrives, see tt_workload_test_stall)
-                    mbar_expect_tx(full_addr, g.tx_bytes + ((it == 0 && split == 0) ? g.extra_tx : 0u));
-                    if (a_tma) {
+                    const bool a_here = a_tma && !(it < n_pref && g.w_operand == 1), b_here = b_tma && !(it < n_pref && g.w_operand == 2);
+                    mbar_expect_tx(full_addr, (a_here ? g.a_stage_bytes : 0u) + (b_here ? g.b_stage_bytes : 0u) +
+                                                  ((it == 0 && split == 0) ? g.extra_tx : 0u));
+                    if (a_here) {
                         uint32_t dst = a_stage;
                         int kc = k0;
 #pragma unroll 1
                         for (int at = 0; at < g.n_atoms; ++at, dst += a_atom, kc += g.atom_k) tma_load_3d(dst, &tmap_a, full_addr, kc, m0, a_bz);
                     }
-                    if (b_tma) {
+                    if (b_here) {
                         uint32_t dst = a_stage + g.a_stage_bytes;
                         int kc = k0;
 #pragma unroll 1
@@ -848,7 +878,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                 }
                 __syncwarp();
-                armed = it + 1;
+                armed = max(armed, it + 1);
                 a_stage += stage_bytes; full_addr += 8u; empty_addr += 8u;
                 if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; a_stage = tiles_base; full_addr = full0; empty_addr = empty0; }
             }
@@ -1419,6 +1449,453 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------------------------
+// GEMM_TC, persistent form (record field `persistent` = 1).  grid = resident CTAs; every CTA walks output tiles
+// t = unit, unit + units, ... (a unit is a CTA, or a pair of CTAs when CG = 2) with
+//   - the operand pipeline running on across tile boundaries (the loads of the next tile are in flight while this
+//     tile's last multiply-accumulates run),
+//   - TWO accumulators in tensor memory, used alternately: the read-out warps drain tile t (bias, activation,
+//     stores) while the MMA warp already accumulates tile t + 1,
+//   - barriers and tensor memory set up once per CTA instead of once per tile.
+// Operands: K-major tensors arrive by TMA straight into the swizzled pipeline stage.  Operands whose ROW index is
+// the contiguous one in memory (the image of a 1x1 convolution: pixels; the second operand of an NN batch_matmul)
+// arrive by TMA as [tile_k][rows] boxes in a staging ring and four warps transpose them into the K-major stage
+// (kind::tf32 has no MN-major operands on this part).  No split-K, one accumulator per tile.
+// Warps: 0 TMA producer, 1 MMA issuer + tensor-memory owner, 2-5 transposers, 6-9 read-out.
+// CG = 2: two CTAs of a cluster work on one 256-row tile.  Each loads its own 128 rows of A and its half of B's
+// rows with ordinary (non-multicast) TMA; the CTA of rank 0 issues tcgen05.mma.cta_group::2, which reads both
+// CTAs' shared memory and writes each CTA's half of the accumulator into that CTA's tensor memory, so an SM reads
+// only half of B per multiply-accumulate.  The rank-1 CTA's warp 1 relays "my stage has landed" to rank 0; a
+// multicast tcgen05.commit frees the stage and publishes the accumulator in both CTAs.
+// ------------------------------------------------------------------------------------------------------------
+template <int CG>
+__device__ __forceinline__ void mma_tf32_cg(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    if constexpr (CG == 1) {
+        mma_tf32(d_tmem, adesc, bdesc, idesc, accumulate);
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+    }
+}
+// Arrive on the barrier at this shared-memory offset once every MMA issued so far has completed: in this CTA (CG 1),
+// or in both CTAs of the pair (CG 2; the arrival is multicast, no data moves).
+template <int CG>
+__device__ __forceinline__ void mma_commit_cg(uint32_t bar) {
+    if constexpr (CG == 1) {
+        mma_commit(bar);
+    } else {
+        const uint16_t mask = 3;
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"(mask) : "memory");
+    }
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Arrive on the barrier at the same offset in the CTA of rank `rank` of this cluster.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank) {
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+        ::"r"(bar), "r"(rank) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait on a barrier that CTAs of the cluster arrive on (acquire at cluster scope).
+__device__ __noinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
+                                               unsigned where, unsigned long long limit_ns) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    unsigned spins = 0;
+    for (;;) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((++spins & 31u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > limit_ns) {
+                *abort_flag = 1;
+                atomicCAS(status, 0u, (unsigned)TT_ERR_TIMEOUT | (where << 8));
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_3d_plain(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2) {
+    tma_load_3d(dst, tmap, bar, c0, c1, c2);
+}
+
+constexpr int kPsTransposeWarps = 4;
+constexpr int kPsEpilogueWarps = 4;
+
+// Transpose one staged box [tile_k][rows] (row index contiguous) into the K-major swizzled stage tile.  A task is a
+// (32-row block, four consecutive reduction indices) pair: lanes walk rows (conflict-free 4-byte loads), each lane
+// assembles its row's four values and writes one 16-byte chunk.
+__device__ __forceinline__ void ps_transpose(uint32_t stg, uint32_t tile, int rows, int tile_k, int atom_k, int row_bytes,
+                                             int swz_mask, int tw, int lane) {
+    const int atom_shift = atom_k == 32 ? 5 : (atom_k == 16 ? 4 : 3);
+    const int shift = row_bytes == 128 ? 0 : (row_bytes == 64 ? 1 : 2);
+    const uint32_t atom_bytes = (uint32_t)rows * (uint32_t)row_bytes;
+    const int n_rb = (rows + 31) >> 5, n_ch = tile_k >> 2;
+    const int n_tasks = n_rb * n_ch;
+    constexpr int kBatch = 4;
+    for (int t0 = tw; t0 < n_tasks; t0 += kPsTransposeWarps * kBatch) {
+        float val[kBatch][4];
+        uint32_t dst[kBatch];
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+            const int t = t0 + b * kPsTransposeWarps;
+            const bool live = t < n_tasks;                   // warp-uniform
+            const int tt = live ? t : 0;
+            const int ci = tt / n_rb, rb = tt - ci * n_rb;
+            const int kk = ci << 2;
+            const int row = rb * 32 + lane;
+            const bool in_tile = live && row < rows;
+            dst[b] = in_tile ? tile + (uint32_t)(kk >> atom_shift) * atom_bytes + (uint32_t)row * (uint32_t)row_bytes +
+                                   ((uint32_t)((kk & (atom_k - 1)) << 2) ^ ((uint32_t)((row >> shift) & swz_mask) << 4))
+                             : 0xffffffffu;
+            const uint32_t src = stg + 4u * (uint32_t)(kk * rows + (row < rows ? row : rows - 1));
+            val[b][0] = ld_shared_f32(src);
+            val[b][1] = ld_shared_f32(src + 4u * (uint32_t)rows);
+            val[b][2] = ld_shared_f32(src + 8u * (uint32_t)rows);
+            val[b][3] = ld_shared_f32(src + 12u * (uint32_t)rows);
+        }
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b)
+            if (dst[b] != 0xffffffffu) st_shared_v4(dst[b], val[b][0], val[b][1], val[b][2], val[b][3]);
+    }
+}
+
+template <int CG>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const GemmArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[kMaxStages];     // a stage's operands are in place (TMA bytes and/or the transposer warps)
+    __shared__ uint64_t empty_bar[kMaxStages];    // every multiply-accumulate that reads the stage has completed
+    __shared__ uint64_t stg_full[kMaxStages];     // a staging box has landed
+    __shared__ uint64_t stg_empty[kMaxStages];    // the transposer warps are done with it
+    __shared__ uint64_t peer_full[kMaxStages];    // CG 2, rank 0: the rank-1 CTA's stage is in place
+    __shared__ uint64_t acc_full[2];              // an accumulator holds a finished tile
+    __shared__ uint64_t acc_empty[2];             // the read-out warps (of both CTAs) have drained it
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ __align__(16) float s_bias[2][256];
+
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
+    volatile int* abortp = &abort_flag;
+    pdl_allow_next();
+    const uint32_t rank = CG == 2 ? cluster_ctarank() : 0u;
+    const int unit = (int)blockIdx.x / CG, n_units = (int)gridDim.x / CG;
+    const int my_tiles = g.total_tiles > unit ? (g.total_tiles - unit + n_units - 1) / n_units : 0;
+    const int tiles_per_batch = g.tiles_m * g.tiles_n;
+    const int kt_n = g.k_tiles;
+
+    const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t stage_bytes = g.a_stage_bytes + g.b_stage_bytes;
+    const bool a_mn = g.a_mn != 0, b_mn = g.b_mn != 0;
+    const bool any_mn = a_mn || b_mn, any_km = !a_mn || !b_mn;
+    const int b_rows = g.b_rows_cta;
+
+    if (threadIdx.x == 32) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+    }
+    if (threadIdx.x == 0) {
+        const uint32_t full_count = (any_km ? 1u : 0u) + (any_mn ? (uint32_t)kPsTransposeWarps : 0u);
+        for (int s = 0; s < g.stages; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), full_count);
+            mbar_init(smem_u32(&empty_bar[s]), 1u);
+            mbar_init(smem_u32(&stg_full[s]), 1u);
+            mbar_init(smem_u32(&stg_empty[s]), (uint32_t)kPsTransposeWarps);
+            mbar_init(smem_u32(&peer_full[s]), 1u);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&acc_full[a]), 1u);
+            mbar_init(smem_u32(&acc_empty[a]), (uint32_t)(kPsEpilogueWarps * CG));
+        }
+        abort_flag = 0;
+        fence_mbar_init();
+        fence_proxy_async_shared();
+    }
+    if (warp == 1) {
+        if constexpr (CG == 1) {
+            tmem_alloc(smem_u32(&tmem_slot), g.tmem_cols);
+            tmem_relinquish();
+        } else {
+            // both CTAs of the pair allocate, with the same warp and the same destination offset
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(g.tmem_cols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if constexpr (CG == 2) cluster_sync_all();           // the peer's barriers exist before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem_base = *(volatile uint32_t*)&tmem_slot;
+    pdl_wait_prev();                                      // the set-up above touched no global memory
+
+    auto decode = [&](int i, int& m0, int& n0, int& bz) {
+        const int t = unit + i * n_units;
+        bz = t / tiles_per_batch;
+        const int r = t - bz * tiles_per_batch;
+        int tm, tn;
+        if (g.raster == 0) { tm = r % g.tiles_m; tn = r / g.tiles_m; }
+        else               { tn = r % g.tiles_n; tm = r / g.tiles_n; }
+        m0 = (tm * CG + (int)rank) * kHwTileM;
+        n0 = tn * g.tile_n;
+    };
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        const bool leader = elect_one();
+        const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes), b_atom = (uint32_t)(b_rows * g.row_bytes);
+        const uint32_t km_bytes = (a_mn ? 0u : g.a_stage_bytes) + (b_mn ? 0u : g.b_stage_bytes);
+        const uint32_t mn_bytes = (a_mn ? g.stg_a_bytes : 0u) + (b_mn ? g.stg_b_bytes : 0u);
+        uint32_t st = 0, ph = 0;
+        long long issued = 0;
+        bool ok = true;
+        for (int i = 0; i < my_tiles && ok; ++i) {
+            int m0, n0, bz;
+            decode(i, m0, n0, bz);
+            const int nb0 = n0 + (int)rank * b_rows;          // CG 2: this CTA's half of the B rows
+            const int a_bz = g.a_tma_batched ? bz : 0, b_bz = g.b_tma_batched ? bz : 0;
+            int k0 = 0;
+            for (int kt = 0; kt < kt_n; ++kt, k0 += g.tile_k) {
+                if (any_mn) {
+                    const bool got = mbar_wait(smem_u32(&stg_empty[st]), ph ^ 1u, abortp, g.status, 11u, g.wait_ns);
+                    if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+                    if (leader) {
+                        const uint32_t bar = smem_u32(&stg_full[st]);
+                        mbar_expect_tx(bar, mn_bytes);
+                        if (a_mn) tma_load_3d(tiles_base + g.a_stg_off + st * g.stg_a_bytes, &tmap_a, bar, m0, k0, a_bz);
+                        if (b_mn) tma_load_3d(tiles_base + g.b_stg_off + st * g.stg_b_bytes, &tmap_b, bar, nb0, k0, b_bz);
+                    }
+                }
+                if (any_km) {
+                    const bool got = mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, abortp, g.status, 1u, g.wait_ns);
+                    if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+                    if (leader) {
+                        const uint32_t bar = smem_u32(&full_bar[st]);
+                        // (test facility: the first stage may be told to expect more than arrives, see tt_workload_test_stall)
+                        mbar_expect_tx(bar, km_bytes + (issued == 0 ? g.extra_tx : 0u));
+                        const uint32_t a_dst = tiles_base + st * stage_bytes;
+                        if (!a_mn) {
+                            uint32_t dst = a_dst;
+                            int kc = k0;
+#pragma unroll 1
+                            for (int at = 0; at < g.n_atoms; ++at, dst += a_atom, kc += g.atom_k) tma_load_3d(dst, &tmap_a, bar, kc, m0, a_bz);
+                        }
+                        if (!b_mn) {
+                            uint32_t dst = a_dst + g.a_stage_bytes;
+                            int kc = k0;
+#pragma unroll 1
+                            for (int at = 0; at < g.n_atoms; ++at, dst += b_atom, kc += g.atom_k) tma_load_3d(dst, &tmap_b, bar, kc, nb0, b_bz);
+                        }
+                    }
+                }
+                __syncwarp();
+                ++issued;
+                if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
+            }
+        }
+        if ((!ok || *abortp) && lane == 0) {
+            // let copies in flight land before shared memory is given back (bounded)
+            const long long first = issued > g.stages ? issued - g.stages : 0;
+            for (long long it = first; it < issued; ++it) {
+                const int s = (int)(it % g.stages);
+                const uint32_t par = (uint32_t)(it / g.stages) & 1u;
+                const unsigned long long t0 = global_timer_ns();
+                if (any_km) while (!mbar_try_wait(smem_u32(&full_bar[s]), par)) { if (global_timer_ns() - t0 > 2000000ull) break; }
+                if (any_mn) while (!mbar_try_wait(smem_u32(&stg_full[s]), par)) { if (global_timer_ns() - t0 > 4000000ull) break; }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (rank 0 of a pair), or the relay of "my stage has landed" (rank 1) ----------------
+        const bool leader = elect_one();
+        uint32_t st = 0, ph = 0;
+        bool ok = true;
+        if (CG == 2 && rank != 0) {
+            for (int i = 0; i < my_tiles && ok; ++i)
+                for (int kt = 0; kt < kt_n; ++kt) {
+                    const bool got = mbar_wait(smem_u32(&full_bar[st]), ph, abortp, g.status, 2u, g.wait_ns);
+                    if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+                    if (leader) mbar_arrive_remote(smem_u32(&peer_full[st]), 0u);
+                    __syncwarp();
+                    if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
+                }
+        } else {
+            const uint64_t d0 = make_desc(0u, g.row_bytes);
+            const uint32_t d_hi = (uint32_t)(d0 >> 32), d_lo = (uint32_t)d0;
+            const uint32_t a_lo0 = d_lo + ((tiles_base & 0x3FFFFu) >> 4);
+            const uint32_t stage_step = stage_bytes >> 4;
+            const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes) >> 4, b_atom = (uint32_t)(b_rows * g.row_bytes) >> 4;
+            const uint32_t b_off = g.a_stage_bytes >> 4;
+            for (int i = 0; i < my_tiles && ok; ++i) {
+                const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
+                // the read-out of the tile that used this accumulator two tiles ago has finished
+                const bool freed = CG == 2 ? mbar_wait_cluster(smem_u32(&acc_empty[acc]), aph ^ 1u, abortp, g.status, 12u, g.wait_ns)
+                                           : mbar_wait(smem_u32(&acc_empty[acc]), aph ^ 1u, abortp, g.status, 12u, g.wait_ns);
+                if (!__all_sync(0xffffffffu, freed)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)g.tile_n;
+                for (int kt = 0; kt < kt_n; ++kt) {
+                    bool got = mbar_wait(smem_u32(&full_bar[st]), ph, abortp, g.status, 2u, g.wait_ns);
+                    if (CG == 2 && got) got = mbar_wait_cluster(smem_u32(&peer_full[st]), ph, abortp, g.status, 13u, g.wait_ns);
+                    if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+                    tc_fence_after();
+                    if (leader) {
+                        const uint32_t a_lo = a_lo0 + st * stage_step, b_lo = a_lo + b_off;
+                        const uint32_t accumulate = kt > 0 ? 1u : 0u;
+#pragma unroll 1
+                        for (int at = 0; at < g.n_atoms; ++at) {
+                            const int k8n = g.atom_k >> 3;
+#pragma unroll 4
+                            for (int k8 = 0; k8 < k8n; ++k8)
+                                mma_tf32_cg<CG>(d_tmem, ((uint64_t)d_hi << 32) | (uint64_t)(a_lo + (uint32_t)at * a_atom + 2u * (uint32_t)k8),
+                                                ((uint64_t)d_hi << 32) | (uint64_t)(b_lo + (uint32_t)at * b_atom + 2u * (uint32_t)k8), g.idesc,
+                                                (at == 0 && k8 == 0) ? accumulate : 1u);
+                        }
+                        mma_commit_cg<CG>(smem_u32(&empty_bar[st]));          // stage reusable once these MMAs have read it
+                    }
+                    __syncwarp();
+                    if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
+                }
+                if (ok && leader) mma_commit_cg<CG>(smem_u32(&acc_full[acc]));   // the tile's accumulator is complete
+                __syncwarp();
+            }
+        }
+    } else if (warp < 2 + kPsTransposeWarps) {
+        // ---------------- transposers ----------------
+        if (any_mn) {
+            const int tw = warp - 2;
+            uint32_t st = 0, ph = 0;
+            bool ok = true;
+            for (int i = 0; i < my_tiles && ok; ++i)
+                for (int kt = 0; kt < kt_n; ++kt) {
+                    if (!mbar_wait(smem_u32(&stg_full[st]), ph, abortp, g.status, 6u, g.wait_ns) ||
+                        !mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, abortp, g.status, 3u, g.wait_ns)) { ok = false; break; }
+                    const uint32_t a_s = tiles_base + st * stage_bytes, b_s = a_s + g.a_stage_bytes;
+                    if (a_mn) ps_transpose(tiles_base + g.a_stg_off + st * g.stg_a_bytes, a_s, kHwTileM, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, tw, lane);
+                    if (b_mn) ps_transpose(tiles_base + g.b_stg_off + st * g.stg_b_bytes, b_s, b_rows, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, tw, lane);
+                    fence_proxy_async_shared();          // generic-proxy stores -> visible to the tensor core's reads
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(smem_u32(&full_bar[st]));
+                        mbar_arrive(smem_u32(&stg_empty[st]));
+                    }
+                    if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
+                }
+        }
+    } else {
+        // ---------------- read-out: tensor memory -> bias, residual, activation -> global memory ----------------
+        const int ew = warp - (2 + kPsTransposeWarps);
+        const int et = (int)threadIdx.x - 32 * (2 + kPsTransposeWarps);
+        const int quad = warp & 3;                       // tensor-memory lane quadrant this warp may read
+        EpiArgs e;
+        e.y_ms = g.y_ms; e.y_ns = g.y_ns; e.M = g.M;
+        e.lo = g.act == TT_ACT_NONE || g.act == TT_ACT_GELU_ERF ? -INFINITY : 0.f;
+        e.hi = g.act == TT_ACT_RELU6 ? 6.f : INFINITY;
+        e.gelu = g.act == TT_ACT_GELU_ERF;
+        e.vec = (g.vec_store & 1) != 0;
+        e.lin_wp = 0; e.lin_q = 0; e.lin_p = 0;
+        const bool transposed = g.y_ns == 1 && g.y_ms != 1;
+        const uint32_t stg = tiles_base + g.epi_off + (uint32_t)ew * (uint32_t)kStageBytesPerWarp;
+        bool ok = true;
+        for (int i = 0; i < my_tiles && ok; ++i) {
+            int m0, n0, bz;
+            decode(i, m0, n0, bz);
+            const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
+            const int m_first = m0 + quad * 32, m = m_first + lane;
+            // this tile's bias values, staged while the tile is still being accumulated (the buffer's previous readers
+            // finished two tiles ago: they passed the barrier below for tile i - 1 since)
+            if (g.bias_mode == 2) for (int c = et; c < g.tile_n; c += 32 * kPsEpilogueWarps) s_bias[acc][c] = (n0 + c < g.N) ? __ldg(g.bias + n0 + c) : 0.f;
+            const float bias_row = (g.bias_mode == 1 && m < g.M) ? __ldg(g.bias + m) : 0.f;
+            const bool have = mbar_wait(smem_u32(&acc_full[acc]), aph, abortp, g.status, 4u, g.wait_ns);
+            uint32_t all_acc;
+            asm volatile(
+                "{\n\t.reg .pred p, q;\n\t"
+                "setp.ne.u32 q, %1, 0;\n\t"
+                "bar.red.and.pred p, 2, %2, q;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(all_acc) : "r"((uint32_t)have), "n"(32 * kPsEpilogueWarps) : "memory");
+            if (!all_acc) { ok = false; break; }
+            tc_fence_after();
+            e.ybase = g.y + (long long)bz * g.y_bs;
+            e.rbase = g.residual ? g.residual + (long long)bz * g.y_bs : nullptr;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * (uint32_t)g.tile_n;
+            uint32_t r[32];
+            tmem_ld32(t_row, r);
+#pragma unroll 1
+            for (int c0 = 0; c0 < g.tile_n; c0 += 32) {
+                float v[32];
+                const int nb = n0 + c0;
+                const int cnt = min(g.N - nb, g.tile_n - c0);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+                if (c0 + 32 < g.tile_n) tmem_ld32(t_row + (uint32_t)(c0 + 32), r);
+                else {
+                    // every value of this accumulator is in registers: hand it back to the MMA warp
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (CG == 2) mbar_arrive_remote(smem_u32(&acc_empty[acc]), 0u);
+                        else mbar_arrive(smem_u32(&acc_empty[acc]));
+                    }
+                }
+                if (cnt <= 0) continue;                  // warp-uniform
+                if (g.bias_mode == 1) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] += bias_row;
+                } else if (g.bias_mode == 2) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 b = *reinterpret_cast<const float4*>(&s_bias[acc][c0 + j]);
+                        v[j] += b.x; v[j + 1] += b.y; v[j + 2] += b.z; v[j + 3] += b.w;
+                    }
+                }
+                const bool full = cnt >= 32 && m_first + 32 <= g.M && (e.vec || !transposed);
+                if (e.rbase == nullptr) {
+                    if (e.gelu) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = fminf(fmaxf(v[j], e.lo), e.hi);
+                    }
+                    if (full) epilogue_block<true, false>(v, e, m_first, nb, cnt, stg, lane, transposed);
+                    else epilogue_block<false, false>(v, e, m_first, nb, cnt, stg, lane, transposed);
+                } else {
+                    if (full) epilogue_block<true, true>(v, e, m_first, nb, cnt, stg, lane, transposed);
+                    else epilogue_block<false, true>(v, e, m_first, nb, cnt, stg, lane, transposed);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    // a pair stays together until neither CTA touches the other's shared memory, barriers or tensor memory any more
+    if constexpr (CG == 2) cluster_sync_all();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        if constexpr (CG == 1) tmem_dealloc(tmem_base, g.tmem_cols);
+        else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(g.tmem_cols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------
 // DW_SIMT: depthwise conv + bias + activation.  One CTA = tile_c channels x tile_h x tile_w outputs of one image.
 // The input halo tile is staged in shared memory with coalesced row reads; each thread then produces `items`
 // consecutive outputs along the width and stores them with vec-wide stores.
@@ -1964,12 +2441,45 @@ cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* t
         ++n_attr;
     }
     cfg.attrs = attr; cfg.numAttrs = (unsigned)n_attr;
-    // Only grids of more than two CTAs per SM take the capped build: that is where sharing an SM pays.  Smaller grids
-    // (the batch-1 layers) keep the uncapped one, which has no register spills; measured in a chained ResNet-18-shaped
-    // pass, a single 196-CTA layer on the capped build cost the pass 10 us.
-    const long long ctas = (long long)I.grid_x * I.grid_y * I.grid_z;
-    if (ctas > 2 * 148 && gemm_two_per_sm(I.smem_bytes, g.tmem_cols)) return cudaLaunchKernelEx(&cfg, tt_gemm_tc_kernel<2>, ta, tb, tx, g);
+    // which build runs is the record's choice (ctas_per_sm), resolved by the legaliser
+    if (g.two_per_sm && gemm_two_per_sm(I.smem_bytes, g.tmem_cols)) return cudaLaunchKernelEx(&cfg, tt_gemm_tc_kernel<2>, ta, tb, tx, g);
     return cudaLaunchKernelEx(&cfg, tt_gemm_tc_kernel<1>, ta, tb, tx, g);
+}
+
+// The persistent form: one CTA (or one pair of CTAs, as a cluster of two) per SM.
+cudaError_t launch_gemm_ps(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, cudaStream_t st) {
+    static int attr_set_for = -1, sm_count = 148;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (attr_set_for != dev) {
+        cudaError_t e = cudaFuncSetAttribute(tt_gemm_ps_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemLimit);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(tt_gemm_ps_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmemLimit);
+        if (e != cudaSuccess) return e;
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        attr_set_for = dev;
+    }
+    CUtensorMap ta, tb;
+    memcpy(&ta, tmap_a, sizeof ta);
+    memcpy(&tb, tmap_b, sizeof tb);
+    const int cg = g.cta_group == 2 ? 2 : 1;
+    const long long units = std::min<long long>(g.total_tiles, sm_count / cg);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(units * cg), 1, 1); cfg.blockDim = dim3(kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)I.smem_bytes; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+    ++n_attr;
+    if (cg == 2) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = 2; attr[n_attr].val.clusterDim.y = 1; attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
+    cfg.attrs = attr; cfg.numAttrs = (unsigned)n_attr;
+    if (cg == 2) return cudaLaunchKernelEx(&cfg, tt_gemm_ps_kernel<2>, ta, tb, g);
+    return cudaLaunchKernelEx(&cfg, tt_gemm_ps_kernel<1>, ta, tb, g);
 }
 
 // Can a cluster of `cluster` CTAs with this much shared memory each be resident at all?

@@ -28,7 +28,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_sizes_match_header_layout():
     assert ctypes.sizeof(B.tt_shapes) == 20 * 4
-    assert ctypes.sizeof(B.tt_schedule_record) == 3 * 4 + 80 + 16 * 4
+    assert ctypes.sizeof(B.tt_schedule_record) == 3 * 4 + 80 + 20 * 4
     assert B.status_string(B.TT_ERR_INVALID_SCHEDULE) != B.status_string(B.TT_OK)
 
 
@@ -489,7 +489,7 @@ def test_pool_file_round_trip_and_rejections(tmp_path):
     B.pool_save(path, recs[:1], None)
     line = [l for l in open(path).read().splitlines() if not l.startswith("#")][0]
     assert "us=-1" in line
-    for bad in (line.replace("tile_n=", "tile_q="), line.replace("version=1", "version=99"), line.replace("stages=2", "stages=two"),
+    for bad in (line.replace("tile_n=", "tile_q="), line.replace("version=2", "version=99"), line.replace("stages=2", "stages=two"),
                 line.replace("origin=1,", "origin=1;")):
         with open(path, "w") as f:
             f.write(bad + "\n")
