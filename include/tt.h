@@ -113,8 +113,10 @@ typedef struct tt_schedule_record {
     int32_t block_x, block_y, items_per_thread, vec_width, unroll, threads;
     int32_t mma_m_axis;    /* GEMM_TC: which output axis rides the 128 accumulator rows: 0 library's choice by shape,
                               1 output rows (conv filters, dense/bmm rows m), 2 output columns (conv pixels, nn) */
-    int32_t slab_tiles;    /* GEMM_TC, conv2d only: reduction tiles served by one staging of the input rows in shared
-                              memory (the cache buffer of the im2col operand); 0 = as many as fit */
+    int32_t slab_tiles;    /* GEMM_TC, conv2d: reduction tiles served by one staging of the input rows in shared
+                              memory (the cache buffer of the im2col operand); 0 = as many as fit.  Persistent form with a
+                              row-contiguous operand: boxes in that operand's staging ring, i.e. how much is in flight
+                              from memory; 0 = as many as fit, at most 8 */
     int32_t acc_split;     /* GEMM_TC: independent accumulators in tensor memory (1, 2, 4 or 8; 0 = 1) to which the
                               8-wide reduction steps are dealt round-robin; they are added in fixed order on read-out.
                               Consecutive multiply-accumulates into one accumulator wait for each other; into several,

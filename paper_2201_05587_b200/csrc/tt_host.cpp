@@ -305,13 +305,22 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
         const bool a_mn = swap ? v_mn : u_mn, b_mn = swap ? u_mn : v_mn;
         const unsigned stg_a = a_mn ? (unsigned)(tk * kHwTileM * 4) : 0u, stg_b = b_mn ? (unsigned)(tk * tn * 4) : 0u;
         const long long epi = 4ll * 32 * 36 * 4;
+        // the staging ring of a row-contiguous operand has its own depth (record field slab_tiles; 0 = as deep as fits,
+        // at most 8): it is what is in flight from DRAM, while the K-major stages only decouple transposing from multiplying
+        if (rec->slab_tiles < 0) return TT_ERR_INVALID_SCHEDULE;
+        const bool any_stg = stg_a + stg_b > 0;
+        int sd = any_stg ? (rec->slab_tiles == 0 ? kMaxStages : std::min(kMaxStages, rec->slab_tiles)) : 0;
         long long smem_p = 0;
         for (;;) {
-            smem_p = (long long)st * (a_stage + b_stage + stg_a + stg_b) + epi + 1024;
-            if (smem_p <= kDynSmemLimit || strict || st <= 1) break;
+            smem_p = (long long)st * (a_stage + b_stage) + (long long)sd * (stg_a + stg_b) + epi + 1024;
+            if (smem_p <= kDynSmemLimit) break;
+            if (any_stg && sd > 1 && (rec->slab_tiles == 0 || !strict) && (rec->slab_tiles == 0 || sd >= st)) { --sd; continue; }
+            if (strict || st <= 1) break;
             --st; changed |= TT_CHG_STAGES;
         }
-        L.stages = st; L.split_k = 1; L.acc_split = 1; L.slab_tiles = 0; L.ctas_per_sm = 1;
+        if (any_stg && rec->slab_tiles != 0 && sd != rec->slab_tiles) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_SLAB; }
+        if (!any_stg && rec->slab_tiles != 0) changed |= TT_CHG_SLAB;
+        L.stages = st; L.split_k = 1; L.acc_split = 1; L.slab_tiles = (any_stg && rec->slab_tiles != 0) ? sd : 0; L.ctas_per_sm = 1;
         if (rec->ctas_per_sm == 2) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_FORM; }
         if (strict && (changed & ~TT_CHG_TILE_M)) return TT_ERR_INVALID_SCHEDULE;
         const int rows_m = kHwTileM * cg;
@@ -341,10 +350,11 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
         g.idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((unsigned)(tn >> 3) << 17) | ((unsigned)(rows_m >> 4) << 24);
         g.persistent = 1; g.cta_group = cg; g.total_tiles = (int)units;
         g.a_mn = a_mn; g.b_mn = b_mn; g.b_rows_cta = tn / cg;
+        g.stg_depth = std::max(sd, 1);
         g.a_stg_off = (unsigned)((long long)st * (a_stage + b_stage));
-        g.b_stg_off = g.a_stg_off + (unsigned)st * stg_a;
+        g.b_stg_off = g.a_stg_off + (unsigned)sd * stg_a;
         g.stg_a_bytes = stg_a; g.stg_b_bytes = stg_b;
-        g.epi_off = g.b_stg_off + (unsigned)st * stg_b;
+        g.epi_off = g.b_stg_off + (unsigned)sd * stg_b;
         struct Opnd { int mode; long long rs, ks, bs; int batched; } U{}, V{};
         long long y_is, y_js, y_bs;
         int bias_on;

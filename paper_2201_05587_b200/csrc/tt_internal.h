@@ -82,7 +82,8 @@ struct GemmArgs {
     int a_mn, b_mn;                             // operand arrives as [tile_k][rows] boxes and is transposed in shared memory
     int b_rows_cta;                             // rows of operand B one CTA loads: tile_n / cta_group
     unsigned a_stg_off, b_stg_off;              // staging rings: byte offsets from the aligned tile base
-    unsigned stg_a_bytes, stg_b_bytes;          // ... and bytes per stage
+    unsigned stg_a_bytes, stg_b_bytes;          // ... and bytes per box
+    int stg_depth;                              // boxes per staging ring (what is in flight from DRAM)
     unsigned epi_off;                           // read-out staging area (one 32 x 36-float block per read-out warp)
 };
 

@@ -53,6 +53,16 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
+// Non-blocking test of a barrier phase.
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
 __device__ __forceinline__ unsigned long long global_timer_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -1464,8 +1474,8 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 // CG = 2: two CTAs of a cluster work on one 256-row tile.  Each loads its own 128 rows of A and its half of B's
 // rows with ordinary (non-multicast) TMA; the CTA of rank 0 issues tcgen05.mma.cta_group::2, which reads both
 // CTAs' shared memory and writes each CTA's half of the accumulator into that CTA's tensor memory, so an SM reads
-// only half of B per multiply-accumulate.  The rank-1 CTA's warp 1 relays "my stage has landed" to rank 0; a
-// multicast tcgen05.commit frees the stage and publishes the accumulator in both CTAs.
+// only half of B per multiply-accumulate.  Both CTAs' loads report their bytes to the stage barrier of rank 0 (which
+// expects the pair's total), a multicast tcgen05.commit frees the stage and publishes the accumulator in both CTAs.
 // ------------------------------------------------------------------------------------------------------------
 template <int CG>
 __device__ __forceinline__ void mma_tf32_cg(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
@@ -1531,6 +1541,13 @@ __device__ __noinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, vo
         }
     }
 }
+// TMA load whose completion is reported to a barrier given by its cluster-wide address, which may lie in the other
+// CTA of the pair (no multicast: the data goes to this CTA's shared memory only).
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const void* tmap, uint32_t bar_cluster, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
 __device__ __forceinline__ void tma_load_3d_plain(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2) {
     tma_load_3d(dst, tmap, bar, c0, c1, c2);
 }
@@ -1584,7 +1601,6 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __shared__ uint64_t empty_bar[kMaxStages];    // every multiply-accumulate that reads the stage has completed
     __shared__ uint64_t stg_full[kMaxStages];     // a staging box has landed
     __shared__ uint64_t stg_empty[kMaxStages];    // the transposer warps are done with it
-    __shared__ uint64_t peer_full[kMaxStages];    // CG 2, rank 0: the rank-1 CTA's stage is in place
     __shared__ uint64_t acc_full[2];              // an accumulator holds a finished tile
     __shared__ uint64_t acc_empty[2];             // the read-out warps (of both CTAs) have drained it
     __shared__ uint32_t tmem_slot;
@@ -1615,9 +1631,10 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         for (int s = 0; s < g.stages; ++s) {
             mbar_init(smem_u32(&full_bar[s]), full_count);
             mbar_init(smem_u32(&empty_bar[s]), 1u);
+        }
+        for (int s = 0; s < g.stg_depth; ++s) {
             mbar_init(smem_u32(&stg_full[s]), 1u);
             mbar_init(smem_u32(&stg_empty[s]), (uint32_t)kPsTransposeWarps);
-            mbar_init(smem_u32(&peer_full[s]), 1u);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&acc_full[a]), 1u);
@@ -1657,83 +1674,125 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
+        // Two independent streams of requests, each with its own ring and cursor: boxes of a row-contiguous operand go
+        // to the staging ring (g.stg_depth deep: what is in flight from DRAM), K-major tiles to the pipeline stages.
+        // The warp polls both rings and serves whichever has a free slot, so the staging ring runs as far ahead as
+        // its depth allows, whatever the multiply-accumulates are doing.
         const bool leader = elect_one();
         const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes), b_atom = (uint32_t)(b_rows * g.row_bytes);
         const uint32_t km_bytes = (a_mn ? 0u : g.a_stage_bytes) + (b_mn ? 0u : g.b_stage_bytes);
         const uint32_t mn_bytes = (a_mn ? g.stg_a_bytes : 0u) + (b_mn ? g.stg_b_bytes : 0u);
-        uint32_t st = 0, ph = 0;
-        long long issued = 0;
+        struct Cursor { int i, kt, m0, n0, bz, slot; uint32_t ph; long long it; };
+        const long long total_it = (long long)my_tiles * kt_n;
+        auto cur_init = [&](Cursor& c) {
+            c.i = 0; c.kt = 0; c.slot = 0; c.ph = 0; c.it = 0; c.m0 = c.n0 = c.bz = 0;
+            if (my_tiles > 0) decode(0, c.m0, c.n0, c.bz);
+        };
+        auto cur_next = [&](Cursor& c, int depth) {
+            ++c.it;
+            if (++c.slot == depth) { c.slot = 0; c.ph ^= 1u; }
+            if (++c.kt == kt_n) {
+                c.kt = 0;
+                if (++c.i < my_tiles) decode(c.i, c.m0, c.n0, c.bz);
+            }
+        };
+        Cursor cs, ck;
+        cur_init(cs); cur_init(ck);
+        if (!any_mn) cs.it = total_it;
+        if (!any_km) ck.it = total_it;
         bool ok = true;
-        for (int i = 0; i < my_tiles && ok; ++i) {
-            int m0, n0, bz;
-            decode(i, m0, n0, bz);
-            const int nb0 = n0 + (int)rank * b_rows;          // CG 2: this CTA's half of the B rows
-            const int a_bz = g.a_tma_batched ? bz : 0, b_bz = g.b_tma_batched ? bz : 0;
-            int k0 = 0;
-            for (int kt = 0; kt < kt_n; ++kt, k0 += g.tile_k) {
-                if (any_mn) {
-                    const bool got = mbar_wait(smem_u32(&stg_empty[st]), ph ^ 1u, abortp, g.status, 11u, g.wait_ns);
-                    if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-                    if (leader) {
-                        const uint32_t bar = smem_u32(&stg_full[st]);
-                        mbar_expect_tx(bar, mn_bytes);
-                        if (a_mn) tma_load_3d(tiles_base + g.a_stg_off + st * g.stg_a_bytes, &tmap_a, bar, m0, k0, a_bz);
-                        if (b_mn) tma_load_3d(tiles_base + g.b_stg_off + st * g.stg_b_bytes, &tmap_b, bar, nb0, k0, b_bz);
-                    }
+        unsigned long long t_last = global_timer_ns();
+        unsigned idle = 0;
+        while (cs.it < total_it || ck.it < total_it) {
+            bool progressed = false;
+            if (cs.it < total_it && mbar_test_wait(smem_u32(&stg_empty[cs.slot]), cs.ph ^ 1u)) {
+                if (leader) {
+                    const uint32_t bar = smem_u32(&stg_full[cs.slot]);
+                    const int k0 = cs.kt * g.tile_k;
+                    mbar_expect_tx(bar, mn_bytes);
+                    if (a_mn) tma_load_3d(tiles_base + g.a_stg_off + (uint32_t)cs.slot * g.stg_a_bytes, &tmap_a, bar, cs.m0, k0, g.a_tma_batched ? cs.bz : 0);
+                    if (b_mn) tma_load_3d(tiles_base + g.b_stg_off + (uint32_t)cs.slot * g.stg_b_bytes, &tmap_b, bar, cs.n0 + (int)rank * b_rows, k0,
+                                          g.b_tma_batched ? cs.bz : 0);
                 }
-                if (any_km) {
-                    const bool got = mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, abortp, g.status, 1u, g.wait_ns);
-                    if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-                    if (leader) {
-                        const uint32_t bar = smem_u32(&full_bar[st]);
-                        // (test facility: the first stage may be told to expect more than arrives, see tt_workload_test_stall)
-                        mbar_expect_tx(bar, km_bytes + (issued == 0 ? g.extra_tx : 0u));
-                        const uint32_t a_dst = tiles_base + st * stage_bytes;
-                        if (!a_mn) {
-                            uint32_t dst = a_dst;
-                            int kc = k0;
+                __syncwarp();
+                cur_next(cs, g.stg_depth);
+                progressed = true;
+            }
+            if (ck.it < total_it && mbar_test_wait(smem_u32(&empty_bar[ck.slot]), ck.ph ^ 1u)) {
+                if (leader) {
+                    uint32_t bar = smem_u32(&full_bar[ck.slot]);
+                    const int k0 = ck.kt * g.tile_k;
+                    const int nb0 = ck.n0 + (int)rank * b_rows;       // CG 2: this CTA's half of the B rows
+                    const int a_bz = g.a_tma_batched ? ck.bz : 0, b_bz = g.b_tma_batched ? ck.bz : 0;
+                    // (test facility: the first stage may be told to expect more than arrives, see tt_workload_test_stall)
+                    if (rank == 0) mbar_expect_tx(bar, (uint32_t)CG * km_bytes + (ck.it == 0 ? g.extra_tx : 0u));
+                    if constexpr (CG == 2) bar = map_to_peer(bar, 0u);       // the pair's loads all report to rank 0
+                    const uint32_t a_dst = tiles_base + (uint32_t)ck.slot * stage_bytes;
+                    if (!a_mn) {
+                        uint32_t dst = a_dst;
+                        int kc = k0;
 #pragma unroll 1
-                            for (int at = 0; at < g.n_atoms; ++at, dst += a_atom, kc += g.atom_k) tma_load_3d(dst, &tmap_a, bar, kc, m0, a_bz);
+                        for (int at = 0; at < g.n_atoms; ++at, dst += a_atom, kc += g.atom_k) {
+                            if constexpr (CG == 2) tma_load_3d_pair(dst, &tmap_a, bar, kc, ck.m0, a_bz);
+                            else tma_load_3d(dst, &tmap_a, bar, kc, ck.m0, a_bz);
                         }
-                        if (!b_mn) {
-                            uint32_t dst = a_dst + g.a_stage_bytes;
-                            int kc = k0;
+                    }
+                    if (!b_mn) {
+                        uint32_t dst = a_dst + g.a_stage_bytes;
+                        int kc = k0;
 #pragma unroll 1
-                            for (int at = 0; at < g.n_atoms; ++at, dst += b_atom, kc += g.atom_k) tma_load_3d(dst, &tmap_b, bar, kc, nb0, b_bz);
+                        for (int at = 0; at < g.n_atoms; ++at, dst += b_atom, kc += g.atom_k) {
+                            if constexpr (CG == 2) tma_load_3d_pair(dst, &tmap_b, bar, kc, nb0, b_bz);
+                            else tma_load_3d(dst, &tmap_b, bar, kc, nb0, b_bz);
                         }
                     }
                 }
                 __syncwarp();
-                ++issued;
-                if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
+                cur_next(ck, g.stages);
+                progressed = true;
+            }
+            if (progressed) { idle = 0; continue; }
+            if ((++idle & 63u) == 0u) {
+                // nothing to do for a while: the same bounded patience as every other wait of the kernel
+                if (idle == 64u) t_last = global_timer_ns();
+                bool give_up = *abortp != 0;
+                if (!give_up && global_timer_ns() - t_last > g.wait_ns) {
+                    *abortp = 1;
+                    atomicCAS(g.status, 0u, (unsigned)TT_ERR_TIMEOUT | (1u << 8));
+                    give_up = true;
+                }
+                if (__any_sync(0xffffffffu, give_up)) { ok = false; break; }
             }
         }
         if ((!ok || *abortp) && lane == 0) {
             // let copies in flight land before shared memory is given back (bounded)
-            const long long first = issued > g.stages ? issued - g.stages : 0;
-            for (long long it = first; it < issued; ++it) {
-                const int s = (int)(it % g.stages);
-                const uint32_t par = (uint32_t)(it / g.stages) & 1u;
+            for (int pass = 0; pass < 2; ++pass) {
+                const long long issued = pass == 0 ? ck.it : cs.it;
+                const int depth = pass == 0 ? g.stages : g.stg_depth;
+                if ((pass == 0 && (!any_km || rank != 0)) || (pass == 1 && !any_mn)) continue;
+                const long long first = issued > depth ? issued - depth : 0;
+                for (long long it = first; it < issued; ++it) {
+                    const uint32_t bar = pass == 0 ? smem_u32(&full_bar[it % depth]) : smem_u32(&stg_full[it % depth]);
+                    const uint32_t par = (uint32_t)(it / depth) & 1u;
+                    const unsigned long long t0 = global_timer_ns();
+                    while (!mbar_try_wait(bar, par)) { if (global_timer_ns() - t0 > 2000000ull) break; }
+                }
+            }
+            if (rank != 0) {
+                // this CTA's K-major loads report to rank 0's barriers: give them time to land instead (the pair leaves
+                // together, after rank 0 has seen the pair's bytes or given up on them)
                 const unsigned long long t0 = global_timer_ns();
-                if (any_km) while (!mbar_try_wait(smem_u32(&full_bar[s]), par)) { if (global_timer_ns() - t0 > 2000000ull) break; }
-                if (any_mn) while (!mbar_try_wait(smem_u32(&stg_full[s]), par)) { if (global_timer_ns() - t0 > 4000000ull) break; }
+                while (global_timer_ns() - t0 < 200000ull) { }
             }
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ---------------- MMA issuer (rank 0 of a pair), or the relay of "my stage has landed" (rank 1) ----------------
+        // ---------------- MMA issuer (of a pair: rank 0's) ----------------
         const bool leader = elect_one();
         uint32_t st = 0, ph = 0;
         bool ok = true;
         if (CG == 2 && rank != 0) {
-            for (int i = 0; i < my_tiles && ok; ++i)
-                for (int kt = 0; kt < kt_n; ++kt) {
-                    const bool got = mbar_wait(smem_u32(&full_bar[st]), ph, abortp, g.status, 2u, g.wait_ns);
-                    if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-                    if (leader) mbar_arrive_remote(smem_u32(&peer_full[st]), 0u);
-                    __syncwarp();
-                    if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
-                }
+            // rank 0 issues for the pair
         } else {
             const uint64_t d0 = make_desc(0u, g.row_bytes);
             const uint32_t d_hi = (uint32_t)(d0 >> 32), d_lo = (uint32_t)d0;
@@ -1750,8 +1809,7 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * (uint32_t)g.tile_n;
                 for (int kt = 0; kt < kt_n; ++kt) {
-                    bool got = mbar_wait(smem_u32(&full_bar[st]), ph, abortp, g.status, 2u, g.wait_ns);
-                    if (CG == 2 && got) got = mbar_wait_cluster(smem_u32(&peer_full[st]), ph, abortp, g.status, 13u, g.wait_ns);
+                    const bool got = mbar_wait(smem_u32(&full_bar[st]), ph, abortp, g.status, 2u, g.wait_ns);
                     if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                     tc_fence_after();
                     if (leader) {
@@ -1779,22 +1837,23 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         // ---------------- transposers ----------------
         if (any_mn) {
             const int tw = warp - 2;
-            uint32_t st = 0, ph = 0;
+            uint32_t st = 0, ph = 0, sst = 0, sph = 0;
             bool ok = true;
             for (int i = 0; i < my_tiles && ok; ++i)
                 for (int kt = 0; kt < kt_n; ++kt) {
-                    if (!mbar_wait(smem_u32(&stg_full[st]), ph, abortp, g.status, 6u, g.wait_ns) ||
+                    if (!mbar_wait(smem_u32(&stg_full[sst]), sph, abortp, g.status, 6u, g.wait_ns) ||
                         !mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, abortp, g.status, 3u, g.wait_ns)) { ok = false; break; }
                     const uint32_t a_s = tiles_base + st * stage_bytes, b_s = a_s + g.a_stage_bytes;
-                    if (a_mn) ps_transpose(tiles_base + g.a_stg_off + st * g.stg_a_bytes, a_s, kHwTileM, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, tw, lane);
-                    if (b_mn) ps_transpose(tiles_base + g.b_stg_off + st * g.stg_b_bytes, b_s, b_rows, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, tw, lane);
+                    if (a_mn) ps_transpose(tiles_base + g.a_stg_off + sst * g.stg_a_bytes, a_s, kHwTileM, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, tw, lane);
+                    if (b_mn) ps_transpose(tiles_base + g.b_stg_off + sst * g.stg_b_bytes, b_s, b_rows, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, tw, lane);
                     fence_proxy_async_shared();          // generic-proxy stores -> visible to the tensor core's reads
                     __syncwarp();
                     if (lane == 0) {
                         mbar_arrive(smem_u32(&full_bar[st]));
-                        mbar_arrive(smem_u32(&stg_empty[st]));
+                        mbar_arrive(smem_u32(&stg_empty[sst]));
                     }
                     if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
+                    if (++sst == (uint32_t)g.stg_depth) { sst = 0; sph ^= 1u; }
                 }
         }
     } else {

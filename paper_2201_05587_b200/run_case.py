@@ -20,7 +20,8 @@ from . import workloads as W
 
 ACTS = {"none": B.TT_ACT_NONE, "relu": B.TT_ACT_RELU, "relu6": B.TT_ACT_RELU6, "gelu": B.TT_ACT_GELU_ERF}
 RECORD_FIELDS = ("tile_m", "tile_n", "tile_k", "stages", "split_k", "raster", "block_x", "block_y",
-                 "items_per_thread", "vec_width", "threads", "unroll", "mma_m_axis", "slab_tiles", "acc_split", "k_order")
+                 "items_per_thread", "vec_width", "threads", "unroll", "mma_m_axis", "slab_tiles", "acc_split", "k_order",
+                 "persistent", "cta_group", "ctas_per_sm")
 
 
 def build_spec(a) -> W.Spec:
@@ -53,6 +54,7 @@ def main(argv=None) -> int:
     ap.add_argument("--iters", type=int, default=3, help="plain launches after the timed batches")
     ap.add_argument("--seed", type=int, default=7)
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of graph replays")
+    ap.add_argument("--constant-weights", action="store_true", help="promise that w and bias are constants (fetched early)")
     a = ap.parse_args(argv)
 
     import torch
@@ -72,6 +74,7 @@ def main(argv=None) -> int:
         rec = best[0][0]
         print(f"grid tuner tried {tried} records")
     info = wl.apply(rec)
+    wl.set_constant_weights(a.constant_weights)
     topts = B.tt_timing_opts()
     topts.use_graph = 0 if a.no_graph else 1            # batches replayed as CUDA graphs: no CPU launch gaps
     tm = wl.time(tt, topts)
