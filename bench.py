@@ -108,7 +108,8 @@ def workload_name(model, specs, pool_sources):
 
 def config_dict(model, specs, pool_sources):
     return {"workload": workload_name(model, specs, pool_sources), "l2": "flushed between steps (256 MB write)",
-            "replay": "one CUDA graph per data-chained model pass", "multi_gpu": "independent replicas"}
+            "replay": "one CUDA graph per data-chained model pass", "multi_gpu": "independent replicas",
+            "weights": "declared constant to the library (a kernel may fetch them before it waits for its predecessor)"}
 
 
 class ClockSampler(threading.Thread):
@@ -265,6 +266,7 @@ class Bench:
         for j, sp in enumerate(W.MODELS[model]()):
             a = W.make_inputs(sp, SEEDS.get(model, 7) + 100, j)
             swl = sp.workload()
+            swl.set_constant_weights(True)
             keep, stt = W.device_tensors(sp, a, self.dev)
             best, tried = swl.grid_tune(stt, self.tune_opts, level=self.args.tune_level, top_k=self.args.top_k)
             self.pool_tried += tried
@@ -342,6 +344,8 @@ class Bench:
         specs = W.MODELS[model]()
         arrays = [W.make_inputs(sp, seed, i) for i, sp in enumerate(specs)]
         wls = [sp.workload() for sp in specs]
+        for w in wls:
+            w.set_constant_weights(True)          # inference: no kernel writes a layer's parameters
         dev_t, tts = zip(*[W.device_tensors(sp, a, dev) for sp, a in zip(specs, arrays)])
         pool = W.single_conv_pool() if model == "single_conv" else [r for src in sources for r in self.pool_of(src)]
 
@@ -481,8 +485,9 @@ def saturating_points(bench):
     dwr = lambda **kw: B.make_record(B.TT_FAMILY_DW_SIMT, **kw)
     cases = [
         (W._dense(4096, 4096, 4096), "tensor",
-         [tc(tile_n=256, tile_k=32, stages=4, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1),
-          tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=2)]),
+         [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=6, mma_m_axis=1, persistent=1, cta_group=2),
+          tc(tile_n=240, tile_k=32, stages=6, mma_m_axis=1, persistent=1, cta_group=2),
+          tc(tile_n=256, tile_k=64, stages=3, mma_m_axis=1, persistent=1, cta_group=2)]),
         (conv(32, 128, 28, 128, 3, 1), "tensor",
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=128, tile_k=32, stages=3, mma_m_axis=2),
           tc(tile_n=128, tile_k=64, stages=2, mma_m_axis=2),
@@ -495,15 +500,21 @@ def saturating_points(bench):
          [tc(tile_n=224, tile_k=96, stages=2, k_order=1, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=5, k_order=1, mma_m_axis=1)]),
         (conv(32, 256, 56, 64, 1, 0), "hbm",
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=2),
-          tc(tile_n=64, tile_k=32, stages=2, mma_m_axis=2, slab_tiles=1), tc(tile_n=64, tile_k=32, stages=3, mma_m_axis=2, slab_tiles=1)]),
+          tc(tile_n=64, tile_k=32, stages=2, mma_m_axis=2, slab_tiles=1), tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=2, persistent=1),
+          tc(tile_n=64, tile_k=32, stages=2, mma_m_axis=2, persistent=1)]),
+        (conv(32, 64, 56, 256, 1, 0), "hbm",
+         [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=2, slab_tiles=1), tc(tile_n=128, tile_k=64, stages=2, mma_m_axis=1, persistent=1),
+          tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1, persistent=1)]),
         # batch_matmul at BERT-base head shapes, 3072 = 12 heads x 256 sequences: scores (NT) and context (NN)
         (W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(3072, 128, 128, 64, True), 1, "bmm_nt_3072x128x128x64", "bert"), "hbm",
-         [tc(tile_n=128, tile_k=64, stages=1, mma_m_axis=1), tc(tile_n=128, tile_k=64, stages=1, mma_m_axis=2),
-          tc(tile_n=128, tile_k=32, stages=2, mma_m_axis=1)]),
+         [tc(tile_n=128, tile_k=64, stages=1, mma_m_axis=2), tc(tile_n=128, tile_k=64, stages=2, mma_m_axis=2, persistent=1),
+          tc(tile_n=128, tile_k=64, stages=2, mma_m_axis=1, persistent=1)]),
         (W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(3072, 128, 64, 128, False), 1, "bmm_nn_3072x128x64x128", "bert"), "hbm",
-         [tc(tile_n=64, tile_k=128, stages=1, mma_m_axis=1), tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=1)]),
+         [tc(tile_n=64, tile_k=128, stages=1, mma_m_axis=1), tc(tile_n=64, tile_k=64, stages=3, mma_m_axis=1, persistent=1),
+          tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=1, persistent=1)]),
         (W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(64, 1024, 1024, 1024, True), 1, "bmm_nt_64x1024x1024x1024", "bert"), "tensor",
-         [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=4, mma_m_axis=1)]),
+         [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=256, tile_k=32, stages=6, mma_m_axis=1, persistent=1, cta_group=2),
+          tc(tile_n=256, tile_k=32, stages=4, mma_m_axis=1, persistent=1)]),
         (dw(64, 144, 56, 1), "hbm",
          [dwr(tile_m=4, block_y=16, block_x=56, items_per_thread=4, vec_width=4, threads=128, unroll=4),
           dwr(tile_m=8, block_y=14, block_x=56, items_per_thread=4, vec_width=4, threads=256, unroll=4, raster=1, stages=2),
@@ -527,6 +538,7 @@ def saturating_points(bench):
     for sp, bound, recs in cases:
         a = W.make_inputs(sp, 7)
         wl = sp.workload()
+        wl.set_constant_weights(True)
         t, tt = W.device_tensors(sp, a, dev)
         f, b = algorithmic_work(sp)
         best = None

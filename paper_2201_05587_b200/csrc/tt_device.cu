@@ -18,7 +18,8 @@ cudaError_t launch_row(const tt_apply_info& I, const RowArgs& row, cudaStream_t 
 cudaError_t gemm_cluster_fits(int smem_bytes, int cluster, int* fits);
 cudaError_t launch_repack(const float* w, float* out, int kout, int C, int RS, int CB, cudaStream_t st);
 cudaError_t launch_floor(const tt_apply_info& I, int cluster, cudaStream_t st);
-cudaError_t launch_gemm_ps(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, cudaStream_t st);
+cudaError_t launch_gemm_ps(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, const void* tmap_x,
+                           cudaStream_t st);
 
 namespace {
 
@@ -183,6 +184,7 @@ tt_status bind_device(tt_workload* w) {
         if (cudaMemcpy(w->ktab_dev, tab.data(), bytes, cudaMemcpyHostToDevice) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
     }
     w->tmaps.clear();
+    w->repacked_for = nullptr;
     return TT_OK;
 }
 
@@ -237,10 +239,16 @@ tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
         GemmArgs g = p.g;
         const void* a_ptr = pick(t, p.a_tensor);
         const void* b_ptr = pick(t, p.b_tensor);
+        bool repacked_now = false;
         if (p.repack) {
-            // tap-major convolution: the filters are brought into [filter][32-channel block][tap][channel] order first
-            if (launch_repack(static_cast<const float*>(t->w), static_cast<float*>(w->workspace), g.M, g.C, g.R * g.S,
-                              p.repack_cb, st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+            // tap-major convolution: the filters are brought into [filter][32-channel block][tap][channel] order first.
+            // Constant weights (the caller's promise) are re-packed once per weight pointer and applied record.
+            if (!(w->constant_weights && w->repacked_for == t->w)) {
+                if (launch_repack(static_cast<const float*>(t->w), static_cast<float*>(w->workspace), g.M, g.C, g.R * g.S,
+                                  p.repack_cb, st) != cudaSuccess) { cudaGetLastError(); return TT_ERR_CUDA; }
+                w->repacked_for = t->w;
+                repacked_now = true;
+            }
             a_ptr = w->workspace;
         }
         const TmapPair* maps = nullptr;
@@ -261,11 +269,11 @@ tt_status launch(tt_workload* w, const tt_tensors* t, void* stream) {
         g.wait_ns = w->wait_ns;
         g.extra_tx = w->extra_tx;
         g.w_operand = 0;
-        if (w->constant_weights && !p.repack && (w->op == TT_OP_DENSE || w->op == TT_OP_CONV2D)) {
+        if (w->constant_weights && !repacked_now && !g.persistent && (w->op == TT_OP_DENSE || w->op == TT_OP_CONV2D)) {
             if (p.a_tensor == 1 && g.a_mode == OPM_TMA) g.w_operand = 1;
             else if (p.b_tensor == 1 && g.b_mode == OPM_TMA) g.w_operand = 2;
         }
-        e = g.persistent ? launch_gemm_ps(p.info, g, maps->a, maps->b, st) : launch_gemm(p.info, g, maps->a, maps->b, maps->x, st);
+        e = g.persistent ? launch_gemm_ps(p.info, g, maps->a, maps->b, maps->x, st) : launch_gemm(p.info, g, maps->a, maps->b, maps->x, st);
     } else if (w->family == TT_FAMILY_DW_SIMT) {
         DwArgs d = p.dw;
         d.x = static_cast<const float*>(t->x); d.w = static_cast<const float*>(t->w);
@@ -610,7 +618,28 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
             r.mma_m_axis = ax; r.tile_m = kHwTileM; r.tile_n = tn; r.tile_k = tk; r.stages = sg; r.split_k = sk; r.raster = ra;
             push(r);
         }
+        // the persistent form (alone and as CTA pairs) and the two-CTAs-per-SM build of the one-tile form; on kernels
+        // without them these legalise back and are dropped as duplicates-to-be
+        for (int ax : {1, 2}) for (int tn : full ? std::vector<int>{32, 64, 128, 192, 240, 256} : std::vector<int>{64, 128, 256})
+            for (int tk : {32, 64}) for (int sg : full ? std::vector<int>{2, 3, 4, 6} : std::vector<int>{2, 4, 6}) for (int cg : {1, 2}) {
+                tt_schedule_record r = base;
+                r.mma_m_axis = ax; r.tile_m = kHwTileM; r.tile_n = tn; r.tile_k = tk; r.stages = sg; r.split_k = 1; r.raster = 0;
+                r.persistent = 1; r.cta_group = cg;
+                push(r);
+            }
+        for (int ax : {1, 2}) for (int tn : {64, 128, 256}) for (int sg : {2, 3}) {
+            tt_schedule_record r = base;
+            r.mma_m_axis = ax; r.tile_m = kHwTileM; r.tile_n = tn; r.tile_k = 32; r.stages = sg; r.split_k = 1; r.raster = 0;
+            r.ctas_per_sm = 2;
+            push(r);
+        }
         if (w->op == TT_OP_CONV2D) {
+            for (int tn : {128, 224, 256}) for (int sg : {2, 4}) {
+                tt_schedule_record r = base;
+                r.mma_m_axis = 1; r.tile_m = kHwTileM; r.tile_n = tn; r.tile_k = 32; r.stages = sg; r.split_k = 1; r.raster = 0;
+                r.k_order = 1; r.persistent = 1;
+                push(r);
+            }
             // a slab that serves one reduction tile per staging: the smallest shared-memory footprint (two CTAs may
             // then share an SM)
             for (int ax : {1, 2}) for (int tn : full ? std::vector<int>{32, 64, 128, 256} : std::vector<int>{64, 128}) for (int sg : {2, 3}) {

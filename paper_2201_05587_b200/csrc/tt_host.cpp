@@ -116,9 +116,10 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     if (rec->persistent < 0 || rec->persistent > 1 || rec->cta_group < 0 || rec->cta_group > 2 || rec->ctas_per_sm < 0 ||
         rec->ctas_per_sm > 2 || rec->warp_layout != 0)
         return TT_ERR_INVALID_SCHEDULE;
-    // this reduction order exists in the one-tile-per-CTA kernel only
-    L.persistent = 0; L.cta_group = 1;
-    if (rec->persistent != 0 || rec->cta_group == 2) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_FORM; }
+    // both kernel forms walk this reduction order; CTA pairs do not
+    const bool persistent = rec->persistent == 1;
+    L.persistent = persistent ? 1 : 0; L.cta_group = 1;
+    if (rec->cta_group == 2) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_FORM; }
     if (rec->tile_m != kHwTileM) changed |= TT_CHG_TILE_M;
     if (rec->tile_k != tk) changed |= TT_CHG_TILE_K;
     if (rec->split_k != 1) changed |= TT_CHG_SPLIT_K;
@@ -127,7 +128,8 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     if (tn != rec->tile_n) changed |= TT_CHG_TILE_N;
     L.tile_n = tn;
     const int k_tiles = CB * RS / tps;
-    int st = std::min(std::min(kMaxStages, rec->stages), k_tiles);
+    // (the persistent form's filter pipeline runs on across tiles: no point in clamping it to one tile's reduction)
+    int st = persistent ? std::min(kMaxStages, rec->stages) : std::min(std::min(kMaxStages, rec->stages), k_tiles);
     if (st != rec->stages) changed |= TT_CHG_STAGES;
     if (strict && (changed & ~TT_CHG_TILE_M)) return TT_ERR_INVALID_SCHEDULE;
     // shared memory: filter stages | NCHW staging of a block (TMA box [32][in_rows][wp], one buffer) | pixel-major slab
@@ -140,20 +142,29 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     // furthest row a tile's views can touch (all tile_n rows are read, also those of pixels past the image)
     const long long pm_rows = (long long)((tn + wp - 2) / wp + s.r) * wp + s.s + gap + 8;
     const long long pm_buf = pm_rows * 128;
-    const int nbuf = CB > 1 ? 2 : 1;
+    const int nbuf = (CB > 1 || persistent) ? 2 : 1;
     long long smem = 0;
     const long long min_pipe = (long long)kGatherWarps * 32 * 36 * 4;
+    // persistent form: the read-out has its own staging area (the pipeline buffers are busy with the next tile), and
+    // the NCHW staging ring is two boxes deep when that fits
+    const long long epi = persistent ? 4ll * 32 * 36 * 4 : 0;
+    int sd = persistent ? 2 : 1;
     for (;;) {
-        const long long pipe = std::max<long long>((long long)st * a_stage, min_pipe);
-        smem = pipe + s_buf + nbuf * pm_buf + 1024;
-        if (smem <= kDynSmemLimit || strict || st <= 1) break;
+        const long long pipe = persistent ? (long long)st * a_stage : std::max<long long>((long long)st * a_stage, min_pipe);
+        smem = pipe + sd * s_buf + nbuf * pm_buf + epi + 1024;
+        if (smem <= kDynSmemLimit) break;
+        if (sd > 1) { --sd; continue; }
+        if (strict || st <= 1) break;
         --st; changed |= TT_CHG_STAGES;
     }
     L.stages = st;
-    const long long pipe = std::max<long long>((long long)st * a_stage, min_pipe);
+    const long long pipe = persistent ? (long long)st * a_stage : std::max<long long>((long long)st * a_stage, min_pipe);
     const int tiles_m = (M + kHwTileM - 1) / kHwTileM, tiles_n = (N + tn - 1) / tn;
-    const int tmem_cols_t = std::max(32, pow2_ceil(tn));
-    {
+    const int tmem_cols_t = std::max(32, pow2_ceil(persistent ? 2 * tn : tn));
+    if (persistent) {
+        L.ctas_per_sm = 1;
+        if (rec->ctas_per_sm == 2) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_FORM; }
+    } else {
         // which build: two CTAs per SM need half the shared memory and half the tensor memory each
         const bool fits2 = smem <= 112 * 1024 && tmem_cols_t <= 256;
         const long long ctas = (long long)tiles_m * tiles_n * B;
@@ -164,8 +175,13 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     I = tt_apply_info{};
     I.legal = L; I.changed = changed;
     I.grid_x = tiles_m * tiles_n; I.grid_y = 1; I.grid_z = B;
+    const long long units = (long long)tiles_m * tiles_n * B;
+    if (persistent) {
+        if (units > 0x7fffffffLL) return TT_ERR_RESOURCE;
+        I.grid_x = (int)std::min<long long>(units, 148); I.grid_z = 1;      // the launcher clamps to the device's SM count
+    }
     I.threads = kGemmThreads;
-    I.smem_bytes = (int)std::min<long long>(smem, 0x7fffffff);
+    I.smem_bytes = (int)std::min<long long>(persistent ? std::max<long long>(smem, 116 * 1024) : smem, 0x7fffffff);
     I.tmem_cols = tmem_cols_t;
     I.workspace_bytes = (int64_t)M * K * 4;              // the re-packed filters
     I.launches = 2;
@@ -196,13 +212,15 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     g.tap_major = 1;
     g.two_per_sm = L.ctas_per_sm == 2;
     g.b_rows_cta = tn; g.cta_group = 1;
+    g.persistent = persistent ? 1 : 0; g.total_tiles = (int)units; g.stg_depth = sd;
+    g.epi_off = (unsigned)(pipe + (long long)sd * s_buf + (long long)nbuf * pm_buf);
     g.slab_tma = 1; g.slab_tiles = RS / tps; g.slab_nbuf = 1; g.pm_nbuf = nbuf;
     g.slab_off = (unsigned)pipe; g.slab_buf_bytes = (unsigned)s_buf;
     g.slab_wp = wp; g.slab_gap = gap; g.slab_chpitch = in_rows * wp; g.slab_in_rows = in_rows; g.slab_rstep = 1;
     g.slab_box_ch = std::min(32, s.c);                   // (fewer than 32 channels: the rest of the staging buffer stays zero)
     g.slab_box_bytes = (unsigned)((long long)g.slab_box_ch * in_rows * wp * 4);
     g.slab_vec16 = 1;
-    g.pm_off = (unsigned)(pipe + s_buf); g.pm_buf_bytes = (unsigned)pm_buf;
+    g.pm_off = (unsigned)(pipe + (long long)sd * s_buf); g.pm_buf_bytes = (unsigned)pm_buf;
     return TT_OK;
 }
 

@@ -148,6 +148,7 @@ struct tt_workload {
     unsigned long long wait_ns = 1000000000ull;   // one second per wait inside a kernel, then the kernel gives up
     unsigned extra_tx = 0;            // test facility (tt_workload_test_stall)
     bool constant_weights = false;    // the caller's promise of tt_workload_set_constant_weights
+    const void* repacked_for = nullptr;   // tap-major convolution: the weight pointer whose re-packed copy the workspace holds
     // device staging buffers of tt_run_host
     void* hbuf[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     size_t hbytes[5] = {0, 0, 0, 0, 0};

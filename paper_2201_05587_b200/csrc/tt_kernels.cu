@@ -1595,12 +1595,15 @@ __device__ __forceinline__ void ps_transpose(uint32_t stg, uint32_t tile, int ro
 
 template <int CG>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const GemmArgs g) {
+tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                  const __grid_constant__ CUtensorMap tmap_x, const GemmArgs g) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages];     // a stage's operands are in place (TMA bytes and/or the transposer warps)
     __shared__ uint64_t empty_bar[kMaxStages];    // every multiply-accumulate that reads the stage has completed
     __shared__ uint64_t stg_full[kMaxStages];     // a staging box has landed
     __shared__ uint64_t stg_empty[kMaxStages];    // the transposer warps are done with it
+    __shared__ uint64_t pm_full[2];               // tap-major convolution: a pixel-major slab buffer has been written
+    __shared__ uint64_t pm_empty[2];              // ... and every multiply-accumulate that reads it has completed
     __shared__ uint64_t acc_full[2];              // an accumulator holds a finished tile
     __shared__ uint64_t acc_empty[2];             // the read-out warps (of both CTAs) have drained it
     __shared__ uint32_t tmem_slot;
@@ -1619,15 +1622,23 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t stage_bytes = g.a_stage_bytes + g.b_stage_bytes;
     const bool a_mn = g.a_mn != 0, b_mn = g.b_mn != 0;
+    // Tap-major convolution (see the one-tile kernel): operand A = re-packed filters by TMA; operand B = views of a
+    // pixel-major slab that the transposer warps write once per 32-channel block from a staged NCHW box.  Here the
+    // staging ring, the two slab buffers and the filter stages all run on across tile boundaries.
+    const bool tapm = g.tap_major != 0;
     const bool any_mn = a_mn || b_mn, any_km = !a_mn || !b_mn;
+    const bool any_stg = any_mn || tapm;
     const int b_rows = g.b_rows_cta;
+    const int RS = g.R * g.S;
+    const int blocks_per_tile = tapm ? kt_n * g.n_atoms / RS : 0;     // 32-channel blocks
 
     if (threadIdx.x == 32) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+        if (!tapm) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+        else asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
     }
     if (threadIdx.x == 0) {
-        const uint32_t full_count = (any_km ? 1u : 0u) + (any_mn ? (uint32_t)kPsTransposeWarps : 0u);
+        const uint32_t full_count = tapm ? 1u : (any_km ? 1u : 0u) + (any_mn ? (uint32_t)kPsTransposeWarps : 0u);
         for (int s = 0; s < g.stages; ++s) {
             mbar_init(smem_u32(&full_bar[s]), full_count);
             mbar_init(smem_u32(&empty_bar[s]), 1u);
@@ -1637,6 +1648,8 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             mbar_init(smem_u32(&stg_empty[s]), (uint32_t)kPsTransposeWarps);
         }
         for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&pm_full[a]), (uint32_t)kPsTransposeWarps);
+            mbar_init(smem_u32(&pm_empty[a]), 1u);
             mbar_init(smem_u32(&acc_full[a]), 1u);
             mbar_init(smem_u32(&acc_empty[a]), (uint32_t)(kPsEpilogueWarps * CG));
         }
@@ -1680,33 +1693,42 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         // its depth allows, whatever the multiply-accumulates are doing.
         const bool leader = elect_one();
         const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes), b_atom = (uint32_t)(b_rows * g.row_bytes);
-        const uint32_t km_bytes = (a_mn ? 0u : g.a_stage_bytes) + (b_mn ? 0u : g.b_stage_bytes);
+        const uint32_t km_bytes = (a_mn ? 0u : g.a_stage_bytes) + ((b_mn || tapm) ? 0u : g.b_stage_bytes);
         const uint32_t mn_bytes = (a_mn ? g.stg_a_bytes : 0u) + (b_mn ? g.stg_b_bytes : 0u);
         struct Cursor { int i, kt, m0, n0, bz, slot; uint32_t ph; long long it; };
         const long long total_it = (long long)my_tiles * kt_n;
+        const int inner_s = tapm ? blocks_per_tile : kt_n;            // staging boxes per tile
+        const long long total_s = (long long)my_tiles * inner_s;
         auto cur_init = [&](Cursor& c) {
             c.i = 0; c.kt = 0; c.slot = 0; c.ph = 0; c.it = 0; c.m0 = c.n0 = c.bz = 0;
             if (my_tiles > 0) decode(0, c.m0, c.n0, c.bz);
         };
-        auto cur_next = [&](Cursor& c, int depth) {
+        auto cur_next = [&](Cursor& c, int depth, int inner) {
             ++c.it;
             if (++c.slot == depth) { c.slot = 0; c.ph ^= 1u; }
-            if (++c.kt == kt_n) {
+            if (++c.kt == inner) {
                 c.kt = 0;
                 if (++c.i < my_tiles) decode(c.i, c.m0, c.n0, c.bz);
             }
         };
         Cursor cs, ck;
         cur_init(cs); cur_init(ck);
-        if (!any_mn) cs.it = total_it;
+        if (!any_stg) cs.it = total_s;
         if (!any_km) ck.it = total_it;
         bool ok = true;
         unsigned long long t_last = global_timer_ns();
         unsigned idle = 0;
-        while (cs.it < total_it || ck.it < total_it) {
+        while (cs.it < total_s || ck.it < total_it) {
             bool progressed = false;
-            if (cs.it < total_it && mbar_test_wait(smem_u32(&stg_empty[cs.slot]), cs.ph ^ 1u)) {
-                if (leader) {
+            if (cs.it < total_s && mbar_test_wait(smem_u32(&stg_empty[cs.slot]), cs.ph ^ 1u)) {
+                if (leader && tapm) {
+                    // the input rows of 32-channel block cs.kt behind this tile's pixels: one box that starts `gap` columns
+                    // left of the image and at the tile's first input row (zero fill supplies padding and gaps)
+                    const uint32_t bar = smem_u32(&stg_full[cs.slot]);
+                    mbar_expect_tx(bar, g.slab_box_bytes);
+                    tma_load_4d(tiles_base + g.slab_off + (uint32_t)cs.slot * g.slab_buf_bytes, &tmap_x, bar, -g.slab_gap,
+                                cs.n0 / g.slab_wp - g.ph, cs.kt * 32, cs.bz);
+                } else if (leader) {
                     const uint32_t bar = smem_u32(&stg_full[cs.slot]);
                     const int k0 = cs.kt * g.tile_k;
                     mbar_expect_tx(bar, mn_bytes);
@@ -1715,7 +1737,7 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                                           g.b_tma_batched ? cs.bz : 0);
                 }
                 __syncwarp();
-                cur_next(cs, g.stg_depth);
+                cur_next(cs, g.stg_depth, inner_s);
                 progressed = true;
             }
             if (ck.it < total_it && mbar_test_wait(smem_u32(&empty_bar[ck.slot]), ck.ph ^ 1u)) {
@@ -1737,7 +1759,7 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                             else tma_load_3d(dst, &tmap_a, bar, kc, ck.m0, a_bz);
                         }
                     }
-                    if (!b_mn) {
+                    if (!b_mn && !tapm) {
                         uint32_t dst = a_dst + g.a_stage_bytes;
                         int kc = k0;
 #pragma unroll 1
@@ -1748,7 +1770,7 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     }
                 }
                 __syncwarp();
-                cur_next(ck, g.stages);
+                cur_next(ck, g.stages, kt_n);
                 progressed = true;
             }
             if (progressed) { idle = 0; continue; }
@@ -1769,7 +1791,7 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             for (int pass = 0; pass < 2; ++pass) {
                 const long long issued = pass == 0 ? ck.it : cs.it;
                 const int depth = pass == 0 ? g.stages : g.stg_depth;
-                if ((pass == 0 && (!any_km || rank != 0)) || (pass == 1 && !any_mn)) continue;
+                if ((pass == 0 && (!any_km || rank != 0)) || (pass == 1 && !any_stg)) continue;
                 const long long first = issued > depth ? issued - depth : 0;
                 for (long long it = first; it < issued; ++it) {
                     const uint32_t bar = pass == 0 ? smem_u32(&full_bar[it % depth]) : smem_u32(&stg_full[it % depth]);
@@ -1800,6 +1822,7 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const uint32_t stage_step = stage_bytes >> 4;
             const uint32_t a_atom = (uint32_t)(kHwTileM * g.row_bytes) >> 4, b_atom = (uint32_t)(b_rows * g.row_bytes) >> 4;
             const uint32_t b_off = g.a_stage_bytes >> 4;
+            uint32_t gblock = 0;                         // tap-major: 32-channel blocks consumed so far, over all tiles
             for (int i = 0; i < my_tiles && ok; ++i) {
                 const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
                 // the read-out of the tile that used this accumulator two tiles ago has finished
@@ -1808,6 +1831,43 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (!__all_sync(0xffffffffu, freed)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * (uint32_t)g.tile_n;
+                if (tapm) {
+                    // the B tile of reduction tile kt = (channel block, taps) is the block's pixel-major slab read from row
+                    // lin0 + r * wp + s on: only the descriptor's start address changes from tap to tap
+                    int m0t, n0t, bzt;
+                    decode(i, m0t, n0t, bzt);
+                    const uint32_t pm0 = tiles_base + g.pm_off;
+                    const int lin0 = (n0t - (n0t / g.slab_wp) * g.slab_wp) + g.slab_gap - g.pw;
+                    int tap = 0, fr = 0, fs = 0;
+                    for (int kt = 0; kt < kt_n; ++kt) {
+                        bool got = mbar_wait(smem_u32(&full_bar[st]), ph, abortp, g.status, 2u, g.wait_ns);        // the filter tile
+                        if (tap == 0 && got) got = mbar_wait(smem_u32(&pm_full[gblock & 1u]), (gblock >> 1) & 1u, abortp, g.status, 7u, g.wait_ns);
+                        if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+                        tc_fence_after();
+                        if (leader) {
+                            uint32_t a_lo = a_lo0 + st * stage_step;
+                            int r2 = fr, s2 = fs;
+#pragma unroll 1
+                            for (int t = 0; t < g.n_atoms; ++t, a_lo += a_atom) {
+                                const uint32_t row = (uint32_t)(lin0 + r2 * g.slab_wp + s2);
+                                const uint32_t b_lo = d_lo + (((pm0 + (gblock & 1u) * g.pm_buf_bytes + row * 128u) & 0x3FFFFu) >> 4);
+#pragma unroll
+                                for (int k8 = 0; k8 < 4; ++k8)
+                                    mma_tf32_cg<CG>(d_tmem, ((uint64_t)d_hi << 32) | (uint64_t)(a_lo + 2u * (uint32_t)k8),
+                                                    ((uint64_t)d_hi << 32) | (uint64_t)(b_lo + 2u * (uint32_t)k8), g.idesc,
+                                                    (kt > 0 || t > 0 || k8 > 0) ? 1u : 0u);
+                                if (++s2 == g.S) { s2 = 0; ++r2; }
+                            }
+                            mma_commit_cg<CG>(smem_u32(&empty_bar[st]));                           // filter stage reusable
+                            if (tap + g.n_atoms == RS) mma_commit_cg<CG>(smem_u32(&pm_empty[gblock & 1u]));   // slab buffer reusable
+                        }
+                        __syncwarp();
+                        for (int t = 0; t < g.n_atoms; ++t) if (++fs == g.S) { fs = 0; ++fr; }
+                        tap += g.n_atoms;
+                        if (tap == RS) { tap = 0; fr = 0; fs = 0; ++gblock; }
+                        if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
+                    }
+                } else
                 for (int kt = 0; kt < kt_n; ++kt) {
                     const bool got = mbar_wait(smem_u32(&full_bar[st]), ph, abortp, g.status, 2u, g.wait_ns);
                     if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
@@ -1835,7 +1895,64 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
     } else if (warp < 2 + kPsTransposeWarps) {
         // ---------------- transposers ----------------
-        if (any_mn) {
+        if (tapm) {
+            // staging box [32 channels][in_rows][wp] -> pixel-major slab: one 128-byte row per staged position (32
+            // channels), 16-byte chunks swizzled by the row's absolute address like a TMA 128-byte tile.  Warp tw moves
+            // the channel groups tw and tw + 4 of every position; lanes walk positions.
+            const int tw = warp - 2;
+            const int tt = (int)threadIdx.x - 64;
+            const uint32_t st0 = tiles_base + g.slab_off, pm0 = tiles_base + g.pm_off;
+            const int npix = g.slab_in_rows * g.slab_wp;
+            // rows a view can touch beyond the transposed range must hold finite numbers: clear both buffers once
+            for (uint32_t o = (uint32_t)tt * 16u; o < 2u * g.pm_buf_bytes; o += 32u * kPsTransposeWarps * 16u)
+                st_shared_v4(pm0 + o, 0.f, 0.f, 0.f, 0.f);
+            if (g.slab_box_ch < 32)                      // channels beyond the TMA box (which may already be landing) read as zero
+                for (int sl = 0; sl < g.stg_depth; ++sl)
+                    for (uint32_t o = g.slab_box_bytes + (uint32_t)tt * 16u; o < g.slab_buf_bytes; o += 32u * kPsTransposeWarps * 16u)
+                        st_shared_v4(st0 + (uint32_t)sl * g.slab_buf_bytes + o, 0.f, 0.f, 0.f, 0.f);
+            asm volatile("bar.sync 3, %0;" ::"n"(32 * kPsTransposeWarps) : "memory");
+            const uint32_t ch_bytes = 4u * (uint32_t)g.slab_chpitch;
+            uint32_t sst = 0, sph = 0, gb = 0;
+            bool ok = true;
+            const long long total_blocks = (long long)my_tiles * blocks_per_tile;
+            for (long long j = 0; j < total_blocks && ok; ++j, ++gb) {
+                const uint32_t b = gb & 1u;
+                if (!mbar_wait(smem_u32(&stg_full[sst]), sph, abortp, g.status, 6u, g.wait_ns) ||
+                    !mbar_wait(smem_u32(&pm_empty[b]), ((gb >> 1) & 1u) ^ 1u, abortp, g.status, 8u, g.wait_ns)) { ok = false; break; }
+                const uint32_t dst = pm0 + b * g.pm_buf_bytes;
+#pragma unroll 1
+                for (int grp = tw; grp < 8; grp += kPsTransposeWarps) {
+                    const uint32_t src = st0 + sst * g.slab_buf_bytes + (uint32_t)(4 * grp) * ch_bytes;
+                    for (int p0 = lane; p0 < npix; p0 += 128) {
+                        float v[4][4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int pix = min(p0 + 32 * u, npix - 1);
+                            const uint32_t a = src + 4u * (uint32_t)pix;
+                            v[u][0] = ld_shared_f32(a);
+                            v[u][1] = ld_shared_f32(a + ch_bytes);
+                            v[u][2] = ld_shared_f32(a + 2u * ch_bytes);
+                            v[u][3] = ld_shared_f32(a + 3u * ch_bytes);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int pix = p0 + 32 * u;
+                            if (pix < npix) {
+                                const uint32_t rowa = dst + 128u * (uint32_t)pix;
+                                st_shared_v4(rowa + ((((uint32_t)grp) ^ ((rowa >> 7) & 7u)) << 4), v[u][0], v[u][1], v[u][2], v[u][3]);
+                            }
+                        }
+                    }
+                }
+                fence_proxy_async_shared();              // generic-proxy stores -> visible to the tensor core's reads
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&pm_full[b]));
+                    mbar_arrive(smem_u32(&stg_empty[sst]));
+                }
+                if (++sst == (uint32_t)g.stg_depth) { sst = 0; sph ^= 1u; }
+            }
+        } else if (any_mn) {
             const int tw = warp - 2;
             uint32_t st = 0, ph = 0, sst = 0, sph = 0;
             bool ok = true;
@@ -1867,7 +1984,7 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         e.hi = g.act == TT_ACT_RELU6 ? 6.f : INFINITY;
         e.gelu = g.act == TT_ACT_GELU_ERF;
         e.vec = (g.vec_store & 1) != 0;
-        e.lin_wp = 0; e.lin_q = 0; e.lin_p = 0;
+        e.lin_wp = tapm ? g.slab_wp : 0; e.lin_q = g.Q; e.lin_p = g.Pout;
         const bool transposed = g.y_ns == 1 && g.y_ms != 1;
         const uint32_t stg = tiles_base + g.epi_off + (uint32_t)ew * (uint32_t)kStageBytesPerWarp;
         bool ok = true;
@@ -1924,7 +2041,7 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         v[j] += b.x; v[j + 1] += b.y; v[j + 2] += b.z; v[j + 3] += b.w;
                     }
                 }
-                const bool full = cnt >= 32 && m_first + 32 <= g.M && (e.vec || !transposed);
+                const bool full = !tapm && cnt >= 32 && m_first + 32 <= g.M && (e.vec || !transposed);
                 if (e.rbase == nullptr) {
                     if (e.gelu) {
 #pragma unroll
@@ -2506,7 +2623,8 @@ cudaError_t launch_gemm(const tt_apply_info& I, const GemmArgs& g, const void* t
 }
 
 // The persistent form: one CTA (or one pair of CTAs, as a cluster of two) per SM.
-cudaError_t launch_gemm_ps(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, cudaStream_t st) {
+cudaError_t launch_gemm_ps(const tt_apply_info& I, const GemmArgs& g, const void* tmap_a, const void* tmap_b, const void* tmap_x,
+                           cudaStream_t st) {
     static int attr_set_for = -1, sm_count = 148;
     int dev = 0;
     cudaGetDevice(&dev);
@@ -2518,9 +2636,10 @@ cudaError_t launch_gemm_ps(const tt_apply_info& I, const GemmArgs& g, const void
         cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
         attr_set_for = dev;
     }
-    CUtensorMap ta, tb;
+    CUtensorMap ta, tb, tx;
     memcpy(&ta, tmap_a, sizeof ta);
     memcpy(&tb, tmap_b, sizeof tb);
+    memcpy(&tx, tmap_x, sizeof tx);
     const int cg = g.cta_group == 2 ? 2 : 1;
     const long long units = std::min<long long>(g.total_tiles, sm_count / cg);
     cudaLaunchConfig_t cfg{};
@@ -2537,8 +2656,8 @@ cudaError_t launch_gemm_ps(const tt_apply_info& I, const GemmArgs& g, const void
         ++n_attr;
     }
     cfg.attrs = attr; cfg.numAttrs = (unsigned)n_attr;
-    if (cg == 2) return cudaLaunchKernelEx(&cfg, tt_gemm_ps_kernel<2>, ta, tb, g);
-    return cudaLaunchKernelEx(&cfg, tt_gemm_ps_kernel<1>, ta, tb, g);
+    if (cg == 2) return cudaLaunchKernelEx(&cfg, tt_gemm_ps_kernel<2>, ta, tb, tx, g);
+    return cudaLaunchKernelEx(&cfg, tt_gemm_ps_kernel<1>, ta, tb, tx, g);
 }
 
 // Can a cluster of `cluster` CTAs with this much shared memory each be resident at all?

@@ -108,6 +108,8 @@ GEMM_RECORDS = [
     tc(tile_n=64, tile_k=32, stages=3, persistent=1, cta_group=2, mma_m_axis=1),
     tc(tile_n=256, tile_k=32, stages=2, persistent=1, cta_group=2, mma_m_axis=2),
     tc(tile_n=32, tile_k=128, stages=2, persistent=1, cta_group=2, raster=1, mma_m_axis=1),
+    tc(tile_n=128, tile_k=32, stages=3, k_order=1, persistent=1, mma_m_axis=1),          # tap-major in the persistent form
+    tc(tile_n=64, tile_k=96, stages=2, k_order=1, persistent=1, raster=1, mma_m_axis=1),
     tc(tile_n=64, tile_k=32, stages=2, ctas_per_sm=2, mma_m_axis=1),
     tc(tile_n=128, tile_k=16, stages=3, ctas_per_sm=1, split_k=2, mma_m_axis=2),
 ]
@@ -123,7 +125,7 @@ def check_all_records(spec, seed, records=GEMM_RECORDS):
     assert all(probe.check(r)[0] in (B.TT_OK, B.TT_ERR_RESOURCE) for r in records)
     assert probe.check(probe.default_schedule())[0] == B.TT_OK
     probe.close()
-    assert len(valid) >= len(records) - 5
+    assert len(valid) >= len(records) - 6
     re = elem_ref(spec, a, ref)
     outs = [run_spec(spec, r, a, ref, ref_elem=re) for r in valid]
     # a schedule changes speed, never semantics: every valid record gives the same output up to the order of the
@@ -800,3 +802,33 @@ def test_constant_weights_are_fetched_early_and_results_do_not_change():
         results.append(y)
         del first
     np.testing.assert_array_equal(results[0], results[1])
+
+
+@pytest.mark.parametrize("spec", [
+    W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(20, 40, 20, 20, 72, 3, 3, 1, 1, True, B.TT_ACT_RELU), 1, "ps_tap_conv3x3_n20", "uniform"),
+    W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(9, 33, 12, 16, 136, 5, 3, 1, 2, True, B.TT_ACT_RELU6), 1, "ps_tap_conv5x3_n9", "uniform"),
+    W.Spec(B.TT_OP_CONV2D, B.conv2d_shapes(30, 8, 8, 8, 16, 3, 3, 1, 1, False, B.TT_ACT_NONE), 1, "ps_tap_small_n30", "uniform"),
+], ids=lambda s: s.name)
+def test_persistent_tap_major_convolution_walks_many_tiles(spec):
+    """The tap-major reduction order in the persistent form: filter stages, the staging ring and the two pixel-major
+    slab buffers all run on across tile boundaries (several tiles per CTA, one or several 32-channel blocks per tile,
+    a partial last block, two filter tiles).  Same values as the one-tile form and as the stored reduction order."""
+    a = W.make_inputs(spec, 92)
+    ref = util.oracle_ref(spec, a)
+    re = elem_ref(spec, a, ref)
+    outs = []
+    probe = spec.workload()
+    for rec in (tc(tile_n=32, tile_k=32, stages=3, mma_m_axis=1),
+                tc(tile_n=48, tile_k=32, stages=3, k_order=1, mma_m_axis=1),
+                tc(tile_n=48, tile_k=32, stages=3, k_order=1, persistent=1, mma_m_axis=1),
+                tc(tile_n=16, tile_k=96, stages=2, k_order=1, persistent=1, raster=1, mma_m_axis=1),
+                tc(tile_n=96, tile_k=32, stages=6, k_order=1, persistent=1, mma_m_axis=1),
+                tc(tile_n=256, tile_k=64, stages=2, k_order=1, persistent=1, mma_m_axis=1)):
+        st, info = probe.check(rec)
+        assert st == B.TT_OK
+        if rec.persistent:
+            assert info.legal.persistent == 1 and info.legal.k_order == 1
+        outs.append(run_spec(spec, rec, a, ref, ref_elem=re))
+    probe.close()
+    for y in outs[1:]:
+        assert util.rel_l2(y, outs[0]) <= INVARIANCE_TOL
