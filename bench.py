@@ -109,7 +109,8 @@ def workload_name(model, specs, pool_sources):
 def config_dict(model, specs, pool_sources):
     return {"workload": workload_name(model, specs, pool_sources), "l2": "flushed between steps (256 MB write)",
             "replay": "one CUDA graph per data-chained model pass", "multi_gpu": "independent replicas",
-            "weights": "declared constant to the library (a kernel may fetch them before it waits for its predecessor)"}
+            "weights": "declared constant to the library (a kernel may fetch them before it waits for its predecessor)",
+            "evaluation": "every (kernel, record) pair timed standalone with warm activations and rotating copies of the weights"}
 
 
 class ClockSampler(threading.Thread):
@@ -308,6 +309,28 @@ class Bench:
             body()
         return graph
 
+    def weight_sets(self, spec, t, cap=64):
+        """Tensor sets for the evaluator that differ only in the layer's parameters: inside a model a layer finds its
+        input in the cache (the previous layer just wrote it) and its weights in memory (every layer has its own), so
+        each kernel is timed walking copies of w and bias whose total footprint exceeds twice the L2 (at most `cap`
+        copies: layers with small weights stay partly warm, as they would next to their neighbours' weights)."""
+        torch, B = self.torch, self.B
+        one = B.tensors(t["x"], t["w"], t["bias"], t["residual"], t["y"])
+        if spec.op in (B.TT_OP_SOFTMAX, B.TT_OP_BATCH_MATMUL) or t["w"] is None:
+            return None, [one]
+        nw, nb = t["w"].numel(), (t["bias"].numel() if t["bias"] is not None else 0)
+        pw, pb = (nw + 63) // 64 * 64, (nb + 63) // 64 * 64
+        n_sets = int(min(cap, max(1, (2 * 126e6) // (4 * (pw + pb)) + 1)))
+        if n_sets == 1:
+            return None, [one]
+        arena = torch.zeros(n_sets, pw + pb, dtype=torch.float32, device=self.dev)
+        arena[:, :nw] = t["w"].reshape(1, -1)
+        if nb:
+            arena[:, pw:pw + nb] = t["bias"].reshape(1, -1)
+        sets = [B.tensors(t["x"], arena[i, :nw].view(t["w"].shape), arena[i, pw:pw + nb] if nb else None, t["residual"], t["y"])
+                for i in range(n_sets)]
+        return arena, sets
+
     def cold_sets(self, spec, arrays, max_sets=2048):
         """Tensor sets carved out of one arena whose total footprint exceeds twice the L2, so that a launch that walks
         them round-robin never finds its operands cached."""
@@ -353,7 +376,9 @@ class Bench:
         o = B.tt_tune_opts()
         o.include_default = 1
         o.timing.warmup_batches, o.timing.batches, o.timing.min_batch_us, o.timing.use_graph = 3, 10, 200, 1
-        res = B.transfer_tune(list(wls), list(tts), pool, o)
+        eval_sets = [self.weight_sets(sp, t) for sp, t in zip(specs, dev_t)]
+        res = B.transfer_tune(list(wls), [sets for _, sets in eval_sets], pool, o)
+        del eval_sets
         n_cols = len(pool) + 1
         chosen = res["chosen"]
         use = [sp.use_count for sp in specs]

@@ -312,6 +312,13 @@ tt_status tt_transfer_tune(tt_workload* const* model_workloads, const tt_tensors
                            const tt_schedule_record* pool, size_t n_pool, const tt_tune_opts* o, void* cuda_stream,
                            tt_tune_result* out);
 
+/* The same with several tensor sets per workload: workload i owns set_counts[i] consecutive entries of `tensors` and
+ * every timed batch walks them round-robin.  Sets that differ only in w and bias, with a total footprint beyond the L2,
+ * time a kernel the way it runs inside a model: weights from memory, activations from the cache. */
+tt_status tt_transfer_tune_sets(tt_workload* const* model_workloads, const tt_tensors* tensors, const size_t* set_counts,
+                                size_t n_wl, const tt_schedule_record* pool, size_t n_pool, const tt_tune_opts* o,
+                                void* cuda_stream, tt_tune_result* out);
+
 /* Native tuning of one workload (stands in for the auto-scheduler that fills a pool, Section 2): exhaustive walk
  * over a grid of records of the workload's family, each timed with `o`; writes the best `top_k` records (fastest
  * first) to out_records/out_us and their number to n_out.  level 0 = coarse grid, 1 = full grid. */

@@ -125,6 +125,9 @@ EXPORTS = {
                             C.POINTER(i32)]),
     "tt_transfer_tune": (i32, [C.POINTER(C.c_void_p), C.POINTER(tt_tensors), C.c_size_t, C.POINTER(tt_schedule_record),
                                C.c_size_t, C.POINTER(tt_tune_opts), C.c_void_p, C.POINTER(tt_tune_result)]),
+    "tt_transfer_tune_sets": (i32, [C.POINTER(C.c_void_p), C.POINTER(tt_tensors), C.POINTER(C.c_size_t), C.c_size_t,
+                                    C.POINTER(tt_schedule_record), C.c_size_t, C.POINTER(tt_tune_opts), C.c_void_p,
+                                    C.POINTER(tt_tune_result)]),
     "tt_grid_tune": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(tt_timing_opts), i32, C.c_size_t,
                            C.POINTER(tt_schedule_record), C.POINTER(f32), C.POINTER(C.c_size_t), C.POINTER(i32)]),
     "tt_record_neighbours": (i32, [C.c_void_p, C.POINTER(tt_schedule_record), C.POINTER(tt_schedule_record), C.c_size_t,
@@ -452,7 +455,12 @@ def transfer_tune(workloads, tensor_sets, pool, opts: tt_tune_opts | None = None
     n_wl, n_pool = len(workloads), len(pool)
     n_cols = n_pool + 1
     handles = (C.c_void_p * n_wl)(*[w.handle for w in workloads])
-    tens = (tt_tensors * n_wl)(*tensor_sets)
+    # an entry of tensor_sets may be one tt_tensors or a list of them (several sets, walked round-robin while timing)
+    multi = any(not isinstance(t, tt_tensors) for t in tensor_sets)
+    groups = [[t] if isinstance(t, tt_tensors) else list(t) for t in tensor_sets]
+    flat_sets = [t for g in groups for t in g]
+    tens = (tt_tensors * len(flat_sets))(*flat_sets)
+    counts = (C.c_size_t * n_wl)(*[len(g) for g in groups])
     parr = (tt_schedule_record * max(n_pool, 1))(*pool)
     chosen = (i32 * n_wl)()
     best = (f32 * n_wl)()
@@ -463,8 +471,12 @@ def transfer_tune(workloads, tensor_sets, pool, opts: tt_tune_opts | None = None
     if opts is None:
         opts = tt_tune_opts()
         opts.include_default = 1
-    _check(lib().tt_transfer_tune(handles, tens, n_wl, parr, n_pool, C.byref(opts), _stream(), C.byref(res)),
-           "tt_transfer_tune")
+    if multi:
+        _check(lib().tt_transfer_tune_sets(handles, tens, counts, n_wl, parr, n_pool, C.byref(opts), _stream(), C.byref(res)),
+               "tt_transfer_tune_sets")
+    else:
+        _check(lib().tt_transfer_tune(handles, tens, n_wl, parr, n_pool, C.byref(opts), _stream(), C.byref(res)),
+               "tt_transfer_tune")
     return {
         "chosen": list(chosen), "best_us": list(best),
         "times_us": [[times[i * n_cols + j] for j in range(n_cols)] for i in range(n_wl)],

@@ -540,8 +540,26 @@ tt_status tt_time(tt_workload* w, const tt_tensors* sets, size_t n_sets, void* c
     return time_applied(w, sets, n_sets, static_cast<cudaStream_t>(cuda_stream), o, out);
 }
 
+static tt_status transfer_tune_impl(tt_workload* const* wls, const tt_tensors* tensors, const size_t* set_counts, size_t n_wl,
+                                    const tt_schedule_record* pool, size_t n_pool, const tt_tune_opts* oin, void* cuda_stream,
+                                    tt_tune_result* out);
+
 tt_status tt_transfer_tune(tt_workload* const* wls, const tt_tensors* tensors, size_t n_wl, const tt_schedule_record* pool,
                            size_t n_pool, const tt_tune_opts* oin, void* cuda_stream, tt_tune_result* out) {
+    return transfer_tune_impl(wls, tensors, nullptr, n_wl, pool, n_pool, oin, cuda_stream, out);
+}
+
+tt_status tt_transfer_tune_sets(tt_workload* const* wls, const tt_tensors* tensors, const size_t* set_counts, size_t n_wl,
+                                const tt_schedule_record* pool, size_t n_pool, const tt_tune_opts* oin, void* cuda_stream,
+                                tt_tune_result* out) {
+    if (!set_counts) return TT_ERR_INVALID_ARG;
+    for (size_t i = 0; i < n_wl; ++i) if (set_counts[i] == 0) return TT_ERR_INVALID_ARG;
+    return transfer_tune_impl(wls, tensors, set_counts, n_wl, pool, n_pool, oin, cuda_stream, out);
+}
+
+static tt_status transfer_tune_impl(tt_workload* const* wls, const tt_tensors* tensors, const size_t* set_counts, size_t n_wl,
+                                    const tt_schedule_record* pool, size_t n_pool, const tt_tune_opts* oin, void* cuda_stream,
+                                    tt_tune_result* out) {
     if (!wls || !tensors || !out || (n_pool && !pool) || !out->chosen || !out->best_us || !out->times_us || !out->status)
         return TT_ERR_INVALID_ARG;
     tt_tune_opts o{};
@@ -553,9 +571,13 @@ tt_status tt_transfer_tune(tt_workload* const* wls, const tt_tensors* tensors, s
     const size_t n_cols = n_pool + 1;
     int timed = 0, invalid = 0;
     std::vector<tt_schedule_record> cols(n_cols);
+    size_t first_set = 0;
     for (size_t i = 0; i < n_wl; ++i) {
         tt_workload* w = wls[i];
         if (!w) return TT_ERR_INVALID_ARG;
+        const size_t n_sets = set_counts ? set_counts[i] : 1;
+        const tt_tensors* sets = tensors + first_set;
+        first_set += n_sets;
         tt_default_schedule(w, &cols[0]);
         for (size_t j = 0; j < n_pool; ++j) cols[j + 1] = pool[j];
         for (size_t j = 0; j < n_cols; ++j) {
@@ -567,7 +589,7 @@ tt_status tt_transfer_tune(tt_workload* const* wls, const tt_tensors* tensors, s
             tt_status s = apply_impl(w, &cols[j], j == 0 ? TT_MODE_LEGALISE : o.mode, j == 0 ? 0 : o.strict_class, nullptr);
             if (s == TT_OK) {
                 tt_timing tm{};
-                s = time_applied(w, &tensors[i], 1, st, &o.timing, &tm);
+                s = time_applied(w, sets, n_sets, st, &o.timing, &tm);
                 if (s == TT_OK) { cell = tm.median_us; ++timed; }
             }
             cst = s;
