@@ -526,7 +526,7 @@ def saturating_points(bench):
         (conv(32, 256, 56, 64, 1, 0), "hbm",
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1), tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=2),
           tc(tile_n=64, tile_k=32, stages=2, mma_m_axis=2, slab_tiles=1), tc(tile_n=64, tile_k=64, stages=2, mma_m_axis=2, persistent=1),
-          tc(tile_n=64, tile_k=32, stages=2, mma_m_axis=2, persistent=1)]),
+          tc(tile_n=64, tile_k=32, stages=4, mma_m_axis=2, persistent=1)]),
         (conv(32, 64, 56, 256, 1, 0), "hbm",
          [tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=2, slab_tiles=1), tc(tile_n=128, tile_k=64, stages=2, mma_m_axis=1, persistent=1),
           tc(tile_n=256, tile_k=32, stages=2, mma_m_axis=1, persistent=1)]),

@@ -1557,39 +1557,58 @@ constexpr int kPsEpilogueWarps = 4;
 
 // Transpose one staged box [tile_k][rows] (row index contiguous) into the K-major swizzled stage tile.  A task is a
 // (32-row block, four consecutive reduction indices) pair: lanes walk rows (conflict-free 4-byte loads), each lane
-// assembles its row's four values and writes one 16-byte chunk.
+// assembles its row's four values and writes one 16-byte chunk.  What bounds this routine is its instruction count, so
+// a warp keeps a row block (or shares one with other warps, taking alternate chunks) and everything that depends on the
+// row is worked out once; per chunk there are four loads, one store and a few additions.
+template <int KB>
+__device__ __forceinline__ void ps_transpose_chunks(uint32_t src, uint32_t src_step, uint32_t dst_row, uint32_t swz, int c0, int step, int n_ch,
+                                                    uint32_t k_bytes, int atom_shift, int atom_k, uint32_t atom_bytes, bool in_tile) {
+    for (; c0 < n_ch; c0 += step * KB, src += src_step * KB) {
+        float val[KB][4];
+#pragma unroll
+        for (int b = 0; b < KB; ++b) {
+            const uint32_t a = src + (c0 + b * step < n_ch ? (uint32_t)b * src_step : 0u);
+            val[b][0] = ld_shared_f32(a);
+            val[b][1] = ld_shared_f32(a + k_bytes);
+            val[b][2] = ld_shared_f32(a + 2u * k_bytes);
+            val[b][3] = ld_shared_f32(a + 3u * k_bytes);
+        }
+#pragma unroll
+        for (int b = 0; b < KB; ++b) {
+            const int ci = c0 + b * step;
+            if (ci < n_ch && in_tile) {
+                const int kk = ci << 2;
+                st_shared_v4(dst_row + (uint32_t)(kk >> atom_shift) * atom_bytes + ((uint32_t)((kk & (atom_k - 1)) << 2) ^ swz),
+                             val[b][0], val[b][1], val[b][2], val[b][3]);
+            }
+        }
+    }
+}
+
 __device__ __forceinline__ void ps_transpose(uint32_t stg, uint32_t tile, int rows, int tile_k, int atom_k, int row_bytes,
-                                             int swz_mask, int tw, int lane) {
+                                             int swz_mask, int tw, int nw, int lane) {
     const int atom_shift = atom_k == 32 ? 5 : (atom_k == 16 ? 4 : 3);
     const int shift = row_bytes == 128 ? 0 : (row_bytes == 64 ? 1 : 2);
     const uint32_t atom_bytes = (uint32_t)rows * (uint32_t)row_bytes;
     const int n_rb = (rows + 31) >> 5, n_ch = tile_k >> 2;
-    const int n_tasks = n_rb * n_ch;
-    constexpr int kBatch = 4;
-    for (int t0 = tw; t0 < n_tasks; t0 += kPsTransposeWarps * kBatch) {
-        float val[kBatch][4];
-        uint32_t dst[kBatch];
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-            const int t = t0 + b * kPsTransposeWarps;
-            const bool live = t < n_tasks;                   // warp-uniform
-            const int tt = live ? t : 0;
-            const int ci = tt / n_rb, rb = tt - ci * n_rb;
-            const int kk = ci << 2;
-            const int row = rb * 32 + lane;
-            const bool in_tile = live && row < rows;
-            dst[b] = in_tile ? tile + (uint32_t)(kk >> atom_shift) * atom_bytes + (uint32_t)row * (uint32_t)row_bytes +
-                                   ((uint32_t)((kk & (atom_k - 1)) << 2) ^ ((uint32_t)((row >> shift) & swz_mask) << 4))
-                             : 0xffffffffu;
-            const uint32_t src = stg + 4u * (uint32_t)(kk * rows + (row < rows ? row : rows - 1));
-            val[b][0] = ld_shared_f32(src);
-            val[b][1] = ld_shared_f32(src + 4u * (uint32_t)rows);
-            val[b][2] = ld_shared_f32(src + 8u * (uint32_t)rows);
-            val[b][3] = ld_shared_f32(src + 12u * (uint32_t)rows);
-        }
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b)
-            if (dst[b] != 0xffffffffu) st_shared_v4(dst[b], val[b][0], val[b][1], val[b][2], val[b][3]);
+    const uint32_t k_bytes = 4u * (uint32_t)rows;                  // distance between consecutive reduction indices in the box
+    // row blocks to the nw warps that work on this machine: with nw or more blocks (or a count that does not divide nw) a warp
+    // takes blocks tw, tw + nw, ... and every chunk of them; with fewer, nw / n_rb warps share a block and take alternate chunks
+    int rb_first, rb_step, c_first, c_step;
+    const bool shared_block = n_rb < nw && (nw % n_rb) == 0;
+    if (!shared_block) { rb_first = tw; rb_step = nw; c_first = 0; c_step = 1; }
+    else { rb_first = tw % n_rb; rb_step = n_rb; c_first = tw / n_rb; c_step = nw / n_rb; }   // (rb_step only ends the loop)
+    for (int rb = rb_first; rb < n_rb; rb += rb_step) {
+        const int row = rb * 32 + lane;
+        const bool in_tile = row < rows;
+        const uint32_t src = stg + 4u * (uint32_t)(in_tile ? row : rows - 1) + (uint32_t)c_first * 4u * k_bytes;
+        const uint32_t dst_row = tile + (uint32_t)row * (uint32_t)row_bytes;
+        const uint32_t swz = (uint32_t)((row >> shift) & swz_mask) << 4;
+        const int mine = (n_ch - c_first + c_step - 1) / c_step;
+        if (mine <= 2) ps_transpose_chunks<2>(src, (uint32_t)c_step * 4u * k_bytes, dst_row, swz, c_first, c_step, n_ch, k_bytes, atom_shift, atom_k, atom_bytes, in_tile);
+        else if (mine <= 4) ps_transpose_chunks<4>(src, (uint32_t)c_step * 4u * k_bytes, dst_row, swz, c_first, c_step, n_ch, k_bytes, atom_shift, atom_k, atom_bytes, in_tile);
+        else ps_transpose_chunks<8>(src, (uint32_t)c_step * 4u * k_bytes, dst_row, swz, c_first, c_step, n_ch, k_bytes, atom_shift, atom_k, atom_bytes, in_tile);
+        if (shared_block) break;                                     // this warp has no other block
     }
 }
 
@@ -1631,6 +1650,10 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const int b_rows = g.b_rows_cta;
     const int RS = g.R * g.S;
     const int blocks_per_tile = tapm ? kt_n * g.n_atoms / RS : 0;     // 32-channel blocks
+    // The transposer warps work as two groups on alternate reduction tiles when both rings are at least two deep: while
+    // one group waits for its buffers and hands its stage over, the other copies.
+    const int tr_groups = (g.stages >= 2 && g.stg_depth >= 2) ? 2 : 1;
+    const int tr_warps = kPsTransposeWarps / tr_groups;               // warps per box
 
     if (threadIdx.x == 32) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
@@ -1638,14 +1661,14 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         else asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_x) : "memory");
     }
     if (threadIdx.x == 0) {
-        const uint32_t full_count = tapm ? 1u : (any_km ? 1u : 0u) + (any_mn ? (uint32_t)kPsTransposeWarps : 0u);
+        const uint32_t full_count = tapm ? 1u : (any_km ? 1u : 0u) + (any_mn ? (uint32_t)tr_warps : 0u);
         for (int s = 0; s < g.stages; ++s) {
             mbar_init(smem_u32(&full_bar[s]), full_count);
             mbar_init(smem_u32(&empty_bar[s]), 1u);
         }
         for (int s = 0; s < g.stg_depth; ++s) {
             mbar_init(smem_u32(&stg_full[s]), 1u);
-            mbar_init(smem_u32(&stg_empty[s]), (uint32_t)kPsTransposeWarps);
+            mbar_init(smem_u32(&stg_empty[s]), (uint32_t)(tapm ? kPsTransposeWarps : tr_warps));
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&pm_full[a]), (uint32_t)kPsTransposeWarps);
@@ -1953,25 +1976,27 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (++sst == (uint32_t)g.stg_depth) { sst = 0; sph ^= 1u; }
             }
         } else if (any_mn) {
-            const int tw = warp - 2;
-            uint32_t st = 0, ph = 0, sst = 0, sph = 0;
-            bool ok = true;
-            for (int i = 0; i < my_tiles && ok; ++i)
-                for (int kt = 0; kt < kt_n; ++kt) {
-                    if (!mbar_wait(smem_u32(&stg_full[sst]), sph, abortp, g.status, 6u, g.wait_ns) ||
-                        !mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, abortp, g.status, 3u, g.wait_ns)) { ok = false; break; }
-                    const uint32_t a_s = tiles_base + st * stage_bytes, b_s = a_s + g.a_stage_bytes;
-                    if (a_mn) ps_transpose(tiles_base + g.a_stg_off + sst * g.stg_a_bytes, a_s, kHwTileM, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, tw, lane);
-                    if (b_mn) ps_transpose(tiles_base + g.b_stg_off + sst * g.stg_b_bytes, b_s, b_rows, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, tw, lane);
-                    fence_proxy_async_shared();          // generic-proxy stores -> visible to the tensor core's reads
-                    __syncwarp();
-                    if (lane == 0) {
-                        mbar_arrive(smem_u32(&full_bar[st]));
-                        mbar_arrive(smem_u32(&stg_empty[sst]));
-                    }
-                    if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
-                    if (++sst == (uint32_t)g.stg_depth) { sst = 0; sph ^= 1u; }
+            const int grp = (warp - 2) / tr_warps, tw = (warp - 2) - grp * tr_warps;
+            int st = grp % g.stages, sst = grp % g.stg_depth;
+            uint32_t ph = (uint32_t)(grp / g.stages) & 1u, sph = (uint32_t)(grp / g.stg_depth) & 1u;
+            const long long total_it = (long long)my_tiles * kt_n;
+            for (long long it = grp; it < total_it; it += tr_groups) {
+                if (!mbar_wait(smem_u32(&stg_full[sst]), sph, abortp, g.status, 6u, g.wait_ns) ||
+                    !mbar_wait(smem_u32(&empty_bar[st]), ph ^ 1u, abortp, g.status, 3u, g.wait_ns)) break;
+                const uint32_t a_s = tiles_base + (uint32_t)st * stage_bytes, b_s = a_s + g.a_stage_bytes;
+                if (a_mn) ps_transpose(tiles_base + g.a_stg_off + (uint32_t)sst * g.stg_a_bytes, a_s, kHwTileM, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, tw, tr_warps, lane);
+                if (b_mn) ps_transpose(tiles_base + g.b_stg_off + (uint32_t)sst * g.stg_b_bytes, b_s, b_rows, g.tile_k, g.atom_k, g.row_bytes, g.swz_mask, tw, tr_warps, lane);
+                fence_proxy_async_shared();              // generic-proxy stores -> visible to the tensor core's reads
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&full_bar[st]));
+                    mbar_arrive(smem_u32(&stg_empty[sst]));
                 }
+                st += tr_groups;
+                while (st >= g.stages) { st -= g.stages; ph ^= 1u; }
+                sst += tr_groups;
+                while (sst >= g.stg_depth) { sst -= g.stg_depth; sph ^= 1u; }
+            }
         }
     } else {
         // ---------------- read-out: tensor memory -> bias, residual, activation -> global memory ----------------
