@@ -1650,10 +1650,8 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const int b_rows = g.b_rows_cta;
     const int RS = g.R * g.S;
     const int blocks_per_tile = tapm ? kt_n * g.n_atoms / RS : 0;     // 32-channel blocks
-    // The transposer warps work as two groups on alternate reduction tiles when both rings are at least two deep: while
-    // one group waits for its buffers and hands its stage over, the other copies.
-    const int tr_groups = (g.stages >= 2 && g.stg_depth >= 2) ? 2 : 1;
-    const int tr_warps = kPsTransposeWarps / tr_groups;               // warps per box
+    constexpr int tr_groups = 1;                                      // all transposer warps work on the same box
+    constexpr int tr_warps = kPsTransposeWarps / tr_groups;
 
     if (threadIdx.x == 32) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
