@@ -51,7 +51,8 @@ typedef enum {
     TT_ERR_CUDA = 6,              /* a CUDA runtime or driver call failed (or no device) */
     TT_ERR_TIMEOUT = 7,           /* a bounded wait inside a kernel expired; the context stays usable */
     TT_ERR_OOM = 8,               /* workspace allocation failed */
-    TT_ERR_NOT_IMPLEMENTED = 9
+    TT_ERR_NOT_IMPLEMENTED = 9,
+    TT_SKIPPED = 10               /* evaluator only: the pair was left out by pool sub-sampling (neither valid nor invalid) */
 } tt_status;
 
 /* Operators (each is one fused kernel; bias and activation are applied as soon as an
@@ -207,7 +208,14 @@ typedef struct tt_tune_opts {
     int32_t strict_class;    /* 1: the record's origin kernel class (op, bias, activation, residual) must equal the
                                 workload's (the paper's rule); 0: same family suffices */
     int32_t include_default; /* 1 (default): column 0 of the table is the workload's default ("untuned") record */
-    int32_t reserved[5];
+    int32_t subsample_percent; /* 0 or 100: every pool record is evaluated.  1..99: per workload, a seeded subset of that
+                                share of the pool (tt_pool_subsample; at least one record) is evaluated first, and the
+                                rest only if the subset's best time is not below the default record's by more than
+                                subsample_gain_percent.  Records left out are marked TT_SKIPPED (time -1).  The paper
+                                notes that a larger pool lengthens the search (Section 5.5); this bounds it. */
+    int32_t subsample_gain_percent; /* the gain over the default record that ends a workload's search early */
+    uint32_t subsample_seed;
+    int32_t reserved[2];
 } tt_tune_opts;
 
 /* Result arrays are allocated by the caller.  n_cols = n_pool + 1; column 0 is the default record, column j+1 is
@@ -219,6 +227,7 @@ typedef struct tt_tune_result {
     int32_t* status;        /* [n_wl*n_cols] tt_status of apply/timing for the pair */
     double search_seconds;  /* wall time of the call: apply + warm-up + timing + selection */
     int32_t pairs_timed, pairs_invalid;
+    int32_t pairs_skipped;  /* pairs left out by pool sub-sampling */
 } tt_tune_result;
 
 typedef struct tt_workload tt_workload;
@@ -336,6 +345,11 @@ tt_status tt_grid_tune(tt_workload* w, const tt_tensors* t, void* cuda_stream, c
  * unknown field or carries another record version: TT_ERR_INVALID_ARG.  A missing file: TT_ERR_INVALID_ARG. */
 tt_status tt_pool_save(const char* path, const tt_schedule_record* records, const float* us, size_t n);
 tt_status tt_pool_load(const char* path, tt_schedule_record* out, float* us, size_t cap, size_t* n_out);
+
+/* Pure host: the first `count` entries of a seeded shuffle of 0 .. n_pool-1 (Fisher-Yates from the front, position i
+ * swapped with i + r mod (n_pool - i), r the next output of the splitmix64 generator started at `seed`).  The subset
+ * of the pool that sub-sampling evaluates first; count > n_pool: TT_ERR_INVALID_ARG. */
+tt_status tt_pool_subsample(size_t n_pool, size_t count, uint64_t seed, int32_t* idx_out);
 
 /* Refining a transferred record (Section 7 names it as the next step: vary the parameters of schedules that were
  * transfer-tuned from another model).  The neighbourhood of a record: every field its family uses is moved one rung

@@ -324,3 +324,44 @@ def refine(start, neighbours, time_us, max_rounds: int, min_gain: float = 0.0):
             break
         cur, cur_us = pick, pick_us
     return cur, cur_us, start_us, timed
+
+
+# ---- pool sub-sampling (the paper notes that a larger pool lengthens the search, Section 5.5) ----
+_M64 = (1 << 64) - 1
+
+
+def splitmix64(state: int):
+    """One step of the splitmix64 generator (Steele, Lea, Flood 2014; Vigna's public-domain reference): the state
+    advances by the golden-ratio increment, the output is the state after two xor-shift-multiply rounds and a final
+    xor-shift.  Returns (new state, output)."""
+    state = (state + 0x9E3779B97F4A7C15) & _M64
+    z = state
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _M64
+    return state, z ^ (z >> 31)
+
+
+def pool_subsample(n_pool: int, count: int, seed: int):
+    """The first `count` entries of a Fisher-Yates shuffle of range(n_pool) taken from the front: position i is swapped
+    with position i + r mod (n_pool - i), r the next splitmix64 output of the generator started at `seed`."""
+    if count > n_pool:
+        raise ValueError("more records asked for than the pool holds")
+    perm = list(range(n_pool))
+    state = seed & _M64
+    for i in range(count):
+        state, r = splitmix64(state)
+        j = i + r % (n_pool - i)
+        perm[i], perm[j] = perm[j], perm[i]
+    return perm[:count]
+
+
+def evaluate_subsampled(times_row, first, gain_percent: float):
+    """Which columns of one kernel's row get evaluated under sub-sampling, given what every column WOULD measure:
+    column 0 (the default record) and the subset `first` (pool indices) always; the rest only if the subset's best
+    valid time is not below the default's by more than gain_percent.  Returns the set of evaluated columns."""
+    cols = {0} | {f + 1 for f in first}
+    valid = [times_row[f + 1] for f in first if times_row[f + 1] >= 0]
+    default = times_row[0]
+    if valid and default >= 0 and min(valid) <= default * (1.0 - gain_percent / 100.0):
+        return cols
+    return set(range(len(times_row)))

@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 
 # enums
 TT_OK, TT_ERR_INVALID_ARG, TT_ERR_INVALID_SCHEDULE, TT_ERR_CLASS_MISMATCH, TT_ERR_RESOURCE, \
-    TT_ERR_NOT_APPLIED, TT_ERR_CUDA, TT_ERR_TIMEOUT, TT_ERR_OOM, TT_ERR_NOT_IMPLEMENTED = range(10)
+    TT_ERR_NOT_APPLIED, TT_ERR_CUDA, TT_ERR_TIMEOUT, TT_ERR_OOM, TT_ERR_NOT_IMPLEMENTED, TT_SKIPPED = range(11)
 TT_OP_CONV2D, TT_OP_DWCONV2D, TT_OP_DENSE, TT_OP_BATCH_MATMUL, TT_OP_SOFTMAX = range(5)
 TT_ACT_NONE, TT_ACT_RELU, TT_ACT_RELU6, TT_ACT_GELU_ERF = range(4)
 TT_FAMILY_GEMM_TC, TT_FAMILY_DW_SIMT, TT_FAMILY_ROW_SIMT = range(3)
@@ -87,13 +87,13 @@ class tt_timing(C.Structure):
 
 class tt_tune_opts(C.Structure):
     _fields_ = [("timing", tt_timing_opts), ("mode", i32), ("strict_class", i32), ("include_default", i32),
-                ("reserved", i32 * 5)]
+                ("subsample_percent", i32), ("subsample_gain_percent", i32), ("subsample_seed", u32), ("reserved", i32 * 2)]
 
 
 class tt_tune_result(C.Structure):
     _fields_ = [("chosen", C.POINTER(i32)), ("best_us", C.POINTER(f32)), ("times_us", C.POINTER(f32)),
                 ("status", C.POINTER(i32)), ("search_seconds", C.c_double), ("pairs_timed", i32),
-                ("pairs_invalid", i32)]
+                ("pairs_invalid", i32), ("pairs_skipped", i32)]
 
 
 EXPORTS = {
@@ -137,6 +137,7 @@ EXPORTS = {
     "tt_refine": (i32, [C.c_void_p, C.POINTER(tt_tensors), C.c_void_p, C.POINTER(tt_timing_opts),
                         C.POINTER(tt_schedule_record), i32, f32, C.POINTER(tt_schedule_record), C.POINTER(f32),
                         C.POINTER(f32), C.POINTER(i32)]),
+    "tt_pool_subsample": (i32, [C.c_size_t, C.c_size_t, C.c_uint64, C.POINTER(i32)]),
     "tt_pool_save": (i32, [C.c_char_p, C.POINTER(tt_schedule_record), C.POINTER(f32), C.c_size_t]),
     "tt_pool_load": (i32, [C.c_char_p, C.POINTER(tt_schedule_record), C.POINTER(f32), C.c_size_t, C.POINTER(C.c_size_t)]),
     "tt_dense_static_scratch": (i32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, i32, i32, i32, i32,
@@ -248,6 +249,13 @@ def rank_pools(class_share, class_kernels):
     od = (i32 * max(n_m, 1))()
     _check(lib().tt_rank_pools(sh, n_c, ck, n_m, sc, od), "tt_rank_pools")
     return list(sc)[:n_m], list(od)[:n_m]
+
+
+def pool_subsample(n_pool, count, seed):
+    """tt_pool_subsample: the first `count` indices of the seeded shuffle of range(n_pool)."""
+    out = (i32 * max(count, 1))()
+    _check(lib().tt_pool_subsample(n_pool, count, seed, out), "tt_pool_subsample")
+    return list(out)[:count]
 
 
 def pool_save(path, records, us=None):
@@ -482,4 +490,5 @@ def transfer_tune(workloads, tensor_sets, pool, opts: tt_tune_opts | None = None
         "times_us": [[times[i * n_cols + j] for j in range(n_cols)] for i in range(n_wl)],
         "status": [[status[i * n_cols + j] for j in range(n_cols)] for i in range(n_wl)],
         "search_seconds": res.search_seconds, "pairs_timed": res.pairs_timed, "pairs_invalid": res.pairs_invalid,
+        "pairs_skipped": res.pairs_skipped,
     }

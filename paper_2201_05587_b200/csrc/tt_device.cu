@@ -569,9 +569,24 @@ static tt_status transfer_tune_impl(tt_workload* const* wls, const tt_tensors* t
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const auto t_begin = std::chrono::steady_clock::now();
     const size_t n_cols = n_pool + 1;
-    int timed = 0, invalid = 0;
+    int timed = 0, invalid = 0, skipped = 0;
     std::vector<tt_schedule_record> cols(n_cols);
     size_t first_set = 0;
+    // pool sub-sampling: the order in which a workload's columns are evaluated -- default first, then the seeded
+    // subset, then (only if the subset gained too little over the default) the rest of the pool
+    const bool sub = o.subsample_percent > 0 && o.subsample_percent < 100 && n_pool > 1;
+    size_t n_first = n_pool;
+    std::vector<int32_t> order(n_pool);
+    for (size_t j = 0; j < n_pool; ++j) order[j] = (int32_t)j;
+    if (sub) {
+        n_first = std::max<size_t>(1, (n_pool * (size_t)o.subsample_percent + 99) / 100);
+        std::vector<int32_t> firsts(n_first);
+        if (tt_pool_subsample(n_pool, n_first, o.subsample_seed, firsts.data()) != TT_OK) return TT_ERR_INVALID_ARG;
+        std::vector<char> taken(n_pool, 0);
+        size_t k = 0;
+        for (int32_t f : firsts) { order[k++] = f; taken[(size_t)f] = 1; }
+        for (size_t j = 0; j < n_pool; ++j) if (!taken[j]) order[k++] = (int32_t)j;
+    }
     for (size_t i = 0; i < n_wl; ++i) {
         tt_workload* w = wls[i];
         if (!w) return TT_ERR_INVALID_ARG;
@@ -580,17 +595,29 @@ static tt_status transfer_tune_impl(tt_workload* const* wls, const tt_tensors* t
         first_set += n_sets;
         tt_default_schedule(w, &cols[0]);
         for (size_t j = 0; j < n_pool; ++j) cols[j + 1] = pool[j];
-        for (size_t j = 0; j < n_cols; ++j) {
+        bool stop_early = false;
+        float best_first = -1.f;                         // fastest time among the subset's records
+        for (size_t step = 0; step < n_cols; ++step) {
+            const size_t j = step == 0 ? 0 : (size_t)order[step - 1] + 1;
             float& cell = out->times_us[i * n_cols + j];
             int32_t& cst = out->status[i * n_cols + j];
             cell = -1.f;
+            if (sub && step == n_first + 1) {
+                // the subset is done: go on only if it did not beat the default record by the asked-for margin
+                const float def = out->times_us[i * n_cols];
+                stop_early = best_first >= 0.f && def >= 0.f && best_first <= def * (1.f - 0.01f * (float)o.subsample_gain_percent);
+            }
+            if (stop_early) { cst = TT_SKIPPED; ++skipped; continue; }
             if (j == 0 && !o.include_default) { cst = TT_ERR_INVALID_SCHEDULE; continue; }
             // the default record is the workload's own: never subject to the class rule
             tt_status s = apply_impl(w, &cols[j], j == 0 ? TT_MODE_LEGALISE : o.mode, j == 0 ? 0 : o.strict_class, nullptr);
             if (s == TT_OK) {
                 tt_timing tm{};
                 s = time_applied(w, sets, n_sets, st, &o.timing, &tm);
-                if (s == TT_OK) { cell = tm.median_us; ++timed; }
+                if (s == TT_OK) {
+                    cell = tm.median_us; ++timed;
+                    if (step >= 1 && step <= n_first && (best_first < 0.f || cell < best_first)) best_first = cell;
+                }
             }
             cst = s;
             if (s != TT_OK) {
@@ -606,7 +633,7 @@ static tt_status transfer_tune_impl(tt_workload* const* wls, const tt_tensors* t
             if (s != TT_OK) return s;
         }
     }
-    out->pairs_timed = timed; out->pairs_invalid = invalid;
+    out->pairs_timed = timed; out->pairs_invalid = invalid; out->pairs_skipped = skipped;
     out->search_seconds = std::chrono::duration<double>(std::chrono::steady_clock::now() - t_begin).count();
     return TT_OK;
 }

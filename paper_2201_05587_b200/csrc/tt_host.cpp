@@ -6,6 +6,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <string>
+#include <vector>
 #include <new>
 #include "tt_internal.h"
 
@@ -762,6 +763,7 @@ const char* tt_status_string(tt_status s) {
         case TT_ERR_TIMEOUT: return "device wait timed out";
         case TT_ERR_OOM: return "out of device memory";
         case TT_ERR_NOT_IMPLEMENTED: return "not implemented";
+        case TT_SKIPPED: return "pair left out by pool sub-sampling";
     }
     return "unknown status";
 }
@@ -1095,6 +1097,25 @@ tt_status tt_pool_load(const char* path, tt_schedule_record* out, float* us, siz
     *n_out = n;
     if (rc != TT_OK) return rc;
     return (cap && n > cap) ? TT_ERR_RESOURCE : TT_OK;
+}
+
+tt_status tt_pool_subsample(size_t n_pool, size_t count, uint64_t seed, int32_t* idx_out) {
+    if (count > n_pool || (count && !idx_out) || n_pool > 0x7fffffffu) return TT_ERR_INVALID_ARG;
+    std::vector<int32_t> perm(n_pool);
+    for (size_t i = 0; i < n_pool; ++i) perm[i] = (int32_t)i;
+    uint64_t state = seed;
+    for (size_t i = 0; i < count; ++i) {
+        // splitmix64: advance the state by the golden-ratio increment, then mix
+        state += 0x9E3779B97F4A7C15ull;
+        uint64_t z = state;
+        z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+        z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+        z ^= z >> 31;
+        const size_t j = i + (size_t)(z % (uint64_t)(n_pool - i));
+        std::swap(perm[i], perm[j]);
+        idx_out[i] = perm[i];
+    }
+    return TT_OK;
 }
 
 tt_status tt_split_check(int64_t extent, const int64_t* factors, size_t n, int32_t reformulate, int32_t* valid) {

@@ -508,3 +508,10 @@ def test_bench_counts_algorithmic_work_like_the_library():
             v = sp.workload().gemm_view()
             f, b = bench.algorithmic_work(sp)
             assert f == pytest.approx(v.flops) and b == pytest.approx(v.bytes), sp.name
+
+
+def test_pool_subsample_matches_the_oracle():
+    for n, c, seed in ((1, 1, 0), (10, 4, 7), (56, 14, 2024), (111, 111, 5), (50, 0, 9)):
+        assert B.pool_subsample(n, c, seed) == orc.pool_subsample(n, c, seed)
+    out = (ctypes.c_int32 * 4)()
+    assert B.lib().tt_pool_subsample(3, 4, 0, out) == B.TT_ERR_INVALID_ARG

@@ -431,3 +431,34 @@ def test_refine_round_limit_gain_threshold_invalid_and_ties():
     assert orc.refine(0, star.__getitem__, {0: 5.0, 1: -1.0, 2: 4.0, 3: 4.0}.__getitem__, 3)[0] == 2
     with pytest.raises(ValueError):
         orc.refine(0, star.__getitem__, {0: -1.0, 1: 1.0, 2: 1.0, 3: 1.0}.__getitem__, 3)
+
+
+def test_splitmix64_published_vector_and_subsample_is_a_shuffle_prefix():
+    """The generator against the test vector published with its reference implementation (seed 1234567), and the
+    subset against what a shuffle must satisfy: distinct indices in range, a prefix property (asking for more records
+    extends the list, never reorders it), the full count is a permutation, another seed gives another order."""
+    state, outs = 1234567, []
+    for _ in range(5):
+        state, v = orc.splitmix64(state)
+        outs.append(v)
+    assert outs == [6457827717110365317, 3203168211198807973, 9817491932198370423, 4593380528125082431, 16408922859458223821]
+    for n in (1, 2, 7, 50, 111):
+        full = orc.pool_subsample(n, n, 42)
+        assert sorted(full) == list(range(n))
+        for c in (0, 1, n // 3, n):
+            assert orc.pool_subsample(n, c, 42) == full[:c]
+    assert orc.pool_subsample(50, 50, 42) != orc.pool_subsample(50, 50, 43)
+    # every index leads the list for some seed: no position is favoured out of existence
+    assert {orc.pool_subsample(5, 1, s)[0] for s in range(200)} == set(range(5))
+    with pytest.raises(ValueError):
+        orc.pool_subsample(3, 4, 0)
+
+
+def test_subsampled_evaluation_rule():
+    row = [10.0, 12.0, 7.0, -1.0, 9.5, 4.0]          # default, then five pool records (one invalid)
+    # the subset {1, 2} holds a record 30 % faster than the default: with a 20 % bar the search stops there
+    assert orc.evaluate_subsampled(row, [1, 2], 20.0) == {0, 2, 3}
+    # with a 40 % bar it does not, and every record is evaluated
+    assert orc.evaluate_subsampled(row, [1, 2], 40.0) == set(range(6))
+    # a subset without a valid record never ends the search
+    assert orc.evaluate_subsampled(row, [2], 0.0) == set(range(6))
