@@ -832,3 +832,34 @@ def test_persistent_tap_major_convolution_walks_many_tiles(spec):
     probe.close()
     for y in outs[1:]:
         assert util.rel_l2(y, outs[0]) <= INVARIANCE_TOL
+
+
+def test_subsampled_evaluator_skips_what_the_rule_says_and_keeps_a_valid_choice():
+    """Pool sub-sampling: the seeded subset is evaluated first; with a bar nothing can clear (100 % gain) every record is
+    still evaluated, with a bar everything clears (a negative gain) only the subset is, the rest is marked TT_SKIPPED,
+    and the chosen record is the argmin over what was evaluated."""
+    spec = W._conv(32, 14, 64, 3, 1, 1)
+    a = W.make_inputs(spec, 44)
+    wl = spec.workload()
+    t, tt = W.device_tensors(spec, a)
+    pool = [tc(tile_n=tn, tile_k=tk, stages=st) for tn in (32, 64, 128) for tk in (16, 32) for st in (2, 3)]   # 12 records
+    o = B.tt_tune_opts()
+    o.include_default = 1
+    o.timing.warmup_batches, o.timing.batches, o.timing.min_batch_us, o.timing.use_graph = 1, 3, 50, 1
+    o.subsample_percent, o.subsample_seed = 25, 11
+    first = B.pool_subsample(len(pool), 3, 11)
+    assert first == orc.pool_subsample(len(pool), 3, 11)
+    o.subsample_gain_percent = 100                       # unreachable: the whole pool gets evaluated
+    res = B.transfer_tune([wl], [tt], pool, o)
+    assert res["pairs_skipped"] == 0 and res["pairs_timed"] == 13
+    o.subsample_gain_percent = -1000                     # any valid subset record ends the search
+    res = B.transfer_tune([wl], [tt], pool, o)
+    st = res["status"][0]
+    evaluated = {0} | {f + 1 for f in first}
+    assert {j for j, s in enumerate(st) if s == B.TT_OK} == evaluated
+    assert all(st[j] == B.TT_SKIPPED and res["times_us"][0][j] == -1.0 for j in range(13) if j not in evaluated)
+    assert res["pairs_skipped"] == 9 and res["pairs_timed"] == 4
+    assert res["chosen"] == orc.select(res["times_us"][0], 1, 13) and res["chosen"][0] in evaluated
+    wl.run(tt)                                           # the chosen record is left applied
+    assert util.rel_l2(t["y"].cpu().numpy(), util.oracle_ref(spec, a)) <= util.TOL_TF32
+    wl.close()
