@@ -417,11 +417,13 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     // (each sends the bands of its partial tile to the CTAs that finish them); beyond 8 the partial tiles go through
     // a global workspace and the split that arrives last adds them up
     const int cluster = (sk >= 2 && sk <= 8) ? sk : 0;
-    const long long min_pipe = (long long)kGatherWarps * 32 * 36 * 4;
+    // the read-out stages through the pipeline buffers (idle by then): a 32 x 36 float block per warp, or, for the
+    // cluster reduction, this split's whole partial tile in the layout of the reduction area
+    const long long min_pipe = std::max<long long>((long long)kGatherWarps * 32 * 36 * 4, cluster ? 4LL * kHwTileM * (tn + 4) : 0);
     // cluster reduction area, apart from the pipeline buffers (peers write into it while this CTA may still be in its
-    // main loop): per source split, this CTA's band of the tile -- rows x (tile_n + 4) or columns x 132 floats
-    const long long red_bytes = cluster ? (4 * std::max<long long>((long long)sk * ((kHwTileM + sk - 1) / sk) * (tn + 4),
-                                                                    (long long)sk * ((tn + sk - 1) / sk) * (kHwTileM + 4)) + 127) / 128 * 128 : 0;
+    // main loop): per OTHER split, this CTA's band of the tile -- rows x (tile_n + 4) or columns x 128 floats
+    const long long red_bytes = cluster ? (4 * std::max<long long>((long long)(sk - 1) * ((kHwTileM + sk - 1) / sk) * (tn + 4),
+                                                                    (long long)(sk - 1) * ((tn + sk - 1) / sk) * kHwTileM) + 127) / 128 * 128 : 0;
     const bool conv = w->op == TT_OP_CONV2D;
     const long long ktab = conv ? (((long long)per_split * tk * 4 + 127) / 128) * 128 : 0;
     int sl_tiles = 0, sl_nbuf = 0, sl_wp = 0, sl_gap = 0, sl_chpitch = 0, sl_in_rows = 0, sl_rstep = 1;

@@ -299,11 +299,25 @@ __device__ __forceinline__ float4 ld_shared_v4f(uint32_t addr) {
 }
 // Split-K over a cluster.  The output tile is cut into one band per CTA, along the direction in which the output is
 // NOT contiguous (bands of rows when outputs are contiguous along columns, bands of columns otherwise).  Every CTA
-// sends each band of its partial tile to the CTA that owns the band (remote shared-memory stores into a reduction
-// area that is not part of the pipeline buffers, so a fast peer cannot disturb a slower one's main loop); after one
-// cluster barrier every CTA adds up what it received, in split order, locally.  Area layout, per source split:
-//   bands of rows:    [row in band][col], pitch tile_n + 4 floats;   bands of columns: [col in band][row], pitch 132.
-constexpr int kRedColPitch = kHwTileM + 4;
+// first writes its partial tile into its own shared memory (the pipeline buffers, idle by then) in the layout of the
+// reduction area, so that a band is one contiguous run of bytes; one thread per peer then sends that peer's band with
+// a single bulk copy (cp.async.bulk, shared::cta -> shared::cluster) into the peer's reduction area, which is not part
+// of the pipeline buffers (a fast peer cannot disturb a slower one's main loop).  The copy reports its bytes to a
+// barrier of the receiving CTA, which expects the bands of all other splits: a CTA starts adding as soon as ITS bands
+// have landed, in split order, its own band read from its own staging copy.  Area layout, per source split (the
+// CTA's own split has no slot):
+//   bands of rows:    [row in band][col], pitch tile_n + 4 floats;   bands of columns: [col in band][row], pitch 128.
+constexpr int kRedColPitch = kHwTileM;
+// One band of this CTA's staged partial tile -> the same band's slot in a peer's reduction area; the bytes are counted
+// on the peer's barrier (both destination addresses are shared::cluster addresses of the same peer).
+__device__ __forceinline__ void bulk_copy_to_peer(uint32_t dst_caddr, uint32_t src_saddr, uint32_t bytes, uint32_t bar_caddr) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_caddr), "r"(src_saddr), "r"(bytes), "r"(bar_caddr) : "memory");
+}
+// Wait until every bulk copy this thread issued has been written at its destination.
+__device__ __forceinline__ void bulk_copies_done() {
+    asm volatile("cp.async.bulk.commit_group;\n\tcp.async.bulk.wait_group 0;" ::: "memory");
+}
 
 // All gather threads meet and learn whether every one of them is still healthy (named barrier 1).
 __device__ __forceinline__ bool gather_vote(bool ok) {
@@ -694,6 +708,44 @@ __device__ __forceinline__ void epilogue_block(float (&v)[32], const EpiArgs& e,
 // Two builds: MIN_CTAS = 1 (all registers), and MIN_CTAS = 2 (registers capped so that two CTAs share an SM when a
 // record's shared memory and tensor memory allow it: one CTA's set-up and read-out then overlap the other's main loop).
 // ------------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait on a barrier that CTAs of the cluster arrive on (acquire at cluster scope).
+__device__ __noinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
+                                               unsigned where, unsigned long long limit_ns) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    unsigned spins = 0;
+    for (;;) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((++spins & 31u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > limit_ns) {
+                *abort_flag = 1;
+                atomicCAS(status, 0u, (unsigned)TT_ERR_TIMEOUT | (where << 8));
+                return false;
+            }
+        }
+    }
+}
+
+// Split-K over a cluster: extent (rows or columns) and bytes of the band of the output tile that split `owner` finishes.
+__device__ __forceinline__ int red_band_extent(const GemmArgs& g, int owner) {
+    const int whole = g.y_ns == 1 ? kHwTileM : g.tile_n;
+    const int per = (whole + g.split_k - 1) / g.split_k;
+    return max(0, min(whole, (owner + 1) * per) - owner * per);
+}
+__device__ __forceinline__ uint32_t red_band_bytes(const GemmArgs& g, int owner) {
+    return (uint32_t)red_band_extent(g, owner) * 4u * (uint32_t)(g.y_ns == 1 ? g.tile_n + 4 : kRedColPitch);
+}
+
 template <int MIN_CTAS>
 __global__ void __launch_bounds__(kGemmThreads, MIN_CTAS)
 tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -706,6 +758,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __shared__ uint64_t slab_empty[2];    // all gather warps are done with a slab buffer
     __shared__ uint64_t pm_full[2];       // tap-major convolution: a pixel-major slab buffer has been written
     __shared__ uint64_t pm_empty[2];      // ... and every multiply-accumulate that reads it has completed
+    __shared__ uint64_t red_bar;          // split-K over a cluster: the other splits' bands of this CTA's output have landed
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int last_split_flag;
@@ -717,9 +770,6 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     volatile int* abortp = &abort_flag;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel of the stream may begin its set-up
-    // A CTA's shared memory may be written by a peer only once the CTA runs: every thread announces itself here and
-    // checks, much later and just before the first remote store could happen, that all peers have done the same.
-    if (g.cluster) cluster_arrive();
 
     // tile coordinates
     int tm, tn;
@@ -777,6 +827,11 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             mbar_init(smem_u32(&pm_full[b]), (uint32_t)kGatherWarps);
             mbar_init(smem_u32(&pm_empty[b]), 1u);
         }
+        if (g.cluster) {
+            // the bands this CTA finishes arrive from the other splits: rows x (tile_n + 4) or columns x 128 floats each
+            mbar_init(smem_u32(&red_bar), 1u);
+            mbar_expect_tx(smem_u32(&red_bar), (uint32_t)(g.split_k - 1) * red_band_bytes(g, split));
+        }
         abort_flag = 0;
         last_split_flag = 0;
         fence_mbar_init();
@@ -790,6 +845,10 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *(volatile uint32_t*)&tmem_slot;
+    // A CTA's reduction area and its barrier may be used by a peer only once they exist: every thread announces
+    // itself here (the barrier above is initialised) and checks, just before the first copy to a peer could be issued,
+    // that all peers have done the same.
+    if (g.cluster) cluster_arrive();
     // Programmatic dependent launch: everything above (barriers, tensor memory) touched no global memory and may
     // run while the previous kernel of the stream is still draining; from here on its results are needed.  The
     // kernel that follows this one was allowed to start its own set-up at this kernel's entry.  (Without the launch
@@ -1196,6 +1255,35 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 while (st >= g.stages) { st -= g.stages; ph ^= 1u; }
             }
         }
+        // split-K over a cluster: everything the reduction needs that does not depend on the accumulator is worked out
+        // here, while the main loop is still running (divisions, 64-bit products, first reads of kernel parameters)
+        struct {
+            int sk, whole, per; uint32_t line, slot, red; bool along_cols, gelu, clamp, vec_ok; int bias_mode;
+            float lo, hi; float* ybase; const float* rbase; long long y_ms, y_ns;
+        } cr;
+        if (g.cluster) {
+            cr.sk = g.split_k;
+            cr.along_cols = g.y_ns == 1;                                 // bands of rows
+            cr.whole = cr.along_cols ? kHwTileM : g.tile_n;
+            cr.per = (cr.whole + cr.sk - 1) / cr.sk;                     // lines (rows or columns) per band
+            cr.line = 4u * (uint32_t)(cr.along_cols ? g.tile_n + 4 : kRedColPitch);   // bytes per line
+            cr.slot = (uint32_t)cr.per * cr.line;                        // bytes between the bands of two consecutive splits
+            cr.red = tiles_base + g.red_off;
+            cr.ybase = g.y + (long long)bz * g.y_bs;
+            cr.rbase = g.residual ? g.residual + (long long)bz * g.y_bs : nullptr;
+            cr.lo = g.act == TT_ACT_NONE || g.act == TT_ACT_GELU_ERF ? -INFINITY : 0.f;
+            cr.hi = g.act == TT_ACT_RELU6 ? 6.f : INFINITY;
+            cr.gelu = g.act == TT_ACT_GELU_ERF; cr.clamp = g.act == TT_ACT_RELU || g.act == TT_ACT_RELU6;
+            cr.bias_mode = g.bias_mode; cr.y_ms = g.y_ms; cr.y_ns = g.y_ns;
+            const long long lead = cr.along_cols ? g.y_ms : g.y_ns;      // stride of the other output axis
+            cr.vec_ok = (lead & 3) == 0 && (g.y_bs & 3) == 0 && (reinterpret_cast<uintptr_t>(cr.ybase) & 15u) == 0 &&
+                        (cr.rbase == nullptr || (reinterpret_cast<uintptr_t>(cr.rbase) & 15u) == 0);
+            if constexpr (MIN_CTAS == 1) {               // (kept in registers; the register-capped build works them out again)
+                int pin = cr.per;
+                asm volatile("" : "+r"(pin), "+r"(cr.slot), "+r"(cr.red), "+l"(cr.ybase), "+l"(cr.rbase), "+l"(cr.y_ms), "+l"(cr.y_ns));
+                cr.per = pin;
+            }
+        }
         // epilogue: warp w owns tensor-memory lanes 32*(w % 4) .. +31; the two warps of a lane quadrant take
         // alternate 32-column blocks
         const bool have_acc = mbar_wait(smem_u32(&accum_bar), 0u, abortp, g.status, 4u, g.wait_ns);
@@ -1208,7 +1296,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             "bar.red.and.pred p, 1, %2, q;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(all_acc) : "r"((uint32_t)have_acc), "n"(kGatherThreads) : "memory");
-        if (g.cluster) cluster_wait();                   // every peer is running: its reduction area may be written
+        if (g.cluster) cluster_wait();                   // every peer is set up: its reduction area and barrier may be used
         if (all_acc) {
             tc_fence_after();
             const int half = gw >> 2;
@@ -1221,7 +1309,10 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             const long long per_split = (long long)g.batch * g.M * (long long)g.N;
             float* pcol = g.partial + (long long)bz * g.M * (long long)g.N + m;
             if (g.cluster) {
-                // split-K over a cluster: send each band of this split's partial tile to the CTA that finishes it
+                // split-K over a cluster, step 1: this split's partial tile goes to the pipeline buffers (idle: every
+                // multiply-accumulate has completed) in the layout of the reduction area, a band being one run of bytes
+                const int row = quad * 32 + lane;
+                const uint32_t row_dst = tiles_base + 4u * (uint32_t)(g.y_ns == 1 ? row * (g.tile_n + 4) : row);
 #pragma unroll 1
                 for (int c0 = half * 32; c0 < g.tile_n; c0 += 64) {
                     uint32_t r[32];
@@ -1235,33 +1326,23 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 #pragma unroll
                         for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(t2[i]));
                     }
-                    const int row = quad * 32 + lane;
-                    const uint32_t red = tiles_base + g.red_off;
                     if (g.y_ns == 1) {
-                        // bands of rows: this lane's row belongs to one CTA
-                        const int per = (kHwTileM + g.split_k - 1) / g.split_k;
-                        const int owner = row / per, rl = row - owner * per;
-                        const uint32_t dst = map_to_peer(red, (uint32_t)owner) + 4u * (uint32_t)((split * per + rl) * (g.tile_n + 4) + c0);
+                        // bands of rows: [row][col], pitch tile_n + 4
+                        const uint32_t dst = row_dst + 4u * (uint32_t)c0;
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
                             if (c0 + j < g.tile_n)           // tile_n is a multiple of 16: groups of four are whole
-                                st_peer_v4(dst + 4u * (uint32_t)j, r[j], r[j + 1], r[j + 2], r[j + 3]);
+                                st_shared_v4(dst + 4u * (uint32_t)j, __uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                             __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
                     } else {
-                        // bands of columns: column c0 + j belongs to CTA (c0 + j) / per; lanes (rows) are contiguous
-                        const int per = (g.tile_n + g.split_k - 1) / g.split_k;
-                        int owner = c0 / per, cl = c0 - owner * per;
-                        uint32_t dst = map_to_peer(red, (uint32_t)owner) + 4u * (uint32_t)((split * per + cl) * kRedColPitch + row);
+                        // bands of columns: [col][row], pitch 128 -- the lanes of a warp write 128 contiguous bytes
+                        uint32_t dst = row_dst + 4u * (uint32_t)(c0 * kRedColPitch);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (c0 + j < g.tile_n) st_peer_u32(dst, r[j]);
-                            dst += 4u * (uint32_t)kRedColPitch;
-                            if (++cl == per) {               // next column starts the next CTA's band
-                                cl = 0; ++owner;
-                                dst = map_to_peer(red, (uint32_t)min(owner, g.split_k - 1)) + 4u * (uint32_t)(split * per * kRedColPitch + row);
-                            }
-                        }
+                        for (int j = 0; j < 32; ++j, dst += 4u * (uint32_t)kRedColPitch)
+                            if (c0 + j < g.tile_n) st_shared_u32(dst, r[j]);
                     }
                 }
+                fence_proxy_async_shared();              // generic-proxy stores -> visible to the bulk copies below
             } else if (split_mode) {
                 // 1. park this split's partial tile in the workspace
                 float* pmine = pcol + (long long)split * per_split;
@@ -1365,7 +1446,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                         if (e.gelu) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
-                        } else {
+                        } else if (g.act != TT_ACT_NONE) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] = fminf(fmaxf(v[j], e.lo), e.hi);
                         }
@@ -1378,76 +1459,105 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             }
         }
-    }
-    if (g.cluster) {
-        // ---------------- split-K over the cluster: add up the bands the peers sent ----------------
-        // Every thread of every CTA of the cluster takes part in the barrier, also after a tripped wait.  After it
-        // nobody writes to or reads from another CTA's shared memory any more, so no second barrier is needed.
-        cluster_sync_all();                              // all bands have arrived
-        if (warp >= 2) {
-            const int gw = warp - 2;
-            const int sk = g.split_k;
-            const uint32_t red = tiles_base + g.red_off;
-            float* ybase = g.y + (long long)bz * g.y_bs;
-            const float* rbase = g.residual ? g.residual + (long long)bz * g.y_bs : nullptr;
-            const float lo = g.act == TT_ACT_NONE || g.act == TT_ACT_GELU_ERF ? -INFINITY : 0.f;
-            const float hi = g.act == TT_ACT_RELU6 ? 6.f : INFINITY;
-            const bool gelu = g.act == TT_ACT_GELU_ERF;
-            const bool along_cols = g.y_ns == 1;
-            const long long lead = along_cols ? g.y_ms : g.y_ns;       // stride of the other output axis
-            const bool vec_ok = (lead & 3) == 0 && (g.y_bs & 3) == 0 && (reinterpret_cast<uintptr_t>(ybase) & 15u) == 0 &&
-                                (rbase == nullptr || (reinterpret_cast<uintptr_t>(rbase) & 15u) == 0);
-            // four outputs that are neighbours in memory, first one (mm, nn): the partial sums of all splits (16 bytes
-            // each, `stride` bytes apart) are added in split order, then bias, residual, activation, one 16-byte store
-            auto finish4 = [&](uint32_t addr, uint32_t stride, int mm, int nn, int valid) {
-                float4 p[8];
+        if (g.cluster) {
+            // step 2: once every read-out warp has staged its part, one thread per peer sends that peer's band
+            asm volatile("bar.sync 1, %0;" ::"n"(kGatherThreads) : "memory");
+            if (all_acc && lane == 0 && gw < cr.sk && gw != split) {
+                const uint32_t bytes = (uint32_t)max(0, min(cr.whole, (gw + 1) * cr.per) - gw * cr.per) * cr.line;
+                if (bytes != 0u) {
+                    // (a CTA keeps no slot for its own split: the splits after it move down by one)
+                    bulk_copy_to_peer(map_to_peer(cr.red + (uint32_t)(split < gw ? split : split - 1) * cr.slot, (uint32_t)gw),
+                                      tiles_base + (uint32_t)gw * cr.slot, bytes, map_to_peer(smem_u32(&red_bar), (uint32_t)gw));
+                    bulk_copies_done();                  // (this CTA's shared memory is no longer read, the peer's no longer written)
+                }
+            }
+            __syncwarp();
+            cluster_arrive();                            // second round: this warp sends nothing to a peer any more
+            // step 3: add up the bands of this CTA once the other splits' copies of them have landed
+            const bool landed = __all_sync(0xffffffffu, mbar_wait_cluster(smem_u32(&red_bar), 0u, abortp, g.status, 14u, g.wait_ns));
+            // four outputs that are neighbours in memory, first one (mm, nn), `off` bytes into the band: the partial
+            // sums of all splits (this split's own from the staging copy, the others' from the reduction area)
+            auto load_sums = [&](uint32_t off, float4 (&p)[8]) {
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
-                    if (q < sk) p[q] = ld_shared_v4f(addr + (uint32_t)q * stride);
+                    if (q < cr.sk) p[q] = ld_shared_v4f((q == split ? tiles_base + (uint32_t)q * cr.slot : cr.red + (uint32_t)(q < split ? q : q - 1) * cr.slot) + off);
+            };
+            // ... are added in split order, then bias, residual, activation, one 16-byte store
+            auto finish4 = [&](const float4 (&p)[8], int mm, int nn, int valid) {
                 float4 acc = p[0];
 #pragma unroll
                 for (int q = 1; q < 8; ++q)
-                    if (q < sk) { acc.x += p[q].x; acc.y += p[q].y; acc.z += p[q].z; acc.w += p[q].w; }
+                    if (q < cr.sk) { acc.x += p[q].x; acc.y += p[q].y; acc.z += p[q].z; acc.w += p[q].w; }
                 float v[4] = {acc.x, acc.y, acc.z, acc.w};
-                const long long o = (long long)mm * g.y_ms + (long long)nn * g.y_ns;   // the four are o, o+1, o+2, o+3
+                const long long o = (long long)mm * cr.y_ms + (long long)nn * cr.y_ns;   // the four are o, o+1, o+2, o+3
+                // the tile's bias values were staged in shared memory before the main loop
+                if (cr.bias_mode == 1) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    if (i < valid) {
-                        // the tile's bias values were staged in shared memory before the main loop
-                        if (g.bias_mode == 1) v[i] += s_bias[mm - m0 + (along_cols ? 0 : i)];
-                        else if (g.bias_mode == 2) v[i] += s_bias[nn - n0 + (along_cols ? i : 0)];
-                        if (rbase) v[i] += __ldg(rbase + o + i);
-                        v[i] = gelu ? gelu_erf(v[i]) : fminf(fmaxf(v[i], lo), hi);
-                    }
+                    for (int i = 0; i < 4; ++i) v[i] += s_bias[mm - m0 + (cr.along_cols ? 0 : i)];
+                } else if (cr.bias_mode == 2) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) v[i] += s_bias[nn - n0 + (cr.along_cols ? i : 0)];
                 }
-                if (valid == 4 && vec_ok) *reinterpret_cast<float4*>(ybase + o) = make_float4(v[0], v[1], v[2], v[3]);
+                if (cr.rbase) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        if (i < valid) v[i] += __ldg(cr.rbase + o + i);
+                }
+                if (cr.gelu) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) v[i] = gelu_erf(v[i]);
+                } else if (cr.clamp) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) v[i] = fminf(fmaxf(v[i], cr.lo), cr.hi);
+                }
+                if (valid == 4 && cr.vec_ok) *reinterpret_cast<float4*>(cr.ybase + o) = make_float4(v[0], v[1], v[2], v[3]);
                 else {
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
-                        if (i < valid) ybase[o + i] = v[i];
+                        if (i < valid) cr.ybase[o + i] = v[i];
                 }
             };
-            if (along_cols) {
-                // this CTA's band of rows; a warp takes a row, its lanes walk the columns four at a time
-                const int per = (kHwTileM + sk - 1) / sk;
-                const int rows_here = min(min(kHwTileM, (split + 1) * per), g.M - m0) - split * per;
+            // a warp takes two lines (rows or columns) of the band at a time, the loads of both under way together (one
+            // line in the register-capped build)
+            constexpr int kLines = MIN_CTAS == 1 ? 2 : 1;
+            if (!landed) {
+                // (the wait recorded the time-out; nothing is stored)
+            } else if (cr.along_cols) {
+                // this CTA's band of rows; the lanes of a warp walk a row's columns four at a time
+                const int rows_here = min(min(kHwTileM, (split + 1) * cr.per), g.M - m0) - split * cr.per;
                 const int c_end = min(g.tile_n, g.N - n0);
-                const int pitch = g.tile_n + 4;
-                for (int rl = gw; rl < rows_here; rl += kGatherWarps)
-                    for (int col = lane * 4; col < c_end; col += 128)
-                        finish4(red + 4u * (uint32_t)(rl * pitch + col), 4u * (uint32_t)(per * pitch), m0 + split * per + rl, n0 + col,
-                                min(4, c_end - col));
+                for (int rl = gw; rl < rows_here; rl += kLines * kGatherWarps) {
+                    const bool two = kLines == 2 && rl + kGatherWarps < rows_here;
+                    for (int col = lane * 4; col < c_end; col += 128) {
+                        float4 pa[8], pb[8];
+                        load_sums((uint32_t)rl * cr.line + 4u * (uint32_t)col, pa);
+                        if (two) load_sums((uint32_t)(rl + kGatherWarps) * cr.line + 4u * (uint32_t)col, pb);
+                        finish4(pa, m0 + split * cr.per + rl, n0 + col, min(4, c_end - col));
+                        if (two) finish4(pb, m0 + split * cr.per + rl + kGatherWarps, n0 + col, min(4, c_end - col));
+                    }
+                }
             } else {
-                // this CTA's band of columns; a warp takes a column, its lanes walk the 128 rows four at a time
-                const int per = (g.tile_n + sk - 1) / sk;
-                const int cols_here = min(min(g.tile_n, (split + 1) * per), g.N - n0) - split * per;
+                // this CTA's band of columns; the lanes of a warp walk a column's 128 rows four at a time
+                const int cols_here = min(min(g.tile_n, (split + 1) * cr.per), g.N - n0) - split * cr.per;
                 const int r_end = min(kHwTileM, g.M - m0);
-                for (int cl = gw; cl < cols_here; cl += kGatherWarps)
-                    if (lane * 4 < r_end)
-                        finish4(red + 4u * (uint32_t)(cl * kRedColPitch + lane * 4), 4u * (uint32_t)(per * kRedColPitch), m0 + lane * 4,
-                                n0 + split * per + cl, min(4, r_end - lane * 4));
+                if (lane * 4 < r_end)
+                    for (int cl = gw; cl < cols_here; cl += kLines * kGatherWarps) {
+                        const bool two = kLines == 2 && cl + kGatherWarps < cols_here;
+                        float4 pa[8], pb[8];
+                        load_sums((uint32_t)cl * cr.line + 16u * (uint32_t)lane, pa);
+                        if (two) load_sums((uint32_t)(cl + kGatherWarps) * cr.line + 16u * (uint32_t)lane, pb);
+                        finish4(pa, m0 + lane * 4, n0 + split * cr.per + cl, min(4, r_end - lane * 4));
+                        if (two) finish4(pb, m0 + lane * 4, n0 + split * cr.per + cl + kGatherWarps, min(4, r_end - lane * 4));
+                    }
             }
         }
+    }
+    if (g.cluster) {
+        // Every thread of every CTA of the cluster takes part in both rounds of the cluster barrier, also after a
+        // tripped wait: the second round completes when no CTA sends any more, so none leaves while a copy into its
+        // shared memory could still be under way.
+        if (warp < 2) cluster_arrive();
+        cluster_wait();
     }
     tc_fence_before();
     __syncthreads();
@@ -1513,33 +1623,6 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank) 
         "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
         "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
         ::"r"(bar), "r"(rank) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok;
-}
-// Bounded wait on a barrier that CTAs of the cluster arrive on (acquire at cluster scope).
-__device__ __noinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned* status,
-                                               unsigned where, unsigned long long limit_ns) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    const unsigned long long t0 = global_timer_ns();
-    unsigned spins = 0;
-    for (;;) {
-        if (mbar_try_wait_cluster(bar, parity)) return true;
-        if ((++spins & 31u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > limit_ns) {
-                *abort_flag = 1;
-                atomicCAS(status, 0u, (unsigned)TT_ERR_TIMEOUT | (where << 8));
-                return false;
-            }
-        }
-    }
 }
 // TMA load whose completion is reported to a barrier given by its cluster-wide address, which may lie in the other
 // CTA of the pair (no multicast: the data goes to this CTA's shared memory only).
@@ -2069,7 +2152,7 @@ tt_gemm_ps_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (e.gelu) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
-                    } else {
+                    } else if (g.act != TT_ACT_NONE) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) v[j] = fminf(fmaxf(v[j], e.lo), e.hi);
                     }
