@@ -108,7 +108,8 @@ def workload_name(model, specs, pool_sources):
 
 def config_dict(model, specs, pool_sources):
     return {"workload": workload_name(model, specs, pool_sources), "l2": "flushed between steps (256 MB write)",
-            "replay": "one CUDA graph per data-chained model pass", "multi_gpu": "independent replicas",
+            "replay": "one CUDA graph per data-chained model pass; layers without a data dependency on side streams of the graph",
+            "multi_gpu": "independent replicas",
             "weights": "declared constant to the library (a kernel may fetch them before it waits for its predecessor)",
             "evaluation": "every (kernel, record) pair timed standalone with warm activations and rotating copies of the weights"}
 
@@ -406,12 +407,25 @@ class Bench:
             bufs, ch_tts = W.chain_device_tensors(steps_, ch_arrays, dev)
             order = [(st.kernel, tt) for st, tt in zip(steps_, ch_tts) if st.spec is not None]
             del ch_arrays
+            # layers that do not depend on one another (the projections of an attention block, a block's downsample
+            # beside its first convolution) go to side streams of the same graph; a kernel whose record keeps scratch
+            # in its workload (split-K workspace, re-packed filters) never runs beside itself
+            serial = {i for i, inf in enumerate(infos) if inf.launches > 1 or inf.legal.split_k > 8}
+            plan = W.chain_lanes(steps_, max_lanes=4, serial_kernels=serial)
+            side_streams = [torch.cuda.Stream(device=dev) for _ in range(3)]
+            out["chain_lanes"] = {"streams": 1 + len({pl[0] for pl in plan if pl} - {0}),
+                                  "cross_stream_waits": sum(len(pl[1]) for pl in plan if pl)}
         else:
-            bufs, order = None, [(i, tt) for i, (tt, u) in enumerate(zip(tts, use)) for _ in range(u)]
+            bufs, order, plan = None, [(i, tt) for i, (tt, u) in enumerate(zip(tts, use)) for _ in range(u)], None
 
-        def chained_pass():
+        def sequential_pass():
             for k, tt in order:
                 wls[k].run(tt)
+
+        def chained_pass():
+            if plan is None:
+                return sequential_pass()
+            W.run_chain(wls, steps_, ch_tts, plan, [torch.cuda.current_stream()] + side_streams)
 
         def independent_pass():
             for w, t, u in zip(wls, tts, use):
@@ -438,6 +452,10 @@ class Bench:
         else:
             chained_cold = self.timed_steps(n_side, graph.replay) / n_side * 1e3
         chained_warm = self.timed_steps(n_side, graph.replay, flush=False) / n_side * 1e3
+        gs = self.capture(sequential_pass)
+        self.timed_steps(3, gs.replay)
+        sequential_cold = self.timed_steps(n_side, gs.replay) / n_side * 1e3
+        del gs
         gi = self.capture(independent_pass)
         self.timed_steps(3, gi.replay)
         indep_cold = self.timed_steps(n_side, gi.replay) / n_side * 1e3
@@ -446,7 +464,7 @@ class Bench:
             st = w.status()
             if st != B.TT_OK:
                 raise SystemExit(f"device status {st} after the timed region of {cname}")
-        out["pass_us"] = {"chained_cold_l2": chained_cold, "chained_warm_l2": chained_warm,
+        out["pass_us"] = {"chained_cold_l2": chained_cold, "chained_warm_l2": chained_warm, "chained_one_stream_cold_l2": sequential_cold,
                           "independent_kernels_cold_l2": indep_cold, "tflops_chained_cold_l2": flops_pass / chained_cold / 1e6}
 
         # per kernel: cold-L2 standalone time and launch floor under the chosen record; per class: roofline fractions

@@ -400,3 +400,74 @@ def chain_device_tensors(steps, arrays, device="cuda"):
         bufs.append(t)
         tts.append(B.tensors(t["x"], t["w"], t["bias"], t["residual"], t["y"]))
     return bufs, tts
+
+
+def chain_lanes(steps, max_lanes=4, serial_kernels=()):
+    """Which layers of a chain may run side by side.  A layer depends only on the nodes it is wired to (x, res, w_from):
+    the three projections of an attention block read the same input, a residual block's 1x1 downsample and its first
+    3x3 convolution read the same block input.  Returns, per node, None (an external tensor) or (lane, waits): the
+    layer is enqueued on stream `lane`, after waiting for the events of the layers in `waits` (its producers on other
+    lanes).  A layer follows its input's producer on that producer's lane when it is the first to do so, otherwise it
+    takes the lane that has been idle longest.  Kernels in `serial_kernels` (their applied record keeps per-workload
+    scratch: a split-K workspace, re-packed filters) never overlap with themselves: each of their layers also waits
+    for the previous one.  Every lane's work is ordered, so any assignment is correct; the choice only decides how
+    much runs concurrently."""
+    lane_of, tail, last_used, plan = {}, [], [], []
+    last_of_kernel = {}
+    for i, st in enumerate(steps):
+        if st.spec is None:
+            plan.append(None)
+            continue
+        prods = [p for p in (st.x, st.w_from, st.res) if p is not None and steps[p].spec is not None]
+        for p in (st.x, st.w_from, st.res):
+            # a stand-in tensor replaces an operator outside the hot path that the model feeds from the layer in front
+            # of it: the dependency stays (the model's own input, node 0, has none)
+            if p is not None and p > 0 and steps[p].spec is None:
+                prods += [q for q in range(p - 1, -1, -1) if steps[q].spec is not None][:1]
+        if st.kernel in serial_kernels and st.kernel in last_of_kernel:
+            prods.append(last_of_kernel[st.kernel])
+        lane = None
+        for p in prods:                                   # continue a producer's lane if nobody has yet
+            if tail[lane_of[p]] == p:
+                lane = lane_of[p]
+                break
+        if lane is None:
+            lane = len(tail) if len(tail) < max_lanes else min(range(len(tail)), key=lambda l: last_used[l])
+        if lane == len(tail):
+            tail.append(None)
+            last_used.append(-1)
+        waits = sorted({p for p in prods if lane_of[p] != lane})
+        # work that ran earlier on this lane is ordered before this layer by the stream itself
+        lane_of[i], tail[lane], last_used[lane] = lane, i, i
+        last_of_kernel[st.kernel] = i
+        plan.append((lane, waits))
+    return plan
+
+
+def run_chain(wls, steps, tts, plan, streams):
+    """Enqueue one pass of a chain: streams[0] is the caller's current stream (under stream capture: the capturing one),
+    the others are side streams that fork from it and join it again at the end."""
+    import torch
+    events, used = {}, set()
+    needed = {p for pl in plan if pl is not None for p in pl[1]}
+    start = torch.cuda.Event()
+    start.record(streams[0])
+    for i, (st, tt, pl) in enumerate(zip(steps, tts, plan)):
+        if pl is None:
+            continue
+        lane, waits = pl
+        s = streams[lane]
+        if lane != 0 and lane not in used:
+            s.wait_event(start)                           # the side stream joins (a capture, or the caller's ordering)
+        used.add(lane)
+        for p in waits:
+            s.wait_event(events[p])
+        with torch.cuda.stream(s):
+            wls[st.kernel].run(tt)
+        if i in needed:
+            events[i] = torch.cuda.Event()
+            events[i].record(s)
+    for lane in sorted(used - {0}):
+        e = torch.cuda.Event()
+        e.record(streams[lane])
+        streams[0].wait_event(e)

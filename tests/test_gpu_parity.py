@@ -863,3 +863,60 @@ def test_subsampled_evaluator_skips_what_the_rule_says_and_keeps_a_valid_choice(
     wl.run(tt)                                           # the chosen record is left applied
     assert util.rel_l2(t["y"].cpu().numpy(), util.oracle_ref(spec, a)) <= util.TOL_TF32
     wl.close()
+
+
+@pytest.mark.parametrize("model,make,seed", [("resnet18", W.resnet18_net, 2), ("bert_base", lambda: W.bert_base_net(layers=2), 5)])
+def test_chain_on_several_streams_matches_the_oracle_chain(model, make, seed):
+    """The same chain with layers that do not depend on one another on side streams (the attention projections, a
+    block's downsample beside its first convolution), enqueued directly and replayed as one captured graph: every
+    layer's output against the oracle chain.  The projections share one workload object and run beside one another."""
+    import torch
+    specs, steps = make()
+    arrays = W.make_chain_inputs(steps, seed, init="bert" if model.startswith("bert") else "he")
+    refs = util.oracle_chain(steps, arrays)
+    depth = _tf32_depth(steps)
+    wls = [sp.workload() for sp in specs]
+    rec = tc(tile_n=64, tile_k=64, stages=2, split_k=4, mma_m_axis=2)
+    for wl in wls:
+        wl.apply(rec if wl.family() == B.TT_FAMILY_GEMM_TC else wl.default_schedule())
+        wl.set_constant_weights(True)
+    bufs, tts = W.chain_device_tensors(steps, arrays)
+    plan = W.chain_lanes(steps, max_lanes=4)
+    assert len({pl[0] for pl in plan if pl}) == 4
+    side = [torch.cuda.Stream() for _ in range(3)]
+
+    def clear():
+        for st, b in zip(steps, bufs):
+            if st.spec is not None:
+                b["y"].fill_(float("nan"))
+
+    def check(what):
+        for wl in wls:
+            assert wl.status() == B.TT_OK
+        for i, (st, b, ref, d) in enumerate(zip(steps, bufs, refs, depth)):
+            if st.spec is None:
+                continue
+            y = b["y"].cpu().numpy()
+            assert not np.isnan(y).any(), (what, model, i, st.spec.name)
+            tol = max(d, 1) * util.TOL_TF32 if d else util.TOL_FP32
+            assert util.rel_l2(y, ref) <= tol, (what, model, i, st.spec.name, d, util.rel_l2(y, ref))
+
+    main = torch.cuda.Stream()
+    with torch.cuda.stream(main):
+        for _ in range(2):
+            clear()
+            W.run_chain(wls, steps, tts, plan, [main] + side)
+        main.synchronize()
+    torch.cuda.synchronize()
+    check("direct")
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=main):
+        W.run_chain(wls, steps, tts, plan, [torch.cuda.current_stream()] + side)
+    for _ in range(3):
+        clear()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+    check("graph")
+    for wl in wls:
+        wl.close()

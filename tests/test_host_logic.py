@@ -515,3 +515,34 @@ def test_pool_subsample_matches_the_oracle():
         assert B.pool_subsample(n, c, seed) == orc.pool_subsample(n, c, seed)
     out = (ctypes.c_int32 * 4)()
     assert B.lib().tt_pool_subsample(3, 4, 0, out) == B.TT_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("model", ["resnet18", "resnet50", "mobilenet_v2", "bert_base"])
+def test_chain_lanes_order_every_dependency(model):
+    """The side-by-side plan of a chain: every producer of a layer (input, skip tensor, second operand, and the layer a
+    stand-in tensor replaces) either ran earlier on the layer's own lane or is waited for; kernels declared serial
+    never overlap with themselves; the attention projections and the downsample convolutions do leave lane 0."""
+    specs, steps = W.CHAINS[model]()
+    serial = {0}
+    plan = W.chain_lanes(steps, max_lanes=4, serial_kernels=serial)
+    assert len(plan) == len(steps)
+    seen_on_lane = {}
+    last_serial = {}
+    for i, (st, pl) in enumerate(zip(steps, plan)):
+        assert (pl is None) == (st.spec is None)
+        if pl is None:
+            continue
+        lane, waits = pl
+        assert 0 <= lane < 4 and all(w < i and plan[w] is not None for w in waits)
+        need = [p for p in (st.x, st.w_from, st.res) if p is not None and steps[p].spec is not None]
+        for p in (st.x, st.w_from, st.res):
+            if p is not None and p > 0 and steps[p].spec is None:
+                need += [q for q in range(p - 1, -1, -1) if steps[q].spec is not None][:1]
+        if st.kernel in serial and st.kernel in last_serial:
+            need.append(last_serial[st.kernel])
+        for p in need:
+            assert plan[p][0] == lane or p in waits, (model, i, p)
+        seen_on_lane.setdefault(lane, []).append(i)
+        last_serial[st.kernel] = i
+    lanes_used = len(seen_on_lane)
+    assert lanes_used == (1 if model == "mobilenet_v2" else 4)
