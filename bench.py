@@ -720,7 +720,7 @@ def main():
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = traffic_per_launch()
     roof["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum, timed region average)"
-    roof.update({"kernel": "tt_gemm_tc_kernel",
+    roof.update({"kernel": "GEMM_TC family: tt_gemm_tc_kernel (one tile per CTA) + tt_gemm_ps_kernel (persistent)",
                  "peak_source": peaks["source"] + (" hbm copy" if roof["bound"] == "hbm" else " bf16 burst / 2 (TF32 issues at half the BF16 rate)"),
                  "launches_per_pass": gemm["launches"], "avg_launch_us": gemm["cold_us"] / max(gemm["launches"], 1),
                  "avg_launch_floor_us": gemm["floor_us"] / max(gemm["launches"], 1),
