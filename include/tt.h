@@ -125,7 +125,7 @@ typedef struct tt_schedule_record {
     int32_t k_order;       /* GEMM_TC, conv2d: order in which the reduction (c, r, s) is walked.  0 = as the filters are
                               stored (channel-major; the im2col operand is expanded stage by stage).  1 = blocks of 32
                               channels, tap by tap inside a block: the filters are re-packed into that order by a small
-                              kernel before each run, the input rows are transposed once per block into a pixel-major
+                              kernel (once per weight pointer: again only when tt_run sees other weights), the input rows are transposed once per block into a pixel-major
                               slab, and every tap's operand tile is a shifted view of that slab -- no expansion.
                               Stride-1 convolutions with 16-byte image rows, filters on the 128 rows, split_k = 1;
                               tile_k = 32 * (taps per pipeline stage), the tap count a divisor of r*s, at most 128. */
