@@ -378,11 +378,22 @@ class Bench:
         o.include_default = 1
         o.timing.warmup_batches, o.timing.batches, o.timing.min_batch_us, o.timing.use_graph = 3, 10, 200, 1
         eval_sets = [self.weight_sets(sp, t) for sp, t in zip(specs, dev_t)]
+        n_cols = len(pool) + 1
+        use = [sp.use_count for sp in specs]
+        sub = None
+        if len(pool) >= 8 and not headline:
+            # the same search with pool sub-sampling: a seeded quarter of the pool first, the rest only for kernels that
+            # are not yet 10 % better than their default record (run first: the full search below leaves its choice applied)
+            o.subsample_percent, o.subsample_gain_percent, o.subsample_seed = 25, 10, 1
+            r2 = B.transfer_tune(list(wls), [sets for _, sets in eval_sets], pool, o)
+            flat2 = [v for row in r2["times_us"] for v in row]
+            sub = {"percent": 25, "gain_percent": 10, "pairs_timed": r2["pairs_timed"], "pairs_skipped": r2["pairs_skipped"],
+                   "seconds": r2["search_seconds"],
+                   "sum_standalone_us": B.model_latency(flat2, len(wls), n_cols, r2["chosen"], use)}
+            o.subsample_percent = 0
         res = B.transfer_tune(list(wls), [sets for _, sets in eval_sets], pool, o)
         del eval_sets
-        n_cols = len(pool) + 1
         chosen = res["chosen"]
-        use = [sp.use_count for sp in specs]
         flat = [v for row in res["times_us"] for v in row]
         lat_best = B.model_latency(flat, len(wls), n_cols, chosen, use)
         lat_default = B.model_latency(flat, len(wls), n_cols, [0] * len(wls), use)
@@ -398,7 +409,7 @@ class Bench:
                "sum_standalone_us": {"transferred": lat_best, "default": lat_default,
                                      "speedup_over_default": lat_default / lat_best if lat_best else None},
                "search": {"pairs_timed": res["pairs_timed"], "pairs_invalid": res["pairs_invalid"],
-                          "seconds": res["search_seconds"], "pool_records": len(pool)}}
+                          "seconds": res["search_seconds"], "pool_records": len(pool), "with_pool_subsampling": sub}}
 
         # the data-chained pass (config 1 is a single kernel: its pass is that kernel)
         if model in W.CHAINS:
