@@ -84,7 +84,7 @@ typedef struct tt_shapes {
     float scale;                                                   /* softmax only */
 } tt_shapes;
 
-#define TT_RECORD_VERSION 2u
+#define TT_RECORD_VERSION 3u
 
 /* A schedule record.  Correspondence with the primitives listed under Algorithm 1:
  *   Split     -> tile_m, tile_n, tile_k (CTA tile of the output and of the reduction), split_k
@@ -95,7 +95,7 @@ typedef struct tt_shapes {
  *                               `stages` shared-memory buffers decouple loading from the multiply
  *   Vectorize -> vec_width;   Unroll -> unroll / items_per_thread
  * GEMM_TC uses tile_m, tile_n, tile_k, stages, split_k, raster, mma_m_axis, slab_tiles, acc_split, k_order, persistent,
- *         cta_group, ctas_per_sm, warp_layout.
+ *         cta_group, ctas_per_sm, warp_layout, precision.
  * DW_SIMT uses tile_m (channels per CTA), block_y x block_x (output rows x columns per CTA tile),
  *         items_per_thread (consecutive outputs along the width per thread), vec_width, threads, and unroll:
  *         0 = shared-memory staged kernel; 1, 2, 4 = register-window kernel with that many output rows per thread
@@ -146,6 +146,13 @@ typedef struct tt_schedule_record {
     int32_t warp_layout;   /* GEMM_TC: warps by role.  0 = the only layout of each kernel form: 1 TMA + 1 MMA + 8 operand
                               producers that then read out (320 threads), or, persistent, 1 TMA + 1 MMA + 4 transposers + 4
                               read-out warps.  Reserved for further layouts; any other value is invalid. */
+    int32_t precision;     /* GEMM_TC: 0 = operands are read by the tensor core as TF32 (their fp32 values truncated to 10
+                              mantissa bits).  1 = error-compensated ("3xTF32"): each operand tile is split in shared memory
+                              into what the tensor core sees and the remainder, and every reduction step issues three
+                              multiply-accumulates (a*b_lo, a_lo*b, a*b), which brings the result to within fp32
+                              accumulation error of the exact product at three times the tensor work and twice the
+                              shared memory per stage.  One-tile form, dense and batch_matmul NT with K a multiple of 4;
+                              elsewhere legalised to 0 (TT_CHG_FORM). */
 } tt_schedule_record;
 
 typedef struct tt_tensors {

@@ -20,7 +20,7 @@ TT_OP_CONV2D, TT_OP_DWCONV2D, TT_OP_DENSE, TT_OP_BATCH_MATMUL, TT_OP_SOFTMAX = r
 TT_ACT_NONE, TT_ACT_RELU, TT_ACT_RELU6, TT_ACT_GELU_ERF = range(4)
 TT_FAMILY_GEMM_TC, TT_FAMILY_DW_SIMT, TT_FAMILY_ROW_SIMT = range(3)
 TT_MODE_LEGALISE, TT_MODE_STRICT = 0, 1
-TT_RECORD_VERSION = 2
+TT_RECORD_VERSION = 3
 TT_CHG_TILE_M, TT_CHG_TILE_N, TT_CHG_TILE_K, TT_CHG_STAGES, TT_CHG_SPLIT_K, TT_CHG_VEC, TT_CHG_BLOCK, TT_CHG_ITEMS, TT_CHG_SLAB, TT_CHG_ACC, TT_CHG_KORDER, TT_CHG_FORM = \
     1, 2, 4, 8, 16, 32, 64, 128, 256, 512, 1024, 2048
 
@@ -37,11 +37,11 @@ class tt_schedule_record(C.Structure):
     _fields_ = [("version", u32), ("family", u32), ("origin_op", i32), ("origin", tt_shapes)] + \
                [(n, i32) for n in ("tile_m", "tile_n", "tile_k", "stages", "split_k", "raster", "block_x", "block_y",
                                    "items_per_thread", "vec_width", "unroll", "threads", "mma_m_axis", "slab_tiles", "acc_split", "k_order",
-                                   "persistent", "cta_group", "ctas_per_sm", "warp_layout")]
+                                   "persistent", "cta_group", "ctas_per_sm", "warp_layout", "precision")]
 
     FIELDS = ("tile_m", "tile_n", "tile_k", "stages", "split_k", "raster", "block_x", "block_y",
               "items_per_thread", "vec_width", "unroll", "threads", "mma_m_axis", "slab_tiles", "acc_split", "k_order",
-              "persistent", "cta_group", "ctas_per_sm", "warp_layout")
+              "persistent", "cta_group", "ctas_per_sm", "warp_layout", "precision")
 
     def as_dict(self):
         d = {"family": int(self.family), "origin_op": int(self.origin_op)}
@@ -54,7 +54,7 @@ class tt_schedule_record(C.Structure):
                     f"r{self.raster} ax{self.mma_m_axis}" + (f" sl{self.slab_tiles}" if self.slab_tiles else "") +
                     (f" acc{self.acc_split}" if self.acc_split > 1 else "") + (" tap" if self.k_order else "") +
                     (" ps" if self.persistent else "") + (" cg2" if self.cta_group == 2 else "") +
-                    (" 2/sm" if self.ctas_per_sm == 2 else "") + "]")
+                    (" 2/sm" if self.ctas_per_sm == 2 else "") + (" x3" if self.precision else "") + "]")
         if self.family == TT_FAMILY_DW_SIMT:
             return (f"dw[c{self.tile_m} {self.block_y}x{self.block_x} it{self.items_per_thread} "
                     f"v{self.vec_width} t{self.threads} u{self.unroll}" + (f" tma st{self.stages}" if self.raster else "") + "]")
@@ -210,7 +210,7 @@ def make_record(family, **kw) -> tt_schedule_record:
     r.family = family
     defaults = dict(tile_m=128, tile_n=128, tile_k=32, stages=4, split_k=1, raster=0, block_x=32, block_y=4,
                     items_per_thread=1, vec_width=1, unroll=1, threads=128, mma_m_axis=0, slab_tiles=0, acc_split=1, k_order=0,
-                    persistent=0, cta_group=1, ctas_per_sm=0, warp_layout=0)
+                    persistent=0, cta_group=1, ctas_per_sm=0, warp_layout=0, precision=0)
     defaults.update(kw)
     for k, v in defaults.items():
         setattr(r, k, v)

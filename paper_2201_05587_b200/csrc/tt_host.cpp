@@ -115,12 +115,14 @@ static tt_status legalise_conv_tapmajor(const tt_workload* w, const tt_schedule_
     if (strict && (rec->mma_m_axis == 2 || rec->tile_k != tk || rec->split_k != 1)) return TT_ERR_INVALID_SCHEDULE;
     L.mma_m_axis = 1; L.tile_m = kHwTileM; L.tile_k = tk; L.split_k = 1; L.acc_split = 1; L.slab_tiles = 0; L.k_order = 1;
     if (rec->persistent < 0 || rec->persistent > 1 || rec->cta_group < 0 || rec->cta_group > 2 || rec->ctas_per_sm < 0 ||
-        rec->ctas_per_sm > 2 || rec->warp_layout != 0)
+        rec->ctas_per_sm > 2 || rec->warp_layout != 0 || rec->precision < 0 || rec->precision > 1)
         return TT_ERR_INVALID_SCHEDULE;
     // both kernel forms walk this reduction order; CTA pairs do not
     const bool persistent = rec->persistent == 1;
     L.persistent = persistent ? 1 : 0; L.cta_group = 1;
     if (rec->cta_group == 2) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_FORM; }
+    L.precision = 0;                                      // (no error-compensated products for convolutions)
+    if (rec->precision != 0) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_FORM; }
     if (rec->tile_m != kHwTileM) changed |= TT_CHG_TILE_M;
     if (rec->tile_k != tk) changed |= TT_CHG_TILE_K;
     if (rec->split_k != 1) changed |= TT_CHG_SPLIT_K;
@@ -238,7 +240,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     if (rec->tile_m <= 0 || rec->tile_n <= 0 || rec->tile_k <= 0 || rec->stages <= 0 || rec->split_k <= 0 ||
         rec->raster < 0 || rec->raster > 1 || rec->mma_m_axis < 0 || rec->mma_m_axis > 2 || rec->persistent < 0 ||
         rec->persistent > 1 || rec->cta_group < 0 || rec->cta_group > 2 || rec->ctas_per_sm < 0 || rec->ctas_per_sm > 2 ||
-        rec->warp_layout != 0)
+        rec->warp_layout != 0 || rec->precision < 0 || rec->precision > 1)
         return TT_ERR_INVALID_SCHEDULE;
     // Which output axis becomes the accumulator's 128 rows.  Left to the library (0), the shorter-than-a-tile
     // axis goes to the MMA's N side, where 16..256 columns are legal.
@@ -276,7 +278,16 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     const int k_tiles = (K + tk - 1) / tk;
     // The persistent form: both operands must be reachable by TMA -- K-major with 16-byte rows, or row-contiguous (the
     // image of a pointwise convolution, the second operand of an NN batch_matmul) with 16-byte row pitch.
+    // Error-compensated products need both operands as K-major TMA tiles (their remainders are worked out in place, tile by
+    // tile) and exist in the one-tile form only: dense and batch_matmul NT with 16-byte rows.
+    bool x3 = rec->precision == 1;
+    if (x3 && !((w->op == TT_OP_DENSE || (w->op == TT_OP_BATCH_MATMUL && w->sh.trans_b)) && (K % 4) == 0)) {
+        if (strict) return TT_ERR_INVALID_SCHEDULE;
+        x3 = false; changed |= TT_CHG_FORM;
+    }
+    L.precision = x3 ? 1 : 0;
     bool persistent = rec->persistent == 1;
+    if (persistent && x3) { if (strict) return TT_ERR_INVALID_SCHEDULE; persistent = false; changed |= TT_CHG_FORM; }
     {
         const tt_shapes& o = w->sh;
         bool can = (K % 4) == 0;
@@ -303,7 +314,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     L.split_k = sk;
     // accumulators: a power of two, all of them inside the 512 columns of tensor memory, none left without a step
     if (rec->acc_split < 0) return TT_ERR_INVALID_SCHEDULE;
-    int nacc = persistent ? 1 : std::min(8, pow2_floor(std::max(1, rec->acc_split)));
+    int nacc = (persistent || x3) ? 1 : std::min(8, pow2_floor(std::max(1, rec->acc_split)));
     while (nacc > 1 && (nacc * tn > 512 || (long long)nacc > (long long)per_split * (tk / 8))) nacc >>= 1;
     if (nacc != std::max(1, rec->acc_split)) { if (strict) return TT_ERR_INVALID_SCHEDULE; changed |= TT_CHG_ACC; }
     L.acc_split = nacc;
@@ -465,7 +476,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     };
     long long smem = 0;
     for (;;) {
-        const long long pipe_try = std::max<long long>((long long)st * (a_stage + b_stage), min_pipe);
+        const long long pipe_try = std::max<long long>((long long)st * (a_stage + b_stage) * (x3 ? 2 : 1), min_pipe);
         long long slab_total = 0;
         bool fits = true;
         if (conv) {
@@ -487,7 +498,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
         changed |= TT_CHG_STAGES;
     }
     L.stages = st;
-    const long long pipe = std::max<long long>((long long)st * (a_stage + b_stage), min_pipe);
+    const long long pipe = std::max<long long>((long long)st * (a_stage + b_stage) * (x3 ? 2 : 1), min_pipe);
     if (conv) {
         if (rec->slab_tiles != 0 && sl_tiles != rec->slab_tiles) {
             if (strict) return TT_ERR_INVALID_SCHEDULE;
@@ -554,6 +565,7 @@ static tt_status legalise_gemm(const tt_workload* w, const tt_schedule_record* r
     g.n_acc = nacc;
     g.cluster = cluster;
     g.two_per_sm = L.ctas_per_sm == 2;
+    g.x3 = x3 ? 1 : 0;
     g.b_rows_cta = tn; g.cta_group = 1;
     // Instruction descriptor, kind::tf32: D = F32 (bits 4-5 = 1), A and B = TF32 (bits 7-9, 10-12 = 2), both
     // K-major (bits 15, 16 = 0), N >> 3 at bits 17-22, M >> 4 at bits 24-28.
@@ -1022,6 +1034,7 @@ const RecField kRecFields[] = {
     {"acc_split", &tt_schedule_record::acc_split}, {"k_order", &tt_schedule_record::k_order},
     {"persistent", &tt_schedule_record::persistent}, {"cta_group", &tt_schedule_record::cta_group},
     {"ctas_per_sm", &tt_schedule_record::ctas_per_sm}, {"warp_layout", &tt_schedule_record::warp_layout},
+    {"precision", &tt_schedule_record::precision},
 };
 int32_t* shape_ints(tt_shapes& s, int i) {
     int32_t* f[] = {&s.n, &s.c, &s.h, &s.w, &s.k, &s.r, &s.s, &s.stride_h, &s.stride_w, &s.pad_h, &s.pad_w,

@@ -76,6 +76,7 @@ struct GemmArgs {
     int w_operand;                              // 1 / 2: operand A / B is constant (weights the caller promised nobody is
                                                 // writing): its first stages are requested before the wait on the kernel in front
     int two_per_sm;                             // the register-capped build, so that two CTAs share an SM
+    int x3;                                     // error-compensated products: a stage holds [A][B][A lo][B lo]
     // persistent kernel (record field persistent = 1)
     int persistent, cta_group;
     int total_tiles;                            // tiles_m * tiles_n * batch; tiles_m counts 128 * cta_group rows

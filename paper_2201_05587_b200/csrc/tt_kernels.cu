@@ -759,6 +759,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     __shared__ uint64_t pm_full[2];       // tap-major convolution: a pixel-major slab buffer has been written
     __shared__ uint64_t pm_empty[2];      // ... and every multiply-accumulate that reads it has completed
     __shared__ uint64_t red_bar;          // split-K over a cluster: the other splits' bands of this CTA's output have landed
+    __shared__ uint64_t lo_bar[kMaxStages];   // error-compensated products: the remainders of a stage's operand tiles are written
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int last_split_flag;
@@ -782,7 +783,9 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     const int iters = kt_end - kt_begin;
 
     const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t stage_bytes = g.a_stage_bytes + g.b_stage_bytes;
+    // (error-compensated products: a stage holds the two operand tiles and, behind them, their remainders)
+    const uint32_t lo_off = g.a_stage_bytes + g.b_stage_bytes;
+    const uint32_t stage_bytes = g.x3 ? 2u * lo_off : lo_off;
     const bool a_tma = g.a_mode == OPM_TMA, b_tma = g.b_mode == OPM_TMA;
     const bool any_tma = a_tma || b_tma, any_gather = !a_tma || !b_tma;
     const bool im2col = g.a_mode == OPM_IM2COL || g.b_mode == OPM_IM2COL;
@@ -821,6 +824,7 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
             mbar_init(smem_u32(&empty_bar[s]), 1u);
         }
         mbar_init(smem_u32(&accum_bar), 1u);
+        if (g.x3) for (int s = 0; s < g.stages; ++s) mbar_init(smem_u32(&lo_bar[s]), (uint32_t)kGatherWarps);
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&slab_full[b]), 1u);
             mbar_init(smem_u32(&slab_empty[b]), (uint32_t)kGatherWarps);
@@ -1028,7 +1032,8 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 }
             } else
             for (int it = 0; it < iters; ++it) {
-                const bool got = mbar_wait(full_addr, ph, abortp, g.status, 2u, g.wait_ns);
+                bool got = mbar_wait(full_addr, ph, abortp, g.status, 2u, g.wait_ns);
+                if (g.x3) got = mbar_wait(smem_u32(&lo_bar[st]), ph, abortp, g.status, 16u, g.wait_ns) && got;   // the remainders too
                 if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 tc_fence_after();
                 if (leader) {
@@ -1037,12 +1042,23 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                     if (g.n_acc == 1) {
                         // one accumulator: nothing to rotate.  The common tile_k values are unrolled completely, so
                         // that an issue is two additions and the instruction.
+                        auto issue_stage = [&](uint32_t a0, uint32_t b0, uint32_t accumulate) {
+                            if (g.tile_k == 64) issue_steps<2, 4>(tmem_base, d_hi, a0, b0, a_atom, b_atom, g.idesc, accumulate);
+                            else if (g.tile_k == 32) issue_steps<1, 4>(tmem_base, d_hi, a0, b0, a_atom, b_atom, g.idesc, accumulate);
+                            else if (g.tile_k == 128) issue_steps<4, 4>(tmem_base, d_hi, a0, b0, a_atom, b_atom, g.idesc, accumulate);
+                            else if (g.tile_k == 16) issue_steps<1, 2>(tmem_base, d_hi, a0, b0, a_atom, b_atom, g.idesc, accumulate);
+                            else issue_steps<1, 1>(tmem_base, d_hi, a0, b0, a_atom, b_atom, g.idesc, accumulate);
+                        };
                         const uint32_t accumulate = it > 0 ? 1u : 0u;
-                        if (g.tile_k == 64) issue_steps<2, 4>(tmem_base, d_hi, a_lo, b_lo, a_atom, b_atom, g.idesc, accumulate);
-                        else if (g.tile_k == 32) issue_steps<1, 4>(tmem_base, d_hi, a_lo, b_lo, a_atom, b_atom, g.idesc, accumulate);
-                        else if (g.tile_k == 128) issue_steps<4, 4>(tmem_base, d_hi, a_lo, b_lo, a_atom, b_atom, g.idesc, accumulate);
-                        else if (g.tile_k == 16) issue_steps<1, 2>(tmem_base, d_hi, a_lo, b_lo, a_atom, b_atom, g.idesc, accumulate);
-                        else issue_steps<1, 1>(tmem_base, d_hi, a_lo, b_lo, a_atom, b_atom, g.idesc, accumulate);
+                        if (g.x3) {
+                            // the two cross terms first (small), then the product of what the tensor core sees of a and b
+                            const uint32_t lo = lo_off >> 4;
+                            issue_stage(a_lo + lo, b_lo, accumulate);
+                            issue_stage(a_lo, b_lo + lo, 1u);
+                            issue_stage(a_lo, b_lo, 1u);
+                        } else {
+                            issue_stage(a_lo, b_lo, accumulate);
+                        }
                     } else
 #pragma unroll 1
                     for (int at = 0; at < g.n_atoms; ++at) {
@@ -1253,6 +1269,28 @@ tt_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
                 if (lane == 0) mbar_arrive(full0 + (uint32_t)st * 8u);
                 st += n_groups;
                 while (st >= g.stages) { st -= g.stages; ph ^= 1u; }
+            }
+        }
+        if (g.x3) {
+            // ---- error-compensated products: once a stage's operand tiles have landed, the eight warps write, 16 bytes
+            // per thread and step, what the tensor core will NOT see of every value (x minus x truncated to TF32's ten
+            // mantissa bits: exact in fp32) into the second half of the stage, in the same swizzled layout ----
+            const uint32_t full0 = smem_u32(&full_bar[0]);
+            uint32_t st = 0, ph = 0;
+            for (int it = 0; it < iters; ++it) {
+                if (!mbar_wait(full0 + st * 8u, ph, abortp, g.status, 15u, g.wait_ns)) break;
+                const uint32_t hi = tiles_base + st * stage_bytes;
+                for (uint32_t off = 16u * (uint32_t)gt; off < lo_off; off += 16u * (uint32_t)kGatherThreads) {
+                    const float4 v = ld_shared_v4f(hi + off);
+                    st_shared_v4(hi + lo_off + off, v.x - __uint_as_float(__float_as_uint(v.x) & 0xFFFFE000u),
+                                 v.y - __uint_as_float(__float_as_uint(v.y) & 0xFFFFE000u),
+                                 v.z - __uint_as_float(__float_as_uint(v.z) & 0xFFFFE000u),
+                                 v.w - __uint_as_float(__float_as_uint(v.w) & 0xFFFFE000u));
+                }
+                fence_proxy_async_shared();              // generic-proxy stores -> visible to the tensor core's reads
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&lo_bar[st]));
+                if (++st == (uint32_t)g.stages) { st = 0; ph ^= 1u; }
             }
         }
         // split-K over a cluster: everything the reduction needs that does not depend on the accumulator is worked out

@@ -21,7 +21,7 @@ from . import workloads as W
 ACTS = {"none": B.TT_ACT_NONE, "relu": B.TT_ACT_RELU, "relu6": B.TT_ACT_RELU6, "gelu": B.TT_ACT_GELU_ERF}
 RECORD_FIELDS = ("tile_m", "tile_n", "tile_k", "stages", "split_k", "raster", "block_x", "block_y",
                  "items_per_thread", "vec_width", "threads", "unroll", "mma_m_axis", "slab_tiles", "acc_split", "k_order",
-                 "persistent", "cta_group", "ctas_per_sm")
+                 "persistent", "cta_group", "ctas_per_sm", "precision")
 
 
 def build_spec(a) -> W.Spec:

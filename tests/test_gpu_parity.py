@@ -46,7 +46,9 @@ def run_spec(spec, rec, arrays, ref=None, tol=None, mode=B.TT_MODE_LEGALISE, ref
     (the tensor core reads its operands truncated to TF32), the exact oracle for the fp32 SIMT families -- so that
     one wrong output in a large tensor cannot hide inside the L2 norm.  The output sits between guard bands."""
     wl = spec.workload()
-    wl.apply(rec, mode=mode)
+    info = wl.apply(rec, mode=mode)
+    if info.legal.precision == 1 and ref is not None:
+        ref_elem = ref if ref_elem is not None else None      # compensated products: bounded against the exact oracle
     t, _ = W.device_tensors(spec, arrays)
     t["y"], buf = guarded_output(spec)
     tt = B.tensors(t["x"], t["w"], t["bias"], t["residual"], t["y"])
@@ -112,6 +114,9 @@ GEMM_RECORDS = [
     tc(tile_n=64, tile_k=96, stages=2, k_order=1, persistent=1, raster=1, mma_m_axis=1),
     tc(tile_n=64, tile_k=32, stages=2, ctas_per_sm=2, mma_m_axis=1),
     tc(tile_n=128, tile_k=16, stages=3, ctas_per_sm=1, split_k=2, mma_m_axis=2),
+    # error-compensated products (dense, batch_matmul NT; legalised away elsewhere)
+    tc(tile_n=64, tile_k=32, stages=2, precision=1, mma_m_axis=1),
+    tc(tile_n=128, tile_k=64, stages=3, precision=1, split_k=3, mma_m_axis=2),
 ]
 
 
@@ -124,14 +129,18 @@ def check_all_records(spec, seed, records=GEMM_RECORDS):
     valid = [r for r in records if probe.check(r)[0] == B.TT_OK]
     assert all(probe.check(r)[0] in (B.TT_OK, B.TT_ERR_RESOURCE) for r in records)
     assert probe.check(probe.default_schedule())[0] == B.TT_OK
+    compensated = [probe.check(r)[1].legal.precision == 1 for r in valid]      # (kept only where the kernel has that form)
     probe.close()
     assert len(valid) >= len(records) - 6
     re = elem_ref(spec, a, ref)
     outs = [run_spec(spec, r, a, ref, ref_elem=re) for r in valid]
     # a schedule changes speed, never semantics: every valid record gives the same output up to the order of the
-    # fp32 additions (tile_k and split_k regroup them): sqrt(K) * 2^-24 is about 4e-6 at the largest K here
-    for y in outs[1:]:
-        assert util.rel_l2(y, outs[0]) <= INVARIANCE_TOL
+    # fp32 additions (tile_k and split_k regroup them): sqrt(K) * 2^-24 is about 4e-6 at the largest K here.  Records
+    # with error-compensated products are another precision path: compared among themselves
+    for group in (False, True):
+        ys = [y for y, c in zip(outs, compensated) if c == group]
+        for y in ys[1:]:
+            assert util.rel_l2(y, ys[0]) <= INVARIANCE_TOL
     return outs
 
 
@@ -548,7 +557,8 @@ def _random_records(family, n, seed):
                            stages=rng.choice([1, 2, 3, 4, 6, 8]), split_k=rng.choice([1, 1, 2, 3, 4, 5, 8, 9, 16]),
                            raster=rng.choice([0, 1]), mma_m_axis=rng.choice([0, 1, 2]), slab_tiles=rng.choice([0, 0, 1, 2, 5]),
                            acc_split=rng.choice([1, 1, 2, 4, 8]), k_order=rng.choice([0, 0, 1]),
-                           persistent=rng.choice([0, 0, 1]), cta_group=rng.choice([1, 1, 2]), ctas_per_sm=rng.choice([0, 1, 2])))
+                           persistent=rng.choice([0, 0, 1]), cta_group=rng.choice([1, 1, 2]), ctas_per_sm=rng.choice([0, 1, 2]),
+                           precision=rng.choice([0, 0, 0, 1])))
         else:
             recs.append(B.make_record(B.TT_FAMILY_DW_SIMT, tile_m=rng.choice([1, 2, 4, 8, 16, 32]), block_y=rng.choice([1, 2, 4, 7, 8, 14, 28]),
                                       block_x=rng.choice([4, 8, 16, 28, 32, 56]), items_per_thread=rng.choice([1, 2, 4, 8]),
@@ -920,3 +930,21 @@ def test_chain_on_several_streams_matches_the_oracle_chain(model, make, seed):
     check("graph")
     for wl in wls:
         wl.close()
+
+
+@pytest.mark.parametrize("spec", [
+    W._dense(300, 1024, 520, act=B.TT_ACT_GELU_ERF, name="x3_dense"),
+    W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(6, 200, 136, 256, True), 1, "x3_bmm_nt", "bert"),
+])
+def test_compensated_products_come_within_fp32_accumulation_of_the_exact_result(spec):
+    """precision = 1: what the tensor core drops of each operand (everything below TF32's ten mantissa bits) is fed
+    back through two more products per step, so the result must sit far inside the TF32 tolerance: at least twenty
+    times closer to the exact oracle than the same record with plain TF32 products, and within 2e-5 in rel-L2 (fp32
+    accumulation of up to 1024 terms plus the dropped second-order term); under a split-K cluster too."""
+    a = W.make_inputs(spec, 91)
+    ref = util.oracle_ref(spec, a)
+    for kw in (dict(tile_n=64, tile_k=32, stages=3, mma_m_axis=1), dict(tile_n=128, tile_k=64, stages=2, split_k=2, mma_m_axis=2)):
+        y0 = run_spec(spec, tc(**kw), a, ref)
+        y3 = run_spec(spec, tc(precision=1, **kw), a, ref)
+        e0, e3 = util.rel_l2(y0, ref), util.rel_l2(y3, ref)
+        assert e3 <= 2e-5 and e3 * 20 <= e0, (spec.name, kw, e0, e3)

@@ -28,7 +28,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_sizes_match_header_layout():
     assert ctypes.sizeof(B.tt_shapes) == 20 * 4
-    assert ctypes.sizeof(B.tt_schedule_record) == 3 * 4 + 80 + 20 * 4
+    assert ctypes.sizeof(B.tt_schedule_record) == 3 * 4 + 80 + 21 * 4
     assert B.status_string(B.TT_ERR_INVALID_SCHEDULE) != B.status_string(B.TT_OK)
 
 
@@ -489,7 +489,7 @@ def test_pool_file_round_trip_and_rejections(tmp_path):
     B.pool_save(path, recs[:1], None)
     line = [l for l in open(path).read().splitlines() if not l.startswith("#")][0]
     assert "us=-1" in line
-    for bad in (line.replace("tile_n=", "tile_q="), line.replace("version=2", "version=99"), line.replace("stages=2", "stages=two"),
+    for bad in (line.replace("tile_n=", "tile_q="), line.replace("version=3", "version=99"), line.replace("stages=2", "stages=two"),
                 line.replace("origin=1,", "origin=1;")):
         with open(path, "w") as f:
             f.write(bad + "\n")
@@ -546,3 +546,31 @@ def test_chain_lanes_order_every_dependency(model):
         last_serial[st.kernel] = i
     lanes_used = len(seen_on_lane)
     assert lanes_used == (1 if model == "mobilenet_v2" else 4)
+
+
+def test_compensated_precision_is_kept_where_it_exists_and_reported_elsewhere():
+    """Record field `precision` = 1 (three TF32 products per step): dense and batch_matmul NT in the one-tile form keep
+    it, with twice the shared memory per stage and one accumulator; convolutions, NN products and the persistent form
+    legalise it away as a change of form (strict mode: invalid)."""
+    rec = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=64, tile_k=32, stages=2, mma_m_axis=1, precision=1, acc_split=4)
+    plain = B.make_record(B.TT_FAMILY_GEMM_TC, tile_n=64, tile_k=32, stages=2, mma_m_axis=1)
+    dense = W._dense(256, 512, 384).workload()
+    st, info = dense.check(rec)
+    st0, info0 = dense.check(plain)
+    assert st == B.TT_OK and st0 == B.TT_OK and info.legal.precision == 1 and info.legal.acc_split == 1
+    assert info.smem_bytes - 1024 == 2 * (info0.smem_bytes - 1024)
+    assert dense.check(rec, mode=B.TT_MODE_STRICT)[0] == B.TT_ERR_INVALID_SCHEDULE       # (acc_split was changed)
+    rec.acc_split = 1
+    assert dense.check(rec, mode=B.TT_MODE_STRICT)[0] == B.TT_OK
+    nt = W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(4, 128, 128, 64, True), 1, "nt").workload()
+    assert nt.check(rec)[1].legal.precision == 1
+    for other in (W._conv(32, 14, 64, 3, 1, 1).workload(), W._conv(64, 28, 64, 1, 1, 0).workload(),
+                  W.Spec(B.TT_OP_BATCH_MATMUL, B.bmm_shapes(4, 128, 64, 128, False), 1, "nn").workload()):
+        st, info = other.check(rec)
+        assert st == B.TT_OK and info.legal.precision == 0 and info.changed & B.TT_CHG_FORM
+        assert other.check(rec, mode=B.TT_MODE_STRICT)[0] == B.TT_ERR_INVALID_SCHEDULE
+    rec.persistent = 1
+    st, info = dense.check(rec)
+    assert st == B.TT_OK and info.legal.precision == 1 and info.legal.persistent == 0 and info.changed & B.TT_CHG_FORM
+    bad = B.make_record(B.TT_FAMILY_GEMM_TC, precision=2)
+    assert dense.check(bad)[0] == B.TT_ERR_INVALID_SCHEDULE
