@@ -644,9 +644,12 @@ def test_bounded_wait_expires_reports_timeout_and_the_workload_recovers():
     a result of the search, which goes on (Section 4.3)."""
     import torch
     # (a) one CTA, no split; (b) twelve splits through the workspace, of which only split 0 stalls: the other eleven
-    # arrive at the tile counters, which the status path has to clear again or the next run finishes tiles early
+    # arrive at the tile counters, which the status path has to clear again or the next run finishes tiles early;
+    # (c) three splits as a thread-block cluster: split 0 gives up and sends nothing, its peers send it their bands, then
+    # give up waiting for its band, and all three leave together
     for spec, rec in ((W._dense(8, 16, 8, name="stall_one_cta"), tc(tile_n=16, tile_k=16, stages=2, mma_m_axis=1)),
-                      (W._dense(96, 1536, 200, name="stall_split12"), tc(tile_n=64, tile_k=32, stages=3, split_k=12, mma_m_axis=1))):
+                      (W._dense(96, 1536, 200, name="stall_split12"), tc(tile_n=64, tile_k=32, stages=3, split_k=12, mma_m_axis=1)),
+                      (W._dense(96, 768, 200, name="stall_cluster3"), tc(tile_n=64, tile_k=32, stages=3, split_k=3, mma_m_axis=2))):
         a = W.make_inputs(spec, 77)
         ref = util.oracle_ref(spec, a)
         wl = spec.workload()
